@@ -1,0 +1,214 @@
+/*
+ * fpsk.h - C ABI of the B200 FP-Sketch verifier.
+ *
+ * FP-Sketch verifies a half-precision tensor-core GEMM after the fact.  The GEMM under
+ * test delivers its FP32 accumulator C (n1 x n3) un-narrowed; the verifier reads the
+ * operands A (n1 x n2, FP16 or BF16) and B (n2 x n3, same type) and C and never forms AB
+ * (paper: Introduction; Section "Mixed Precision GEMM and Where to Verify").
+ *
+ * Conventions for every entry point
+ *   - All matrices are row-major.  lda, ldb, ldc are leading dimensions in ELEMENTS.
+ *   - Pointers named d_* or documented "device" must be device memory of the current
+ *     device; pointers named h_* are host memory.  A, B, C, workspace are device memory
+ *     unless an entry point says otherwise.
+ *   - The caller owns every buffer.  The library allocates no memory and never writes to
+ *     A, B or C (paper, Section "Overview": localization does not modify C).
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
+ *   - Indices are 0-based.  The 1-based index weights of the paper are internal.
+ *   - Errors are return codes.  Nothing throws, aborts or resets the device.  After
+ *     FPSK_ERR_CUDA the CUDA error is left for the caller to query.
+ *   - Fast paths use 128-bit loads when the base pointers are 16-byte aligned and the
+ *     leading dimensions are multiples of 8 (A, B) / 4 (C) elements; otherwise a scalar
+ *     path with the same arithmetic order runs.
+ */
+#ifndef FPSK_H
+#define FPSK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum { FPSK_FP16 = 0, FPSK_BF16 = 1 } fpsk_dtype;   /* operand type of A and B */
+
+typedef enum {
+    FPSK_OK = 0,
+    FPSK_ERR_NULL = 1,       /* a required pointer is NULL                                  */
+    FPSK_ERR_SHAPE = 2,      /* a dimension < 1, a leading dimension too small, or too large */
+    FPSK_ERR_DTYPE = 3,      /* unknown operand type, or C is not FP32                       */
+    FPSK_ERR_ALIGN = 4,      /* workspace not 256-byte aligned                               */
+    FPSK_ERR_WORKSPACE = 5,  /* workspace smaller than the matching *_workspace_bytes()      */
+    FPSK_ERR_BUCKETS = 6,    /* bucket count < 1 or beyond what the kernels support          */
+    FPSK_ERR_CAPACITY = 7,   /* fault list or an internal list was truncated                 */
+    FPSK_ERR_CUDA = 8,       /* a CUDA call failed                                           */
+    FPSK_ERR_TIMEOUT = 9,    /* a bounded device-side wait gave up                           */
+    FPSK_ERR_PARAM = 10      /* a parameter is out of range                                  */
+} fpsk_status;
+
+/* Verdict of the probe; lives in device memory so that it can stay there until the caller
+ * reads it once per step (paper, Section "The Cheap S Only Probe"). */
+typedef struct {
+    int32_t fired;       /* 1: dirty (max|s| > thr, or s not finite); 0: clean            */
+    int32_t nonfinite;   /* 1: some sketch entry is Inf or NaN (Section "Nonfinite")       */
+    int32_t argmax_col;  /* column with the largest |s_j|                                  */
+    int32_t status;      /* fpsk_status set by the device (FPSK_ERR_TIMEOUT) else FPSK_OK  */
+    float max_abs;       /* max_j |s_j| over the finite entries                            */
+    float sigma_hat;     /* 1.2533 mean(min(|s|, 5 mean|s|))                               */
+    float thr;           /* min(tau, mu sqrt(2 ln N_b) sigma_hat), N_b = max(n3, 2)        */
+    float tau;           /* 100 n2 2^-23 max|A| max|B|                                     */
+} fpsk_probe_result;
+
+/* One confirmed fault (paper, Section "Validation"; Algorithm 1). */
+typedef struct {
+    int32_t i, j;        /* 0-based coordinate in C                                        */
+    double delta;        /* correction gamma - C_ij, i.e. E_ij; an injected +d reads -d    */
+    double recompute;    /* gamma = A_i,* . B_*,j accumulated in FP64                      */
+    float c_value;       /* the delivered C_ij                                             */
+    int32_t round;       /* hash round that found it                                       */
+    int32_t bucket_a, bucket_b;   /* its bucket (h1(i), h2(j)) in that round               */
+} fpsk_fault;
+
+/* Engine parameters; fpsk_default_params() fills the paper's defaults
+ * (Section "Methodology": k=3, rho_min=0.02, r*=4, r_max=16; Section "Validation": c=100;
+ *  Section "Thresholds": mu=4; Section "Sketch Noise Sets the Bucket Count": B*=0.3, c=2). */
+typedef struct {
+    int32_t rounds;      /* k hash rounds, 1..8                                            */
+    int32_t r_star;      /* target radius                                                  */
+    int32_t r_max;       /* largest radius, <= 16                                          */
+    int32_t radius;      /* search radius; -1 = derive it from the measured noise          */
+    int32_t s_budget;    /* declared fault count s (sets K = max(64, 8 s) and m_comb)      */
+    int32_t delta_max;   /* declared bound Delta on faults per row or column               */
+    int32_t mad_of_abs;  /* 1: MAD of |S| as printed in the paper; 0: signed MAD of S      */
+    int32_t reserved;
+    double rho_min;      /* smallest fault to localize, in units of rms(C)                 */
+    double c_valid;      /* c of tau_ij = c eps sum_k |A_ik||B_kj|                         */
+    double mu;           /* probe margin                                                   */
+    double b_star;       /* target index budget                                            */
+    double c_coll;       /* collision constant of m_comb                                   */
+} fpsk_params;
+
+/* Result of the run-time noise measurement (Section "Fault Magnitude, Calibration, and the
+ * Neighbourhood Search"). */
+typedef struct {
+    double sigma_clip;       /* clipped-mean estimate on S at m0                            */
+    double sigma_mad;        /* MAD estimate on the same S                                  */
+    double rms_c;            /* strided, clipped rms of C                                   */
+    double c_hat;            /* sigma_clip m0 / (2^-24 sqrt(n1 n2 n3) rms_c)                */
+    double index_budget_B;   /* B = max(n1,n3) sigma / (rho_min rms)                        */
+    int32_t m0;              /* bucket count the measurement ran at                         */
+    int32_t m_probe;         /* recalibrated probe bucket count m'                          */
+    int32_t m_loc;           /* bucket count for localization                               */
+    int32_t radius;          /* search radius r for localization                            */
+} fpsk_noise;
+
+const char *fpsk_status_string(fpsk_status s);
+void fpsk_default_params(fpsk_params *p);
+
+/* ---- host-only scalar planning (no device work) --------------------------------------- */
+
+/* Starting bucket count of Eq. (mstart): min(max(m_comb, m_num, 16), max(m_comb, m_max)) with
+ * m_num from Eq. (mnum) at delta = rms(C).  Returns the count, or -1 on bad arguments.
+ * (m,k,n) = (n1,n2,n3). */
+int32_t fpsk_law_m_start(int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, const fpsk_params *p);
+
+/* Calibration plan of Section "Calibration": from a noise estimate sigma_hat measured at
+ * bucket count m_cur and an rms estimate of C, the localization bucket count and radius.
+ * A non-positive or non-finite estimate falls back to Eq. (sigma).  Outputs are host
+ * pointers; index_budget may be NULL. */
+fpsk_status fpsk_plan(int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, double sigma_hat,
+                      double rms_c, int32_t m_cur, const fpsk_params *p,
+                      int32_t *m_loc, int32_t *radius, double *index_budget);
+
+/* ---- probe: detection on every call ------------------------------------------------------ */
+
+/* Bytes of device workspace fpsk_probe needs for this shape (0 on bad arguments). */
+size_t fpsk_probe_workspace_bytes(int64_t m, int64_t k, int64_t n);
+
+/* One-time preparation of a probe workspace: zeroes its synchronisation words (async on
+ * `stream`).  Call once after allocating the workspace, and again after a probe reported
+ * FPSK_ERR_TIMEOUT in its result.  A workspace serves one probe at a time: probes sharing a
+ * workspace must be ordered on one stream. */
+fpsk_status fpsk_probe_init(void *workspace, size_t ws_bytes, void *stream);
+
+/* The detection sketch (Eq. (S) with H1 = 1^T, H2 = I): s = (1^T A) B - 1^T C, its noise
+ * estimate, threshold and one-bit verdict (Section "Thresholds"; Algorithm 2, probe part),
+ * in ONE kernel launch, asynchronous on `stream`, no host synchronisation.
+ *   A, B       device, m x k and k x n, type `dtype`
+ *   C          device, m x n FP32; c_is_fp32 must be 1: a narrowed C is rejected
+ *              (Algorithm 2 line 1) with FPSK_ERR_DTYPE
+ *   d_result   device, written by the kernel; valid once `stream` has been synchronised
+ *   d_residual device, n floats receiving s, or NULL
+ * Reads 2mk + 2kn + 4mn bytes.  Deterministic: fixed summation order, no float atomics. */
+fpsk_status fpsk_probe(const void *A, int64_t lda, const void *B, int64_t ldb,
+                       const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                       fpsk_dtype dtype, int c_is_fp32, const fpsk_params *p,
+                       void *workspace, size_t ws_bytes, void *stream,
+                       fpsk_probe_result *d_result, float *d_residual);
+
+/* The same probe for operands in (pinned) HOST memory: copies A, B, C into staging space
+ * inside the workspace, runs fpsk_probe, copies the verdict back and synchronises `stream`.
+ * The workspace must hold fpsk_probe_workspace_bytes() + 2mk + 2kn + 4mn (+ 3*256) bytes;
+ * host matrices are dense (leading dimension = column count). */
+size_t fpsk_probe_host_workspace_bytes(int64_t m, int64_t k, int64_t n);
+fpsk_status fpsk_probe_host(const void *hA, const void *hB, const float *hC,
+                            int64_t m, int64_t k, int64_t n, fpsk_dtype dtype,
+                            const fpsk_params *p, void *workspace, size_t ws_bytes,
+                            void *stream, fpsk_probe_result *h_result);
+
+/* ---- hashed moment sketches --------------------------------------------------------------- */
+
+/* Hash round `round` of `seed` (Section "Moment Sketches": h1, v1 for side 0 = rows,
+ * h2, v2 for side 1 = columns): d_bucket[idx] in [0, n_buckets), d_sign[idx] = +1 or -1,
+ * idx = 0..count-1.  Device outputs, asynchronous. */
+fpsk_status fpsk_hash_tables(uint64_t seed, int32_t round, int32_t side, int64_t count,
+                             int32_t n_buckets, int32_t *d_bucket, int32_t *d_sign, void *stream);
+
+/* Bytes of device workspace for fpsk_sketches / fpsk_measure_noise / fpsk_localize. */
+size_t fpsk_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, const fpsk_params *p);
+
+/* Largest bucket count the kernels accept for this shape (shared-memory limits). */
+int32_t fpsk_max_buckets(int64_t m, int64_t k, int64_t n);
+
+/* Sum and first-moment sketches of E = AB - C for one hash round (Eq. (S) and the weighted
+ * forms R, T of Section "Moment Sketches"), from compressed operands
+ * (H1 A)(B H2^T) - H1 C H2^T, without forming AB.  d_S, d_R, d_T: device, n_buckets^2 floats
+ * each, row-major [a][b]; d_R and d_T may both be NULL for the S-only form.  Asynchronous. */
+fpsk_status fpsk_sketches(const void *A, int64_t lda, const void *B, int64_t ldb,
+                          const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                          fpsk_dtype dtype, uint64_t seed, int32_t round, int32_t n_buckets,
+                          void *workspace, size_t ws_bytes, void *stream,
+                          float *d_S, float *d_R, float *d_T);
+
+/* Run-time noise measurement on a (clean) product: S of round 0 at m0 buckets (m0 <= 0: the
+ * law's starting count), both noise estimates, the strided clipped rms of C, the normalized
+ * constant and the plan (Section "Calibration" and "Recalibrating the probe").
+ * h_out is a host pointer; the call synchronises `stream`. */
+fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_t ldb,
+                               const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                               fpsk_dtype dtype, uint64_t seed, int32_t m0, const fpsk_params *p,
+                               void *workspace, size_t ws_bytes, void *stream, fpsk_noise *h_out);
+
+/* Localization (Algorithm 2 lines "Localize"; Algorithm 1 per round): p->rounds fresh hash
+ * rounds at n_buckets, peeling confirmed faults across rounds, candidates from moment ratios
+ * (Eq. (recover)), each confirmed by an FP64 recomputation of its inner product over the
+ * (2r+1)^2 window, so no clean entry is ever reported (Lemma 1).
+ *   n_buckets  bucket count m_loc used verbatim
+ *   p->radius  search radius, or -1 to derive it from sigma_MAD of the first round's S
+ *   h_faults   host array of `capacity` records, sorted by (i, j) on return
+ *   h_count    host, number of faults found (may exceed capacity with FPSK_ERR_CAPACITY)
+ * The call synchronises `stream` once per round. */
+fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb,
+                          const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                          fpsk_dtype dtype, uint64_t seed, int32_t n_buckets, const fpsk_params *p,
+                          void *workspace, size_t ws_bytes, void *stream,
+                          fpsk_fault *h_faults, int32_t capacity, int32_t *h_count);
+
+/* Number of kernels launched by this library since load (all entry points, all threads). */
+uint64_t fpsk_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* FPSK_H */

@@ -1,0 +1,515 @@
+// C ABI of the FP-Sketch verifier: argument checks, workspace carving, the scalar planner
+// (Sections "Sketch Noise Sets the Bucket Count" and "Calibration") and the round loop of
+// Algorithm 2's localize part with the ordered replay of Algorithm 1's search over the hits.
+#include "sketch.cuh"
+
+#include <math.h>
+#include <string.h>
+#include <algorithm>
+#include <vector>
+
+namespace fpsk {
+std::atomic<unsigned long long> g_launches{0};
+
+constexpr int kHitCap = 2048;
+constexpr int kPeelCap = 4096;
+
+// ---------------------------------------------------------------- scalar planner
+static double cf_of(fpsk_dtype d) { return d == FPSK_BF16 ? 0.19 : 1.76 * 0.19; }
+
+static double law_sigma(double n1, double n2, double n3, fpsk_dtype d, double rms, double m)
+{
+    return cf_of(d) * ldexp(1.0, -24) * sqrt(n1 * n3 * n2) * pow(n2 / 8192.0, 0.07) * rms / m;
+}
+static int m_comb_of(const fpsk_params &p)
+{
+    return (int)ceil(std::max(3.0 * p.c_coll * p.delta_max, sqrt(3.0 * p.c_coll * p.s_budget)));
+}
+static long long isqrt_ll(long long x)
+{
+    long long r = (long long)sqrt((double)x);
+    while (r * r > x) --r;
+    while ((r + 1) * (r + 1) <= x) ++r;
+    return r;
+}
+static int m_max_of(long long n1, long long n3) { return (int)std::max(16LL, isqrt_ll((n1 * n3) / 16)); }
+static int m_mem_of(long long n2)
+{
+    const long long lim = (1LL << 31) / 4;     // 3 m^2 + 6 m n2 <= lim
+    long long m = (long long)((-6.0 * n2 + sqrt(36.0 * (double)n2 * n2 + 12.0 * lim)) / 6.0);
+    while (3 * (m + 1) * (m + 1) + 6 * (m + 1) * n2 <= lim) ++m;
+    while (m > 0 && 3 * m * m + 6 * m * n2 > lim) --m;
+    return (int)std::min(m, 1LL << 30);
+}
+static int m_start_of(long long n1, long long n2, long long n3, fpsk_dtype d, const fpsk_params &p)
+{
+    const double x = (double)std::max(n1, n3) / p.b_star * law_sigma((double)n1, (double)n2, (double)n3, d, 1.0, 1.0);
+    const double mnum = ceil(x);
+    const int mc = m_comb_of(p);
+    const double lo = std::max({(double)mc, mnum, 16.0});
+    const double hi = (double)std::max(mc, m_max_of(n1, n3));
+    return (int)std::min(lo, hi);
+}
+static int radius_of_budget(double B) { return B <= 0.05 ? 0 : std::max(2, (int)ceil(2.5 * B)); }
+
+static void plan_of(long long n1, long long n2, long long n3, fpsk_dtype d, double sigma, double rms, int m_cur,
+                    const fpsk_params &p, int &m_loc, int &radius, double &Bout)
+{
+    const bool ok = std::isfinite(sigma) && sigma > 0 && std::isfinite(rms) && rms > 0;
+    if (!ok) {
+        sigma = law_sigma((double)n1, (double)n2, (double)n3, d, 1.0, (double)m_cur);
+        rms = 1.0;
+    }
+    const double B = (double)std::max(n1, n3) * sigma / (p.rho_min * rms);
+    Bout = B;
+    const int rB = radius_of_budget(B);
+    if (rB <= p.r_star) {
+        m_loc = m_cur;
+        radius = rB;
+        return;
+    }
+    const double grown = 16.0 * ceil(ceil((double)m_cur * rB / p.r_star) / 16.0);
+    const double capped = std::min({grown, (double)m_max_of(n1, n3), (double)m_mem_of(n2)});
+    m_loc = (int)std::max((double)m_cur, capped);
+    const double Bp = B * m_cur / m_loc;
+    radius = Bp <= 0.05 ? 0 : std::min(p.r_max, std::max(2, (int)ceil(2.5 * Bp)));
+}
+
+static bool params_ok(const fpsk_params &p)
+{
+    return p.rounds >= 1 && p.rounds <= 8 && p.r_star >= 0 && p.r_max >= 0 && p.r_max <= 16 && p.radius >= -1 &&
+           p.radius <= 16 && p.s_budget >= 1 && p.delta_max >= 1 && p.rho_min > 0 && p.c_valid > 0 && p.mu > 0 &&
+           p.b_star > 0 && p.c_coll > 1.0 - 1e-12;
+}
+
+static fpsk_params resolve_params(const fpsk_params *p)
+{
+    fpsk_params q;
+    if (p) q = *p;
+    else fpsk_default_params(&q);
+    return q;
+}
+
+static fpsk_status check_mats(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
+                              int64_t m, int64_t k, int64_t n, fpsk_dtype dtype)
+{
+    if (!A || !B || !C) return FPSK_ERR_NULL;
+    if (dtype != FPSK_FP16 && dtype != FPSK_BF16) return FPSK_ERR_DTYPE;
+    if (m < 1 || k < 1 || n < 1 || lda < k || ldb < n || ldc < n) return FPSK_ERR_SHAPE;
+    if (m >= (1LL << 30) || k >= (1LL << 30) || n >= (1LL << 30)) return FPSK_ERR_SHAPE;
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- localize workspace
+struct LocWs {
+    SketchWs sk;
+    float *S, *R, *T;
+    SelectWs sel;
+    float *samples;
+    float *misc;              // [0] max|A| [1] max|B| [2] tau [3] rms_c ; [8..] uint scratch
+    PeelEntry *peel;
+    Hit *hits;
+    int *n_hits;
+};
+
+static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b)
+{
+    const size_t mm = (size_t)m_b * m_b;
+    size_t b = sketch_ws_bytes(n1, n2, n3, m_b);
+    b += align_up(mm * 4, 256) * 3;
+    b += align_up(select_ws_bytes(), 256);
+    b += align_up((size_t)131072 * 4, 256);
+    b += 256;
+    b += align_up(sizeof(PeelEntry) * kPeelCap, 256);
+    b += align_up(sizeof(Hit) * kHitCap, 256);
+    b += 256;
+    return b;
+}
+
+static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, LocWs &w)
+{
+    if (ws_bytes < loc_ws_bytes(n1, n2, n3, m_b)) return false;
+    const size_t mm = (size_t)m_b * m_b;
+    const size_t skb = sketch_ws_bytes(n1, n2, n3, m_b);
+    if (!sketch_carve(ws, skb, n1, n2, n3, m_b, w.sk)) return false;
+    char *p = static_cast<char *>(ws) + skb;
+    auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
+    w.S = (float *)take(mm * 4); w.R = (float *)take(mm * 4); w.T = (float *)take(mm * 4);
+    select_carve(take(select_ws_bytes()), w.sel);
+    w.samples = (float *)take((size_t)131072 * 4);
+    w.misc = (float *)take(256);
+    w.peel = (PeelEntry *)take(sizeof(PeelEntry) * kPeelCap);
+    w.hits = (Hit *)take(sizeof(Hit) * kHitCap);
+    w.n_hits = (int *)take(256);
+    return true;
+}
+
+__global__ void tau_kernel(float *misc, float n2)
+{
+    if (threadIdx.x == 0) misc[2] = 100.f * n2 * 1.1920928955078125e-07f * misc[0] * misc[1];
+}
+
+static int offset_rank_key(int di, int dj, int r)
+{
+    // Chebyshev, then Manhattan, then d_i, then d_j (all ascending) packed into one integer
+    const int ch = std::max(abs(di), abs(dj)), mh = abs(di) + abs(dj);
+    return ((ch * 64 + mh) * 64 + (di + r)) * 64 + (dj + r);
+}
+
+}  // namespace fpsk
+
+using namespace fpsk;
+
+extern "C" {
+
+const char *fpsk_status_string(fpsk_status s)
+{
+    switch (s) {
+    case FPSK_OK: return "ok";
+    case FPSK_ERR_NULL: return "null pointer";
+    case FPSK_ERR_SHAPE: return "bad shape or leading dimension";
+    case FPSK_ERR_DTYPE: return "bad operand type, or C is not FP32";
+    case FPSK_ERR_ALIGN: return "workspace not 256-byte aligned";
+    case FPSK_ERR_WORKSPACE: return "workspace too small";
+    case FPSK_ERR_BUCKETS: return "bucket count out of range";
+    case FPSK_ERR_CAPACITY: return "list truncated";
+    case FPSK_ERR_CUDA: return "CUDA error";
+    case FPSK_ERR_TIMEOUT: return "bounded device wait gave up";
+    case FPSK_ERR_PARAM: return "parameter out of range";
+    }
+    return "unknown";
+}
+
+void fpsk_default_params(fpsk_params *p)
+{
+    if (!p) return;
+    memset(p, 0, sizeof(*p));
+    p->rounds = 3; p->r_star = 4; p->r_max = 16; p->radius = -1;
+    p->s_budget = 8; p->delta_max = 8; p->mad_of_abs = 1;
+    p->rho_min = 0.02; p->c_valid = 100.0; p->mu = 4.0; p->b_star = 0.3; p->c_coll = 2.0;
+}
+
+int32_t fpsk_law_m_start(int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, const fpsk_params *p)
+{
+    const fpsk_params q = resolve_params(p);
+    if (m < 1 || k < 1 || n < 1 || (dtype != FPSK_FP16 && dtype != FPSK_BF16) || !params_ok(q)) return -1;
+    return m_start_of(m, k, n, dtype, q);
+}
+
+fpsk_status fpsk_plan(int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, double sigma_hat, double rms_c,
+                      int32_t m_cur, const fpsk_params *p, int32_t *m_loc, int32_t *radius, double *index_budget)
+{
+    if (!m_loc || !radius) return FPSK_ERR_NULL;
+    const fpsk_params q = resolve_params(p);
+    if (m < 1 || k < 1 || n < 1 || m_cur < 1) return FPSK_ERR_SHAPE;
+    if (dtype != FPSK_FP16 && dtype != FPSK_BF16) return FPSK_ERR_DTYPE;
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    int ml, r;
+    double B;
+    plan_of(m, k, n, dtype, sigma_hat, rms_c, m_cur, q, ml, r, B);
+    *m_loc = ml;
+    *radius = r;
+    if (index_budget) *index_budget = B;
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- probe
+size_t fpsk_probe_workspace_bytes(int64_t m, int64_t k, int64_t n) { return probe_ws_bytes(m, k, n); }
+
+fpsk_status fpsk_probe_init(void *workspace, size_t ws_bytes, void *stream)
+{
+    if (!workspace) return FPSK_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    if (ws_bytes < 256) return FPSK_ERR_WORKSPACE;
+    FPSK_CUDA_OK(cudaMemsetAsync(workspace, 0, 256, static_cast<cudaStream_t>(stream)));
+    return FPSK_OK;
+}
+
+fpsk_status fpsk_probe(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
+                       int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, int c_is_fp32, const fpsk_params *p,
+                       void *workspace, size_t ws_bytes, void *stream, fpsk_probe_result *d_result,
+                       float *d_residual)
+{
+    if (!c_is_fp32) return FPSK_ERR_DTYPE;      // a narrowed C is rejected, not tolerated
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (!workspace || !d_result) return FPSK_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    ProbeDims d{m, k, n, lda, ldb, ldc};
+    return probe_launch(A, B, C, d, dtype, q.mu, workspace, ws_bytes, static_cast<cudaStream_t>(stream), d_result,
+                        d_residual);
+}
+
+size_t fpsk_probe_host_workspace_bytes(int64_t m, int64_t k, int64_t n)
+{
+    const size_t base = probe_ws_bytes(m, k, n);
+    if (!base) return 0;
+    return align_up(base, 256) + align_up((size_t)m * k * 2, 256) + align_up((size_t)k * n * 2, 256) +
+           align_up((size_t)m * n * 4, 256) + 256;
+}
+
+fpsk_status fpsk_probe_host(const void *hA, const void *hB, const float *hC, int64_t m, int64_t k, int64_t n,
+                            fpsk_dtype dtype, const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream,
+                            fpsk_probe_result *h_result)
+{
+    fpsk_status rc = check_mats(hA, k, hB, n, hC, n, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (!workspace || !h_result) return FPSK_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    if (ws_bytes < fpsk_probe_host_workspace_bytes(m, k, n)) return FPSK_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *w = static_cast<char *>(workspace);
+    const size_t base = align_up(probe_ws_bytes(m, k, n), 256);
+    char *dA = w + base;
+    char *dB = dA + align_up((size_t)m * k * 2, 256);
+    char *dC = dB + align_up((size_t)k * n * 2, 256);
+    char *dres = dC + align_up((size_t)m * n * 4, 256);
+    FPSK_CUDA_OK(cudaMemcpyAsync(dA, hA, (size_t)m * k * 2, cudaMemcpyHostToDevice, st));
+    FPSK_CUDA_OK(cudaMemcpyAsync(dB, hB, (size_t)k * n * 2, cudaMemcpyHostToDevice, st));
+    FPSK_CUDA_OK(cudaMemcpyAsync(dC, hC, (size_t)m * n * 4, cudaMemcpyHostToDevice, st));
+    rc = fpsk_probe(dA, k, dB, n, reinterpret_cast<const float *>(dC), n, m, k, n, dtype, 1, p, workspace, base, stream,
+                    reinterpret_cast<fpsk_probe_result *>(dres), nullptr);
+    if (rc != FPSK_OK) return rc;
+    FPSK_CUDA_OK(cudaMemcpyAsync(h_result, dres, sizeof(fpsk_probe_result), cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaStreamSynchronize(st));
+    return (fpsk_status)h_result->status;
+}
+
+// ---------------------------------------------------------------- sketches
+fpsk_status fpsk_hash_tables(uint64_t seed, int32_t round, int32_t side, int64_t count, int32_t n_buckets,
+                             int32_t *d_bucket, int32_t *d_sign, void *stream)
+{
+    if (!d_bucket || !d_sign) return FPSK_ERR_NULL;
+    if (count < 1 || count >= (1LL << 30)) return FPSK_ERR_SHAPE;
+    if (n_buckets < 1) return FPSK_ERR_BUCKETS;
+    if (round < 0 || side < 0 || side > 1) return FPSK_ERR_PARAM;
+    return build_hash_side(seed, round, side, (int)count, n_buckets, d_bucket, d_sign, nullptr, nullptr, nullptr,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int32_t fpsk_max_buckets(int64_t m, int64_t k, int64_t n)
+{
+    if (m < 1 || k < 1 || n < 1) return 0;
+    return sketch_max_buckets(m, k, n);
+}
+
+size_t fpsk_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, const fpsk_params *p)
+{
+    if (m < 1 || k < 1 || n < 1) return 0;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return 0;
+    // n_buckets <= 0: size for the law's starting count of either operand type
+    if (n_buckets <= 0) n_buckets = std::max(m_start_of(m, k, n, FPSK_FP16, q), m_start_of(m, k, n, FPSK_BF16, q));
+    if (n_buckets > sketch_max_buckets(m, k, n)) return 0;
+    return loc_ws_bytes(m, k, n, n_buckets);
+}
+
+fpsk_status fpsk_sketches(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
+                          int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t round,
+                          int32_t n_buckets, void *workspace, size_t ws_bytes, void *stream, float *d_S, float *d_R,
+                          float *d_T)
+{
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (!workspace || !d_S) return FPSK_ERR_NULL;
+    if ((d_R == nullptr) != (d_T == nullptr)) return FPSK_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
+    if (round < 0) return FPSK_ERR_PARAM;
+    SketchWs w;
+    if (!sketch_carve(workspace, ws_bytes, m, k, n, n_buckets, w)) return FPSK_ERR_WORKSPACE;
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+    return build_sketches(in, dtype, seed, round, n_buckets, d_R != nullptr, w, static_cast<cudaStream_t>(stream), d_S,
+                          d_R, d_T);
+}
+
+fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
+                               int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t m0,
+                               const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream, fpsk_noise *h_out)
+{
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (!workspace || !h_out) return FPSK_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    if (m0 <= 0) m0 = m_start_of(m, k, n, dtype, q);
+    if (m0 > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
+    LocWs w;
+    if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w)) return FPSK_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+    rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
+    if (rc != FPSK_OK) return rc;
+    const long long mm = (long long)m0 * m0;
+    rc = sigma_clip_launch(w.S, mm, w.sel, st);
+    if (rc != FPSK_OK) return rc;
+    rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+    if (rc != FPSK_OK) return rc;
+    float h_scal[8];
+    FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
+    rc = rms_c_launch(C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
+    if (rc != FPSK_OK) return rc;
+    float h_rms = 0.f;
+    FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaStreamSynchronize(st));
+
+    fpsk_noise out;
+    memset(&out, 0, sizeof(out));
+    out.sigma_clip = h_scal[3];
+    out.sigma_mad = h_scal[1];
+    out.rms_c = h_rms;
+    out.m0 = m0;
+    const bool rms_ok = std::isfinite(out.rms_c) && out.rms_c > 0;
+    out.c_hat = rms_ok ? out.sigma_clip * m0 / (ldexp(1.0, -24) * sqrt((double)m * (double)k * (double)n) * out.rms_c)
+                       : nan("");
+    int ml, r;
+    double B_;
+    plan_of(m, k, n, dtype, out.sigma_clip, out.rms_c, m0, q, ml, r, B_);
+    out.m_loc = ml;
+    out.radius = r;
+    out.index_budget_B = B_;
+    if (rms_ok && std::isfinite(out.sigma_clip) && out.sigma_clip > 0) {
+        const double B1 = (double)std::max(m, n) * out.sigma_clip / out.rms_c;
+        const double grown = std::min(ceil(m0 * B1 / q.b_star), (double)m_max_of(m, n));
+        out.m_probe = (int)std::max({(double)m_comb_of(q), 16.0, grown});
+    } else {
+        out.m_probe = m0;
+    }
+    *h_out = out;
+    return FPSK_OK;
+}
+
+fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
+                          int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t n_buckets,
+                          const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream, fpsk_fault *h_faults,
+                          int32_t capacity, int32_t *h_count)
+{
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (!workspace || !h_count || (capacity > 0 && !h_faults)) return FPSK_ERR_NULL;
+    if (capacity < 0) return FPSK_ERR_PARAM;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
+    const int m_b = n_buckets;
+    LocWs w;
+    if (!loc_carve(workspace, ws_bytes, m, k, n, m_b, w)) return FPSK_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+    const long long mm = (long long)m_b * m_b;
+    const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
+    *h_count = 0;
+
+    // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
+    unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
+    rc = max_abs_half_launch(A, lda, m, k, dtype, w.misc + 0, uscr, st);
+    if (rc != FPSK_OK) return rc;
+    rc = max_abs_half_launch(B, ldb, k, n, dtype, w.misc + 1, uscr + 1, st);
+    if (rc != FPSK_OK) return rc;
+    tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
+    FPSK_LAUNCH_CHECK();
+
+    int radius = q.radius;
+    bool round0_built = false;
+    if (radius < 0) {
+        // no calibration handed in: sigma_MAD of the first round's S and the strided rms of C
+        rc = build_sketches(in, dtype, seed, 0, m_b, true, w.sk, st, w.S, w.R, w.T);
+        if (rc != FPSK_OK) return rc;
+        round0_built = true;
+        rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+        if (rc != FPSK_OK) return rc;
+        float h_scal[8], h_rms = 0.f;
+        FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
+        rc = rms_c_launch(C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
+        if (rc != FPSK_OK) return rc;
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        double sig = h_scal[1], rms = h_rms;
+        if (!(std::isfinite(sig) && sig > 0 && std::isfinite(rms) && rms > 0)) {
+            sig = law_sigma((double)m, (double)k, (double)n, dtype, 1.0, (double)m_b);
+            rms = 1.0;
+        }
+        radius = std::min(q.r_max, radius_of_budget((double)std::max(m, n) * sig / (q.rho_min * rms)));
+    }
+
+    std::vector<fpsk_fault> F;
+    std::vector<PeelEntry> peel;
+    std::vector<Hit> hits(kHitCap);
+    std::vector<Candidate> cand(kSelMaxK);
+    bool truncated = false;
+    for (int t = 0; t < q.rounds; ++t) {
+        if (!(t == 0 && round0_built)) {
+            rc = build_sketches(in, dtype, seed, t, m_b, true, w.sk, st, w.S, w.R, w.T);
+            if (rc != FPSK_OK) return rc;
+        }
+        if (!peel.empty()) {
+            const int np = (int)std::min<size_t>(peel.size(), kPeelCap);
+            if ((int)peel.size() > kPeelCap) truncated = true;
+            FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, st));
+            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, w.R, w.T, st);
+            if (rc != FPSK_OK) return rc;
+        }
+        if (!(t == 0 && round0_built)) {
+            rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+            if (rc != FPSK_OK) return rc;
+        }
+        rc = select_candidates_launch(w.S, w.R, w.T, m_b, m, n, w.misc + 2, radius, K, w.sel, st);
+        if (rc != FPSK_OK) return rc;
+        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, w.hits, w.n_hits, kHitCap, st);
+        if (rc != FPSK_OK) return rc;
+        int h_counts[4] = {0, 0, 0, 0}, h_nhits = 0;
+        FPSK_CUDA_OK(cudaMemcpyAsync(h_counts, w.sel.counts, sizeof(h_counts), cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_nhits, w.n_hits, 4, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * kHitCap, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
+        const int nU = std::min(h_counts[2], K);
+
+        // replay of Algorithm 1's search: offsets in Chebyshev-then-Manhattan order, buckets of U
+        // in selection order; a bucket leaves U at its first accepted entry
+        std::sort(hits.begin(), hits.begin() + h_nhits, [&](const Hit &x, const Hit &y) {
+            const int kx = offset_rank_key(x.di, x.dj, radius), ky = offset_rank_key(y.di, y.dj, radius);
+            if (kx != ky) return kx < ky;
+            return x.cand < y.cand;
+        });
+        std::vector<char> alive((size_t)std::max(nU, 1), 1);
+        for (int h = 0; h < h_nhits; ++h) {
+            const Hit &x = hits[h];
+            if (x.cand < 0 || x.cand >= nU || !alive[x.cand]) continue;
+            bool inF = false;
+            for (const fpsk_fault &f : F)
+                if (f.i == x.i && f.j == x.j) { inF = true; break; }
+            if (inF) continue;
+            fpsk_fault f;
+            memset(&f, 0, sizeof(f));
+            f.i = x.i; f.j = x.j;
+            f.recompute = x.gamma;
+            f.c_value = x.c_value;
+            f.delta = x.gamma - (double)x.c_value;
+            f.round = t;
+            f.bucket_a = cand[x.cand].flat / m_b;
+            f.bucket_b = cand[x.cand].flat % m_b;
+            F.push_back(f);
+            // only finite faults are peeled (Section "Peeling Across Hash Rounds")
+            if (std::isfinite(f.delta)) peel.push_back(PeelEntry{f.i, f.j, f.delta});
+            alive[x.cand] = 0;
+        }
+    }
+    std::sort(F.begin(), F.end(), [](const fpsk_fault &x, const fpsk_fault &y) {
+        return x.i != y.i ? x.i < y.i : x.j < y.j;
+    });
+    *h_count = (int32_t)F.size();
+    const int ncopy = std::min<int>((int)F.size(), capacity);
+    for (int f = 0; f < ncopy; ++f) h_faults[f] = F[f];
+    if ((int)F.size() > capacity || truncated) return FPSK_ERR_CAPACITY;
+    return FPSK_OK;
+}
+
+uint64_t fpsk_launch_count(void) { return g_launches.load(); }
+
+}  // extern "C"

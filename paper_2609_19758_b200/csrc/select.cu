@@ -1,0 +1,430 @@
+// Noise estimates, thresholds and candidate selection on a sketch S (Section "Thresholds";
+// Algorithm 1: MAD estimate, tau_c, tau_d, the K largest buckets, the set U and the moment
+// ratios of Eq. (recover)).  Medians and the K-th largest key come from an exact radix select
+// (integer histograms only), so every decision is deterministic.
+#include "sketch.cuh"
+
+#include <math.h>
+
+namespace fpsk {
+
+enum SelMode {
+    SEL_ABS = 0,        // key = bits(|S|)                         (median of |S|)
+    SEL_SIGNED = 1,     // key = order-preserving bits of S        (median of S)
+    SEL_DEV_ABS = 2,    // key = bits(||S| - med|)
+    SEL_DEV_SIGNED = 3, // key = bits(|S - med|)
+    SEL_TOPK = 4,       // valid iff |S| > thr; key = bits(|S|) << 32 | ~idx   (all keys distinct)
+    SEL_SAMPLE = 5      // valid iff S >= 0 (sentinel -1 marks dropped samples); key = bits(S)
+};
+
+// state words
+enum { ST_PREFIX = 0, ST_K = 1, ST_SKIP = 2, ST_WORDS = 4 };
+// scal slots
+enum { SC_MED = 0, SC_MAD = 1, SC_MEAN = 2, SC_CLIP = 3, SC_THR = 4, SC_TAUC = 5, SC_TAUD = 6, SC_WORDS = 16 };
+
+__device__ __forceinline__ uint32_t ordered_bits(float x)
+{
+    uint32_t b = __float_as_uint(x);
+    return b ^ ((b >> 31) ? 0xFFFFFFFFu : 0x80000000u);
+}
+__device__ __forceinline__ float from_ordered_bits(uint32_t k)
+{
+    uint32_t b = (k >> 31) ? (k ^ 0x80000000u) : ~k;
+    return __uint_as_float(b);
+}
+
+__device__ __forceinline__ bool make_key(int mode, const float *S, long long idx, const float *scal,
+                                         unsigned long long &key)
+{
+    const float x = S[idx];
+    switch (mode) {
+    case SEL_ABS: key = __float_as_uint(fabsf(x)); return true;
+    case SEL_SIGNED: key = ordered_bits(x); return true;
+    case SEL_DEV_ABS: key = __float_as_uint(fabsf(fabsf(x) - scal[SC_MED])); return true;
+    case SEL_DEV_SIGNED: key = __float_as_uint(fabsf(x - scal[SC_MED])); return true;
+    case SEL_TOPK: {
+        const float a = fabsf(x);
+        if (!(a > scal[SC_THR])) return false;
+        key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
+        return true;
+    }
+    default:
+        if (!(x >= 0.f)) return false;
+        key = __float_as_uint(x);
+        return true;
+    }
+}
+
+// counts[0] = number of valid keys (SEL_TOPK, SEL_SAMPLE)
+__global__ void count_valid_kernel(int mode, const float *S, long long mm, const float *scal, int *counts)
+{
+    int c = 0;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < mm; i += (long long)gridDim.x * blockDim.x) {
+        unsigned long long k;
+        c += make_key(mode, S, i, scal, k) ? 1 : 0;
+    }
+    c = __reduce_add_sync(0xFFFFFFFFu, c);
+    if ((threadIdx.x & 31) == 0 && c) atomicAdd(counts, c);
+}
+
+// rank to select: median of N keys, or (count - K) for the K largest, from device counts
+__global__ void select_init_kernel(int mode, long long n_all, int K, const int *counts, unsigned long long *state,
+                                   unsigned int *hist)
+{
+    if (threadIdx.x != 0) return;
+    state[ST_PREFIX] = 0;
+    state[ST_SKIP] = 0;
+    if (mode == SEL_TOPK) {
+        const int cnt = counts[0];
+        if (cnt <= K) state[ST_SKIP] = 1;      // take everything above the threshold
+        else state[ST_K] = (unsigned long long)(cnt - K);
+    } else if (mode == SEL_SAMPLE) {
+        const int cnt = counts[0];
+        if (cnt <= 0) state[ST_SKIP] = 1;
+        else state[ST_K] = (unsigned long long)((cnt - 1) / 2);
+    } else {
+        state[ST_K] = (unsigned long long)((n_all - 1) / 2);
+    }
+    for (int b = 0; b < 257; ++b) hist[b] = 0;
+}
+
+// One 8-bit digit of the radix select.  The last CTA to finish picks the digit.
+__global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, int shift, const float *S, long long mm,
+                                                         const float *scal, unsigned long long *state, unsigned int *hist)
+{
+    __shared__ unsigned int sh[256];
+    __shared__ int last;
+    if (state[ST_SKIP]) return;
+    sh[threadIdx.x] = 0;
+    __syncthreads();
+    const unsigned long long prefix = state[ST_PREFIX];
+    const int hs = shift + 8;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < mm; i += (long long)gridDim.x * blockDim.x) {
+        unsigned long long k;
+        if (!make_key(mode, S, i, scal, k)) continue;
+        if (hs < nbits && (k >> hs) != (prefix >> hs)) continue;
+        atomicAdd(&sh[(unsigned)(k >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    if (sh[threadIdx.x]) atomicAdd(&hist[threadIdx.x], sh[threadIdx.x]);
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = (atomicAdd(&hist[256], 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    if (threadIdx.x == 0) {
+        unsigned long long k = state[ST_K], cum = 0;
+        int bin = 255;
+        for (int b = 0; b < 256; ++b) {
+            const unsigned int h = __ldcg(&hist[b]);
+            if (cum + h > k) { bin = b; break; }
+            cum += h;
+        }
+        state[ST_K] = k - cum;
+        state[ST_PREFIX] = prefix | ((unsigned long long)bin << shift);
+        hist[256] = 0;
+    }
+    __syncthreads();
+    hist[threadIdx.x] = 0;
+}
+
+// after the passes: turn the selected key into a value
+__global__ void select_finish_kernel(int mode, const unsigned long long *state, float *scal)
+{
+    if (threadIdx.x != 0) return;
+    const unsigned long long key = state[ST_PREFIX];
+    if (mode == SEL_ABS) scal[SC_MED] = __uint_as_float((uint32_t)key);
+    else if (mode == SEL_SIGNED) scal[SC_MED] = from_ordered_bits((uint32_t)key);
+    else if (mode == SEL_DEV_ABS || mode == SEL_DEV_SIGNED) scal[SC_MAD] = 1.4826f * __uint_as_float((uint32_t)key);
+    else if (mode == SEL_SAMPLE) scal[SC_MED] = state[ST_SKIP] ? __uint_as_float(0x7FC00000u) : __uint_as_float((uint32_t)key);
+}
+
+static fpsk_status run_select(int mode, int nbits, const float *S, long long mm, int K, SelectWs &w, cudaStream_t st)
+{
+    select_init_kernel<<<1, 32, 0, st>>>(mode, mm, K, w.counts, w.state, w.hist);
+    FPSK_LAUNCH_CHECK();
+    long long want = (mm + 256 * 16 - 1) / (256 * 16);
+    const int grid = (int)(want < 1 ? 1 : (want > 1184 ? 1184 : want));
+    for (int shift = nbits - 8; shift >= 0; shift -= 8) {
+        radix_pass_kernel<<<grid, 256, 0, st>>>(mode, nbits, shift, S, mm, w.scal, w.state, w.hist);
+        FPSK_LAUNCH_CHECK();
+    }
+    select_finish_kernel<<<1, 32, 0, st>>>(mode, w.state, w.scal);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+fpsk_status sigma_mad_launch(const float *S, long long mm, int mad_of_abs, SelectWs &w, cudaStream_t st)
+{
+    fpsk_status rc = run_select(mad_of_abs ? SEL_ABS : SEL_SIGNED, 32, S, mm, 0, w, st);
+    if (rc != FPSK_OK) return rc;
+    return run_select(mad_of_abs ? SEL_DEV_ABS : SEL_DEV_SIGNED, 32, S, mm, 0, w, st);
+}
+
+// ---------------------------------------------------------------- clipped mean
+// mode 0: sum |S| -> scal[SC_MEAN] = mean; mode 1: sum min(|S|, 5 mean) -> scal[SC_CLIP].
+// Fixed grid, fixed per-CTA tree, partials summed in CTA order by the last CTA: deterministic.
+constexpr int kSumGrid = 256;
+__global__ void __launch_bounds__(256) abs_sum_kernel(int mode, const float *S, long long mm, float *scal, float *partial,
+                                                      unsigned int *ticket)
+{
+    __shared__ float sh[256];
+    __shared__ int last;
+    const float clip = mode ? 5.f * scal[SC_MEAN] : 0.f;
+    float acc = 0.f;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < mm; i += (long long)gridDim.x * blockDim.x) {
+        const float a = fabsf(S[i]);
+        acc += mode ? fminf(a, clip) : a;
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = 128; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        __stcg(partial + blockIdx.x, sh[0]);
+        __threadfence();
+        last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!last || threadIdx.x != 0) return;
+    __threadfence();
+    float tot = 0.f;
+    for (int b = 0; b < (int)gridDim.x; ++b) tot += __ldcg(partial + b);
+    const float mean = tot / (float)mm;
+    if (mode) scal[SC_CLIP] = 1.2533f * mean;
+    else scal[SC_MEAN] = mean;
+    *ticket = 0;
+}
+
+fpsk_status sigma_clip_launch(const float *S, long long mm, SelectWs &w, cudaStream_t st)
+{
+    FPSK_CUDA_OK(cudaMemsetAsync(w.hist + 257, 0, 4, st));
+    for (int mode = 0; mode < 2; ++mode) {
+        abs_sum_kernel<<<kSumGrid, 256, 0, st>>>(mode, S, mm, w.scal, w.partial, w.hist + 257);
+        FPSK_LAUNCH_CHECK();
+    }
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- thresholds and candidates
+__global__ void thresholds_kernel(const float *taup, float nmax, float rad, float *scal, int *counts)
+{
+    if (threadIdx.x != 0) return;
+    const float tau = *taup;
+    const float sig = scal[SC_MAD];
+    const float tau_c = fminf(tau, 2.f * sig);
+    const float tau_d = nmax * sig / fmaxf(rad, 0.5f);
+    scal[SC_TAUC] = tau_c;
+    scal[SC_TAUD] = tau_d;
+    scal[SC_THR] = fmaxf(tau_c, tau_d);
+    counts[0] = 0; counts[1] = 0; counts[2] = 0;
+}
+
+__global__ void collect_kernel(const float *S, long long mm, const float *scal, const unsigned long long *state,
+                               int cap, unsigned long long *keys, int *counts)
+{
+    const unsigned long long kth = state[ST_SKIP] ? 0ull : state[ST_PREFIX];
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < mm; i += (long long)gridDim.x * blockDim.x) {
+        unsigned long long k;
+        if (!make_key(SEL_TOPK, S, i, scal, k)) continue;
+        if (k < kth) continue;
+        const int slot = atomicAdd(counts + 1, 1);
+        if (slot < cap) keys[slot] = k;
+    }
+}
+
+// Sort the selected keys (descending |S|, ties by ascending flat index), keep those with
+// S != 0 and S, R, T finite (the set U), decode Eq. (recover) with 1-based -> 0-based indices.
+__global__ void __launch_bounds__(1024) decode_kernel(const float *S, const float *R, const float *T, int p1, int p3,
+                                                      const unsigned long long *keys, int *counts, int cap, Candidate *cand)
+{
+    __shared__ unsigned long long sk[kSelMaxK];
+    __shared__ int flag[kSelMaxK];
+    const int t = threadIdx.x;
+    int n = counts[1];
+    if (n > cap) n = cap;
+    sk[t] = t < n ? keys[t] : 0ull;
+    __syncthreads();
+    for (int k = 2; k <= kSelMaxK; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const int ixj = t ^ j;
+            if (ixj > t) {
+                const bool desc = (t & k) == 0;
+                const unsigned long long a = sk[t], b = sk[ixj];
+                if (desc ? (a < b) : (a > b)) { sk[t] = b; sk[ixj] = a; }
+            }
+            __syncthreads();
+        }
+    }
+    Candidate c;
+    c.flat = -1; c.ih = 0; c.jh = 0; c.s_abs = 0.f;
+    int keep = 0;
+    if (t < n) {
+        const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sk[t] & 0xFFFFFFFFull);
+        const float s = S[idx], r = R ? R[idx] : 0.f, q = T ? T[idx] : 0.f;
+        const bool fin = (fabsf(s) <= 3.402823466e38f) && (fabsf(r) <= 3.402823466e38f) && (fabsf(q) <= 3.402823466e38f);
+        if (s != 0.f && fin) {
+            float fi = rintf(ldexpf(r / s, p1)) - 1.f;
+            float fj = rintf(ldexpf(q / s, p3)) - 1.f;
+            const float lim = 1073741824.f;
+            if (!(fabsf(fi) < lim)) fi = -lim;
+            if (!(fabsf(fj) < lim)) fj = -lim;
+            c.flat = (int)idx; c.ih = (int)fi; c.jh = (int)fj; c.s_abs = fabsf(s);
+            keep = 1;
+        }
+    }
+    flag[t] = keep;
+    __syncthreads();
+    // inclusive scan of the keep flags (order-preserving compaction)
+    for (int o = 1; o < kSelMaxK; o <<= 1) {
+        const int v = t >= o ? flag[t - o] : 0;
+        __syncthreads();
+        flag[t] += v;
+        __syncthreads();
+    }
+    if (keep) cand[flag[t] - 1] = c;
+    if (t == kSelMaxK - 1) counts[2] = flag[t];
+}
+
+fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
+                                     long long n3, const float *d_tau, int radius, int K, SelectWs &w, cudaStream_t st)
+{
+    if (K > kSelMaxK) K = kSelMaxK;
+    const long long mm = (long long)m_b * m_b;
+    thresholds_kernel<<<1, 32, 0, st>>>(d_tau, (float)(n1 > n3 ? n1 : n3), (float)radius, w.scal, w.counts);
+    FPSK_LAUNCH_CHECK();
+    long long want = (mm + 256 * 16 - 1) / (256 * 16);
+    const int grid = (int)(want < 1 ? 1 : (want > 1184 ? 1184 : want));
+    count_valid_kernel<<<grid, 256, 0, st>>>(SEL_TOPK, S, mm, w.scal, w.counts);
+    FPSK_LAUNCH_CHECK();
+    fpsk_status rc = run_select(SEL_TOPK, 64, S, mm, K, w, st);
+    if (rc != FPSK_OK) return rc;
+    collect_kernel<<<grid, 256, 0, st>>>(S, mm, w.scal, w.state, kSelMaxK, w.keys, w.counts);
+    FPSK_LAUNCH_CHECK();
+    int p1 = 0, p3 = 0;
+    while ((1LL << p1) < n1) ++p1;
+    while ((1LL << p3) < n3) ++p3;
+    decode_kernel<<<1, kSelMaxK, 0, st>>>(S, R, T, p1, p3, w.keys, w.counts, kSelMaxK, w.cand);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- max |X| of a half matrix
+template <typename T>
+__global__ void max_abs_half_kernel(const unsigned short *X, long long ld, long long rows, long long cols, unsigned int *out)
+{
+    unsigned int m = 0;
+    const long long total = rows * cols;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const long long r = i / cols, c = i - r * cols;
+        m = max(m, (unsigned int)(X[r * ld + c] & 0x7FFFu));
+    }
+    m = __reduce_max_sync(0xFFFFFFFFu, m);
+    if ((threadIdx.x & 31) == 0) atomicMax(out, m);
+}
+template <typename T>
+__global__ void max_abs_finish_kernel(const unsigned int *bits, float *out)
+{
+    if (threadIdx.x == 0) out[0] = bits16_to_float<T>(bits[0]);
+}
+
+fpsk_status max_abs_half_launch(const void *X, long long ld, long long rows, long long cols, fpsk_dtype dtype,
+                                float *out, unsigned int *scratch, cudaStream_t st)
+{
+    FPSK_CUDA_OK(cudaMemsetAsync(scratch, 0, 4, st));
+    const unsigned short *x = static_cast<const unsigned short *>(X);
+    long long want = (rows * cols + 256 * 32 - 1) / (256 * 32);
+    const int grid = (int)(want < 1 ? 1 : (want > 2368 ? 2368 : want));
+    if (dtype == FPSK_FP16) {
+        max_abs_half_kernel<__half><<<grid, 256, 0, st>>>(x, ld, rows, cols, scratch);
+        FPSK_LAUNCH_CHECK();
+        max_abs_finish_kernel<__half><<<1, 32, 0, st>>>(scratch, out);
+    } else {
+        max_abs_half_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(x, ld, rows, cols, scratch);
+        FPSK_LAUNCH_CHECK();
+        max_abs_finish_kernel<__nv_bfloat16><<<1, 32, 0, st>>>(scratch, out);
+    }
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- strided, clipped rms of C
+__global__ void sample_c_kernel(const float *C, long long ldc, long long n3, long long total, long long stride,
+                                long long nsamp, float *samples)
+{
+    const long long t = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= nsamp) return;
+    const long long flat = t * stride;
+    const long long r = flat / n3, c = flat - r * n3;
+    const float a = fabsf(C[r * ldc + c]);
+    samples[t] = (a <= 3.402823466e38f) ? a : -1.f;      // sentinel for Inf / NaN
+}
+
+// single CTA, FP64 accumulation in a fixed order
+__global__ void __launch_bounds__(1024) clipped_rms_kernel(const float *samples, long long nsamp, const float *scal,
+                                                           const int *counts, float *out)
+{
+    __shared__ double sh[1024];
+    const float clip = 64.f * scal[SC_MED];
+    double acc = 0.0;
+    for (long long i = threadIdx.x; i < nsamp; i += 1024) {
+        const float a = samples[i];
+        if (a >= 0.f) {
+            const double v = (double)fminf(a, clip);
+            acc += v * v;
+        }
+    }
+    sh[threadIdx.x] = acc;
+    __syncthreads();
+    for (int s = 512; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) sh[threadIdx.x] += sh[threadIdx.x + s];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const int n = counts[0];
+        out[0] = n > 0 ? (float)sqrt(sh[0] / (double)n) : __uint_as_float(0x7FC00000u);
+    }
+}
+
+fpsk_status rms_c_launch(const float *C, long long ldc, long long n1, long long n3, float *samples,
+                         SelectWs &w, float *out, cudaStream_t st)
+{
+    const long long total = n1 * n3;
+    long long stride = total / 65536;
+    if (stride < 1) stride = 1;
+    const long long nsamp = (total + stride - 1) / stride;
+    sample_c_kernel<<<(unsigned)((nsamp + 255) / 256), 256, 0, st>>>(C, ldc, n3, total, stride, nsamp, samples);
+    FPSK_LAUNCH_CHECK();
+    FPSK_CUDA_OK(cudaMemsetAsync(w.counts, 0, 4 * 4, st));
+    count_valid_kernel<<<64, 256, 0, st>>>(SEL_SAMPLE, samples, nsamp, w.scal, w.counts);
+    FPSK_LAUNCH_CHECK();
+    fpsk_status rc = run_select(SEL_SAMPLE, 32, samples, nsamp, 0, w, st);
+    if (rc != FPSK_OK) return rc;
+    clipped_rms_kernel<<<1, 1024, 0, st>>>(samples, nsamp, w.scal, w.counts, out);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- workspace
+size_t select_ws_bytes()
+{
+    return 4096 /*hist+ticket*/ + 256 /*state*/ + 256 /*scal*/ + align_up(kSumGrid * 4, 256) +
+           align_up(kSelMaxK * 8, 256) + 256 /*counts*/ + align_up(kSelMaxK * sizeof(Candidate), 256);
+}
+
+void select_carve(void *ws, SelectWs &w)
+{
+    char *p = static_cast<char *>(ws);
+    w.hist = (unsigned int *)p; p += 4096;
+    w.state = (unsigned long long *)p; p += 256;
+    w.scal = (float *)p; p += 256;
+    w.partial = (float *)p; p += align_up(kSumGrid * 4, 256);
+    w.keys = (unsigned long long *)p; p += align_up(kSelMaxK * 8, 256);
+    w.counts = (int *)p; p += 256;
+    w.cand = (Candidate *)p;
+}
+
+}  // namespace fpsk

@@ -1,0 +1,567 @@
+// Hashed moment sketches S, R, T of E = AB - C for one hash round, without forming AB
+// (Section "Moment Sketches", Eq. (S)):  (H1 A)(B H2^T) - H1 C H2^T and the index-weighted
+// forms.  All accumulation is FP32 in a fixed order: no float atomics anywhere, so results
+// are bit-reproducible run to run.
+//
+//   hash_kernel / scan_kernel / place_kernel   hash tables and bucket-sorted permutations
+//   compress_a_kernel   P = H1 A, Pw = H1 W1 A          (m_b x n2, rows grouped by bucket)
+//   compress_b_kernel   Q = B H2^T, Qw = B W2 H2^T      (n2 x m_b, one row of B per pass)
+//   sgemm_kernel        S_AB = P Q, R_AB = Pw Q, T_AB = P Qw   (FP32 SIMT, split-K partials)
+//   scatter_c_kernel    S_C, R_C, T_C: one streaming pass over C per round
+//   combine_kernel      S = sum of AB partials - sum of C partials
+#include "sketch.cuh"
+
+namespace fpsk {
+
+// ---------------------------------------------------------------- hash tables
+__global__ void hash_kernel(uint32_t key, int n, int m_b, int *bucket, int *sign, int *count)
+{
+    int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= n) return;
+    int b, s;
+    hash_index(key, (uint32_t)idx, (uint32_t)m_b, b, s);
+    bucket[idx] = b;
+    sign[idx] = s;
+    if (count) atomicAdd(count + b, 1);
+}
+
+// exclusive scan of count[0..m_b) into start[0..m_b]; single CTA
+__global__ void scan_kernel(const int *count, int m_b, int *start)
+{
+    __shared__ int carry;
+    __shared__ int buf[1024];
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < m_b; base += 1024) {
+        int i = base + threadIdx.x;
+        int v = i < m_b ? count[i] : 0;
+        buf[threadIdx.x] = v;
+        __syncthreads();
+        for (int o = 1; o < 1024; o <<= 1) {
+            int t = threadIdx.x >= o ? buf[threadIdx.x - o] : 0;
+            __syncthreads();
+            buf[threadIdx.x] += t;
+            __syncthreads();
+        }
+        if (i < m_b) start[i] = carry + buf[threadIdx.x] - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry += buf[1023];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) start[m_b] = carry;
+}
+
+// Stable placement: entry idx goes to start[b] + (number of idx' < idx in the same bucket).
+// perm packs the index (low 31 bits) and the sign (bit 31 set = -1).
+__global__ void place_kernel(const int *bucket, const int *sign, const int *start, int n, uint32_t *perm)
+{
+    __shared__ int tile[1024];
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = idx < n ? bucket[idx] : -1;
+    int rank = 0;
+    const int hi = min(n, (int)((blockIdx.x + 1) * blockDim.x));
+    for (int base = 0; base < hi; base += 1024) {
+        __syncthreads();
+        int t = base + threadIdx.x;
+        tile[threadIdx.x] = t < n ? bucket[t] : -2;
+        __syncthreads();
+        int lim = min(1024, idx - base);   // only earlier indices count
+        for (int q = 0; q < lim; ++q) rank += (tile[q] == b);
+    }
+    if (idx < n) perm[start[b] + rank] = (uint32_t)idx | (sign[idx] < 0 ? 0x80000000u : 0u);
+}
+
+fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, int *bucket, int *sign,
+                            int *count, int *start, uint32_t *perm, cudaStream_t st)
+{
+    const uint32_t key = round_key(seed, rnd, side);
+    if (count) FPSK_CUDA_OK(cudaMemsetAsync(count, 0, sizeof(int) * (size_t)m_b, st));
+    hash_kernel<<<(n + 255) / 256, 256, 0, st>>>(key, n, m_b, bucket, sign, count);
+    FPSK_LAUNCH_CHECK();
+    if (!perm) return FPSK_OK;
+    scan_kernel<<<1, 1024, 0, st>>>(count, m_b, start);
+    FPSK_LAUNCH_CHECK();
+    place_kernel<<<(n + 1023) / 1024, 1024, 0, st>>>(bucket, sign, start, n, perm);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- A compression
+// CTA (x: group of 8-column vectors, y: bucket a).  Thread owns 8 adjacent columns and walks
+// the rows of bucket a in ascending row order.
+template <typename T, bool VEC, bool MOM>
+__global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A, long long lda, int n1, int n2,
+                                                         int kpad, float inv_p1, const uint32_t *rowperm,
+                                                         const int *rowstart, float *P, float *Pw)
+{
+    const int a = blockIdx.y;
+    const long long col0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    if (col0 >= kpad) return;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, accw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (col0 < n2) {
+        const int s0 = rowstart[a], s1 = rowstart[a + 1];
+        for (int s = s0; s < s1; ++s) {
+            const uint32_t e = __ldg(rowperm + s);
+            const int i = (int)(e & 0x7FFFFFFFu);
+            const float sg = (e >> 31) ? -1.f : 1.f;
+            uint4 v;
+            if (VEC) v = ldg_nc_v4(A + (long long)i * lda + col0);
+            else {
+                unsigned int w[4] = {0, 0, 0, 0};
+                for (int q = 0; q < 8; ++q)
+                    if (col0 + q < n2) w[q >> 1] |= (unsigned int)A[(long long)i * lda + col0 + q] << ((q & 1) * 16);
+                v = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            const float swi = sg * ((float)(i + 1) * inv_p1);
+            const unsigned int ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float2 f = HalfTraits<T>::unpack2(ww[q]);
+                acc[2 * q] += sg * f.x;
+                acc[2 * q + 1] += sg * f.y;
+                if (MOM) {
+                    accw[2 * q] = fmaf(swi, f.x, accw[2 * q]);
+                    accw[2 * q + 1] = fmaf(swi, f.y, accw[2 * q + 1]);
+                }
+            }
+        }
+    }
+    float4 *dp = reinterpret_cast<float4 *>(P + (long long)a * kpad + col0);
+    dp[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    dp[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+    if (MOM) {
+        float4 *dw = reinterpret_cast<float4 *>(Pw + (long long)a * kpad + col0);
+        dw[0] = make_float4(accw[0], accw[1], accw[2], accw[3]);
+        dw[1] = make_float4(accw[4], accw[5], accw[6], accw[7]);
+    }
+}
+
+// ---------------------------------------------------------------- B compression
+// One row of B at a time staged in shared memory; thread b folds the columns of bucket b in
+// ascending column order.  Rows k >= n2 (padding of the contraction) are written as zeros.
+template <typename T, bool MOM>
+__global__ void __launch_bounds__(256) compress_b_kernel(const unsigned short *B, long long ldb, int n2, int n3,
+                                                         int kpad, int m_b, int npad, float inv_p3,
+                                                         const uint32_t *colperm, const int *colstart,
+                                                         float *Q, float *Qw)
+{
+    extern __shared__ __align__(16) unsigned short rowbuf[];
+    for (int k = blockIdx.x; k < kpad; k += gridDim.x) {
+        if (k >= n2) {
+            for (int b = threadIdx.x; b < npad; b += blockDim.x) {
+                Q[(long long)k * npad + b] = 0.f;
+                if (MOM) Qw[(long long)k * npad + b] = 0.f;
+            }
+            continue;
+        }
+        __syncthreads();
+        const unsigned short *src = B + (long long)k * ldb;
+        if (((reinterpret_cast<uintptr_t>(src) & 15) == 0) && (n3 % 8 == 0)) {
+            for (int j = threadIdx.x * 8; j < n3; j += blockDim.x * 8)
+                *reinterpret_cast<uint4 *>(rowbuf + j) = ldg_nc_v4(src + j);
+        } else {
+            for (int j = threadIdx.x; j < n3; j += blockDim.x) rowbuf[j] = src[j];
+        }
+        __syncthreads();
+        for (int b = threadIdx.x; b < npad; b += blockDim.x) {
+            float q = 0.f, qw = 0.f;
+            if (b < m_b) {
+                const int s0 = __ldg(colstart + b), s1 = __ldg(colstart + b + 1);
+                for (int s = s0; s < s1; ++s) {
+                    const uint32_t e = __ldg(colperm + s);
+                    const int j = (int)(e & 0x7FFFFFFFu);
+                    const float sg = (e >> 31) ? -1.f : 1.f;
+                    const float x = bits16_to_float<T>(rowbuf[j]);
+                    q += sg * x;
+                    if (MOM) qw = fmaf(sg * ((float)(j + 1) * inv_p3), x, qw);
+                }
+            }
+            Q[(long long)k * npad + b] = q;
+            if (MOM) Qw[(long long)k * npad + b] = qw;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- C scatter
+// CTA (x: bucket row a, y: split).  The rows of bucket a (ascending) are divided among the
+// splits; each row of C is staged in shared memory and folded over its columns by bucket;
+// the three accumulators of bucket row a live in shared memory, one owner thread per b.
+template <bool MOM>
+__global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long long ldc, int n1, int n3, int m_b,
+                                                        float inv_p1, float inv_p3, const uint32_t *rowperm,
+                                                        const int *rowstart, const uint32_t *colperm,
+                                                        const int *colstart, int nsplit, float *part)
+{
+    extern __shared__ __align__(16) float sm[];
+    float *rowbuf = sm;                       // n3 (padded to 4)
+    float *accS = sm + ((n3 + 3) & ~3);
+    float *accR = accS + m_b;
+    float *accT = accR + m_b;
+    const int a = blockIdx.x, sp = blockIdx.y;
+    for (int b = threadIdx.x; b < m_b; b += blockDim.x) {
+        accS[b] = 0.f;
+        if (MOM) { accR[b] = 0.f; accT[b] = 0.f; }
+    }
+    const int s0 = rowstart[a], s1 = rowstart[a + 1];
+    const int cnt = s1 - s0;
+    const int q0 = s0 + (int)((long long)cnt * sp / nsplit), q1 = s0 + (int)((long long)cnt * (sp + 1) / nsplit);
+    for (int s = q0; s < q1; ++s) {
+        const uint32_t e = __ldg(rowperm + s);
+        const int i = (int)(e & 0x7FFFFFFFu);
+        const float v1 = (e >> 31) ? -1.f : 1.f;
+        const float v1w = v1 * ((float)(i + 1) * inv_p1);
+        __syncthreads();
+        const float *src = C + (long long)i * ldc;
+        if (((reinterpret_cast<uintptr_t>(src) & 15) == 0) && (n3 % 4 == 0)) {
+            for (int j = threadIdx.x * 4; j < n3; j += blockDim.x * 4) {
+                uint4 v = ldg_nc_v4(src + j);
+                *reinterpret_cast<uint4 *>(rowbuf + j) = v;
+            }
+        } else {
+            for (int j = threadIdx.x; j < n3; j += blockDim.x) rowbuf[j] = src[j];
+        }
+        __syncthreads();
+        for (int b = threadIdx.x; b < m_b; b += blockDim.x) {
+            const int c0 = __ldg(colstart + b), c1 = __ldg(colstart + b + 1);
+            float rs = 0.f, rt = 0.f;
+            for (int c = c0; c < c1; ++c) {
+                const uint32_t ce = __ldg(colperm + c);
+                const int j = (int)(ce & 0x7FFFFFFFu);
+                const float sg = (ce >> 31) ? -1.f : 1.f;
+                const float x = rowbuf[j];
+                rs += sg * x;
+                if (MOM) rt = fmaf(sg * ((float)(j + 1) * inv_p3), x, rt);
+            }
+            accS[b] += v1 * rs;
+            if (MOM) {
+                accR[b] = fmaf(v1w, rs, accR[b]);
+                accT[b] += v1 * rt;
+            }
+        }
+    }
+    const long long mm = (long long)m_b * m_b;
+    float *dst = part + (long long)sp * 3 * mm + (long long)a * m_b;
+    for (int b = threadIdx.x; b < m_b; b += blockDim.x) {
+        dst[b] = accS[b];
+        if (MOM) { dst[mm + b] = accR[b]; dst[2 * mm + b] = accT[b]; }
+    }
+}
+
+// ---------------------------------------------------------------- FP32 SIMT contraction
+// C[M x N] = A[M x K] * B[K x N], all row-major, K a multiple of BK, FP32 FMA only (the
+// sketch noise is the measured quantity, so no reduced-precision tensor-core path here).
+// blockIdx.z = problem * ksplit + split; each split writes its own partial output.
+struct GemmBatch {
+    const float *A[3];
+    const float *B[3];
+    float *Cpart;     // [ksplit][3][M*N]
+    int M, N, K, lda, ldb, ksplit, kchunk;
+};
+
+template <int BM, int BN, int T>   // T = 4 or 8 outputs per thread per dimension; 256 threads
+__global__ void __launch_bounds__(256) sgemm_kernel(const GemmBatch g)
+{
+    constexpr int BK = 16;
+    constexpr int PADM = BM + 4, PADN = BN + 4;
+    __shared__ __align__(16) float As[2][BK][PADM];
+    __shared__ __align__(16) float Bs[2][BK][PADN];
+    const int prob = blockIdx.z / g.ksplit, ks = blockIdx.z % g.ksplit;
+    const float *__restrict__ A = g.A[prob];
+    const float *__restrict__ B = g.B[prob];
+    const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
+    const int k_begin = ks * g.kchunk, k_end = min(g.K, k_begin + g.kchunk);
+    const int tid = threadIdx.x;
+    constexpr int TX = BN / T;               // threads along N
+    const int tx = tid % TX, ty = tid / TX;
+    constexpr int HALF = T / 4;              // 1 or 2 groups of 4
+    // global -> smem assignment
+    constexpr int A_F4 = BM * BK / 4 / 256;  // float4 per thread for the A tile
+    constexpr int B_F4 = BK * BN / 4 / 256;
+    float4 ra[A_F4], rb[B_F4];
+    float acc[T][T];
+#pragma unroll
+    for (int i = 0; i < T; ++i)
+#pragma unroll
+        for (int j = 0; j < T; ++j) acc[i][j] = 0.f;
+
+    auto gload = [&](int k0) {
+#pragma unroll
+        for (int q = 0; q < A_F4; ++q) {
+            int f = tid + q * 256;           // float4 index in tile: row = f / 4, kq = f % 4
+            int row = f >> 2, kq = f & 3;
+            int gr = m0 + row;
+            ra[q] = (gr < g.M) ? *reinterpret_cast<const float4 *>(A + (long long)gr * g.lda + k0 + kq * 4)
+                               : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int q = 0; q < B_F4; ++q) {
+            int f = tid + q * 256;           // row k = f / (BN/4), c4 = f % (BN/4)
+            int kr = f / (BN / 4), c4 = f % (BN / 4);
+            int gc = n0 + c4 * 4;
+            rb[q] = (gc < g.ldb) ? *reinterpret_cast<const float4 *>(B + (long long)(k0 + kr) * g.ldb + gc)
+                                 : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    };
+    auto sstore = [&](int buf) {
+#pragma unroll
+        for (int q = 0; q < A_F4; ++q) {
+            int f = tid + q * 256;
+            int row = f >> 2, kq = f & 3;
+            As[buf][kq * 4 + 0][row] = ra[q].x;
+            As[buf][kq * 4 + 1][row] = ra[q].y;
+            As[buf][kq * 4 + 2][row] = ra[q].z;
+            As[buf][kq * 4 + 3][row] = ra[q].w;
+        }
+#pragma unroll
+        for (int q = 0; q < B_F4; ++q) {
+            int f = tid + q * 256;
+            int kr = f / (BN / 4), c4 = f % (BN / 4);
+            *reinterpret_cast<float4 *>(&Bs[buf][kr][c4 * 4]) = rb[q];
+        }
+    };
+
+    if (k_begin < k_end) {
+        gload(k_begin);
+        sstore(0);
+        __syncthreads();
+        int buf = 0;
+        for (int k0 = k_begin; k0 < k_end; k0 += BK) {
+            const bool more = (k0 + BK) < k_end;
+            if (more) gload(k0 + BK);
+#pragma unroll
+            for (int kk = 0; kk < BK; ++kk) {
+                float a[T], b[T];
+#pragma unroll
+                for (int h = 0; h < HALF; ++h) {
+                    float4 va = *reinterpret_cast<const float4 *>(&As[buf][kk][h * (BM / 2) + ty * 4]);
+                    float4 vb = *reinterpret_cast<const float4 *>(&Bs[buf][kk][h * (BN / 2) + tx * 4]);
+                    a[h * 4 + 0] = va.x; a[h * 4 + 1] = va.y; a[h * 4 + 2] = va.z; a[h * 4 + 3] = va.w;
+                    b[h * 4 + 0] = vb.x; b[h * 4 + 1] = vb.y; b[h * 4 + 2] = vb.z; b[h * 4 + 3] = vb.w;
+                }
+#pragma unroll
+                for (int i = 0; i < T; ++i)
+#pragma unroll
+                    for (int j = 0; j < T; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+            }
+            if (more) {
+                sstore(buf ^ 1);
+                __syncthreads();
+                buf ^= 1;
+            }
+        }
+    }
+    float *Cout = g.Cpart + ((long long)ks * 3 + prob) * (long long)g.M * g.N;
+#pragma unroll
+    for (int i = 0; i < T; ++i) {
+        const int row = m0 + (i / 4) * (BM / 2) * (HALF - 1) + (HALF == 1 ? ty * 4 + i : ty * 4 + (i & 3));
+        if (row >= g.M) continue;
+#pragma unroll
+        for (int j = 0; j < T; ++j) {
+            const int col = n0 + (j / 4) * (BN / 2) * (HALF - 1) + (HALF == 1 ? tx * 4 + j : tx * 4 + (j & 3));
+            if (col < g.N) Cout[(long long)row * g.N + col] = acc[i][j];
+        }
+    }
+}
+
+// ---------------------------------------------------------------- combine
+__global__ void combine_kernel(const float *partAB, int ksplit, const float *partC, int nsplit, long long mm,
+                               int nsk, float *S, float *R, float *T)
+{
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= mm) return;
+    for (int q = 0; q < nsk; ++q) {
+        float ab = partAB[(long long)q * mm + idx];
+        for (int s = 1; s < ksplit; ++s) ab += partAB[((long long)s * 3 + q) * mm + idx];
+        float c = partC[(long long)q * mm + idx];
+        for (int s = 1; s < nsplit; ++s) c += partC[((long long)s * 3 + q) * mm + idx];
+        float *dst = q == 0 ? S : (q == 1 ? R : T);
+        dst[idx] = ab - c;
+    }
+}
+
+// Subtract every confirmed fault from its bucket (Algorithm 1, peeling loop).  One thread:
+// the list is short and the order of subtractions is then fixed.
+__global__ void peel_kernel(const PeelEntry *F, int nF, uint32_t key1, uint32_t key2, int m_b, float inv_p1,
+                            float inv_p3, float *S, float *R, float *T)
+{
+    if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    for (int f = 0; f < nF; ++f) {
+        int a, b, s1, s2;
+        hash_index(key1, (uint32_t)F[f].i, (uint32_t)m_b, a, s1);
+        hash_index(key2, (uint32_t)F[f].j, (uint32_t)m_b, b, s2);
+        const double g = (double)(s1 * s2) * F[f].delta;
+        const long long o = (long long)a * m_b + b;
+        S[o] = (float)((double)S[o] - g);
+        R[o] = (float)((double)R[o] - g * ((double)(F[f].i + 1) * (double)inv_p1));
+        T[o] = (float)((double)T[o] - g * ((double)(F[f].j + 1) * (double)inv_p3));
+    }
+}
+
+// ---------------------------------------------------------------- host orchestration
+static int pow2_exp(long long n)
+{
+    int p = 0;
+    while ((1LL << p) < n) ++p;
+    return p;
+}
+
+void sketch_plan(long long n1, long long n2, long long n3, int m_b, SketchPlan &pl)
+{
+    pl.kpad = (int)((n2 + 15) / 16 * 16);
+    pl.npad = (m_b + 3) / 4 * 4;
+    int ns = (512 + m_b - 1) / m_b;
+    if (ns > 16) ns = 16;
+    long long avg_rows = n1 / m_b;
+    if (ns > avg_rows) ns = (int)(avg_rows > 1 ? avg_rows : 1);
+    pl.nsplit = ns < 1 ? 1 : ns;
+    pl.tile = m_b <= 192 ? 64 : 128;
+    const int tiles = ((m_b + pl.tile - 1) / pl.tile) * ((m_b + pl.tile - 1) / pl.tile) * 3;
+    int ks = (600 + tiles - 1) / tiles;
+    const int maxks = pl.kpad / 256 > 1 ? pl.kpad / 256 : 1;   // at least 256 of K per split
+    if (ks > maxks) ks = maxks;
+    if (ks > 32) ks = 32;
+    if (ks < 1) ks = 1;
+    int kchunk = ((pl.kpad + ks - 1) / ks + 15) / 16 * 16;
+    ks = (pl.kpad + kchunk - 1) / kchunk;
+    pl.ksplit = ks;
+    pl.kchunk = kchunk;
+}
+
+size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b)
+{
+    SketchPlan pl;
+    sketch_plan(n1, n2, n3, m_b, pl);
+    const size_t mm = (size_t)m_b * m_b;
+    size_t b = 0;
+    b += align_up((size_t)n1 * 4, 256) * 3;          // h1, v1, rowperm
+    b += align_up((size_t)n3 * 4, 256) * 3;          // h2, v2, colperm
+    b += align_up((size_t)(m_b + 1) * 4, 256) * 4;   // rowcount, rowstart, colcount, colstart
+    b += align_up((size_t)m_b * pl.kpad * 4, 256) * 2;       // P, Pw
+    b += align_up((size_t)pl.kpad * pl.npad * 4, 256) * 2;   // Q, Qw
+    b += align_up((size_t)pl.ksplit * 3 * mm * 4, 256);      // AB partials
+    b += align_up((size_t)pl.nsplit * 3 * mm * 4, 256);      // C partials
+    return b;
+}
+
+bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, SketchWs &w)
+{
+    if (ws_bytes < sketch_ws_bytes(n1, n2, n3, m_b)) return false;
+    sketch_plan(n1, n2, n3, m_b, w.pl);
+    const size_t mm = (size_t)m_b * m_b;
+    char *p = static_cast<char *>(ws);
+    auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
+    w.h1 = (int *)take((size_t)n1 * 4); w.v1 = (int *)take((size_t)n1 * 4); w.rowperm = (uint32_t *)take((size_t)n1 * 4);
+    w.h2 = (int *)take((size_t)n3 * 4); w.v2 = (int *)take((size_t)n3 * 4); w.colperm = (uint32_t *)take((size_t)n3 * 4);
+    w.rowcount = (int *)take((size_t)(m_b + 1) * 4); w.rowstart = (int *)take((size_t)(m_b + 1) * 4);
+    w.colcount = (int *)take((size_t)(m_b + 1) * 4); w.colstart = (int *)take((size_t)(m_b + 1) * 4);
+    w.P = (float *)take((size_t)m_b * w.pl.kpad * 4); w.Pw = (float *)take((size_t)m_b * w.pl.kpad * 4);
+    w.Q = (float *)take((size_t)w.pl.kpad * w.pl.npad * 4); w.Qw = (float *)take((size_t)w.pl.kpad * w.pl.npad * 4);
+    w.partAB = (float *)take((size_t)w.pl.ksplit * 3 * mm * 4);
+    w.partC = (float *)take((size_t)w.pl.nsplit * 3 * mm * 4);
+    return true;
+}
+
+int sketch_max_buckets(long long n1, long long n2, long long n3)
+{
+    // scatter_c_kernel keeps one row of C and three m_b-vectors in shared memory
+    const long long budget = 200 * 1024 - ((n3 + 3) / 4 * 4) * 4;
+    if (budget < 3 * 4) return 0;
+    long long m = budget / 12;
+    if (m > 16384) m = 16384;
+    return (int)m;
+}
+
+template <typename T>
+static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, int m_b, bool mom, SketchWs &w,
+                                    cudaStream_t st, float *S, float *R, float *Tt)
+{
+    const int n1 = (int)in.n1, n2 = (int)in.n2, n3 = (int)in.n3;
+    const float inv_p1 = 1.0f / (float)(1LL << pow2_exp(n1));
+    const float inv_p3 = 1.0f / (float)(1LL << pow2_exp(n3));
+    fpsk_status rc;
+    rc = build_hash_side(seed, rnd, 0, n1, m_b, w.h1, w.v1, w.rowcount, w.rowstart, w.rowperm, st);
+    if (rc != FPSK_OK) return rc;
+    rc = build_hash_side(seed, rnd, 1, n3, m_b, w.h2, w.v2, w.colcount, w.colstart, w.colperm, st);
+    if (rc != FPSK_OK) return rc;
+
+    const unsigned short *A = static_cast<const unsigned short *>(in.A);
+    const unsigned short *B = static_cast<const unsigned short *>(in.B);
+    const SketchPlan &pl = w.pl;
+    {
+        const bool vec = (reinterpret_cast<uintptr_t>(in.A) & 15) == 0 && in.lda % 8 == 0 && n2 % 8 == 0;
+        dim3 grid((pl.kpad / 8 + 127) / 128, m_b);
+#define FPSK_CA(V, M) compress_a_kernel<T, V, M><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw)
+        if (vec) { if (mom) FPSK_CA(true, true); else FPSK_CA(true, false); }
+        else     { if (mom) FPSK_CA(false, true); else FPSK_CA(false, false); }
+#undef FPSK_CA
+        FPSK_LAUNCH_CHECK();
+    }
+    {
+        const size_t smem = ((size_t)n3 * 2 + 15) / 16 * 16;
+        int grid = pl.kpad < 1184 ? pl.kpad : 1184;
+        if (mom) {
+            FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            compress_b_kernel<T, true><<<grid, 256, smem, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw);
+        } else {
+            FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            compress_b_kernel<T, false><<<grid, 256, smem, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw);
+        }
+        FPSK_LAUNCH_CHECK();
+    }
+    {
+        GemmBatch g;
+        g.A[0] = w.P; g.B[0] = w.Q;
+        g.A[1] = w.Pw; g.B[1] = w.Q;
+        g.A[2] = w.P; g.B[2] = w.Qw;
+        g.Cpart = w.partAB;
+        g.M = m_b; g.N = m_b; g.K = pl.kpad; g.lda = pl.kpad; g.ldb = pl.npad;
+        g.ksplit = pl.ksplit; g.kchunk = pl.kchunk;
+        const int nprob = mom ? 3 : 1;
+        if (pl.tile == 64) {
+            dim3 grid((m_b + 63) / 64, (m_b + 63) / 64, nprob * pl.ksplit);
+            sgemm_kernel<64, 64, 4><<<grid, 256, 0, st>>>(g);
+        } else {
+            dim3 grid((m_b + 127) / 128, (m_b + 127) / 128, nprob * pl.ksplit);
+            sgemm_kernel<128, 128, 8><<<grid, 256, 0, st>>>(g);
+        }
+        FPSK_LAUNCH_CHECK();
+    }
+    {
+        const size_t smem = ((size_t)((n3 + 3) & ~3) + 3 * (size_t)m_b) * 4;
+        dim3 grid(m_b, pl.nsplit);
+        if (mom) {
+            FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            scatter_c_kernel<true><<<grid, 256, smem, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, w.colperm, w.colstart, pl.nsplit, w.partC);
+        } else {
+            FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            scatter_c_kernel<false><<<grid, 256, smem, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, w.colperm, w.colstart, pl.nsplit, w.partC);
+        }
+        FPSK_LAUNCH_CHECK();
+    }
+    {
+        const long long mm = (long long)m_b * m_b;
+        combine_kernel<<<(unsigned)((mm + 255) / 256), 256, 0, st>>>(w.partAB, pl.ksplit, w.partC, pl.nsplit, mm, mom ? 3 : 1, S, R, Tt);
+        FPSK_LAUNCH_CHECK();
+    }
+    return FPSK_OK;
+}
+
+fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
+                           SketchWs &w, cudaStream_t st, float *S, float *R, float *T)
+{
+    if (dtype == FPSK_FP16) return build_sketches_t<__half>(in, seed, rnd, m_b, mom, w, st, S, R, T);
+    return build_sketches_t<__nv_bfloat16>(in, seed, rnd, m_b, mom, w, st, S, R, T);
+}
+
+fpsk_status peel_launch(const PeelEntry *dF, int nF, uint64_t seed, int rnd, long long n1, long long n3, int m_b,
+                        float *S, float *R, float *T, cudaStream_t st)
+{
+    if (nF <= 0) return FPSK_OK;
+    const float inv_p1 = 1.0f / (float)(1LL << pow2_exp(n1));
+    const float inv_p3 = 1.0f / (float)(1LL << pow2_exp(n3));
+    peel_kernel<<<1, 32, 0, st>>>(dF, nF, round_key(seed, rnd, 0), round_key(seed, rnd, 1), m_b, inv_p1, inv_p3, S, R, T);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+}  // namespace fpsk

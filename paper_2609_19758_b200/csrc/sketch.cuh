@@ -1,0 +1,95 @@
+// Internal interfaces between the sketch builder, the selection / confirmation kernels and
+// the C ABI layer.
+#pragma once
+#include "fpsk_common.cuh"
+
+namespace fpsk {
+
+struct PeelEntry {          // a confirmed fault as the peeling kernel needs it
+    int i, j;
+    double delta;
+};
+
+struct SketchPlan {
+    int kpad;      // n2 rounded up to 16: K extent of the contraction
+    int npad;      // m_b rounded up to 4: leading dimension of Q, Qw
+    int nsplit;    // row splits per bucket row in the C scatter
+    int ksplit;    // K splits of the contraction
+    int kchunk;    // K extent per split (multiple of 16)
+    int tile;      // 64 or 128
+};
+
+struct SketchWs {
+    SketchPlan pl;
+    int *h1, *v1, *h2, *v2;
+    uint32_t *rowperm, *colperm;
+    int *rowcount, *rowstart, *colcount, *colstart;
+    float *P, *Pw, *Q, *Qw, *partAB, *partC;
+};
+
+struct SketchIn {
+    const void *A, *B;
+    const float *C;
+    long long n1, n2, n3, lda, ldb, ldc;
+};
+
+void sketch_plan(long long n1, long long n2, long long n3, int m_b, SketchPlan &pl);
+size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b);
+bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, SketchWs &w);
+int sketch_max_buckets(long long n1, long long n2, long long n3);
+
+fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, int *bucket, int *sign,
+                            int *count, int *start, uint32_t *perm, cudaStream_t st);
+fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
+                           SketchWs &w, cudaStream_t st, float *S, float *R, float *T);
+fpsk_status peel_launch(const PeelEntry *dF, int nF, uint64_t seed, int rnd, long long n1, long long n3, int m_b,
+                        float *S, float *R, float *T, cudaStream_t st);
+
+// ---- selection (select.cu) -----------------------------------------------------------------
+struct Candidate {          // one decoded bucket of the set U (Algorithm 1)
+    int flat;               // a*m_b + b
+    int ih, jh;             // rounded 0-based coordinate estimate
+    float s_abs;
+};
+
+struct SelectWs {           // all device memory
+    unsigned int *hist;     // 256 bins + control words
+    unsigned long long *state;   // radix-select state
+    float *scal;            // scalar results: [0] median, [1] sigma_mad, [2] mean|S|, [3] sigma_clip,
+                            //                 [4] thr, [5] tau_c, [6] tau_d
+    float *partial;         // per-CTA partial sums
+    unsigned long long *keys;    // selected keys (<= kmax)
+    int *counts;            // [0] above-threshold count, [1] collected, [2] n_U
+    Candidate *cand;        // <= kmax
+};
+constexpr int kSelMaxK = 1024;
+size_t select_ws_bytes();
+void select_carve(void *ws, SelectWs &w);
+
+// sigma_MAD of S (mad_of_abs: of |S| as printed, else signed) -> scal[1]; median -> scal[0]
+fpsk_status sigma_mad_launch(const float *S, long long mm, int mad_of_abs, SelectWs &w, cudaStream_t st);
+// clipped-mean estimate 1.2533 mean(min(|S|, 5 mean|S|)) -> scal[3]
+fpsk_status sigma_clip_launch(const float *S, long long mm, SelectWs &w, cudaStream_t st);
+// thresholds from scal[1] and tau, K largest |S| above max(tau_c, tau_d), decoded candidates
+fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
+                                     long long n3, const float *d_tau, int radius, int K, SelectWs &w, cudaStream_t st);
+// device max |X| of a half matrix -> out[0] (float)
+fpsk_status max_abs_half_launch(const void *X, long long ld, long long rows, long long cols, fpsk_dtype dtype,
+                                float *out, unsigned int *scratch, cudaStream_t st);
+// strided, clipped rms of C (Section "Calibration") -> scal_out[0]; uses SelectWs for the median
+fpsk_status rms_c_launch(const float *C, long long ldc, long long n1, long long n3, float *samples,
+                         SelectWs &w, float *out, cudaStream_t st);
+
+// ---- confirmation (confirm.cu) ---------------------------------------------------------------
+struct Hit {                // an accepted window entry
+    int cand;               // index into the candidate list
+    int di, dj;             // offset from the candidate's estimate
+    int i, j;
+    float c_value;
+    double gamma;           // FP64 recomputation
+};
+fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
+                           int max_cand, int radius, double c_valid, Hit *hits, int *n_hits, int hit_cap,
+                           cudaStream_t st);
+
+}  // namespace fpsk

@@ -1,0 +1,275 @@
+"""Thin ctypes binding over ``libfpsk.so`` (the C ABI declared in ``include/fpsk.h``).
+
+Argument marshalling only: every step of the verifier runs inside the CUDA library.  PyTorch
+supplies device memory and streams.  If the library has not been built this module raises;
+there is no fallback path.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libfpsk.so")
+
+FP16, BF16 = 0, 1
+STATUS_OK = 0
+ERR_NULL, ERR_SHAPE, ERR_DTYPE, ERR_ALIGN, ERR_WORKSPACE, ERR_BUCKETS, ERR_CAPACITY, ERR_CUDA, ERR_TIMEOUT, ERR_PARAM = range(1, 11)
+
+
+class ProbeResult(C.Structure):
+    _fields_ = [("fired", C.c_int32), ("nonfinite", C.c_int32), ("argmax_col", C.c_int32), ("status", C.c_int32),
+                ("max_abs", C.c_float), ("sigma_hat", C.c_float), ("thr", C.c_float), ("tau", C.c_float)]
+
+
+class Fault(C.Structure):
+    _fields_ = [("i", C.c_int32), ("j", C.c_int32), ("delta", C.c_double), ("recompute", C.c_double),
+                ("c_value", C.c_float), ("round", C.c_int32), ("bucket_a", C.c_int32), ("bucket_b", C.c_int32)]
+
+
+class Params(C.Structure):
+    _fields_ = [("rounds", C.c_int32), ("r_star", C.c_int32), ("r_max", C.c_int32), ("radius", C.c_int32),
+                ("s_budget", C.c_int32), ("delta_max", C.c_int32), ("mad_of_abs", C.c_int32), ("reserved", C.c_int32),
+                ("rho_min", C.c_double), ("c_valid", C.c_double), ("mu", C.c_double), ("b_star", C.c_double),
+                ("c_coll", C.c_double)]
+
+
+class Noise(C.Structure):
+    _fields_ = [("sigma_clip", C.c_double), ("sigma_mad", C.c_double), ("rms_c", C.c_double), ("c_hat", C.c_double),
+                ("index_budget_B", C.c_double), ("m0", C.c_int32), ("m_probe", C.c_int32), ("m_loc", C.c_int32),
+                ("radius", C.c_int32)]
+
+
+class FpskError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: fpsk status {status} ({status_string(status)})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """The loaded shared library; raises if it is missing (build it with
+    ``python -m paper_2609_19758_b200.build``)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise FileNotFoundError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_19758_b200.build`")
+        L = C.CDLL(LIB_PATH)
+        vp, i64, i32, u64, sz = C.c_void_p, C.c_int64, C.c_int32, C.c_uint64, C.c_size_t
+        L.fpsk_status_string.restype = C.c_char_p
+        L.fpsk_status_string.argtypes = [C.c_int]
+        L.fpsk_default_params.restype = None
+        L.fpsk_default_params.argtypes = [C.POINTER(Params)]
+        L.fpsk_law_m_start.restype = i32
+        L.fpsk_law_m_start.argtypes = [i64, i64, i64, C.c_int, C.POINTER(Params)]
+        L.fpsk_plan.restype = C.c_int
+        L.fpsk_plan.argtypes = [i64, i64, i64, C.c_int, C.c_double, C.c_double, i32, C.POINTER(Params),
+                                C.POINTER(i32), C.POINTER(i32), C.POINTER(C.c_double)]
+        L.fpsk_probe_workspace_bytes.restype = sz
+        L.fpsk_probe_workspace_bytes.argtypes = [i64, i64, i64]
+        L.fpsk_probe_init.restype = C.c_int
+        L.fpsk_probe_init.argtypes = [vp, sz, vp]
+        L.fpsk_probe.restype = C.c_int
+        L.fpsk_probe.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, C.c_int, C.POINTER(Params),
+                                 vp, sz, vp, vp, vp]
+        L.fpsk_probe_host_workspace_bytes.restype = sz
+        L.fpsk_probe_host_workspace_bytes.argtypes = [i64, i64, i64]
+        L.fpsk_probe_host.restype = C.c_int
+        L.fpsk_probe_host.argtypes = [vp, vp, vp, i64, i64, i64, C.c_int, C.POINTER(Params), vp, sz, vp,
+                                      C.POINTER(ProbeResult)]
+        L.fpsk_hash_tables.restype = C.c_int
+        L.fpsk_hash_tables.argtypes = [u64, i32, i32, i64, i32, vp, vp, vp]
+        L.fpsk_workspace_bytes.restype = sz
+        L.fpsk_workspace_bytes.argtypes = [i64, i64, i64, i32, C.POINTER(Params)]
+        L.fpsk_max_buckets.restype = i32
+        L.fpsk_max_buckets.argtypes = [i64, i64, i64]
+        L.fpsk_sketches.restype = C.c_int
+        L.fpsk_sketches.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32, i32, vp, sz, vp,
+                                    vp, vp, vp]
+        L.fpsk_measure_noise.restype = C.c_int
+        L.fpsk_measure_noise.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32,
+                                         C.POINTER(Params), vp, sz, vp, C.POINTER(Noise)]
+        L.fpsk_localize.restype = C.c_int
+        L.fpsk_localize.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32, C.POINTER(Params),
+                                    vp, sz, vp, C.POINTER(Fault), i32, C.POINTER(i32)]
+        L.fpsk_launch_count.restype = u64
+        L.fpsk_launch_count.argtypes = []
+        _lib = L
+    return _lib
+
+
+def status_string(s: int) -> str:
+    return lib().fpsk_status_string(int(s)).decode()
+
+
+def default_params(**kw) -> Params:
+    p = Params()
+    lib().fpsk_default_params(C.byref(p))
+    for k, v in kw.items():
+        setattr(p, k, v)
+    return p
+
+
+def launch_count() -> int:
+    return int(lib().fpsk_launch_count())
+
+
+def dtype_of(t: torch.Tensor) -> int:
+    if t.dtype == torch.float16:
+        return FP16
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"operands must be float16 or bfloat16, got {t.dtype}")
+
+
+def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return int(s.cuda_stream)
+
+
+def _mat_args(A: torch.Tensor, B: torch.Tensor, Cm: torch.Tensor):
+    assert A.is_cuda and B.is_cuda and Cm.is_cuda, "A, B, C must be device tensors"
+    assert A.dim() == 2 and B.dim() == 2 and Cm.dim() == 2
+    assert A.stride(1) == 1 and B.stride(1) == 1 and Cm.stride(1) == 1, "row-major (unit column stride) required"
+    m, k = A.shape
+    k2, n = B.shape
+    assert k2 == k and tuple(Cm.shape) == (m, n) and A.dtype == B.dtype
+    return (A.data_ptr(), A.stride(0) if m > 1 else max(k, A.stride(0)), B.data_ptr(),
+            B.stride(0) if k > 1 else max(n, B.stride(0)), Cm.data_ptr(), Cm.stride(0) if m > 1 else max(n, Cm.stride(0)),
+            m, k, n, dtype_of(A))
+
+
+def law_m_start(m: int, k: int, n: int, dtype: int, params: Optional[Params] = None) -> int:
+    return int(lib().fpsk_law_m_start(m, k, n, dtype, C.byref(params) if params is not None else None))
+
+
+def plan(m: int, k: int, n: int, dtype: int, sigma_hat: float, rms_c: float, m_cur: int,
+         params: Optional[Params] = None) -> Tuple[int, int, float]:
+    ml, r, B = C.c_int32(), C.c_int32(), C.c_double()
+    rc = lib().fpsk_plan(m, k, n, dtype, sigma_hat, rms_c, m_cur, C.byref(params) if params is not None else None,
+                         C.byref(ml), C.byref(r), C.byref(B))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_plan")
+    return ml.value, r.value, B.value
+
+
+def probe_workspace(m: int, k: int, n: int, device=None, stream=None) -> torch.Tensor:
+    """Allocate and prepare a probe workspace (torch owns the memory)."""
+    nbytes = int(lib().fpsk_probe_workspace_bytes(m, k, n))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+    rc = lib().fpsk_probe_init(ws.data_ptr(), nbytes, _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_init")
+    return ws
+
+
+def probe(A, B, Cm, workspace: torch.Tensor, result: torch.Tensor, residual: Optional[torch.Tensor] = None,
+          params: Optional[Params] = None, stream=None, c_is_fp32: Optional[bool] = None) -> None:
+    """Asynchronous probe; `result` is a device uint8 tensor of sizeof(ProbeResult) bytes."""
+    a = _mat_args(A, B, Cm)
+    if c_is_fp32 is None:
+        c_is_fp32 = Cm.dtype == torch.float32
+    rc = lib().fpsk_probe(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], 1 if c_is_fp32 else 0,
+                          C.byref(params) if params is not None else None, workspace.data_ptr(), workspace.numel(),
+                          _stream_ptr(stream), result.data_ptr(), residual.data_ptr() if residual is not None else None)
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe")
+
+
+def new_probe_result(device=None) -> torch.Tensor:
+    return torch.zeros(C.sizeof(ProbeResult), dtype=torch.uint8, device=device or "cuda")
+
+
+def read_probe_result(result: torch.Tensor) -> ProbeResult:
+    """Synchronising read of a device verdict."""
+    host = result.cpu().numpy().tobytes()
+    return ProbeResult.from_buffer_copy(host)
+
+
+def probe_host(hA: torch.Tensor, hB: torch.Tensor, hC: torch.Tensor, workspace: torch.Tensor,
+               params: Optional[Params] = None, stream=None) -> ProbeResult:
+    """Probe of operands that live in (pinned) host memory; returns the verdict on the host."""
+    assert not hA.is_cuda and not hB.is_cuda and not hC.is_cuda
+    assert hA.is_contiguous() and hB.is_contiguous() and hC.is_contiguous() and hC.dtype == torch.float32
+    m, k = hA.shape
+    n = hB.shape[1]
+    res = ProbeResult()
+    rc = lib().fpsk_probe_host(hA.data_ptr(), hB.data_ptr(), hC.data_ptr(), m, k, n, dtype_of(hA),
+                               C.byref(params) if params is not None else None, workspace.data_ptr(),
+                               workspace.numel(), _stream_ptr(stream), C.byref(res))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_host")
+    return res
+
+
+def probe_host_workspace(m: int, k: int, n: int, device=None, stream=None) -> torch.Tensor:
+    nbytes = int(lib().fpsk_probe_host_workspace_bytes(m, k, n))
+    ws = torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+    rc = lib().fpsk_probe_init(ws.data_ptr(), nbytes, _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_init")
+    return ws
+
+
+def hash_tables(seed: int, rnd: int, side: int, count: int, n_buckets: int, device=None, stream=None):
+    b = torch.empty(count, dtype=torch.int32, device=device or "cuda")
+    s = torch.empty(count, dtype=torch.int32, device=device or "cuda")
+    rc = lib().fpsk_hash_tables(seed, rnd, side, count, n_buckets, b.data_ptr(), s.data_ptr(), _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_hash_tables")
+    return b, s
+
+
+def workspace(m: int, k: int, n: int, n_buckets: int, params: Optional[Params] = None, device=None) -> torch.Tensor:
+    nbytes = int(lib().fpsk_workspace_bytes(m, k, n, n_buckets, C.byref(params) if params is not None else None))
+    if nbytes == 0:
+        raise FpskError(ERR_BUCKETS, "fpsk_workspace_bytes")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+
+
+def max_buckets(m: int, k: int, n: int) -> int:
+    return int(lib().fpsk_max_buckets(m, k, n))
+
+
+def sketches(A, B, Cm, seed: int, rnd: int, n_buckets: int, ws: torch.Tensor, moments: bool = True, stream=None):
+    a = _mat_args(A, B, Cm)
+    S = torch.empty((n_buckets, n_buckets), dtype=torch.float32, device=A.device)
+    R = torch.empty_like(S) if moments else None
+    T = torch.empty_like(S) if moments else None
+    rc = lib().fpsk_sketches(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, rnd, n_buckets,
+                             ws.data_ptr(), ws.numel(), _stream_ptr(stream), S.data_ptr(),
+                             R.data_ptr() if moments else None, T.data_ptr() if moments else None)
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_sketches")
+    return S, R, T
+
+
+def measure_noise(A, B, Cm, seed: int, ws: torch.Tensor, m0: int = 0, params: Optional[Params] = None,
+                  stream=None) -> Noise:
+    a = _mat_args(A, B, Cm)
+    out = Noise()
+    rc = lib().fpsk_measure_noise(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, m0,
+                                  C.byref(params) if params is not None else None, ws.data_ptr(), ws.numel(),
+                                  _stream_ptr(stream), C.byref(out))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_measure_noise")
+    return out
+
+
+def localize(A, B, Cm, seed: int, n_buckets: int, ws: torch.Tensor, params: Optional[Params] = None,
+             capacity: int = 1024, stream=None) -> List[Fault]:
+    a = _mat_args(A, B, Cm)
+    buf = (Fault * capacity)()
+    cnt = C.c_int32(0)
+    rc = lib().fpsk_localize(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, n_buckets,
+                             C.byref(params) if params is not None else None, ws.data_ptr(), ws.numel(),
+                             _stream_ptr(stream), buf, capacity, C.byref(cnt))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_localize")
+    return [buf[i] for i in range(cnt.value)]
