@@ -1,0 +1,386 @@
+#!/usr/bin/env python
+"""Benchmark of the FP-Sketch verifier hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input:
+    probe (detection sketch + verdict)  ->  run-time noise measurement on the clean product
+    ->  localization of the injected faults (hash rounds, candidates, FP64 confirmation).
+Workload: square BF16 product m=k=n=4096, A ~ N(0,1), B ~ N(0, sd 1/sqrt(k)), FP32 C from the
+vendor GEMM, 4 additive faults of 2-9 % of rms(C) per batch; batches rotate so that no input
+is served from L2, and a 256 MiB read flushes L2 before every probe.
+
+Prints ONE JSON line.  The headline metric is the clean-path probe's HBM throughput
+(algorithmic bytes 2mk + 2kn + 4mn over the probe kernel's device time); probe ms, vendor
+GEMM ms, localize ms, recovery and the measured noise constant ride along.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+FALLBACK_HBM_GBS = 6650.0
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--shape", default="4096,4096,4096", help="m,k,n (default: the benchmark configuration)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"])
+    ap.add_argument("--kind", default="gauss_scaled")
+    ap.add_argument("--sets", type=int, default=3, help="rotating input batches")
+    ap.add_argument("--probe-only", action="store_true", help="time only the probe (profiling aid)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(p) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(index), "--query-gpu=" + self.Q,
+                                       "--format=csv,noheader,nounits", "-lms", "100"],
+                                      stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        time.sleep(0.15)
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 8:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[4:8]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        try:
+            os.unlink(self.f.name)
+        except OSError:
+            pass
+        if sm:
+            # "under load": samples within 25 % of the highest clock seen are the loaded ones
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = max(mx)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+def algorithmic_bytes(m, k, n):
+    return 2 * m * k + 2 * k * n + 4 * m * n
+
+
+def make_batches(args, m, k, n, dt, nsets, seed0=0):
+    from paper_2609_19758_b200 import harness, workloads as W
+    batches = []
+    for s in range(nsets):
+        A, B = W.operands(args.kind, m, k, n, dt, seed0 + s)
+        dA, dB = A.cuda(), B.cuda()
+        C = harness.vendor_gemm_fp32(dA, dB)
+        rms = float(torch.sqrt(torch.mean(C.double() ** 2)))
+        faults = W.faults_additive(m, n, rms, seed0 + s, 4, 0.02, 0.09, "small")
+        Cf = C.clone()
+        for f in faults:
+            Cf[f.i, f.j] += f.value
+        batches.append(dict(A=dA, B=dB, C=C, Cf=Cf, faults=faults, rms=rms, hA=A, hB=B))
+    return batches
+
+
+def run_ours(args):
+    from paper_2609_19758_b200 import build as Bld
+    from paper_2609_19758_b200 import fpsk, harness, workloads as W
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    if rank == 0:
+        Bld.build()
+    if dist is not None:
+        dist.barrier()
+    fpsk.lib()
+
+    m, k, n = (int(x) for x in args.shape.split(","))
+    dt = W.BF16 if args.dtype == "bf16" else W.FP16
+    K, Wm = args.steps, max(args.warmup, 3)
+    nsets = max(args.sets, 3 if algorithmic_bytes(m, k, n) < 512e6 else 2)
+    batches = make_batches(args, m, k, n, dt, nsets, seed0=100 * rank)
+    params = fpsk.default_params(s_budget=4)
+    pws = fpsk.probe_workspace(m, k, n)
+    res = fpsk.new_probe_result()
+    resid = torch.empty(n, dtype=torch.float32, device="cuda")
+    # workspace sized for the largest bucket count the plan can ask for
+    mb_cap = min(fpsk.max_buckets(m, k, n), max(16, int((m * n // 16) ** 0.5)))
+    mb_cap = max(mb_cap, fpsk.law_m_start(m, k, n, dt, params))
+    ws = fpsk.workspace(m, k, n, mb_cap, params)
+    flush = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")     # 256 MiB, read (not written) to evict L2
+    nbytes = algorithmic_bytes(m, k, n)
+
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    pe = [(ev(), ev()) for _ in range(K)]
+    ne = [(ev(), ev()) for _ in range(K)]
+    le = [(ev(), ev()) for _ in range(K)]
+    t0, t1 = ev(), ev()
+    found = injected = false_pos = fired_n = 0
+    c_hats, plans = [], []
+    launches0 = 0
+    sampler = None
+    for s in range(Wm + K):
+        if s == Wm:
+            if dist is not None:
+                dist.barrier()
+            torch.cuda.synchronize()
+            sampler = ClockSampler(local) if rank == 0 else None
+            launches0 = fpsk.launch_count()
+            t0.record()
+        b = batches[s % nsets]
+        i = s - Wm
+        flush_sink = flush.max()                        # a 256 MiB READ evicts the inputs from L2 and leaves no dirty lines
+        if i >= 0:
+            pe[i][0].record()
+        fpsk.probe(b["A"], b["B"], b["Cf"], pws, res, resid, params)
+        if i >= 0:
+            pe[i][1].record()
+        if args.probe_only:
+            continue
+        verdict = fpsk.read_probe_result(res)           # the one host read of the verdict
+        if i >= 0:
+            ne[i][0].record()
+        nz = fpsk.measure_noise(b["A"], b["B"], b["C"], 1000 + s, ws, 0, params)
+        if i >= 0:
+            ne[i][1].record()
+            le[i][0].record()
+        params.radius = nz.radius
+        got = fpsk.localize(b["A"], b["B"], b["Cf"], 1000 + s, min(nz.m_loc, mb_cap), ws, params)
+        if i >= 0:
+            le[i][1].record()
+            want = {(f.i, f.j) for f in b["faults"]}
+            have = {(f.i, f.j) for f in got}
+            found += len(want & have)
+            injected += len(want)
+            false_pos += len(have - want)
+            fired_n += int(verdict.fired)
+            c_hats.append(nz.c_hat)
+            plans.append((nz.m0, nz.m_loc, nz.radius))
+    t1.record()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    launches = fpsk.launch_count() - launches0
+    clocks = sampler.stop() if sampler else None
+    total_ms = t0.elapsed_time(t1)
+    probe_ms = [a.elapsed_time(b_) for a, b_ in pe]
+    noise_ms = [a.elapsed_time(b_) for a, b_ in ne] if not args.probe_only else [0.0]
+    loc_ms = [a.elapsed_time(b_) for a, b_ in le] if not args.probe_only else [0.0]
+    probe_mean = sum(probe_ms) / len(probe_ms)
+
+    # vendor GEMM under test, timed alongside (not part of the product)
+    g0, g1 = ev(), ev()
+    b = batches[0]
+    for _ in range(3):
+        harness.vendor_gemm_fp32(b["A"], b["B"])
+    torch.cuda.synchronize()
+    g0.record()
+    for q in range(10):
+        bb = batches[q % nsets]
+        harness.vendor_gemm_fp32(bb["A"], bb["B"])
+    g1.record()
+    torch.cuda.synchronize()
+    gemm_ms = g0.elapsed_time(g1) / 10
+
+    # end to end through the C ABI with HOST buffers: H2D of A, B, C and D2H of the verdict inside
+    hws = fpsk.probe_host_workspace(m, k, n)
+    hb = [dict(A=x["hA"].pin_memory(), B=x["hB"].pin_memory(), C=x["Cf"].cpu().pin_memory()) for x in batches[:2]]
+    Ke = min(K, 20)
+    for q in range(2):
+        fpsk.probe_host(hb[q % 2]["A"], hb[q % 2]["B"], hb[q % 2]["C"], hws, params)
+    torch.cuda.synchronize()
+    w0 = time.perf_counter()
+    for q in range(Ke):
+        r_ = fpsk.probe_host(hb[q % 2]["A"], hb[q % 2]["B"], hb[q % 2]["C"], hws, params)
+    torch.cuda.synchronize()
+    e2e_ms = (time.perf_counter() - w0) * 1e3 / Ke
+
+    # max over ranks
+    stats = torch.tensor([probe_mean, total_ms / K, e2e_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
+    probe_mean_x, step_ms_x, e2e_ms_x = (float(x) for x in stats.cpu())
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    peak, peak_src = measured_peak()
+    gbs = nbytes / (probe_mean_x * 1e-3) / 1e9
+    out = {
+        "metric": "clean-path probe HBM GB/s (probe ms beside vendor GEMM ms; fault recovery rate)",
+        "value": gbs * world,
+        "unit": "GB/s",
+        "n_gpus": world,
+        "steps": K,
+        "warmup": Wm,
+        "ms_per_step": step_ms_x,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": args.dtype,
+        "data": "synthetic",
+        "config": {
+            "workload": f"square {args.dtype.upper()} product m=k=n={m}" if m == k == n else f"{m}x{k}x{n} {args.dtype}",
+            "recipe": f"{args.kind}: A~N(0,1), B~N(0,1/sqrt(k)); FP32 C from the vendor GEMM; 4 faults of 2-9% rms(C) per batch",
+            "step": "probe + noise measurement (clean C) + localize (3 hash rounds, FP64 confirm)",
+            "l2": f"256 MiB flush read before every probe; {nsets} rotating input batches (each 134 MB > L2)",
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+        },
+        "probe_ms": probe_mean_x,
+        "probe_ms_median": statistics.median(probe_ms),
+        "probe_ms_min": min(probe_ms),
+        "gemm_ms": gemm_ms,
+        "probe_over_gemm": probe_mean_x / gemm_ms,
+        "measure_noise_ms": statistics.median(noise_ms),
+        "localize_ms": statistics.median(loc_ms),
+        "recovery": {"found": found, "injected": injected, "rate": (found / injected) if injected else None,
+                     "false_positives": false_pos, "probe_fired": fired_n, "steps": K},
+        "noise": {"c_hat_median": statistics.median(c_hats) if c_hats else None,
+                  "plan_m0_mloc_r": list(plans[len(plans) // 2]) if plans else None},
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
+                     "peak_source": peak_src + " copy bandwidth (MEASURED_PEAKS.json)" if peak_src == "measured" else "fallback 6650",
+                     "frac_of_nominal_8TBs": gbs / 8000.0, "kernel": "probe_kernel", "bytes_per_launch": nbytes,
+                     "traffic": None},
+        "e2e": {"value": nbytes / (e2e_ms_x * 1e-3) / 1e9 * world, "unit": "GB/s", "ms": e2e_ms_x,
+                "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 32},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    traffic_file = os.path.join(ROOT, "profiles", "probe_traffic.json")
+    try:
+        with open(traffic_file) as f:
+            tj = json.load(f)
+        key = f"{m}x{k}x{n}_{args.dtype}"
+        if key in tj:
+            out["roofline"]["traffic"] = tj[key]
+    except Exception:
+        pass
+    if not args.no_cpu_baseline and not args.probe_only:
+        out["cpu_baseline"] = cpu_baseline(args, batches[0], m, k, n, dt, nbytes)
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def oracle_probe_once(A64, B64, C64):
+    import oracle as O
+    E = O.error_matrix(A64, B64, C64)
+    s = O.probe_sketch(E)
+    return O.probe_verdict(s, O.analytic_tau(A64, B64, A64.shape[1]))
+
+
+def cpu_baseline(args, batch, m, k, n, dt, nbytes):
+    """The oracle as it stands, timed on this machine's host cores: one full-size probe
+    (explicit E = AB - C in FP64, column sums, verdict)."""
+    A64 = batch["hA"].double().numpy()
+    B64 = batch["hB"].double().numpy()
+    C64 = batch["Cf"].cpu().numpy()
+    t = time.perf_counter()
+    v = oracle_probe_once(A64, B64, C64)
+    dt_s = time.perf_counter() - t
+    return {"value": nbytes / dt_s / 1e9, "unit": "GB/s", "ms": dt_s * 1e3, "cores": os.cpu_count(), "kind": "oracle",
+            "fired": bool(v.fired),
+            "sample": f"one full-size oracle probe of the {m}x{k}x{n} workload (FP64 explicit E, numpy/OpenBLAS threads)"}
+
+
+def run_reference(args):
+    """The CPU oracle timed as the reference arm: each step is one oracle probe of the same
+    workload (bounded: a step is a few seconds at 4096^3)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2609_19758_b200 import workloads as W
+    m, k, n = (int(x) for x in args.shape.split(","))
+    dt = W.BF16 if args.dtype == "bf16" else W.FP16
+    nbytes = algorithmic_bytes(m, k, n)
+    A, B = W.operands(args.kind, m, k, n, dt, 0)
+    C = W.cpu_fp32_product(A, B)
+    C[3, 5] += 0.05
+    A64, B64, C64 = A.double().numpy(), B.double().numpy(), C.numpy()
+    K = min(args.steps, 30)
+    Wm = min(max(args.warmup, 1), 2)
+    for _ in range(Wm):
+        oracle_probe_once(A64, B64, C64)
+    t = time.perf_counter()
+    for _ in range(K):
+        oracle_probe_once(A64, B64, C64)
+    ms = (time.perf_counter() - t) * 1e3 / K
+    gbs = nbytes / (ms * 1e-3) / 1e9
+    sample = f"{K} oracle probes of the full {m}x{k}x{n} workload (steps capped at 30 to bound the run)"
+    print(json.dumps({
+        "impl": "reference", "metric": "clean-path probe HBM GB/s (probe ms beside vendor GEMM ms; fault recovery rate)",
+        "value": gbs, "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": Wm,
+        "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": f"square {args.dtype.upper()} product m=k=n={m}" if m == k == n else f"{m}x{k}x{n}"},
+        "probe_ms": ms,
+        "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": os.cpu_count(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -78,10 +78,21 @@ template <> struct HalfTraits<__nv_bfloat16> {
     }
 };
 
-// |x| of two packed 16-bit floats, as raw bits (sign bits cleared); for finite values the
-// unsigned 16-bit order of these bits is the order of the magnitudes in both formats.
-__device__ __forceinline__ uint32_t abs2_bits(uint32_t w) { return w & 0x7FFF7FFFu; }
-__device__ __forceinline__ uint32_t max2_u16(uint32_t a, uint32_t b) { return __vmaxu2(a, b); }
+// Running max of |x| over packed pairs of 16-bit floats, kept as a packed pair: one abs and
+// one max instruction per two elements (native HMNMX2).  NaN operands are ignored by the max.
+template <typename T> __device__ __forceinline__ uint32_t absmax2(uint32_t acc, uint32_t w);
+template <> __device__ __forceinline__ uint32_t absmax2<__half>(uint32_t acc, uint32_t w)
+{
+    __half2 a = *reinterpret_cast<__half2 *>(&acc), b = *reinterpret_cast<__half2 *>(&w);
+    a = __hmax2(a, __habs2(b));
+    return *reinterpret_cast<uint32_t *>(&a);
+}
+template <> __device__ __forceinline__ uint32_t absmax2<__nv_bfloat16>(uint32_t acc, uint32_t w)
+{
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&acc), b = *reinterpret_cast<__nv_bfloat162 *>(&w);
+    a = __hmax2(a, __habs2(b));
+    return *reinterpret_cast<uint32_t *>(&a);
+}
 
 template <typename T> __device__ __forceinline__ float bits16_to_float(uint32_t b);
 template <> __device__ __forceinline__ float bits16_to_float<__half>(uint32_t b)

@@ -9,6 +9,8 @@
 #include "fpsk_common.cuh"
 
 #include <math.h>
+#include <stdlib.h>
+#include <string.h>
 #include <mutex>
 
 namespace fpsk {
@@ -16,7 +18,6 @@ namespace fpsk {
 constexpr int kProbeThreads = 512;
 constexpr int kMaxTpr = 128;      // threads that share one row segment (x8 halves / x4 floats)
 constexpr int kUChunk = 2048;     // u values staged in shared memory per GEMV chunk
-constexpr int kCtrlWords = 64;
 
 struct Decomp {
     int cg;      // column groups
@@ -36,7 +37,18 @@ struct ProbeArgs {
     float *s;                 // n3 floats
     fpsk_probe_result *result;
     float mu;
+    long long *trace;         // optional per-CTA phase timestamps (NULL = off)
+    float4 *vstat;            // per-CTA statistics of its slice of s: (sum|s|, bad, max|s|, argmax as bits)
 };
+
+__device__ __forceinline__ void trace_mark(const ProbeArgs &p, int c, int k)
+{
+    if (p.trace) {
+        unsigned long long t;
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        p.trace[c * 32 + k] = (long long)t;
+    }
+}
 
 template <bool VEC>
 __device__ __forceinline__ uint4 load8h(const unsigned short *X, long long ld, long long row,
@@ -77,8 +89,7 @@ __device__ __forceinline__ void add8(float (&acc)[8], const uint4 &v, unsigned i
     f = HalfTraits<T>::unpack2(v.y); acc[2] += f.x; acc[3] += f.y;
     f = HalfTraits<T>::unpack2(v.z); acc[4] += f.x; acc[5] += f.y;
     f = HalfTraits<T>::unpack2(v.w); acc[6] += f.x; acc[7] += f.y;
-    mx = max2_u16(mx, max2_u16(max2_u16(abs2_bits(v.x), abs2_bits(v.y)),
-                               max2_u16(abs2_bits(v.z), abs2_bits(v.w))));
+    mx = absmax2<T>(absmax2<T>(absmax2<T>(absmax2<T>(mx, v.x), v.y), v.z), v.w);
 }
 
 template <typename T>
@@ -89,8 +100,108 @@ __device__ __forceinline__ void fma8(float (&acc)[8], const uint4 &v, float u, u
     f = HalfTraits<T>::unpack2(v.y); acc[2] = fmaf(u, f.x, acc[2]); acc[3] = fmaf(u, f.y, acc[3]);
     f = HalfTraits<T>::unpack2(v.z); acc[4] = fmaf(u, f.x, acc[4]); acc[5] = fmaf(u, f.y, acc[5]);
     f = HalfTraits<T>::unpack2(v.w); acc[6] = fmaf(u, f.x, acc[6]); acc[7] = fmaf(u, f.y, acc[7]);
-    mx = max2_u16(mx, max2_u16(max2_u16(abs2_bits(v.x), abs2_bits(v.y)),
-                               max2_u16(abs2_bits(v.z), abs2_bits(v.w))));
+    mx = absmax2<T>(absmax2<T>(absmax2<T>(absmax2<T>(mx, v.x), v.y), v.z), v.w);
+}
+
+// The same with packed FP32 pairs (add.f32x2 / fma.rn.f32x2 of sm_100): half the FP32
+// instructions per 16-byte vector.  Each lane of a pair is an ordinary round-to-nearest op.
+template <typename T>
+__device__ __forceinline__ void add8p(float2 (&acc)[4], const uint4 &v, unsigned int &mx)
+{
+    acc[0] = __fadd2_rn(acc[0], HalfTraits<T>::unpack2(v.x));
+    acc[1] = __fadd2_rn(acc[1], HalfTraits<T>::unpack2(v.y));
+    acc[2] = __fadd2_rn(acc[2], HalfTraits<T>::unpack2(v.z));
+    acc[3] = __fadd2_rn(acc[3], HalfTraits<T>::unpack2(v.w));
+    mx = absmax2<T>(absmax2<T>(absmax2<T>(absmax2<T>(mx, v.x), v.y), v.z), v.w);
+}
+
+template <typename T>
+__device__ __forceinline__ void fma8p(float2 (&acc)[4], const uint4 &v, float u, unsigned int &mx)
+{
+    const float2 uu = make_float2(u, u);
+    acc[0] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.x), acc[0]);
+    acc[1] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.y), acc[1]);
+    acc[2] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.z), acc[2]);
+    acc[3] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.w), acc[3]);
+    mx = absmax2<T>(absmax2<T>(absmax2<T>(absmax2<T>(mx, v.x), v.y), v.z), v.w);
+}
+
+// Running min and max of packed pairs of 16-bit floats (two HMNMX2 per word, no integer work;
+// NaN operands are ignored).  max|x| follows from both at the end.
+template <typename T> struct MinMax2 {
+    uint32_t mx, mn;
+    __device__ __forceinline__ void init();
+    __device__ __forceinline__ void upd(uint32_t w);
+    __device__ __forceinline__ float absmax() const;   // >= 0; 0 when nothing was seen
+};
+template <> __device__ __forceinline__ void MinMax2<__half>::init() { mx = 0xFC00FC00u; mn = 0x7C007C00u; }
+template <> __device__ __forceinline__ void MinMax2<__nv_bfloat16>::init() { mx = 0xFF80FF80u; mn = 0x7F807F80u; }
+template <> __device__ __forceinline__ void MinMax2<__half>::upd(uint32_t w)
+{
+    __half2 a = *reinterpret_cast<__half2 *>(&mx), b = *reinterpret_cast<__half2 *>(&mn), x = *reinterpret_cast<__half2 *>(&w);
+    a = __hmax2(a, x);
+    b = __hmin2(b, x);
+    mx = *reinterpret_cast<uint32_t *>(&a);
+    mn = *reinterpret_cast<uint32_t *>(&b);
+}
+template <> __device__ __forceinline__ void MinMax2<__nv_bfloat16>::upd(uint32_t w)
+{
+    __nv_bfloat162 a = *reinterpret_cast<__nv_bfloat162 *>(&mx), b = *reinterpret_cast<__nv_bfloat162 *>(&mn),
+                   x = *reinterpret_cast<__nv_bfloat162 *>(&w);
+    a = __hmax2(a, x);
+    b = __hmin2(b, x);
+    mx = *reinterpret_cast<uint32_t *>(&a);
+    mn = *reinterpret_cast<uint32_t *>(&b);
+}
+template <typename T> __device__ __forceinline__ float MinMax2<T>::absmax() const
+{
+    const float a = fmaxf(bits16_to_float<T>(mx & 0xFFFFu), bits16_to_float<T>(mx >> 16));
+    const float b = fminf(bits16_to_float<T>(mn & 0xFFFFu), bits16_to_float<T>(mn >> 16));
+    return fmaxf(fmaxf(a, -b), 0.f);
+}
+// exact 16-bit pattern of a non-negative value that is representable in T
+template <typename T> __device__ __forceinline__ unsigned int float_to_bits16(float x);
+template <> __device__ __forceinline__ unsigned int float_to_bits16<__half>(float x)
+{
+    return (unsigned int)__half_as_ushort(__float2half_rn(x));
+}
+template <> __device__ __forceinline__ unsigned int float_to_bits16<__nv_bfloat16>(float x)
+{
+    return __float_as_uint(x) >> 16;
+}
+
+// acc[e] += x_e for the 8 half-precision values of a 16-byte vector, with the mixed-precision
+// add of sm_100 (add.f32.f16 / add.f32.bf16: FP32 accumulate of a 16-bit operand, one FP
+// instruction per element and no unpacking on the integer pipe).
+template <typename T> __device__ __forceinline__ void madd2(float &a0, float &a1, uint32_t w);
+template <> __device__ __forceinline__ void madd2<__half>(float &a0, float &a1, uint32_t w)
+{
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.f32.f16 %0, lo, %0;\n\tadd.f32.f16 %1, hi, %1;\n\t}"
+        : "+f"(a0), "+f"(a1) : "r"(w));
+}
+template <> __device__ __forceinline__ void madd2<__nv_bfloat16>(float &a0, float &a1, uint32_t w)
+{
+    asm("{\n\t.reg .b16 lo, hi;\n\tmov.b32 {lo, hi}, %2;\n\tadd.f32.bf16 %0, lo, %0;\n\tadd.f32.bf16 %1, hi, %1;\n\t}"
+        : "+f"(a0), "+f"(a1) : "r"(w));
+}
+template <typename T>
+__device__ __forceinline__ void add8m(float2 (&acc)[4], const uint4 &v, MinMax2<T> &mm)
+{
+    madd2<T>(acc[0].x, acc[0].y, v.x);
+    madd2<T>(acc[1].x, acc[1].y, v.y);
+    madd2<T>(acc[2].x, acc[2].y, v.z);
+    madd2<T>(acc[3].x, acc[3].y, v.w);
+    mm.upd(v.x); mm.upd(v.y); mm.upd(v.z); mm.upd(v.w);
+}
+template <typename T>
+__device__ __forceinline__ void fma8m(float2 (&acc)[4], const uint4 &v, float u, MinMax2<T> &mm)
+{
+    const float2 uu = make_float2(u, u);
+    acc[0] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.x), acc[0]);
+    acc[1] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.y), acc[1]);
+    acc[2] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.z), acc[2]);
+    acc[3] = __ffma2_rn(uu, HalfTraits<T>::unpack2(v.w), acc[3]);
+    mm.upd(v.x); mm.upd(v.y); mm.upd(v.z); mm.upd(v.w);
 }
 
 // Sum the per-row-lane accumulators of a CTA in lane order and store the partial vector.
@@ -273,61 +384,131 @@ __device__ __forceinline__ ArgMax amax(ArgMax a, ArgMax b)
     return a;
 }
 
-// Deterministic block sum: per-thread values combined by a fixed tree.
-__device__ __forceinline__ float block_sum(float v, float *sm)
+struct SyncAll {
+    static __device__ __forceinline__ void sync() { __syncthreads(); }
+};
+struct SyncConsumers {   // named barrier over the 512 consumer threads of the TMA kernel
+    static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+};
+
+// Deterministic block reductions over NT threads: xor-shuffle tree inside each warp, then the
+// warp results combined in warp order.  Two barriers each.
+template <int NT, typename Sync>
+__device__ __forceinline__ float block_sum(float v, float *sm, int tid)
 {
-    __syncthreads();
-    sm[threadIdx.x] = v;
-    __syncthreads();
-    for (int s = kProbeThreads / 2; s > 0; s >>= 1) {
-        if ((int)threadIdx.x < s) sm[threadIdx.x] += sm[threadIdx.x + s];
-        __syncthreads();
-    }
-    return sm[0];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    Sync::sync();
+    if ((tid & 31) == 0) sm[tid >> 5] = v;
+    Sync::sync();
+    float r = sm[0];
+    for (int w = 1; w < NT / 32; ++w) r += sm[w];
+    return r;
 }
 
-template <typename T>
-__device__ void verdict(const ProbeArgs &p, int grid, float *red, int status)
+template <int NT, typename Sync>
+__device__ __forceinline__ ArgMax block_argmax(ArgMax v, float *sm, int tid)
 {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ArgMax t;
+        t.v = __shfl_xor_sync(0xFFFFFFFFu, v.v, o);
+        t.i = __shfl_xor_sync(0xFFFFFFFFu, v.i, o);
+        v = amax(v, t);
+    }
+    ArgMax *ams = reinterpret_cast<ArgMax *>(sm);
+    Sync::sync();
+    if ((tid & 31) == 0) ams[tid >> 5] = v;
+    Sync::sync();
+    ArgMax r = ams[0];
+    for (int w = 1; w < NT / 32; ++w) r = amax(r, ams[w]);
+    return r;
+}
+
+// Verdict over the n3 sketch entries by NT threads of one CTA (Section "Thresholds";
+// Algorithm 2 probe part; the explicit finiteness test of Section "Nonfinite").  The entries
+// are fetched with batches of independent loads and kept in registers for the second pass.
+template <typename T, int NT, typename Sync>
+__device__ void verdict(const ProbeArgs &p, int grid, float *red, int status, int tid)
+{
+    constexpr int CACHE = 8192 / NT;
     const int n = (int)p.n3;
+    float cache[CACHE];
+#pragma unroll
+    for (int q = 0; q < CACHE; ++q) {
+        const int j = tid + q * NT;
+        const float x = __ldcg(p.s + (j < n ? j : n - 1));     // clamped: no branch, one batch of loads
+        cache[q] = j < n ? fabsf(x) : 0.f;
+    }
     float sum = 0.f;
     ArgMax am = {-1.f, 0x7FFFFFFF};
     int bad = 0;
-    for (int j = threadIdx.x; j < n; j += kProbeThreads) {
-        float a = fabsf(__ldcg(p.s + j));
-        sum += a;
-        if (!(a <= 3.402823466e38f)) bad = 1;          // Inf or NaN
-        am = amax(am, ArgMax{(a != a) ? -1.f : a, j});
+#pragma unroll
+    for (int q = 0; q < CACHE; ++q) {
+        const int j = tid + q * NT;
+        if (j < n) {
+            const float a = cache[q];
+            sum += a;
+            if (!(a <= 3.402823466e38f)) bad = 1;          // Inf or NaN
+            am = amax(am, ArgMax{(a != a) ? -1.f : a, j});
+        }
     }
-    const float mean_abs = block_sum(sum, red) / (float)n;
+    for (int j0 = tid + CACHE * NT; j0 < n; j0 += 8 * NT) {     // only when n3 > 32 NT
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = fabsf(__ldcg(p.s + min(j0 + q * NT, n - 1)));
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            if (j0 + q * NT < n) {
+                sum += v[q];
+                if (!(v[q] <= 3.402823466e38f)) bad = 1;
+                am = amax(am, ArgMax{(v[q] != v[q]) ? -1.f : v[q], j0 + q * NT});
+            }
+        }
+    }
+    if (tid == 0) trace_mark(p, blockIdx.x, 13);
+    const float mean_abs = block_sum<NT, Sync>(sum, red, tid) / (float)n;
+    if (tid == 0) trace_mark(p, blockIdx.x, 14);
     float csum = 0.f;
     const float clip = 5.f * mean_abs;
-    for (int j = threadIdx.x; j < n; j += kProbeThreads) csum += fminf(fabsf(__ldcg(p.s + j)), clip);
-    const float sigma = 1.2533f * (block_sum(csum, red) / (float)n);
-    // arg max and flags
-    __syncthreads();
-    ArgMax *ams = reinterpret_cast<ArgMax *>(red);
-    ams[threadIdx.x] = am;
-    __syncthreads();
-    for (int s = kProbeThreads / 2; s > 0; s >>= 1) {
-        if ((int)threadIdx.x < s) ams[threadIdx.x] = amax(ams[threadIdx.x], ams[threadIdx.x + s]);
-        __syncthreads();
+#pragma unroll
+    for (int q = 0; q < CACHE; ++q)
+        if (tid + q * NT < n) csum += fminf(cache[q], clip);
+    for (int j0 = tid + CACHE * NT; j0 < n; j0 += 8 * NT) {
+        float v[8];
+#pragma unroll
+        for (int q = 0; q < 8; ++q) v[q] = fabsf(__ldcg(p.s + min(j0 + q * NT, n - 1)));
+#pragma unroll
+        for (int q = 0; q < 8; ++q)
+            if (j0 + q * NT < n) csum += fminf(v[q], clip);
     }
-    am = ams[0];
-    const int anybad = __syncthreads_or(bad);
-    if (threadIdx.x == 0) {
-        unsigned int ma = 0, mb = 0;
-        for (int c = 0; c < grid; ++c) {
-            ma = max(ma, __ldcg(p.maxA + c));
-            mb = max(mb, __ldcg(p.maxB + c));
-        }
+    const float sigma = 1.2533f * (block_sum<NT, Sync>(csum, red, tid) / (float)n);
+    const float anybad = block_sum<NT, Sync>(bad ? 1.f : 0.f, red, tid);
+    am = block_argmax<NT, Sync>(am, red, tid);
+    unsigned int ma = 0, mb = 0;
+    for (int c = tid; c < grid; c += NT) {
+        ma = max(ma, __ldcg(p.maxA + c));
+        mb = max(mb, __ldcg(p.maxB + c));
+    }
+    Sync::sync();     // red is reused below
+    if (tid == 0) trace_mark(p, blockIdx.x, 15);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        ma = max(ma, __shfl_xor_sync(0xFFFFFFFFu, ma, o));
+        mb = max(mb, __shfl_xor_sync(0xFFFFFFFFu, mb, o));
+    }
+    unsigned int *um = reinterpret_cast<unsigned int *>(red);
+    if ((tid & 31) == 0) { um[tid >> 5] = ma; um[NT / 32 + (tid >> 5)] = mb; }
+    Sync::sync();
+    if (tid == 0) {
+        for (int w = 1; w < NT / 32; ++w) { ma = max(ma, um[w]); mb = max(mb, um[NT / 32 + w]); }
         const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) *
                           bits16_to_float<T>(mb);
         const float nb = (float)(n > 2 ? n : 2);
         const float thr = fminf(tau, p.mu * sqrtf(2.f * logf(nb)) * sigma);
         fpsk_probe_result r;
-        r.nonfinite = anybad ? 1 : 0;
-        r.fired = (anybad || am.v > thr) ? 1 : 0;
+        r.nonfinite = anybad > 0.f ? 1 : 0;
+        r.fired = (anybad > 0.f || am.v > thr) ? 1 : 0;
         r.argmax_col = am.i;
         r.status = status;
         r.max_abs = am.v;
@@ -391,7 +572,7 @@ __global__ void __launch_bounds__(kProbeThreads, 2) probe_kernel(const ProbeArgs
     if (s_flag) {   // the last CTA through: everything is published
         __threadfence();
         const int failed = (int)__ldcg(p.ctrl + 3);
-        verdict<T>(p, G, red, failed ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK);
+        verdict<T, kProbeThreads, SyncAll>(p, G, red, failed ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK, (int)threadIdx.x);
         __syncthreads();
         if (threadIdx.x == 0 && !failed) {
             // self-reset for the next launch (after a timeout the host must re-initialise)
@@ -400,10 +581,645 @@ __global__ void __launch_bounds__(kProbeThreads, 2) probe_kernel(const ProbeArgs
     }
 }
 
+// ================================================================ TMA pipeline variant
+// Same arithmetic plan, but all data movement is done by the bulk-copy engine
+// (cp.async.bulk completing on mbarriers) and the threads only do arithmetic.  One producer
+// warp streams tiles into a ring of shared-memory stages; 16 consumer warps reduce stage after
+// stage.  The tile stream of a CTA is
+//     A tiles | C tiles | U tiles | B tiles
+// where the U tiles carry the published partial column sums of A that this CTA's rows of B
+// need: they travel through the same ring, so u is in shared memory when the B tiles arrive
+// and the producer never drains the pipeline.  The final combine fetches the partial vectors
+// of a column slice with bulk copies as well.  One CTA per SM.
+//
+// Everything outside the streaming loops runs once per CTA (cold code, L2 round trips of
+// several hundred cycles), so those parts are short loops with as few dependent global round
+// trips as possible.
+constexpr int kTmaConsumers = 512;
+constexpr int kTmaThreads = kTmaConsumers + 32;   // + producer warp
+constexpr int kStageBytes = 32768;
+constexpr int kStages = 6;
+constexpr int kSegMax = 4096;                 // bytes of one row segment: 256 x 16 B; two row lanes of consumers
+constexpr int kGatherFloats = 5120;           // staging of partial vectors in the final combine; lane-reduce scratch
+constexpr int kUChunkT = 1024;                // u values kept in shared memory
+constexpr int kTmaSmem = kStages * kStageBytes + (kGatherFloats + kUChunkT) * 4 + 256;
+
+struct TDecomp {
+    int cg;       // column groups
+    int rg;       // row groups; cg*rg <= grid
+    int segb;     // bytes per row segment (multiple of 16, <= kSegMax)
+    int tr;       // rows per stage
+    int stride;   // floats per partial row
+    int unit;     // rows are dealt out in units of this many (4 for B: keeps u slices 16-byte aligned)
+    int uq, urem; // (rows/unit) / rg and % rg: group g owns unit*(uq + (g < urem)) rows
+};
+
+struct TmaArgs {
+    ProbeArgs p;
+    TDecomp tA, tB, tC;
+    int sq, srem;        // (n3/4) / grid and % grid: column slice of each CTA in the final combine, in units of 4
+    float thr_scale;     // mu sqrt(2 ln N_b)
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Bounded wait on an mbarrier phase: gives up (returns false) after about a second of polling
+// instead of spinning forever.
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    const long long t_end = clock64() + 2000000000LL;
+    for (;;) {
+#pragma unroll 1
+        for (int it = 0; it < 1024; ++it) {
+            uint32_t ok;
+            asm volatile(
+                "{\n\t.reg .pred p;\n\t"
+                "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                "selp.u32 %0, 1, 0, p;\n\t}"
+                : "=r"(ok)
+                : "r"(bar), "r"(parity)
+                : "memory");
+            if (ok) return true;
+        }
+        if (clock64() > t_end) return false;
+    }
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+// Orders this thread's earlier generic-proxy observations before its later async-proxy
+// (bulk copy) accesses.
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
+
+// Partition of `units` items over groups: the first urem groups own uq+1 items, the others uq.
+// Finds the group of item u, its offset inside the group, the group's first item and its size.
+__device__ __forceinline__ void locate_unit(int u, int uq, int urem, int &g, int &off, int &first, int &cnt)
+{
+    const int big = urem * (uq + 1);
+    if (u < big) {
+        g = u / (uq + 1);
+        off = u - g * (uq + 1);
+        first = g * (uq + 1);
+        cnt = uq + 1;
+    } else {
+        const int v = u - big;
+        const int gg = v / uq;            // uq > 0 here: with uq == 0 every item lies in the first urem groups
+        g = urem + gg;
+        off = v - gg * uq;
+        first = big + gg * uq;
+        cnt = uq;
+    }
+}
+
+struct Piece {          // what one CTA streams of one matrix
+    const char *base;   // first byte of the piece's first row segment
+    long long ldb;      // leading dimension in bytes
+    int r0, r1;         // rows [r0, r1)
+    int wbytes;         // bytes of this piece's row segment (<= segb; the last group may be narrower)
+    int segb, tr;
+    int cg, rg;         // this CTA's column group and row group
+    bool has;
+};
+
+__device__ __forceinline__ Piece make_piece(const void *X, long long ld_elems, long long rowbytes, int elt,
+                                            const TDecomp &d, int c)
+{
+    Piece pc;
+    pc.rg = c / d.cg;
+    pc.cg = c - pc.rg * d.cg;
+    pc.has = pc.rg < d.rg;
+    pc.ldb = ld_elems * elt;
+    pc.segb = d.segb;
+    pc.tr = d.tr;
+    const long long cb0 = (long long)pc.cg * d.segb;
+    long long w = rowbytes - cb0;
+    if (w > d.segb) w = d.segb;
+    if (w <= 0) { w = 0; pc.has = false; }
+    pc.wbytes = (int)w;
+    pc.r0 = pc.has ? d.unit * (pc.rg * d.uq + min(pc.rg, d.urem)) : 0;
+    pc.r1 = pc.has ? pc.r0 + d.unit * (d.uq + (pc.rg < d.urem ? 1 : 0)) : 0;
+    pc.base = static_cast<const char *>(X) + cb0;
+    return pc;
+}
+
+// Verdict by the 512 consumers of the last CTA (Section "Thresholds"; Algorithm 2 probe part;
+// the finiteness test of Section "Nonfinite").  s is brought into shared memory by one bulk
+// copy per chunk, then reduced by short loops; the block reductions are fixed trees.
+struct VStat {
+    float sum;
+    float bad;
+    ArgMax am;
+};
+
+template <typename T>
+__device__ __noinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr_scale, float *sbuf, int sbuf_cap, float *red,
+                                         uint32_t gbar, uint32_t gpar, int status, int ctid)
+{
+    const int n = (int)p.n3;
+    // thread 0 fetches the two operand maxima early; they are only needed at the very end
+    unsigned int ma = 0, mb = 0;
+    if (ctid == 0) { ma = __ldcg(p.ctrl + 4); mb = __ldcg(p.ctrl + 5); }
+    // per-CTA slice statistics -> sum|s|, non-finite flag, max|s| and its column (fixed tree)
+    float sum = 0.f, bad = 0.f;
+    ArgMax am = {-1.f, 0x7FFFFFFF};
+    for (int g = ctid; g < grid; g += kTmaConsumers) {
+        const float4 st = __ldcg(p.vstat + g);
+        sum += st.x;
+        bad += st.y;
+        am = amax(am, ArgMax{st.z, __float_as_int(st.w)});
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        bad += __shfl_xor_sync(0xFFFFFFFFu, bad, o);
+        ArgMax t;
+        t.v = __shfl_xor_sync(0xFFFFFFFFu, am.v, o);
+        t.i = __shfl_xor_sync(0xFFFFFFFFu, am.i, o);
+        am = amax(am, t);
+    }
+    VStat *vs = reinterpret_cast<VStat *>(red);
+    SyncConsumers::sync();
+    if ((ctid & 31) == 0) vs[ctid >> 5] = VStat{sum, bad, am};
+    SyncConsumers::sync();
+    {
+        VStat r = vs[0];
+        for (int w = 1; w < kTmaConsumers / 32; ++w) {
+            r.sum += vs[w].sum;
+            r.bad += vs[w].bad;
+            r.am = amax(r.am, vs[w].am);
+        }
+        sum = r.sum; bad = r.bad; am = r.am;
+    }
+    const float clip = 5.f * (sum / (float)n);
+    float csum_total = sum;                 // nothing is clipped when max|s| <= 5 mean|s|
+    if (bad > 0.f || !(am.v <= clip)) {
+        // some entry exceeds the clip level (or is not finite): second pass over all of s
+        const bool al16 = (reinterpret_cast<uintptr_t>(p.s) & 15) == 0;
+        float csum = 0.f;
+        for (int base = 0; base < n; base += sbuf_cap) {
+            const int cntv = min(sbuf_cap, n - base);
+            SyncConsumers::sync();
+            if (al16 && (cntv & 3) == 0) {
+                if (ctid == 0) {
+                    fence_proxy_async();
+                    mbar_expect_tx(gbar, (uint32_t)cntv * 4u);
+                    bulk_g2s(smem_u32(sbuf), p.s + base, (uint32_t)cntv * 4u, gbar);
+                }
+                mbar_wait_bounded(gbar, gpar);
+                gpar ^= 1u;
+            } else {
+                for (int e = ctid; e < cntv; e += kTmaConsumers) sbuf[e] = __ldcg(p.s + base + e);
+                SyncConsumers::sync();
+            }
+            for (int j = ctid; j < cntv; j += kTmaConsumers) csum += fminf(fabsf(sbuf[j]), clip);
+        }
+        csum_total = block_sum<kTmaConsumers, SyncConsumers>(csum, red + 256, ctid);
+    }
+    if (ctid == 0) {
+        const float sigma = 1.2533f * (csum_total / (float)n);
+        const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) * bits16_to_float<T>(mb);
+        const float thr = fminf(tau, thr_scale * sigma);
+        fpsk_probe_result r;
+        r.nonfinite = bad > 0.f ? 1 : 0;
+        r.fired = (bad > 0.f || am.v > thr) ? 1 : 0;
+        r.argmax_col = am.i;
+        r.status = status;
+        r.max_abs = am.v;
+        r.sigma_hat = sigma;
+        r.thr = thr;
+        r.tau = tau;
+        *p.result = r;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *ring = smem;
+    float *red = reinterpret_cast<float *>(smem + kStages * kStageBytes);          // kGatherFloats
+    float *us = red + kGatherFloats;                                               // kUChunkT floats
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(us + kUChunkT);
+    __shared__ int s_flag;
+    __shared__ int s_err;
+    const ProbeArgs &p = a.p;
+    const int c = blockIdx.x, G = gridDim.x;
+    const int tid = threadIdx.x;
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages), gbar = smem_u32(bars + 2 * kStages);
+    if (tid == 0) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, kTmaConsumers / 32);
+        }
+        mbar_init(gbar, 1);
+        s_err = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    // With programmatic dependent launch this kernel may start while its predecessor in the
+    // stream is still draining; nothing produced by earlier work is touched before this point.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    __syncthreads();
+
+    Piece pc[3];
+    pc[0] = make_piece(p.A, p.lda, p.n2 * 2, 2, a.tA, c);
+    pc[1] = make_piece(p.C, p.ldc, p.n3 * 4, 4, a.tC, c);
+    pc[2] = make_piece(p.B, p.ldb, p.n3 * 2, 2, a.tB, c);
+    // U tiles: the rgA partial rows of column sums of A, restricted to this CTA's rows of B
+    const int ucnt = pc[2].has ? pc[2].r1 - pc[2].r0 : 0;                 // multiple of 4
+    const bool use_ut = ucnt > 0 && ucnt <= kUChunkT;
+    const int ut_rows = use_ut ? kStageBytes / (ucnt * 4) : 1;            // partial rows per U tile
+    const int ngA = a.tA.rg;
+
+    if (tid >= kTmaConsumers) {
+        // ------------------------------------------------------------ producer warp
+        const int lane = tid - kTmaConsumers;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const Piece &q = pc[m];
+            if (m == 2 && use_ut && ok) {
+                // the partial sums must be published by every CTA before they are fetched
+                int w = 1;
+                if (lane == 0) w = bounded_wait_ge(p.ctrl + 0, (unsigned)G) ? 1 : 0;
+                w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                if (!w) ok = false;
+                fence_proxy_async();
+                for (int t0 = 0; t0 < ngA && ok; t0 += ut_rows) {
+                    const int nt = min(ut_rows, ngA - t0);
+                    w = 1;
+                    if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                    w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                    if (!w) { ok = false; break; }
+                    if (lane == 0) {
+                        // this row group's block of partA is [ngA][ucnt]: rows t0..t0+nt are contiguous
+                        const uint32_t bytes = (uint32_t)nt * (uint32_t)ucnt * 4u;
+                        mbar_expect_tx(full0 + 8 * stage, bytes);
+                        bulk_g2s(smem_u32(ring + (size_t)stage * kStageBytes),
+                                 p.partA + (long long)pc[2].r0 * ngA + (long long)t0 * ucnt, bytes, full0 + 8 * stage);
+                    }
+                    __syncwarp();
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) continue;
+            if (!q.has) continue;
+            for (int row = q.r0; row < q.r1 && ok; row += q.tr) {
+                const int nr = min(q.tr, q.r1 - row);
+                int w = 1;
+                if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                if (!w) { ok = false; break; }
+                if (lane == 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)nr * (uint32_t)q.wbytes);
+                __syncwarp();
+                const uint32_t dst0 = smem_u32(ring + (size_t)stage * kStageBytes);
+                for (int r = lane; r < nr; r += 32)
+                    bulk_g2s(dst0 + (uint32_t)r * (uint32_t)q.segb, q.base + (long long)(row + r) * q.ldb, (uint32_t)q.wbytes,
+                             full0 + 8 * stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok && lane == 0) {
+            s_err = 1;
+            atomicOr(p.ctrl + 3, 1u);
+        }
+    } else {
+        // ------------------------------------------------------------ consumer warps
+        const int ctid = tid;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        if (ctid == 0) trace_mark(p, c, 0);
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const Piece &q = pc[m];
+            const int tpr = q.segb / 16;
+            const int RL = kTmaConsumers / tpr;
+            const int rl = ctid / tpr, tc = ctid - rl * tpr;
+            const bool active = q.has && rl < RL && tc * 16 < q.wbytes;
+            float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+            MinMax2<T> mm;
+            mm.init();
+            int us_base = 0, us_cnt = 0;
+            if (m == 2 && q.has) {
+                if (use_ut) {
+                    // U tiles: u_k = sum over the published partial rows.  Thread (sub, k) adds the
+                    // rows t = sub, sub + NSUB, ... of column k over all tiles; the NSUB sub-sums are
+                    // then combined in sub order (fixed order, deterministic).
+                    int uw = 64;
+                    while (uw < ucnt) uw <<= 1;                     // columns per pass (<= 1024)
+                    const int nsub = uw <= kTmaConsumers ? kTmaConsumers / uw : 1;
+                    const int sub = uw <= kTmaConsumers ? ctid / uw : 0;
+                    const int kk = uw <= kTmaConsumers ? ctid - sub * uw : ctid;
+                    float u0 = 0.f, u1 = 0.f;
+                    for (int t0 = 0; t0 < ngA; t0 += ut_rows) {
+                        const int nt = min(ut_rows, ngA - t0);
+                        if (ok) {
+                            int w = 1;
+                            if ((ctid & 31) == 0) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
+                            w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                            if (w) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
+                            if (!w) { ok = false; s_err = 1; }
+                        }
+                        if (ok) {
+                            const float *tb = reinterpret_cast<const float *>(ring + (size_t)stage * kStageBytes);
+                            // global partial-row index t0 + t must be congruent to sub: keeps the order fixed
+                            int t = (sub - t0 % nsub + nsub) % nsub;
+                            if (kk < ucnt) {
+#pragma unroll 4
+                                for (; t < nt; t += nsub) u0 += tb[t * ucnt + kk];
+                            }
+                            if (uw > kTmaConsumers && kk + kTmaConsumers < ucnt) {
+#pragma unroll 4
+                                for (int t2 = 0; t2 < nt; ++t2) u1 += tb[t2 * ucnt + kk + kTmaConsumers];
+                            }
+                        }
+                        __syncwarp();
+                        if ((ctid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
+                        if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                    }
+                    if (nsub > 1) {
+                        SyncConsumers::sync();
+                        red[sub * uw + kk] = u0;
+                        SyncConsumers::sync();
+                        if (sub == 0 && kk < ucnt) {
+                            float u = red[kk];
+                            for (int s2 = 1; s2 < nsub; ++s2) u += red[s2 * uw + kk];
+                            us[kk] = u;
+                        }
+                    } else {
+                        if (kk < ucnt) us[kk] = u0;
+                        if (kk + kTmaConsumers < ucnt) us[kk + kTmaConsumers] = u1;
+                    }
+                    us_base = q.r0;
+                    us_cnt = ucnt;
+                    SyncConsumers::sync();
+                } else {
+                    // large slices: wait (bounded) until every CTA has published its column sums of A
+                    if (ctid == 0) s_flag = bounded_wait_ge(p.ctrl + 0, (unsigned)G) ? 1 : 0;
+                    SyncConsumers::sync();
+                    if (!s_flag) ok = false;
+                    SyncConsumers::sync();
+                }
+                if (ctid == 0) trace_mark(p, c, 4);
+            }
+            if (q.has) {
+                for (int row = q.r0; row < q.r1; row += q.tr) {
+                    const int nr = min(q.tr, q.r1 - row);
+                    if (m == 2 && !use_ut && row + nr > us_base + us_cnt) {
+                        // fallback for very tall slices of B: u from plain loads, in partial-row order
+                        us_base = row;
+                        us_cnt = min(kUChunkT, q.r1 - row);
+                        SyncConsumers::sync();
+                        for (int k = ctid; k < us_cnt; k += kTmaConsumers) {
+                            float u = 0.f;
+                            for (int t = 0; t < ngA; ++t)
+                                u += __ldcg(p.partA + (long long)q.r0 * ngA + (long long)t * (q.r1 - q.r0) + (us_base - q.r0) + k);
+                            us[k] = u;
+                        }
+                        SyncConsumers::sync();
+                    }
+                    if (ok) {
+                        // lane 0 polls (bounded); the verdict is warp-uniform; every lane then
+                        // observes the completed phase itself before reading the stage
+                        int w = 1;
+                        if ((ctid & 31) == 0) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
+                        w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                        if (w) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
+                        if (!w) { ok = false; s_err = 1; }
+                    }
+                    if (ok && active) {
+                        const unsigned char *sb = ring + (size_t)stage * kStageBytes + tc * 16;
+                        if (m == 1) {
+#pragma unroll 4
+                            for (int r = rl; r < nr; r += RL) {
+                                const float4 v = *reinterpret_cast<const float4 *>(sb + (size_t)r * q.segb);
+                                acc[0] = __fadd2_rn(acc[0], make_float2(v.x, v.y));
+                                acc[1] = __fadd2_rn(acc[1], make_float2(v.z, v.w));
+                            }
+                        } else if (m == 0) {
+#pragma unroll 4
+                            for (int r = rl; r < nr; r += RL) {
+                                const uint4 v = *reinterpret_cast<const uint4 *>(sb + (size_t)r * q.segb);
+                                add8m<T>(acc, v, mm);
+                            }
+                        } else {
+                            const float *uu = us + (row - us_base);
+#pragma unroll 4
+                            for (int r = rl; r < nr; r += RL) {
+                                const uint4 v = *reinterpret_cast<const uint4 *>(sb + (size_t)r * q.segb);
+                                fma8m<T>(acc, v, uu[r], mm);
+                            }
+                        }
+                    }
+                    __syncwarp();
+                    if ((ctid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (ctid == 0) trace_mark(p, c, m == 0 ? 1 : (m == 1 ? 3 : 6));
+            // ---- epilogue of the piece: combine row lanes (fixed order) and publish the partial
+            // Layouts are blocked by their reader, so that every later gather is one contiguous copy:
+            //   partA : for each row group g of B, a block [t < ngA][rows of g] of partial column sums of A
+            //   partP : for each column slice c' of the final combine, a block [t < ngP + ngC][columns of c']
+            //           holding the partial p rows (t < ngP) and the partial column sums of C (t >= ngP)
+            const TDecomp &d = m == 0 ? a.tA : (m == 1 ? a.tC : a.tB);
+            const int nv = m == 1 ? 4 : 8;
+            if (q.has) {
+                float4 lo = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+                float4 hi = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
+                float4 *r4 = reinterpret_cast<float4 *>(red);
+                SyncConsumers::sync();
+                if (active && rl > 0) {
+                    r4[((rl - 1) * tpr + tc) * 2] = lo;
+                    r4[((rl - 1) * tpr + tc) * 2 + 1] = hi;
+                }
+                SyncConsumers::sync();
+                if (active && rl == 0) {
+                    for (int l = 1; l < RL; ++l) {
+                        const float4 x = r4[((l - 1) * tpr + tc) * 2], y = r4[((l - 1) * tpr + tc) * 2 + 1];
+                        lo.x += x.x; lo.y += x.y; lo.z += x.z; lo.w += x.w;
+                        hi.x += y.x; hi.y += y.y; hi.z += y.z; hi.w += y.w;
+                    }
+                    const int col0 = q.cg * (d.segb / (m == 1 ? 4 : 2)) + tc * nv;     // first column of this thread
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        if (h == 1 && nv == 4) break;
+                        const int u = (col0 >> 2) + h;                                  // unit of 4 columns
+                        int g, off, first, cnt;
+                        float *dst;
+                        if (m == 0) {
+                            locate_unit(u, a.tB.uq, a.tB.urem, g, off, first, cnt);
+                            dst = p.partA + (long long)first * 4 * ngA + (long long)q.rg * (cnt * 4) + off * 4;
+                        } else {
+                            locate_unit(u, a.sq, a.srem, g, off, first, cnt);
+                            const int t = m == 2 ? q.rg : a.tB.rg + q.rg;
+                            dst = p.partP + (long long)first * 4 * (a.tB.rg + a.tC.rg) + (long long)t * (cnt * 4) + off * 4;
+                        }
+                        __stcg(reinterpret_cast<float4 *>(dst), h == 0 ? lo : hi);
+                    }
+                }
+            }
+            if (m != 1) {
+                // max |.| of the half-precision operand (for tau): integer atomic, order-independent
+                unsigned int mbits = float_to_bits16<T>(mm.absmax());
+                mbits = __reduce_max_sync(0xFFFFFFFFu, mbits);
+                if ((ctid & 31) == 0 && mbits) atomicMax(p.ctrl + (m == 0 ? 4 : 5), mbits);
+            }
+            if (m == 0) {
+                SyncConsumers::sync();
+                if (ctid == 0) {
+                    __threadfence();
+                    atomicAdd(p.ctrl + 0, 1u);
+                    trace_mark(p, c, 2);
+                }
+            }
+            if (m == 2 && ctid == 0) trace_mark(p, c, 7);
+        }
+        // ---- all partials of this CTA are written: grid-wide publication, then the slices
+        SyncConsumers::sync();
+        if (ctid == 0) {
+            __threadfence();
+            if (!ok) atomicOr(p.ctrl + 3, 1u);
+            atomicAdd(p.ctrl + 1, 1u);
+            s_flag = (ok && bounded_wait_ge(p.ctrl + 1, (unsigned)G)) ? 1 : 0;
+        }
+        SyncConsumers::sync();
+        const bool ok2 = s_flag != 0;
+        if (ctid == 0) trace_mark(p, c, 8);
+        uint32_t gpar = 0;
+        float lsum = 0.f, lbad = 0.f;
+        ArgMax lam = {-1.f, 0x7FFFFFFF};
+        if (ok2) {
+            // this CTA's slice of columns: s_j = (sum of partial p) - (sum of partial column sums of C);
+            // the partial rows of the slice arrive by bulk copies, all in flight together
+            const int j0 = 4 * (c * a.sq + min(c, a.srem)), jn = 4 * (a.sq + (c < a.srem ? 1 : 0));
+            const int ngP = a.tB.rg, ngC = a.tC.rg, ntot = ngP + ngC;
+            const float *blk = p.partP + (long long)j0 * ntot;          // [ntot][jn], contiguous
+            const int tmax = jn > 0 ? kGatherFloats / jn : ntot;        // partial rows per pass (>= 1: jn <= kGatherFloats)
+            float sp0 = 0.f, sc0 = 0.f, sp1 = 0.f, sc1 = 0.f;           // columns ctid and ctid + 512
+            for (int t0 = 0; t0 < ntot && jn > 0; t0 += tmax) {
+                const int nt = min(tmax, ntot - t0);
+                if (ctid == 0) {
+                    fence_proxy_async();
+                    const uint32_t bytes = (uint32_t)nt * (uint32_t)jn * 4u;
+                    mbar_expect_tx(gbar, bytes);
+                    bulk_g2s(smem_u32(red), blk + (long long)t0 * jn, bytes, gbar);
+                }
+                const bool got = mbar_wait_bounded(gbar, gpar);
+                gpar ^= 1u;
+                if (!got) s_err = 1;
+                if (ctid < jn) {
+#pragma unroll 4
+                    for (int t = 0; t < nt; ++t) {
+                        const float v = red[t * jn + ctid];
+                        if (t0 + t < ngP) sp0 += v; else sc0 += v;
+                    }
+                }
+                if (ctid + kTmaConsumers < jn) {
+#pragma unroll 4
+                    for (int t = 0; t < nt; ++t) {
+                        const float v = red[t * jn + ctid + kTmaConsumers];
+                        if (t0 + t < ngP) sp1 += v; else sc1 += v;
+                    }
+                }
+                SyncConsumers::sync();
+            }
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int k = ctid + h * kTmaConsumers;
+                if (k < jn) {
+                    const float sv = h == 0 ? sp0 - sc0 : sp1 - sc1;
+                    __stcg(p.s + j0 + k, sv);
+                    const float av = fabsf(sv);
+                    lsum += av;
+                    if (!(av <= 3.402823466e38f)) lbad = 1.f;
+                    lam = amax(lam, ArgMax{(av != av) ? -1.f : av, j0 + k});
+                }
+            }
+        }
+        // statistics of this CTA's slice (fixed tree: warp shuffles, then warp order)
+        {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+                lbad += __shfl_xor_sync(0xFFFFFFFFu, lbad, o);
+                ArgMax t;
+                t.v = __shfl_xor_sync(0xFFFFFFFFu, lam.v, o);
+                t.i = __shfl_xor_sync(0xFFFFFFFFu, lam.i, o);
+                lam = amax(lam, t);
+            }
+            VStat *vs = reinterpret_cast<VStat *>(red);
+            if ((ctid & 31) == 0) vs[ctid >> 5] = VStat{lsum, lbad, lam};
+            SyncConsumers::sync();
+            if (ctid == 0) {
+                VStat r = vs[0];
+                for (int w = 1; w < kTmaConsumers / 32; ++w) {
+                    r.sum += vs[w].sum;
+                    r.bad += vs[w].bad;
+                    r.am = amax(r.am, vs[w].am);
+                }
+                __stcg(p.vstat + c, make_float4(r.sum, r.bad, r.am.v, __int_as_float(r.am.i)));
+            }
+        }
+        SyncConsumers::sync();
+        if (ctid == 0) {
+            trace_mark(p, c, 9);
+            __threadfence();
+            if (!ok2 || s_err) atomicOr(p.ctrl + 3, 1u);
+            const unsigned int t = atomicAdd(p.ctrl + 2, 1u);
+            s_flag = (t == (unsigned)G - 1) ? 1 : 0;
+            if (s_flag) {
+                __threadfence();
+                s_flag = 1 + (int)__ldcg(p.ctrl + 3);      // 1: all good, 2: some CTA gave up
+            }
+            trace_mark(p, c, 10);
+        }
+        SyncConsumers::sync();
+        if (s_flag) {     // the last CTA through: every slice of s is published
+            const int failed = s_flag - 1;
+            // the ring is idle by now (every stage was consumed): reuse it to stage s
+            verdict_tma<T>(p, G, a.thr_scale, reinterpret_cast<float *>(ring), kStages * kStageBytes / 4, red, gbar, gpar,
+                           failed ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK, ctid);
+            if (ctid == 0) {
+                trace_mark(p, c, 11);
+                if (!failed) { p.ctrl[0] = 0; p.ctrl[1] = 0; p.ctrl[2] = 0; p.ctrl[4] = 0; p.ctrl[5] = 0; }
+            }
+        }
+    }
+    // Error path only: before the CTA leaves, wait (bounded) for bulk copies that may still be
+    // landing in its shared memory.
+    __syncthreads();
+    if (s_err && tid == kTmaConsumers) {
+        for (int s = 0; s < kStages; ++s) {
+            mbar_wait_bounded(full0 + 8 * s, 0);
+            mbar_wait_bounded(full0 + 8 * s, 1);
+        }
+        mbar_wait_bounded(gbar, 0);
+        mbar_wait_bounded(gbar, 1);
+    }
+}
+
 // ---------------------------------------------------------------- host side
 struct DevInfo {
     int sms = 0;
     int grid = 0;
+    int tma_grid = 0;
 };
 static DevInfo g_dev[64];
 static std::mutex g_dev_mu;
@@ -435,7 +1251,7 @@ static fpsk_status probe_grid(int &grid)
 }
 
 // Upper bound used for workspace sizing when no device is present / before the first launch.
-constexpr int kMaxGrid = 1024;
+constexpr int kMaxGrid = 512;
 
 static bool make_decomp(long long cols, int vec, int grid, Decomp &d)
 {
@@ -449,15 +1265,41 @@ static bool make_decomp(long long cols, int vec, int grid, Decomp &d)
     return true;
 }
 
+static bool make_tdecomp(long long rows, int unit, long long rowbytes, int elt, int grid, TDecomp &d)
+{
+    long long cg = (rowbytes + kSegMax - 1) / kSegMax;
+    if (cg > grid || rowbytes % 16 != 0 || rows % unit != 0) return false;
+    long long seg = (rowbytes + cg - 1) / cg;
+    seg = (seg + 15) / 16 * 16;
+    d.cg = (int)cg;
+    d.segb = (int)seg;
+    d.rg = grid / d.cg;
+    d.tr = kStageBytes / d.segb;
+    d.stride = (int)(cg * seg / elt);
+    d.unit = unit;
+    d.uq = (int)((rows / unit) / d.rg);
+    d.urem = (int)((rows / unit) % d.rg);
+    return true;
+}
+
 static size_t part_floats(long long cols, int vec)
 {
-    // rows of partials <= kMaxGrid/cg; stride <= cols + cg*vec  ->  bounded by kMaxGrid*kMaxTpr*vec + slack
+    // plain kernel: rows of partials <= kMaxGrid/cg, stride = cg*gwv*vec
     long long wv = (cols + vec - 1) / vec;
     long long cg = (wv + kMaxTpr - 1) / kMaxTpr;
     long long gwv = (wv + cg - 1) / cg;
     long long rg = kMaxGrid / cg;
     if (rg < 1) rg = 1;
-    return (size_t)(rg * cg * gwv * vec);
+    size_t plain = (size_t)(rg * cg * gwv * vec);
+    // TMA kernel: rows <= kMaxGrid/cg, stride = cg*segb/elt
+    const int elt = vec == 8 ? 2 : 4;
+    long long rowbytes = cols * elt;
+    long long tcg = (rowbytes + kSegMax - 1) / kSegMax;
+    long long seg = ((rowbytes + tcg - 1) / tcg + 15) / 16 * 16;
+    long long trg = kMaxGrid / tcg;
+    if (trg < 1) trg = 1;
+    size_t tma = (size_t)(trg * tcg * seg / elt);
+    return plain > tma ? plain : tma;
 }
 
 size_t probe_ws_bytes(int64_t n1, int64_t n2, int64_t n3)
@@ -469,24 +1311,41 @@ size_t probe_ws_bytes(int64_t n1, int64_t n2, int64_t n3)
     b += align_up(part_floats(n3, 4) * 4, 256);          // partC
     b += align_up((size_t)kMaxGrid * 4, 256) * 2;        // maxA, maxB
     b += align_up((size_t)n3 * 4, 256);                  // s
+    b += (size_t)kMaxGrid * 32 * 8;                      // optional phase trace
+    b += (size_t)kMaxGrid * 16;                          // per-CTA slice statistics
     return b;
+}
+
+static fpsk_status tma_grid(int &grid)
+{
+    int dev = 0;
+    FPSK_CUDA_OK(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return FPSK_ERR_CUDA;
+    std::lock_guard<std::mutex> lk(g_dev_mu);
+    if (g_dev[dev].tma_grid == 0) {
+        int sms = 0, occ = 0, o2 = 0;
+        FPSK_CUDA_OK(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        FPSK_CUDA_OK(cudaFuncSetAttribute(probe_tma_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTmaSmem));
+        FPSK_CUDA_OK(cudaFuncSetAttribute(probe_tma_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kTmaSmem));
+        FPSK_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, probe_tma_kernel<__half>, kTmaThreads, kTmaSmem));
+        FPSK_CUDA_OK(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&o2, probe_tma_kernel<__nv_bfloat16>, kTmaThreads, kTmaSmem));
+        occ = occ < o2 ? occ : o2;
+        if (occ < 1 || sms < 1) return FPSK_ERR_CUDA;
+        g_dev[dev].tma_grid = sms;        // one CTA per SM
+    }
+    grid = g_dev[dev].tma_grid;
+    return FPSK_OK;
 }
 
 fpsk_status probe_launch(const void *A, const void *B, const float *C, const ProbeDims &d,
                          fpsk_dtype dtype, double mu, void *ws, size_t ws_bytes, cudaStream_t st,
                          fpsk_probe_result *d_result, float *d_residual)
 {
-    int grid = 0;
-    fpsk_status rc = probe_grid(grid);
-    if (rc != FPSK_OK) return rc;
-    if (grid > kMaxGrid) grid = kMaxGrid;
-    ProbeArgs p;
+    if (ws_bytes < probe_ws_bytes(d.n1, d.n2, d.n3)) return FPSK_ERR_WORKSPACE;
+    TmaArgs ta;
+    ProbeArgs &p = ta.p;
     p.A = A; p.B = B; p.C = C;
     p.n1 = d.n1; p.n2 = d.n2; p.n3 = d.n3; p.lda = d.lda; p.ldb = d.ldb; p.ldc = d.ldc;
-    if (!make_decomp(d.n2, 8, grid, p.dA) || !make_decomp(d.n3, 8, grid, p.dB) ||
-        !make_decomp(d.n3, 4, grid, p.dC))
-        return FPSK_ERR_SHAPE;
-    if (ws_bytes < probe_ws_bytes(d.n1, d.n2, d.n3)) return FPSK_ERR_WORKSPACE;
     char *w = static_cast<char *>(ws);
     p.ctrl = reinterpret_cast<unsigned int *>(w); w += 256;
     p.partA = reinterpret_cast<float *>(w); w += align_up(part_floats(d.n2, 8) * 4, 256);
@@ -495,6 +1354,12 @@ fpsk_status probe_launch(const void *A, const void *B, const float *C, const Pro
     p.maxA = reinterpret_cast<unsigned int *>(w); w += align_up((size_t)kMaxGrid * 4, 256);
     p.maxB = reinterpret_cast<unsigned int *>(w); w += align_up((size_t)kMaxGrid * 4, 256);
     p.s = d_residual ? d_residual : reinterpret_cast<float *>(w);
+    w += align_up((size_t)d.n3 * 4, 256);
+    // FPSK_PROBE_TRACE=1 records per-CTA phase timestamps in the workspace tail (a measurement aid)
+    static const bool want_trace = [] { const char *e = getenv("FPSK_PROBE_TRACE"); return e && e[0] == '1'; }();
+    p.trace = want_trace ? reinterpret_cast<long long *>(w) : nullptr;
+    w += (size_t)kMaxGrid * 32 * 8;
+    p.vstat = reinterpret_cast<float4 *>(w);
     p.result = d_result;
     p.mu = (float)mu;
 
@@ -502,6 +1367,50 @@ fpsk_status probe_launch(const void *A, const void *B, const float *C, const Pro
                        reinterpret_cast<uintptr_t>(C)) & 15) == 0 &&
                      d.lda % 8 == 0 && d.ldb % 8 == 0 && d.ldc % 4 == 0 && d.n2 % 8 == 0 &&
                      d.n3 % 8 == 0;
+    // FPSK_PROBE_PLAIN=1 forces the plain-load kernel (a measurement aid)
+    static const bool force_plain = [] { const char *e = getenv("FPSK_PROBE_PLAIN"); return e && e[0] == '1'; }();
+    if (vec && !force_plain) {
+        int grid = 0;
+        fpsk_status rc = tma_grid(grid);
+        if (rc != FPSK_OK) return rc;
+        if (grid > kMaxGrid) grid = kMaxGrid;
+        if (make_tdecomp(d.n1, 1, d.n2 * 2, 2, grid, ta.tA) && make_tdecomp(d.n2, 4, d.n3 * 2, 2, grid, ta.tB) &&
+            make_tdecomp(d.n1, 1, d.n3 * 4, 4, grid, ta.tC) && ((d.n3 / 4) / grid + 1) * 4 <= 2 * kTmaConsumers) {
+            ta.sq = (int)((d.n3 / 4) / grid);
+            ta.srem = (int)((d.n3 / 4) % grid);
+            ta.thr_scale = (float)(mu * sqrt(2.0 * log((double)(d.n3 > 2 ? d.n3 : 2))));
+            void *args[] = {&ta};
+            const void *fn = dtype == FPSK_FP16 ? (const void *)probe_tma_kernel<__half>
+                                                : (const void *)probe_tma_kernel<__nv_bfloat16>;
+            // FPSK_PROBE_PDL=1: programmatic dependent launch instead of a cooperative launch (measurement aid)
+            static const bool pdl = [] { const char *e = getenv("FPSK_PROBE_PDL"); return e && e[0] == '1'; }();
+            if (pdl) {
+                cudaLaunchConfig_t cfg;
+                memset(&cfg, 0, sizeof(cfg));
+                cfg.gridDim = dim3(grid);
+                cfg.blockDim = dim3(kTmaThreads);
+                cfg.dynamicSmemBytes = kTmaSmem;
+                cfg.stream = st;
+                cudaLaunchAttribute at[1];
+                at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+                at[0].val.programmaticStreamSerializationAllowed = 1;
+                cfg.attrs = at;
+                cfg.numAttrs = 1;
+                FPSK_CUDA_OK(cudaLaunchKernelExC(&cfg, fn, args));
+            } else {
+                FPSK_CUDA_OK(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kTmaThreads), args, kTmaSmem, st));
+            }
+            FPSK_LAUNCH_CHECK();
+            return FPSK_OK;
+        }
+    }
+    int grid = 0;
+    fpsk_status rc = probe_grid(grid);
+    if (rc != FPSK_OK) return rc;
+    if (grid > kMaxGrid) grid = kMaxGrid;
+    if (!make_decomp(d.n2, 8, grid, p.dA) || !make_decomp(d.n3, 8, grid, p.dB) ||
+        !make_decomp(d.n3, 4, grid, p.dC))
+        return FPSK_ERR_SHAPE;
     void *args[] = {&p};
     const void *fn;
     if (dtype == FPSK_FP16)
