@@ -157,6 +157,31 @@ fpsk_status fpsk_probe_host(const void *hA, const void *hB, const float *hC,
                             const fpsk_params *p, void *workspace, size_t ws_bytes,
                             void *stream, fpsk_probe_result *h_result);
 
+/* The probe without caller-provided scratch.  (No counterpart in the paper: this is a
+ * deployment convenience of this library.)
+ *
+ * For callers that cannot allocate device memory where they verify a GEMM - inside a
+ * stream-capture region, on a latency-critical or fault-handling path that must not enter the
+ * allocator, or in a plug-in that is handed tensors but owns no memory pool - the scratch
+ * that fpsk_probe takes as `workspace` lives in a fixed array of
+ * FPSK_PROBE_STATIC_SCRATCH_BYTES inside the library (held by every GPU that loads the
+ * library, until the process exits).  Arguments and results are those of fpsk_probe, minus
+ * the workspace; A, B, C and the outputs are still the caller's device buffers.
+ *   - Calls no cudaMalloc / cudaFree and no allocating library routine.
+ *   - The first call on each device looks up the array's device address (with that device
+ *     current); make that first call outside any stream capture.
+ *   - Shapes whose scratch would not fit (fpsk_probe_workspace_bytes(m,k,n) >
+ *     FPSK_PROBE_STATIC_SCRATCH_BYTES) are refused with FPSK_ERR_WORKSPACE; nothing is launched.
+ *     12 MiB covers every shape up to 16384 x 16384 x 16384.
+ *   - All calls on a device share the one array, which keeps the previous call's contents; the
+ *     call re-zeroes the words that must start at zero.  Two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them. */
+#define FPSK_PROBE_STATIC_SCRATCH_BYTES (12u << 20)
+fpsk_status fpsk_probe_static(const void *A, int64_t lda, const void *B, int64_t ldb,
+                              const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                              fpsk_dtype dtype, int c_is_fp32, const fpsk_params *p, void *stream,
+                              fpsk_probe_result *d_result, float *d_residual);
+
 /* ---- hashed moment sketches --------------------------------------------------------------- */
 
 /* Hash round `round` of `seed` (Section "Moment Sketches": h1, v1 for side 0 = rows,

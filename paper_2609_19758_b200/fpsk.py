@@ -83,6 +83,9 @@ def lib() -> C.CDLL:
         L.fpsk_probe_host.restype = C.c_int
         L.fpsk_probe_host.argtypes = [vp, vp, vp, i64, i64, i64, C.c_int, C.POINTER(Params), vp, sz, vp,
                                       C.POINTER(ProbeResult)]
+        L.fpsk_probe_static.restype = C.c_int
+        L.fpsk_probe_static.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, C.c_int, C.POINTER(Params),
+                                        vp, vp, vp]
         L.fpsk_hash_tables.restype = C.c_int
         L.fpsk_hash_tables.argtypes = [u64, i32, i32, i64, i32, vp, vp, vp]
         L.fpsk_workspace_bytes.restype = sz
@@ -180,6 +183,23 @@ def probe(A, B, Cm, workspace: torch.Tensor, result: torch.Tensor, residual: Opt
                           _stream_ptr(stream), result.data_ptr(), residual.data_ptr() if residual is not None else None)
     if rc != STATUS_OK:
         raise FpskError(rc, "fpsk_probe")
+
+
+PROBE_STATIC_SCRATCH_BYTES = 12 << 20
+
+
+def probe_static(A, B, Cm, result: torch.Tensor, residual: Optional[torch.Tensor] = None,
+                 params: Optional[Params] = None, stream=None) -> None:
+    """The probe for callers that cannot allocate device memory (no workspace argument: the
+    scratch is a fixed array inside the library).  Same outputs as `probe`.  Calls sharing a
+    device must not overlap on the GPU."""
+    a = _mat_args(A, B, Cm)
+    rc = lib().fpsk_probe_static(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9],
+                                 1 if Cm.dtype == torch.float32 else 0,
+                                 C.byref(params) if params is not None else None, _stream_ptr(stream),
+                                 result.data_ptr(), residual.data_ptr() if residual is not None else None)
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_static")
 
 
 def new_probe_result(device=None) -> torch.Tensor:
