@@ -325,7 +325,7 @@ def oracle_probe_once(A64, B64, C64):
     import oracle as O
     E = O.error_matrix(A64, B64, C64)
     s = O.probe_sketch(E)
-    return O.probe_verdict(s, O.analytic_tau(A64, B64, A64.shape[1]))
+    return O.probe_verdict(s, O.analytic_tau(A64, B64, A64.shape[1]), n_rows=A64.shape[0])
 
 
 def cpu_baseline(args, batch, m, k, n, dt, nbytes):

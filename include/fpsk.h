@@ -56,7 +56,7 @@ typedef struct {
     int32_t status;      /* fpsk_status set by the device (FPSK_ERR_TIMEOUT) else FPSK_OK  */
     float max_abs;       /* max_j |s_j| over the finite entries                            */
     float sigma_hat;     /* 1.2533 mean(min(|s|, 5 mean|s|))                               */
-    float thr;           /* min(tau, mu sqrt(2 ln N_b) sigma_hat), N_b = max(n3, 2)        */
+    float thr;           /* min(tau sqrt(n1), mu sqrt(2 ln N_b) sigma_hat), N_b = max(n3, 2) */
     float tau;           /* 100 n2 2^-23 max|A| max|B|                                     */
 } fpsk_probe_result;
 
@@ -133,7 +133,8 @@ size_t fpsk_probe_workspace_bytes(int64_t m, int64_t k, int64_t n);
 fpsk_status fpsk_probe_init(void *workspace, size_t ws_bytes, void *stream);
 
 /* The detection sketch (Eq. (S) with H1 = 1^T, H2 = I): s = (1^T A) B - 1^T C, its noise
- * estimate, threshold and one-bit verdict (Section "Thresholds"; Algorithm 2, probe part),
+ * estimate, threshold and one-bit verdict (Section "Thresholds"; Algorithm 2, probe part;
+ * each entry of s sums n1 entries of E, so the analytic cap tau enters as tau sqrt(n1)),
  * in ONE kernel launch, asynchronous on `stream`, no host synchronisation.
  *   A, B       device, m x k and k x n, type `dtype`
  *   C          device, m x n FP32; c_is_fp32 must be 1: a narrowed C is rejected

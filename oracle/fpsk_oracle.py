@@ -188,16 +188,20 @@ def sigma_clip(S) -> float:
     return float(1.2533 * np.minimum(a, 5.0 * mean_abs).mean())
 
 
-def probe_verdict(s: np.ndarray, tau: float, params: Params = None) -> ProbeResult:
-    """thr = min(tau, mu sqrt(2 ln N_b) sigma_hat); dirty iff max|s| > thr or s is not
-    finite (Section "Thresholds", Algorithm 2 probe part, Section "Nonfinite").
-    N_b is the number of sketch entries: n3 here, m^2 in the paper's hashed probe."""
+def probe_verdict(s: np.ndarray, tau: float, params: Params = None, n_rows: int = 1) -> ProbeResult:
+    """thr = min(tau sqrt(n_rows), mu sqrt(2 ln N_b) sigma_hat); dirty iff max|s| > thr or s is
+    not finite (Section "Thresholds", Algorithm 2 probe part, Section "Nonfinite").
+    N_b is the number of sketch entries: n3 here, m^2 in the paper's hashed probe.
+    n_rows is the number of entries of E that one sketch entry sums (n1 for the column
+    sketch): the analytic cap tau bounds the rounding of ONE inner product (with slack 100),
+    and a sum of n_rows of them grows like sqrt(n_rows); with n_rows = 1 this is the paper's
+    rule verbatim.  (Reading for the un-hashed sketch; unpinned by the paper.)"""
     params = params or Params()
     s = np.asarray(s, dtype=np.float64)
     n_b = max(int(s.size), 2)
     nonfinite = bool(np.any(~np.isfinite(s)))
     sig = sigma_clip(s)
-    thr = min(tau, params.mu * math.sqrt(2.0 * math.log(n_b)) * sig)
+    thr = min(tau * math.sqrt(float(n_rows)), params.mu * math.sqrt(2.0 * math.log(n_b)) * sig)
     a = np.abs(s)
     if s.size:
         # NaN entries never win the argmax of the finite comparison

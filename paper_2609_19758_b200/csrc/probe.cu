@@ -505,7 +505,7 @@ __device__ void verdict(const ProbeArgs &p, int grid, float *red, int status, in
         const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) *
                           bits16_to_float<T>(mb);
         const float nb = (float)(n > 2 ? n : 2);
-        const float thr = fminf(tau, p.mu * sqrtf(2.f * logf(nb)) * sigma);
+        const float thr = fminf(tau * sqrtf((float)p.n1), p.mu * sqrtf(2.f * logf(nb)) * sigma);
         fpsk_probe_result r;
         r.nonfinite = anybad > 0.f ? 1 : 0;
         r.fired = (anybad > 0.f || am.v > thr) ? 1 : 0;
@@ -791,7 +791,8 @@ __device__ __noinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr
     if (ctid == 0) {
         const float sigma = 1.2533f * (csum_total / (float)n);
         const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) * bits16_to_float<T>(mb);
-        const float thr = fminf(tau, thr_scale * sigma);
+        // each s_j sums n1 entries of E: the per-entry cap tau grows like sqrt(n1) for the column sketch
+        const float thr = fminf(tau * sqrtf((float)p.n1), thr_scale * sigma);
         fpsk_probe_result r;
         r.nonfinite = bad > 0.f ? 1 : 0;
         r.fired = (bad > 0.f || am.v > thr) ? 1 : 0;

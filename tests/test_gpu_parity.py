@@ -84,7 +84,7 @@ def test_probe_residual_and_verdict(shape, dtype):
     assert np.all(np.abs(resid - s_ref) <= TOL * abs_j + 1e-30)
     assert got.tau == pytest.approx(tau, rel=1e-6)
     # the verdict formula applied to the GPU's own residual, in FP64
-    v = O.probe_verdict(resid, tau)
+    v = O.probe_verdict(resid, tau, n_rows=n1)
     assert got.sigma_hat == pytest.approx(v.sigma_hat, rel=1e-4, abs=1e-30)
     assert got.thr == pytest.approx(v.thr, rel=1e-4, abs=1e-30)
     assert got.max_abs == pytest.approx(v.max_abs, rel=1e-6, abs=1e-30)
@@ -92,7 +92,7 @@ def test_probe_residual_and_verdict(shape, dtype):
     if abs(v.max_abs - v.thr) > 1e-3 * v.thr:
         assert bool(got.fired) == v.fired
     if n3 >= 256:
-        assert not got.fired and not O.probe_verdict(s_ref, tau).fired      # clean product
+        assert not got.fired and not O.probe_verdict(s_ref, tau, n_rows=n1).fired      # clean product
 
 
 def test_probe_fires_on_faults_and_not_on_clean_with_the_oracle():
@@ -106,7 +106,7 @@ def test_probe_fires_on_faults_and_not_on_clean_with_the_oracle():
         f = W.faults_additive(n, n, rms, s, 1, 0.02, 0.09, "small")
         Cf, ch = W.inject(Cm, f)
         got, resid, _ = _run_probe(A, Bm, Cf)
-        ref = O.probe_verdict(O.probe_sketch(AB - Cf.double().numpy()), tau)
+        ref = O.probe_verdict(O.probe_sketch(AB - Cf.double().numpy()), tau, n_rows=n)
         assert ref.fired and got.fired == 1
         assert got.argmax_col == ref.argmax_col == f[0].j
         assert got.max_abs == pytest.approx(abs(ch[0]), rel=0.05)

@@ -119,7 +119,7 @@ def test_clean_integer_product_is_clean():
     A, B, C, _ = _int_case(24, 9, 20, 11)
     E = O.error_matrix(A, B, C)
     assert not E.any()
-    v = O.probe_verdict(O.probe_sketch(E), O.analytic_tau(A, B, 9))
+    v = O.probe_verdict(O.probe_sketch(E), O.analytic_tau(A, B, 9), n_rows=24)
     assert not v.fired and not v.nonfinite and v.thr == 0.0
     assert O.localize(A, B, C, seed=3, m_b=4, dtype=W.FP16, params=O.Params(radius=2)) == []
 
@@ -136,7 +136,7 @@ def test_clean_fp32_product_reports_nothing_and_lemma1_scan():
     st = {}
     F = O.localize(A, B, C, seed=8, m_b=4, dtype=W.FP16, params=O.Params(radius=3), stats=st)
     assert F == []
-    v = O.probe_verdict(O.probe_sketch(O.error_matrix(A, B, C)), O.analytic_tau(A, B, 64))
+    v = O.probe_verdict(O.probe_sketch(O.error_matrix(A, B, C)), O.analytic_tau(A, B, 64), n_rows=48)
     assert not v.fired
 
 
@@ -157,6 +157,9 @@ def test_probe_threshold_formula_on_known_vector():
     assert v.thr == pytest.approx(4 * math.sqrt(2 * math.log(100)) * 1.2533 * 0.5, rel=1e-12)
     assert not v.fired          # 0.5 < thr
     assert O.probe_verdict(s, tau=0.4).fired and O.probe_verdict(s, tau=0.4).thr == 0.4
+    # a sketch entry that sums n_rows entries of E: the analytic cap grows like sqrt(n_rows)
+    assert O.probe_verdict(s, tau=0.1, n_rows=16).thr == pytest.approx(0.4) and O.probe_verdict(s, tau=0.1, n_rows=16).fired
+    assert not O.probe_verdict(s, tau=0.2, n_rows=16).fired
     # one outlier is clipped at 5 mean|s| in the estimate
     s2 = np.ones(10)
     s2[0] = 91.0                      # mean|s| = 10, clip at 50

@@ -23,7 +23,7 @@ def test_small_square_fp16_clean_and_single_faults():
     assert 0.02 < nz.c_hat < 1.0            # same order as the paper's normalized constant
     tau = O.analytic_tau(A64, B64, 256)
     E = O.error_matrix(A64, B64, C.numpy())
-    assert not O.probe_verdict(O.probe_sketch(E), tau).fired
+    assert not O.probe_verdict(O.probe_sketch(E), tau, n_rows=256).fired
     p.radius = nz.radius
     assert O.localize(A64, B64, C.numpy(), 7, nz.m_loc, O.FP16, p, E=E) == []
     rms = W.rms(C)
@@ -31,7 +31,7 @@ def test_small_square_fp16_clean_and_single_faults():
         f = W.faults_additive(256, 256, rms, s, 1, 0.5, 0.5, "typical")
         Cf, changes = W.inject(C, f)
         Ef = O.error_matrix(A64, B64, Cf.numpy())
-        v = O.probe_verdict(O.probe_sketch(Ef), tau)
+        v = O.probe_verdict(O.probe_sketch(Ef), tau, n_rows=256)
         assert v.fired and v.argmax_col == f[0].j
         F = O.localize(A64, B64, Cf.numpy(), 7, nz.m_loc, O.FP16, p, E=Ef)
         assert [(x.i, x.j) for x in F] == [(f[0].i, f[0].j)]
