@@ -636,24 +636,42 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar)
 }
 // Bounded wait on an mbarrier phase: gives up (returns false) after about a second of polling
 // instead of spinning forever.
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity)
 {
     const long long t_end = clock64() + 2000000000LL;
     for (;;) {
 #pragma unroll 1
-        for (int it = 0; it < 1024; ++it) {
-            uint32_t ok;
-            asm volatile(
-                "{\n\t.reg .pred p;\n\t"
-                "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-                "selp.u32 %0, 1, 0, p;\n\t}"
-                : "=r"(ok)
-                : "r"(bar), "r"(parity)
-                : "memory");
-            if (ok) return true;
-        }
+        for (int it = 0; it < 1024; ++it)
+            if (mbar_try(bar, parity)) return true;
         if (clock64() > t_end) return false;
     }
+}
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity)
+{
+    if (mbar_try(bar, parity)) return true;       // the common case: one instruction
+    return mbar_wait_slow(bar, parity);
+}
+// The same for a whole warp: lane 0 polls, the outcome is broadcast, and __syncwarp orders the
+// other lanes' later reads after lane 0's observation of the completed phase.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity)
+{
+    int w = 1;
+    if ((threadIdx.x & 31) == 0) w = mbar_wait_bounded(bar, parity) ? 1 : 0;
+    w = __shfl_sync(0xFFFFFFFFu, w, 0);
+    __syncwarp();
+    return w != 0;
 }
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
@@ -725,7 +743,7 @@ struct VStat {
 };
 
 template <typename T>
-__device__ __noinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr_scale, float *sbuf, int sbuf_cap, float *red,
+__device__ __forceinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr_scale, float *sbuf, int sbuf_cap, float *red,
                                          uint32_t gbar, uint32_t gpar, int status, int ctid)
 {
     const int n = (int)p.n3;
@@ -778,7 +796,7 @@ __device__ __noinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr
                     mbar_expect_tx(gbar, (uint32_t)cntv * 4u);
                     bulk_g2s(smem_u32(sbuf), p.s + base, (uint32_t)cntv * 4u, gbar);
                 }
-                mbar_wait_bounded(gbar, gpar);
+                mbar_wait_warp(gbar, gpar);
                 gpar ^= 1u;
             } else {
                 for (int e = ctid; e < cntv; e += kTmaConsumers) sbuf[e] = __ldcg(p.s + base + e);
@@ -931,11 +949,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                     for (int t0 = 0; t0 < ngA; t0 += ut_rows) {
                         const int nt = min(ut_rows, ngA - t0);
                         if (ok) {
-                            int w = 1;
-                            if ((ctid & 31) == 0) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
-                            w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                            if (w) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
-                            if (!w) { ok = false; s_err = 1; }
+                            if (!mbar_wait_warp(full0 + 8 * stage, phase)) { ok = false; s_err = 1; }
                         }
                         if (ok) {
                             const float *tb = reinterpret_cast<const float *>(ring + (size_t)stage * kStageBytes);
@@ -996,13 +1010,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                         SyncConsumers::sync();
                     }
                     if (ok) {
-                        // lane 0 polls (bounded); the verdict is warp-uniform; every lane then
-                        // observes the completed phase itself before reading the stage
-                        int w = 1;
-                        if ((ctid & 31) == 0) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
-                        w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                        if (w) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
-                        if (!w) { ok = false; s_err = 1; }
+                        if (!mbar_wait_warp(full0 + 8 * stage, phase)) { ok = false; s_err = 1; }
                     }
                     if (ok && active) {
                         const unsigned char *sb = ring + (size_t)stage * kStageBytes + tc * 16;
@@ -1122,7 +1130,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                     mbar_expect_tx(gbar, bytes);
                     bulk_g2s(smem_u32(red), blk + (long long)t0 * jn, bytes, gbar);
                 }
-                const bool got = mbar_wait_bounded(gbar, gpar);
+                const bool got = mbar_wait_warp(gbar, gpar);
                 gpar ^= 1u;
                 if (!got) s_err = 1;
                 if (ctid < jn) {
