@@ -298,20 +298,20 @@ def run_ours(args):
                   "plan_m0_mloc_r": list(plans[len(plans) // 2]) if plans else None},
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                      "peak_source": peak_src + " copy bandwidth (MEASURED_PEAKS.json)" if peak_src == "measured" else "fallback 6650",
-                     "frac_of_nominal_8TBs": gbs / 8000.0, "kernel": "probe_kernel", "bytes_per_launch": nbytes,
+                     "frac_of_nominal_8TBs": gbs / 8000.0, "kernel": "probe_tma_kernel", "bytes_per_launch": nbytes,
                      "traffic": None},
         "e2e": {"value": nbytes / (e2e_ms_x * 1e-3) / 1e9 * world, "unit": "GB/s", "ms": e2e_ms_x,
                 "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 32},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
-    traffic_file = os.path.join(ROOT, "profiles", "probe_traffic.json")
+    # DRAM traffic per launch of the probe kernel, from the committed ncu summary (text, "key bytes")
     try:
-        with open(traffic_file) as f:
-            tj = json.load(f)
-        key = f"{m}x{k}x{n}_{args.dtype}"
-        if key in tj:
-            out["roofline"]["traffic"] = tj[key]
+        with open(os.path.join(ROOT, "profiles", "probe_traffic.txt")) as f:
+            for line in f:
+                parts = line.split("#")[0].split()
+                if len(parts) == 2 and parts[0] == f"{m}x{k}x{n}_{args.dtype}":
+                    out["roofline"]["traffic"] = int(parts[1])
     except Exception:
         pass
     if not args.no_cpu_baseline and not args.probe_only:

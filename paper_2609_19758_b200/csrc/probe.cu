@@ -837,6 +837,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
     const ProbeArgs &p = a.p;
     const int c = blockIdx.x, G = gridDim.x;
     const int tid = threadIdx.x;
+    if (tid == 0) trace_mark(p, c, 12);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages), gbar = smem_u32(bars + 2 * kStages);
     if (tid == 0) {
         for (int s = 0; s < kStages; ++s) {
@@ -1214,6 +1215,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
     // Error path only: before the CTA leaves, wait (bounded) for bulk copies that may still be
     // landing in its shared memory.
     __syncthreads();
+    if (tid == 0) trace_mark(p, c, 13);
     if (s_err && tid == kTmaConsumers) {
         for (int s = 0; s < kStages; ++s) {
             mbar_wait_bounded(full0 + 8 * s, 0);
