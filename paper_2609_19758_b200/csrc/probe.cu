@@ -603,6 +603,7 @@ constexpr int kSegMax = 4096;                 // bytes of one row segment: 256 x
 constexpr int kGatherFloats = 5120;           // staging of partial vectors in the final combine; lane-reduce scratch
 constexpr int kUChunkT = 1024;                // u values kept in shared memory
 constexpr int kTmaSmem = kStages * kStageBytes + (kGatherFloats + kUChunkT) * 4 + 256;
+constexpr int kMaxGridC = 256;                // grids up to this size combine their statistics in one batch of loads
 
 struct TDecomp {
     int cg;       // column groups
@@ -678,8 +679,22 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
 }
-// Orders this thread's earlier generic-proxy observations before its later async-proxy
-// (bulk copy) accesses.
+// Publication counters: a release-add makes everything this thread has observed (its own writes
+// and, through the preceding CTA barrier, its CTA's) visible before the count; the ticket is an
+// acquire-release add, so the last arriver also sees what every earlier arriver published.
+__device__ __forceinline__ void red_release_add(unsigned int *ctr)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(ctr), "r"(1u) : "memory");
+}
+__device__ __forceinline__ unsigned int atom_acq_rel_add(unsigned int *ctr)
+{
+    unsigned int old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(ctr), "r"(1u) : "memory");
+    return old;
+}
+// Cross-proxy fence between the generic proxy (ordinary loads/stores) and the async proxy (bulk
+// copies): a thread that has observed a publication (acquire) executes it before it issues bulk
+// copies of the published data.
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async;" ::: "memory"); }
 
 // Partition of `units` items over groups: the first urem groups own uq+1 items, the others uq.
@@ -743,85 +758,111 @@ struct VStat {
 };
 
 template <typename T>
-__device__ __forceinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr_scale, float *sbuf, int sbuf_cap, float *red,
-                                         uint32_t gbar, uint32_t gpar, int status, int ctid)
+__device__ __forceinline__ void write_verdict(const ProbeArgs &p, float thr_scale, float csum_total, float bad, ArgMax am,
+                                              unsigned int ma, unsigned int mb, int status)
 {
     const int n = (int)p.n3;
-    // thread 0 fetches the two operand maxima early; they are only needed at the very end
+    const float sigma = 1.2533f * (csum_total / (float)n);
+    const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) * bits16_to_float<T>(mb);
+    // each s_j sums n1 entries of E: the per-entry cap tau grows like sqrt(n1) for the column sketch
+    const float thr = fminf(tau * sqrtf((float)p.n1), thr_scale * sigma);
+    fpsk_probe_result r;
+    r.nonfinite = bad > 0.f ? 1 : 0;
+    r.fired = (bad > 0.f || am.v > thr) ? 1 : 0;
+    r.argmax_col = am.i;
+    r.status = status;
+    r.max_abs = am.v;
+    r.sigma_hat = sigma;
+    r.thr = thr;
+    r.tau = tau;
+    *p.result = r;
+}
+
+// Verdict in the last CTA.  Warp 0 combines the per-slice statistics (one batch of loads, warp
+// shuffles, no block barrier) and finishes alone when nothing exceeds the clip level; otherwise
+// all consumers make the second pass over s (staged into shared memory by one bulk copy).
+template <typename T>
+__device__ __forceinline__ void verdict_tma(const ProbeArgs &p, int grid, float thr_scale, float *sbuf, int sbuf_cap, float *red,
+                                            uint32_t gbar, uint32_t gpar, int status, int ctid, int *s_slow)
+{
+    const int n = (int)p.n3;
     unsigned int ma = 0, mb = 0;
-    if (ctid == 0) { ma = __ldcg(p.ctrl + 4); mb = __ldcg(p.ctrl + 5); }
-    // per-CTA slice statistics -> sum|s|, non-finite flag, max|s| and its column (fixed tree)
-    float sum = 0.f, bad = 0.f;
+    float sum = 0.f, bad = 0.f, clip = 0.f;
     ArgMax am = {-1.f, 0x7FFFFFFF};
-    for (int g = ctid; g < grid; g += kTmaConsumers) {
-        const float4 st = __ldcg(p.vstat + g);
-        sum += st.x;
-        bad += st.y;
-        am = amax(am, ArgMax{st.z, __float_as_int(st.w)});
-    }
+    if (ctid < 32) {
+        // the per-CTA records (slice statistics, operand maxima) come in by three bulk copies:
+        // one round trip and a few instructions, then a short loop over shared memory
+        float4 *sv = reinterpret_cast<float4 *>(red);
+        unsigned int *sa = reinterpret_cast<unsigned int *>(red + 4 * 512), *sb = sa + 512;
+        const uint32_t mbytes = ((uint32_t)grid * 4u + 15u) & ~15u;
+        if (ctid == 0) {
+            fence_proxy_async();
+            mbar_expect_tx(gbar, (uint32_t)grid * 16u + 2u * mbytes);
+            bulk_g2s(smem_u32(sv), p.vstat, (uint32_t)grid * 16u, gbar);
+            bulk_g2s(smem_u32(sa), p.maxA, mbytes, gbar);
+            bulk_g2s(smem_u32(sb), p.maxB, mbytes, gbar);
+        }
+        mbar_wait_warp(gbar, gpar);
+        for (int g = ctid; g < grid; g += 32) {
+            const float4 st = sv[g];
+            sum += st.x;
+            bad += st.y;
+            am = amax(am, ArgMax{st.z, __float_as_int(st.w)});
+            ma = max(ma, sa[g]);
+            mb = max(mb, sb[g]);
+        }
+        ma = __reduce_max_sync(0xFFFFFFFFu, ma);
+        mb = __reduce_max_sync(0xFFFFFFFFu, mb);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
-        bad += __shfl_xor_sync(0xFFFFFFFFu, bad, o);
-        ArgMax t;
-        t.v = __shfl_xor_sync(0xFFFFFFFFu, am.v, o);
-        t.i = __shfl_xor_sync(0xFFFFFFFFu, am.i, o);
-        am = amax(am, t);
-    }
-    VStat *vs = reinterpret_cast<VStat *>(red);
-    SyncConsumers::sync();
-    if ((ctid & 31) == 0) vs[ctid >> 5] = VStat{sum, bad, am};
-    SyncConsumers::sync();
-    {
-        VStat r = vs[0];
-        for (int w = 1; w < kTmaConsumers / 32; ++w) {
-            r.sum += vs[w].sum;
-            r.bad += vs[w].bad;
-            r.am = amax(r.am, vs[w].am);
+        for (int o = 16; o > 0; o >>= 1) {
+            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+            bad += __shfl_xor_sync(0xFFFFFFFFu, bad, o);
+            ArgMax t;
+            t.v = __shfl_xor_sync(0xFFFFFFFFu, am.v, o);
+            t.i = __shfl_xor_sync(0xFFFFFFFFu, am.i, o);
+            am = amax(am, t);
         }
-        sum = r.sum; bad = r.bad; am = r.am;
-    }
-    const float clip = 5.f * (sum / (float)n);
-    float csum_total = sum;                 // nothing is clipped when max|s| <= 5 mean|s|
-    if (bad > 0.f || !(am.v <= clip)) {
-        // some entry exceeds the clip level (or is not finite): second pass over all of s
-        const bool al16 = (reinterpret_cast<uintptr_t>(p.s) & 15) == 0;
-        float csum = 0.f;
-        for (int base = 0; base < n; base += sbuf_cap) {
-            const int cntv = min(sbuf_cap, n - base);
-            SyncConsumers::sync();
-            if (al16 && (cntv & 3) == 0) {
-                if (ctid == 0) {
-                    fence_proxy_async();
-                    mbar_expect_tx(gbar, (uint32_t)cntv * 4u);
-                    bulk_g2s(smem_u32(sbuf), p.s + base, (uint32_t)cntv * 4u, gbar);
-                }
-                mbar_wait_warp(gbar, gpar);
-                gpar ^= 1u;
-            } else {
-                for (int e = ctid; e < cntv; e += kTmaConsumers) sbuf[e] = __ldcg(p.s + base + e);
-                SyncConsumers::sync();
+        clip = 5.f * (sum / (float)n);
+        const bool slow = bad > 0.f || !(am.v <= clip);
+        if (ctid == 0) {
+            *s_slow = slow ? 1 : 0;
+            if (!slow) write_verdict<T>(p, thr_scale, sum, bad, am, ma, mb, status);   // nothing clipped: sum of min = sum
+            else {
+                VStat *vs = reinterpret_cast<VStat *>(red);
+                vs[0] = VStat{sum, bad, am};
             }
-            for (int j = ctid; j < cntv; j += kTmaConsumers) csum += fminf(fabsf(sbuf[j]), clip);
         }
-        csum_total = block_sum<kTmaConsumers, SyncConsumers>(csum, red + 256, ctid);
     }
-    if (ctid == 0) {
-        const float sigma = 1.2533f * (csum_total / (float)n);
-        const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) * bits16_to_float<T>(mb);
-        // each s_j sums n1 entries of E: the per-entry cap tau grows like sqrt(n1) for the column sketch
-        const float thr = fminf(tau * sqrtf((float)p.n1), thr_scale * sigma);
-        fpsk_probe_result r;
-        r.nonfinite = bad > 0.f ? 1 : 0;
-        r.fired = (bad > 0.f || am.v > thr) ? 1 : 0;
-        r.argmax_col = am.i;
-        r.status = status;
-        r.max_abs = am.v;
-        r.sigma_hat = sigma;
-        r.thr = thr;
-        r.tau = tau;
-        *p.result = r;
+    gpar ^= 1u;                 // warp 0 has used one phase of gbar; every thread tracks it
+    SyncConsumers::sync();
+    if (!*s_slow) return;
+    // some entry exceeds the clip level (or is not finite): second pass over all of s
+    {
+        const VStat r = reinterpret_cast<VStat *>(red)[0];
+        sum = r.sum; bad = r.bad; am = r.am;
+        clip = 5.f * (sum / (float)n);
     }
+    const bool al16 = (reinterpret_cast<uintptr_t>(p.s) & 15) == 0;
+    float csum = 0.f;
+    for (int base = 0; base < n; base += sbuf_cap) {
+        const int cntv = min(sbuf_cap, n - base);
+        SyncConsumers::sync();
+        if (al16 && (cntv & 3) == 0) {
+            if (ctid == 0) {
+                fence_proxy_async();
+                mbar_expect_tx(gbar, (uint32_t)cntv * 4u);
+                bulk_g2s(smem_u32(sbuf), p.s + base, (uint32_t)cntv * 4u, gbar);
+            }
+            mbar_wait_warp(gbar, gpar);
+            gpar ^= 1u;
+        } else {
+            for (int e = ctid; e < cntv; e += kTmaConsumers) sbuf[e] = __ldcg(p.s + base + e);
+            SyncConsumers::sync();
+        }
+        for (int j = ctid; j < cntv; j += kTmaConsumers) csum += fminf(fabsf(sbuf[j]), clip);
+    }
+    const float csum_total = block_sum<kTmaConsumers, SyncConsumers>(csum, red + 256, ctid);
+    if (ctid == 0) write_verdict<T>(p, thr_scale, csum_total, bad, am, ma, mb, status);
 }
 
 template <typename T>
@@ -834,6 +875,8 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
     unsigned long long *bars = reinterpret_cast<unsigned long long *>(us + kUChunkT);
     __shared__ int s_flag;
     __shared__ int s_err;
+    __shared__ int s_slow;
+    __shared__ unsigned int smx[kTmaConsumers / 32];
     const ProbeArgs &p = a.p;
     const int c = blockIdx.x, G = gridDim.x;
     const int tid = threadIdx.x;
@@ -924,6 +967,39 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
+        // Where this thread's partial sums go (offsets into partA / partP, in floats).  Worked out
+        // now, while the first tiles are still in flight, so that the epilogues are short.
+        // Layouts are blocked by their reader, so that every later gather is one contiguous copy:
+        //   partA : for each row group g of B, a block [t < ngA][rows of g] of partial column sums of A
+        //   partP : for each column slice c' of the final combine, a block [t < ngP + ngC][columns of c']
+        //           holding the partial p rows (t < ngP) and the partial column sums of C (t >= ngP)
+        long long eoff[3][2];
+#pragma unroll
+        for (int m = 0; m < 3; ++m) {
+            const Piece &q = pc[m];
+            const TDecomp &d = m == 0 ? a.tA : (m == 1 ? a.tC : a.tB);
+            const int tpr = q.segb / 16;
+            const int rl = ctid / tpr, tc = ctid - rl * tpr;
+            const int nv = m == 1 ? 4 : 8;
+            const int col0 = q.cg * (d.segb / (m == 1 ? 4 : 2)) + tc * nv;
+            eoff[m][0] = eoff[m][1] = 0;
+            if (q.has && rl == 0 && tc * 16 < q.wbytes) {
+#pragma unroll
+                for (int h = 0; h < 2; ++h) {
+                    if (h == 1 && nv == 4) break;
+                    const int u = (col0 >> 2) + h;
+                    int g, off, first, cnt;
+                    if (m == 0) {
+                        locate_unit(u, a.tB.uq, a.tB.urem, g, off, first, cnt);
+                        eoff[m][h] = (long long)first * 4 * ngA + (long long)q.rg * (cnt * 4) + off * 4;
+                    } else {
+                        locate_unit(u, a.sq, a.srem, g, off, first, cnt);
+                        const int t = m == 2 ? q.rg : a.tB.rg + q.rg;
+                        eoff[m][h] = (long long)first * 4 * (a.tB.rg + a.tC.rg) + (long long)t * (cnt * 4) + off * 4;
+                    }
+                }
+            }
+        }
         if (ctid == 0) trace_mark(p, c, 0);
 #pragma unroll
         for (int m = 0; m < 3; ++m) {
@@ -1044,11 +1120,6 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
             }
             if (ctid == 0) trace_mark(p, c, m == 0 ? 1 : (m == 1 ? 3 : 6));
             // ---- epilogue of the piece: combine row lanes (fixed order) and publish the partial
-            // Layouts are blocked by their reader, so that every later gather is one contiguous copy:
-            //   partA : for each row group g of B, a block [t < ngA][rows of g] of partial column sums of A
-            //   partP : for each column slice c' of the final combine, a block [t < ngP + ngC][columns of c']
-            //           holding the partial p rows (t < ngP) and the partial column sums of C (t >= ngP)
-            const TDecomp &d = m == 0 ? a.tA : (m == 1 ? a.tC : a.tB);
             const int nv = m == 1 ? 4 : 8;
             if (q.has) {
                 float4 lo = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
@@ -1066,37 +1137,27 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                         lo.x += x.x; lo.y += x.y; lo.z += x.z; lo.w += x.w;
                         hi.x += y.x; hi.y += y.y; hi.z += y.z; hi.w += y.w;
                     }
-                    const int col0 = q.cg * (d.segb / (m == 1 ? 4 : 2)) + tc * nv;     // first column of this thread
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        if (h == 1 && nv == 4) break;
-                        const int u = (col0 >> 2) + h;                                  // unit of 4 columns
-                        int g, off, first, cnt;
-                        float *dst;
-                        if (m == 0) {
-                            locate_unit(u, a.tB.uq, a.tB.urem, g, off, first, cnt);
-                            dst = p.partA + (long long)first * 4 * ngA + (long long)q.rg * (cnt * 4) + off * 4;
-                        } else {
-                            locate_unit(u, a.sq, a.srem, g, off, first, cnt);
-                            const int t = m == 2 ? q.rg : a.tB.rg + q.rg;
-                            dst = p.partP + (long long)first * 4 * (a.tB.rg + a.tC.rg) + (long long)t * (cnt * 4) + off * 4;
-                        }
-                        __stcg(reinterpret_cast<float4 *>(dst), h == 0 ? lo : hi);
-                    }
+                    float *pbase = m == 0 ? p.partA : p.partP;
+                    __stcg(reinterpret_cast<float4 *>(pbase + eoff[m][0]), lo);
+                    if (nv == 8) __stcg(reinterpret_cast<float4 *>(pbase + eoff[m][1]), hi);
                 }
             }
             if (m != 1) {
-                // max |.| of the half-precision operand (for tau): integer atomic, order-independent
+                // max |.| of the half-precision operand (for tau): one value per CTA, combined by the verdict
                 unsigned int mbits = float_to_bits16<T>(mm.absmax());
                 mbits = __reduce_max_sync(0xFFFFFFFFu, mbits);
-                if ((ctid & 31) == 0 && mbits) atomicMax(p.ctrl + (m == 0 ? 4 : 5), mbits);
+                if ((ctid & 31) == 0) smx[ctid >> 5] = mbits;
             }
-            if (m == 0) {
+            if (m != 1) {
                 SyncConsumers::sync();
                 if (ctid == 0) {
-                    __threadfence();
-                    atomicAdd(p.ctrl + 0, 1u);
-                    trace_mark(p, c, 2);
+                    unsigned int r_ = 0;
+                    for (int w = 0; w < kTmaConsumers / 32; ++w) r_ = max(r_, smx[w]);
+                    __stcg((m == 0 ? p.maxA : p.maxB) + c, r_);
+                    if (m == 0) {
+                        red_release_add(p.ctrl + 0);
+                        trace_mark(p, c, 2);
+                    }
                 }
             }
             if (m == 2 && ctid == 0) trace_mark(p, c, 7);
@@ -1104,9 +1165,8 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
         // ---- all partials of this CTA are written: grid-wide publication, then the slices
         SyncConsumers::sync();
         if (ctid == 0) {
-            __threadfence();
             if (!ok) atomicOr(p.ctrl + 3, 1u);
-            atomicAdd(p.ctrl + 1, 1u);
+            red_release_add(p.ctrl + 1);
             s_flag = (ok && bounded_wait_ge(p.ctrl + 1, (unsigned)G)) ? 1 : 0;
         }
         SyncConsumers::sync();
@@ -1121,8 +1181,16 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
             const int j0 = 4 * (c * a.sq + min(c, a.srem)), jn = 4 * (a.sq + (c < a.srem ? 1 : 0));
             const int ngP = a.tB.rg, ngC = a.tC.rg, ntot = ngP + ngC;
             const float *blk = p.partP + (long long)j0 * ntot;          // [ntot][jn], contiguous
-            const int tmax = jn > 0 ? kGatherFloats / jn : ntot;        // partial rows per pass (>= 1: jn <= kGatherFloats)
-            float sp0 = 0.f, sc0 = 0.f, sp1 = 0.f, sc1 = 0.f;           // columns ctid and ctid + 512
+            // thread (sub, kk) adds the partial rows t = sub, sub + nsub, ... of column kk; the sub-sums are
+            // then combined in sub order (fixed order: deterministic).  Wide slices: one thread per column pair.
+            int uw = 32;
+            while (uw < jn && uw < kTmaConsumers) uw <<= 1;
+            const int nsub = jn <= kTmaConsumers ? kTmaConsumers / uw : 1;
+            const int sub = jn <= kTmaConsumers ? ctid / uw : 0;
+            const int kk = jn <= kTmaConsumers ? ctid - sub * uw : ctid;
+            constexpr int kData = kGatherFloats - 2 * kTmaConsumers;    // staging; the tail of `red` holds the sub-sums
+            const int tmax = jn > 0 ? kData / jn : ntot;                 // partial rows per pass (>= 1: jn <= 1024)
+            float sp0 = 0.f, sc0 = 0.f, sp1 = 0.f, sc1 = 0.f;
             for (int t0 = 0; t0 < ntot && jn > 0; t0 += tmax) {
                 const int nt = min(tmax, ntot - t0);
                 if (ctid == 0) {
@@ -1134,26 +1202,41 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                 const bool got = mbar_wait_warp(gbar, gpar);
                 gpar ^= 1u;
                 if (!got) s_err = 1;
-                if (ctid < jn) {
+                if (kk < jn) {
+                    int t = (sub - t0 % nsub + nsub) % nsub;              // global row t0 + t is congruent to sub
 #pragma unroll 4
-                    for (int t = 0; t < nt; ++t) {
-                        const float v = red[t * jn + ctid];
+                    for (; t < nt; t += nsub) {
+                        const float v = red[t * jn + kk];
                         if (t0 + t < ngP) sp0 += v; else sc0 += v;
                     }
                 }
-                if (ctid + kTmaConsumers < jn) {
+                if (kk + kTmaConsumers < jn) {
 #pragma unroll 4
                     for (int t = 0; t < nt; ++t) {
-                        const float v = red[t * jn + ctid + kTmaConsumers];
+                        const float v = red[t * jn + kk + kTmaConsumers];
                         if (t0 + t < ngP) sp1 += v; else sc1 += v;
                     }
                 }
                 SyncConsumers::sync();
             }
+            if (nsub > 1) {
+                float *tmp = red + kData;
+                tmp[sub * uw + kk] = sp0;
+                tmp[kTmaConsumers + sub * uw + kk] = sc0;
+                SyncConsumers::sync();
+                if (sub == 0 && kk < jn) {
+                    sp0 = tmp[kk];
+                    sc0 = tmp[kTmaConsumers + kk];
+                    for (int s2 = 1; s2 < nsub; ++s2) {
+                        sp0 += tmp[s2 * uw + kk];
+                        sc0 += tmp[kTmaConsumers + s2 * uw + kk];
+                    }
+                }
+            }
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-                const int k = ctid + h * kTmaConsumers;
-                if (k < jn) {
+                const int k = kk + h * kTmaConsumers;
+                if (sub == 0 && k < jn) {
                     const float sv = h == 0 ? sp0 - sc0 : sp1 - sc1;
                     __stcg(p.s + j0 + k, sv);
                     const float av = fabsf(sv);
@@ -1165,39 +1248,43 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
         }
         // statistics of this CTA's slice (fixed tree: warp shuffles, then warp order)
         {
+            const int jn_ = 4 * (a.sq + (c < a.srem ? 1 : 0));
+            const bool one_warp = jn_ <= 32;              // then only warp 0 holds columns
+            if (!one_warp || ctid < 32) {
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
-                lbad += __shfl_xor_sync(0xFFFFFFFFu, lbad, o);
-                ArgMax t;
-                t.v = __shfl_xor_sync(0xFFFFFFFFu, lam.v, o);
-                t.i = __shfl_xor_sync(0xFFFFFFFFu, lam.i, o);
-                lam = amax(lam, t);
-            }
-            VStat *vs = reinterpret_cast<VStat *>(red);
-            if ((ctid & 31) == 0) vs[ctid >> 5] = VStat{lsum, lbad, lam};
-            SyncConsumers::sync();
-            if (ctid == 0) {
-                VStat r = vs[0];
-                for (int w = 1; w < kTmaConsumers / 32; ++w) {
-                    r.sum += vs[w].sum;
-                    r.bad += vs[w].bad;
-                    r.am = amax(r.am, vs[w].am);
+                for (int o = 16; o > 0; o >>= 1) {
+                    lsum += __shfl_xor_sync(0xFFFFFFFFu, lsum, o);
+                    lbad += __shfl_xor_sync(0xFFFFFFFFu, lbad, o);
+                    ArgMax t;
+                    t.v = __shfl_xor_sync(0xFFFFFFFFu, lam.v, o);
+                    t.i = __shfl_xor_sync(0xFFFFFFFFu, lam.i, o);
+                    lam = amax(lam, t);
                 }
-                __stcg(p.vstat + c, make_float4(r.sum, r.bad, r.am.v, __int_as_float(r.am.i)));
+            }
+            if (one_warp) {
+                if (ctid == 0) __stcg(p.vstat + c, make_float4(lsum, lbad, lam.v, __int_as_float(lam.i)));
+            } else {
+                VStat *vs = reinterpret_cast<VStat *>(red);
+                if ((ctid & 31) == 0) vs[ctid >> 5] = VStat{lsum, lbad, lam};
+                SyncConsumers::sync();
+                if (ctid == 0) {
+                    VStat r = vs[0];
+                    for (int w = 1; w < kTmaConsumers / 32; ++w) {
+                        r.sum += vs[w].sum;
+                        r.bad += vs[w].bad;
+                        r.am = amax(r.am, vs[w].am);
+                    }
+                    __stcg(p.vstat + c, make_float4(r.sum, r.bad, r.am.v, __int_as_float(r.am.i)));
+                }
             }
         }
         SyncConsumers::sync();
         if (ctid == 0) {
             trace_mark(p, c, 9);
-            __threadfence();
             if (!ok2 || s_err) atomicOr(p.ctrl + 3, 1u);
-            const unsigned int t = atomicAdd(p.ctrl + 2, 1u);
+            const unsigned int t = atom_acq_rel_add(p.ctrl + 2);
             s_flag = (t == (unsigned)G - 1) ? 1 : 0;
-            if (s_flag) {
-                __threadfence();
-                s_flag = 1 + (int)__ldcg(p.ctrl + 3);      // 1: all good, 2: some CTA gave up
-            }
+            if (s_flag) s_flag = 1 + (int)__ldcg(p.ctrl + 3);      // 1: all good, 2: some CTA gave up
             trace_mark(p, c, 10);
         }
         SyncConsumers::sync();
@@ -1205,10 +1292,10 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
             const int failed = s_flag - 1;
             // the ring is idle by now (every stage was consumed): reuse it to stage s
             verdict_tma<T>(p, G, a.thr_scale, reinterpret_cast<float *>(ring), kStages * kStageBytes / 4, red, gbar, gpar,
-                           failed ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK, ctid);
+                           failed ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK, ctid, &s_slow);
             if (ctid == 0) {
                 trace_mark(p, c, 11);
-                if (!failed) { p.ctrl[0] = 0; p.ctrl[1] = 0; p.ctrl[2] = 0; p.ctrl[4] = 0; p.ctrl[5] = 0; }
+                if (!failed) { p.ctrl[0] = 0; p.ctrl[1] = 0; p.ctrl[2] = 0; }
             }
         }
     }
