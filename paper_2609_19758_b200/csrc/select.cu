@@ -313,17 +313,32 @@ fpsk_status select_candidates_launch(const float *S, const float *R, const float
 }
 
 // ---------------------------------------------------------------- max |X| of a half matrix
+// max |x| over a half-precision matrix as a 16-bit pattern (sign cleared; for finite values the
+// unsigned order of the patterns is the order of the magnitudes in both formats).
 template <typename T>
-__global__ void max_abs_half_kernel(const unsigned short *X, long long ld, long long rows, long long cols, unsigned int *out)
+__global__ void __launch_bounds__(256) max_abs_half_kernel(const unsigned short *X, long long ld, long long rows, long long cols,
+                                                           int vec_ok, unsigned int *out)
 {
     unsigned int m = 0;
-    const long long total = rows * cols;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-        const long long r = i / cols, c = i - r * cols;
-        m = max(m, (unsigned int)(X[r * ld + c] & 0x7FFFu));
+    if (vec_ok) {
+        const long long cv = cols / 8;               // 16-byte vectors per row
+        const long long total = rows * cv;
+        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+            const long long r = i / cv, c = i - r * cv;
+            const uint4 v = ldg_nc_v4(X + r * ld + c * 8);
+            const unsigned int w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                m = max(m, (w[q] >> 16) & 0x7FFFu);
+                m = max(m, w[q] & 0x7FFFu);
+            }
+        }
+    } else {
+        for (long long r = blockIdx.x; r < rows; r += gridDim.x)
+            for (long long c = threadIdx.x; c < cols; c += blockDim.x) m = max(m, (unsigned int)(X[r * ld + c] & 0x7FFFu));
     }
     m = __reduce_max_sync(0xFFFFFFFFu, m);
-    if ((threadIdx.x & 31) == 0) atomicMax(out, m);
+    if ((threadIdx.x & 31) == 0 && m) atomicMax(out, m);
 }
 template <typename T>
 __global__ void max_abs_finish_kernel(const unsigned int *bits, float *out)
@@ -336,14 +351,15 @@ fpsk_status max_abs_half_launch(const void *X, long long ld, long long rows, lon
 {
     FPSK_CUDA_OK(cudaMemsetAsync(scratch, 0, 4, st));
     const unsigned short *x = static_cast<const unsigned short *>(X);
-    long long want = (rows * cols + 256 * 32 - 1) / (256 * 32);
+    const int vec_ok = ((reinterpret_cast<uintptr_t>(X) & 15) == 0 && ld % 8 == 0 && cols % 8 == 0) ? 1 : 0;
+    long long want = vec_ok ? (rows * (cols / 8) + 256 * 4 - 1) / (256 * 4) : rows;
     const int grid = (int)(want < 1 ? 1 : (want > 2368 ? 2368 : want));
     if (dtype == FPSK_FP16) {
-        max_abs_half_kernel<__half><<<grid, 256, 0, st>>>(x, ld, rows, cols, scratch);
+        max_abs_half_kernel<__half><<<grid, 256, 0, st>>>(x, ld, rows, cols, vec_ok, scratch);
         FPSK_LAUNCH_CHECK();
         max_abs_finish_kernel<__half><<<1, 32, 0, st>>>(scratch, out);
     } else {
-        max_abs_half_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(x, ld, rows, cols, scratch);
+        max_abs_half_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(x, ld, rows, cols, vec_ok, scratch);
         FPSK_LAUNCH_CHECK();
         max_abs_finish_kernel<__nv_bfloat16><<<1, 32, 0, st>>>(scratch, out);
     }

@@ -52,23 +52,24 @@ __global__ void scan_kernel(const int *count, int m_b, int *start)
 }
 
 // Stable placement: entry idx goes to start[b] + (number of idx' < idx in the same bucket).
-// perm packs the index (low 31 bits) and the sign (bit 31 set = -1).
-__global__ void place_kernel(const int *bucket, const int *sign, const int *start, int n, uint32_t *perm)
+// perm packs the index (low 31 bits) and the sign (bit 31 set = -1).  One warp per entry: the
+// lanes share the scan over the earlier entries, so the O(n^2 / 2) comparisons spread over the
+// whole GPU.
+__global__ void __launch_bounds__(256) place_kernel(const int *bucket, const int *sign, const int *start, int n, uint32_t *perm)
 {
-    __shared__ int tile[1024];
-    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
-    const int b = idx < n ? bucket[idx] : -1;
-    int rank = 0;
-    const int hi = min(n, (int)((blockIdx.x + 1) * blockDim.x));
-    for (int base = 0; base < hi; base += 1024) {
-        __syncthreads();
-        int t = base + threadIdx.x;
-        tile[threadIdx.x] = t < n ? bucket[t] : -2;
-        __syncthreads();
-        int lim = min(1024, idx - base);   // only earlier indices count
-        for (int q = 0; q < lim; ++q) rank += (tile[q] == b);
+    const int idx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (idx >= n) return;
+    const int b = __ldg(bucket + idx);
+    int cnt = 0;
+    int j = lane;
+    for (; j + 96 < idx; j += 128) {
+        const int b0 = __ldg(bucket + j), b1 = __ldg(bucket + j + 32), b2 = __ldg(bucket + j + 64), b3 = __ldg(bucket + j + 96);
+        cnt += (b0 == b) + (b1 == b) + (b2 == b) + (b3 == b);
     }
-    if (idx < n) perm[start[b] + rank] = (uint32_t)idx | (sign[idx] < 0 ? 0x80000000u : 0u);
+    for (; j < idx; j += 32) cnt += (__ldg(bucket + j) == b);
+    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    if (lane == 0) perm[__ldg(start + b) + cnt] = (uint32_t)idx | (__ldg(sign + idx) < 0 ? 0x80000000u : 0u);
 }
 
 fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, int *bucket, int *sign,
@@ -81,7 +82,7 @@ fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, in
     if (!perm) return FPSK_OK;
     scan_kernel<<<1, 1024, 0, st>>>(count, m_b, start);
     FPSK_LAUNCH_CHECK();
-    place_kernel<<<(n + 1023) / 1024, 1024, 0, st>>>(bucket, sign, start, n, perm);
+    place_kernel<<<(n + 7) / 8, 256, 0, st>>>(bucket, sign, start, n, perm);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
@@ -252,22 +253,22 @@ __global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long lon
 // sketch noise is the measured quantity, so no reduced-precision tensor-core path here).
 // blockIdx.z = problem * ksplit + split; each split writes its own partial output.
 struct GemmBatch {
-    const float *A[3];
-    const float *B[3];
+    const float *P, *Pw;      // problems: 0 = P Q, 1 = Pw Q, 2 = P Qw
+    const float *Q, *Qw;
     float *Cpart;     // [ksplit][3][M*N]
     int M, N, K, lda, ldb, ksplit, kchunk;
 };
 
 template <int BM, int BN, int T>   // T = 4 or 8 outputs per thread per dimension; 256 threads
-__global__ void __launch_bounds__(256) sgemm_kernel(const GemmBatch g)
+__global__ void __launch_bounds__(256, 2) sgemm_kernel(const GemmBatch g)
 {
     constexpr int BK = 16;
     constexpr int PADM = BM + 4, PADN = BN + 4;
     __shared__ __align__(16) float As[2][BK][PADM];
     __shared__ __align__(16) float Bs[2][BK][PADN];
     const int prob = blockIdx.z / g.ksplit, ks = blockIdx.z % g.ksplit;
-    const float *__restrict__ A = g.A[prob];
-    const float *__restrict__ B = g.B[prob];
+    const float *__restrict__ A = prob == 1 ? g.Pw : g.P;
+    const float *__restrict__ B = prob == 2 ? g.Qw : g.Q;
     const int m0 = blockIdx.y * BM, n0 = blockIdx.x * BN;
     const int k_begin = ks * g.kchunk, k_end = min(g.K, k_begin + g.kchunk);
     const int tid = threadIdx.x;
@@ -510,9 +511,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     }
     {
         GemmBatch g;
-        g.A[0] = w.P; g.B[0] = w.Q;
-        g.A[1] = w.Pw; g.B[1] = w.Q;
-        g.A[2] = w.P; g.B[2] = w.Qw;
+        g.P = w.P; g.Pw = w.Pw; g.Q = w.Q; g.Qw = w.Qw;
         g.Cpart = w.partAB;
         g.M = m_b; g.N = m_b; g.K = pl.kpad; g.lda = pl.kpad; g.ldb = pl.npad;
         g.ksplit = pl.ksplit; g.kchunk = pl.kchunk;
