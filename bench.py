@@ -135,7 +135,7 @@ def make_batches(args, m, k, n, dt, nsets, seed0=0):
 
 def run_ours(args):
     from paper_2609_19758_b200 import build as Bld
-    from paper_2609_19758_b200 import fpsk, harness, workloads as W
+    from paper_2609_19758_b200 import fpsk, harness, replicas, workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -253,11 +253,8 @@ def run_ours(args):
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - w0) * 1e3 / Ke
 
-    # max over ranks
-    stats = torch.tensor([probe_mean, total_ms / K, e2e_ms], dtype=torch.float64, device="cuda")
-    if dist is not None:
-        dist.all_reduce(stats, op=dist.ReduceOp.MAX)
-    probe_mean_x, step_ms_x, e2e_ms_x = (float(x) for x in stats.cpu())
+    # max over ranks (replicas only: no data-path collective)
+    probe_mean_x, step_ms_x, e2e_ms_x = replicas.max_over_ranks([probe_mean, total_ms / K, e2e_ms], dist, device="cuda")
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
@@ -267,7 +264,7 @@ def run_ours(args):
     gbs = nbytes / (probe_mean_x * 1e-3) / 1e9
     out = {
         "metric": "clean-path probe HBM GB/s (probe ms beside vendor GEMM ms; fault recovery rate)",
-        "value": gbs * world,
+        "value": replicas.whole_job_throughput(nbytes / 1e9, probe_mean_x * 1e-3, world),
         "unit": "GB/s",
         "n_gpus": world,
         "steps": K,
@@ -300,7 +297,7 @@ def run_ours(args):
                      "peak_source": peak_src + " copy bandwidth (MEASURED_PEAKS.json)" if peak_src == "measured" else "fallback 6650",
                      "frac_of_nominal_8TBs": gbs / 8000.0, "kernel": "probe_tma_kernel", "bytes_per_launch": nbytes,
                      "traffic": None},
-        "e2e": {"value": nbytes / (e2e_ms_x * 1e-3) / 1e9 * world, "unit": "GB/s", "ms": e2e_ms_x,
+        "e2e": {"value": replicas.whole_job_throughput(nbytes / 1e9, e2e_ms_x * 1e-3, world), "unit": "GB/s", "ms": e2e_ms_x,
                 "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 32},
         "gpu_launches": int(launches),
         "clocks": clocks,
