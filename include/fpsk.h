@@ -231,6 +231,43 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
                           void *workspace, size_t ws_bytes, void *stream,
                           fpsk_fault *h_faults, int32_t capacity, int32_t *h_count);
 
+/* ---- Algorithm 2 complete: verify, localize, repair in place ------------------------------ */
+
+typedef struct {
+    int32_t state;        /* 0: clean (only the probe ran); 1: repaired, the second probe is clean;
+                             2: the second probe still fires - the caller must recompute C = AB */
+    int32_t n_faults;     /* faults found (absolute ones included)                              */
+    int32_t n_absolute;   /* entries found by the exact scan (not finite, or |C_ij| > fp32max/16) */
+    int32_t m_loc;        /* bucket count localization ran at                                   */
+    int32_t radius;       /* search radius it used                                              */
+    int32_t reserved;
+    fpsk_probe_result first_probe, second_probe;
+} fpsk_repair_report;
+
+/* Bytes of workspace for fpsk_verify_repair (n_buckets <= 0: sized for any plan). */
+size_t fpsk_repair_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, const fpsk_params *p);
+
+/* Algorithm 2: probe; on a dirty product the exact scan for entries that are not finite or
+ * larger than fp32max/16 (at most K, recomputed as absolute values; C holds the recomputed
+ * values while the sketches are built and gets them back afterwards - Section "Nonfinite and
+ * Out of Range Entries"), the plan from the noise measured on this call (sigma_MAD of a fresh S
+ * at the law's bucket count and the strided rms of C; n_buckets > 0 skips the plan), k rounds
+ * of Algorithm 1, then Apply: C_ij <- delta for the absolute entries, C_ij <- C_ij + delta for
+ * the others, and a second probe.  C is MODIFIED in place (device, m x n FP32).
+ * Faults come back sorted by (i, j); absolute entries have round = -1, bucket_a = bucket_b = -1
+ * and delta = recompute = the repaired value.  Host outputs; the call synchronises `stream`. */
+fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_t ldb, float *C, int64_t ldc,
+                               int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed,
+                               int32_t n_buckets, const fpsk_params *p, void *workspace, size_t ws_bytes,
+                               void *stream, fpsk_fault *h_faults, int32_t capacity,
+                               fpsk_repair_report *h_report);
+
+/* The Apply step alone (Algorithm 2, "Apply"): writes a fault list into C.  Entries with
+ * round < 0 are absolute (C_ij <- delta), the others corrections (C_ij <- C_ij + delta).
+ * h_faults is a host array; workspace needs 256 KiB; at most 4096 entries per call. */
+fpsk_status fpsk_apply_corrections(float *C, int64_t ldc, int64_t m, int64_t n, const fpsk_fault *h_faults,
+                                   int32_t count, void *workspace, size_t ws_bytes, void *stream);
+
 /* Number of kernels launched by this library since load (all entry points, all threads). */
 uint64_t fpsk_launch_count(void);
 

@@ -41,7 +41,7 @@ __all__ = [
     "localize_round", "localize",
     "c_f", "law_sigma", "m_comb", "m_max", "m_mem", "m_num", "m_start", "cap_K",
     "rms_c_estimate", "index_budget", "radius_from_budget", "plan", "recalibrated_m",
-    "measure_noise",
+    "measure_noise", "scan_out_of_range", "apply_corrections", "verify_repair", "FP32_MAX",
 ]
 
 EPS32 = 2.0 ** -23          # FP32 machine epsilon used by the thresholds (Section "Validation")
@@ -560,3 +560,123 @@ def measure_noise(A, B, C, seed: int, dtype: int, m0: int = 0, params: Params = 
     else:
         m_probe = m0
     return NoiseResult(s_clip, s_mad, rms, c_hat, Bv, m0, m_probe, m_loc, r)
+
+
+# ----------------------------------------------------------------------------
+# Algorithm 2 complete: exact scan, absolute repairs, apply, second probe
+# (Section "Nonfinite and Out of Range Entries"; Algorithm 2)
+# ----------------------------------------------------------------------------
+FP32_MAX = float(np.finfo(np.float32).max)
+
+
+def scan_out_of_range(C, K: int):
+    """Coordinates of entries that are not finite or larger than fp32max/16 in magnitude, in
+    row-major order, at most K of them."""
+    C = np.asarray(C)
+    with np.errstate(invalid="ignore"):
+        bad = ~(np.abs(C.astype(np.float64)) <= FP32_MAX / 16.0)
+    ii, jj = np.nonzero(bad)
+    return [(int(i), int(j)) for i, j in zip(ii[:K], jj[:K])]
+
+
+def apply_corrections(C, F: List[Fault]) -> np.ndarray:
+    """C_ij <- delta for absolute entries (round < 0), C_ij <- C_ij + delta otherwise, in FP32."""
+    out = np.array(C, dtype=np.float32, copy=True)
+    for f in F:
+        if f.round < 0:
+            out[f.i, f.j] = np.float32(f.delta)
+        else:
+            out[f.i, f.j] = np.float32(np.float64(out[f.i, f.j]) + f.delta)
+    return out
+
+
+def verify_repair(A, B, C, seed: int, dtype: int, params: Params = None, m_b: int = 0):
+    """Algorithm 2: probe; scan; absolute repairs held in C while the sketches are built; plan
+    from sigma_MAD of a fresh S at the law's bucket count and the strided rms of C (unless m_b
+    is given); k rounds of Algorithm 1; restore; apply; second probe.
+    Returns (C_out, F sorted by (i, j), report dict)."""
+    params = params or Params()
+    A64, B64 = _f64(A), _f64(B)
+    C = np.array(C, dtype=np.float32, copy=True)
+    n1, n2 = A64.shape
+    n3 = B64.shape[1]
+    tau = analytic_tau(A64, B64, n2)
+    AB = A64 @ B64
+    first = probe_verdict(probe_sketch(AB - C.astype(np.float64)), tau, params, n_rows=n1)
+    rep = dict(state=0, n_faults=0, n_absolute=0, m_loc=0, radius=0, first_probe=first, second_probe=None)
+    if not first.fired:
+        return C, [], rep
+    K = cap_K(params)
+    F: List[Fault] = []
+    work = C.copy()
+    for (i, j) in scan_out_of_range(C, K):
+        gamma = float(np.dot(A64[i, :], B64[:, j]))
+        F.append(Fault(i, j, gamma, gamma, float(C[i, j]), -1, -1, -1))
+        work[i, j] = np.float32(gamma)
+    rep["n_absolute"] = len(F)
+    E = AB - work.astype(np.float64)
+    r = params.radius
+    if m_b <= 0:
+        m0 = m_start(n1, n2, n3, dtype, params)
+        h1, v1 = hash_round(seed, 0, 0, n1, m0)
+        h2, v2 = hash_round(seed, 0, 1, n3, m0)
+        S0, _, _ = moment_sketches(E, h1, v1, h2, v2, m0)
+        m_b, r_plan, _ = plan(n1, n2, n3, dtype, sigma_mad(S0, params.mad_of_abs), rms_c_estimate(work), m0, params)
+        if r < 0:
+            r = r_plan
+    if r < 0:
+        h1, v1 = hash_round(seed, 0, 0, n1, m_b)
+        h2, v2 = hash_round(seed, 0, 1, n3, m_b)
+        S0, _, _ = moment_sketches(E, h1, v1, h2, v2, m_b)
+        sig0, rms = sigma_mad(S0, params.mad_of_abs), rms_c_estimate(work)
+        if not (np.isfinite(sig0) and sig0 > 0 and np.isfinite(rms) and rms > 0):
+            sig0, rms = law_sigma(n1, n2, n3, dtype, 1.0, m_b), 1.0
+        r = min(params.r_max, radius_from_budget(index_budget(n1, n3, sig0, rms, params.rho_min)))
+    rep["m_loc"], rep["radius"] = m_b, r
+    for t in range(params.rounds):
+        # absolute entries are in F (never revisited) but are not peeled
+        peeled = [f for f in F if f.round >= 0]
+        known = [f for f in F if f.round < 0]
+        Ft = list(peeled)
+        Ft = _round_with_known(A64, B64, work, E, seed, t, m_b, r, Ft, known, params, tau)
+        F = known + Ft
+    F = sorted(F, key=lambda f: (f.i, f.j))
+    C_out = apply_corrections(C, F)
+    second = probe_verdict(probe_sketch(AB - C_out.astype(np.float64)), tau, params, n_rows=n1)
+    rep["second_probe"] = second
+    rep["n_faults"] = len(F)
+    rep["state"] = 2 if second.fired else 1
+    return C_out, F, rep
+
+
+def _round_with_known(A64, B64, C, E, seed, rnd, m_b, r, F_finite, F_abs, params, tau):
+    """One round of Algorithm 1 where F = F_finite + F_abs: only F_finite is peeled, both are
+    skipped by the search."""
+    n1, n3 = E.shape
+    h1, v1 = hash_round(seed, rnd, 0, n1, m_b)
+    h2, v2 = hash_round(seed, rnd, 1, n3, m_b)
+    S, R, T = moment_sketches(E, h1, v1, h2, v2, m_b)
+    peel(S, R, T, F_finite, h1, v1, h2, v2, n1, n3)
+    sig = sigma_mad(S, params.mad_of_abs)
+    thr = max(min(tau, 2.0 * sig), max(n1, n3) * sig / max(float(r), 0.5))
+    U = decode_candidates(S, R, T, select_candidates(S, thr, cap_K(params)), n1, n3)
+    inF = {(f.i, f.j) for f in F_finite} | {(f.i, f.j) for f in F_abs}
+    alive = list(U)
+    for (di, dj) in search_offsets(r):
+        if not alive:
+            break
+        still = []
+        for (flat, ih, jh) in alive:
+            i, j = ih + di, jh + dj
+            if i < 0 or i >= n1 or j < 0 or j >= n3 or (i, j) in inF:
+                still.append((flat, ih, jh))
+                continue
+            ok, gamma, _ = validate_entry(A64, B64, C, i, j, params.c_valid)
+            if ok:
+                cij = float(C[i, j])
+                F_finite.append(Fault(i, j, gamma - cij, gamma, cij, rnd, flat // m_b, flat % m_b))
+                inF.add((i, j))
+            else:
+                still.append((flat, ih, jh))
+        alive = still
+    return F_finite

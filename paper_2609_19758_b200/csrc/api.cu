@@ -156,6 +156,114 @@ static int offset_rank_key(int di, int dj, int r)
     return ((ch * 64 + mh) * 64 + (di + r)) * 64 + (dj + r);
 }
 
+// The localize part of Algorithm 2: p.rounds rounds of Algorithm 1 at m_b buckets, carrying F.
+// Entries already in F with round < 0 are absolute repairs (Section "Nonfinite"): they count as
+// found but are not peeled, their error is already absent from the sketches.
+static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int m_b, const fpsk_params &q, LocWs &w,
+                                 cudaStream_t st, std::vector<fpsk_fault> &F, bool &truncated, int &radius_used)
+{
+    const long long m = in.n1, k = in.n2, n = in.n3;
+    const long long mm = (long long)m_b * m_b;
+    const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
+    fpsk_status rc;
+    // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
+    unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
+    rc = max_abs_half_launch(in.A, in.lda, m, k, dtype, w.misc + 0, uscr, st);
+    if (rc != FPSK_OK) return rc;
+    rc = max_abs_half_launch(in.B, in.ldb, k, n, dtype, w.misc + 1, uscr + 1, st);
+    if (rc != FPSK_OK) return rc;
+    tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
+    FPSK_LAUNCH_CHECK();
+
+    int radius = q.radius;
+    bool round0_built = false;
+    if (radius < 0) {
+        // no calibration handed in: sigma_MAD of the first round's S and the strided rms of C
+        rc = build_sketches(in, dtype, seed, 0, m_b, true, w.sk, st, w.S, w.R, w.T);
+        if (rc != FPSK_OK) return rc;
+        round0_built = true;
+        rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+        if (rc != FPSK_OK) return rc;
+        float h_scal[8], h_rms = 0.f;
+        FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
+        rc = rms_c_launch(in.C, in.ldc, m, n, w.samples, w.sel, w.misc + 3, st);
+        if (rc != FPSK_OK) return rc;
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        double sig = h_scal[1], rms = h_rms;
+        if (!(std::isfinite(sig) && sig > 0 && std::isfinite(rms) && rms > 0)) {
+            sig = law_sigma((double)m, (double)k, (double)n, dtype, 1.0, (double)m_b);
+            rms = 1.0;
+        }
+        radius = std::min(q.r_max, radius_of_budget((double)std::max(m, n) * sig / (q.rho_min * rms)));
+    }
+    radius_used = radius;
+
+    std::vector<PeelEntry> peel;
+    std::vector<Hit> hits(kHitCap);
+    std::vector<Candidate> cand(kSelMaxK);
+    for (int t = 0; t < q.rounds; ++t) {
+        if (!(t == 0 && round0_built)) {
+            rc = build_sketches(in, dtype, seed, t, m_b, true, w.sk, st, w.S, w.R, w.T);
+            if (rc != FPSK_OK) return rc;
+        }
+        if (!peel.empty()) {
+            const int np = (int)std::min<size_t>(peel.size(), kPeelCap);
+            if ((int)peel.size() > kPeelCap) truncated = true;
+            FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, st));
+            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, w.R, w.T, st);
+            if (rc != FPSK_OK) return rc;
+        }
+        if (!(t == 0 && round0_built)) {
+            rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+            if (rc != FPSK_OK) return rc;
+        }
+        rc = select_candidates_launch(w.S, w.R, w.T, m_b, m, n, w.misc + 2, radius, K, w.sel, st);
+        if (rc != FPSK_OK) return rc;
+        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, st);
+        if (rc != FPSK_OK) return rc;
+        int h_counts[4] = {0, 0, 0, 0}, h_nhits = 0;
+        FPSK_CUDA_OK(cudaMemcpyAsync(h_counts, w.sel.counts, sizeof(h_counts), cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_nhits, w.n_hits, 4, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * kHitCap, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
+        const int nU = std::min(h_counts[2], K);
+
+        // replay of Algorithm 1's search: offsets in Chebyshev-then-Manhattan order, buckets of U
+        // in selection order; a bucket leaves U at its first accepted entry
+        std::sort(hits.begin(), hits.begin() + h_nhits, [&](const Hit &x, const Hit &y) {
+            const int kx = offset_rank_key(x.di, x.dj, radius), ky = offset_rank_key(y.di, y.dj, radius);
+            if (kx != ky) return kx < ky;
+            return x.cand < y.cand;
+        });
+        std::vector<char> alive((size_t)std::max(nU, 1), 1);
+        for (int h = 0; h < h_nhits; ++h) {
+            const Hit &x = hits[h];
+            if (x.cand < 0 || x.cand >= nU || !alive[x.cand]) continue;
+            bool inF = false;
+            for (const fpsk_fault &f : F)
+                if (f.i == x.i && f.j == x.j) { inF = true; break; }
+            if (inF) continue;
+            fpsk_fault f;
+            memset(&f, 0, sizeof(f));
+            f.i = x.i; f.j = x.j;
+            f.recompute = x.gamma;
+            f.c_value = x.c_value;
+            f.delta = x.gamma - (double)x.c_value;
+            f.round = t;
+            f.bucket_a = cand[x.cand].flat / m_b;
+            f.bucket_b = cand[x.cand].flat % m_b;
+            F.push_back(f);
+            // only finite faults are peeled (Section "Peeling Across Hash Rounds")
+            if (std::isfinite(f.delta)) peel.push_back(PeelEntry{f.i, f.j, f.delta});
+            alive[x.cand] = 0;
+        }
+    }
+    return FPSK_OK;
+}
+
 }  // namespace fpsk
 
 using namespace fpsk;
@@ -395,117 +503,209 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
     const fpsk_params q = resolve_params(p);
     if (!params_ok(q)) return FPSK_ERR_PARAM;
     if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
-    const int m_b = n_buckets;
     LocWs w;
-    if (!loc_carve(workspace, ws_bytes, m, k, n, m_b, w)) return FPSK_ERR_WORKSPACE;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w)) return FPSK_ERR_WORKSPACE;
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
-    const long long mm = (long long)m_b * m_b;
-    const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
     *h_count = 0;
-
-    // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
-    unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
-    rc = max_abs_half_launch(A, lda, m, k, dtype, w.misc + 0, uscr, st);
-    if (rc != FPSK_OK) return rc;
-    rc = max_abs_half_launch(B, ldb, k, n, dtype, w.misc + 1, uscr + 1, st);
-    if (rc != FPSK_OK) return rc;
-    tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
-    FPSK_LAUNCH_CHECK();
-
-    int radius = q.radius;
-    bool round0_built = false;
-    if (radius < 0) {
-        // no calibration handed in: sigma_MAD of the first round's S and the strided rms of C
-        rc = build_sketches(in, dtype, seed, 0, m_b, true, w.sk, st, w.S, w.R, w.T);
-        if (rc != FPSK_OK) return rc;
-        round0_built = true;
-        rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
-        if (rc != FPSK_OK) return rc;
-        float h_scal[8], h_rms = 0.f;
-        FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
-        rc = rms_c_launch(C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
-        if (rc != FPSK_OK) return rc;
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaStreamSynchronize(st));
-        double sig = h_scal[1], rms = h_rms;
-        if (!(std::isfinite(sig) && sig > 0 && std::isfinite(rms) && rms > 0)) {
-            sig = law_sigma((double)m, (double)k, (double)n, dtype, 1.0, (double)m_b);
-            rms = 1.0;
-        }
-        radius = std::min(q.r_max, radius_of_budget((double)std::max(m, n) * sig / (q.rho_min * rms)));
-    }
-
     std::vector<fpsk_fault> F;
-    std::vector<PeelEntry> peel;
-    std::vector<Hit> hits(kHitCap);
-    std::vector<Candidate> cand(kSelMaxK);
     bool truncated = false;
-    for (int t = 0; t < q.rounds; ++t) {
-        if (!(t == 0 && round0_built)) {
-            rc = build_sketches(in, dtype, seed, t, m_b, true, w.sk, st, w.S, w.R, w.T);
-            if (rc != FPSK_OK) return rc;
-        }
-        if (!peel.empty()) {
-            const int np = (int)std::min<size_t>(peel.size(), kPeelCap);
-            if ((int)peel.size() > kPeelCap) truncated = true;
-            FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, st));
-            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, w.R, w.T, st);
-            if (rc != FPSK_OK) return rc;
-        }
-        if (!(t == 0 && round0_built)) {
-            rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
-            if (rc != FPSK_OK) return rc;
-        }
-        rc = select_candidates_launch(w.S, w.R, w.T, m_b, m, n, w.misc + 2, radius, K, w.sel, st);
-        if (rc != FPSK_OK) return rc;
-        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, w.hits, w.n_hits, kHitCap, st);
-        if (rc != FPSK_OK) return rc;
-        int h_counts[4] = {0, 0, 0, 0}, h_nhits = 0;
-        FPSK_CUDA_OK(cudaMemcpyAsync(h_counts, w.sel.counts, sizeof(h_counts), cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_nhits, w.n_hits, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * kHitCap, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaStreamSynchronize(st));
-        if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
-        const int nU = std::min(h_counts[2], K);
-
-        // replay of Algorithm 1's search: offsets in Chebyshev-then-Manhattan order, buckets of U
-        // in selection order; a bucket leaves U at its first accepted entry
-        std::sort(hits.begin(), hits.begin() + h_nhits, [&](const Hit &x, const Hit &y) {
-            const int kx = offset_rank_key(x.di, x.dj, radius), ky = offset_rank_key(y.di, y.dj, radius);
-            if (kx != ky) return kx < ky;
-            return x.cand < y.cand;
-        });
-        std::vector<char> alive((size_t)std::max(nU, 1), 1);
-        for (int h = 0; h < h_nhits; ++h) {
-            const Hit &x = hits[h];
-            if (x.cand < 0 || x.cand >= nU || !alive[x.cand]) continue;
-            bool inF = false;
-            for (const fpsk_fault &f : F)
-                if (f.i == x.i && f.j == x.j) { inF = true; break; }
-            if (inF) continue;
-            fpsk_fault f;
-            memset(&f, 0, sizeof(f));
-            f.i = x.i; f.j = x.j;
-            f.recompute = x.gamma;
-            f.c_value = x.c_value;
-            f.delta = x.gamma - (double)x.c_value;
-            f.round = t;
-            f.bucket_a = cand[x.cand].flat / m_b;
-            f.bucket_b = cand[x.cand].flat % m_b;
-            F.push_back(f);
-            // only finite faults are peeled (Section "Peeling Across Hash Rounds")
-            if (std::isfinite(f.delta)) peel.push_back(PeelEntry{f.i, f.j, f.delta});
-            alive[x.cand] = 0;
-        }
-    }
+    int radius_used = 0;
+    rc = localize_core(in, dtype, seed, n_buckets, q, w, static_cast<cudaStream_t>(stream), F, truncated, radius_used);
+    if (rc != FPSK_OK) return rc;
     std::sort(F.begin(), F.end(), [](const fpsk_fault &x, const fpsk_fault &y) {
         return x.i != y.i ? x.i < y.i : x.j < y.j;
     });
     *h_count = (int32_t)F.size();
     const int ncopy = std::min<int>((int)F.size(), capacity);
     for (int f = 0; f < ncopy; ++f) h_faults[f] = F[f];
+    if ((int)F.size() > capacity || truncated) return FPSK_ERR_CAPACITY;
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- Algorithm 2, complete
+size_t fpsk_repair_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, const fpsk_params *p)
+{
+    if (m < 1 || k < 1 || n < 1) return 0;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return 0;
+    int mb = n_buckets;
+    if (mb <= 0) {   // calibrated on the call: size for the largest count the plan can ask for
+        mb = std::max({m_start_of(m, k, n, FPSK_FP16, q), m_start_of(m, k, n, FPSK_BF16, q), m_max_of(m, n)});
+        mb = std::min(mb, m_mem_of(k));
+        mb = std::min(mb, sketch_max_buckets(m, k, n));
+    }
+    if (mb < 1 || mb > sketch_max_buckets(m, k, n)) return 0;
+    return align_up(probe_ws_bytes(m, k, n), 256) + align_up(loc_ws_bytes(m, k, n, mb), 256) +
+           align_up(repair_scratch_bytes(), 256) + 256;
+}
+
+fpsk_status fpsk_apply_corrections(float *C, int64_t ldc, int64_t m, int64_t n, const fpsk_fault *h_faults,
+                                   int32_t count, void *workspace, size_t ws_bytes, void *stream)
+{
+    if (!C || (count > 0 && !h_faults) || !workspace) return FPSK_ERR_NULL;
+    if (m < 1 || n < 1 || ldc < n || count < 0) return FPSK_ERR_SHAPE;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    if (count > kRepairCap) return FPSK_ERR_CAPACITY;
+    if (ws_bytes < repair_scratch_bytes()) return FPSK_ERR_WORKSPACE;
+    for (int f = 0; f < count; ++f)
+        if (h_faults[f].i < 0 || h_faults[f].i >= m || h_faults[f].j < 0 || h_faults[f].j >= n) return FPSK_ERR_SHAPE;
+    if (count == 0) return FPSK_OK;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    std::vector<PatchEntry> pe((size_t)count);
+    for (int f = 0; f < count; ++f) {
+        pe[f].i = h_faults[f].i;
+        pe[f].j = h_faults[f].j;
+        pe[f].value = h_faults[f].delta;
+        pe[f].mode = h_faults[f].round < 0 ? PATCH_SET : PATCH_ADD;     // absolute entries carry the value itself
+    }
+    PatchEntry *d = static_cast<PatchEntry *>(workspace);
+    FPSK_CUDA_OK(cudaMemcpyAsync(d, pe.data(), sizeof(PatchEntry) * count, cudaMemcpyHostToDevice, st));
+    fpsk_status rc = patch_launch(C, ldc, d, count, st);
+    if (rc != FPSK_OK) return rc;
+    FPSK_CUDA_OK(cudaStreamSynchronize(st));      // pe is read by the copy until here
+    return FPSK_OK;
+}
+
+fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_t ldb, float *C, int64_t ldc, int64_t m,
+                               int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t n_buckets,
+                               const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream, fpsk_fault *h_faults,
+                               int32_t capacity, fpsk_repair_report *h_report)
+{
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (!workspace || !h_report || (capacity > 0 && !h_faults)) return FPSK_ERR_NULL;
+    if (capacity < 0) return FPSK_ERR_PARAM;
+    if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    if (n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
+    if (ws_bytes < fpsk_repair_workspace_bytes(m, k, n, n_buckets, p) || fpsk_repair_workspace_bytes(m, k, n, n_buckets, p) == 0)
+        return FPSK_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    memset(h_report, 0, sizeof(*h_report));
+
+    // workspace: [probe | verdict | repair scratch | localize]
+    char *wp = static_cast<char *>(workspace);
+    void *probe_ws = wp;
+    const size_t pws = align_up(probe_ws_bytes(m, k, n), 256);
+    fpsk_probe_result *d_res = reinterpret_cast<fpsk_probe_result *>(wp + pws);
+    void *rep_ws = wp + pws + 256;
+    char *loc_ws = wp + pws + 256 + align_up(repair_scratch_bytes(), 256);
+    const size_t loc_bytes = ws_bytes - (size_t)(loc_ws - wp);
+    const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
+
+    // ---- S-only probe (every call)
+    FPSK_CUDA_OK(cudaMemsetAsync(probe_ws, 0, 256, st));
+    ProbeDims pd{m, k, n, lda, ldb, ldc};
+    rc = probe_launch(A, B, C, pd, dtype, q.mu, probe_ws, pws, st, d_res, nullptr);
+    if (rc != FPSK_OK) return rc;
+    FPSK_CUDA_OK(cudaMemcpyAsync(&h_report->first_probe, d_res, sizeof(fpsk_probe_result), cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaStreamSynchronize(st));
+    if (h_report->first_probe.status != FPSK_OK) return (fpsk_status)h_report->first_probe.status;
+    if (!h_report->first_probe.fired) {
+        h_report->state = 0;       // clean: nothing else runs
+        return FPSK_OK;
+    }
+
+    // ---- exact scan for nonfinite / out-of-range entries, recomputed as absolute values
+    std::vector<fpsk_fault> F;
+    std::vector<PatchEntry> restore;
+    {
+        int n_abs = 0;
+        std::vector<ScanEntry> ent((size_t)K);
+        rc = scan_launch(C, ldc, m, n, K, rep_ws, st, ent.data(), &n_abs);
+        if (rc != FPSK_OK) return rc;
+        if (n_abs > 0) {
+            std::vector<double> gam((size_t)n_abs);
+            std::vector<float> oldv((size_t)n_abs);
+            SketchIn in0{A, B, C, m, k, n, lda, ldb, ldc};
+            rc = recompute_entries(in0, dtype, ent.data(), n_abs, rep_ws, st, gam.data(), oldv.data());
+            if (rc != FPSK_OK) return rc;
+            std::vector<PatchEntry> pe((size_t)n_abs);
+            for (int e = 0; e < n_abs; ++e) {
+                fpsk_fault f;
+                memset(&f, 0, sizeof(f));
+                f.i = ent[e].i; f.j = ent[e].j;
+                f.delta = gam[e];                 // absolute: the repaired value itself
+                f.recompute = gam[e];
+                f.c_value = oldv[e];
+                f.round = -1; f.bucket_a = -1; f.bucket_b = -1;
+                F.push_back(f);
+                pe[e] = PatchEntry{f.i, f.j, PATCH_SET, gam[e]};
+                restore.push_back(PatchEntry{f.i, f.j, PATCH_SET_BITS, 0.0});
+                memcpy(&restore.back().value, &oldv[e], sizeof(float));      // exact bit pattern of the old entry
+            }
+            // C holds the recomputed values while the sketches are built
+            PatchEntry *d = static_cast<PatchEntry *>(rep_ws);
+            FPSK_CUDA_OK(cudaMemcpyAsync(d, pe.data(), sizeof(PatchEntry) * n_abs, cudaMemcpyHostToDevice, st));
+            rc = patch_launch(C, ldc, d, n_abs, st);
+            if (rc != FPSK_OK) return rc;
+            FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        }
+        h_report->n_absolute = n_abs;
+    }
+
+    // ---- plan from the noise measured on this call, then k rounds of Algorithm 1
+    fpsk_params qq = q;
+    int m_loc = n_buckets;
+    if (m_loc <= 0) {
+        const int m0 = std::min(m_start_of(m, k, n, dtype, q), sketch_max_buckets(m, k, n));
+        LocWs w0;
+        if (!loc_carve(loc_ws, loc_bytes, m, k, n, m0, w0)) return FPSK_ERR_WORKSPACE;
+        SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+        rc = build_sketches(in, dtype, seed, 0, m0, false, w0.sk, st, w0.S, nullptr, nullptr);
+        if (rc != FPSK_OK) return rc;
+        rc = sigma_mad_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, w0.sel, st);
+        if (rc != FPSK_OK) return rc;
+        float h_scal[8], h_rms = 0.f;
+        FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w0.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
+        rc = rms_c_launch(C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);
+        if (rc != FPSK_OK) return rc;
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w0.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        int r;
+        double B_;
+        plan_of(m, k, n, dtype, h_scal[1], h_rms, m0, q, m_loc, r, B_);
+        m_loc = std::min(m_loc, sketch_max_buckets(m, k, n));
+        if (qq.radius < 0) qq.radius = r;
+    }
+    LocWs w;
+    if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w)) return FPSK_ERR_WORKSPACE;
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+    bool truncated = false;
+    int radius_used = 0;
+    rc = localize_core(in, dtype, seed, m_loc, qq, w, st, F, truncated, radius_used);
+    // ---- the absolute entries go back into C whatever happened above
+    if (!restore.empty()) {
+        PatchEntry *d = static_cast<PatchEntry *>(rep_ws);
+        FPSK_CUDA_OK(cudaMemcpyAsync(d, restore.data(), sizeof(PatchEntry) * restore.size(), cudaMemcpyHostToDevice, st));
+        fpsk_status rc2 = patch_launch(C, ldc, d, (int)restore.size(), st);
+        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        if (rc2 != FPSK_OK) return rc2;
+    }
+    if (rc != FPSK_OK) return rc;
+    h_report->m_loc = m_loc;
+    h_report->radius = radius_used;
+
+    // ---- apply: C_ij <- delta for the absolute entries, C_ij <- C_ij + delta for the others
+    std::sort(F.begin(), F.end(), [](const fpsk_fault &x, const fpsk_fault &y) {
+        return x.i != y.i ? x.i < y.i : x.j < y.j;
+    });
+    h_report->n_faults = (int32_t)F.size();
+    const int ncopy = std::min<int>((int)F.size(), capacity);
+    for (int f = 0; f < ncopy; ++f) h_faults[f] = F[f];
+    if ((int)F.size() > kRepairCap) truncated = true;
+    rc = fpsk_apply_corrections(C, ldc, m, n, F.data(), (int)std::min<size_t>(F.size(), kRepairCap), rep_ws,
+                                repair_scratch_bytes(), stream);
+    if (rc != FPSK_OK) return rc;
+
+    // ---- probe once more; if it still fires the caller must recompute the product
+    rc = probe_launch(A, B, C, pd, dtype, q.mu, probe_ws, pws, st, d_res, nullptr);
+    if (rc != FPSK_OK) return rc;
+    FPSK_CUDA_OK(cudaMemcpyAsync(&h_report->second_probe, d_res, sizeof(fpsk_probe_result), cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaStreamSynchronize(st));
+    if (h_report->second_probe.status != FPSK_OK) return (fpsk_status)h_report->second_probe.status;
+    h_report->state = h_report->second_probe.fired ? 2 : 1;
     if ((int)F.size() > capacity || truncated) return FPSK_ERR_CAPACITY;
     return FPSK_OK;
 }

@@ -15,7 +15,7 @@ constexpr int kConfirmThreads = 256;
 template <typename T>
 __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
     const unsigned short *A, long long lda, const unsigned short *B, long long ldb, const float *C, long long ldc,
-    long long n1, long long n2, long long n3, const Candidate *cand, const int *n_cand, int r, double c_valid,
+    long long n1, long long n2, long long n3, const Candidate *cand, const int *n_cand, int r, double c_valid, int force,
     Hit *hits, int *n_hits, int hit_cap)
 {
     __shared__ double sg[kConfirmThreads];
@@ -52,7 +52,7 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
         }
         const float cij = C[i * ldc + j];
         const double tau_ij = c_valid * 1.1920928955078125e-07 * ab;
-        if (fabs(g - (double)cij) > tau_ij) {
+        if (force || fabs(g - (double)cij) > tau_ij) {
             const int slot = atomicAdd(n_hits, 1);
             if (slot < hit_cap) {
                 Hit h;
@@ -65,7 +65,7 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
 }
 
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
-                           int max_cand, int radius, double c_valid, Hit *hits, int *n_hits, int hit_cap,
+                           int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
                            cudaStream_t st)
 {
     if (radius < 0 || 2 * radius + 1 > kConfirmThreads) return FPSK_ERR_PARAM;
@@ -75,10 +75,10 @@ fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate
     const unsigned short *B = static_cast<const unsigned short *>(in.B);
     if (dtype == FPSK_FP16)
         confirm_kernel<__half><<<grid, kConfirmThreads, 0, st>>>(A, in.lda, B, in.ldb, in.C, in.ldc, in.n1, in.n2, in.n3,
-                                                                 cand, n_cand, radius, c_valid, hits, n_hits, hit_cap);
+                                                                 cand, n_cand, radius, c_valid, force, hits, n_hits, hit_cap);
     else
         confirm_kernel<__nv_bfloat16><<<grid, kConfirmThreads, 0, st>>>(A, in.lda, B, in.ldb, in.C, in.ldc, in.n1, in.n2,
-                                                                        in.n3, cand, n_cand, radius, c_valid, hits, n_hits,
+                                                                        in.n3, cand, n_cand, radius, c_valid, force, hits, n_hits,
                                                                         hit_cap);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;

@@ -88,8 +88,27 @@ struct Hit {                // an accepted window entry
     float c_value;
     double gamma;           // FP64 recomputation
 };
+// force != 0: report every in-range window entry, whatever its test says
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
-                           int max_cand, int radius, double c_valid, Hit *hits, int *n_hits, int hit_cap,
+                           int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
                            cudaStream_t st);
+
+// ---- scan / patch / apply (repair.cu) ----------------------------------------------------------
+constexpr int kRepairCap = 4096;      // entries one call can scan out, patch or apply
+struct ScanEntry {
+    int i, j;
+};
+enum { PATCH_SET = 0, PATCH_ADD = 1, PATCH_SET_BITS = 2 };
+struct PatchEntry {
+    int i, j;
+    int mode;          // PATCH_SET: C_ij = value; PATCH_ADD: C_ij += value; PATCH_SET_BITS: raw float bits in value
+    double value;
+};
+size_t repair_scratch_bytes();
+fpsk_status scan_launch(const float *C, long long ldc, long long n1, long long n3, int cap, void *scratch, cudaStream_t st,
+                        ScanEntry *h_entries, int *h_count);
+fpsk_status recompute_entries(const SketchIn &in, fpsk_dtype dtype, const ScanEntry *h_entries, int n, void *scratch,
+                              cudaStream_t st, double *h_gamma, float *h_old);
+fpsk_status patch_launch(float *C, long long ldc, const PatchEntry *d_entries, int n, cudaStream_t st);
 
 }  // namespace fpsk

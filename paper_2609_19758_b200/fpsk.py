@@ -44,6 +44,11 @@ class Noise(C.Structure):
                 ("radius", C.c_int32)]
 
 
+class RepairReport(C.Structure):
+    _fields_ = [("state", C.c_int32), ("n_faults", C.c_int32), ("n_absolute", C.c_int32), ("m_loc", C.c_int32),
+                ("radius", C.c_int32), ("reserved", C.c_int32), ("first_probe", ProbeResult), ("second_probe", ProbeResult)]
+
+
 class FpskError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -101,6 +106,13 @@ def lib() -> C.CDLL:
         L.fpsk_localize.restype = C.c_int
         L.fpsk_localize.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32, C.POINTER(Params),
                                     vp, sz, vp, C.POINTER(Fault), i32, C.POINTER(i32)]
+        L.fpsk_repair_workspace_bytes.restype = sz
+        L.fpsk_repair_workspace_bytes.argtypes = [i64, i64, i64, i32, C.POINTER(Params)]
+        L.fpsk_verify_repair.restype = C.c_int
+        L.fpsk_verify_repair.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32, C.POINTER(Params),
+                                         vp, sz, vp, C.POINTER(Fault), i32, C.POINTER(RepairReport)]
+        L.fpsk_apply_corrections.restype = C.c_int
+        L.fpsk_apply_corrections.argtypes = [vp, i64, i64, i64, C.POINTER(Fault), i32, vp, sz, vp]
         L.fpsk_launch_count.restype = u64
         L.fpsk_launch_count.argtypes = []
         _lib = L
@@ -293,3 +305,35 @@ def localize(A, B, Cm, seed: int, n_buckets: int, ws: torch.Tensor, params: Opti
     if rc != STATUS_OK:
         raise FpskError(rc, "fpsk_localize")
     return [buf[i] for i in range(cnt.value)]
+
+
+def repair_workspace(m: int, k: int, n: int, n_buckets: int = 0, params: Optional[Params] = None, device=None) -> torch.Tensor:
+    nbytes = int(lib().fpsk_repair_workspace_bytes(m, k, n, n_buckets, C.byref(params) if params is not None else None))
+    if nbytes == 0:
+        raise FpskError(ERR_BUCKETS, "fpsk_repair_workspace_bytes")
+    return torch.empty(nbytes, dtype=torch.uint8, device=device or "cuda")
+
+
+def verify_repair(A, B, Cm, seed: int, ws: torch.Tensor, n_buckets: int = 0, params: Optional[Params] = None,
+                  capacity: int = 1024, stream=None):
+    """Algorithm 2 in place on Cm (device FP32): returns (faults, report)."""
+    a = _mat_args(A, B, Cm)
+    assert Cm.dtype == torch.float32
+    buf = (Fault * capacity)()
+    rep = RepairReport()
+    rc = lib().fpsk_verify_repair(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, n_buckets,
+                                  C.byref(params) if params is not None else None, ws.data_ptr(), ws.numel(),
+                                  _stream_ptr(stream), buf, capacity, C.byref(rep))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_verify_repair")
+    return [buf[i] for i in range(min(rep.n_faults, capacity))], rep
+
+
+def apply_corrections(Cm: torch.Tensor, faults, ws: torch.Tensor, stream=None) -> None:
+    n = len(faults)
+    buf = (Fault * max(n, 1))(*faults)
+    m, ncol = Cm.shape
+    rc = lib().fpsk_apply_corrections(Cm.data_ptr(), Cm.stride(0), m, ncol, buf, n, ws.data_ptr(), ws.numel(),
+                                      _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_apply_corrections")
