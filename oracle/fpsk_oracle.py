@@ -42,6 +42,7 @@ __all__ = [
     "c_f", "law_sigma", "m_comb", "m_max", "m_mem", "m_num", "m_start", "cap_K",
     "rms_c_estimate", "index_budget", "radius_from_budget", "plan", "recalibrated_m",
     "measure_noise", "scan_out_of_range", "apply_corrections", "verify_repair", "FP32_MAX",
+    "hashed_sum_sketch", "probe_hashed",
 ]
 
 EPS32 = 2.0 ** -23          # FP32 machine epsilon used by the thresholds (Section "Validation")
@@ -212,6 +213,40 @@ def probe_verdict(s: np.ndarray, tau: float, params: Params = None, n_rows: int 
         arg, mx = -1, 0.0
     fired = bool(nonfinite or (mx > thr))
     return ProbeResult(fired, nonfinite, arg, mx, sig, thr, tau)
+
+
+# ----------------------------------------------------------------------------
+# the paper's own probe: S alone at the probe's bucket count m
+# (Section "The Cheap S Only Probe", Eq. (S), Section "Thresholds")
+# ----------------------------------------------------------------------------
+def hashed_sum_sketch(E, h1, v1, h2, v2, m_b: int) -> np.ndarray:
+    """S = H1 E H2^T, entry by entry from the definition (no R, no T)."""
+    E = np.asarray(E, dtype=np.float64)
+    flat = (np.asarray(h1, dtype=np.int64)[:, None] * m_b + np.asarray(h2, dtype=np.int64)[None, :]).ravel()
+    sE = (np.asarray(v1)[:, None] * np.asarray(v2)[None, :]) * E
+    with np.errstate(invalid="ignore"):
+        return np.bincount(flat, weights=sE.ravel(), minlength=m_b * m_b).reshape(m_b, m_b)
+
+
+def probe_hashed(A, B, C, seed: int, rnd: int, m_b: int, params: Params = None):
+    """The S only probe: hash round (seed, rnd) with m_b buckets per side, S = H1 (AB - C) H2^T,
+    sigma_hat = clipped mean over the m_b^2 buckets, thr = min(cap, mu sqrt(2 ln m_b^2) sigma_hat),
+    dirty iff max|S| > thr or S is not finite.  The analytic cap enters as tau sqrt(n1 n3 / m_b^2):
+    tau bounds one inner product's rounding and a bucket sums n1 n3 / m_b^2 of them on average
+    (the reading taken for the un-hashed sketch, applied to the bucket population).
+    Returns (ProbeResult with argmax_col = flat bucket index a*m_b + b, S)."""
+    params = params or Params()
+    A64, B64 = _f64(A), _f64(B)
+    n1, n2 = A64.shape
+    n3 = B64.shape[1]
+    h1, v1 = hash_round(seed, rnd, 0, n1, m_b)
+    h2, v2 = hash_round(seed, rnd, 1, n3, m_b)
+    with np.errstate(invalid="ignore", over="ignore"):
+        E = A64 @ B64 - np.asarray(C, dtype=np.float64)
+    S = hashed_sum_sketch(E, h1, v1, h2, v2, m_b)
+    tau = analytic_tau(A64, B64, n2)
+    pop = float(n1) * float(n3) / (float(m_b) * float(m_b))
+    return probe_verdict(S.ravel(), tau, params, n_rows=pop), S
 
 
 # ----------------------------------------------------------------------------
