@@ -183,6 +183,56 @@ fpsk_status fpsk_probe_static(const void *A, int64_t lda, const void *B, int64_t
                               fpsk_dtype dtype, int c_is_fp32, const fpsk_params *p, void *stream,
                               fpsk_probe_result *d_result, float *d_residual);
 
+/* ---- the paper's own probe: S alone, B side cached ------------------------------------------ */
+
+/* Host-side record of a cached B side (Section "Implementation": the sketch of the B side is
+ * cached and keyed on tensor identity and version, so an in-place optimizer update invalidates
+ * it).  Zero-initialise it once (valid = 0); fpsk_probe_hashed fills and checks it.  The key is
+ * (B pointer, ldb, b_version, shape, dtype, seed, round, n_buckets, cache pointer). */
+typedef struct {
+    const void *B;
+    void *cache;
+    int64_t ldb, m, k, n;
+    uint64_t seed, version;
+    int32_t dtype, n_buckets, round;
+    int32_t valid;        /* 0: nothing cached                                                 */
+    int32_t rebuilds;     /* how many times the B side was (re)built through this record       */
+    int32_t reserved;
+} fpsk_bside;
+
+/* Bytes of device memory for the cached B side (hash tables and bucket-sorted permutations of
+ * rows and columns, Q = B H2^T as k x n_buckets FP32, max|B|) and for the per-call workspace
+ * (P = H1 A, H1 C, split-K partials, S).  0 on bad arguments. */
+size_t fpsk_probe_hashed_cache_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets);
+size_t fpsk_probe_hashed_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets);
+
+/* 1 when `side` already holds the B side for exactly this key (the call would read A and C only),
+ * else 0.  Host only. */
+int32_t fpsk_bside_matches(const fpsk_bside *side, const void *B, int64_t ldb, uint64_t b_version,
+                           int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed,
+                           int32_t round, int32_t n_buckets, const void *cache);
+
+/* The S only probe (Section "The Cheap S Only Probe"): S = (H1 A)(B H2^T) - H1 C H2^T for hash
+ * round `round` of `seed` at n_buckets buckets per side, sigma_hat = 1.2533 mean(min(|S|, 5 mean|S|))
+ * over the n_buckets^2 buckets, thr = min(tau sqrt(m n / n_buckets^2), mu sqrt(2 ln n_buckets^2) sigma_hat)
+ * (Section "Thresholds"; a bucket sums m n / n_buckets^2 entries of E on average, so the analytic
+ * cap enters with the root of that population), dirty iff max|S| > thr or S is not finite.
+ *   side, cache   the B side.  When `side` does not match the key (see fpsk_bside), it is rebuilt
+ *                 into `cache` first (reads B once; side->rebuilds is incremented); on a match B
+ *                 is not read: the call reads 2mk + 4mn bytes.  Bump b_version after every in-place
+ *                 change of B.
+ *   workspace     per-call scratch; its first 256 bytes must be zero before the first call
+ *                 (fpsk_probe_init does that) and again after a result with status FPSK_ERR_TIMEOUT
+ *   d_result      device; argmax_col holds the flat bucket index a * n_buckets + b
+ *   d_S           device, n_buckets^2 floats receiving S, or NULL
+ * sigma_hat is the noise at this bucket count and feeds fpsk_plan directly.
+ * Asynchronous on `stream`, no host synchronisation; deterministic. */
+fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, const void *B, int64_t ldb,
+                              uint64_t b_version, const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                              fpsk_dtype dtype, int c_is_fp32, uint64_t seed, int32_t round, int32_t n_buckets,
+                              const fpsk_params *p, void *cache, size_t cache_bytes, void *workspace,
+                              size_t ws_bytes, void *stream, fpsk_probe_result *d_result, float *d_S);
+
 /* ---- hashed moment sketches --------------------------------------------------------------- */
 
 /* Hash round `round` of `seed` (Section "Moment Sketches": h1, v1 for side 0 = rows,

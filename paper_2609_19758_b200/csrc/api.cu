@@ -386,6 +386,60 @@ fpsk_status fpsk_probe_host(const void *hA, const void *hB, const float *hC, int
 }
 
 // ---------------------------------------------------------------- sketches
+// ---------------------------------------------------------------- S only probe, cached B side
+size_t fpsk_probe_hashed_cache_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets)
+{
+    if (m < 1 || k < 1 || n < 1 || n_buckets < 1 || n_buckets > 4096) return 0;
+    if (m >= (1LL << 30) || k >= (1LL << 30) || n >= (1LL << 30)) return 0;
+    return hprobe_cache_bytes(m, k, n, n_buckets);
+}
+
+size_t fpsk_probe_hashed_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets)
+{
+    if (m < 1 || k < 1 || n < 1 || n_buckets < 1 || n_buckets > 4096) return 0;
+    if (m >= (1LL << 30) || k >= (1LL << 30) || n >= (1LL << 30)) return 0;
+    return hprobe_ws_bytes(m, k, n, n_buckets);
+}
+
+int32_t fpsk_bside_matches(const fpsk_bside *side, const void *B, int64_t ldb, uint64_t b_version, int64_t m,
+                           int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t round, int32_t n_buckets,
+                           const void *cache)
+{
+    if (!side || !side->valid) return 0;
+    return side->B == B && side->cache == cache && side->ldb == ldb && side->version == b_version && side->m == m &&
+                   side->k == k && side->n == n && side->dtype == (int32_t)dtype && side->seed == seed &&
+                   side->round == round && side->n_buckets == n_buckets
+               ? 1 : 0;
+}
+
+fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, const void *B, int64_t ldb,
+                              uint64_t b_version, const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
+                              fpsk_dtype dtype, int c_is_fp32, uint64_t seed, int32_t round, int32_t n_buckets,
+                              const fpsk_params *p, void *cache, size_t cache_bytes, void *workspace, size_t ws_bytes,
+                              void *stream, fpsk_probe_result *d_result, float *d_S)
+{
+    if (!c_is_fp32) return FPSK_ERR_DTYPE;      // a narrowed C is rejected, not tolerated
+    if (!side || !cache || !workspace || !d_result) return FPSK_ERR_NULL;
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    if (rc != FPSK_OK) return rc;
+    if (n_buckets < 1 || n_buckets > 4096 || round < 0) return FPSK_ERR_BUCKETS;
+    if ((reinterpret_cast<uintptr_t>(cache) & 255) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return FPSK_ERR_ALIGN;
+    if (cache_bytes < hprobe_cache_bytes(m, k, n, n_buckets) || ws_bytes < hprobe_ws_bytes(m, k, n, n_buckets))
+        return FPSK_ERR_WORKSPACE;
+    const fpsk_params q = resolve_params(p);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!fpsk_bside_matches(side, B, ldb, b_version, m, k, n, dtype, seed, round, n_buckets, cache)) {
+        side->valid = 0;
+        rc = hprobe_prepare(B, ldb, m, k, n, dtype, seed, round, n_buckets, cache, cache_bytes, st);
+        if (rc != FPSK_OK) return rc;
+        side->B = B; side->cache = cache; side->ldb = ldb; side->m = m; side->k = k; side->n = n;
+        side->seed = seed; side->version = b_version; side->dtype = (int32_t)dtype; side->n_buckets = n_buckets;
+        side->round = round; side->valid = 1; side->rebuilds += 1;
+    }
+    return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, cache, cache_bytes, workspace, ws_bytes, st,
+                         d_result, d_S);
+}
+
 fpsk_status fpsk_hash_tables(uint64_t seed, int32_t round, int32_t side, int64_t count, int32_t n_buckets,
                              int32_t *d_bucket, int32_t *d_sign, void *stream)
 {

@@ -1,0 +1,656 @@
+// The S only probe at the probe's own bucket count (Section "The Cheap S Only Probe"):
+//   S = (H1 A)(B H2^T) - H1 C H2^T,   sigma_hat, threshold and one-bit verdict (Section "Thresholds").
+// The B side (hash round, bucket-sorted permutations, Q = B H2^T, max|B|) is built once per weight
+// tensor and kept by the caller; a call on a cached B reads A once and C once.
+//
+//   hp_partition_kernel     balanced split of the (matrix, column segment, row bucket) units over CTAs
+//   hp_stream_kernel        P = H1 A (m x n2) and Tc = H1 C (m x n3): signed row-bucket sums, one
+//                           persistent CTA per SM, rows gathered by bulk copies into a shared-memory ring
+//   hp_rowsum_plain_kernel  the same sums with plain loads (inputs that bulk copies cannot address)
+//   sgemm (sketch.cu)       P Q as split-K partials, FP32 FMA
+//   hp_verdict_kernel       S = sum of partials - Tc H2^T (column fold), statistics, verdict
+// Every sum has a fixed order (no float atomics): results are bit-reproducible.
+#include "sketch.cuh"
+#include "stream_pipe.cuh"
+
+#include <math.h>
+#include <stdlib.h>
+#include <mutex>
+#include <type_traits>
+
+namespace fpsk {
+
+constexpr int kHpConsumers = 512;
+constexpr int kHpThreads = kHpConsumers + 32;     // + producer warp
+constexpr int kHpStages = 6;
+constexpr int kHpStageBytes = 32768;
+constexpr int kHpPieceBytes = 4096;               // one row of one column segment
+constexpr int kHpPieces = kHpStageBytes / kHpPieceBytes;
+constexpr int kHpSegA = kHpPieceBytes / 2;        // columns of A per segment
+constexpr int kHpSegC = kHpPieceBytes / 4;        // columns of C per segment
+constexpr int kHpRedBytes = 256 * 32;             // lane-combine scratch: 256 threads x 8 floats
+constexpr int kHpSmem = kHpStages * kHpStageBytes + kHpRedBytes + 256 /*barriers*/ + kHpStages * 16 /*stage records*/;
+
+struct HpArgs {
+    const unsigned short *A;
+    long long lda;
+    const float *C;
+    long long ldc;
+    int n1, n2, n3, m, kpad;
+    int segsA, segsC;              // column segments of A and of C
+    const uint32_t *rowperm;       // rows sorted by bucket; bit 31 = sign -1
+    const int *rowstart;           // [m + 1]
+    const int *first_unit;         // [grid + 1]
+    float *P;                      // m x kpad
+    float *Tc;                     // m x n3
+    unsigned int *maxA;            // per CTA: bits of max|A| over what it streamed
+    unsigned int *ctrl;            // [0] verdict ticket, [1] error flag
+};
+
+// cumulative bytes streamed before unit u, with units ordered (matrix, segment, bucket)
+__device__ __forceinline__ long long hp_unit_start(const HpArgs &p, int u)
+{
+    const int UA = p.m * p.segsA, U = UA + p.m * p.segsC;
+    if (u >= U) return 2LL * p.n1 * p.n2 + 4LL * p.n1 * p.n3;
+    if (u < UA) {
+        const int s = u / p.m, a = u - s * p.m;
+        const int w = min(kHpSegA, p.n2 - s * kHpSegA);
+        return 2LL * p.n1 * ((long long)s * kHpSegA) + 2LL * __ldg(p.rowstart + a) * w;
+    }
+    const int v = u - UA;
+    const int s = v / p.m, a = v - s * p.m;
+    const int w = min(kHpSegC, p.n3 - s * kHpSegC);
+    return 2LL * p.n1 * p.n2 + 4LL * p.n1 * ((long long)s * kHpSegC) + 4LL * __ldg(p.rowstart + a) * w;
+}
+
+// first_unit[c] = smallest unit whose start is >= c W / grid  (W = all bytes); first_unit[grid] = U
+__global__ void hp_partition_kernel(HpArgs p, int grid, int *first_unit)
+{
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c > grid) return;
+    const int U = p.m * (p.segsA + p.segsC);
+    if (c == grid) { first_unit[c] = U; return; }
+    const long long W = 2LL * p.n1 * p.n2 + 4LL * p.n1 * p.n3;
+    const long long target = (W / grid) * c + (W % grid) * c / grid;
+    int lo = 0, hi = U;                 // smallest u in [0, U] with start(u) >= target
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (hp_unit_start(p, mid) >= target) hi = mid; else lo = mid + 1;
+    }
+    first_unit[c] = lo;
+}
+
+struct HpStageRec {     // what the producer tells the consumers about one stage
+    int unit;           // -1: no more work
+    int info;           // pieces | last << 8 | sign bits << 16
+    int pad0, pad1;
+};
+
+// Barrier over the consumer warps on an mbarrier (one arrival per warp), so that this wait is
+// bounded like every other wait of the kernel.  Returns false when it gave up.
+__device__ __forceinline__ bool hp_consumer_sync(uint32_t cbar, uint32_t &cpar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(cbar);
+    const bool w = mbar_wait_warp(cbar, cpar);
+    cpar ^= 1u;
+    return w;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    unsigned char *ring = smem;
+    float4 *red4 = reinterpret_cast<float4 *>(smem + kHpStages * kHpStageBytes);
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + kHpStages * kHpStageBytes + kHpRedBytes);
+    HpStageRec *recs = reinterpret_cast<HpStageRec *>(smem + kHpStages * kHpStageBytes + kHpRedBytes + 256);
+    __shared__ unsigned int smx[kHpConsumers / 32];
+    const int c = blockIdx.x;
+    const int tid = threadIdx.x;
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kHpStages), cbar = smem_u32(bars + 2 * kHpStages);
+    if (tid == 0) {
+        for (int s = 0; s < kHpStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, kHpConsumers / 32);
+        }
+        mbar_init(cbar, kHpConsumers / 32);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    __syncthreads();
+    const int UA = p.m * p.segsA;
+    const int u0 = __ldg(p.first_unit + c), u1 = __ldg(p.first_unit + c + 1);
+
+    if (tid >= kHpConsumers) {
+        // ------------------------------------------------------------ producer warp
+        const int lane = tid - kHpConsumers;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        for (int u = u0; u < u1 && ok; ++u) {
+            const bool isC = u >= UA;
+            const int v = isC ? u - UA : u;
+            const int seg = v / p.m, a = v - seg * p.m;
+            const int s0 = __ldg(p.rowstart + a), s1 = __ldg(p.rowstart + a + 1);
+            const int wbytes = isC ? 4 * min(kHpSegC, p.n3 - seg * kHpSegC) : 2 * min(kHpSegA, p.n2 - seg * kHpSegA);
+            const unsigned char *base = isC ? reinterpret_cast<const unsigned char *>(p.C + (long long)seg * kHpSegC)
+                                            : reinterpret_cast<const unsigned char *>(p.A + (long long)seg * kHpSegA);
+            const long long ldb = isC ? p.ldc * 4 : p.lda * 2;
+            int pos = s0;
+            do {
+                const int np = min(kHpPieces, s1 - pos);
+                const bool last = pos + np >= s1;
+                uint32_t e = 0;
+                if (lane < np) e = __ldg(p.rowperm + pos + lane);
+                int w = 1;
+                if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                if (!w) { ok = false; break; }
+                const unsigned int signs = __ballot_sync(0xFFFFFFFFu, lane < np && (e >> 31));
+                if (lane == 0) {
+                    HpStageRec r;
+                    r.unit = u;
+                    r.info = np | (last ? 0x100 : 0) | (int)(signs << 16);
+                    r.pad0 = r.pad1 = 0;
+                    recs[stage] = r;
+                    if (np > 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)np * (uint32_t)wbytes);
+                    else mbar_arrive(full0 + 8 * stage);
+                }
+                __syncwarp();
+                if (lane < np)
+                    bulk_g2s(smem_u32(ring + (size_t)stage * kHpStageBytes) + (uint32_t)lane * kHpPieceBytes,
+                             base + (long long)(e & 0x7FFFFFFFu) * ldb, (uint32_t)wbytes, full0 + 8 * stage);
+                if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
+                pos += np;
+            } while (pos < s1);
+        }
+        if (ok) {
+            // end of work: one empty stage with unit = -1
+            int w = 1;
+            if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+            w = __shfl_sync(0xFFFFFFFFu, w, 0);
+            if (w) {
+                if (lane == 0) {
+                    HpStageRec r;
+                    r.unit = -1; r.info = 0; r.pad0 = r.pad1 = 0;
+                    recs[stage] = r;
+                    mbar_arrive(full0 + 8 * stage);
+                }
+            } else ok = false;
+        }
+        if (!ok && lane == 0) atomicOr(p.ctrl + 1, 1u);
+    } else {
+        // ------------------------------------------------------------ consumer warps
+        const int ctid = tid;
+        const int tc = ctid & 255, rl = ctid >> 8;     // 256 x 16 B across a piece; two row lanes
+        int stage = 0;
+        uint32_t phase = 0, cpar = 0;
+        bool ok = true;
+        float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
+        MinMax2<T> mm;
+        mm.init();
+        for (;;) {
+            if (!mbar_wait_warp(full0 + 8 * stage, phase)) { ok = false; break; }
+            const HpStageRec r = recs[stage];
+            if (r.unit < 0) break;
+            const int u = r.unit;
+            const int np = r.info & 0xFF;
+            const bool last = (r.info & 0x100) != 0;
+            const unsigned int signs = ((unsigned int)r.info) >> 16;
+            const bool isC = u >= UA;
+            const int v = isC ? u - UA : u;
+            const int seg = v / p.m, a = v - seg * p.m;
+            const int wbytes = isC ? 4 * min(kHpSegC, p.n3 - seg * kHpSegC) : 2 * min(kHpSegA, p.n2 - seg * kHpSegA);
+            const bool active = tc * 16 < wbytes;
+            if (active) {
+                const unsigned char *sb = ring + (size_t)stage * kHpStageBytes + tc * 16;
+                if (isC) {
+#pragma unroll
+                    for (int q = rl; q < kHpPieces; q += 2) {
+                        if (q < np) {
+                            const float4 x = *reinterpret_cast<const float4 *>(sb + q * kHpPieceBytes);
+                            const float sg = ((signs >> q) & 1u) ? -1.f : 1.f;
+                            acc[0] = __ffma2_rn(make_float2(sg, sg), make_float2(x.x, x.y), acc[0]);
+                            acc[1] = __ffma2_rn(make_float2(sg, sg), make_float2(x.z, x.w), acc[1]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int q = rl; q < kHpPieces; q += 2) {
+                        if (q < np) {
+                            uint4 x = *reinterpret_cast<const uint4 *>(sb + q * kHpPieceBytes);
+                            const uint32_t flip = ((signs >> q) & 1u) ? 0x80008000u : 0u;
+                            x.x ^= flip; x.y ^= flip; x.z ^= flip; x.w ^= flip;
+                            add8m<T>(acc, x, mm);
+                        }
+                    }
+                }
+            }
+            __syncwarp();
+            if ((ctid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
+            if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
+            if (last) {
+                // unit complete: row lane 1 hands its sums to row lane 0, which stores the row segment
+                if (!hp_consumer_sync(cbar, cpar)) { ok = false; break; }
+                if (rl == 1) {
+                    red4[tc * 2] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+                    red4[tc * 2 + 1] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
+                }
+                if (!hp_consumer_sync(cbar, cpar)) { ok = false; break; }
+                if (rl == 0) {
+                    if (isC) {
+                        if (active) {
+                            const float4 y = red4[tc * 2];
+                            __stcg(reinterpret_cast<float4 *>(p.Tc + (long long)a * p.n3 + seg * kHpSegC + tc * 4),
+                                   make_float4(acc[0].x + y.x, acc[0].y + y.y, acc[1].x + y.z, acc[1].y + y.w));
+                        }
+                    } else {
+                        const int col = seg * kHpSegA + tc * 8;
+                        if (active) {
+                            const float4 y0 = red4[tc * 2], y1 = red4[tc * 2 + 1];
+                            float4 *dst = reinterpret_cast<float4 *>(p.P + (long long)a * p.kpad + col);
+                            __stcg(dst, make_float4(acc[0].x + y0.x, acc[0].y + y0.y, acc[1].x + y0.z, acc[1].y + y0.w));
+                            __stcg(dst + 1, make_float4(acc[2].x + y1.x, acc[2].y + y1.y, acc[3].x + y1.z, acc[3].y + y1.w));
+                        } else if (col < p.kpad) {
+                            // padding columns of the contraction's K extent
+                            float4 *dst = reinterpret_cast<float4 *>(p.P + (long long)a * p.kpad + col);
+                            __stcg(dst, make_float4(0.f, 0.f, 0.f, 0.f));
+                            __stcg(dst + 1, make_float4(0.f, 0.f, 0.f, 0.f));
+                        }
+                    }
+                }
+                acc[0] = acc[1] = acc[2] = acc[3] = make_float2(0.f, 0.f);
+            }
+        }
+        // max|A| over what this CTA streamed (for tau)
+        unsigned int mbits = float_to_bits16<T>(mm.absmax());
+        mbits = __reduce_max_sync(0xFFFFFFFFu, mbits);
+        if ((ctid & 31) == 0) {
+            smx[ctid >> 5] = mbits;
+            if (!ok) atomicOr(p.ctrl + 1, 1u);
+        }
+        if (ok && hp_consumer_sync(cbar, cpar) && ctid == 0) {
+            unsigned int r_ = 0;
+            for (int w = 0; w < kHpConsumers / 32; ++w) r_ = max(r_, smx[w]);
+            p.maxA[c] = r_;
+        }
+    }
+}
+
+// The same signed row-bucket sums with plain loads, for inputs the bulk copies cannot address
+// (base not 16-byte aligned, leading dimension or width not a multiple of 16 bytes).
+// Thread (bucket a, column): rows of the bucket in ascending row order.
+template <typename T>
+__global__ void __launch_bounds__(256) hp_rowsum_plain_kernel(const HpArgs p)
+{
+    const int a = blockIdx.y;
+    const int col = blockIdx.x * blockDim.x + threadIdx.x;
+    const int s0 = __ldg(p.rowstart + a), s1 = __ldg(p.rowstart + a + 1);
+    if (blockIdx.z == 0) {
+        if (col >= p.kpad) return;
+        constexpr unsigned int kInf = std::is_same<T, __half>::value ? 0x7C00u : 0x7F80u;
+        float acc = 0.f;
+        unsigned int mx = 0;
+        if (col < p.n2) {
+            for (int s = s0; s < s1; ++s) {
+                const uint32_t e = __ldg(p.rowperm + s);
+                const unsigned short h = p.A[(long long)(e & 0x7FFFFFFFu) * p.lda + col];
+                const float x = bits16_to_float<T>(h);
+                acc += (e >> 31) ? -x : x;
+                const unsigned int mag = h & 0x7FFFu;       // |x| of a 16-bit float orders like its bit pattern
+                if (mag <= kInf) mx = max(mx, mag);         // NaN operands are ignored, as in the streaming path
+            }
+        }
+        p.P[(long long)a * p.kpad + col] = acc;
+        mx = __reduce_max_sync(0xFFFFFFFFu, mx);
+        if ((threadIdx.x & 31) == 0 && mx) atomicMax(p.maxA, mx);
+    } else {
+        if (col >= p.n3) return;
+        float acc = 0.f;
+        for (int s = s0; s < s1; ++s) {
+            const uint32_t e = __ldg(p.rowperm + s);
+            const float x = p.C[(long long)(e & 0x7FFFFFFFu) * p.ldc + col];
+            acc += (e >> 31) ? -x : x;
+        }
+        p.Tc[(long long)a * p.n3 + col] = acc;
+    }
+}
+
+// ---------------------------------------------------------------- combine + verdict
+struct HvArgs {
+    const float *partAB;     // [ksplit][m*m]
+    int ksplit;
+    const float *Tc;         // m x n3
+    const uint32_t *colperm; // columns sorted by bucket; bit 31 = sign -1
+    const int *colstart;     // [m + 1]
+    int m, n1, n2, n3;
+    const unsigned int *maxA;
+    int n_maxA;
+    const float *maxB;           // [1] max|B|
+    float thr_scale;         // mu sqrt(2 ln max(m^2, 2))
+    float cap_scale;         // sqrt(n1 n3 / m^2)
+    float *S;                // m*m
+    float4 *vstat;           // per CTA: sum|S|, nonfinite count, max, argmax (as int bits)
+    unsigned int *ctrl;      // [0] ticket, [1] error flag
+    fpsk_probe_result *result;
+};
+
+struct HvMax {
+    float v;
+    int i;
+};
+__device__ __forceinline__ HvMax hv_better(HvMax a, HvMax b)
+{
+    if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
+    return a;
+}
+
+// CTA a computes row a of S.  The last CTA to finish (ticket) combines the per-row statistics in row
+// order and writes the verdict; when some bucket exceeds the clip level it makes the second pass
+// over S alone (fixed order).
+template <typename T>
+__global__ void __launch_bounds__(256) hp_verdict_kernel(const HvArgs p)
+{
+    __shared__ float ssum[256], sbad[256];
+    __shared__ HvMax smax[256];
+    __shared__ int s_last;
+    const int a = blockIdx.x, tid = threadIdx.x;
+    const long long mm = (long long)p.m * p.m;
+    float lsum = 0.f, lbad = 0.f;
+    HvMax lmax = {-1.f, 0x7FFFFFFF};
+    const float *trow = p.Tc + (long long)a * p.n3;
+    for (int b = tid; b < p.m; b += 256) {
+        const long long idx = (long long)a * p.m + b;
+        float ab = __ldcg(p.partAB + idx);
+        for (int s = 1; s < p.ksplit; ++s) ab += __ldcg(p.partAB + (long long)s * mm + idx);
+        float cf = 0.f;
+        const int c0 = __ldg(p.colstart + b), c1 = __ldg(p.colstart + b + 1);
+        for (int s = c0; s < c1; ++s) {
+            const uint32_t e = __ldg(p.colperm + s);
+            const float x = __ldcg(trow + (e & 0x7FFFFFFFu));
+            cf += (e >> 31) ? -x : x;
+        }
+        const float sv = ab - cf;
+        p.S[idx] = sv;
+        const float av = fabsf(sv);
+        lsum += av;
+        if (!(av <= 3.4028234663852886e38f)) lbad += 1.f;          // Inf or NaN
+        else lmax = hv_better(lmax, HvMax{av, (int)idx});
+    }
+    ssum[tid] = lsum; sbad[tid] = lbad; smax[tid] = lmax;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (tid < o) {
+            ssum[tid] += ssum[tid + o];
+            sbad[tid] += sbad[tid + o];
+            smax[tid] = hv_better(smax[tid], smax[tid + o]);
+        }
+        __syncthreads();
+    }
+    if (tid == 0) {
+        p.vstat[a] = make_float4(ssum[0], sbad[0], smax[0].v, __int_as_float(smax[0].i));
+        __threadfence();
+        const unsigned int t = atom_acq_rel_add(p.ctrl + 0);
+        s_last = (t == (unsigned int)(gridDim.x - 1)) ? 1 : 0;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    // ---- last CTA: statistics in row order
+    float tsum = 0.f, tbad = 0.f;
+    HvMax tmax = {-1.f, 0x7FFFFFFF};
+    unsigned int ma = 0;
+    if (tid == 0) {
+        for (int r = 0; r < p.m; ++r) {
+            const float4 v = __ldcg(p.vstat + r);
+            tsum += v.x;
+            tbad += v.y;
+            tmax = hv_better(tmax, HvMax{v.z, __float_as_int(v.w)});
+        }
+        ssum[0] = tsum; sbad[0] = tbad; smax[0] = tmax;
+    }
+    for (int r = tid; r < p.n_maxA; r += 256) ma = max(ma, __ldcg(p.maxA + r));
+    __syncthreads();
+    tsum = ssum[0]; tbad = sbad[0]; tmax = smax[0];
+    __syncthreads();
+    // max|A| across the per-CTA records
+    {
+        unsigned int *um = reinterpret_cast<unsigned int *>(ssum);
+        um[tid] = ma;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if (tid < o) um[tid] = max(um[tid], um[tid + o]);
+            __syncthreads();
+        }
+        ma = um[0];
+        __syncthreads();
+    }
+    const float mean = tsum / (float)mm;
+    float clipped = tsum;
+    if (!(tmax.v <= 5.f * mean) || tbad > 0.f) {
+        // second pass: sum of min(|S|, 5 mean|S|), thread-strided then tree (fixed order)
+        const float clip = 5.f * mean;
+        float cs = 0.f;
+        for (long long i = tid; i < mm; i += 256) cs += fminf(fabsf(__ldcg(p.S + i)), clip);
+        ssum[tid] = cs;
+        __syncthreads();
+        for (int o = 128; o > 0; o >>= 1) {
+            if (tid < o) ssum[tid] += ssum[tid + o];
+            __syncthreads();
+        }
+        clipped = ssum[0];
+    }
+    if (tid == 0) {
+        const float sigma = 1.2533f * (clipped / (float)mm);
+        const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) *
+                          __ldcg(p.maxB);
+        // a bucket sums n1 n3 / m^2 entries of E on average: the per-entry cap grows like the root of that
+        const float thr = fminf(tau * p.cap_scale, p.thr_scale * sigma);
+        fpsk_probe_result r;
+        r.nonfinite = tbad > 0.f ? 1 : 0;
+        r.fired = (tbad > 0.f || tmax.v > thr) ? 1 : 0;
+        r.argmax_col = tmax.v >= 0.f ? tmax.i : -1;
+        r.status = __ldcg(p.ctrl + 1) ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK;
+        r.max_abs = tmax.v >= 0.f ? tmax.v : 0.f;
+        r.sigma_hat = sigma;
+        r.thr = thr;
+        r.tau = tau;
+        *p.result = r;
+        p.ctrl[0] = 0;          // ticket and error flag ready for the next call on this workspace
+        p.ctrl[1] = 0;
+    }
+}
+
+// ---------------------------------------------------------------- host side
+struct HpPlan {
+    int kpad, npad, segsA, segsC, tile, ksplit, kchunk;
+};
+
+static void hp_plan(long long n2, long long n3, int m, int sms, HpPlan &pl)
+{
+    pl.kpad = (int)((n2 + 15) / 16 * 16);
+    pl.npad = (m + 3) / 4 * 4;
+    pl.segsA = (int)((n2 + kHpSegA - 1) / kHpSegA);
+    pl.segsC = (int)((n3 + kHpSegC - 1) / kHpSegC);
+    pl.tile = m <= 512 ? 64 : 128;
+    const int t1 = (m + pl.tile - 1) / pl.tile;
+    const int tiles = t1 * t1;
+    int ks = (2 * sms + tiles - 1) / tiles;                     // two resident CTAs per SM
+    const int maxks = pl.kpad / 128 > 1 ? pl.kpad / 128 : 1;    // at least 128 of K per split
+    if (ks > maxks) ks = maxks;
+    if (ks > 64) ks = 64;
+    if (ks < 1) ks = 1;
+    int kchunk = ((pl.kpad + ks - 1) / ks + 15) / 16 * 16;
+    pl.ksplit = (pl.kpad + kchunk - 1) / kchunk;
+    pl.kchunk = kchunk;
+}
+
+struct HpCache {          // the B side, device memory kept by the caller across calls
+    int *h1, *v1, *rowcount, *rowstart;
+    uint32_t *rowperm;
+    int *h2, *v2, *colcount, *colstart;
+    uint32_t *colperm;
+    int *first_unit;
+    float *Q;
+    float *maxB;          // [0] max|B|
+    unsigned int *scratch;
+};
+
+static size_t hp_cache_layout(void *base, long long n1, long long n2, long long n3, int m, int sms, HpCache *c)
+{
+    HpPlan pl;
+    hp_plan(n2, n3, m, sms, pl);
+    char *p = static_cast<char *>(base);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { void *r = p ? p + off : nullptr; off += align_up(bytes, 256); return r; };
+    HpCache t;
+    t.h1 = (int *)take((size_t)n1 * 4); t.v1 = (int *)take((size_t)n1 * 4); t.rowperm = (uint32_t *)take((size_t)n1 * 4);
+    t.rowcount = (int *)take((size_t)(m + 1) * 4); t.rowstart = (int *)take((size_t)(m + 1) * 4);
+    t.h2 = (int *)take((size_t)n3 * 4); t.v2 = (int *)take((size_t)n3 * 4); t.colperm = (uint32_t *)take((size_t)n3 * 4);
+    t.colcount = (int *)take((size_t)(m + 1) * 4); t.colstart = (int *)take((size_t)(m + 1) * 4);
+    t.first_unit = (int *)take((size_t)(sms + 1) * 4);
+    t.Q = (float *)take((size_t)pl.kpad * pl.npad * 4);
+    t.maxB = (float *)take(256);
+    t.scratch = (unsigned int *)take(256);
+    if (c) *c = t;
+    return off;
+}
+
+struct HpWork {           // per-call scratch
+    unsigned int *ctrl;   // first 256 bytes: zero before the first call (fpsk_probe_init)
+    unsigned int *maxA;
+    float4 *vstat;
+    float *P, *Tc, *partAB, *S;
+};
+
+static size_t hp_work_layout(void *base, long long n1, long long n2, long long n3, int m, int sms, HpWork *w)
+{
+    HpPlan pl;
+    hp_plan(n2, n3, m, sms, pl);
+    char *p = static_cast<char *>(base);
+    size_t off = 0;
+    auto take = [&](size_t bytes) { void *r = p ? p + off : nullptr; off += align_up(bytes, 256); return r; };
+    HpWork t;
+    t.ctrl = (unsigned int *)take(256);
+    t.maxA = (unsigned int *)take((size_t)(sms > 1 ? sms : 1) * 4);
+    t.vstat = (float4 *)take((size_t)m * 16);
+    t.P = (float *)take((size_t)m * pl.kpad * 4);
+    t.Tc = (float *)take((size_t)m * n3 * 4);
+    t.partAB = (float *)take((size_t)pl.ksplit * m * m * 4);
+    t.S = (float *)take((size_t)m * m * 4);
+    if (w) *w = t;
+    return off;
+}
+
+static int hp_sm_count()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
+    return sms;
+}
+
+size_t hprobe_cache_bytes(long long n1, long long n2, long long n3, int m)
+{
+    return hp_cache_layout(nullptr, n1, n2, n3, m, hp_sm_count(), nullptr);
+}
+
+size_t hprobe_ws_bytes(long long n1, long long n2, long long n3, int m)
+{
+    return hp_work_layout(nullptr, n1, n2, n3, m, hp_sm_count(), nullptr);
+}
+
+static HpArgs hp_args(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2, long long n3,
+                      int m, const HpPlan &pl, const HpCache &c, const HpWork *w)
+{
+    HpArgs a;
+    a.A = static_cast<const unsigned short *>(A); a.lda = lda;
+    a.C = C; a.ldc = ldc;
+    a.n1 = (int)n1; a.n2 = (int)n2; a.n3 = (int)n3; a.m = m; a.kpad = pl.kpad;
+    a.segsA = pl.segsA; a.segsC = pl.segsC;
+    a.rowperm = c.rowperm; a.rowstart = c.rowstart; a.first_unit = c.first_unit;
+    a.P = w ? w->P : nullptr; a.Tc = w ? w->Tc : nullptr;
+    a.maxA = w ? w->maxA : nullptr; a.ctrl = w ? w->ctrl : nullptr;
+    return a;
+}
+
+// Build the B side: both hash tables of the round, Q = B H2^T, max|B| and the unit partition.
+fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long n2, long long n3, fpsk_dtype dtype,
+                           uint64_t seed, int rnd, int m, void *cache, size_t cache_bytes, cudaStream_t st)
+{
+    const int sms = hp_sm_count();
+    HpCache c;
+    if (cache_bytes < hp_cache_layout(cache, n1, n2, n3, m, sms, &c)) return FPSK_ERR_WORKSPACE;
+    HpPlan pl;
+    hp_plan(n2, n3, m, sms, pl);
+    fpsk_status rc = build_hash_side(seed, rnd, 0, (int)n1, m, c.h1, c.v1, c.rowcount, c.rowstart, c.rowperm, st);
+    if (rc != FPSK_OK) return rc;
+    rc = build_hash_side(seed, rnd, 1, (int)n3, m, c.h2, c.v2, c.colcount, c.colstart, c.colperm, st);
+    if (rc != FPSK_OK) return rc;
+    rc = build_b_side(B, ldb, n2, n3, dtype, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q, st);
+    if (rc != FPSK_OK) return rc;
+    rc = max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
+    if (rc != FPSK_OK) return rc;
+    const HpArgs a = hp_args(nullptr, 0, nullptr, 0, n1, n2, n3, m, pl, c, nullptr);
+    hp_partition_kernel<<<(sms + 1 + 127) / 128, 128, 0, st>>>(a, sms, c.first_unit);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// One probe on a prepared B side.  d_S may be NULL (S then stays in the workspace).
+fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
+                          long long n3, fpsk_dtype dtype, int m, double mu, void *cache, size_t cache_bytes, void *ws,
+                          size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S)
+{
+    const int sms = hp_sm_count();
+    HpCache c;
+    HpWork w;
+    if (cache_bytes < hp_cache_layout(cache, n1, n2, n3, m, sms, &c)) return FPSK_ERR_WORKSPACE;
+    if (ws_bytes < hp_work_layout(ws, n1, n2, n3, m, sms, &w)) return FPSK_ERR_WORKSPACE;
+    HpPlan pl;
+    hp_plan(n2, n3, m, sms, pl);
+    const HpArgs a = hp_args(A, lda, C, ldc, n1, n2, n3, m, pl, c, &w);
+    static const bool force_plain = getenv("FPSK_HPROBE_PLAIN") != nullptr;
+    const bool bulk_ok = !force_plain && (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 &&
+                         lda % 8 == 0 && ldc % 4 == 0 && n2 % 8 == 0 && n3 % 4 == 0;
+    int n_maxA = sms;
+    if (bulk_ok) {
+        static std::once_flag once;
+        static cudaError_t attr_err = cudaSuccess;
+        std::call_once(once, [] {
+            attr_err = cudaFuncSetAttribute(hp_stream_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHpSmem);
+            if (attr_err == cudaSuccess)
+                attr_err = cudaFuncSetAttribute(hp_stream_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHpSmem);
+        });
+        FPSK_CUDA_OK(attr_err);
+        if (dtype == FPSK_FP16) hp_stream_kernel<__half><<<sms, kHpThreads, kHpSmem, st>>>(a);
+        else hp_stream_kernel<__nv_bfloat16><<<sms, kHpThreads, kHpSmem, st>>>(a);
+        FPSK_LAUNCH_CHECK();
+    } else {
+        n_maxA = 1;
+        FPSK_CUDA_OK(cudaMemsetAsync(w.maxA, 0, 4, st));
+        const int cols = pl.kpad > (int)n3 ? pl.kpad : (int)n3;
+        dim3 grid((cols + 255) / 256, m, 2);
+        if (dtype == FPSK_FP16) hp_rowsum_plain_kernel<__half><<<grid, 256, 0, st>>>(a);
+        else hp_rowsum_plain_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
+        FPSK_LAUNCH_CHECK();
+    }
+    fpsk_status rc = contraction_launch(w.P, c.Q, w.partAB, m, m, pl.kpad, pl.kpad, pl.npad, pl.ksplit, pl.kchunk, pl.tile, st);
+    if (rc != FPSK_OK) return rc;
+    HvArgs v;
+    v.partAB = w.partAB; v.ksplit = pl.ksplit; v.Tc = w.Tc; v.colperm = c.colperm; v.colstart = c.colstart;
+    v.m = m; v.n1 = (int)n1; v.n2 = (int)n2; v.n3 = (int)n3;
+    v.maxA = w.maxA; v.n_maxA = n_maxA; v.maxB = c.maxB;
+    const double mm = (double)m * (double)m;
+    v.thr_scale = (float)(mu * sqrt(2.0 * log(mm > 2.0 ? mm : 2.0)));
+    v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);
+    v.S = d_S ? d_S : w.S;
+    v.vstat = w.vstat; v.ctrl = w.ctrl; v.result = d_result;
+    if (dtype == FPSK_FP16) hp_verdict_kernel<__half><<<m, 256, 0, st>>>(v);
+    else hp_verdict_kernel<__nv_bfloat16><<<m, 256, 0, st>>>(v);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+}  // namespace fpsk

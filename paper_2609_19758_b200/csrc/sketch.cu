@@ -255,8 +255,9 @@ __global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long lon
 struct GemmBatch {
     const float *P, *Pw;      // problems: 0 = P Q, 1 = Pw Q, 2 = P Qw
     const float *Q, *Qw;
-    float *Cpart;     // [ksplit][3][M*N]
+    float *Cpart;     // [ksplit][nprob][M*N]
     int M, N, K, lda, ldb, ksplit, kchunk;
+    int nprob;        // problems per split in Cpart
 };
 
 template <int BM, int BN, int T>   // T = 4 or 8 outputs per thread per dimension; 256 threads
@@ -351,7 +352,7 @@ __global__ void __launch_bounds__(256, 2) sgemm_kernel(const GemmBatch g)
             }
         }
     }
-    float *Cout = g.Cpart + ((long long)ks * 3 + prob) * (long long)g.M * g.N;
+    float *Cout = g.Cpart + ((long long)ks * g.nprob + prob) * (long long)g.M * g.N;
 #pragma unroll
     for (int i = 0; i < T; ++i) {
         const int row = m0 + (i / 4) * (BM / 2) * (HALF - 1) + (HALF == 1 ? ty * 4 + i : ty * 4 + (i & 3));
@@ -515,6 +516,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         g.Cpart = w.partAB;
         g.M = m_b; g.N = m_b; g.K = pl.kpad; g.lda = pl.kpad; g.ldb = pl.npad;
         g.ksplit = pl.ksplit; g.kchunk = pl.kchunk;
+        g.nprob = 3;          // combine_kernel reads a stride of three problems per split
         const int nprob = mom ? 3 : 1;
         if (pl.tile == 64) {
             dim3 grid((m_b + 63) / 64, (m_b + 63) / 64, nprob * pl.ksplit);
@@ -542,6 +544,42 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         combine_kernel<<<(unsigned)((mm + 255) / 256), 256, 0, st>>>(w.partAB, pl.ksplit, w.partC, pl.nsplit, mm, mom ? 3 : 1, S, R, Tt);
         FPSK_LAUNCH_CHECK();
     }
+    return FPSK_OK;
+}
+
+fpsk_status contraction_launch(const float *P, const float *Q, float *part, int M, int N, int K, int lda, int ldb,
+                               int ksplit, int kchunk, int tile, cudaStream_t st)
+{
+    GemmBatch g;
+    g.P = P; g.Pw = P; g.Q = Q; g.Qw = Q;
+    g.Cpart = part;
+    g.M = M; g.N = N; g.K = K; g.lda = lda; g.ldb = ldb;
+    g.ksplit = ksplit; g.kchunk = kchunk; g.nprob = 1;
+    if (tile == 64) {
+        dim3 grid((N + 63) / 64, (M + 63) / 64, ksplit);
+        sgemm_kernel<64, 64, 4><<<grid, 256, 0, st>>>(g);
+    } else {
+        dim3 grid((N + 127) / 128, (M + 127) / 128, ksplit);
+        sgemm_kernel<128, 128, 8><<<grid, 256, 0, st>>>(g);
+    }
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+fpsk_status build_b_side(const void *B, long long ldb, long long n2, long long n3, fpsk_dtype dtype, int m_b, int kpad,
+                         int npad, const uint32_t *colperm, const int *colstart, float *Q, cudaStream_t st)
+{
+    const unsigned short *Bp = static_cast<const unsigned short *>(B);
+    const size_t smem = ((size_t)n3 * 2 + 15) / 16 * 16;
+    int grid = kpad < 1184 ? kpad : 1184;
+    if (dtype == FPSK_FP16) {
+        FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b_kernel<__half, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        compress_b_kernel<__half, false><<<grid, 256, smem, st>>>(Bp, ldb, (int)n2, (int)n3, kpad, m_b, npad, 0.f, colperm, colstart, Q, nullptr);
+    } else {
+        FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b_kernel<__nv_bfloat16, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        compress_b_kernel<__nv_bfloat16, false><<<grid, 256, smem, st>>>(Bp, ldb, (int)n2, (int)n3, kpad, m_b, npad, 0.f, colperm, colstart, Q, nullptr);
+    }
+    FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
 

@@ -42,6 +42,12 @@ fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, in
                             int *count, int *start, uint32_t *perm, cudaStream_t st);
 fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
                            SketchWs &w, cudaStream_t st, float *S, float *R, float *T);
+// one FP32 contraction part[ks] = P[:, ks-th K chunk] Q[ks-th K chunk, :]  (M x K by K x N, K a multiple of 16)
+fpsk_status contraction_launch(const float *P, const float *Q, float *part, int M, int N, int K, int lda, int ldb,
+                               int ksplit, int kchunk, int tile, cudaStream_t st);
+// Q = B H2^T (kpad x npad, rows >= n2 zero) from the bucket-sorted column permutation
+fpsk_status build_b_side(const void *B, long long ldb, long long n2, long long n3, fpsk_dtype dtype, int m_b, int kpad,
+                         int npad, const uint32_t *colperm, const int *colstart, float *Q, cudaStream_t st);
 fpsk_status peel_launch(const PeelEntry *dF, int nF, uint64_t seed, int rnd, long long n1, long long n3, int m_b,
                         float *S, float *R, float *T, cudaStream_t st);
 
@@ -110,5 +116,14 @@ fpsk_status scan_launch(const float *C, long long ldc, long long n1, long long n
 fpsk_status recompute_entries(const SketchIn &in, fpsk_dtype dtype, const ScanEntry *h_entries, int n, void *scratch,
                               cudaStream_t st, double *h_gamma, float *h_old);
 fpsk_status patch_launch(float *C, long long ldc, const PatchEntry *d_entries, int n, cudaStream_t st);
+
+// ---- the S only probe with a cached B side (hprobe.cu) ------------------------------------------
+size_t hprobe_cache_bytes(long long n1, long long n2, long long n3, int m);
+size_t hprobe_ws_bytes(long long n1, long long n2, long long n3, int m);
+fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long n2, long long n3, fpsk_dtype dtype,
+                           uint64_t seed, int rnd, int m, void *cache, size_t cache_bytes, cudaStream_t st);
+fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
+                          long long n3, fpsk_dtype dtype, int m, double mu, void *cache, size_t cache_bytes, void *ws,
+                          size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S);
 
 }  // namespace fpsk

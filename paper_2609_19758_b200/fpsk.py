@@ -49,6 +49,14 @@ class RepairReport(C.Structure):
                 ("radius", C.c_int32), ("reserved", C.c_int32), ("first_probe", ProbeResult), ("second_probe", ProbeResult)]
 
 
+class BSide(C.Structure):
+    """Host record of a cached B side (fpsk_bside)."""
+    _fields_ = [("B", C.c_void_p), ("cache", C.c_void_p), ("ldb", C.c_int64), ("m", C.c_int64), ("k", C.c_int64),
+                ("n", C.c_int64), ("seed", C.c_uint64), ("version", C.c_uint64), ("dtype", C.c_int32),
+                ("n_buckets", C.c_int32), ("round", C.c_int32), ("valid", C.c_int32), ("rebuilds", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
 class FpskError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -91,6 +99,15 @@ def lib() -> C.CDLL:
         L.fpsk_probe_static.restype = C.c_int
         L.fpsk_probe_static.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, C.c_int, C.POINTER(Params),
                                         vp, vp, vp]
+        L.fpsk_probe_hashed_cache_bytes.restype = sz
+        L.fpsk_probe_hashed_cache_bytes.argtypes = [i64, i64, i64, i32]
+        L.fpsk_probe_hashed_workspace_bytes.restype = sz
+        L.fpsk_probe_hashed_workspace_bytes.argtypes = [i64, i64, i64, i32]
+        L.fpsk_bside_matches.restype = i32
+        L.fpsk_bside_matches.argtypes = [C.POINTER(BSide), vp, i64, u64, i64, i64, i64, C.c_int, u64, i32, i32, vp]
+        L.fpsk_probe_hashed.restype = C.c_int
+        L.fpsk_probe_hashed.argtypes = [C.POINTER(BSide), vp, i64, vp, i64, u64, vp, i64, i64, i64, i64, C.c_int, C.c_int,
+                                        u64, i32, i32, C.POINTER(Params), vp, sz, vp, sz, vp, vp, vp]
         L.fpsk_hash_tables.restype = C.c_int
         L.fpsk_hash_tables.argtypes = [u64, i32, i32, i64, i32, vp, vp, vp]
         L.fpsk_workspace_bytes.restype = sz
@@ -212,6 +229,45 @@ def probe_static(A, B, Cm, result: torch.Tensor, residual: Optional[torch.Tensor
                                  result.data_ptr(), residual.data_ptr() if residual is not None else None)
     if rc != STATUS_OK:
         raise FpskError(rc, "fpsk_probe_static")
+
+
+class HashedProbe:
+    """Buffers of the S only probe with a cached B side: the host record, the device cache and the
+    per-call workspace (torch owns the memory).  ``__call__`` is one asynchronous probe."""
+
+    def __init__(self, m: int, k: int, n: int, n_buckets: int, seed: int, rnd: int = 0, device=None, stream=None):
+        self.shape = (m, k, n)
+        self.n_buckets, self.seed, self.round = n_buckets, seed, rnd
+        cb = int(lib().fpsk_probe_hashed_cache_bytes(m, k, n, n_buckets))
+        wb = int(lib().fpsk_probe_hashed_workspace_bytes(m, k, n, n_buckets))
+        if cb == 0 or wb == 0:
+            raise FpskError(ERR_SHAPE, "fpsk_probe_hashed_cache_bytes")
+        self.cache = torch.empty(cb, dtype=torch.uint8, device=device or "cuda")
+        self.ws = torch.empty(wb, dtype=torch.uint8, device=device or "cuda")
+        rc = lib().fpsk_probe_init(self.ws.data_ptr(), wb, _stream_ptr(stream))
+        if rc != STATUS_OK:
+            raise FpskError(rc, "fpsk_probe_init")
+        self.side = BSide()
+
+    def matches(self, B: torch.Tensor, b_version: int) -> bool:
+        m, k, n = self.shape
+        ldb = B.stride(0) if k > 1 else max(n, B.stride(0))
+        return bool(lib().fpsk_bside_matches(C.byref(self.side), B.data_ptr(), ldb, b_version, m, k, n, dtype_of(B),
+                                             self.seed, self.round, self.n_buckets, self.cache.data_ptr()))
+
+    def __call__(self, A, B, Cm, result: torch.Tensor, b_version: int = 0, S: Optional[torch.Tensor] = None,
+                 params: Optional[Params] = None, stream=None, c_is_fp32: Optional[bool] = None) -> None:
+        a = _mat_args(A, B, Cm)
+        assert (a[6], a[7], a[8]) == self.shape
+        if c_is_fp32 is None:
+            c_is_fp32 = Cm.dtype == torch.float32
+        rc = lib().fpsk_probe_hashed(C.byref(self.side), a[0], a[1], a[2], a[3], b_version, a[4], a[5], a[6], a[7],
+                                     a[8], a[9], 1 if c_is_fp32 else 0, self.seed, self.round, self.n_buckets,
+                                     C.byref(params) if params is not None else None, self.cache.data_ptr(),
+                                     self.cache.numel(), self.ws.data_ptr(), self.ws.numel(), _stream_ptr(stream),
+                                     result.data_ptr(), S.data_ptr() if S is not None else None)
+        if rc != STATUS_OK:
+            raise FpskError(rc, "fpsk_probe_hashed")
 
 
 def new_probe_result(device=None) -> torch.Tensor:

@@ -1,0 +1,185 @@
+"""Parity of the S only probe with a cached B side (Section "The Cheap S Only Probe") with the oracle.
+
+S within 1e-5 of the bucket's sum of sum_k |A_ik||B_kj|; the verdict through the oracle's rule applied
+to the GPU's own S; bit-exact on integer products; the cache key logic on the device path.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2609_19758_b200 import build as B
+from paper_2609_19758_b200 import fpsk, harness, workloads as W
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    B.build()
+    fpsk.lib()
+
+
+def _f64(t):
+    return t.double().numpy()
+
+
+def _case(kind, n1, n2, n3, dtype, seed):
+    A, Bm = W.operands(kind, n1, n2, n3, dtype, seed)
+    if n1 % 8 == 0 and n2 % 8 == 0 and n3 % 8 == 0:
+        Cm = harness.vendor_gemm_fp32(A.cuda(), Bm.cuda()).cpu()
+    else:
+        Cm = W.cpu_fp32_product(A, Bm)
+    return A, Bm, Cm
+
+
+def _run(hp, A, Bm, Cm, version=0, params=None):
+    m = hp.n_buckets
+    res = fpsk.new_probe_result()
+    S = torch.full((m, m), float("nan"), dtype=torch.float32, device="cuda")
+    hp(A, Bm, Cm, res, b_version=version, S=S, params=params)
+    torch.cuda.synchronize()
+    return fpsk.read_probe_result(res), S.cpu().numpy().astype(np.float64)
+
+
+SHAPES = [
+    # (n1, n2, n3, m)   bulk-copy path: n2 % 8 == 0, n3 % 4 == 0
+    (64, 64, 64, 4), (256, 256, 256, 16), (512, 2056, 1028, 48), (1024, 512, 2048, 64), (1000, 4104, 1500, 100),
+    (2048, 1384, 4104, 256), (300, 8, 4, 7), (96, 4096, 96, 1),
+    # plain path: odd sizes
+    (7, 5, 9, 3), (33, 17, 40, 5), (255, 256, 257, 16), (257, 255, 33, 48),
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+@pytest.mark.parametrize("dtype", [W.FP16, W.BF16])
+def test_sketch_and_verdict(shape, dtype):
+    n1, n2, n3, m = shape
+    A, Bm, Cm = _case("uniform" if dtype == W.FP16 else "gauss_scaled", n1, n2, n3, dtype, 5)
+    A64, B64 = _f64(A), _f64(Bm)
+    ref, S_ref = O.probe_hashed(A64, B64, Cm.numpy(), 21, 4, m)
+    h1, _ = O.hash_round(21, 4, 0, n1, m)
+    h2, _ = O.hash_round(21, 4, 1, n3, m)
+    denom = O.abs_sketch(O.abs_product(A64, B64), h1, h2, m)
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=21, rnd=4)
+    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda())
+    assert got.status == 0
+    assert np.all(np.abs(S - S_ref) <= TOL * denom + 1e-30)
+    assert got.tau == pytest.approx(ref.tau, rel=1e-6)
+    v = O.probe_verdict(S.ravel(), ref.tau, n_rows=n1 * n3 / float(m * m))     # the rule on the GPU's own S
+    assert got.sigma_hat == pytest.approx(v.sigma_hat, rel=1e-4, abs=1e-30)
+    assert got.thr == pytest.approx(v.thr, rel=1e-4, abs=1e-30)
+    assert got.max_abs == pytest.approx(v.max_abs, rel=1e-6, abs=1e-30)
+    assert got.argmax_col == v.argmax_col
+    assert got.nonfinite == 0
+    if abs(v.max_abs - v.thr) > 1e-3 * v.thr:
+        assert bool(got.fired) == v.fired
+
+
+@pytest.mark.parametrize("shape", [(96, 64, 80, 8), (512, 2048, 1024, 32), (130, 72, 100, 5), (31, 9, 27, 4)])
+def test_integer_products_are_bit_exact(shape):
+    n1, n2, n3, m = shape
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 5)
+    Cm = W.cpu_fp32_product(A, Bm)
+    Cm[n1 // 3, n3 // 2] += 3.0
+    Cm[n1 - 1, 0] -= 5.0
+    ref, S_ref = O.probe_hashed(_f64(A), _f64(Bm), Cm.numpy(), 11, 7, m)
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=11, rnd=7)
+    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda())
+    assert np.array_equal(S, S_ref)
+    assert got.fired == 1 and ref.fired and got.argmax_col == ref.argmax_col and got.max_abs == ref.max_abs
+
+
+def test_detection_agrees_with_the_oracle_on_small_faults():
+    n, m = 1024, 64
+    A, Bm, Cm = _case("gauss_scaled", n, n, n, W.BF16, 11)
+    A64, B64 = _f64(A), _f64(Bm)
+    rms = W.rms(Cm)
+    hp = fpsk.HashedProbe(n, n, n, m, seed=3, rnd=0)
+    dA, dB = A.cuda(), Bm.cuda()
+    got, _ = _run(hp, dA, dB, Cm.cuda())
+    ref, _ = O.probe_hashed(A64, B64, Cm.numpy(), 3, 0, m)
+    assert not ref.fired and got.fired == 0
+    h1, _ = O.hash_round(3, 0, 0, n, m)
+    h2, _ = O.hash_round(3, 0, 1, n, m)
+    for s in range(4):
+        f = W.faults_additive(n, n, rms, s, 1, 0.02, 0.09, "small")
+        Cf, ch = W.inject(Cm, f)
+        got, _ = _run(hp, dA, dB, Cf.cuda())
+        ref, _ = O.probe_hashed(A64, B64, Cf.numpy(), 3, 0, m)
+        assert ref.fired and got.fired == 1
+        assert got.argmax_col == ref.argmax_col == int(h1[f[0].i]) * m + int(h2[f[0].j])
+    assert hp.side.rebuilds == 1                      # one B side served every call
+
+
+def test_nonfinite_entries_fire():
+    A, Bm, Cm = _case("uniform", 128, 64, 128, W.FP16, 3)
+    hp = fpsk.HashedProbe(128, 64, 128, 8, seed=1)
+    for bad in (float("nan"), float("inf"), float("-inf")):
+        Cn = Cm.clone()
+        Cn[5, 7] = bad
+        got, S = _run(hp, A.cuda(), Bm.cuda(), Cn.cuda())
+        assert got.fired == 1 and got.nonfinite == 1 and got.status == 0
+        assert np.count_nonzero(~np.isfinite(S)) == 1
+
+
+def test_cache_is_keyed_on_identity_and_version():
+    n1, n2, n3, m = 256, 128, 192, 16
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, W.BF16, 9)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=5)
+    assert not hp.matches(dB, 0)
+    r0, S0 = _run(hp, dA, dB, dC, version=0)
+    assert hp.matches(dB, 0) and hp.side.rebuilds == 1
+    before = fpsk.launch_count()
+    r1, S1 = _run(hp, dA, dB, dC, version=0)
+    per_call = fpsk.launch_count() - before
+    assert hp.side.rebuilds == 1 and np.array_equal(S0, S1)         # cached: same result, nothing rebuilt
+    assert per_call == 3                                             # row sums, contraction, verdict
+    # an in-place update of B with a new version rebuilds; the product no longer matches C
+    dB.mul_(2.0)
+    r2, S2 = _run(hp, dA, dB, dC, version=1)
+    assert hp.side.rebuilds == 2 and r2.fired == 1
+    ref, S_ref = O.probe_hashed(_f64(A), 2.0 * _f64(Bm), Cm.numpy(), 5, 0, m)
+    h1, _ = O.hash_round(5, 0, 0, n1, m)
+    h2, _ = O.hash_round(5, 0, 1, n3, m)
+    denom = O.abs_sketch(O.abs_product(_f64(A), 2.0 * _f64(Bm)), h1, h2, m)
+    assert np.all(np.abs(S2 - S_ref) <= TOL * denom)
+    # another tensor with the same contents is another identity
+    dB2 = dB.clone()
+    _run(hp, dA, dB2, dC, version=1)
+    assert hp.side.rebuilds == 3
+
+
+def test_rejections():
+    A, Bm, Cm = _case("uniform", 64, 64, 64, W.FP16, 3)
+    hp = fpsk.HashedProbe(64, 64, 64, 8, seed=1)
+    res = fpsk.new_probe_result()
+    with pytest.raises(fpsk.FpskError) as e:
+        hp(A.cuda(), Bm.cuda(), Cm.cuda(), res, c_is_fp32=False)
+    assert e.value.status == fpsk.ERR_DTYPE
+    assert hp.side.rebuilds == 0
+
+
+def test_reruns_are_bit_identical_and_paths_agree():
+    n1, n2, n3, m = 1536, 1024, 2048, 96
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, W.FP16, 4)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=8, rnd=2)
+    r0, S0 = _run(hp, dA, dB, dC)
+    for _ in range(3):
+        r, S = _run(hp, dA, dB, dC)
+        assert np.array_equal(S, S0) and r.sigma_hat == r0.sigma_hat and r.thr == r0.thr
+    # a view with an odd column offset takes the plain-load path: same sketch within rounding
+    big = torch.zeros(n1, n2 + 8, dtype=dA.dtype, device="cuda")
+    big[:, 1:n2 + 1] = dA
+    hp2 = fpsk.HashedProbe(n1, n2, n3, m, seed=8, rnd=2)
+    r2, S2 = _run(hp2, big[:, 1:n2 + 1], dB, dC)
+    h1, _ = O.hash_round(8, 2, 0, n1, m)
+    h2, _ = O.hash_round(8, 2, 1, n3, m)
+    denom = O.abs_sketch(O.abs_product(_f64(A), _f64(Bm)), h1, h2, m)
+    assert np.all(np.abs(S2 - S0) <= 2 * TOL * denom)
+    assert r2.tau == r0.tau

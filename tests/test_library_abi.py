@@ -95,3 +95,43 @@ def test_argument_validation_needs_no_device(lib):
     assert lib.fpsk_workspace_bytes(4096, 4096, 4096, 384, None) > 3 * 384 * 384 * 4
     assert lib.fpsk_workspace_bytes(4096, 4096, 4096, 10 ** 6, None) == 0
     assert fpsk.max_buckets(4096, 4096, 4096) >= 4096 and fpsk.max_buckets(16384, 16384, 16384) >= 4096
+
+
+def test_bside_record_and_key_logic(lib):
+    """The cache key of the B side (tensor identity and version; Section "Implementation") is host logic."""
+    assert C.sizeof(fpsk.BSide) == 88 and fpsk.BSide.valid.offset == 76
+    s = fpsk.BSide()
+    Bp, cache = C.c_void_p(0x1000), C.c_void_p(0x2000)
+    args = (Bp, 64, 7, 32, 48, 64, fpsk.BF16, 99, 3, 16, cache)
+    assert lib.fpsk_bside_matches(C.byref(s), *args) == 0            # nothing cached yet
+    s.B, s.cache, s.ldb, s.version, s.m, s.k, s.n = 0x1000, 0x2000, 64, 7, 32, 48, 64
+    s.dtype, s.seed, s.round, s.n_buckets, s.valid = fpsk.BF16, 99, 3, 16, 1
+    assert lib.fpsk_bside_matches(C.byref(s), *args) == 1
+    for pos, other in ((0, C.c_void_p(0x1040)), (1, 128), (2, 8), (3, 33), (4, 49), (5, 65), (6, fpsk.FP16), (7, 98),
+                       (8, 2), (9, 17), (10, C.c_void_p(0x3000))):
+        changed = list(args)
+        changed[pos] = other
+        assert lib.fpsk_bside_matches(C.byref(s), *changed) == 0, pos   # any field of the key invalidates
+    s.valid = 0
+    assert lib.fpsk_bside_matches(C.byref(s), *args) == 0
+
+
+def test_hashed_probe_validation_needs_no_device(lib):
+    one = C.c_void_p(4096)
+    s = fpsk.BSide()
+    f = lib.fpsk_probe_hashed
+
+    def call(side=s, A=one, c_is_fp32=1, nb=16, rnd=0, cache=one, cbytes=1 << 30, ws=one, wbytes=1 << 30, m=64):
+        return f(C.byref(side) if side is not None else None, A, 64, one, 64, 0, one, 64, m, 64, 64, fpsk.FP16, c_is_fp32,
+                 1, rnd, nb, None, cache, cbytes, ws, wbytes, None, one, None)
+
+    assert call(c_is_fp32=0) == fpsk.ERR_DTYPE          # a narrowed C is rejected
+    assert call(side=None) == fpsk.ERR_NULL
+    assert call(A=None) == fpsk.ERR_NULL
+    assert call(m=0) == fpsk.ERR_SHAPE
+    assert call(nb=0) == fpsk.ERR_BUCKETS and call(nb=5000) == fpsk.ERR_BUCKETS and call(rnd=-1) == fpsk.ERR_BUCKETS
+    assert call(cache=C.c_void_p(4096 + 8)) == fpsk.ERR_ALIGN
+    assert call(cbytes=16) == fpsk.ERR_WORKSPACE and call(wbytes=16) == fpsk.ERR_WORKSPACE
+    assert s.valid == 0 and s.rebuilds == 0
+    assert lib.fpsk_probe_hashed_cache_bytes(0, 8, 8, 4) == 0
+    assert lib.fpsk_probe_hashed_workspace_bytes(64, 64, 64, 16) >= 4 * (16 * 64 * 2 + 16 * 16)
