@@ -1,9 +1,12 @@
 // The S only probe at the probe's own bucket count (Section "The Cheap S Only Probe"):
 //   S = (H1 A)(B H2^T) - H1 C H2^T,   sigma_hat, threshold and one-bit verdict (Section "Thresholds").
-// The B side (hash round, bucket-sorted permutations, Q = B H2^T, max|B|) is built once per weight
-// tensor and kept by the caller; a call on a cached B reads A once and C once.
+// The B side (hash round, bucket-sorted permutations, Q = B H2^T, max|B|, and the work list of the
+// streaming kernel, which depends on the hash round only) is built once per weight tensor and kept
+// by the caller; a call on a cached B reads A once and C once.
 //
-//   hp_partition_kernel     balanced split of the (matrix, column segment, row bucket) units over CTAs
+//   hp_count_chunks_kernel, hp_fill_stages_kernel
+//                           the work list: for every (matrix, column segment, row bucket) unit the ring
+//                           stages (rows, signs) that stream it
 //   hp_stream_kernel        P = H1 A (m x n2) and Tc = H1 C (m x n3): signed row-bucket sums, one
 //                           persistent CTA per SM, rows gathered by bulk copies into a shared-memory ring
 //   hp_rowsum_plain_kernel  the same sums with plain loads (inputs that bulk copies cannot address)
@@ -21,15 +24,17 @@
 namespace fpsk {
 
 constexpr int kHpConsumers = 512;
-constexpr int kHpThreads = kHpConsumers + 32;     // + producer warp
-constexpr int kHpStages = 6;
-constexpr int kHpStageBytes = 32768;
+constexpr int kHpTeamThreads = 256;               // consumer threads of one team
+constexpr int kHpThreads = kHpConsumers + 64;     // + one producer warp per team
+constexpr int kHpStages = 6;                      // ring stages per team
+constexpr int kHpStageBytes = 16384;
 constexpr int kHpPieceBytes = 4096;               // one row of one column segment
 constexpr int kHpPieces = kHpStageBytes / kHpPieceBytes;
+static_assert(kHpPieces == 4, "a stage record's row indices sit in one 16-byte lane word");
+static_assert(2 * 2 * kHpStages * 8 + 8 <= 256, "barrier block");
 constexpr int kHpSegA = kHpPieceBytes / 2;        // columns of A per segment
 constexpr int kHpSegC = kHpPieceBytes / 4;        // columns of C per segment
-constexpr int kHpRedBytes = 256 * 32;             // lane-combine scratch: 256 threads x 8 floats
-constexpr int kHpSmem = kHpStages * kHpStageBytes + kHpRedBytes + 256 /*barriers*/ + kHpStages * 16 /*stage records*/;
+constexpr int kHpSmem = 2 * kHpStages * kHpStageBytes + 256 /*barriers*/ + 2 * kHpStages * 16 /*stage records*/;
 
 struct HpArgs {
     const unsigned short *A;
@@ -40,51 +45,70 @@ struct HpArgs {
     int segsA, segsC;              // column segments of A and of C
     const uint32_t *rowperm;       // rows sorted by bucket; bit 31 = sign -1
     const int *rowstart;           // [m + 1]
-    const int *first_unit;         // [grid + 1]
+    const int *stages;             // chunks of 8 stage records, 16 ints per record:
+                                   //   [0] bucket | isC << 30   [1] segment   [2] pieces | last-of-unit << 8 | signs << 16
+                                   //   [4 .. 4 + pieces) row indices;  [15] of the chunk's last record: next chunk of the unit
+                                   // chunk u is the first chunk of unit u; longer units continue in chunks >= units
     float *P;                      // m x kpad
     float *Tc;                     // m x n3
     unsigned int *maxA;            // per CTA: bits of max|A| over what it streamed
-    unsigned int *ctrl;            // [0] verdict ticket, [1] error flag
+    unsigned int *ctrl;            // [0] verdict ticket, [1] error flag, [2] next unit to hand out
+    int trace_on;
+    unsigned long long *trace;     // 8 time stamps per CTA when trace_on
 };
 
-// cumulative bytes streamed before unit u, with units ordered (matrix, segment, bucket)
-__device__ __forceinline__ long long hp_unit_start(const HpArgs &p, int u)
-{
-    const int UA = p.m * p.segsA, U = UA + p.m * p.segsC;
-    if (u >= U) return 2LL * p.n1 * p.n2 + 4LL * p.n1 * p.n3;
-    if (u < UA) {
-        const int s = u / p.m, a = u - s * p.m;
-        const int w = min(kHpSegA, p.n2 - s * kHpSegA);
-        return 2LL * p.n1 * ((long long)s * kHpSegA) + 2LL * __ldg(p.rowstart + a) * w;
-    }
-    const int v = u - UA;
-    const int s = v / p.m, a = v - s * p.m;
-    const int w = min(kHpSegC, p.n3 - s * kHpSegC);
-    return 2LL * p.n1 * p.n2 + 4LL * p.n1 * ((long long)s * kHpSegC) + 4LL * __ldg(p.rowstart + a) * w;
-}
+// Units are (matrix, column segment, row bucket), ordered that way: A units first.  A unit's rows go
+// out in ring stages of up to kHpPieces rows; a stage never mixes units; an empty bucket still gets
+// one stage (its sums are written as zeros).  Stage records come in chunks of eight, so that one
+// warp-wide 16-byte load brings a whole chunk.
+constexpr int kHpChunk = 8;
 
-// first_unit[c] = smallest unit whose start is >= c W / grid  (W = all bytes); first_unit[grid] = U
-__global__ void hp_partition_kernel(HpArgs p, int grid, int *first_unit)
+__global__ void hp_count_chunks_kernel(HpArgs p, int *extra)
 {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c > grid) return;
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
     const int U = p.m * (p.segsA + p.segsC);
-    if (c == grid) { first_unit[c] = U; return; }
-    const long long W = 2LL * p.n1 * p.n2 + 4LL * p.n1 * p.n3;
-    const long long target = (W / grid) * c + (W % grid) * c / grid;
-    int lo = 0, hi = U;                 // smallest u in [0, U] with start(u) >= target
-    while (lo < hi) {
-        const int mid = (lo + hi) >> 1;
-        if (hp_unit_start(p, mid) >= target) hi = mid; else lo = mid + 1;
-    }
-    first_unit[c] = lo;
+    if (u >= U) return;
+    const int a = u % p.m;
+    const int rows = __ldg(p.rowstart + a + 1) - __ldg(p.rowstart + a);
+    const int nst = rows > 0 ? (rows + kHpPieces - 1) / kHpPieces : 1;
+    extra[u] = (nst + kHpChunk - 1) / kHpChunk - 1;        // chunks beyond the first
 }
 
-struct HpStageRec {     // what the producer tells the consumers about one stage
-    int unit;           // -1: no more work
-    int info;           // pieces | last << 8 | sign bits << 16
-    int pad0, pad1;
-};
+__global__ void hp_fill_stages_kernel(HpArgs p, const int *extra_start, int *stages)
+{
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    const int UA = p.m * p.segsA, U = UA + p.m * p.segsC;
+    if (u >= U) return;
+    const bool isC = u >= UA;
+    const int v = isC ? u - UA : u;
+    const int seg = v / p.m, a = v - seg * p.m;
+    const int s0 = __ldg(p.rowstart + a), s1 = __ldg(p.rowstart + a + 1);
+    const int nst = s1 > s0 ? (s1 - s0 + kHpPieces - 1) / kHpPieces : 1;
+    const int nchunk = (nst + kHpChunk - 1) / kHpChunk;
+    int pos = s0;
+    for (int k = 0; k < nchunk; ++k) {
+        const int ci = k == 0 ? u : U + extra_start[u] + (k - 1);
+        for (int j = 0; j < kHpChunk; ++j) {
+            int *rec = stages + ((long long)ci * kHpChunk + j) * 16;
+            const int st = k * kHpChunk + j;
+            for (int q = 0; q < 16; ++q) rec[q] = 0;
+            if (st < nst) {
+                const int np = min(kHpPieces, s1 - pos);
+                unsigned int signs = 0;
+                for (int q = 0; q < np; ++q) {
+                    const uint32_t e = __ldg(p.rowperm + pos + q);
+                    rec[4 + q] = (int)(e & 0x7FFFFFFFu);
+                    signs |= (e >> 31) << q;
+                }
+                rec[0] = a | (isC ? (1 << 30) : 0);
+                rec[1] = seg;
+                rec[2] = np | (st == nst - 1 ? 0x100 : 0) | (int)(signs << 16);
+                pos += np;
+            }
+            if (j == kHpChunk - 1) rec[15] = k + 1 < nchunk ? U + extra_start[u] + k : -1;
+        }
+    }
+}
 
 // Barrier over the consumer warps on an mbarrier (one arrival per warp), so that this wait is
 // bounded like every other wait of the kernel.  Returns false when it gave up.
@@ -97,130 +121,198 @@ __device__ __forceinline__ bool hp_consumer_sync(uint32_t cbar, uint32_t &cpar)
     return w;
 }
 
+__device__ __forceinline__ unsigned long long hp_gtime()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+
+// One CTA per SM, two independent teams per CTA.  A team is one producer warp, eight consumer warps
+// (256 threads x 16 bytes = one row piece) and its own ring of kHpStages stages; it takes whole
+// units, so nothing is shared between teams.  Two producer warps matter: one warp issues a bulk
+// copy about every 90 ns, which at 4 KB per copy is just the SM's share of the memory bandwidth.
+//
+// Units are handed out by a counter (ctrl[2]): a team that streams faster takes more of them, so
+// all teams finish together whatever their share of the memory system.  Which team sums a unit
+// does not change the sum (fixed order inside the unit).  The producer keeps the counter two units
+// ahead and a unit's stage records one unit ahead, so no round trip to L2 sits between two stages.
 template <typename T>
 __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned char *ring = smem;
-    float4 *red4 = reinterpret_cast<float4 *>(smem + kHpStages * kHpStageBytes);
-    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + kHpStages * kHpStageBytes + kHpRedBytes);
-    HpStageRec *recs = reinterpret_cast<HpStageRec *>(smem + kHpStages * kHpStageBytes + kHpRedBytes + 256);
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + 2 * kHpStages * kHpStageBytes);
+    int *recs_all = reinterpret_cast<int *>(smem + 2 * kHpStages * kHpStageBytes + 256);
     __shared__ unsigned int smx[kHpConsumers / 32];
     const int c = blockIdx.x;
     const int tid = threadIdx.x;
-    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kHpStages), cbar = smem_u32(bars + 2 * kHpStages);
+    const bool tr = p.trace_on != 0;
+    const int team = tid < kHpConsumers ? tid >> 8 : (tid - kHpConsumers) >> 5;
+    unsigned char *ring = smem + (size_t)team * kHpStages * kHpStageBytes;
+    int *recs = recs_all + team * kHpStages * 4;
+    const uint32_t full0 = smem_u32(bars) + team * (2 * kHpStages * 8), empty0 = full0 + kHpStages * 8;
+    const uint32_t cbar = smem_u32(bars) + 2 * (2 * kHpStages * 8);
     if (tid == 0) {
-        for (int s = 0; s < kHpStages; ++s) {
-            mbar_init(full0 + 8 * s, 1);
-            mbar_init(empty0 + 8 * s, kHpConsumers / 32);
+        for (int s = 0; s < 2 * kHpStages; ++s) {
+            const int tm = s / kHpStages, ss = s % kHpStages;
+            mbar_init(smem_u32(bars) + tm * (2 * kHpStages * 8) + 8 * ss, 1);
+            mbar_init(smem_u32(bars) + tm * (2 * kHpStages * 8) + kHpStages * 8 + 8 * ss, kHpTeamThreads / 32);
         }
         mbar_init(cbar, kHpConsumers / 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     __syncthreads();
-    const int UA = p.m * p.segsA;
-    const int u0 = __ldg(p.first_unit + c), u1 = __ldg(p.first_unit + c + 1);
+    if (tr && (tid == 0 || tid == kHpTeamThreads)) p.trace[(c * 2 + team) * 8 + 0] = hp_gtime();
 
     if (tid >= kHpConsumers) {
-        // ------------------------------------------------------------ producer warp
-        const int lane = tid - kHpConsumers;
+        // ------------------------------------------------------------ producer warp of the team
+        const int lane = tid & 31;
+        const int U = p.m * (p.segsA + p.segsC);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
-        for (int u = u0; u < u1 && ok; ++u) {
-            const bool isC = u >= UA;
-            const int v = isC ? u - UA : u;
-            const int seg = v / p.m, a = v - seg * p.m;
-            const int s0 = __ldg(p.rowstart + a), s1 = __ldg(p.rowstart + a + 1);
-            const int wbytes = isC ? 4 * min(kHpSegC, p.n3 - seg * kHpSegC) : 2 * min(kHpSegA, p.n2 - seg * kHpSegA);
-            const unsigned char *base = isC ? reinterpret_cast<const unsigned char *>(p.C + (long long)seg * kHpSegC)
-                                            : reinterpret_cast<const unsigned char *>(p.A + (long long)seg * kHpSegA);
-            const long long ldb = isC ? p.ldc * 4 : p.lda * 2;
-            int pos = s0;
-            do {
-                const int np = min(kHpPieces, s1 - pos);
-                const bool last = pos + np >= s1;
-                uint32_t e = 0;
-                if (lane < np) e = __ldg(p.rowperm + pos + lane);
-                int w = 1;
-                if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
-                w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                if (!w) { ok = false; break; }
-                const unsigned int signs = __ballot_sync(0xFFFFFFFFu, lane < np && (e >> 31));
-                if (lane == 0) {
-                    HpStageRec r;
-                    r.unit = u;
-                    r.info = np | (last ? 0x100 : 0) | (int)(signs << 16);
-                    r.pad0 = r.pad1 = 0;
-                    recs[stage] = r;
-                    if (np > 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)np * (uint32_t)wbytes);
-                    else mbar_arrive(full0 + 8 * stage);
+        bool first = true;
+        // uA: unit being streamed; uB: the next one; both known, and so are their first chunks RA, RB
+        // (lane l holds 16 bytes: ints 4 (l % 4) .. of record l / 4).  uC is fetched while uA streams.
+        const int4 *chunks = reinterpret_cast<const int4 *>(p.stages);
+        int uA = 0, uB = 0;
+        if (lane == 0) {
+            uA = (int)atomicAdd(p.ctrl + 2, 1u);
+            uB = (int)atomicAdd(p.ctrl + 2, 1u);
+        }
+        uA = __shfl_sync(0xFFFFFFFFu, uA, 0);
+        uB = __shfl_sync(0xFFFFFFFFu, uB, 0);
+        const int4 zero4 = make_int4(0, 0, 0, 0);
+        int4 RA = uA < U ? __ldg(chunks + (long long)uA * 32 + lane) : zero4;
+        int4 RB = uB < U ? __ldg(chunks + (long long)uB * 32 + lane) : zero4;
+        while (uA < U && ok) {
+            int uC = 0;
+            if (lane == 0) uC = (int)atomicAdd(p.ctrl + 2, 1u);          // needed when this unit is done
+            int4 R = RA;
+            for (;;) {
+                const unsigned int lastmask = __ballot_sync(0xFFFFFFFFu, (lane & 3) == 0 && (R.z & 0x100));
+                const int nxt = __shfl_sync(0xFFFFFFFFu, R.w, 31);
+                int4 Rn = zero4;
+                if (!lastmask && nxt >= 0) Rn = __ldg(chunks + (long long)nxt * 32 + lane);    // continuation, in flight meanwhile
+                const int jn = lastmask ? ((__ffs(lastmask) - 1) >> 2) + 1 : kHpChunk;
+                for (int j = 0; j < jn; ++j) {
+                    const int h0 = __shfl_sync(0xFFFFFFFFu, R.x, 4 * j), h1 = __shfl_sync(0xFFFFFFFFu, R.y, 4 * j),
+                              h2 = __shfl_sync(0xFFFFFFFFu, R.z, 4 * j);
+                    const int src = 4 * j + 1;                  // ints 4..7 of record j: the row indices
+                    const int v0 = __shfl_sync(0xFFFFFFFFu, R.x, src), v1 = __shfl_sync(0xFFFFFFFFu, R.y, src),
+                              v2 = __shfl_sync(0xFFFFFFFFu, R.z, src), v3 = __shfl_sync(0xFFFFFFFFu, R.w, src);
+                    const int row = (lane & 2) ? ((lane & 1) ? v3 : v2) : ((lane & 1) ? v1 : v0);
+                    const int np = h2 & 0xFF;
+                    const bool isC = (h0 >> 30) != 0;
+                    const int seg = h1;
+                    const int wbytes = isC ? 4 * min(kHpSegC, p.n3 - seg * kHpSegC) : 2 * min(kHpSegA, p.n2 - seg * kHpSegA);
+                    const unsigned char *base = isC ? reinterpret_cast<const unsigned char *>(p.C + (long long)seg * kHpSegC)
+                                                    : reinterpret_cast<const unsigned char *>(p.A + (long long)seg * kHpSegA);
+                    const long long ldb = isC ? p.ldc * 4 : p.lda * 2;
+                    int w = 1;
+                    if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                    w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                    if (!w) { ok = false; break; }
+                    if (lane == 0) {
+                        *reinterpret_cast<int4 *>(recs + stage * 4) = make_int4(h0, h1, h2, 0);
+                        if (np > 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)np * (uint32_t)wbytes);
+                        else mbar_arrive(full0 + 8 * stage);
+                    }
+                    __syncwarp();
+                    if (tr && lane == 0 && first) { p.trace[(c * 2 + team) * 8 + 1] = hp_gtime(); first = false; }
+                    if (lane < np)
+                        bulk_g2s(smem_u32(ring + (size_t)stage * kHpStageBytes) + (uint32_t)lane * kHpPieceBytes,
+                                 base + (long long)row * ldb, (uint32_t)wbytes, full0 + 8 * stage);
+                    if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
                 }
-                __syncwarp();
-                if (lane < np)
-                    bulk_g2s(smem_u32(ring + (size_t)stage * kHpStageBytes) + (uint32_t)lane * kHpPieceBytes,
-                             base + (long long)(e & 0x7FFFFFFFu) * ldb, (uint32_t)wbytes, full0 + 8 * stage);
-                if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
-                pos += np;
-            } while (pos < s1);
+                if (lastmask || !ok || nxt < 0) break;
+                R = Rn;
+            }
+            uC = __shfl_sync(0xFFFFFFFFu, uC, 0);
+            uA = uB; RA = RB;
+            uB = uC;
+            RB = uB < U ? __ldg(chunks + (long long)uB * 32 + lane) : zero4;     // used one unit from now
         }
         if (ok) {
-            // end of work: one empty stage with unit = -1
+            // end of work: one empty stage marked -1
             int w = 1;
             if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
             w = __shfl_sync(0xFFFFFFFFu, w, 0);
             if (w) {
                 if (lane == 0) {
-                    HpStageRec r;
-                    r.unit = -1; r.info = 0; r.pad0 = r.pad1 = 0;
-                    recs[stage] = r;
+                    recs[stage * 4] = -1;
                     mbar_arrive(full0 + 8 * stage);
                 }
             } else ok = false;
         }
+        if (tr && lane == 0) p.trace[(c * 2 + team) * 8 + 2] = hp_gtime();
         if (!ok && lane == 0) atomicOr(p.ctrl + 1, 1u);
     } else {
-        // ------------------------------------------------------------ consumer warps
-        const int ctid = tid;
-        const int tc = ctid & 255, rl = ctid >> 8;     // 256 x 16 B across a piece; two row lanes
+        // ------------------------------------------------------------ consumer warps of the team
+        const int tc = tid & (kHpTeamThreads - 1);     // 256 x 16 B across a piece
         int stage = 0;
         uint32_t phase = 0, cpar = 0;
+        unsigned int nunit = 0;
         bool ok = true;
+        bool first = true;
         float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
         MinMax2<T> mm;
         mm.init();
         for (;;) {
             if (!mbar_wait_warp(full0 + 8 * stage, phase)) { ok = false; break; }
-            const HpStageRec r = recs[stage];
-            if (r.unit < 0) break;
-            const int u = r.unit;
-            const int np = r.info & 0xFF;
-            const bool last = (r.info & 0x100) != 0;
-            const unsigned int signs = ((unsigned int)r.info) >> 16;
-            const bool isC = u >= UA;
-            const int v = isC ? u - UA : u;
-            const int seg = v / p.m, a = v - seg * p.m;
+            if (tr && first && tc == 0) { p.trace[(c * 2 + team) * 8 + 3] = hp_gtime(); first = false; }
+            const int4 r = *reinterpret_cast<const int4 *>(recs + stage * 4);
+            if (r.x < 0) break;
+            const int a = r.x & 0x3FFFFFFF;
+            const bool isC = (r.x >> 30) != 0;
+            const int seg = r.y;
+            const int np = r.z & 0xFF;
+            const bool last = (r.z & 0x100) != 0;
+            const unsigned int sg = ((unsigned int)r.z) >> 16;
             const int wbytes = isC ? 4 * min(kHpSegC, p.n3 - seg * kHpSegC) : 2 * min(kHpSegA, p.n2 - seg * kHpSegA);
             const bool active = tc * 16 < wbytes;
             if (active) {
                 const unsigned char *sb = ring + (size_t)stage * kHpStageBytes + tc * 16;
-                if (isC) {
+                if (np == kHpPieces) {
+                    // full stage: all loads in flight before the first use
+                    if (isC) {
+                        float4 x[kHpPieces];
 #pragma unroll
-                    for (int q = rl; q < kHpPieces; q += 2) {
+                        for (int q = 0; q < kHpPieces; ++q) x[q] = *reinterpret_cast<const float4 *>(sb + q * kHpPieceBytes);
+#pragma unroll
+                        for (int q = 0; q < kHpPieces; ++q) {
+                            const float f = ((sg >> q) & 1u) ? -1.f : 1.f;
+                            acc[0] = __ffma2_rn(make_float2(f, f), make_float2(x[q].x, x[q].y), acc[0]);
+                            acc[1] = __ffma2_rn(make_float2(f, f), make_float2(x[q].z, x[q].w), acc[1]);
+                        }
+                    } else {
+                        uint4 x[kHpPieces];
+#pragma unroll
+                        for (int q = 0; q < kHpPieces; ++q) x[q] = *reinterpret_cast<const uint4 *>(sb + q * kHpPieceBytes);
+#pragma unroll
+                        for (int q = 0; q < kHpPieces; ++q) {
+                            const uint32_t flip = ((sg >> q) & 1u) ? 0x80008000u : 0u;
+                            x[q].x ^= flip; x[q].y ^= flip; x[q].z ^= flip; x[q].w ^= flip;
+                            add8m<T>(acc, x[q], mm);
+                        }
+                    }
+                } else if (isC) {
+#pragma unroll
+                    for (int q = 0; q < kHpPieces; ++q) {
                         if (q < np) {
                             const float4 x = *reinterpret_cast<const float4 *>(sb + q * kHpPieceBytes);
-                            const float sg = ((signs >> q) & 1u) ? -1.f : 1.f;
-                            acc[0] = __ffma2_rn(make_float2(sg, sg), make_float2(x.x, x.y), acc[0]);
-                            acc[1] = __ffma2_rn(make_float2(sg, sg), make_float2(x.z, x.w), acc[1]);
+                            const float f = ((sg >> q) & 1u) ? -1.f : 1.f;
+                            acc[0] = __ffma2_rn(make_float2(f, f), make_float2(x.x, x.y), acc[0]);
+                            acc[1] = __ffma2_rn(make_float2(f, f), make_float2(x.z, x.w), acc[1]);
                         }
                     }
                 } else {
 #pragma unroll
-                    for (int q = rl; q < kHpPieces; q += 2) {
+                    for (int q = 0; q < kHpPieces; ++q) {
                         if (q < np) {
                             uint4 x = *reinterpret_cast<const uint4 *>(sb + q * kHpPieceBytes);
-                            const uint32_t flip = ((signs >> q) & 1u) ? 0x80008000u : 0u;
+                            const uint32_t flip = ((sg >> q) & 1u) ? 0x80008000u : 0u;
                             x.x ^= flip; x.y ^= flip; x.z ^= flip; x.w ^= flip;
                             add8m<T>(acc, x, mm);
                         }
@@ -228,49 +320,35 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
                 }
             }
             __syncwarp();
-            if ((ctid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
+            if ((tid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
             if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
             if (last) {
-                // unit complete: row lane 1 hands its sums to row lane 0, which stores the row segment
-                if (!hp_consumer_sync(cbar, cpar)) { ok = false; break; }
-                if (rl == 1) {
-                    red4[tc * 2] = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
-                    red4[tc * 2 + 1] = make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y);
-                }
-                if (!hp_consumer_sync(cbar, cpar)) { ok = false; break; }
-                if (rl == 0) {
-                    if (isC) {
-                        if (active) {
-                            const float4 y = red4[tc * 2];
-                            __stcg(reinterpret_cast<float4 *>(p.Tc + (long long)a * p.n3 + seg * kHpSegC + tc * 4),
-                                   make_float4(acc[0].x + y.x, acc[0].y + y.y, acc[1].x + y.z, acc[1].y + y.w));
-                        }
-                    } else {
-                        const int col = seg * kHpSegA + tc * 8;
-                        if (active) {
-                            const float4 y0 = red4[tc * 2], y1 = red4[tc * 2 + 1];
-                            float4 *dst = reinterpret_cast<float4 *>(p.P + (long long)a * p.kpad + col);
-                            __stcg(dst, make_float4(acc[0].x + y0.x, acc[0].y + y0.y, acc[1].x + y0.z, acc[1].y + y0.w));
-                            __stcg(dst + 1, make_float4(acc[2].x + y1.x, acc[2].y + y1.y, acc[3].x + y1.z, acc[3].y + y1.w));
-                        } else if (col < p.kpad) {
-                            // padding columns of the contraction's K extent
-                            float4 *dst = reinterpret_cast<float4 *>(p.P + (long long)a * p.kpad + col);
-                            __stcg(dst, make_float4(0.f, 0.f, 0.f, 0.f));
-                            __stcg(dst + 1, make_float4(0.f, 0.f, 0.f, 0.f));
-                        }
+                // unit complete: every thread stores its columns of the row segment
+                if (isC) {
+                    if (active)
+                        __stcg(reinterpret_cast<float4 *>(p.Tc + (long long)a * p.n3 + seg * kHpSegC + tc * 4),
+                               make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y));
+                } else {
+                    const int col = seg * kHpSegA + tc * 8;
+                    if (active || col < p.kpad) {        // inactive columns below kpad: padding of the contraction's K extent (zeros)
+                        float4 *dst = reinterpret_cast<float4 *>(p.P + (long long)a * p.kpad + col);
+                        __stcg(dst, make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y));
+                        __stcg(dst + 1, make_float4(acc[2].x, acc[2].y, acc[3].x, acc[3].y));
                     }
                 }
+                ++nunit;
                 acc[0] = acc[1] = acc[2] = acc[3] = make_float2(0.f, 0.f);
             }
         }
+        if (tr && tc == 0) { p.trace[(c * 2 + team) * 8 + 4] = hp_gtime(); p.trace[(c * 2 + team) * 8 + 7] = nunit; }
         // max|A| over what this CTA streamed (for tau)
         unsigned int mbits = float_to_bits16<T>(mm.absmax());
         mbits = __reduce_max_sync(0xFFFFFFFFu, mbits);
-        if ((ctid & 31) == 0) {
-            smx[ctid >> 5] = mbits;
+        if ((tid & 31) == 0) {
+            smx[tid >> 5] = mbits;
             if (!ok) atomicOr(p.ctrl + 1, 1u);
         }
-        if (ok && hp_consumer_sync(cbar, cpar) && ctid == 0) {
+        if (ok && hp_consumer_sync(cbar, cpar) && tid == 0) {
             unsigned int r_ = 0;
             for (int w = 0; w < kHpConsumers / 32; ++w) r_ = max(r_, smx[w]);
             p.maxA[c] = r_;
@@ -346,30 +424,64 @@ __device__ __forceinline__ HvMax hv_better(HvMax a, HvMax b)
     return a;
 }
 
-// CTA a computes row a of S.  The last CTA to finish (ticket) combines the per-row statistics in row
-// order and writes the verdict; when some bucket exceeds the clip level it makes the second pass
-// over S alone (fixed order).
+// CTA a computes row a of S: the row of Tc is staged in shared memory (coalesced), thread b folds the
+// columns of bucket b in ascending column order and subtracts the fold from the sum of the split-K
+// partials.  The last CTA to finish (ticket) combines the per-row statistics (fixed tree) and writes
+// the verdict; when some bucket exceeds the clip level it makes the second pass over S alone.
+constexpr int kHvThreads = 256;
+constexpr int kHvRowMax = 49152;      // floats of one row of Tc that fit in shared memory
+
 template <typename T>
-__global__ void __launch_bounds__(256) hp_verdict_kernel(const HvArgs p)
+__global__ void __launch_bounds__(kHvThreads) hp_verdict_kernel(const HvArgs p, int stage_row)
 {
-    __shared__ float ssum[256], sbad[256];
-    __shared__ HvMax smax[256];
+    extern __shared__ __align__(16) float trow_s[];
+    __shared__ float ssum[kHvThreads], sbad[kHvThreads];
+    __shared__ HvMax smax[kHvThreads];
     __shared__ int s_last;
     const int a = blockIdx.x, tid = threadIdx.x;
     const long long mm = (long long)p.m * p.m;
     float lsum = 0.f, lbad = 0.f;
     HvMax lmax = {-1.f, 0x7FFFFFFF};
     const float *trow = p.Tc + (long long)a * p.n3;
-    for (int b = tid; b < p.m; b += 256) {
+    if (stage_row) {
+        if ((p.n3 & 3) == 0) {
+            for (int j = tid * 4; j < p.n3; j += kHvThreads * 4)
+                *reinterpret_cast<float4 *>(trow_s + j) = __ldcg(reinterpret_cast<const float4 *>(trow + j));
+        } else {
+            for (int j = tid; j < p.n3; j += kHvThreads) trow_s[j] = __ldcg(trow + j);
+        }
+        __syncthreads();
+    }
+    for (int b = tid; b < p.m; b += kHvThreads) {
         const long long idx = (long long)a * p.m + b;
-        float ab = __ldcg(p.partAB + idx);
-        for (int s = 1; s < p.ksplit; ++s) ab += __ldcg(p.partAB + (long long)s * mm + idx);
-        float cf = 0.f;
         const int c0 = __ldg(p.colstart + b), c1 = __ldg(p.colstart + b + 1);
-        for (int s = c0; s < c1; ++s) {
-            const uint32_t e = __ldg(p.colperm + s);
-            const float x = __ldcg(trow + (e & 0x7FFFFFFFu));
-            cf += (e >> 31) ? -x : x;
+        float ab = 0.f;
+        for (int s0 = 0; s0 < p.ksplit; s0 += 8) {
+            // eight partials in flight, then added in split order
+            float v[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) v[q] = s0 + q < p.ksplit ? __ldcg(p.partAB + (long long)(s0 + q) * mm + idx) : 0.f;
+#pragma unroll
+            for (int q = 0; q < 8; ++q) ab += v[q];
+        }
+        float cf = 0.f;
+        if (stage_row) {
+            for (int s0 = c0; s0 < c1; s0 += 8) {
+                uint32_t e[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) e[q] = s0 + q < c1 ? __ldg(p.colperm + s0 + q) : 0u;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    const float x = trow_s[e[q] & 0x7FFFFFFFu];
+                    if (s0 + q < c1) cf += (e[q] >> 31) ? -x : x;
+                }
+            }
+        } else {
+            for (int s = c0; s < c1; ++s) {
+                const uint32_t e = __ldg(p.colperm + s);
+                const float x = __ldcg(trow + (e & 0x7FFFFFFFu));
+                cf += (e >> 31) ? -x : x;
+            }
         }
         const float sv = ab - cf;
         p.S[idx] = sv;
@@ -380,7 +492,7 @@ __global__ void __launch_bounds__(256) hp_verdict_kernel(const HvArgs p)
     }
     ssum[tid] = lsum; sbad[tid] = lbad; smax[tid] = lmax;
     __syncthreads();
-    for (int o = 128; o > 0; o >>= 1) {
+    for (int o = kHvThreads / 2; o > 0; o >>= 1) {
         if (tid < o) {
             ssum[tid] += ssum[tid + o];
             sbad[tid] += sbad[tid + o];
@@ -397,45 +509,44 @@ __global__ void __launch_bounds__(256) hp_verdict_kernel(const HvArgs p)
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    // ---- last CTA: statistics in row order
+    // ---- last CTA: per-row records, thread-strided in row order, then a fixed tree
     float tsum = 0.f, tbad = 0.f;
     HvMax tmax = {-1.f, 0x7FFFFFFF};
     unsigned int ma = 0;
-    if (tid == 0) {
-        for (int r = 0; r < p.m; ++r) {
-            const float4 v = __ldcg(p.vstat + r);
-            tsum += v.x;
-            tbad += v.y;
-            tmax = hv_better(tmax, HvMax{v.z, __float_as_int(v.w)});
-        }
-        ssum[0] = tsum; sbad[0] = tbad; smax[0] = tmax;
+    for (int r = tid; r < p.m; r += kHvThreads) {
+        const float4 v = __ldcg(p.vstat + r);
+        tsum += v.x;
+        tbad += v.y;
+        tmax = hv_better(tmax, HvMax{v.z, __float_as_int(v.w)});
     }
-    for (int r = tid; r < p.n_maxA; r += 256) ma = max(ma, __ldcg(p.maxA + r));
+    for (int r = tid; r < p.n_maxA; r += kHvThreads) ma = max(ma, __ldcg(p.maxA + r));
+    ma = __reduce_max_sync(0xFFFFFFFFu, ma);
+    __shared__ unsigned int sma[kHvThreads / 32];
+    if ((tid & 31) == 0) sma[tid >> 5] = ma;
+    ssum[tid] = tsum; sbad[tid] = tbad; smax[tid] = tmax;
     __syncthreads();
+    for (int o = kHvThreads / 2; o > 0; o >>= 1) {
+        if (tid < o) {
+            ssum[tid] += ssum[tid + o];
+            sbad[tid] += sbad[tid + o];
+            smax[tid] = hv_better(smax[tid], smax[tid + o]);
+        }
+        __syncthreads();
+    }
     tsum = ssum[0]; tbad = sbad[0]; tmax = smax[0];
+    ma = 0;
+    for (int w = 0; w < kHvThreads / 32; ++w) ma = max(ma, sma[w]);
     __syncthreads();
-    // max|A| across the per-CTA records
-    {
-        unsigned int *um = reinterpret_cast<unsigned int *>(ssum);
-        um[tid] = ma;
-        __syncthreads();
-        for (int o = 128; o > 0; o >>= 1) {
-            if (tid < o) um[tid] = max(um[tid], um[tid + o]);
-            __syncthreads();
-        }
-        ma = um[0];
-        __syncthreads();
-    }
     const float mean = tsum / (float)mm;
     float clipped = tsum;
     if (!(tmax.v <= 5.f * mean) || tbad > 0.f) {
         // second pass: sum of min(|S|, 5 mean|S|), thread-strided then tree (fixed order)
         const float clip = 5.f * mean;
         float cs = 0.f;
-        for (long long i = tid; i < mm; i += 256) cs += fminf(fabsf(__ldcg(p.S + i)), clip);
+        for (long long i = tid; i < mm; i += kHvThreads) cs += fminf(fabsf(__ldcg(p.S + i)), clip);
         ssum[tid] = cs;
         __syncthreads();
-        for (int o = 128; o > 0; o >>= 1) {
+        for (int o = kHvThreads / 2; o > 0; o >>= 1) {
             if (tid < o) ssum[tid] += ssum[tid + o];
             __syncthreads();
         }
@@ -443,8 +554,7 @@ __global__ void __launch_bounds__(256) hp_verdict_kernel(const HvArgs p)
     }
     if (tid == 0) {
         const float sigma = 1.2533f * (clipped / (float)mm);
-        const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) *
-                          __ldcg(p.maxB);
+        const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) * __ldcg(p.maxB);
         // a bucket sums n1 n3 / m^2 entries of E on average: the per-entry cap grows like the root of that
         const float thr = fminf(tau * p.cap_scale, p.thr_scale * sigma);
         fpsk_probe_result r;
@@ -457,8 +567,9 @@ __global__ void __launch_bounds__(256) hp_verdict_kernel(const HvArgs p)
         r.thr = thr;
         r.tau = tau;
         *p.result = r;
-        p.ctrl[0] = 0;          // ticket and error flag ready for the next call on this workspace
+        p.ctrl[0] = 0;          // ticket, error flag and unit counter ready for the next call on this workspace
         p.ctrl[1] = 0;
+        p.ctrl[2] = 0;
     }
 }
 
@@ -491,7 +602,8 @@ struct HpCache {          // the B side, device memory kept by the caller across
     uint32_t *rowperm;
     int *h2, *v2, *colcount, *colstart;
     uint32_t *colperm;
-    int *first_unit;
+    int *extra_count, *extra_start;
+    int *stages;
     float *Q;
     float *maxB;          // [0] max|B|
     unsigned int *scratch;
@@ -509,7 +621,11 @@ static size_t hp_cache_layout(void *base, long long n1, long long n2, long long 
     t.rowcount = (int *)take((size_t)(m + 1) * 4); t.rowstart = (int *)take((size_t)(m + 1) * 4);
     t.h2 = (int *)take((size_t)n3 * 4); t.v2 = (int *)take((size_t)n3 * 4); t.colperm = (uint32_t *)take((size_t)n3 * 4);
     t.colcount = (int *)take((size_t)(m + 1) * 4); t.colstart = (int *)take((size_t)(m + 1) * 4);
-    t.first_unit = (int *)take((size_t)(sms + 1) * 4);
+    const size_t units = (size_t)m * (pl.segsA + pl.segsC);
+    t.extra_count = (int *)take((units + 1) * 4);
+    t.extra_start = (int *)take((units + 1) * 4);
+    // one chunk per unit, plus continuation chunks: at most (stages of all units) / 8 of them
+    t.stages = (int *)take((units + (size_t)(pl.segsA + pl.segsC) * ((size_t)n1 / (kHpPieces * kHpChunk) + (size_t)m / kHpChunk + 1)) * kHpChunk * 64);
     t.Q = (float *)take((size_t)pl.kpad * pl.npad * 4);
     t.maxB = (float *)take(256);
     t.scratch = (unsigned int *)take(256);
@@ -522,6 +638,7 @@ struct HpWork {           // per-call scratch
     unsigned int *maxA;
     float4 *vstat;
     float *P, *Tc, *partAB, *S;
+    unsigned long long *trace;
 };
 
 static size_t hp_work_layout(void *base, long long n1, long long n2, long long n3, int m, int sms, HpWork *w)
@@ -539,6 +656,7 @@ static size_t hp_work_layout(void *base, long long n1, long long n2, long long n
     t.Tc = (float *)take((size_t)m * n3 * 4);
     t.partAB = (float *)take((size_t)pl.ksplit * m * m * 4);
     t.S = (float *)take((size_t)m * m * 4);
+    t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 128);       // 8 stamps per team
     if (w) *w = t;
     return off;
 }
@@ -569,9 +687,12 @@ static HpArgs hp_args(const void *A, long long lda, const float *C, long long ld
     a.C = C; a.ldc = ldc;
     a.n1 = (int)n1; a.n2 = (int)n2; a.n3 = (int)n3; a.m = m; a.kpad = pl.kpad;
     a.segsA = pl.segsA; a.segsC = pl.segsC;
-    a.rowperm = c.rowperm; a.rowstart = c.rowstart; a.first_unit = c.first_unit;
+    a.rowperm = c.rowperm; a.rowstart = c.rowstart; a.stages = c.stages;
     a.P = w ? w->P : nullptr; a.Tc = w ? w->Tc : nullptr;
     a.maxA = w ? w->maxA : nullptr; a.ctrl = w ? w->ctrl : nullptr;
+    a.trace = w ? w->trace : nullptr;
+    static const bool trace_env = getenv("FPSK_HPROBE_TRACE") != nullptr;
+    a.trace_on = trace_env ? 1 : 0;
     return a;
 }
 
@@ -593,7 +714,12 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
     rc = max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
     if (rc != FPSK_OK) return rc;
     const HpArgs a = hp_args(nullptr, 0, nullptr, 0, n1, n2, n3, m, pl, c, nullptr);
-    hp_partition_kernel<<<(sms + 1 + 127) / 128, 128, 0, st>>>(a, sms, c.first_unit);
+    const int units = m * (pl.segsA + pl.segsC);
+    hp_count_chunks_kernel<<<(units + 255) / 256, 256, 0, st>>>(a, c.extra_count);
+    FPSK_LAUNCH_CHECK();
+    rc = exclusive_scan_launch(c.extra_count, units, c.extra_start, st);
+    if (rc != FPSK_OK) return rc;
+    hp_fill_stages_kernel<<<(units + 255) / 256, 256, 0, st>>>(a, c.extra_start, c.stages);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
@@ -647,8 +773,20 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);
     v.S = d_S ? d_S : w.S;
     v.vstat = w.vstat; v.ctrl = w.ctrl; v.result = d_result;
-    if (dtype == FPSK_FP16) hp_verdict_kernel<__half><<<m, 256, 0, st>>>(v);
-    else hp_verdict_kernel<__nv_bfloat16><<<m, 256, 0, st>>>(v);
+    const int stage_row = n3 <= kHvRowMax ? 1 : 0;
+    const size_t vsmem = stage_row ? (size_t)((n3 + 3) / 4 * 4) * 4 : 0;
+    if (vsmem > 48 * 1024) {
+        static std::once_flag once2;
+        static cudaError_t attr_err2 = cudaSuccess;
+        std::call_once(once2, [] {
+            attr_err2 = cudaFuncSetAttribute(hp_verdict_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHvRowMax * 4);
+            if (attr_err2 == cudaSuccess)
+                attr_err2 = cudaFuncSetAttribute(hp_verdict_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHvRowMax * 4);
+        });
+        FPSK_CUDA_OK(attr_err2);
+    }
+    if (dtype == FPSK_FP16) hp_verdict_kernel<__half><<<m, kHvThreads, vsmem, st>>>(v, stage_row);
+    else hp_verdict_kernel<__nv_bfloat16><<<m, kHvThreads, vsmem, st>>>(v, stage_row);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }

@@ -547,6 +547,13 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     return FPSK_OK;
 }
 
+fpsk_status exclusive_scan_launch(const int *count, int n, int *start, cudaStream_t st)
+{
+    scan_kernel<<<1, 1024, 0, st>>>(count, n, start);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
 fpsk_status contraction_launch(const float *P, const float *Q, float *part, int M, int N, int K, int lda, int ldb,
                                int ksplit, int kchunk, int tile, cudaStream_t st)
 {

@@ -42,6 +42,8 @@ fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, in
                             int *count, int *start, uint32_t *perm, cudaStream_t st);
 fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
                            SketchWs &w, cudaStream_t st, float *S, float *R, float *T);
+// start[0..n] = exclusive prefix sums of count[0..n)  (one CTA, any n)
+fpsk_status exclusive_scan_launch(const int *count, int n, int *start, cudaStream_t st);
 // one FP32 contraction part[ks] = P[:, ks-th K chunk] Q[ks-th K chunk, :]  (M x K by K x N, K a multiple of 16)
 fpsk_status contraction_launch(const float *P, const float *Q, float *part, int M, int N, int K, int lda, int ldb,
                                int ksplit, int kchunk, int tile, cudaStream_t st);
