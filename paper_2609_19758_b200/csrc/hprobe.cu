@@ -7,11 +7,12 @@
 //   hp_count_chunks_kernel, hp_fill_stages_kernel
 //                           the work list: for every (matrix, column segment, row bucket) unit the ring
 //                           stages (rows, signs) that stream it
-//   hp_stream_kernel        P = H1 A (m x n2) and Tc = H1 C (m x n3): signed row-bucket sums, one
-//                           persistent CTA per SM, rows gathered by bulk copies into a shared-memory ring
+//   hp_stream_kernel        P = H1 A (m x n2) and H1 C H2^T per column segment: signed row-bucket sums
+//                           (and the column fold for C), one persistent CTA per SM, rows gathered by
+//                           bulk copies into shared-memory rings
 //   hp_rowsum_plain_kernel  the same sums with plain loads (inputs that bulk copies cannot address)
 //   sgemm (sketch.cu)       P Q as split-K partials, FP32 FMA
-//   hp_verdict_kernel       S = sum of partials - Tc H2^T (column fold), statistics, verdict
+//   hp_combine_kernel       S = sum of split-K partials - sum of segment partials, statistics, verdict
 // Every sum has a fixed order (no float atomics): results are bit-reproducible.
 #include "sketch.cuh"
 #include "stream_pipe.cuh"
@@ -31,10 +32,11 @@ constexpr int kHpStageBytes = 16384;
 constexpr int kHpPieceBytes = 4096;               // one row of one column segment
 constexpr int kHpPieces = kHpStageBytes / kHpPieceBytes;
 static_assert(kHpPieces == 4, "a stage record's row indices sit in one 16-byte lane word");
-static_assert(2 * 2 * kHpStages * 8 + 8 <= 256, "barrier block");
+static_assert(2 * 2 * kHpStages * 8 + 8 + 16 <= 256, "barrier block");
 constexpr int kHpSegA = kHpPieceBytes / 2;        // columns of A per segment
 constexpr int kHpSegC = kHpPieceBytes / 4;        // columns of C per segment
-constexpr int kHpSmem = 2 * kHpStages * kHpStageBytes + 256 /*barriers*/ + 2 * kHpStages * 16 /*stage records*/;
+constexpr int kHpFoldBytes = 2 * 2 * kHpSegC * 4; // per team, two buffers of one segment of row-bucket sums of C
+constexpr int kHpSmem = 2 * kHpStages * kHpStageBytes + kHpFoldBytes + 256 /*barriers*/ + 2 * kHpStages * 16 /*stage records*/;
 
 struct HpArgs {
     const unsigned short *A;
@@ -48,9 +50,12 @@ struct HpArgs {
     const int *stages;             // chunks of 8 stage records, 16 ints per record:
                                    //   [0] bucket | isC << 30   [1] segment   [2] pieces | last-of-unit << 8 | signs << 16
                                    //   [4 .. 4 + pieces) row indices;  [15] of the chunk's last record: next chunk of the unit
-                                   // chunk u is the first chunk of unit u; longer units continue in chunks >= units
+                                   // chunk k is the first chunk of the k-th unit handed out; longer units continue in chunks >= units
+    const uint32_t *segperm;       // per column segment of C: its columns (local index, bit 31 = sign -1) sorted by bucket
+    const int *segstart;           // [segsC][m + 1] bucket boundaries in segperm, relative to the segment
     float *P;                      // m x kpad
-    float *Tc;                     // m x n3
+    float *Tc;                     // m x n3 (plain-load path only)
+    float *partC;                  // [segsC][m*m]: H1 C H2^T restricted to the columns of one segment
     unsigned int *maxA;            // per CTA: bits of max|A| over what it streamed
     unsigned int *ctrl;            // [0] verdict ticket, [1] error flag, [2] next unit to hand out
     int trace_on;
@@ -63,18 +68,41 @@ struct HpArgs {
 // warp-wide 16-byte load brings a whole chunk.
 constexpr int kHpChunk = 8;
 
-__global__ void hp_count_chunks_kernel(HpArgs p, int *extra)
+// Buckets ranked by row count, largest first (ties by index).  Units are handed out in rank order, so
+// the last units to go out are the smallest and all teams finish close together.
+__global__ void hp_rank_kernel(const int *rowstart, int m, int *rank)
 {
-    const int u = blockIdx.x * blockDim.x + threadIdx.x;
-    const int U = p.m * (p.segsA + p.segsC);
-    if (u >= U) return;
-    const int a = u % p.m;
-    const int rows = __ldg(p.rowstart + a + 1) - __ldg(p.rowstart + a);
-    const int nst = rows > 0 ? (rows + kHpPieces - 1) / kHpPieces : 1;
-    extra[u] = (nst + kHpChunk - 1) / kHpChunk - 1;        // chunks beyond the first
+    const int a = blockIdx.x * blockDim.x + threadIdx.x;
+    if (a >= m) return;
+    const int rows = __ldg(rowstart + a + 1) - __ldg(rowstart + a);
+    int r = 0;
+    for (int o = 0; o < m; ++o) {
+        const int ro = __ldg(rowstart + o + 1) - __ldg(rowstart + o);
+        r += (ro > rows) || (ro == rows && o < a);
+    }
+    rank[a] = r;
 }
 
-__global__ void hp_fill_stages_kernel(HpArgs p, const int *extra_start, int *stages)
+// position of unit (isC, seg, a) in the hand-out order
+__device__ __forceinline__ int hp_unit_pos(const HpArgs &p, const int *rank, bool isC, int seg, int a)
+{
+    return __ldg(rank + a) * (p.segsA + p.segsC) + (isC ? p.segsA + seg : seg);
+}
+
+__global__ void hp_count_chunks_kernel(HpArgs p, const int *rank, int *extra)
+{
+    const int u = blockIdx.x * blockDim.x + threadIdx.x;
+    const int UA = p.m * p.segsA, U = UA + p.m * p.segsC;
+    if (u >= U) return;
+    const bool isC = u >= UA;
+    const int v = isC ? u - UA : u;
+    const int seg = v / p.m, a = v - seg * p.m;
+    const int rows = __ldg(p.rowstart + a + 1) - __ldg(p.rowstart + a);
+    const int nst = rows > 0 ? (rows + kHpPieces - 1) / kHpPieces : 1;
+    extra[hp_unit_pos(p, rank, isC, seg, a)] = (nst + kHpChunk - 1) / kHpChunk - 1;        // chunks beyond the first
+}
+
+__global__ void hp_fill_stages_kernel(HpArgs p, const int *rank, const int *extra_start, int *stages)
 {
     const int u = blockIdx.x * blockDim.x + threadIdx.x;
     const int UA = p.m * p.segsA, U = UA + p.m * p.segsC;
@@ -85,9 +113,10 @@ __global__ void hp_fill_stages_kernel(HpArgs p, const int *extra_start, int *sta
     const int s0 = __ldg(p.rowstart + a), s1 = __ldg(p.rowstart + a + 1);
     const int nst = s1 > s0 ? (s1 - s0 + kHpPieces - 1) / kHpPieces : 1;
     const int nchunk = (nst + kHpChunk - 1) / kHpChunk;
+    const int up = hp_unit_pos(p, rank, isC, seg, a);
     int pos = s0;
     for (int k = 0; k < nchunk; ++k) {
-        const int ci = k == 0 ? u : U + extra_start[u] + (k - 1);
+        const int ci = k == 0 ? up : U + extra_start[up] + (k - 1);
         for (int j = 0; j < kHpChunk; ++j) {
             int *rec = stages + ((long long)ci * kHpChunk + j) * 16;
             const int st = k * kHpChunk + j;
@@ -105,8 +134,41 @@ __global__ void hp_fill_stages_kernel(HpArgs p, const int *extra_start, int *sta
                 rec[2] = np | (st == nst - 1 ? 0x100 : 0) | (int)(signs << 16);
                 pos += np;
             }
-            if (j == kHpChunk - 1) rec[15] = k + 1 < nchunk ? U + extra_start[u] + k : -1;
+            if (j == kHpChunk - 1) rec[15] = k + 1 < nchunk ? U + extra_start[up] + k : -1;
         }
+    }
+}
+
+// Column lists of one segment of C (CTA = segment): the segment's columns sorted by bucket, stable in
+// the column index, so that a bucket's fold adds its columns in ascending order.
+__global__ void __launch_bounds__(256) hp_segment_lists_kernel(const int *h2, const int *v2, int n3, int m, uint32_t *segperm,
+                                                               int *segstart)
+{
+    __shared__ int sh[kHpSegC];
+    extern __shared__ int cnt[];                // m + 1
+    const int seg = blockIdx.x;
+    const int c0 = seg * kHpSegC, w = min(kHpSegC, n3 - c0);
+    for (int j = threadIdx.x; j < w; j += blockDim.x) sh[j] = h2[c0 + j];
+    for (int b = threadIdx.x; b <= m; b += blockDim.x) cnt[b] = 0;
+    __syncthreads();
+    for (int j = threadIdx.x; j < w; j += blockDim.x) atomicAdd(&cnt[sh[j]], 1);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int run = 0;
+        for (int b = 0; b < m; ++b) {
+            const int n = cnt[b];
+            cnt[b] = run;
+            run += n;
+        }
+        cnt[m] = run;
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b <= m; b += blockDim.x) segstart[(long long)seg * (m + 1) + b] = cnt[b];
+    for (int j = threadIdx.x; j < w; j += blockDim.x) {
+        const int b = sh[j];
+        int rank = 0;
+        for (int i = 0; i < j; ++i) rank += (sh[i] == b);
+        segperm[c0 + cnt[b] + rank] = (uint32_t)j | (v2[c0 + j] < 0 ? 0x80000000u : 0u);
     }
 }
 
@@ -118,6 +180,16 @@ __device__ __forceinline__ bool hp_consumer_sync(uint32_t cbar, uint32_t &cpar)
     if ((threadIdx.x & 31) == 0) mbar_arrive(cbar);
     const bool w = mbar_wait_warp(cbar, cpar);
     cpar ^= 1u;
+    return w;
+}
+
+// The same over the eight consumer warps of one team.
+__device__ __forceinline__ bool hp_team_sync(uint32_t tbar, uint32_t &tpar)
+{
+    __syncwarp();
+    if ((threadIdx.x & 31) == 0) mbar_arrive(tbar);
+    const bool w = mbar_wait_warp(tbar, tpar);
+    tpar ^= 1u;
     return w;
 }
 
@@ -141,8 +213,9 @@ template <typename T>
 __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p)
 {
     extern __shared__ __align__(128) unsigned char smem[];
-    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + 2 * kHpStages * kHpStageBytes);
-    int *recs_all = reinterpret_cast<int *>(smem + 2 * kHpStages * kHpStageBytes + 256);
+    float *fold_all = reinterpret_cast<float *>(smem + 2 * kHpStages * kHpStageBytes);
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + 2 * kHpStages * kHpStageBytes + kHpFoldBytes);
+    int *recs_all = reinterpret_cast<int *>(smem + 2 * kHpStages * kHpStageBytes + kHpFoldBytes + 256);
     __shared__ unsigned int smx[kHpConsumers / 32];
     const int c = blockIdx.x;
     const int tid = threadIdx.x;
@@ -152,6 +225,7 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
     int *recs = recs_all + team * kHpStages * 4;
     const uint32_t full0 = smem_u32(bars) + team * (2 * kHpStages * 8), empty0 = full0 + kHpStages * 8;
     const uint32_t cbar = smem_u32(bars) + 2 * (2 * kHpStages * 8);
+    const uint32_t tbar = cbar + 8 + 8 * team;           // barrier over the team's consumer warps
     if (tid == 0) {
         for (int s = 0; s < 2 * kHpStages; ++s) {
             const int tm = s / kHpStages, ss = s % kHpStages;
@@ -159,6 +233,8 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
             mbar_init(smem_u32(bars) + tm * (2 * kHpStages * 8) + kHpStages * 8 + 8 * ss, kHpTeamThreads / 32);
         }
         mbar_init(cbar, kHpConsumers / 32);
+        mbar_init(cbar + 8, kHpTeamThreads / 32);
+        mbar_init(cbar + 16, kHpTeamThreads / 32);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -252,10 +328,14 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
         // ------------------------------------------------------------ consumer warps of the team
         const int tc = tid & (kHpTeamThreads - 1);     // 256 x 16 B across a piece
         int stage = 0;
-        uint32_t phase = 0, cpar = 0;
-        unsigned int nunit = 0;
+        uint32_t phase = 0, cpar = 0, tpar = 0;
+        unsigned int nunit = 0, ncunit = 0;
         bool ok = true;
         bool first = true;
+        bool fresh = true;                             // the next stage opens a unit
+        int fs0 = 0, fs1 = 0;                          // this thread's first bucket in the open C unit's segment list
+        float *fold = fold_all + team * (2 * kHpSegC);
+        const long long mm2 = (long long)p.m * p.m;
         float2 acc[4] = {{0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}, {0.f, 0.f}};
         MinMax2<T> mm;
         mm.init();
@@ -272,6 +352,12 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
             const unsigned int sg = ((unsigned int)r.z) >> 16;
             const int wbytes = isC ? 4 * min(kHpSegC, p.n3 - seg * kHpSegC) : 2 * min(kHpSegA, p.n2 - seg * kHpSegA);
             const bool active = tc * 16 < wbytes;
+            if (fresh && isC && tc < p.m) {
+                // needed when the unit is complete: in flight while its rows stream
+                fs0 = __ldg(p.segstart + (long long)seg * (p.m + 1) + tc);
+                fs1 = __ldg(p.segstart + (long long)seg * (p.m + 1) + tc + 1);
+            }
+            fresh = false;
             if (active) {
                 const unsigned char *sb = ring + (size_t)stage * kHpStageBytes + tc * 16;
                 if (np == kHpPieces) {
@@ -323,11 +409,36 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
             if ((tid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
             if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
             if (last) {
-                // unit complete: every thread stores its columns of the row segment
+                // unit complete
                 if (isC) {
-                    if (active)
-                        __stcg(reinterpret_cast<float4 *>(p.Tc + (long long)a * p.n3 + seg * kHpSegC + tc * 4),
-                               make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y));
+                    // the segment's signed row-bucket sums go through shared memory; thread b then folds the
+                    // columns of bucket b (ascending) into partC[seg][a][b].  Two buffers: the barrier of
+                    // the next C unit separates this unit's reads from the writes of the one after.
+                    float *tb = fold + (ncunit & 1u) * kHpSegC;
+                    if (active) *reinterpret_cast<float4 *>(tb + tc * 4) = make_float4(acc[0].x, acc[0].y, acc[1].x, acc[1].y);
+                    if (!hp_team_sync(tbar, tpar)) { ok = false; break; }
+                    const uint32_t *sp = p.segperm + (long long)seg * kHpSegC;
+                    float *dst = p.partC + (long long)seg * mm2 + (long long)a * p.m;
+                    for (int b = tc; b < p.m; b += kHpTeamThreads) {
+                        int s0 = fs0, s1 = fs1;
+                        if (b != tc) {
+                            s0 = __ldg(p.segstart + (long long)seg * (p.m + 1) + b);
+                            s1 = __ldg(p.segstart + (long long)seg * (p.m + 1) + b + 1);
+                        }
+                        float cf = 0.f;
+                        for (int s = s0; s < s1; s += 4) {
+                            uint32_t e[4];
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) e[q] = s + q < s1 ? __ldg(sp + s + q) : 0u;
+#pragma unroll
+                            for (int q = 0; q < 4; ++q) {
+                                const float x = tb[e[q] & 0x7FFFFFFFu];
+                                if (s + q < s1) cf += (e[q] >> 31) ? -x : x;
+                            }
+                        }
+                        __stcg(dst + b, cf);
+                    }
+                    ++ncunit;
                 } else {
                     const int col = seg * kHpSegA + tc * 8;
                     if (active || col < p.kpad) {        // inactive columns below kpad: padding of the contraction's K extent (zeros)
@@ -337,6 +448,7 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
                     }
                 }
                 ++nunit;
+                fresh = true;
                 acc[0] = acc[1] = acc[2] = acc[3] = make_float2(0.f, 0.f);
             }
         }
@@ -395,22 +507,42 @@ __global__ void __launch_bounds__(256) hp_rowsum_plain_kernel(const HpArgs p)
     }
 }
 
+// partC from Tc for the plain-load path: CTA (bucket row a, segment), thread b folds the segment's
+// columns of bucket b in ascending order (same order as the streaming kernel).
+__global__ void __launch_bounds__(256) hp_fold_plain_kernel(const HpArgs p)
+{
+    const int a = blockIdx.x, seg = blockIdx.y;
+    const long long mm = (long long)p.m * p.m;
+    const float *trow = p.Tc + (long long)a * p.n3 + (long long)seg * kHpSegC;
+    const uint32_t *sp = p.segperm + (long long)seg * kHpSegC;
+    for (int b = threadIdx.x; b < p.m; b += blockDim.x) {
+        const int s0 = __ldg(p.segstart + (long long)seg * (p.m + 1) + b), s1 = __ldg(p.segstart + (long long)seg * (p.m + 1) + b + 1);
+        float cf = 0.f;
+        for (int s = s0; s < s1; ++s) {
+            const uint32_t e = __ldg(sp + s);
+            const float x = trow[e & 0x7FFFFFFFu];
+            cf += (e >> 31) ? -x : x;
+        }
+        p.partC[(long long)seg * mm + (long long)a * p.m + b] = cf;
+    }
+}
+
 // ---------------------------------------------------------------- combine + verdict
 struct HvArgs {
     const float *partAB;     // [ksplit][m*m]
     int ksplit;
-    const float *Tc;         // m x n3
-    const uint32_t *colperm; // columns sorted by bucket; bit 31 = sign -1
-    const int *colstart;     // [m + 1]
+    const float *partC;      // [nseg][m*m]
+    int nseg;
     int m, n1, n2, n3;
     const unsigned int *maxA;
     int n_maxA;
-    const float *maxB;           // [1] max|B|
+    const float *maxB;       // [1] max|B|
     float thr_scale;         // mu sqrt(2 ln max(m^2, 2))
     float cap_scale;         // sqrt(n1 n3 / m^2)
     float *S;                // m*m
     float4 *vstat;           // per CTA: sum|S|, nonfinite count, max, argmax (as int bits)
-    unsigned int *ctrl;      // [0] ticket, [1] error flag
+    float *cstat;            // per CTA: sum of min(|S|, clip)
+    unsigned int *ctrl;      // [0] ticket, [1] error flag, [2] unit counter of the streaming kernel, [3] statistics published
     fpsk_probe_result *result;
 };
 
@@ -424,152 +556,155 @@ __device__ __forceinline__ HvMax hv_better(HvMax a, HvMax b)
     return a;
 }
 
-// CTA a computes row a of S: the row of Tc is staged in shared memory (coalesced), thread b folds the
-// columns of bucket b in ascending column order and subtracts the fold from the sum of the split-K
-// partials.  The last CTA to finish (ticket) combines the per-row statistics (fixed tree) and writes
-// the verdict; when some bucket exceeds the clip level it makes the second pass over S alone.
-constexpr int kHvThreads = 256;
-constexpr int kHvRowMax = 49152;      // floats of one row of Tc that fit in shared memory
+constexpr int kHvThreads = 512;
+constexpr int kHvWarps = kHvThreads / 32;
+constexpr int kHvMaxGrid = 512;
 
-template <typename T>
-__global__ void __launch_bounds__(kHvThreads) hp_verdict_kernel(const HvArgs p, int stage_row)
+struct HvStat {
+    float sum, bad;
+    HvMax mx;
+};
+__device__ __forceinline__ HvStat hv_join(HvStat a, HvStat b)
 {
-    extern __shared__ __align__(16) float trow_s[];
-    __shared__ float ssum[kHvThreads], sbad[kHvThreads];
-    __shared__ HvMax smax[kHvThreads];
-    __shared__ int s_last;
-    const int a = blockIdx.x, tid = threadIdx.x;
-    const long long mm = (long long)p.m * p.m;
-    float lsum = 0.f, lbad = 0.f;
-    HvMax lmax = {-1.f, 0x7FFFFFFF};
-    const float *trow = p.Tc + (long long)a * p.n3;
-    if (stage_row) {
-        if ((p.n3 & 3) == 0) {
-            for (int j = tid * 4; j < p.n3; j += kHvThreads * 4)
-                *reinterpret_cast<float4 *>(trow_s + j) = __ldcg(reinterpret_cast<const float4 *>(trow + j));
-        } else {
-            for (int j = tid; j < p.n3; j += kHvThreads) trow_s[j] = __ldcg(trow + j);
-        }
-        __syncthreads();
+    HvStat r;
+    r.sum = a.sum + b.sum;
+    r.bad = a.bad + b.bad;
+    r.mx = hv_better(a.mx, b.mx);
+    return r;
+}
+// Block-wide combination in a fixed shape (butterfly inside a warp, then the warps in order): every
+// thread returns the same value.  `slot` must hold kHvWarps entries; two uses need two slot arrays
+// or a barrier between them.
+__device__ __forceinline__ HvStat hv_block_join(HvStat v, HvStat *slot)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        HvStat w;
+        w.sum = __shfl_xor_sync(0xFFFFFFFFu, v.sum, o);
+        w.bad = __shfl_xor_sync(0xFFFFFFFFu, v.bad, o);
+        w.mx.v = __shfl_xor_sync(0xFFFFFFFFu, v.mx.v, o);
+        w.mx.i = __shfl_xor_sync(0xFFFFFFFFu, v.mx.i, o);
+        // lower lane first: the same operand order in both partners
+        v = (threadIdx.x & o) ? hv_join(w, v) : hv_join(v, w);
     }
-    for (int b = tid; b < p.m; b += kHvThreads) {
-        const long long idx = (long long)a * p.m + b;
-        const int c0 = __ldg(p.colstart + b), c1 = __ldg(p.colstart + b + 1);
+    if ((threadIdx.x & 31) == 0) slot[threadIdx.x >> 5] = v;
+    __syncthreads();
+    HvStat r = slot[0];
+#pragma unroll
+    for (int w = 1; w < kHvWarps; ++w) r = hv_join(r, slot[w]);
+    return r;
+}
+
+// Cooperative grid, CTA c owns a contiguous range of the m^2 buckets.
+//   1. S = (split-K partials, in split order) - (segment partials of H1 C H2^T, in segment order);
+//      per-CTA sum|S|, count of non-finite entries, max and argmax; publish (release) and wait
+//      (bounded) for all CTAs.
+//   2. every CTA forms the same total in the same order, hence the same clip level 5 mean|S|; when
+//      some bucket exceeds it, it re-reads its own range of S (still in L2) for the clipped sum.
+//   3. the last CTA to finish (ticket) adds the clipped sums in CTA order and writes the verdict.
+template <typename T>
+__global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
+{
+    __shared__ HvStat slot0[kHvWarps], slot1[kHvWarps], slot2[kHvWarps], slot3[kHvWarps];
+    __shared__ unsigned int sma[kHvWarps];
+    __shared__ int s_flag;
+    const int c = blockIdx.x, G = gridDim.x, tid = threadIdx.x;
+    const long long mm = (long long)p.m * p.m;
+    // ranges in units of 4 buckets (the tail CTA takes the remainder of an m^2 that is not a multiple of 4)
+    const long long q4 = (mm + 3) / 4;
+    const long long i0 = 4 * (q4 * c / G), i1 = min(mm, 4 * (q4 * (c + 1) / G));
+    HvStat l = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
+    for (long long i = i0 + tid; i < i1; i += kHvThreads) {
         float ab = 0.f;
         for (int s0 = 0; s0 < p.ksplit; s0 += 8) {
-            // eight partials in flight, then added in split order
-            float v[8];
+            float v[8];                 // eight partials in flight, then added in split order
 #pragma unroll
-            for (int q = 0; q < 8; ++q) v[q] = s0 + q < p.ksplit ? __ldcg(p.partAB + (long long)(s0 + q) * mm + idx) : 0.f;
+            for (int q = 0; q < 8; ++q) v[q] = s0 + q < p.ksplit ? __ldcg(p.partAB + (long long)(s0 + q) * mm + i) : 0.f;
 #pragma unroll
             for (int q = 0; q < 8; ++q) ab += v[q];
         }
         float cf = 0.f;
-        if (stage_row) {
-            for (int s0 = c0; s0 < c1; s0 += 8) {
-                uint32_t e[8];
+        for (int s0 = 0; s0 < p.nseg; s0 += 8) {
+            float v[8];
 #pragma unroll
-                for (int q = 0; q < 8; ++q) e[q] = s0 + q < c1 ? __ldg(p.colperm + s0 + q) : 0u;
+            for (int q = 0; q < 8; ++q) v[q] = s0 + q < p.nseg ? __ldcg(p.partC + (long long)(s0 + q) * mm + i) : 0.f;
 #pragma unroll
-                for (int q = 0; q < 8; ++q) {
-                    const float x = trow_s[e[q] & 0x7FFFFFFFu];
-                    if (s0 + q < c1) cf += (e[q] >> 31) ? -x : x;
-                }
-            }
-        } else {
-            for (int s = c0; s < c1; ++s) {
-                const uint32_t e = __ldg(p.colperm + s);
-                const float x = __ldcg(trow + (e & 0x7FFFFFFFu));
-                cf += (e >> 31) ? -x : x;
-            }
+            for (int q = 0; q < 8; ++q) cf += v[q];
         }
         const float sv = ab - cf;
-        p.S[idx] = sv;
+        __stcg(p.S + i, sv);
         const float av = fabsf(sv);
-        lsum += av;
-        if (!(av <= 3.4028234663852886e38f)) lbad += 1.f;          // Inf or NaN
-        else lmax = hv_better(lmax, HvMax{av, (int)idx});
+        l.sum += av;
+        if (!(av <= 3.4028234663852886e38f)) l.bad += 1.f;          // Inf or NaN
+        else l.mx = hv_better(l.mx, HvMax{av, (int)i});
     }
-    ssum[tid] = lsum; sbad[tid] = lbad; smax[tid] = lmax;
+    l = hv_block_join(l, slot0);
+    if (tid == 0) {
+        __stcg(p.vstat + c, make_float4(l.sum, l.bad, l.mx.v, __int_as_float(l.mx.i)));
+        red_release_add(p.ctrl + 3);
+        s_flag = bounded_wait_ge(p.ctrl + 3, (unsigned)G) ? 1 : 0;
+        if (!s_flag) atomicOr(p.ctrl + 1, 1u);
+    }
     __syncthreads();
-    for (int o = kHvThreads / 2; o > 0; o >>= 1) {
-        if (tid < o) {
-            ssum[tid] += ssum[tid + o];
-            sbad[tid] += sbad[tid + o];
-            smax[tid] = hv_better(smax[tid], smax[tid + o]);
+    const bool ok = s_flag != 0;
+    // ---- the same totals in every CTA: records in CTA order, thread-strided, then the fixed shape
+    HvStat t = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
+    if (ok) {
+        for (int r = tid; r < G; r += kHvThreads) {
+            const float4 v = __ldcg(p.vstat + r);
+            t = hv_join(t, HvStat{v.x, v.y, {v.z, __float_as_int(v.w)}});
         }
-        __syncthreads();
+    }
+    t = hv_block_join(t, slot1);
+    const float mean = t.sum / (float)mm;
+    const bool slow = !(t.mx.v <= 5.f * mean) || t.bad > 0.f;
+    if (slow) {
+        const float clip = 5.f * mean;
+        HvStat cs = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
+        for (long long i = i0 + tid; i < i1; i += kHvThreads) cs.sum += fminf(fabsf(__ldcg(p.S + i)), clip);
+        cs = hv_block_join(cs, slot2);
+        if (tid == 0) __stcg(p.cstat + c, cs.sum);
     }
     if (tid == 0) {
-        p.vstat[a] = make_float4(ssum[0], sbad[0], smax[0].v, __int_as_float(smax[0].i));
         __threadfence();
-        const unsigned int t = atom_acq_rel_add(p.ctrl + 0);
-        s_last = (t == (unsigned int)(gridDim.x - 1)) ? 1 : 0;
+        const unsigned int tk = atom_acq_rel_add(p.ctrl + 0);
+        s_flag = (tk == (unsigned int)(G - 1)) ? 1 : 0;
     }
     __syncthreads();
-    if (!s_last) return;
+    if (!s_flag) return;
     __threadfence();
-    // ---- last CTA: per-row records, thread-strided in row order, then a fixed tree
-    float tsum = 0.f, tbad = 0.f;
-    HvMax tmax = {-1.f, 0x7FFFFFFF};
-    unsigned int ma = 0;
-    for (int r = tid; r < p.m; r += kHvThreads) {
-        const float4 v = __ldcg(p.vstat + r);
-        tsum += v.x;
-        tbad += v.y;
-        tmax = hv_better(tmax, HvMax{v.z, __float_as_int(v.w)});
+    // ---- last CTA
+    float clipped = t.sum;
+    if (slow) {
+        HvStat cs = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
+        for (int r = tid; r < G; r += kHvThreads) cs.sum += __ldcg(p.cstat + r);
+        cs = hv_block_join(cs, slot3);
+        clipped = cs.sum;
     }
+    unsigned int ma = 0;
     for (int r = tid; r < p.n_maxA; r += kHvThreads) ma = max(ma, __ldcg(p.maxA + r));
     ma = __reduce_max_sync(0xFFFFFFFFu, ma);
-    __shared__ unsigned int sma[kHvThreads / 32];
     if ((tid & 31) == 0) sma[tid >> 5] = ma;
-    ssum[tid] = tsum; sbad[tid] = tbad; smax[tid] = tmax;
     __syncthreads();
-    for (int o = kHvThreads / 2; o > 0; o >>= 1) {
-        if (tid < o) {
-            ssum[tid] += ssum[tid + o];
-            sbad[tid] += sbad[tid + o];
-            smax[tid] = hv_better(smax[tid], smax[tid + o]);
-        }
-        __syncthreads();
-    }
-    tsum = ssum[0]; tbad = sbad[0]; tmax = smax[0];
-    ma = 0;
-    for (int w = 0; w < kHvThreads / 32; ++w) ma = max(ma, sma[w]);
-    __syncthreads();
-    const float mean = tsum / (float)mm;
-    float clipped = tsum;
-    if (!(tmax.v <= 5.f * mean) || tbad > 0.f) {
-        // second pass: sum of min(|S|, 5 mean|S|), thread-strided then tree (fixed order)
-        const float clip = 5.f * mean;
-        float cs = 0.f;
-        for (long long i = tid; i < mm; i += kHvThreads) cs += fminf(fabsf(__ldcg(p.S + i)), clip);
-        ssum[tid] = cs;
-        __syncthreads();
-        for (int o = kHvThreads / 2; o > 0; o >>= 1) {
-            if (tid < o) ssum[tid] += ssum[tid + o];
-            __syncthreads();
-        }
-        clipped = ssum[0];
-    }
     if (tid == 0) {
+        ma = 0;
+        for (int w = 0; w < kHvWarps; ++w) ma = max(ma, sma[w]);
         const float sigma = 1.2533f * (clipped / (float)mm);
         const float tau = 100.f * (float)p.n2 * 1.1920928955078125e-07f * bits16_to_float<T>(ma) * __ldcg(p.maxB);
         // a bucket sums n1 n3 / m^2 entries of E on average: the per-entry cap grows like the root of that
         const float thr = fminf(tau * p.cap_scale, p.thr_scale * sigma);
         fpsk_probe_result r;
-        r.nonfinite = tbad > 0.f ? 1 : 0;
-        r.fired = (tbad > 0.f || tmax.v > thr) ? 1 : 0;
-        r.argmax_col = tmax.v >= 0.f ? tmax.i : -1;
-        r.status = __ldcg(p.ctrl + 1) ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK;
-        r.max_abs = tmax.v >= 0.f ? tmax.v : 0.f;
+        r.nonfinite = t.bad > 0.f ? 1 : 0;
+        r.fired = (t.bad > 0.f || t.mx.v > thr) ? 1 : 0;
+        r.argmax_col = t.mx.v >= 0.f ? t.mx.i : -1;
+        r.status = (!ok || __ldcg(p.ctrl + 1)) ? (int)FPSK_ERR_TIMEOUT : (int)FPSK_OK;
+        r.max_abs = t.mx.v >= 0.f ? t.mx.v : 0.f;
         r.sigma_hat = sigma;
         r.thr = thr;
         r.tau = tau;
         *p.result = r;
-        p.ctrl[0] = 0;          // ticket, error flag and unit counter ready for the next call on this workspace
-        p.ctrl[1] = 0;
-        p.ctrl[2] = 0;
+        // counters ready for the next call on this workspace
+        p.ctrl[0] = 0; p.ctrl[1] = 0; p.ctrl[2] = 0; p.ctrl[3] = 0;
     }
 }
 
@@ -602,8 +737,10 @@ struct HpCache {          // the B side, device memory kept by the caller across
     uint32_t *rowperm;
     int *h2, *v2, *colcount, *colstart;
     uint32_t *colperm;
-    int *extra_count, *extra_start;
+    int *extra_count, *extra_start, *rank;
     int *stages;
+    uint32_t *segperm;
+    int *segstart;
     float *Q;
     float *maxB;          // [0] max|B|
     unsigned int *scratch;
@@ -624,8 +761,11 @@ static size_t hp_cache_layout(void *base, long long n1, long long n2, long long 
     const size_t units = (size_t)m * (pl.segsA + pl.segsC);
     t.extra_count = (int *)take((units + 1) * 4);
     t.extra_start = (int *)take((units + 1) * 4);
+    t.rank = (int *)take((size_t)m * 4);
     // one chunk per unit, plus continuation chunks: at most (stages of all units) / 8 of them
     t.stages = (int *)take((units + (size_t)(pl.segsA + pl.segsC) * ((size_t)n1 / (kHpPieces * kHpChunk) + (size_t)m / kHpChunk + 1)) * kHpChunk * 64);
+    t.segperm = (uint32_t *)take((size_t)n3 * 4);
+    t.segstart = (int *)take((size_t)pl.segsC * (m + 1) * 4);
     t.Q = (float *)take((size_t)pl.kpad * pl.npad * 4);
     t.maxB = (float *)take(256);
     t.scratch = (unsigned int *)take(256);
@@ -637,7 +777,7 @@ struct HpWork {           // per-call scratch
     unsigned int *ctrl;   // first 256 bytes: zero before the first call (fpsk_probe_init)
     unsigned int *maxA;
     float4 *vstat;
-    float *P, *Tc, *partAB, *S;
+    float *P, *Tc, *partAB, *partC, *S, *cstat;
     unsigned long long *trace;
 };
 
@@ -651,10 +791,12 @@ static size_t hp_work_layout(void *base, long long n1, long long n2, long long n
     HpWork t;
     t.ctrl = (unsigned int *)take(256);
     t.maxA = (unsigned int *)take((size_t)(sms > 1 ? sms : 1) * 4);
-    t.vstat = (float4 *)take((size_t)m * 16);
+    t.vstat = (float4 *)take((size_t)kHvMaxGrid * 16);
+    t.cstat = (float *)take((size_t)kHvMaxGrid * 4);
     t.P = (float *)take((size_t)m * pl.kpad * 4);
     t.Tc = (float *)take((size_t)m * n3 * 4);
     t.partAB = (float *)take((size_t)pl.ksplit * m * m * 4);
+    t.partC = (float *)take((size_t)pl.segsC * m * m * 4);
     t.S = (float *)take((size_t)m * m * 4);
     t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 128);       // 8 stamps per team
     if (w) *w = t;
@@ -688,7 +830,8 @@ static HpArgs hp_args(const void *A, long long lda, const float *C, long long ld
     a.n1 = (int)n1; a.n2 = (int)n2; a.n3 = (int)n3; a.m = m; a.kpad = pl.kpad;
     a.segsA = pl.segsA; a.segsC = pl.segsC;
     a.rowperm = c.rowperm; a.rowstart = c.rowstart; a.stages = c.stages;
-    a.P = w ? w->P : nullptr; a.Tc = w ? w->Tc : nullptr;
+    a.segperm = c.segperm; a.segstart = c.segstart;
+    a.P = w ? w->P : nullptr; a.Tc = w ? w->Tc : nullptr; a.partC = w ? w->partC : nullptr;
     a.maxA = w ? w->maxA : nullptr; a.ctrl = w ? w->ctrl : nullptr;
     a.trace = w ? w->trace : nullptr;
     static const bool trace_env = getenv("FPSK_HPROBE_TRACE") != nullptr;
@@ -714,12 +857,16 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
     rc = max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
     if (rc != FPSK_OK) return rc;
     const HpArgs a = hp_args(nullptr, 0, nullptr, 0, n1, n2, n3, m, pl, c, nullptr);
+    hp_segment_lists_kernel<<<pl.segsC, 256, (size_t)(m + 1) * 4, st>>>(c.h2, c.v2, (int)n3, m, c.segperm, c.segstart);
+    FPSK_LAUNCH_CHECK();
     const int units = m * (pl.segsA + pl.segsC);
-    hp_count_chunks_kernel<<<(units + 255) / 256, 256, 0, st>>>(a, c.extra_count);
+    hp_rank_kernel<<<(m + 127) / 128, 128, 0, st>>>(c.rowstart, m, c.rank);
+    FPSK_LAUNCH_CHECK();
+    hp_count_chunks_kernel<<<(units + 255) / 256, 256, 0, st>>>(a, c.rank, c.extra_count);
     FPSK_LAUNCH_CHECK();
     rc = exclusive_scan_launch(c.extra_count, units, c.extra_start, st);
     if (rc != FPSK_OK) return rc;
-    hp_fill_stages_kernel<<<(units + 255) / 256, 256, 0, st>>>(a, c.extra_start, c.stages);
+    hp_fill_stages_kernel<<<(units + 255) / 256, 256, 0, st>>>(a, c.rank, c.extra_start, c.stages);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
@@ -761,33 +908,30 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
         if (dtype == FPSK_FP16) hp_rowsum_plain_kernel<__half><<<grid, 256, 0, st>>>(a);
         else hp_rowsum_plain_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(a);
         FPSK_LAUNCH_CHECK();
+        hp_fold_plain_kernel<<<dim3(m, pl.segsC), 256, 0, st>>>(a);
+        FPSK_LAUNCH_CHECK();
     }
     fpsk_status rc = contraction_launch(w.P, c.Q, w.partAB, m, m, pl.kpad, pl.kpad, pl.npad, pl.ksplit, pl.kchunk, pl.tile, st);
     if (rc != FPSK_OK) return rc;
     HvArgs v;
-    v.partAB = w.partAB; v.ksplit = pl.ksplit; v.Tc = w.Tc; v.colperm = c.colperm; v.colstart = c.colstart;
+    v.partAB = w.partAB; v.ksplit = pl.ksplit; v.partC = w.partC; v.nseg = pl.segsC;
     v.m = m; v.n1 = (int)n1; v.n2 = (int)n2; v.n3 = (int)n3;
     v.maxA = w.maxA; v.n_maxA = n_maxA; v.maxB = c.maxB;
     const double mm = (double)m * (double)m;
     v.thr_scale = (float)(mu * sqrt(2.0 * log(mm > 2.0 ? mm : 2.0)));
     v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);
     v.S = d_S ? d_S : w.S;
-    v.vstat = w.vstat; v.ctrl = w.ctrl; v.result = d_result;
-    const int stage_row = n3 <= kHvRowMax ? 1 : 0;
-    const size_t vsmem = stage_row ? (size_t)((n3 + 3) / 4 * 4) * 4 : 0;
-    if (vsmem > 48 * 1024) {
-        static std::once_flag once2;
-        static cudaError_t attr_err2 = cudaSuccess;
-        std::call_once(once2, [] {
-            attr_err2 = cudaFuncSetAttribute(hp_verdict_kernel<__half>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHvRowMax * 4);
-            if (attr_err2 == cudaSuccess)
-                attr_err2 = cudaFuncSetAttribute(hp_verdict_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kHvRowMax * 4);
-        });
-        FPSK_CUDA_OK(attr_err2);
+    v.vstat = w.vstat; v.cstat = w.cstat; v.ctrl = w.ctrl; v.result = d_result;
+    {
+        // cooperative: every CTA waits (bounded) for the statistics of all others
+        int grid = sms < kHvMaxGrid ? sms : kHvMaxGrid;
+        const long long q4 = ((long long)m * m + 3) / 4;
+        if (grid > q4) grid = (int)q4;
+        void *args[] = {(void *)&v};
+        const void *fn = dtype == FPSK_FP16 ? (const void *)hp_combine_kernel<__half> : (const void *)hp_combine_kernel<__nv_bfloat16>;
+        FPSK_CUDA_OK(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kHvThreads), args, 0, st));
+        count_launch();
     }
-    if (dtype == FPSK_FP16) hp_verdict_kernel<__half><<<m, kHvThreads, vsmem, st>>>(v, stage_row);
-    else hp_verdict_kernel<__nv_bfloat16><<<m, kHvThreads, vsmem, st>>>(v, stage_row);
-    FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
 

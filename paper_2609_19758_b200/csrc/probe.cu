@@ -520,7 +520,8 @@ __global__ void __launch_bounds__(kProbeThreads, 2) probe_kernel(const ProbeArgs
 // several hundred cycles), so those parts are short loops with as few dependent global round
 // trips as possible.
 constexpr int kTmaConsumers = 512;
-constexpr int kTmaThreads = kTmaConsumers + 32;   // + producer warp
+constexpr int kTmaProducers = 2;                  // producer warps: one warp issues a bulk copy about every 90 ns
+constexpr int kTmaThreads = kTmaConsumers + 32 * kTmaProducers;
 constexpr int kStageBytes = 32768;
 constexpr int kStages = 6;
 constexpr int kSegMax = 4096;                 // bytes of one row segment: 256 x 16 B; two row lanes of consumers
@@ -758,8 +759,12 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
     const int ngA = a.tA.rg;
 
     if (tid >= kTmaConsumers) {
-        // ------------------------------------------------------------ producer warp
-        const int lane = tid - kTmaConsumers;
+        // ------------------------------------------------------------ producer warps
+        // Both walk the same sequence of stages; warp w fills the stages whose running number is
+        // congruent to w, so two streams of copy instructions are in flight.
+        const int lane = tid & 31;
+        const int pw = (tid - kTmaConsumers) >> 5;
+        unsigned int nstage = 0;
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -775,18 +780,20 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                 fence_proxy_async();
                 for (int t0 = 0; t0 < ngA && ok; t0 += ut_rows) {
                     const int nt = min(ut_rows, ngA - t0);
-                    w = 1;
-                    if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
-                    w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                    if (!w) { ok = false; break; }
-                    if (lane == 0) {
-                        // this row group's block of partA is [ngA][ucnt]: rows t0..t0+nt are contiguous
-                        const uint32_t bytes = (uint32_t)nt * (uint32_t)ucnt * 4u;
-                        mbar_expect_tx(full0 + 8 * stage, bytes);
-                        bulk_g2s(smem_u32(ring + (size_t)stage * kStageBytes),
-                                 p.partA + (long long)pc[2].r0 * ngA + (long long)t0 * ucnt, bytes, full0 + 8 * stage);
+                    if ((nstage++ % kTmaProducers) == (unsigned)pw) {
+                        w = 1;
+                        if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                        w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                        if (!w) { ok = false; break; }
+                        if (lane == 0) {
+                            // this row group's block of partA is [ngA][ucnt]: rows t0..t0+nt are contiguous
+                            const uint32_t bytes = (uint32_t)nt * (uint32_t)ucnt * 4u;
+                            mbar_expect_tx(full0 + 8 * stage, bytes);
+                            bulk_g2s(smem_u32(ring + (size_t)stage * kStageBytes),
+                                     p.partA + (long long)pc[2].r0 * ngA + (long long)t0 * ucnt, bytes, full0 + 8 * stage);
+                        }
+                        __syncwarp();
                     }
-                    __syncwarp();
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -794,16 +801,18 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
             if (!q.has) continue;
             for (int row = q.r0; row < q.r1 && ok; row += q.tr) {
                 const int nr = min(q.tr, q.r1 - row);
-                int w = 1;
-                if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
-                w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                if (!w) { ok = false; break; }
-                if (lane == 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)nr * (uint32_t)q.wbytes);
-                __syncwarp();
-                const uint32_t dst0 = smem_u32(ring + (size_t)stage * kStageBytes);
-                for (int r = lane; r < nr; r += 32)
-                    bulk_g2s(dst0 + (uint32_t)r * (uint32_t)q.segb, q.base + (long long)(row + r) * q.ldb, (uint32_t)q.wbytes,
-                             full0 + 8 * stage);
+                if ((nstage++ % kTmaProducers) == (unsigned)pw) {
+                    int w = 1;
+                    if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                    w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                    if (!w) { ok = false; break; }
+                    if (lane == 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)nr * (uint32_t)q.wbytes);
+                    __syncwarp();
+                    const uint32_t dst0 = smem_u32(ring + (size_t)stage * kStageBytes);
+                    for (int r = lane; r < nr; r += 32)
+                        bulk_g2s(dst0 + (uint32_t)r * (uint32_t)q.segb, q.base + (long long)(row + r) * q.ldb, (uint32_t)q.wbytes,
+                                 full0 + 8 * stage);
+                }
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
         }

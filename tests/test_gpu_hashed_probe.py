@@ -138,7 +138,7 @@ def test_cache_is_keyed_on_identity_and_version():
     r1, S1 = _run(hp, dA, dB, dC, version=0)
     per_call = fpsk.launch_count() - before
     assert hp.side.rebuilds == 1 and np.array_equal(S0, S1)         # cached: same result, nothing rebuilt
-    assert per_call == 3                                             # row sums, contraction, verdict
+    assert per_call == 3                                             # row-bucket sums + fold, contraction, combine + verdict
     # an in-place update of B with a new version rebuilds; the product no longer matches C
     dB.mul_(2.0)
     r2, S2 = _run(hp, dA, dB, dC, version=1)
