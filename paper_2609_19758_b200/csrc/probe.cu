@@ -520,7 +520,10 @@ __global__ void __launch_bounds__(kProbeThreads, 2) probe_kernel(const ProbeArgs
 // several hundred cycles), so those parts are short loops with as few dependent global round
 // trips as possible.
 constexpr int kTmaConsumers = 512;
-constexpr int kTmaProducers = 2;                  // producer warps: one warp issues a bulk copy about every 90 ns
+#ifndef FPSK_TMA_PRODUCERS
+#define FPSK_TMA_PRODUCERS 1
+#endif
+constexpr int kTmaProducers = FPSK_TMA_PRODUCERS;   // producer warps (a second one gains 1 % at 16384^3 and costs 2 us at 4096^3)
 constexpr int kTmaThreads = kTmaConsumers + 32 * kTmaProducers;
 constexpr int kStageBytes = 32768;
 constexpr int kStages = 6;
