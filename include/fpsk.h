@@ -200,6 +200,16 @@ typedef struct {
     int32_t reserved;
 } fpsk_bside;
 
+/* State of a probe across calls; see "what the probe keeps between calls" below. */
+typedef struct {
+    uint32_t calls;             /* probes accumulated since the reset                              */
+    uint32_t clean_calls;       /* those that reported clean                                       */
+    uint32_t fired_any;         /* OR of the verdicts since the reset                              */
+    uint32_t first_fired_call;  /* 1-based index of the first dirty call since the reset, 0 = none */
+    double sigma_sum;           /* sum of sigma_hat over the clean calls                           */
+    double reserved;
+} fpsk_probe_state;
+
 /* Bytes of device memory for the cached B side (hash tables and bucket-sorted permutations of
  * rows and columns, Q = B H2^T as k x n_buckets FP32, max|B|) and for the per-call workspace
  * (P = H1 A, H1 C, split-K partials, S).  0 on bad arguments. */
@@ -225,13 +235,40 @@ int32_t fpsk_bside_matches(const fpsk_bside *side, const void *B, int64_t ldb, u
  *                 (fpsk_probe_init does that) and again after a result with status FPSK_ERR_TIMEOUT
  *   d_result      device; argmax_col holds the flat bucket index a * n_buckets + b
  *   d_S           device, n_buckets^2 floats receiving S, or NULL
+ *   d_state       device, accumulated into by the last kernel of the call, or NULL
  * sigma_hat is the noise at this bucket count and feeds fpsk_plan directly.
  * Asynchronous on `stream`, no host synchronisation; deterministic. */
 fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, const void *B, int64_t ldb,
                               uint64_t b_version, const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
                               fpsk_dtype dtype, int c_is_fp32, uint64_t seed, int32_t round, int32_t n_buckets,
                               const fpsk_params *p, void *cache, size_t cache_bytes, void *workspace,
-                              size_t ws_bytes, void *stream, fpsk_probe_result *d_result, float *d_S);
+                              size_t ws_bytes, void *stream, fpsk_probe_result *d_result, float *d_S,
+                              fpsk_probe_state *d_state);
+
+/* ---- what the probe keeps between calls ------------------------------------------------------ */
+
+/* fpsk_probe_state (declared above, device memory, 32 bytes): the probe averages sigma_hat over the
+ * calls it reports clean without a host synchronisation, and accumulates the verdicts into one flag,
+ * so that a caller synchronises once per step instead of once per GEMM (Section "Calibration",
+ * "Recalibrating the probe"; Section "Implementation").  fpsk_probe_hashed updates it inside its
+ * last kernel when d_state is not NULL; fpsk_probe_accumulate does the same for the result of any
+ * probe of this library (one single-thread kernel).  Updates are plain read-modify-writes: the calls
+ * that share a state must be ordered on one stream.  Everything here can be captured into a CUDA
+ * graph (first call of each entry point outside the capture) and replayed. */
+fpsk_status fpsk_probe_state_reset(fpsk_probe_state *d_state, void *stream);
+fpsk_status fpsk_probe_accumulate(const fpsk_probe_result *d_result, fpsk_probe_state *d_state, void *stream);
+
+/* Cadence of the recalibration: 1 when `calls` is 16 or a later multiple of 1024 ("after 16 calls
+ * and then every 1024"), else 0.  Host only. */
+int32_t fpsk_recalibration_due(uint32_t calls);
+
+/* m' = max(m_comb, 16, min(ceil(n_buckets B1 / B*), m_max)) with B1 = max(m, n) sigma_bar / rms_c, and
+ * whether m' lies outside [n_buckets / 1.25, 1.25 n_buckets] (then the caller rebuilds its hashes,
+ * buffers, caches and graphs at m').  sigma_bar = sigma_sum / clean_calls of a state read back by
+ * the caller.  A sigma_bar or rms_c that is not a positive finite number leaves n_buckets unchanged.
+ * Host only; outputs are host pointers. */
+fpsk_status fpsk_probe_recalibrate(int64_t m, int64_t n, double sigma_bar, double rms_c, int32_t n_buckets,
+                                   const fpsk_params *p, int32_t *m_new, int32_t *rebuild);
 
 /* ---- hashed moment sketches --------------------------------------------------------------- */
 

@@ -42,7 +42,7 @@ __all__ = [
     "c_f", "law_sigma", "m_comb", "m_max", "m_mem", "m_num", "m_start", "cap_K",
     "rms_c_estimate", "index_budget", "radius_from_budget", "plan", "recalibrated_m",
     "measure_noise", "scan_out_of_range", "apply_corrections", "verify_repair", "FP32_MAX",
-    "hashed_sum_sketch", "probe_hashed",
+    "hashed_sum_sketch", "probe_hashed", "ProbeState", "recalibration_due", "recalibrate_probe",
 ]
 
 EPS32 = 2.0 ** -23          # FP32 machine epsilon used by the thresholds (Section "Validation")
@@ -564,6 +564,50 @@ def recalibrated_m(n1, n3, sigma_bar, rms_c, m_cur, params: Params = None) -> in
     params = params or Params()
     B1 = max(n1, n3) * sigma_bar / rms_c
     return max(m_comb(params), 16, min(int(math.ceil(m_cur * B1 / params.b_star)), m_max(n1, n3)))
+
+
+# ----------------------------------------------------------------------------
+# stateful probe  (Section "Calibration", paragraph "Recalibrating the probe";
+# Section "Implementation": verdict accumulated into one flag per step)
+# ----------------------------------------------------------------------------
+@dataclass
+class ProbeState:
+    """What the probe keeps between calls: how many calls, how many it reported clean, the sum of
+    sigma_hat over the clean ones, and the OR of the verdicts since the last reset."""
+    calls: int = 0
+    clean_calls: int = 0
+    fired_any: int = 0
+    first_fired_call: int = 0       # 1-based index of the first dirty call since the reset, 0 = none
+    sigma_sum: float = 0.0
+
+    def accumulate(self, r: ProbeResult) -> None:
+        self.calls += 1
+        if r.fired:
+            if not self.fired_any:
+                self.first_fired_call = self.calls
+            self.fired_any = 1
+        else:
+            self.clean_calls += 1
+            self.sigma_sum += float(np.float32(r.sigma_hat))
+
+    def sigma_bar(self) -> float:
+        return self.sigma_sum / self.clean_calls if self.clean_calls else float("nan")
+
+
+def recalibration_due(calls: int) -> bool:
+    """After 16 calls and then every 1024: taken as call counts 16, 1024, 2048, ..."""
+    return calls == 16 or (calls > 16 and calls % 1024 == 0)
+
+
+def recalibrate_probe(n1, n3, sigma_bar, rms_c, m_cur, params: Params = None):
+    """(m', rebuild): m' from the averaged clean-call noise; the engine rebuilds at m' only when m'
+    lies outside [m / 1.25, 1.25 m].  A noise or rms estimate that is not a positive finite number
+    leaves m unchanged."""
+    ok = all(math.isfinite(x) and x > 0 for x in (sigma_bar, rms_c))
+    if not ok:
+        return m_cur, False
+    m_new = recalibrated_m(n1, n3, sigma_bar, rms_c, m_cur, params)
+    return m_new, (m_new < m_cur / 1.25 or m_new > 1.25 * m_cur)
 
 
 def measure_noise(A, B, C, seed: int, dtype: int, m0: int = 0, params: Params = None,

@@ -416,7 +416,7 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
                               uint64_t b_version, const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
                               fpsk_dtype dtype, int c_is_fp32, uint64_t seed, int32_t round, int32_t n_buckets,
                               const fpsk_params *p, void *cache, size_t cache_bytes, void *workspace, size_t ws_bytes,
-                              void *stream, fpsk_probe_result *d_result, float *d_S)
+                              void *stream, fpsk_probe_result *d_result, float *d_S, fpsk_probe_state *d_state)
 {
     if (!c_is_fp32) return FPSK_ERR_DTYPE;      // a narrowed C is rejected, not tolerated
     if (!side || !cache || !workspace || !d_result) return FPSK_ERR_NULL;
@@ -437,7 +437,41 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
         side->round = round; side->valid = 1; side->rebuilds += 1;
     }
     return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, cache, cache_bytes, workspace, ws_bytes, st,
-                         d_result, d_S);
+                         d_result, d_S, d_state);
+}
+
+// ---------------------------------------------------------------- stateful probe
+fpsk_status fpsk_probe_state_reset(fpsk_probe_state *d_state, void *stream)
+{
+    if (!d_state) return FPSK_ERR_NULL;
+    FPSK_CUDA_OK(cudaMemsetAsync(d_state, 0, sizeof(fpsk_probe_state), static_cast<cudaStream_t>(stream)));
+    return FPSK_OK;
+}
+
+fpsk_status fpsk_probe_accumulate(const fpsk_probe_result *d_result, fpsk_probe_state *d_state, void *stream)
+{
+    if (!d_result || !d_state) return FPSK_ERR_NULL;
+    return probe_accumulate_launch(d_result, d_state, static_cast<cudaStream_t>(stream));
+}
+
+int32_t fpsk_recalibration_due(uint32_t calls) { return (calls == 16u || (calls > 16u && calls % 1024u == 0u)) ? 1 : 0; }
+
+fpsk_status fpsk_probe_recalibrate(int64_t m, int64_t n, double sigma_bar, double rms_c, int32_t n_buckets,
+                                   const fpsk_params *p, int32_t *m_new, int32_t *rebuild)
+{
+    if (!m_new || !rebuild) return FPSK_ERR_NULL;
+    if (m < 1 || n < 1) return FPSK_ERR_SHAPE;
+    if (n_buckets < 1) return FPSK_ERR_BUCKETS;
+    const fpsk_params q = resolve_params(p);
+    *m_new = n_buckets;
+    *rebuild = 0;
+    if (!(std::isfinite(sigma_bar) && sigma_bar > 0 && std::isfinite(rms_c) && rms_c > 0)) return FPSK_OK;
+    const double B1 = (double)std::max(m, n) * sigma_bar / rms_c;
+    const double grown = std::min(ceil(n_buckets * B1 / q.b_star), (double)m_max_of(m, n));
+    const int mn = (int)std::max({(double)m_comb_of(q), 16.0, grown});
+    *m_new = mn;
+    *rebuild = ((double)mn < n_buckets / 1.25 || (double)mn > 1.25 * n_buckets) ? 1 : 0;
+    return FPSK_OK;
 }
 
 fpsk_status fpsk_hash_tables(uint64_t seed, int32_t round, int32_t side, int64_t count, int32_t n_buckets,

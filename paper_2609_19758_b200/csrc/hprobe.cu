@@ -544,6 +544,7 @@ struct HvArgs {
     float *cstat;            // per CTA: sum of min(|S|, clip)
     unsigned int *ctrl;      // [0] ticket, [1] error flag, [2] unit counter of the streaming kernel, [3] statistics published
     fpsk_probe_result *result;
+    fpsk_probe_state *state; // accumulated into when not null
 };
 
 struct HvMax {
@@ -554,6 +555,33 @@ __device__ __forceinline__ HvMax hv_better(HvMax a, HvMax b)
 {
     if (b.v > a.v || (b.v == a.v && b.i < a.i)) return b;
     return a;
+}
+
+// One probe result into the running state (single thread; calls sharing a state are stream-ordered).
+__device__ __forceinline__ void state_accumulate(fpsk_probe_state *st, const fpsk_probe_result &r)
+{
+    fpsk_probe_state s = *st;
+    s.calls += 1;
+    if (r.fired) {
+        if (!s.fired_any) s.first_fired_call = s.calls;
+        s.fired_any = 1;
+    } else {
+        s.clean_calls += 1;
+        s.sigma_sum += (double)r.sigma_hat;
+    }
+    *st = s;
+}
+
+__global__ void state_accumulate_kernel(const fpsk_probe_result *r, fpsk_probe_state *st)
+{
+    if (blockIdx.x == 0 && threadIdx.x == 0) state_accumulate(st, *r);
+}
+
+fpsk_status probe_accumulate_launch(const fpsk_probe_result *d_result, fpsk_probe_state *d_state, cudaStream_t st)
+{
+    state_accumulate_kernel<<<1, 32, 0, st>>>(d_result, d_state);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
 }
 
 constexpr int kHvThreads = 512;
@@ -703,6 +731,7 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
         r.thr = thr;
         r.tau = tau;
         *p.result = r;
+        if (p.state) state_accumulate(p.state, r);
         // counters ready for the next call on this workspace
         p.ctrl[0] = 0; p.ctrl[1] = 0; p.ctrl[2] = 0; p.ctrl[3] = 0;
     }
@@ -874,7 +903,7 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
 // One probe on a prepared B side.  d_S may be NULL (S then stays in the workspace).
 fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
                           long long n3, fpsk_dtype dtype, int m, double mu, void *cache, size_t cache_bytes, void *ws,
-                          size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S)
+                          size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S, fpsk_probe_state *d_state)
 {
     const int sms = hp_sm_count();
     HpCache c;
@@ -921,7 +950,7 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     v.thr_scale = (float)(mu * sqrt(2.0 * log(mm > 2.0 ? mm : 2.0)));
     v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);
     v.S = d_S ? d_S : w.S;
-    v.vstat = w.vstat; v.cstat = w.cstat; v.ctrl = w.ctrl; v.result = d_result;
+    v.vstat = w.vstat; v.cstat = w.cstat; v.ctrl = w.ctrl; v.result = d_result; v.state = d_state;
     {
         // cooperative: every CTA waits (bounded) for the statistics of all others
         int grid = sms < kHvMaxGrid ? sms : kHvMaxGrid;

@@ -57,6 +57,12 @@ class BSide(C.Structure):
                 ("reserved", C.c_int32)]
 
 
+class ProbeState(C.Structure):
+    """fpsk_probe_state: what a probe keeps between calls (device memory, 32 bytes)."""
+    _fields_ = [("calls", C.c_uint32), ("clean_calls", C.c_uint32), ("fired_any", C.c_uint32),
+                ("first_fired_call", C.c_uint32), ("sigma_sum", C.c_double), ("reserved", C.c_double)]
+
+
 class FpskError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
@@ -107,7 +113,16 @@ def lib() -> C.CDLL:
         L.fpsk_bside_matches.argtypes = [C.POINTER(BSide), vp, i64, u64, i64, i64, i64, C.c_int, u64, i32, i32, vp]
         L.fpsk_probe_hashed.restype = C.c_int
         L.fpsk_probe_hashed.argtypes = [C.POINTER(BSide), vp, i64, vp, i64, u64, vp, i64, i64, i64, i64, C.c_int, C.c_int,
-                                        u64, i32, i32, C.POINTER(Params), vp, sz, vp, sz, vp, vp, vp]
+                                        u64, i32, i32, C.POINTER(Params), vp, sz, vp, sz, vp, vp, vp, vp]
+        L.fpsk_probe_state_reset.restype = C.c_int
+        L.fpsk_probe_state_reset.argtypes = [vp, vp]
+        L.fpsk_probe_accumulate.restype = C.c_int
+        L.fpsk_probe_accumulate.argtypes = [vp, vp, vp]
+        L.fpsk_recalibration_due.restype = i32
+        L.fpsk_recalibration_due.argtypes = [C.c_uint32]
+        L.fpsk_probe_recalibrate.restype = C.c_int
+        L.fpsk_probe_recalibrate.argtypes = [i64, i64, C.c_double, C.c_double, i32, C.POINTER(Params),
+                                             C.POINTER(i32), C.POINTER(i32)]
         L.fpsk_hash_tables.restype = C.c_int
         L.fpsk_hash_tables.argtypes = [u64, i32, i32, i64, i32, vp, vp, vp]
         L.fpsk_workspace_bytes.restype = sz
@@ -256,7 +271,8 @@ class HashedProbe:
                                              self.seed, self.round, self.n_buckets, self.cache.data_ptr()))
 
     def __call__(self, A, B, Cm, result: torch.Tensor, b_version: int = 0, S: Optional[torch.Tensor] = None,
-                 params: Optional[Params] = None, stream=None, c_is_fp32: Optional[bool] = None) -> None:
+                 params: Optional[Params] = None, stream=None, c_is_fp32: Optional[bool] = None,
+                 state: Optional[torch.Tensor] = None) -> None:
         a = _mat_args(A, B, Cm)
         assert (a[6], a[7], a[8]) == self.shape
         if c_is_fp32 is None:
@@ -265,9 +281,51 @@ class HashedProbe:
                                      a[8], a[9], 1 if c_is_fp32 else 0, self.seed, self.round, self.n_buckets,
                                      C.byref(params) if params is not None else None, self.cache.data_ptr(),
                                      self.cache.numel(), self.ws.data_ptr(), self.ws.numel(), _stream_ptr(stream),
-                                     result.data_ptr(), S.data_ptr() if S is not None else None)
+                                     result.data_ptr(), S.data_ptr() if S is not None else None,
+                                     state.data_ptr() if state is not None else None)
         if rc != STATUS_OK:
             raise FpskError(rc, "fpsk_probe_hashed")
+
+
+def new_probe_state(device=None, stream=None) -> torch.Tensor:
+    """A zeroed fpsk_probe_state in device memory (uint8 tensor of 32 bytes)."""
+    st = torch.empty(C.sizeof(ProbeState), dtype=torch.uint8, device=device or "cuda")
+    rc = lib().fpsk_probe_state_reset(st.data_ptr(), _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_state_reset")
+    return st
+
+
+def reset_probe_state(state: torch.Tensor, stream=None) -> None:
+    rc = lib().fpsk_probe_state_reset(state.data_ptr(), _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_state_reset")
+
+
+def read_probe_state(state: torch.Tensor) -> ProbeState:
+    """Synchronising read of the state (the once-per-step host read)."""
+    host = state.cpu().numpy().tobytes()
+    return ProbeState.from_buffer_copy(host)
+
+
+def probe_accumulate(result: torch.Tensor, state: torch.Tensor, stream=None) -> None:
+    rc = lib().fpsk_probe_accumulate(result.data_ptr(), state.data_ptr(), _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_accumulate")
+
+
+def recalibration_due(calls: int) -> bool:
+    return bool(lib().fpsk_recalibration_due(calls))
+
+
+def probe_recalibrate(m: int, n: int, sigma_bar: float, rms_c: float, n_buckets: int,
+                      params: Optional[Params] = None) -> Tuple[int, bool]:
+    mn, rb = C.c_int32(), C.c_int32()
+    rc = lib().fpsk_probe_recalibrate(m, n, sigma_bar, rms_c, n_buckets, C.byref(params) if params is not None else None,
+                                      C.byref(mn), C.byref(rb))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_probe_recalibrate")
+    return mn.value, bool(rb.value)
 
 
 def new_probe_result(device=None) -> torch.Tensor:

@@ -183,3 +183,100 @@ def test_reruns_are_bit_identical_and_paths_agree():
     denom = O.abs_sketch(O.abs_product(_f64(A), _f64(Bm)), h1, h2, m)
     assert np.all(np.abs(S2 - S0) <= 2 * TOL * denom)
     assert r2.tau == r0.tau
+
+
+# ---------------------------------------------------------------- state across calls, graph replay
+def test_state_accumulates_like_the_oracle():
+    n1, n2, n3, m = 512, 256, 512, 32
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, W.BF16, 13)
+    Cf = Cm.clone()
+    Cf[17, 300] += 1.0
+    dA, dB, dC, dF = A.cuda(), Bm.cuda(), Cm.cuda(), Cf.cuda()
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=9)
+    res = fpsk.new_probe_result()
+    state = fpsk.new_probe_state()
+    ref = O.ProbeState()
+    for which in (0, 0, 1, 0, 1, 0, 0):
+        hp(dA, dB, dF if which else dC, res, state=state)
+        torch.cuda.synchronize()
+        r = fpsk.read_probe_result(res)
+        assert r.fired == which
+        ref.accumulate(O.ProbeResult(bool(r.fired), bool(r.nonfinite), r.argmax_col, r.max_abs, r.sigma_hat, r.thr, r.tau))
+    got = fpsk.read_probe_state(state)
+    assert (got.calls, got.clean_calls, got.fired_any, got.first_fired_call) == (7, 5, 1, 3)
+    assert (got.calls, got.clean_calls, got.fired_any, got.first_fired_call) == \
+           (ref.calls, ref.clean_calls, ref.fired_any, ref.first_fired_call)
+    assert got.sigma_sum == ref.sigma_sum                       # same values added in the same order, in FP64
+    # the same bookkeeping for the column-sum probe, through the stand-alone kernel
+    fpsk.reset_probe_state(state)
+    pws = fpsk.probe_workspace(n1, n2, n3)
+    ref = O.ProbeState()
+    for which in (1, 0, 0):
+        fpsk.probe(dA, dB, dF if which else dC, pws, res)
+        fpsk.probe_accumulate(res, state)
+        torch.cuda.synchronize()
+        r = fpsk.read_probe_result(res)
+        ref.accumulate(O.ProbeResult(bool(r.fired), bool(r.nonfinite), r.argmax_col, r.max_abs, r.sigma_hat, r.thr, r.tau))
+    got = fpsk.read_probe_state(state)
+    assert (got.calls, got.clean_calls, got.fired_any, got.first_fired_call, got.sigma_sum) == \
+           (ref.calls, ref.clean_calls, ref.fired_any, ref.first_fired_call, ref.sigma_sum)
+    assert (got.calls, got.fired_any, got.first_fired_call) == (3, 1, 1)
+
+
+def test_probe_replays_from_a_cuda_graph():
+    """One host read per step: the captured probe accumulates its verdicts and its noise on the device."""
+    n1, n2, n3, m = 1024, 512, 1024, 64
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, W.FP16, 21)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda().clone()
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=4)
+    res = fpsk.new_probe_result()
+    S = torch.zeros(m, m, dtype=torch.float32, device="cuda")
+    state = fpsk.new_probe_state()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        hp(dA, dB, dC, res, S=S)                     # builds the B side and sets kernel attributes outside the capture
+    side.synchronize()
+    r0 = fpsk.read_probe_result(res)
+    S0 = S.cpu().numpy().copy()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        hp(dA, dB, dC, res, S=S, state=state)
+    rebuilds = hp.side.rebuilds
+    for _ in range(5):
+        g.replay()
+    torch.cuda.synchronize()
+    st = fpsk.read_probe_state(state)
+    assert (st.calls, st.clean_calls, st.fired_any) == (5, 5, 0)
+    assert st.sigma_sum == 5 * float(np.float32(r0.sigma_hat))
+    assert np.array_equal(S.cpu().numpy(), S0) and hp.side.rebuilds == rebuilds
+    # the graph reads C in place: a fault written into the same buffer is seen by the next replay
+    dC[100, 200] += 0.5
+    g.replay()
+    g.replay()
+    torch.cuda.synchronize()
+    st = fpsk.read_probe_state(state)
+    assert (st.calls, st.clean_calls, st.fired_any, st.first_fired_call) == (7, 5, 1, 6)
+    assert fpsk.read_probe_result(res).fired == 1
+
+
+def test_recalibration_from_the_accumulated_noise():
+    n1 = n2 = n3 = 1024
+    m = 64
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, W.BF16, 31)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=6)
+    res = fpsk.new_probe_result()
+    state = fpsk.new_probe_state()
+    calls = 0
+    while not fpsk.recalibration_due(calls):
+        hp(dA, dB, dC, res, state=state)
+        calls += 1
+    st = fpsk.read_probe_state(state)
+    assert calls == 16 and st.calls == 16 and st.clean_calls == 16
+    sigma_bar = st.sigma_sum / st.clean_calls
+    rms = O.rms_c_estimate(Cm.numpy())
+    got = fpsk.probe_recalibrate(n1, n3, sigma_bar, rms, m)
+    assert got == O.recalibrate_probe(n1, n3, sigma_bar, rms, m)
+    # the oracle's sketch at the same bucket count gives the same plan input
+    ref, _ = O.probe_hashed(_f64(A), _f64(Bm), Cm.numpy(), 6, 0, m)
+    assert sigma_bar == pytest.approx(ref.sigma_hat, rel=0.05)

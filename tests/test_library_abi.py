@@ -123,7 +123,7 @@ def test_hashed_probe_validation_needs_no_device(lib):
 
     def call(side=s, A=one, c_is_fp32=1, nb=16, rnd=0, cache=one, cbytes=1 << 30, ws=one, wbytes=1 << 30, m=64):
         return f(C.byref(side) if side is not None else None, A, 64, one, 64, 0, one, 64, m, 64, 64, fpsk.FP16, c_is_fp32,
-                 1, rnd, nb, None, cache, cbytes, ws, wbytes, None, one, None)
+                 1, rnd, nb, None, cache, cbytes, ws, wbytes, None, one, None, None)
 
     assert call(c_is_fp32=0) == fpsk.ERR_DTYPE          # a narrowed C is rejected
     assert call(side=None) == fpsk.ERR_NULL
@@ -135,3 +135,20 @@ def test_hashed_probe_validation_needs_no_device(lib):
     assert s.valid == 0 and s.rebuilds == 0
     assert lib.fpsk_probe_hashed_cache_bytes(0, 8, 8, 4) == 0
     assert lib.fpsk_probe_hashed_workspace_bytes(64, 64, 64, 16) >= 4 * (16 * 64 * 2 + 16 * 16)
+
+
+def test_probe_state_layout_cadence_and_recalibration_match_the_oracle(lib):
+    assert C.sizeof(fpsk.ProbeState) == 32 and fpsk.ProbeState.sigma_sum.offset == 16
+    for calls in list(range(0, 40)) + [1023, 1024, 1025, 1040, 2048, 4096, 5000]:
+        assert fpsk.recalibration_due(calls) == O.recalibration_due(calls), calls
+    for (n1, n3) in ((4096, 4096), (2048, 11008), (16384, 512)):
+        for m_cur in (16, 48, 100, 256, 1000):
+            for sig in (1e-9, 3e-6, 7.3e-5, 1e-4, 2e-3, 1.0, float("nan"), 0.0, float("inf")):
+                for rms in (1.0, 0.37, 12.0, 0.0):
+                    assert fpsk.probe_recalibrate(n1, n3, sig, rms, m_cur) == O.recalibrate_probe(n1, n3, sig, rms, m_cur)
+    mn, rb = C.c_int32(), C.c_int32()
+    assert lib.fpsk_probe_recalibrate(0, 4, 1.0, 1.0, 16, None, C.byref(mn), C.byref(rb)) == fpsk.ERR_SHAPE
+    assert lib.fpsk_probe_recalibrate(4, 4, 1.0, 1.0, 0, None, C.byref(mn), C.byref(rb)) == fpsk.ERR_BUCKETS
+    assert lib.fpsk_probe_recalibrate(4, 4, 1.0, 1.0, 16, None, None, C.byref(rb)) == fpsk.ERR_NULL
+    assert lib.fpsk_probe_state_reset(None, None) == fpsk.ERR_NULL
+    assert lib.fpsk_probe_accumulate(None, None, None) == fpsk.ERR_NULL

@@ -117,3 +117,35 @@ def test_detects_fault_above_floor_and_stays_clean_below():
     C[100, 17] += 20.0 * res.thr
     res2, _ = o.probe_hashed(A, B, C, 3, 0, 16)
     assert res2.fired
+
+
+# ---------------------------------------------------------------- stateful probe
+def test_state_accumulates_clean_noise_and_ors_the_verdicts():
+    st = o.ProbeState()
+    clean = o.ProbeResult(False, False, 3, 0.1, 0.25, 1.0, 2.0)
+    dirty = o.ProbeResult(True, False, 5, 9.0, 0.75, 1.0, 2.0)
+    for r in (clean, clean, dirty, clean, dirty):
+        st.accumulate(r)
+    assert (st.calls, st.clean_calls, st.fired_any, st.first_fired_call) == (5, 3, 1, 3)
+    assert st.sigma_sum == 0.75 and st.sigma_bar() == 0.25          # dirty calls do not enter the average
+    assert math.isnan(o.ProbeState().sigma_bar())
+
+
+def test_recalibration_cadence():
+    due = [c for c in range(1, 3100) if o.recalibration_due(c)]
+    assert due == [16, 1024, 2048, 3072]
+
+
+def test_recalibration_band_and_formula():
+    # B1 = max(n1, n3) sigma / rms; m' = max(m_comb, 16, min(ceil(m B1 / B*), m_max)); B* = 0.3, m_comb = 48
+    n = 4096
+    assert o.recalibrate_probe(n, n, 0.3 / n, 1.0, 100) == (100, False)              # B1 = B*: m' = m
+    assert o.recalibrate_probe(n, n, 0.3 * 1.25 / n, 1.0, 100) == (125, False)       # edge of the band: keep
+    assert o.recalibrate_probe(n, n, 0.3 * 1.26 / n, 1.0, 100) == (126, True)        # outside: rebuild
+    assert o.recalibrate_probe(n, n, 0.3 * 0.8 / n, 1.0, 100) == (80, False)         # m / 1.25 exactly: keep
+    assert o.recalibrate_probe(n, n, 0.3 * 0.79 / n, 1.0, 100) == (79, True)
+    assert o.recalibrate_probe(n, n, 1e-9, 1.0, 100) == (48, True)                   # floor m_comb
+    assert o.recalibrate_probe(n, n, 1.0, 1.0, 100) == (1024, True)                  # cap m_max
+    for bad in (float("nan"), 0.0, -1.0, float("inf")):
+        assert o.recalibrate_probe(n, n, bad, 1.0, 100) == (100, False)
+        assert o.recalibrate_probe(n, n, 1e-4, bad, 100) == (100, False)
