@@ -47,6 +47,8 @@ def parse_args():
     ap.add_argument("--sets", type=int, default=3, help="rotating input batches")
     ap.add_argument("--probe-only", action="store_true", help="time only the probe (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tensor-cores", type=int, default=1, choices=[0, 1],
+                    help="contraction of the moment sketches: 1 = split-BF16 tcgen05 (bucket counts >= 384), 0 = FP32 FMA")
     ap.add_argument("--probe-buckets", type=int, default=256, help="bucket count of the S only probe leg (0: skip it)")
     return ap.parse_args()
 
@@ -158,7 +160,7 @@ def run_ours(args):
     K, Wm = args.steps, max(args.warmup, 3)
     nsets = max(args.sets, 3 if algorithmic_bytes(m, k, n) < 512e6 else 2)
     batches = make_batches(args, m, k, n, dt, nsets, seed0=100 * rank)
-    params = fpsk.default_params(s_budget=4)
+    params = fpsk.default_params(s_budget=4, tensor_cores=args.tensor_cores)
     pws = fpsk.probe_workspace(m, k, n)
     res = fpsk.new_probe_result()
     resid = torch.empty(n, dtype=torch.float32, device="cuda")
@@ -338,6 +340,7 @@ def run_ours(args):
             "workload": f"square {args.dtype.upper()} product m=k=n={m}" if m == k == n else f"{m}x{k}x{n} {args.dtype}",
             "recipe": f"{args.kind}: A~N(0,1), B~N(0,1/sqrt(k)); FP32 C from the vendor GEMM; 4 faults of 2-9% rms(C) per batch",
             "step": "probe + noise measurement (clean C) + localize (3 hash rounds, FP64 confirm)",
+            "contraction": "split-BF16 tcgen05 at >= 384 buckets, FP32 FMA below" if args.tensor_cores else "FP32 FMA",
             "l2": f"256 MiB flush read before every probe; {nsets} rotating input batches (each 134 MB > L2)",
             "parallelism": "replicas only" if world > 1 else "single GPU",
         },

@@ -81,7 +81,7 @@ typedef struct {
     int32_t s_budget;    /* declared fault count s (sets K = max(64, 8 s) and m_comb)      */
     int32_t delta_max;   /* declared bound Delta on faults per row or column               */
     int32_t mad_of_abs;  /* 1: MAD of |S| as printed in the paper; 0: signed MAD of S      */
-    int32_t reserved;
+    int32_t tensor_cores;/* 0: FP32 FMA contraction; 1: split-BF16 tcgen05 contraction     */
     double rho_min;      /* smallest fault to localize, in units of rms(C)                 */
     double c_valid;      /* c of tau_ij = c eps sum_k |A_ik||B_kj|                         */
     double mu;           /* probe margin                                                   */

@@ -112,10 +112,10 @@ struct LocWs {
     int *n_hits;
 };
 
-static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b)
+static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool tc = false)
 {
     const size_t mm = (size_t)m_b * m_b;
-    size_t b = sketch_ws_bytes(n1, n2, n3, m_b);
+    size_t b = sketch_ws_bytes(n1, n2, n3, m_b, tc);
     b += align_up(mm * 4, 256) * 3;
     b += align_up(select_ws_bytes(), 256);
     b += align_up((size_t)131072 * 4, 256);
@@ -126,12 +126,12 @@ static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b)
     return b;
 }
 
-static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, LocWs &w)
+static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, LocWs &w, bool tc = false)
 {
-    if (ws_bytes < loc_ws_bytes(n1, n2, n3, m_b)) return false;
+    if (ws_bytes < loc_ws_bytes(n1, n2, n3, m_b, tc)) return false;
     const size_t mm = (size_t)m_b * m_b;
-    const size_t skb = sketch_ws_bytes(n1, n2, n3, m_b);
-    if (!sketch_carve(ws, skb, n1, n2, n3, m_b, w.sk)) return false;
+    const size_t skb = sketch_ws_bytes(n1, n2, n3, m_b, tc);
+    if (!sketch_carve(ws, skb, n1, n2, n3, m_b, w.sk, tc)) return false;
     char *p = static_cast<char *>(ws) + skb;
     auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
     w.S = (float *)take(mm * 4); w.R = (float *)take(mm * 4); w.T = (float *)take(mm * 4);
@@ -227,7 +227,10 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
         FPSK_CUDA_OK(cudaMemcpyAsync(&h_nhits, w.n_hits, 4, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * kHitCap, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
+        unsigned int h_tc_err = 0;
+        if (w.sk.tc) FPSK_CUDA_OK(cudaMemcpyAsync(&h_tc_err, w.sk.tc_err, 4, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_tc_err) return FPSK_ERR_TIMEOUT;        // a bounded wait of the tensor-core contraction gave up
         if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
         const int nU = std::min(h_counts[2], K);
 
@@ -436,7 +439,7 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
         side->seed = seed; side->version = b_version; side->dtype = (int32_t)dtype; side->n_buckets = n_buckets;
         side->round = round; side->valid = 1; side->rebuilds += 1;
     }
-    return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, cache, cache_bytes, workspace, ws_bytes, st,
+    return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, q.tensor_cores, cache, cache_bytes, workspace, ws_bytes, st,
                          d_result, d_S, d_state);
 }
 
@@ -499,7 +502,7 @@ size_t fpsk_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, 
     // n_buckets <= 0: size for the law's starting count of either operand type
     if (n_buckets <= 0) n_buckets = std::max(m_start_of(m, k, n, FPSK_FP16, q), m_start_of(m, k, n, FPSK_BF16, q));
     if (n_buckets > sketch_max_buckets(m, k, n)) return 0;
-    return loc_ws_bytes(m, k, n, n_buckets);
+    return loc_ws_bytes(m, k, n, n_buckets, q.tensor_cores != 0);
 }
 
 fpsk_status fpsk_sketches(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
@@ -534,7 +537,7 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     if (m0 <= 0) m0 = m_start_of(m, k, n, dtype, q);
     if (m0 > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     LocWs w;
-    if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w)) return FPSK_ERR_WORKSPACE;
+    if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
     rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
@@ -592,7 +595,7 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
     if (!params_ok(q)) return FPSK_ERR_PARAM;
     if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     LocWs w;
-    if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w)) return FPSK_ERR_WORKSPACE;
+    if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
     *h_count = 0;
     std::vector<fpsk_fault> F;
@@ -623,7 +626,7 @@ size_t fpsk_repair_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_bu
         mb = std::min(mb, sketch_max_buckets(m, k, n));
     }
     if (mb < 1 || mb > sketch_max_buckets(m, k, n)) return 0;
-    return align_up(probe_ws_bytes(m, k, n), 256) + align_up(loc_ws_bytes(m, k, n, mb), 256) +
+    return align_up(probe_ws_bytes(m, k, n), 256) + align_up(loc_ws_bytes(m, k, n, mb, q.tensor_cores != 0), 256) +
            align_up(repair_scratch_bytes(), 256) + 256;
 }
 
@@ -739,7 +742,7 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
     if (m_loc <= 0) {
         const int m0 = std::min(m_start_of(m, k, n, dtype, q), sketch_max_buckets(m, k, n));
         LocWs w0;
-        if (!loc_carve(loc_ws, loc_bytes, m, k, n, m0, w0)) return FPSK_ERR_WORKSPACE;
+        if (!loc_carve(loc_ws, loc_bytes, m, k, n, m0, w0, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
         SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
         rc = build_sketches(in, dtype, seed, 0, m0, false, w0.sk, st, w0.S, nullptr, nullptr);
         if (rc != FPSK_OK) return rc;
@@ -758,7 +761,7 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
         if (qq.radius < 0) qq.radius = r;
     }
     LocWs w;
-    if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w)) return FPSK_ERR_WORKSPACE;
+    if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
     bool truncated = false;
     int radius_used = 0;

@@ -740,6 +740,7 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
 // ---------------------------------------------------------------- host side
 struct HpPlan {
     int kpad, npad, segsA, segsC, tile, ksplit, kchunk;
+    int tc_ksplit;     // K splits of the tensor-core contraction (128 x 128 tiles, K blocks of 64)
 };
 
 static void hp_plan(long long n2, long long n3, int m, int sms, HpPlan &pl)
@@ -759,6 +760,7 @@ static void hp_plan(long long n2, long long n3, int m, int sms, HpPlan &pl)
     int kchunk = ((pl.kpad + ks - 1) / ks + 15) / 16 * 16;
     pl.ksplit = (pl.kpad + kchunk - 1) / kchunk;
     pl.kchunk = kchunk;
+    pl.tc_ksplit = tc_plan_ksplit(m, m, pl.kpad, 1, sms);
 }
 
 struct HpCache {          // the B side, device memory kept by the caller across calls
@@ -771,6 +773,7 @@ struct HpCache {          // the B side, device memory kept by the caller across
     uint32_t *segperm;
     int *segstart;
     float *Q;
+    unsigned char *Qplanes;   // Q^T as tiled BF16 planes (tensor-core contraction)
     float *maxB;          // [0] max|B|
     unsigned int *scratch;
 };
@@ -796,6 +799,7 @@ static size_t hp_cache_layout(void *base, long long n1, long long n2, long long 
     t.segperm = (uint32_t *)take((size_t)n3 * 4);
     t.segstart = (int *)take((size_t)pl.segsC * (m + 1) * 4);
     t.Q = (float *)take((size_t)pl.kpad * pl.npad * 4);
+    t.Qplanes = (unsigned char *)take(tc_planes_bytes(m, pl.kpad));
     t.maxB = (float *)take(256);
     t.scratch = (unsigned int *)take(256);
     if (c) *c = t;
@@ -807,6 +811,7 @@ struct HpWork {           // per-call scratch
     unsigned int *maxA;
     float4 *vstat;
     float *P, *Tc, *partAB, *partC, *S, *cstat;
+    unsigned char *Pplanes;
     unsigned long long *trace;
 };
 
@@ -824,7 +829,8 @@ static size_t hp_work_layout(void *base, long long n1, long long n2, long long n
     t.cstat = (float *)take((size_t)kHvMaxGrid * 4);
     t.P = (float *)take((size_t)m * pl.kpad * 4);
     t.Tc = (float *)take((size_t)m * n3 * 4);
-    t.partAB = (float *)take((size_t)pl.ksplit * m * m * 4);
+    t.partAB = (float *)take((size_t)(pl.ksplit > pl.tc_ksplit ? pl.ksplit : pl.tc_ksplit) * m * m * 4);
+    t.Pplanes = (unsigned char *)take(tc_planes_bytes(m, pl.kpad));
     t.partC = (float *)take((size_t)pl.segsC * m * m * 4);
     t.S = (float *)take((size_t)m * m * 4);
     t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 128);       // 8 stamps per team
@@ -883,6 +889,8 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
     if (rc != FPSK_OK) return rc;
     rc = build_b_side(B, ldb, n2, n3, dtype, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q, st);
     if (rc != FPSK_OK) return rc;
+    rc = tc_split_launch(c.Q, 1, pl.npad, m, pl.kpad, c.Qplanes, st);      // row b of Q^T is column b of Q
+    if (rc != FPSK_OK) return rc;
     rc = max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
     if (rc != FPSK_OK) return rc;
     const HpArgs a = hp_args(nullptr, 0, nullptr, 0, n1, n2, n3, m, pl, c, nullptr);
@@ -902,7 +910,7 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
 
 // One probe on a prepared B side.  d_S may be NULL (S then stays in the workspace).
 fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
-                          long long n3, fpsk_dtype dtype, int m, double mu, void *cache, size_t cache_bytes, void *ws,
+                          long long n3, fpsk_dtype dtype, int m, double mu, int tensor_cores, void *cache, size_t cache_bytes, void *ws,
                           size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S, fpsk_probe_state *d_state)
 {
     const int sms = hp_sm_count();
@@ -940,10 +948,21 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
         hp_fold_plain_kernel<<<dim3(m, pl.segsC), 256, 0, st>>>(a);
         FPSK_LAUNCH_CHECK();
     }
-    fpsk_status rc = contraction_launch(w.P, c.Q, w.partAB, m, m, pl.kpad, pl.kpad, pl.npad, pl.ksplit, pl.kchunk, pl.tile, st);
+    fpsk_status rc;
+    int ksplit = pl.ksplit;
+    if (tensor_cores) {
+        rc = tc_split_launch(w.P, pl.kpad, 1, m, pl.kpad, w.Pplanes, st);
+        if (rc != FPSK_OK) return rc;
+        const unsigned char *pa[2] = {w.Pplanes, w.Pplanes}, *pb[2] = {c.Qplanes, c.Qplanes};
+        const int sel[3] = {0, 0, 0};
+        ksplit = pl.tc_ksplit;
+        rc = tc_contract_launch(pa, pb, sel, sel, 1, 1, w.partAB, m, m, pl.kpad, ksplit, w.ctrl + 1, st);
+    } else {
+        rc = contraction_launch(w.P, c.Q, w.partAB, m, m, pl.kpad, pl.kpad, pl.npad, pl.ksplit, pl.kchunk, pl.tile, st);
+    }
     if (rc != FPSK_OK) return rc;
     HvArgs v;
-    v.partAB = w.partAB; v.ksplit = pl.ksplit; v.partC = w.partC; v.nseg = pl.segsC;
+    v.partAB = w.partAB; v.ksplit = ksplit; v.partC = w.partC; v.nseg = pl.segsC;
     v.m = m; v.n1 = (int)n1; v.n2 = (int)n2; v.n3 = (int)n3;
     v.maxA = w.maxA; v.n_maxA = n_maxA; v.maxB = c.maxB;
     const double mm = (double)m * (double)m;

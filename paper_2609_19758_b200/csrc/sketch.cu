@@ -429,25 +429,37 @@ void sketch_plan(long long n1, long long n2, long long n3, int m_b, SketchPlan &
     pl.kchunk = kchunk;
 }
 
-size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b)
+static int sketch_sms()
+{
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
+    return sms;
+}
+
+size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool tc)
 {
     SketchPlan pl;
     sketch_plan(n1, n2, n3, m_b, pl);
     const size_t mm = (size_t)m_b * m_b;
+    tc = tc && m_b >= kTcMinBuckets;
+    const int tcks = tc ? tc_plan_ksplit(m_b, m_b, pl.kpad, 3, sketch_sms()) : 0;
     size_t b = 0;
     b += align_up((size_t)n1 * 4, 256) * 3;          // h1, v1, rowperm
     b += align_up((size_t)n3 * 4, 256) * 3;          // h2, v2, colperm
     b += align_up((size_t)(m_b + 1) * 4, 256) * 4;   // rowcount, rowstart, colcount, colstart
     b += align_up((size_t)m_b * pl.kpad * 4, 256) * 2;       // P, Pw
     b += align_up((size_t)pl.kpad * pl.npad * 4, 256) * 2;   // Q, Qw
-    b += align_up((size_t)pl.ksplit * 3 * mm * 4, 256);      // AB partials
+    b += align_up((size_t)(pl.ksplit > tcks ? pl.ksplit : tcks) * 3 * mm * 4, 256);      // AB partials
+    if (tc) b += align_up(tc_planes_bytes(m_b, pl.kpad), 256) * 4 + 256;          // BF16 planes of P, Pw, Q^T, Qw^T; error word
     b += align_up((size_t)pl.nsplit * 3 * mm * 4, 256);      // C partials
     return b;
 }
 
-bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, SketchWs &w)
+bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, SketchWs &w, bool tc)
 {
-    if (ws_bytes < sketch_ws_bytes(n1, n2, n3, m_b)) return false;
+    if (ws_bytes < sketch_ws_bytes(n1, n2, n3, m_b, tc)) return false;
+    tc = tc && m_b >= kTcMinBuckets;
     sketch_plan(n1, n2, n3, m_b, w.pl);
     const size_t mm = (size_t)m_b * m_b;
     char *p = static_cast<char *>(ws);
@@ -458,7 +470,11 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
     w.colcount = (int *)take((size_t)(m_b + 1) * 4); w.colstart = (int *)take((size_t)(m_b + 1) * 4);
     w.P = (float *)take((size_t)m_b * w.pl.kpad * 4); w.Pw = (float *)take((size_t)m_b * w.pl.kpad * 4);
     w.Q = (float *)take((size_t)w.pl.kpad * w.pl.npad * 4); w.Qw = (float *)take((size_t)w.pl.kpad * w.pl.npad * 4);
-    w.partAB = (float *)take((size_t)w.pl.ksplit * 3 * mm * 4);
+    w.tc = tc;
+    w.tc_ksplit = tc ? tc_plan_ksplit(m_b, m_b, w.pl.kpad, 3, sketch_sms()) : 0;
+    w.partAB = (float *)take((size_t)(w.pl.ksplit > w.tc_ksplit ? w.pl.ksplit : w.tc_ksplit) * 3 * mm * 4);
+    for (int i = 0; i < 4; ++i) w.planes[i] = tc ? (unsigned char *)take(tc_planes_bytes(m_b, w.pl.kpad)) : nullptr;
+    w.tc_err = tc ? (unsigned int *)take(256) : nullptr;
     w.partC = (float *)take((size_t)w.pl.nsplit * 3 * mm * 4);
     return true;
 }
@@ -510,6 +526,26 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         }
         FPSK_LAUNCH_CHECK();
     }
+    int ab_splits = pl.ksplit;
+    if (w.tc) {
+        // split-BF16 contraction on the tensor cores: operands as tiled planes, then one launch for all problems
+        FPSK_CUDA_OK(cudaMemsetAsync(w.tc_err, 0, 4, st));
+        rc = tc_split_launch(w.P, pl.kpad, 1, m_b, pl.kpad, w.planes[0], st);
+        if (rc != FPSK_OK) return rc;
+        rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, w.planes[2], st);        // row b of Q^T is column b of Q
+        if (rc != FPSK_OK) return rc;
+        if (mom) {
+            rc = tc_split_launch(w.Pw, pl.kpad, 1, m_b, pl.kpad, w.planes[1], st);
+            if (rc != FPSK_OK) return rc;
+            rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, w.planes[3], st);
+            if (rc != FPSK_OK) return rc;
+        }
+        const unsigned char *pa[2] = {w.planes[0], w.planes[1]}, *pb[2] = {w.planes[2], w.planes[3]};
+        const int selA[3] = {0, 1, 0}, selB[3] = {0, 0, 1};
+        ab_splits = w.tc_ksplit;
+        rc = tc_contract_launch(pa, pb, selA, selB, mom ? 3 : 1, 3, w.partAB, m_b, m_b, pl.kpad, ab_splits, w.tc_err, st);
+        if (rc != FPSK_OK) return rc;
+    } else
     {
         GemmBatch g;
         g.P = w.P; g.Pw = w.Pw; g.Q = w.Q; g.Qw = w.Qw;
@@ -541,7 +577,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     }
     {
         const long long mm = (long long)m_b * m_b;
-        combine_kernel<<<(unsigned)((mm + 255) / 256), 256, 0, st>>>(w.partAB, pl.ksplit, w.partC, pl.nsplit, mm, mom ? 3 : 1, S, R, Tt);
+        combine_kernel<<<(unsigned)((mm + 255) / 256), 256, 0, st>>>(w.partAB, ab_splits, w.partC, pl.nsplit, mm, mom ? 3 : 1, S, R, Tt);
         FPSK_LAUNCH_CHECK();
     }
     return FPSK_OK;

@@ -25,6 +25,10 @@ struct SketchWs {
     uint32_t *rowperm, *colperm;
     int *rowcount, *rowstart, *colcount, *colstart;
     float *P, *Pw, *Q, *Qw, *partAB, *partC;
+    bool tc;                     // split-BF16 tensor-core contraction
+    int tc_ksplit;
+    unsigned char *planes[4];    // P, Pw, Q^T, Qw^T as tiled BF16 planes
+    unsigned int *tc_err;        // set by the contraction when a wait gave up
 };
 
 struct SketchIn {
@@ -34,8 +38,8 @@ struct SketchIn {
 };
 
 void sketch_plan(long long n1, long long n2, long long n3, int m_b, SketchPlan &pl);
-size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b);
-bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, SketchWs &w);
+size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool tc = false);
+bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, SketchWs &w, bool tc = false);
 int sketch_max_buckets(long long n1, long long n2, long long n3);
 
 fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, int *bucket, int *sign,
@@ -119,13 +123,25 @@ fpsk_status recompute_entries(const SketchIn &in, fpsk_dtype dtype, const ScanEn
                               cudaStream_t st, double *h_gamma, float *h_old);
 fpsk_status patch_launch(float *C, long long ldc, const PatchEntry *d_entries, int n, cudaStream_t st);
 
+// ---- split-precision tensor-core contraction (tc_contract.cu) -------------------------------------
+// bytes of the three tiled BF16 planes of a rows x kk FP32 matrix
+size_t tc_planes_bytes(int rows, int kk);
+// planes of X(r, k) = src[r * ldr + k * ldk]
+fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, unsigned char *planes, cudaStream_t st);
+// part[ks][prob] = A_selA[prob] (M x K) times B_selB[prob] (N x K) transposed, over the ks-th range of K
+fpsk_status tc_contract_launch(const unsigned char *const *planesA, const unsigned char *const *planesB, const int *selA,
+                               const int *selB, int nprob, int pstride, float *part, int M, int N, int K, int ksplit,
+                               unsigned int *d_err, cudaStream_t st);
+int tc_plan_ksplit(int M, int N, int K, int nprob, int sms);
+constexpr int kTcMinBuckets = 384;      // below this the FP32 FMA contraction is the faster one (measured)
+
 // ---- the S only probe with a cached B side (hprobe.cu) ------------------------------------------
 size_t hprobe_cache_bytes(long long n1, long long n2, long long n3, int m);
 size_t hprobe_ws_bytes(long long n1, long long n2, long long n3, int m);
 fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long n2, long long n3, fpsk_dtype dtype,
                            uint64_t seed, int rnd, int m, void *cache, size_t cache_bytes, cudaStream_t st);
 fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
-                          long long n3, fpsk_dtype dtype, int m, double mu, void *cache, size_t cache_bytes, void *ws,
+                          long long n3, fpsk_dtype dtype, int m, double mu, int tensor_cores, void *cache, size_t cache_bytes, void *ws,
                           size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S, fpsk_probe_state *d_state);
 fpsk_status probe_accumulate_launch(const fpsk_probe_result *d_result, fpsk_probe_state *d_state, cudaStream_t st);
 

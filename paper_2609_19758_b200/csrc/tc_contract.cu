@@ -1,0 +1,330 @@
+// Split-precision contraction on the 5th-generation tensor cores (tcgen05, accumulators in TMEM).
+//
+// The sketches need S_AB = P Q (and the weighted forms) to FP32 accuracy: the sketch noise is the
+// measured quantity, and a single-pass reduced-precision product raises it by orders of magnitude
+// (Section "Implementation": TF32 raised the floor 419x).  An FP32 value is therefore split into
+// three BF16 terms x = hi + mid + lo (8 + 8 + 8 significand bits, each remainder exact in FP32), and
+// the product is formed from the six term pairs whose weight is above 2^-24:
+//   (hi,hi) (hi,mid) (mid,hi) (hi,lo) (lo,hi) (mid,mid),
+// every pair one BF16 tcgen05.mma with FP32 accumulation into the same TMEM accumulator.
+//
+//   tc_split_kernel      FP32 matrix -> three BF16 planes, laid out tile by tile exactly as the
+//                        tensor core reads shared memory (K-major, no swizzle: 8 x 16-byte core
+//                        matrices), so that a 128 x 64 operand tile is one contiguous 16 KB block
+//   tc_contract_kernel   one 128 x 128 output tile per CTA and K split: a producer warp brings the six
+//                        operand tiles of a K block with six bulk copies (mbarrier complete_tx), one
+//                        thread issues the 24 MMAs of the block and commits them to the stage's
+//                        "empty" barrier, four warps read the accumulator back (tcgen05.ld) and
+//                        store the split-K partial.
+// Every wait is bounded; on expiry the CTA flags the error word, frees its TMEM and leaves.
+#include "sketch.cuh"
+#include "stream_pipe.cuh"
+
+#include <mutex>
+
+namespace fpsk {
+
+constexpr int kTcBM = 128, kTcBN = 128, kTcBK = 64;
+constexpr int kTcTileBytes = kTcBM * kTcBK * 2;          // one BF16 plane of one operand tile
+constexpr int kTcStageBytes = 6 * kTcTileBytes;          // A hi, mid, lo; B hi, mid, lo
+constexpr int kTcStages = 2;
+constexpr int kTcSmem = kTcStages * kTcStageBytes + 256;
+constexpr int kTcThreads = 192;                          // warps 0-3 epilogue, warp 4 producer, warp 5 MMA
+constexpr int kTcCols = 128;                             // TMEM columns of the accumulator
+
+// ---------------------------------------------------------------- FP32 -> three BF16 planes, tiled
+// X(r, k) = src[r * ldr + k * ldk] for r < rows, k < kk, else 0.  Output: plane p, row tile rt, K block
+// kb at ((p * rtiles + rt) * kblocks + kb) * 16 KB; inside a tile the 16-byte chunk (row r, k chunk kc)
+// sits at (kc * 16 + r / 8) * 128 + (r % 8) * 16.
+__global__ void __launch_bounds__(256) tc_split_kernel(const float *src, long long ldr, long long ldk, int rows, int kk,
+                                                       int rtiles, int kblocks, unsigned char *planes)
+{
+    __shared__ float tile[kTcBM][kTcBK + 1];
+    const int kb = blockIdx.x, rt = blockIdx.y;
+    const int r0 = rt * kTcBM, k0 = kb * kTcBK;
+    if (ldk == 1) {
+        // rows contiguous in k: a warp reads 2 rows x 64 floats
+        for (int e = threadIdx.x; e < kTcBM * kTcBK; e += 256) {
+            const int r = e / kTcBK, k = e % kTcBK;
+            tile[r][k] = (r0 + r < rows && k0 + k < kk) ? src[(long long)(r0 + r) * ldr + (k0 + k)] : 0.f;
+        }
+    } else {
+        // columns contiguous in r: a warp reads 32 consecutive r of one k
+        for (int e = threadIdx.x; e < kTcBM * kTcBK; e += 256) {
+            const int k = e / kTcBM, r = e % kTcBM;
+            tile[r][k] = (r0 + r < rows && k0 + k < kk) ? src[(long long)(r0 + r) * ldr + (long long)(k0 + k) * ldk] : 0.f;
+        }
+    }
+    __syncthreads();
+    const size_t plane_stride = (size_t)rtiles * kblocks * kTcTileBytes;
+    unsigned char *out = planes + ((size_t)rt * kblocks + kb) * kTcTileBytes;
+    for (int id = threadIdx.x; id < kTcBM * (kTcBK / 8); id += 256) {
+        const int kc = id / kTcBM, r = id % kTcBM;
+        unsigned short h[8], m[8], l[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float x = tile[r][kc * 8 + j];
+            const __nv_bfloat16 bh = __float2bfloat16_rn(x);
+            const float r1 = x - __bfloat162float(bh);           // exact
+            const __nv_bfloat16 bm = __float2bfloat16_rn(r1);
+            const float r2 = r1 - __bfloat162float(bm);          // exact
+            const __nv_bfloat16 bl = __float2bfloat16_rn(r2);
+            h[j] = __bfloat16_as_ushort(bh);
+            m[j] = __bfloat16_as_ushort(bm);
+            l[j] = __bfloat16_as_ushort(bl);
+        }
+        const size_t off = (size_t)(kc * 16 + r / 8) * 128 + (size_t)(r % 8) * 16;
+        auto pack = [](const unsigned short *v) {
+            return make_uint4(v[0] | ((unsigned)v[1] << 16), v[2] | ((unsigned)v[3] << 16), v[4] | ((unsigned)v[5] << 16),
+                              v[6] | ((unsigned)v[7] << 16));
+        };
+        *reinterpret_cast<uint4 *>(out + off) = pack(h);
+        *reinterpret_cast<uint4 *>(out + plane_stride + off) = pack(m);
+        *reinterpret_cast<uint4 *>(out + 2 * plane_stride + off) = pack(l);
+    }
+}
+
+// ---------------------------------------------------------------- tcgen05 wrappers
+__device__ __forceinline__ void tc_alloc(uint32_t smem_slot, uint32_t cols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_slot), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_relinquish() { asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_dealloc(uint32_t taddr, uint32_t cols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, BF16 operands, FP32 accumulate; 128 x 128 x 16
+__device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
+        : "memory");
+}
+// shared-memory operand descriptor: K-major, no swizzle; leading (K) byte offset between the two
+// 16-byte K halves of a 16-deep step, stride (M/N) byte offset between 8-row groups
+__device__ __forceinline__ uint64_t tc_smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((saddr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;                       // descriptor version of this architecture
+    return d;                                     // base offset 0, layout type 0 (no swizzle)
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct TcArgs {
+    const unsigned char *planesA[2];   // operand matrices of the A side (P, Pw), tiled planes
+    const unsigned char *planesB[2];   // of the B side (Q^T, Qw^T)
+    int selA[3], selB[3];              // which matrix each problem multiplies
+    float *Cpart;                      // [ksplit][nprob][M * N]
+    int M, N;                          // valid extent of the output
+    int mtiles, ntiles, kblocks;       // tiles of 128 rows of the A and B planes, K blocks of 64
+    int ksplit, kb_per_split, nprob, pstride;   // partial (ks, prob) at (ks * pstride + prob) * M * N
+    unsigned int *err;                 // set to 1 when a wait gave up
+};
+
+__global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs g)
+{
+    extern __shared__ __align__(1024) unsigned char smem[];
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(smem + kTcStages * kTcStageBytes);
+    uint32_t *tslot = reinterpret_cast<uint32_t *>(bars + 8);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kTcStages), accb = smem_u32(bars + 2 * kTcStages);
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int nt = blockIdx.x, mt = blockIdx.y;
+    const int prob = blockIdx.z / g.ksplit, ks = blockIdx.z % g.ksplit;
+    const int kb0 = ks * g.kb_per_split, kb1 = min(g.kblocks, kb0 + g.kb_per_split);
+    if (tid == 0) {
+        for (int s = 0; s < kTcStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, 1);
+        }
+        mbar_init(accb, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 5) {
+        tc_alloc(smem_u32(tslot), kTcCols);
+        tc_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tslot;
+
+    if (warp == 4) {
+        // ------------------------------------------------------------ producer
+        const unsigned char *pa = g.planesA[g.selA[prob]], *pb = g.planesB[g.selB[prob]];
+        const size_t strideA = (size_t)g.mtiles * g.kblocks * kTcTileBytes, strideB = (size_t)g.ntiles * g.kblocks * kTcTileBytes;
+        int stage = 0;
+        uint32_t phase = 0;
+        for (int kb = kb0; kb < kb1; ++kb) {
+            int w = 1;
+            if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+            w = __shfl_sync(0xFFFFFFFFu, w, 0);
+            if (!w) { if (lane == 0) { atomicOr(g.err, 1u); } break; }
+            if (lane == 0) mbar_expect_tx(full0 + 8 * stage, kTcStageBytes);
+            __syncwarp();
+            if (lane < 6) {
+                const bool isB = lane >= 3;
+                const int p = isB ? lane - 3 : lane;
+                const unsigned char *src = isB ? pb + p * strideB + ((size_t)nt * g.kblocks + kb) * kTcTileBytes
+                                               : pa + p * strideA + ((size_t)mt * g.kblocks + kb) * kTcTileBytes;
+                bulk_g2s(smem_u32(smem + (size_t)stage * kTcStageBytes + (size_t)lane * kTcTileBytes), src, kTcTileBytes,
+                         full0 + 8 * stage);
+            }
+            if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------------------ MMA issue (one thread)
+        // instruction descriptor: FP32 accumulator, BF16 x BF16, both K-major, N = 128, M = 128
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        uint32_t acc = 0;
+        for (int kb = kb0; kb < kb1 && ok; ++kb) {
+            int w = 1;
+            if (lane == 0) w = mbar_wait_bounded(full0 + 8 * stage, phase) ? 1 : 0;
+            w = __shfl_sync(0xFFFFFFFFu, w, 0);
+            if (!w) { ok = false; break; }
+            tc_fence_after();
+            if (lane == 0) {
+                const uint32_t sbase = smem_u32(smem + (size_t)stage * kTcStageBytes);
+                // term pairs (A plane, B plane), small weights first
+                const int pairA[6] = {2, 0, 1, 1, 0, 0}, pairB[6] = {0, 2, 1, 0, 1, 0};
+#pragma unroll
+                for (int kstep = 0; kstep < kTcBK / 16; ++kstep) {
+#pragma unroll
+                    for (int q = 0; q < 6; ++q) {
+                        const uint32_t sa = sbase + pairA[q] * kTcTileBytes + kstep * 2 * (kTcBM / 8) * 128;
+                        const uint32_t sb = sbase + (3 + pairB[q]) * kTcTileBytes + kstep * 2 * (kTcBN / 8) * 128;
+                        tc_mma(tmem, tc_smem_desc(sa, (kTcBM / 8) * 128, 128), tc_smem_desc(sb, (kTcBN / 8) * 128, 128), idesc, acc);
+                        acc = 1;
+                    }
+                }
+                tc_commit(empty0 + 8 * stage);        // the stage is free once these MMAs have read it
+            }
+            __syncwarp();
+            if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
+        }
+        if (lane == 0) {
+            if (!ok) atomicOr(g.err, 1u);
+            tc_commit(accb);                          // arrives when every MMA issued above is complete
+        }
+        __syncwarp();
+    } else {
+        // ------------------------------------------------------------ epilogue: warp w owns TMEM lanes 32 w ..
+        const bool got = mbar_wait_warp(accb, 0);
+        tc_fence_after();
+        if (!got) { if (lane == 0) atomicOr(g.err, 1u); }
+        else if (kb1 > kb0) {
+            const int row = mt * kTcBM + warp * 32 + lane;
+            float *dst = g.Cpart + ((size_t)ks * g.pstride + prob) * (size_t)g.M * g.N + (size_t)row * g.N;
+#pragma unroll 1
+            for (int c = 0; c < kTcBN / 32; ++c) {
+                uint32_t v[32];
+                tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
+                const int col0 = nt * kTcBN + c * 32;
+                if (row < g.M) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j)
+                        if (col0 + j < g.N) dst[col0 + j] = __uint_as_float(v[j]);
+                }
+            }
+        } else {
+            // an empty K range (more splits than K blocks): the partial is zero
+            const int row = mt * kTcBM + warp * 32 + lane;
+            if (row < g.M) {
+                float *dst = g.Cpart + ((size_t)ks * g.pstride + prob) * (size_t)g.M * g.N + (size_t)row * g.N;
+                for (int j = 0; j < kTcBN; ++j)
+                    if (nt * kTcBN + j < g.N) dst[nt * kTcBN + j] = 0.f;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) tc_dealloc(tmem, kTcCols);
+}
+
+// ---------------------------------------------------------------- host side
+size_t tc_planes_bytes(int rows, int kk)
+{
+    const size_t rt = (size_t)(rows + kTcBM - 1) / kTcBM, kb = (size_t)(kk + kTcBK - 1) / kTcBK;
+    return 3 * rt * kb * kTcTileBytes;
+}
+
+fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, unsigned char *planes, cudaStream_t st)
+{
+    const int rt = (rows + kTcBM - 1) / kTcBM, kb = (kk + kTcBK - 1) / kTcBK;
+    tc_split_kernel<<<dim3(kb, rt), 256, 0, st>>>(src, ldr, ldk, rows, kk, rt, kb, planes);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// K splits: enough CTAs to fill the GPU, and no accumulation chain longer than kTcMaxChain K blocks.
+// The tensor core's FP32 accumulation is not round-to-nearest: measured on sketches of clean products,
+// chains of 1024 terms give the lowest noise (about a third below the FP32 FMA contraction), chains of
+// 8192 terms double it; shorter chains move the additions into the FP32 combine and approach its noise.
+constexpr int kTcMaxChain = 16;
+int tc_plan_ksplit(int M, int N, int K, int nprob, int sms)
+{
+    const int tiles = ((M + kTcBM - 1) / kTcBM) * ((N + kTcBN - 1) / kTcBN) * nprob;
+    const int kblocks = (K + kTcBK - 1) / kTcBK;
+    int s = sms / (tiles > 0 ? tiles : 1);
+    if (s < 1) s = 1;
+    if (s > kblocks) s = kblocks;
+    int per = (kblocks + s - 1) / s;
+    if (per > kTcMaxChain) per = kTcMaxChain;
+    return (kblocks + per - 1) / per;
+}
+
+// part[ks][prob] = A_sel(prob) B_sel(prob)^T over the ks-th range of K blocks.  planesA[i] holds an M x K
+// matrix, planesB[i] an N x K matrix (both as tiled BF16 planes of tc_split_launch).
+fpsk_status tc_contract_launch(const unsigned char *const *planesA, const unsigned char *const *planesB, const int *selA,
+                               const int *selB, int nprob, int pstride, float *part, int M, int N, int K, int ksplit,
+                               unsigned int *d_err, cudaStream_t st)
+{
+    static std::once_flag once;
+    static cudaError_t attr_err = cudaSuccess;
+    std::call_once(once, [] {
+        attr_err = cudaFuncSetAttribute(tc_contract_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
+    });
+    FPSK_CUDA_OK(attr_err);
+    TcArgs g;
+    g.planesA[0] = planesA[0]; g.planesA[1] = planesA[1];
+    g.planesB[0] = planesB[0]; g.planesB[1] = planesB[1];
+    for (int i = 0; i < 3; ++i) { g.selA[i] = i < nprob ? selA[i] : 0; g.selB[i] = i < nprob ? selB[i] : 0; }
+    g.Cpart = part; g.M = M; g.N = N;
+    g.mtiles = (M + kTcBM - 1) / kTcBM; g.ntiles = (N + kTcBN - 1) / kTcBN; g.kblocks = (K + kTcBK - 1) / kTcBK;
+    g.ksplit = ksplit; g.kb_per_split = (g.kblocks + ksplit - 1) / ksplit; g.nprob = nprob; g.pstride = pstride;
+    g.err = d_err;
+    tc_contract_kernel<<<dim3(g.ntiles, g.mtiles, nprob * ksplit), kTcThreads, kTcSmem, st>>>(g);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+}  // namespace fpsk

@@ -33,7 +33,7 @@ class Fault(C.Structure):
 
 class Params(C.Structure):
     _fields_ = [("rounds", C.c_int32), ("r_star", C.c_int32), ("r_max", C.c_int32), ("radius", C.c_int32),
-                ("s_budget", C.c_int32), ("delta_max", C.c_int32), ("mad_of_abs", C.c_int32), ("reserved", C.c_int32),
+                ("s_budget", C.c_int32), ("delta_max", C.c_int32), ("mad_of_abs", C.c_int32), ("tensor_cores", C.c_int32),
                 ("rho_min", C.c_double), ("c_valid", C.c_double), ("mu", C.c_double), ("b_star", C.c_double),
                 ("c_coll", C.c_double)]
 

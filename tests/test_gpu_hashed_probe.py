@@ -56,7 +56,8 @@ SHAPES = [
 
 @pytest.mark.parametrize("shape", SHAPES)
 @pytest.mark.parametrize("dtype", [W.FP16, W.BF16])
-def test_sketch_and_verdict(shape, dtype):
+@pytest.mark.parametrize("tensor_cores", [0, 1])
+def test_sketch_and_verdict(shape, dtype, tensor_cores):
     n1, n2, n3, m = shape
     A, Bm, Cm = _case("uniform" if dtype == W.FP16 else "gauss_scaled", n1, n2, n3, dtype, 5)
     A64, B64 = _f64(A), _f64(Bm)
@@ -65,7 +66,7 @@ def test_sketch_and_verdict(shape, dtype):
     h2, _ = O.hash_round(21, 4, 1, n3, m)
     denom = O.abs_sketch(O.abs_product(A64, B64), h1, h2, m)
     hp = fpsk.HashedProbe(n1, n2, n3, m, seed=21, rnd=4)
-    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda())
+    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda(), params=fpsk.default_params(tensor_cores=tensor_cores))
     assert got.status == 0
     assert np.all(np.abs(S - S_ref) <= TOL * denom + 1e-30)
     assert got.tau == pytest.approx(ref.tau, rel=1e-6)
@@ -79,8 +80,10 @@ def test_sketch_and_verdict(shape, dtype):
         assert bool(got.fired) == v.fired
 
 
-@pytest.mark.parametrize("shape", [(96, 64, 80, 8), (512, 2048, 1024, 32), (130, 72, 100, 5), (31, 9, 27, 4)])
-def test_integer_products_are_bit_exact(shape):
+@pytest.mark.parametrize("shape", [(96, 64, 80, 8), (512, 2048, 1024, 32), (130, 72, 100, 5), (31, 9, 27, 4),
+                                   (640, 1000, 768, 200)])
+@pytest.mark.parametrize("tensor_cores", [0, 1])
+def test_integer_products_are_bit_exact(shape, tensor_cores):
     n1, n2, n3, m = shape
     A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 5)
     Cm = W.cpu_fp32_product(A, Bm)
@@ -88,7 +91,7 @@ def test_integer_products_are_bit_exact(shape):
     Cm[n1 - 1, 0] -= 5.0
     ref, S_ref = O.probe_hashed(_f64(A), _f64(Bm), Cm.numpy(), 11, 7, m)
     hp = fpsk.HashedProbe(n1, n2, n3, m, seed=11, rnd=7)
-    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda())
+    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda(), params=fpsk.default_params(tensor_cores=tensor_cores))
     assert np.array_equal(S, S_ref)
     assert got.fired == 1 and ref.fired and got.argmax_col == ref.argmax_col and got.max_abs == ref.max_abs
 

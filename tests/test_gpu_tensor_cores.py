@@ -1,0 +1,105 @@
+"""The split-BF16 tensor-core contraction (tcgen05) behind `tensor_cores = 1`: same results as the FP32
+FMA contraction within the 1e-5 tolerance, bit-exact on integer products, and a measured sketch noise
+that is not above the FMA path's (the gate for using it; Section "Implementation" warns that a
+single-pass reduced-precision product raised the floor 419x)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+from paper_2609_19758_b200 import build as B
+from paper_2609_19758_b200 import fpsk, harness, workloads as W
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _lib():
+    B.build()
+    fpsk.lib()
+
+
+def _f64(t):
+    return t.double().numpy()
+
+
+def _case(kind, n1, n2, n3, dtype, seed):
+    A, Bm = W.operands(kind, n1, n2, n3, dtype, seed)
+    return A, Bm, harness.vendor_gemm_fp32(A.cuda(), Bm.cuda()).cpu()
+
+
+@pytest.mark.parametrize("shape,m_b,dtype", [((1024, 1024, 1024), 384, W.BF16), ((1536, 520, 1280), 400, W.FP16),
+                                             ((2048, 2048, 2048), 512, W.BF16)])
+def test_localize_agrees_with_the_oracle_and_with_the_fma_path(shape, m_b, dtype):
+    n1, n2, n3 = shape
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, dtype, 5)
+    rms = W.rms(Cm)
+    faults = W.faults_additive(n1, n3, rms, 3, 4, 0.03, 0.09, "small")
+    Cf, ch = W.inject(Cm, faults)
+    dA, dB, dF = A.cuda(), Bm.cuda(), Cf.cuda()
+    A64, B64 = _f64(A), _f64(Bm)
+    ref = O.localize(A64, B64, Cf.numpy(), 77, m_b, dtype, O.Params(s_budget=4, radius=4))
+    rset = {(f.i, f.j) for f in ref}
+    rmap = {(f.i, f.j): f for f in ref}
+    results = {}
+    for tc in (0, 1):
+        p = fpsk.default_params(s_budget=4, radius=4, tensor_cores=tc)
+        ws = fpsk.workspace(n1, n2, n3, m_b, p)
+        got = fpsk.localize(dA, dB, dF, 77, m_b, ws, p)
+        results[tc] = got
+        assert {(f.i, f.j) for f in got} == rset == {(f.i, f.j) for f in faults}
+        for f in got:
+            a = np.abs(A64[f.i, :]) @ np.abs(B64[:, f.j])
+            assert abs(f.delta - rmap[(f.i, f.j)].delta) <= TOL * a
+    assert [(f.i, f.j, f.delta, f.round) for f in results[0]] == [(f.i, f.j, f.delta, f.round) for f in results[1]]
+
+
+def test_integer_products_localize_exactly():
+    n1, n2, n3, m_b = 768, 256, 640, 384
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 31, lim=8)
+    Cm = W.cpu_fp32_product(A, Bm)
+    coords = [(5, 1), (5, 9), (300, 630), (767, 639), (0, 0), (412, 77)]
+    faults = [W.InjectedFault(i, j, "add", 3.0 + t, "typical") for t, (i, j) in enumerate(coords)]
+    Cf, ch = W.inject(Cm, faults)
+    p = fpsk.default_params(radius=1, rounds=3, tensor_cores=1)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    got = fpsk.localize(A.cuda(), Bm.cuda(), Cf.cuda(), 2024, m_b, ws, p)
+    assert {(f.i, f.j) for f in got} == set(coords)
+    for f in got:
+        assert f.delta == -(3.0 + coords.index((f.i, f.j)))
+
+
+@pytest.mark.parametrize("n,dtype", [(2048, W.BF16), (2048, W.FP16)])
+def test_measured_noise_is_not_above_the_fma_path(n, dtype):
+    A, Bm, Cm = _case("gauss_scaled", n, n, n, dtype, 9)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    sig = {}
+    for tc in (0, 1):
+        p = fpsk.default_params(tensor_cores=tc)
+        ws = fpsk.workspace(n, n, n, 512, p)
+        sig[tc] = fpsk.measure_noise(dA, dB, dC, 5, ws, 512, p)
+    # what an exact verifier would see: the GEMM's own rounding, sketched in FP64
+    h1, v1 = O.hash_round(5, 0, 0, n, 512)
+    h2, v2 = O.hash_round(5, 0, 1, n, 512)
+    E = _f64(A) @ _f64(Bm) - Cm.numpy().astype(np.float64)
+    ref = O.sigma_clip(O.hashed_sum_sketch(E, h1, v1, h2, v2, 512))
+    assert sig[1].sigma_clip <= 1.02 * sig[0].sigma_clip
+    # It may even fall below the exact verifier's: the product under test comes from the same tensor cores, and
+    # the part of its rounding that is systematic (accumulation that is not round-to-nearest) is reproduced by
+    # the verifier's own contraction and cancels in the sketch.
+    assert 0.5 * ref <= sig[1].sigma_clip <= 1.5 * ref
+    assert sig[0].rms_c == sig[1].rms_c
+
+
+def test_small_bucket_counts_keep_the_fma_contraction():
+    """Below the crossover the flag changes nothing (same kernels, same bits)."""
+    n, m_b = 512, 128
+    A, Bm, Cm = _case("gauss_scaled", n, n, n, W.BF16, 17)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    out = []
+    for tc in (0, 1):
+        p = fpsk.default_params(tensor_cores=tc)
+        ws = fpsk.workspace(n, n, n, m_b, p)
+        out.append(fpsk.measure_noise(dA, dB, dC, 5, ws, m_b, p))
+    assert out[0].sigma_clip == out[1].sigma_clip and out[0].sigma_mad == out[1].sigma_mad
