@@ -99,11 +99,17 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, in
     __syncthreads();
     const unsigned long long prefix = state[ST_PREFIX];
     const int hs = shift + 8;
-    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < mm; i += (long long)gridDim.x * blockDim.x) {
-        unsigned long long k;
-        if (!make_key(mode, S, i, scal, k)) continue;
-        if (hs < nbits && (k >> hs) != (prefix >> hs)) continue;
-        atomicAdd(&sh[(unsigned)(k >> shift) & 255u], 1u);
+    // Keys of a noise sketch crowd into a few bins of the leading digits: lanes with the same bin are
+    // combined first (match_any), so a warp issues one shared-memory atomic per distinct bin.
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long i0 = (long long)blockIdx.x * blockDim.x; i0 < mm; i0 += stride) {
+        const long long i = i0 + threadIdx.x;
+        unsigned long long k = 0;
+        bool valid = i < mm && make_key(mode, S, i, scal, k);
+        if (valid && hs < nbits && (k >> hs) != (prefix >> hs)) valid = false;
+        const unsigned int bin = valid ? ((unsigned)(k >> shift) & 255u) : 256u;
+        const unsigned int peers = __match_any_sync(0xFFFFFFFFu, bin);
+        if (valid && (threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(&sh[bin], (unsigned)__popc(peers));
     }
     __syncthreads();
     if (sh[threadIdx.x]) atomicAdd(&hist[threadIdx.x], sh[threadIdx.x]);
@@ -113,17 +119,39 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, in
     __syncthreads();
     if (!last) return;
     __threadfence();
-    if (threadIdx.x == 0) {
-        unsigned long long k = state[ST_K], cum = 0;
-        int bin = 255;
-        for (int b = 0; b < 256; ++b) {
-            const unsigned int h = __ldcg(&hist[b]);
-            if (cum + h > k) { bin = b; break; }
-            cum += h;
+    // the bin holding the k-th key: inclusive scan of the 256 counts (one per thread), then the first
+    // thread whose running count passes k
+    {
+        __shared__ unsigned long long wsum[8];
+        __shared__ int s_bin;
+        __shared__ unsigned long long s_before;
+        const unsigned long long k = state[ST_K];
+        const unsigned int h = __ldcg(&hist[threadIdx.x]);
+        unsigned long long inc = h;
+        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+            if (lane >= o) inc += v;
         }
-        state[ST_K] = k - cum;
-        state[ST_PREFIX] = prefix | ((unsigned long long)bin << shift);
-        hist[256] = 0;
+        if (lane == 31) wsum[wid] = inc;
+        if (threadIdx.x == 0) { s_bin = 255; s_before = 0; }
+        __syncthreads();
+        unsigned long long base = 0;
+        for (int w = 0; w < wid; ++w) base += wsum[w];
+        inc += base;                                   // keys in bins 0 .. threadIdx.x
+        const unsigned long long before = inc - h;     // keys in bins below this one
+        unsigned long long total = 0;
+        for (int w = 0; w < 8; ++w) total += wsum[w];
+        __syncthreads();
+        if (before <= k && k < inc) { s_bin = threadIdx.x; s_before = before; }        // exactly one thread, when k < total
+        if (threadIdx.x == 255 && k >= total) { s_bin = 255; s_before = total; }       // k beyond the keys (not reached: k is clamped to the count)
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            state[ST_K] = k - s_before;
+            state[ST_PREFIX] = prefix | ((unsigned long long)s_bin << shift);
+            hist[256] = 0;
+        }
     }
     __syncthreads();
     hist[threadIdx.x] = 0;
