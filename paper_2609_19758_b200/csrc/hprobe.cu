@@ -889,7 +889,7 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
     if (rc != FPSK_OK) return rc;
     rc = build_b_side(B, ldb, n2, n3, dtype, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q, st);
     if (rc != FPSK_OK) return rc;
-    rc = tc_split_launch(c.Q, 1, pl.npad, m, pl.kpad, c.Qplanes, st);      // row b of Q^T is column b of Q
+    rc = tc_split_launch(c.Q, 1, pl.npad, m, pl.kpad, 1, c.Qplanes, st);      // row b of Q^T is column b of Q
     if (rc != FPSK_OK) return rc;
     rc = max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
     if (rc != FPSK_OK) return rc;
@@ -951,7 +951,7 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     fpsk_status rc;
     int ksplit = pl.ksplit;
     if (tensor_cores) {
-        rc = tc_split_launch(w.P, pl.kpad, 1, m, pl.kpad, w.Pplanes, st);
+        rc = tc_split_launch(w.P, pl.kpad, 1, m, pl.kpad, 0, w.Pplanes, st);
         if (rc != FPSK_OK) return rc;
         const unsigned char *pa[2] = {w.Pplanes, w.Pplanes}, *pb[2] = {c.Qplanes, c.Qplanes};
         const int sel[3] = {0, 0, 0};

@@ -530,14 +530,14 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     if (w.tc) {
         // split-BF16 contraction on the tensor cores: operands as tiled planes, then one launch for all problems
         FPSK_CUDA_OK(cudaMemsetAsync(w.tc_err, 0, 4, st));
-        rc = tc_split_launch(w.P, pl.kpad, 1, m_b, pl.kpad, w.planes[0], st);
+        rc = tc_split_launch(w.P, pl.kpad, 1, m_b, pl.kpad, 0, w.planes[0], st);
         if (rc != FPSK_OK) return rc;
-        rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, w.planes[2], st);        // row b of Q^T is column b of Q
+        rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], st);        // row b of Q^T is column b of Q
         if (rc != FPSK_OK) return rc;
         if (mom) {
-            rc = tc_split_launch(w.Pw, pl.kpad, 1, m_b, pl.kpad, w.planes[1], st);
+            rc = tc_split_launch(w.Pw, pl.kpad, 1, m_b, pl.kpad, 0, w.planes[1], st);
             if (rc != FPSK_OK) return rc;
-            rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, w.planes[3], st);
+            rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], st);
             if (rc != FPSK_OK) return rc;
         }
         const unsigned char *pa[2] = {w.planes[0], w.planes[1]}, *pb[2] = {w.planes[2], w.planes[3]};

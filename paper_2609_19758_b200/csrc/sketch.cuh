@@ -126,8 +126,9 @@ fpsk_status patch_launch(float *C, long long ldc, const PatchEntry *d_entries, i
 // ---- split-precision tensor-core contraction (tc_contract.cu) -------------------------------------
 // bytes of the three tiled BF16 planes of a rows x kk FP32 matrix
 size_t tc_planes_bytes(int rows, int kk);
-// planes of X(r, k) = src[r * ldr + k * ldk]
-fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, unsigned char *planes, cudaStream_t st);
+// planes of X(r, k) = src[r * ldr + k * ldk], tiled for the A side (b_side = 0) or the B side (1) of the contraction
+fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, int b_side, unsigned char *planes,
+                            cudaStream_t st);
 // part[ks][prob] = A_selA[prob] (M x K) times B_selB[prob] (N x K) transposed, over the ks-th range of K
 fpsk_status tc_contract_launch(const unsigned char *const *planesA, const unsigned char *const *planesB, const int *selA,
                                const int *selB, int nprob, int pstride, float *part, int M, int N, int K, int ksplit,

@@ -10,10 +10,10 @@
 //
 //   tc_split_kernel      FP32 matrix -> three BF16 planes, laid out tile by tile exactly as the
 //                        tensor core reads shared memory (K-major, no swizzle: 8 x 16-byte core
-//                        matrices), so that a 128 x 64 operand tile is one contiguous 16 KB block
-//   tc_contract_kernel   one 128 x 128 output tile per CTA and K split: a producer warp brings the six
-//                        operand tiles of a K block with six bulk copies (mbarrier complete_tx), one
-//                        thread issues the 24 MMAs of the block and commits them to the stage's
+//                        matrices), so that the three planes of an operand tile are one contiguous block
+//   tc_contract_kernel   one 128 x 256 output tile per CTA and K split: a producer warp brings the operand
+//                        tiles of a 32-deep K block with two bulk copies (mbarrier complete_tx), one
+//                        thread issues the 12 MMAs of the block and commits them to the stage's
 //                        "empty" barrier, four warps read the accumulator back (tcgen05.ld) and
 //                        store the split-K partial.
 // Every wait is bounded; on expiry the CTA flags the error word, frees its TMEM and leaves.
@@ -24,42 +24,46 @@
 
 namespace fpsk {
 
-constexpr int kTcBM = 128, kTcBN = 128, kTcBK = 64;
-constexpr int kTcTileBytes = kTcBM * kTcBK * 2;          // one BF16 plane of one operand tile
-constexpr int kTcStageBytes = 6 * kTcTileBytes;          // A hi, mid, lo; B hi, mid, lo
-constexpr int kTcStages = 2;
+constexpr int kTcBM = 128, kTcBN = 256, kTcBK = 32;
+constexpr int kTcTileA = kTcBM * kTcBK * 2;              // one BF16 plane of an A tile (8 KB)
+constexpr int kTcTileB = kTcBN * kTcBK * 2;              // of a B tile (16 KB)
+constexpr int kTcStageBytes = 3 * kTcTileA + 3 * kTcTileB;   // A hi, mid, lo; B hi, mid, lo (72 KB)
+constexpr int kTcStages = 3;
 constexpr int kTcSmem = kTcStages * kTcStageBytes + 256;
 constexpr int kTcThreads = 192;                          // warps 0-3 epilogue, warp 4 producer, warp 5 MMA
-constexpr int kTcCols = 128;                             // TMEM columns of the accumulator
+constexpr int kTcCols = 256;                             // TMEM columns of the accumulator
+static_assert(kTcBM * (kTcBN + 1) * 4 <= kTcStages * kTcStageBytes, "epilogue tile fits in the operand stages");
 
 // ---------------------------------------------------------------- FP32 -> three BF16 planes, tiled
-// X(r, k) = src[r * ldr + k * ldk] for r < rows, k < kk, else 0.  Output: plane p, row tile rt, K block
-// kb at ((p * rtiles + rt) * kblocks + kb) * 16 KB; inside a tile the 16-byte chunk (row r, k chunk kc)
-// sits at (kc * 16 + r / 8) * 128 + (r % 8) * 16.
+// X(r, k) = src[r * ldr + k * ldk] for r < rows, k < kk, else 0.  Tiles of R rows (128 for the A side, 256
+// for the B side) by 32 k.  Output: row tile rt, K block kb, plane p at ((rt * kblocks + kb) * 3 + p) * R * 64
+// bytes, so the three planes of an operand tile are one contiguous block (one bulk copy); inside a plane
+// tile the 16-byte chunk (row r, k chunk kc) sits at (kc * (R / 8) + r / 8) * 128 + (r % 8) * 16.
+template <int R>
 __global__ void __launch_bounds__(256) tc_split_kernel(const float *src, long long ldr, long long ldk, int rows, int kk,
-                                                       int rtiles, int kblocks, unsigned char *planes)
+                                                       int kblocks, unsigned char *planes)
 {
-    __shared__ float tile[kTcBM][kTcBK + 1];
+    __shared__ float tile[R][kTcBK + 1];
+    constexpr int kTile = R * kTcBK * 2;
     const int kb = blockIdx.x, rt = blockIdx.y;
-    const int r0 = rt * kTcBM, k0 = kb * kTcBK;
+    const int r0 = rt * R, k0 = kb * kTcBK;
     if (ldk == 1) {
-        // rows contiguous in k: a warp reads 2 rows x 64 floats
-        for (int e = threadIdx.x; e < kTcBM * kTcBK; e += 256) {
+        // rows contiguous in k: a warp reads one row of 32 floats
+        for (int e = threadIdx.x; e < R * kTcBK; e += 256) {
             const int r = e / kTcBK, k = e % kTcBK;
             tile[r][k] = (r0 + r < rows && k0 + k < kk) ? src[(long long)(r0 + r) * ldr + (k0 + k)] : 0.f;
         }
     } else {
         // columns contiguous in r: a warp reads 32 consecutive r of one k
-        for (int e = threadIdx.x; e < kTcBM * kTcBK; e += 256) {
-            const int k = e / kTcBM, r = e % kTcBM;
+        for (int e = threadIdx.x; e < R * kTcBK; e += 256) {
+            const int k = e / R, r = e % R;
             tile[r][k] = (r0 + r < rows && k0 + k < kk) ? src[(long long)(r0 + r) * ldr + (long long)(k0 + k) * ldk] : 0.f;
         }
     }
     __syncthreads();
-    const size_t plane_stride = (size_t)rtiles * kblocks * kTcTileBytes;
-    unsigned char *out = planes + ((size_t)rt * kblocks + kb) * kTcTileBytes;
-    for (int id = threadIdx.x; id < kTcBM * (kTcBK / 8); id += 256) {
-        const int kc = id / kTcBM, r = id % kTcBM;
+    unsigned char *out = planes + ((size_t)rt * kblocks + kb) * 3 * kTile;
+    for (int id = threadIdx.x; id < R * (kTcBK / 8); id += 256) {
+        const int kc = id / R, r = id % R;
         unsigned short h[8], m[8], l[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -73,14 +77,14 @@ __global__ void __launch_bounds__(256) tc_split_kernel(const float *src, long lo
             m[j] = __bfloat16_as_ushort(bm);
             l[j] = __bfloat16_as_ushort(bl);
         }
-        const size_t off = (size_t)(kc * 16 + r / 8) * 128 + (size_t)(r % 8) * 16;
+        const size_t off = (size_t)(kc * (R / 8) + r / 8) * 128 + (size_t)(r % 8) * 16;
         auto pack = [](const unsigned short *v) {
             return make_uint4(v[0] | ((unsigned)v[1] << 16), v[2] | ((unsigned)v[3] << 16), v[4] | ((unsigned)v[5] << 16),
                               v[6] | ((unsigned)v[7] << 16));
         };
         *reinterpret_cast<uint4 *>(out + off) = pack(h);
-        *reinterpret_cast<uint4 *>(out + plane_stride + off) = pack(m);
-        *reinterpret_cast<uint4 *>(out + 2 * plane_stride + off) = pack(l);
+        *reinterpret_cast<uint4 *>(out + kTile + off) = pack(m);
+        *reinterpret_cast<uint4 *>(out + 2 * kTile + off) = pack(l);
     }
 }
 
@@ -100,7 +104,7 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, BF16 operands, FP32 accumulate; 128 x 128 x 16
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, BF16 operands, FP32 accumulate; 128 x 256 x 16
 __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
@@ -142,7 +146,7 @@ struct TcArgs {
     int selA[3], selB[3];              // which matrix each problem multiplies
     float *Cpart;                      // [ksplit][nprob][M * N]
     int M, N;                          // valid extent of the output
-    int mtiles, ntiles, kblocks;       // tiles of 128 rows of the A and B planes, K blocks of 64
+    int mtiles, ntiles, kblocks;       // tiles of 128 rows of the A planes, of 256 rows of the B planes, K blocks of 32
     int ksplit, kb_per_split, nprob, pstride;   // partial (ks, prob) at (ks * pstride + prob) * M * N
     unsigned int *err;                 // set to 1 when a wait gave up
 };
@@ -178,7 +182,6 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
     if (warp == 4) {
         // ------------------------------------------------------------ producer
         const unsigned char *pa = g.planesA[g.selA[prob]], *pb = g.planesB[g.selB[prob]];
-        const size_t strideA = (size_t)g.mtiles * g.kblocks * kTcTileBytes, strideB = (size_t)g.ntiles * g.kblocks * kTcTileBytes;
         int stage = 0;
         uint32_t phase = 0;
         for (int kb = kb0; kb < kb1; ++kb) {
@@ -188,13 +191,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
             if (!w) { if (lane == 0) { atomicOr(g.err, 1u); } break; }
             if (lane == 0) mbar_expect_tx(full0 + 8 * stage, kTcStageBytes);
             __syncwarp();
-            if (lane < 6) {
-                const bool isB = lane >= 3;
-                const int p = isB ? lane - 3 : lane;
-                const unsigned char *src = isB ? pb + p * strideB + ((size_t)nt * g.kblocks + kb) * kTcTileBytes
-                                               : pa + p * strideA + ((size_t)mt * g.kblocks + kb) * kTcTileBytes;
-                bulk_g2s(smem_u32(smem + (size_t)stage * kTcStageBytes + (size_t)lane * kTcTileBytes), src, kTcTileBytes,
-                         full0 + 8 * stage);
+            if (lane < 2) {
+                // lane 0: the three planes of the A tile (24 KB), lane 1: of the B tile (48 KB)
+                const unsigned char *src = lane ? pb + ((size_t)nt * g.kblocks + kb) * 3 * kTcTileB
+                                                : pa + ((size_t)mt * g.kblocks + kb) * 3 * kTcTileA;
+                bulk_g2s(smem_u32(smem + (size_t)stage * kTcStageBytes + (size_t)lane * 3 * kTcTileA), src,
+                         lane ? 3 * kTcTileB : 3 * kTcTileA, full0 + 8 * stage);
             }
             if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
         }
@@ -220,8 +222,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
                 for (int kstep = 0; kstep < kTcBK / 16; ++kstep) {
 #pragma unroll
                     for (int q = 0; q < 6; ++q) {
-                        const uint32_t sa = sbase + pairA[q] * kTcTileBytes + kstep * 2 * (kTcBM / 8) * 128;
-                        const uint32_t sb = sbase + (3 + pairB[q]) * kTcTileBytes + kstep * 2 * (kTcBN / 8) * 128;
+                        const uint32_t sa = sbase + pairA[q] * kTcTileA + kstep * 2 * (kTcBM / 8) * 128;
+                        const uint32_t sb = sbase + 3 * kTcTileA + pairB[q] * kTcTileB + kstep * 2 * (kTcBN / 8) * 128;
                         tc_mma(tmem, tc_smem_desc(sa, (kTcBM / 8) * 128, 128), tc_smem_desc(sb, (kTcBN / 8) * 128, 128), idesc, acc);
                         acc = 1;
                     }
@@ -242,17 +244,27 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
         tc_fence_after();
         if (!got) { if (lane == 0) atomicOr(g.err, 1u); }
         else if (kb1 > kb0) {
-            const int row = mt * kTcBM + warp * 32 + lane;
-            float *dst = g.Cpart + ((size_t)ks * g.pstride + prob) * (size_t)g.M * g.N + (size_t)row * g.N;
+            // accumulator rows through shared memory (the operand stages are free now), so that the partial
+            // goes out as full 128-byte lines: thread = row on the way in, lane = column on the way out
+            float *tile = reinterpret_cast<float *>(smem);                 // [128][kTcBN + 1]
+            const int rloc = warp * 32 + lane;
 #pragma unroll 1
             for (int c = 0; c < kTcBN / 32; ++c) {
                 uint32_t v[32];
                 tc_ld32(tmem + ((uint32_t)(warp * 32) << 16) + (uint32_t)(c * 32), v);
-                const int col0 = nt * kTcBN + c * 32;
-                if (row < g.M) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (col0 + j < g.N) dst[col0 + j] = __uint_as_float(v[j]);
+                for (int j = 0; j < 32; ++j) tile[rloc * (kTcBN + 1) + c * 32 + j] = __uint_as_float(v[j]);
+            }
+            __syncwarp();                                                  // a warp reads back only the rows it wrote
+            float *dst0 = g.Cpart + ((size_t)ks * g.pstride + prob) * (size_t)g.M * g.N;
+            for (int r = 0; r < 32; ++r) {
+                const int row = mt * kTcBM + warp * 32 + r;
+                if (row >= g.M) break;
+                float *dst = dst0 + (size_t)row * g.N + nt * kTcBN;
+#pragma unroll
+                for (int q = 0; q < kTcBN / 32; ++q) {
+                    const int col = q * 32 + lane;
+                    if (nt * kTcBN + col < g.N) dst[col] = tile[(warp * 32 + r) * (kTcBN + 1) + col];
                 }
             }
         } else {
@@ -273,14 +285,17 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
 // ---------------------------------------------------------------- host side
 size_t tc_planes_bytes(int rows, int kk)
 {
-    const size_t rt = (size_t)(rows + kTcBM - 1) / kTcBM, kb = (size_t)(kk + kTcBK - 1) / kTcBK;
-    return 3 * rt * kb * kTcTileBytes;
+    // sized for either side: rows rounded up to the B side's 256
+    const size_t rt = (size_t)(rows + kTcBN - 1) / kTcBN, kb = (size_t)(kk + kTcBK - 1) / kTcBK;
+    return 3 * rt * kb * kTcTileB;
 }
 
-fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, unsigned char *planes, cudaStream_t st)
+fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, int b_side, unsigned char *planes,
+                            cudaStream_t st)
 {
-    const int rt = (rows + kTcBM - 1) / kTcBM, kb = (kk + kTcBK - 1) / kTcBK;
-    tc_split_kernel<<<dim3(kb, rt), 256, 0, st>>>(src, ldr, ldk, rows, kk, rt, kb, planes);
+    const int kb = (kk + kTcBK - 1) / kTcBK;
+    if (b_side) tc_split_kernel<kTcBN><<<dim3(kb, (rows + kTcBN - 1) / kTcBN), 256, 0, st>>>(src, ldr, ldk, rows, kk, kb, planes);
+    else tc_split_kernel<kTcBM><<<dim3(kb, (rows + kTcBM - 1) / kTcBM), 256, 0, st>>>(src, ldr, ldk, rows, kk, kb, planes);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
@@ -289,7 +304,7 @@ fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int 
 // The tensor core's FP32 accumulation is not round-to-nearest: measured on sketches of clean products,
 // chains of 1024 terms give the lowest noise (about a third below the FP32 FMA contraction), chains of
 // 8192 terms double it; shorter chains move the additions into the FP32 combine and approach its noise.
-constexpr int kTcMaxChain = 16;
+constexpr int kTcMaxChain = 32;        // K blocks of 32: 1024 terms
 int tc_plan_ksplit(int M, int N, int K, int nprob, int sms)
 {
     const int tiles = ((M + kTcBM - 1) / kTcBM) * ((N + kTcBN - 1) / kTcBN) * nprob;
@@ -303,7 +318,7 @@ int tc_plan_ksplit(int M, int N, int K, int nprob, int sms)
 }
 
 // part[ks][prob] = A_sel(prob) B_sel(prob)^T over the ks-th range of K blocks.  planesA[i] holds an M x K
-// matrix, planesB[i] an N x K matrix (both as tiled BF16 planes of tc_split_launch).
+// matrix (A-side planes of tc_split_launch), planesB[i] an N x K matrix (B-side planes).
 fpsk_status tc_contract_launch(const unsigned char *const *planesA, const unsigned char *const *planesB, const int *selA,
                                const int *selB, int nprob, int pstride, float *part, int M, int N, int K, int ksplit,
                                unsigned int *d_err, cudaStream_t st)
