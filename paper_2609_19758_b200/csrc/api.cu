@@ -202,11 +202,21 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
     std::vector<PeelEntry> peel;
     std::vector<Hit> hits(kHitCap);
     std::vector<Candidate> cand(kSelMaxK);
+    // The sketches of round t + 1 do not depend on what round t finds (only the peeling does), so they
+    // are enqueued before the host waits for round t's results: the GPU builds them while the host
+    // replays the search.  The event marks the end of round t's copies.
+    struct EventGuard {
+        cudaEvent_t e = nullptr;
+        ~EventGuard() { if (e) cudaEventDestroy(e); }
+    } round_done;
+    FPSK_CUDA_OK(cudaEventCreateWithFlags(&round_done.e, cudaEventDisableTiming));
+    bool built_ahead = false;
     for (int t = 0; t < q.rounds; ++t) {
-        if (!(t == 0 && round0_built)) {
+        if (!(t == 0 && round0_built) && !built_ahead) {
             rc = build_sketches(in, dtype, seed, t, m_b, true, w.sk, st, w.S, w.R, w.T);
             if (rc != FPSK_OK) return rc;
         }
+        built_ahead = false;
         if (!peel.empty()) {
             const int np = (int)std::min<size_t>(peel.size(), kPeelCap);
             if ((int)peel.size() > kPeelCap) truncated = true;
@@ -229,7 +239,13 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
         FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
         unsigned int h_tc_err = 0;
         if (w.sk.tc) FPSK_CUDA_OK(cudaMemcpyAsync(&h_tc_err, w.sk.tc_err, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        FPSK_CUDA_OK(cudaEventRecord(round_done.e, st));
+        if (t + 1 < q.rounds) {
+            rc = build_sketches(in, dtype, seed, t + 1, m_b, true, w.sk, st, w.S, w.R, w.T);
+            if (rc != FPSK_OK) return rc;
+            built_ahead = true;
+        }
+        FPSK_CUDA_OK(cudaEventSynchronize(round_done.e));
         if (h_tc_err) return FPSK_ERR_TIMEOUT;        // a bounded wait of the tensor-core contraction gave up
         if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
         const int nU = std::min(h_counts[2], K);
