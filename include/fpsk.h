@@ -11,8 +11,10 @@
  *   - Pointers named d_* or documented "device" must be device memory of the current
  *     device; pointers named h_* are host memory.  A, B, C, workspace are device memory
  *     unless an entry point says otherwise.
- *   - The caller owns every buffer.  The library allocates no memory and never writes to
- *     A, B or C (paper, Section "Overview": localization does not modify C).
+ *   - The caller owns every buffer.  The library allocates no device memory and never writes
+ *     to A or B; C is written only by fpsk_verify_repair and fpsk_apply_corrections (paper,
+ *     Section "Overview": localization does not modify C; Algorithm 2, "Apply").
+ *     fpsk_localize creates one CUDA event for the duration of the call.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Indices are 0-based.  The 1-based index weights of the paper are internal.
  *   - Errors are return codes.  Nothing throws, aborts or resets the device.  After
