@@ -7,7 +7,7 @@
 //   compress_a_kernel   P = H1 A, Pw = H1 W1 A          (m_b x n2, rows grouped by bucket)
 //   compress_b_kernel   Q = B H2^T, Qw = B W2 H2^T      (n2 x m_b, one row of B per pass)
 //   sgemm_kernel        S_AB = P Q, R_AB = Pw Q, T_AB = P Qw   (FP32 SIMT, split-K partials)
-//   scatter_c_kernel    S_C, R_C, T_C: one streaming pass over C per round
+//   scatter_c_kernel    S_C, R_C, T_C: one streaming pass over C per round (row sums in registers, one fold per chunk)
 //   combine_kernel      S = sum of AB partials - sum of C partials
 #include "sketch.cuh"
 
@@ -87,17 +87,46 @@ fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, in
     return FPSK_OK;
 }
 
+// Eight FP32 values -> the 16-byte chunks of their three BF16 terms (x = hi + mid + lo, remainders exact).
+__device__ __forceinline__ void split8_bf16(const float (&x)[8], uint4 &hi, uint4 &mid, uint4 &lo)
+{
+    unsigned short h[8], m[8], l[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        const __nv_bfloat16 bh = __float2bfloat16_rn(x[j]);
+        const float r1 = x[j] - __bfloat162float(bh);
+        const __nv_bfloat16 bm = __float2bfloat16_rn(r1);
+        const float r2 = r1 - __bfloat162float(bm);
+        const __nv_bfloat16 bl = __float2bfloat16_rn(r2);
+        h[j] = __bfloat16_as_ushort(bh); m[j] = __bfloat16_as_ushort(bm); l[j] = __bfloat16_as_ushort(bl);
+    }
+    hi = make_uint4(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16), h[4] | ((unsigned)h[5] << 16), h[6] | ((unsigned)h[7] << 16));
+    mid = make_uint4(m[0] | ((unsigned)m[1] << 16), m[2] | ((unsigned)m[3] << 16), m[4] | ((unsigned)m[5] << 16), m[6] | ((unsigned)m[7] << 16));
+    lo = make_uint4(l[0] | ((unsigned)l[1] << 16), l[2] | ((unsigned)l[3] << 16), l[4] | ((unsigned)l[5] << 16), l[6] | ((unsigned)l[7] << 16));
+}
+// Where the chunk (row r, eight k starting at k0) of a tiled operand plane sits (layout of tc_contract.cu):
+// tiles of R rows by 32 k, the three planes of a tile back to back.
+template <int R>
+__device__ __forceinline__ size_t plane_chunk_offset(int r, int k0, int kblocks)
+{
+    const int rt = r / R, rr = r % R, kb = k0 >> 5, kc = (k0 & 31) >> 3;
+    return ((size_t)rt * kblocks + kb) * 3 * (size_t)(R * 64) + (size_t)(kc * (R / 8) + rr / 8) * 128 + (size_t)(rr % 8) * 16;
+}
+
 // ---------------------------------------------------------------- A compression
 // CTA (x: group of 8-column vectors, y: bucket a).  Thread owns 8 adjacent columns and walks
 // the rows of bucket a in ascending row order.
-template <typename T, bool VEC, bool MOM>
+// PLANES: the sums go out as tiled BF16 planes for the tensor-core contraction (K extent kblocks * 32,
+// zero beyond n2) instead of FP32 rows of P, Pw.
+template <typename T, bool VEC, bool MOM, bool PLANES>
 __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A, long long lda, int n1, int n2,
                                                          int kpad, float inv_p1, const uint32_t *rowperm,
-                                                         const int *rowstart, float *P, float *Pw)
+                                                         const int *rowstart, float *P, float *Pw, int kblocks,
+                                                         unsigned char *planesP, unsigned char *planesPw)
 {
     const int a = blockIdx.y;
     const long long col0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
-    if (col0 >= kpad) return;
+    if (col0 >= (PLANES ? kblocks * 32 : kpad)) return;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, accw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (col0 < n2) {
         const int s0 = rowstart[a], s1 = rowstart[a + 1];
@@ -126,6 +155,21 @@ __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A
                 }
             }
         }
+    }
+    if (PLANES) {
+        const size_t off = plane_chunk_offset<128>(a, (int)col0, kblocks);
+        uint4 hi, mid, lo;
+        split8_bf16(acc, hi, mid, lo);
+        *reinterpret_cast<uint4 *>(planesP + off) = hi;
+        *reinterpret_cast<uint4 *>(planesP + off + 128 * 64) = mid;
+        *reinterpret_cast<uint4 *>(planesP + off + 2 * 128 * 64) = lo;
+        if (MOM) {
+            split8_bf16(accw, hi, mid, lo);
+            *reinterpret_cast<uint4 *>(planesPw + off) = hi;
+            *reinterpret_cast<uint4 *>(planesPw + off + 128 * 64) = mid;
+            *reinterpret_cast<uint4 *>(planesPw + off + 2 * 128 * 64) = lo;
+        }
+        return;
     }
     float4 *dp = reinterpret_cast<float4 *>(P + (long long)a * kpad + col0);
     dp[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
@@ -187,15 +231,95 @@ __global__ void __launch_bounds__(256) compress_b_kernel(const unsigned short *B
 // CTA (x: bucket row a, y: split).  The rows of bucket a (ascending) are divided among the
 // splits; each row of C is staged in shared memory and folded over its columns by bucket;
 // the three accumulators of bucket row a live in shared memory, one owner thread per b.
-template <bool MOM>
+// The same with eight consecutive rows of B per pass: the column lists are walked once for eight rows,
+// the barriers are amortised, and the eight sums of a bucket are exactly one 16-byte chunk of the tiled
+// BF16 planes (PLANES: emitted directly, K extent kblocks * 32 and bucket extent btiles * 256, zero
+// padded; otherwise FP32 rows of Q, Qw as above).  Same order of additions per row as the kernel above.
+template <typename T, bool MOM, bool PLANES>
+__global__ void __launch_bounds__(256) compress_b8_kernel(const unsigned short *B, long long ldb, int n2, int n3,
+                                                          int kpad, int m_b, int npad, float inv_p3,
+                                                          const uint32_t *colperm, const int *colstart, float *Q,
+                                                          float *Qw, int kblocks, int btiles, unsigned char *planesQ,
+                                                          unsigned char *planesQw)
+{
+    extern __shared__ __align__(16) unsigned short rowbuf8[];
+    const int n3p = (n3 + 7) & ~7;
+    const int kend = PLANES ? kblocks * 32 : kpad;
+    const int bmax = PLANES ? btiles * 256 : npad;
+    for (int k0 = blockIdx.x * 8; k0 < kend; k0 += gridDim.x * 8) {
+        __syncthreads();
+        for (int r = 0; r < 8; ++r) {
+            unsigned short *dstrow = rowbuf8 + (size_t)r * n3p;
+            if (k0 + r >= n2) {
+                for (int j = threadIdx.x * 8; j < n3p; j += blockDim.x * 8) *reinterpret_cast<uint4 *>(dstrow + j) = make_uint4(0, 0, 0, 0);
+                continue;
+            }
+            const unsigned short *src = B + (long long)(k0 + r) * ldb;
+            if (((reinterpret_cast<uintptr_t>(src) & 15) == 0) && (n3 % 8 == 0)) {
+                for (int j = threadIdx.x * 8; j < n3; j += blockDim.x * 8) *reinterpret_cast<uint4 *>(dstrow + j) = ldg_nc_v4(src + j);
+            } else {
+                for (int j = threadIdx.x; j < n3; j += blockDim.x) dstrow[j] = src[j];
+            }
+        }
+        __syncthreads();
+        for (int b = threadIdx.x; b < bmax; b += blockDim.x) {
+            float q[8] = {0, 0, 0, 0, 0, 0, 0, 0}, qw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            if (b < m_b) {
+                const int s0 = __ldg(colstart + b), s1 = __ldg(colstart + b + 1);
+                for (int s = s0; s < s1; ++s) {
+                    const uint32_t e = __ldg(colperm + s);
+                    const int j = (int)(e & 0x7FFFFFFFu);
+                    const float sg = (e >> 31) ? -1.f : 1.f;
+                    const float swj = sg * ((float)(j + 1) * inv_p3);
+#pragma unroll
+                    for (int r = 0; r < 8; ++r) {
+                        const float x = bits16_to_float<T>(rowbuf8[(size_t)r * n3p + j]);
+                        q[r] += sg * x;
+                        if (MOM) qw[r] = fmaf(swj, x, qw[r]);
+                    }
+                }
+            }
+            if (PLANES) {
+                const size_t off = plane_chunk_offset<256>(b, k0, kblocks);
+                uint4 hi, mid, lo;
+                split8_bf16(q, hi, mid, lo);
+                *reinterpret_cast<uint4 *>(planesQ + off) = hi;
+                *reinterpret_cast<uint4 *>(planesQ + off + 256 * 64) = mid;
+                *reinterpret_cast<uint4 *>(planesQ + off + 2 * 256 * 64) = lo;
+                if (MOM) {
+                    split8_bf16(qw, hi, mid, lo);
+                    *reinterpret_cast<uint4 *>(planesQw + off) = hi;
+                    *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = mid;
+                    *reinterpret_cast<uint4 *>(planesQw + off + 2 * 256 * 64) = lo;
+                }
+            } else {
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    if (k0 + r < kpad) {
+                        Q[(long long)(k0 + r) * npad + b] = q[r];
+                        if (MOM) Qw[(long long)(k0 + r) * npad + b] = qw[r];
+                    }
+                }
+            }
+        }
+    }
+}
+
+// CTA (bucket a, row split).  Columns go in chunks of kScChunk: every thread sums the signed (and
+// row-weighted) rows of the bucket for its own columns in registers - no barrier per row, sixteen
+// independent loads per thread and row in flight - then the chunk's column sums go through shared
+// memory once and thread b folds the columns of bucket b (ascending) into S, R, T.
+constexpr int kScChunk = 4096;
+template <bool MOM, bool VEC>
 __global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long long ldc, int n1, int n3, int m_b,
                                                         float inv_p1, float inv_p3, const uint32_t *rowperm,
                                                         const int *rowstart, const uint32_t *colperm,
                                                         const int *colstart, int nsplit, float *part)
 {
     extern __shared__ __align__(16) float sm[];
-    float *rowbuf = sm;                       // n3 (padded to 4)
-    float *accS = sm + ((n3 + 3) & ~3);
+    float *tS = sm;                           // kScChunk
+    float *tR = sm + kScChunk;                // kScChunk
+    float *accS = sm + 2 * kScChunk;
     float *accR = accS + m_b;
     float *accT = accR + m_b;
     const int a = blockIdx.x, sp = blockIdx.y;
@@ -206,40 +330,68 @@ __global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long lon
     const int s0 = rowstart[a], s1 = rowstart[a + 1];
     const int cnt = s1 - s0;
     const int q0 = s0 + (int)((long long)cnt * sp / nsplit), q1 = s0 + (int)((long long)cnt * (sp + 1) / nsplit);
-    for (int s = q0; s < q1; ++s) {
-        const uint32_t e = __ldg(rowperm + s);
-        const int i = (int)(e & 0x7FFFFFFFu);
-        const float v1 = (e >> 31) ? -1.f : 1.f;
-        const float v1w = v1 * ((float)(i + 1) * inv_p1);
-        __syncthreads();
-        const float *src = C + (long long)i * ldc;
-        if (((reinterpret_cast<uintptr_t>(src) & 15) == 0) && (n3 % 4 == 0)) {
-            for (int j = threadIdx.x * 4; j < n3; j += blockDim.x * 4) {
-                uint4 v = ldg_nc_v4(src + j);
-                *reinterpret_cast<uint4 *>(rowbuf + j) = v;
+    for (int c0 = 0; c0 < n3; c0 += kScChunk) {
+        const int cw = min(kScChunk, n3 - c0);
+        float4 rs[4], rr[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) { rs[q] = make_float4(0.f, 0.f, 0.f, 0.f); rr[q] = make_float4(0.f, 0.f, 0.f, 0.f); }
+        for (int s = q0; s < q1; ++s) {
+            const uint32_t e = __ldg(rowperm + s);
+            const int i = (int)(e & 0x7FFFFFFFu);
+            const float v1 = (e >> 31) ? -1.f : 1.f;
+            const float v1w = v1 * ((float)(i + 1) * inv_p1);
+            const float *src = C + (long long)i * ldc + c0;
+            float4 x[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int j = q * 1024 + threadIdx.x * 4;
+                if (VEC) {
+                    x[q] = j < cw ? __ldg(reinterpret_cast<const float4 *>(src + j)) : make_float4(0.f, 0.f, 0.f, 0.f);
+                } else {
+                    x[q].x = j + 0 < cw ? src[j + 0] : 0.f;
+                    x[q].y = j + 1 < cw ? src[j + 1] : 0.f;
+                    x[q].z = j + 2 < cw ? src[j + 2] : 0.f;
+                    x[q].w = j + 3 < cw ? src[j + 3] : 0.f;
+                }
             }
-        } else {
-            for (int j = threadIdx.x; j < n3; j += blockDim.x) rowbuf[j] = src[j];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                rs[q].x = fmaf(v1, x[q].x, rs[q].x); rs[q].y = fmaf(v1, x[q].y, rs[q].y);
+                rs[q].z = fmaf(v1, x[q].z, rs[q].z); rs[q].w = fmaf(v1, x[q].w, rs[q].w);
+                if (MOM) {
+                    rr[q].x = fmaf(v1w, x[q].x, rr[q].x); rr[q].y = fmaf(v1w, x[q].y, rr[q].y);
+                    rr[q].z = fmaf(v1w, x[q].z, rr[q].z); rr[q].w = fmaf(v1w, x[q].w, rr[q].w);
+                }
+            }
+        }
+        __syncthreads();                      // the previous chunk's fold has finished reading tS, tR
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int j = q * 1024 + threadIdx.x * 4;
+            *reinterpret_cast<float4 *>(tS + j) = rs[q];
+            if (MOM) *reinterpret_cast<float4 *>(tR + j) = rr[q];
         }
         __syncthreads();
         for (int b = threadIdx.x; b < m_b; b += blockDim.x) {
-            const int c0 = __ldg(colstart + b), c1 = __ldg(colstart + b + 1);
-            float rs = 0.f, rt = 0.f;
-            for (int c = c0; c < c1; ++c) {
+            const int k0 = __ldg(colstart + b), k1 = __ldg(colstart + b + 1);
+            float fs = 0.f, fr = 0.f, ft = 0.f;
+            for (int c = k0; c < k1; ++c) {
                 const uint32_t ce = __ldg(colperm + c);
-                const int j = (int)(ce & 0x7FFFFFFFu);
+                const int j = (int)(ce & 0x7FFFFFFFu) - c0;
+                if (j < 0 || j >= cw) continue;
                 const float sg = (ce >> 31) ? -1.f : 1.f;
-                const float x = rowbuf[j];
-                rs += sg * x;
-                if (MOM) rt = fmaf(sg * ((float)(j + 1) * inv_p3), x, rt);
+                const float x = tS[j];
+                fs += sg * x;
+                if (MOM) {
+                    ft = fmaf(sg * ((float)(j + c0 + 1) * inv_p3), x, ft);
+                    fr += sg * tR[j];
+                }
             }
-            accS[b] += v1 * rs;
-            if (MOM) {
-                accR[b] = fmaf(v1w, rs, accR[b]);
-                accT[b] += v1 * rt;
-            }
+            accS[b] += fs;
+            if (MOM) { accR[b] += fr; accT[b] += ft; }
         }
     }
+    __syncthreads();
     const long long mm = (long long)m_b * m_b;
     float *dst = part + (long long)sp * 3 * mm + (long long)a * m_b;
     for (int b = threadIdx.x; b < m_b; b += blockDim.x) {
@@ -481,8 +633,9 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
 
 int sketch_max_buckets(long long n1, long long n2, long long n3)
 {
-    // scatter_c_kernel keeps one row of C and three m_b-vectors in shared memory
-    const long long budget = 200 * 1024 - ((n3 + 3) / 4 * 4) * 4;
+    // scatter_c_kernel keeps two column-sum chunks and three m_b-vectors in shared memory
+    (void)n3;
+    const long long budget = 200 * 1024 - 2LL * kScChunk * 4;
     if (budget < 3 * 4) return 0;
     long long m = budget / 12;
     if (m > 16384) m = 16384;
@@ -505,16 +658,40 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     const unsigned short *A = static_cast<const unsigned short *>(in.A);
     const unsigned short *B = static_cast<const unsigned short *>(in.B);
     const SketchPlan &pl = w.pl;
+    // With the tensor-core contraction the compressions emit the tiled BF16 planes themselves (no FP32 P, Q).
+    const int kblocks = (pl.kpad + 31) / 32;
+    const int btiles = (m_b + 255) / 256;
+    const bool b8 = (size_t)16 * ((n3 + 7) & ~7) <= 160 * 1024;      // eight rows of B fit in shared memory
     {
         const bool vec = (reinterpret_cast<uintptr_t>(in.A) & 15) == 0 && in.lda % 8 == 0 && n2 % 8 == 0;
-        dim3 grid((pl.kpad / 8 + 127) / 128, m_b);
-#define FPSK_CA(V, M) compress_a_kernel<T, V, M><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw)
-        if (vec) { if (mom) FPSK_CA(true, true); else FPSK_CA(true, false); }
-        else     { if (mom) FPSK_CA(false, true); else FPSK_CA(false, false); }
+        const int kcols = w.tc ? kblocks * 32 : pl.kpad;
+        dim3 grid((kcols / 8 + 127) / 128, m_b);
+#define FPSK_CA(V, M, PL) compress_a_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw, kblocks, w.planes[0], w.planes[1])
+        if (w.tc) {
+            if (vec) { if (mom) FPSK_CA(true, true, true); else FPSK_CA(true, false, true); }
+            else     { if (mom) FPSK_CA(false, true, true); else FPSK_CA(false, false, true); }
+        } else {
+            if (vec) { if (mom) FPSK_CA(true, true, false); else FPSK_CA(true, false, false); }
+            else     { if (mom) FPSK_CA(false, true, false); else FPSK_CA(false, false, false); }
+        }
 #undef FPSK_CA
         FPSK_LAUNCH_CHECK();
     }
-    {
+    if (b8) {
+        const size_t smem = (size_t)16 * ((n3 + 7) & ~7);
+        const int groups = (w.tc ? kblocks * 32 : pl.kpad) / 8;
+        const int grid = groups < 888 ? groups : 888;
+#define FPSK_CB8(M, PL)                                                                                                          \
+    do {                                                                                                                         \
+        FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b8_kernel<T, M, PL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        compress_b8_kernel<T, M, PL><<<grid, 256, smem, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm,      \
+                                                              w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3]); \
+    } while (0)
+        if (w.tc) { if (mom) FPSK_CB8(true, true); else FPSK_CB8(false, true); }
+        else      { if (mom) FPSK_CB8(true, false); else FPSK_CB8(false, false); }
+#undef FPSK_CB8
+        FPSK_LAUNCH_CHECK();
+    } else {
         const size_t smem = ((size_t)n3 * 2 + 15) / 16 * 16;
         int grid = pl.kpad < 1184 ? pl.kpad : 1184;
         if (mom) {
@@ -528,17 +705,16 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     }
     int ab_splits = pl.ksplit;
     if (w.tc) {
-        // split-BF16 contraction on the tensor cores: operands as tiled planes, then one launch for all problems
+        // split-BF16 contraction on the tensor cores, one launch for all problems
         FPSK_CUDA_OK(cudaMemsetAsync(w.tc_err, 0, 4, st));
-        rc = tc_split_launch(w.P, pl.kpad, 1, m_b, pl.kpad, 0, w.planes[0], st);
-        if (rc != FPSK_OK) return rc;
-        rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], st);        // row b of Q^T is column b of Q
-        if (rc != FPSK_OK) return rc;
-        if (mom) {
-            rc = tc_split_launch(w.Pw, pl.kpad, 1, m_b, pl.kpad, 0, w.planes[1], st);
+        if (!b8) {
+            // wide B: Q, Qw came out as FP32 rows; split them here (row b of Q^T is column b of Q)
+            rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], st);
             if (rc != FPSK_OK) return rc;
-            rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], st);
-            if (rc != FPSK_OK) return rc;
+            if (mom) {
+                rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], st);
+                if (rc != FPSK_OK) return rc;
+            }
         }
         const unsigned char *pa[2] = {w.planes[0], w.planes[1]}, *pb[2] = {w.planes[2], w.planes[3]};
         const int selA[3] = {0, 1, 0}, selB[3] = {0, 0, 1};
@@ -564,15 +740,18 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         FPSK_LAUNCH_CHECK();
     }
     {
-        const size_t smem = ((size_t)((n3 + 3) & ~3) + 3 * (size_t)m_b) * 4;
+        const size_t smem = ((size_t)2 * kScChunk + 3 * (size_t)m_b) * 4;
         dim3 grid(m_b, pl.nsplit);
-        if (mom) {
-            FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            scatter_c_kernel<true><<<grid, 256, smem, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, w.colperm, w.colstart, pl.nsplit, w.partC);
-        } else {
-            FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            scatter_c_kernel<false><<<grid, 256, smem, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, w.colperm, w.colstart, pl.nsplit, w.partC);
-        }
+        const bool vec = (reinterpret_cast<uintptr_t>(in.C) & 15) == 0 && in.ldc % 4 == 0 && n3 % 4 == 0;
+#define FPSK_SC(M, V)                                                                                                        \
+    do {                                                                                                                     \
+        FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<M, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        scatter_c_kernel<M, V><<<grid, 256, smem, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart,  \
+                                                        w.colperm, w.colstart, pl.nsplit, w.partC);                          \
+    } while (0)
+        if (mom) { if (vec) FPSK_SC(true, true); else FPSK_SC(true, false); }
+        else     { if (vec) FPSK_SC(false, true); else FPSK_SC(false, false); }
+#undef FPSK_SC
         FPSK_LAUNCH_CHECK();
     }
     {
