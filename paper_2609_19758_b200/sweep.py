@@ -36,6 +36,8 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--sizes", default="1024,2048,4096,8192,16384")
     ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--tensor-cores", type=int, default=0, choices=[0, 1],
+                    help="contraction of the moment sketches: 1 = split-BF16 tcgen05 at >= 384 buckets")
     args = ap.parse_args()
     B.build()
     fpsk.lib()
@@ -50,7 +52,7 @@ def main():
             Bm = torch.randn(n, n, device="cuda", generator=gen).to(dt)
             C = harness.vendor_gemm_fp32(A, Bm)
             d = fpsk.BF16 if dt == torch.bfloat16 else fpsk.FP16
-            p = fpsk.default_params()
+            p = fpsk.default_params(tensor_cores=args.tensor_cores)
             ws0 = fpsk.workspace(n, n, n, 0, p)
             nz = fpsk.measure_noise(A, Bm, C, 7, ws0, 0, p)
             pws = fpsk.probe_workspace(n, n, n)
@@ -67,7 +69,7 @@ def main():
             found = []
             loc_ms, _ = _time(lambda: found.append(len(fpsk.localize(A, Bm, C, 7, m_loc, ws, p))), max(3, it // 4), flush)
             nbytes = 2 * n * n + 2 * n * n + 4 * n * n
-            row = dict(n=n, dtype=dt_name, c_hat=nz.c_hat, sigma_clip=nz.sigma_clip, sigma_mad=nz.sigma_mad, rms_c=nz.rms_c,
+            row = dict(n=n, dtype=dt_name, tensor_cores=args.tensor_cores, c_hat=nz.c_hat, sigma_clip=nz.sigma_clip, sigma_mad=nz.sigma_mad, rms_c=nz.rms_c,
                        m0=nz.m0, m_probe=nz.m_probe, m_loc=nz.m_loc, radius=nz.radius, probe_ms=probe_ms, probe_ms_min=probe_min,
                        probe_gbs=nbytes / probe_ms / 1e6, gemm_ms=gemm_ms, measure_noise_ms=noise_ms, localize_ms=loc_ms,
                        clean_fired=int(verdict.fired), clean_faults_reported=max(found) if found else 0)
