@@ -4,14 +4,17 @@
 // streaming kernel, which depends on the hash round only) is built once per weight tensor and kept
 // by the caller; a call on a cached B reads A once and C once.
 //
-//   hp_count_chunks_kernel, hp_fill_stages_kernel
-//                           the work list: for every (matrix, column segment, row bucket) unit the ring
-//                           stages (rows, signs) that stream it
+//   hp_rank_kernel, hp_count_chunks_kernel, hp_fill_stages_kernel, hp_segment_lists_kernel
+//                           once per B side: the work list (for every (matrix, column segment, row bucket)
+//                           unit the ring stages (rows, signs) that stream it, largest buckets first) and
+//                           the per-segment column lists of the fold
 //   hp_stream_kernel        P = H1 A (m x n2) and H1 C H2^T per column segment: signed row-bucket sums
 //                           (and the column fold for C), one persistent CTA per SM, rows gathered by
 //                           bulk copies into shared-memory rings
-//   hp_rowsum_plain_kernel  the same sums with plain loads (inputs that bulk copies cannot address)
-//   sgemm (sketch.cu)       P Q as split-K partials, FP32 FMA
+//   hp_rowsum_plain_kernel, hp_fold_plain_kernel
+//                           the same with plain loads (inputs that bulk copies cannot address)
+//   sgemm (sketch.cu) or tc_contract (tc_contract.cu)
+//                           P Q as split-K partials: FP32 FMA, or split-BF16 on the tensor cores
 //   hp_combine_kernel       S = sum of split-K partials - sum of segment partials, statistics, verdict
 // Every sum has a fixed order (no float atomics): results are bit-reproducible.
 #include "sketch.cuh"
