@@ -68,36 +68,59 @@ __global__ void count_valid_kernel(int mode, const float *S, long long mm, const
 }
 
 // rank to select: median of N keys, or (count - K) for the K largest, from device counts
-__global__ void select_init_kernel(int mode, long long n_all, int K, const int *counts, unsigned long long *state,
-                                   unsigned int *hist)
+__device__ __forceinline__ void select_initial(int mode, long long n_all, int K, const int *counts, bool &skip,
+                                               unsigned long long &k)
 {
-    if (threadIdx.x != 0) return;
-    state[ST_PREFIX] = 0;
-    state[ST_SKIP] = 0;
+    skip = false;
+    k = 0;
     if (mode == SEL_TOPK) {
         const int cnt = counts[0];
-        if (cnt <= K) state[ST_SKIP] = 1;      // take everything above the threshold
-        else state[ST_K] = (unsigned long long)(cnt - K);
+        if (cnt <= K) skip = true;             // take everything above the threshold
+        else k = (unsigned long long)(cnt - K);
     } else if (mode == SEL_SAMPLE) {
         const int cnt = counts[0];
-        if (cnt <= 0) state[ST_SKIP] = 1;
-        else state[ST_K] = (unsigned long long)((cnt - 1) / 2);
+        if (cnt <= 0) skip = true;
+        else k = (unsigned long long)((cnt - 1) / 2);
     } else {
-        state[ST_K] = (unsigned long long)((n_all - 1) / 2);
+        k = (unsigned long long)((n_all - 1) / 2);
     }
-    for (int b = 0; b < 257; ++b) hist[b] = 0;
 }
 
-// One 8-bit digit of the radix select.  The last CTA to finish picks the digit.
+// what the selected key means, written once the last digit is known (or at once when nothing is selected)
+__device__ __forceinline__ void select_result(int mode, unsigned long long key, bool skip, float *scal)
+{
+    if (mode == SEL_ABS) scal[SC_MED] = __uint_as_float((uint32_t)key);
+    else if (mode == SEL_SIGNED) scal[SC_MED] = from_ordered_bits((uint32_t)key);
+    else if (mode == SEL_DEV_ABS || mode == SEL_DEV_SIGNED) scal[SC_MAD] = 1.4826f * __uint_as_float((uint32_t)key);
+    else if (mode == SEL_SAMPLE) scal[SC_MED] = skip ? __uint_as_float(0x7FC00000u) : __uint_as_float((uint32_t)key);
+}
+
+// One 8-bit digit of the radix select.  The last CTA to finish picks the digit.  The first pass of a
+// select derives the rank from the device counts itself and the last one writes the result, so a select
+// is nothing but its passes.  The histogram is left at zero by every pass (and zeroed once per call of
+// the library before the first select).
 __global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, int shift, const float *S, long long mm,
-                                                         const float *scal, unsigned long long *state, unsigned int *hist)
+                                                         float *scal, unsigned long long *state, unsigned int *hist,
+                                                         long long n_all, int K, const int *counts)
 {
     __shared__ unsigned int sh[256];
     __shared__ int last;
-    if (state[ST_SKIP]) return;
+    const bool first = shift == nbits - 8, final_ = shift == 0;
+    bool skip;
+    unsigned long long k_first = 0;
+    if (first) select_initial(mode, n_all, K, counts, skip, k_first);
+    else skip = state[ST_SKIP] != 0;
+    if (skip) {
+        if (first && blockIdx.x == 0 && threadIdx.x == 0) {
+            state[ST_SKIP] = 1;
+            state[ST_PREFIX] = 0;
+            select_result(mode, 0, true, scal);
+        }
+        return;
+    }
     sh[threadIdx.x] = 0;
     __syncthreads();
-    const unsigned long long prefix = state[ST_PREFIX];
+    const unsigned long long prefix = first ? 0ull : state[ST_PREFIX];
     const int hs = shift + 8;
     // Keys of a noise sketch crowd into a few bins of the leading digits: lanes with the same bin are
     // combined first (match_any), so a warp issues one shared-memory atomic per distinct bin.
@@ -125,7 +148,7 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, in
         __shared__ unsigned long long wsum[8];
         __shared__ int s_bin;
         __shared__ unsigned long long s_before;
-        const unsigned long long k = state[ST_K];
+        const unsigned long long k = first ? k_first : state[ST_K];
         const unsigned int h = __ldcg(&hist[threadIdx.x]);
         unsigned long long inc = h;
         const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
@@ -148,8 +171,11 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, in
         if (threadIdx.x == 255 && k >= total) { s_bin = 255; s_before = total; }       // k beyond the keys (not reached: k is clamped to the count)
         __syncthreads();
         if (threadIdx.x == 0) {
+            const unsigned long long key = prefix | ((unsigned long long)s_bin << shift);
             state[ST_K] = k - s_before;
-            state[ST_PREFIX] = prefix | ((unsigned long long)s_bin << shift);
+            state[ST_PREFIX] = key;
+            if (first) state[ST_SKIP] = 0;
+            if (final_) select_result(mode, key, false, scal);
             hist[256] = 0;
         }
     }
@@ -158,28 +184,19 @@ __global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, in
 }
 
 // after the passes: turn the selected key into a value
-__global__ void select_finish_kernel(int mode, const unsigned long long *state, float *scal)
-{
-    if (threadIdx.x != 0) return;
-    const unsigned long long key = state[ST_PREFIX];
-    if (mode == SEL_ABS) scal[SC_MED] = __uint_as_float((uint32_t)key);
-    else if (mode == SEL_SIGNED) scal[SC_MED] = from_ordered_bits((uint32_t)key);
-    else if (mode == SEL_DEV_ABS || mode == SEL_DEV_SIGNED) scal[SC_MAD] = 1.4826f * __uint_as_float((uint32_t)key);
-    else if (mode == SEL_SAMPLE) scal[SC_MED] = state[ST_SKIP] ? __uint_as_float(0x7FC00000u) : __uint_as_float((uint32_t)key);
-}
 
 static fpsk_status run_select(int mode, int nbits, const float *S, long long mm, int K, SelectWs &w, cudaStream_t st)
 {
-    select_init_kernel<<<1, 32, 0, st>>>(mode, mm, K, w.counts, w.state, w.hist);
-    FPSK_LAUNCH_CHECK();
+    if (!w.hist_clean) {
+        FPSK_CUDA_OK(cudaMemsetAsync(w.hist, 0, 257 * sizeof(unsigned int), st));
+        w.hist_clean = true;
+    }
     long long want = (mm + 256 * 16 - 1) / (256 * 16);
     const int grid = (int)(want < 1 ? 1 : (want > 1184 ? 1184 : want));
     for (int shift = nbits - 8; shift >= 0; shift -= 8) {
-        radix_pass_kernel<<<grid, 256, 0, st>>>(mode, nbits, shift, S, mm, w.scal, w.state, w.hist);
+        radix_pass_kernel<<<grid, 256, 0, st>>>(mode, nbits, shift, S, mm, w.scal, w.state, w.hist, mm, K, w.counts);
         FPSK_LAUNCH_CHECK();
     }
-    select_finish_kernel<<<1, 32, 0, st>>>(mode, w.state, w.scal);
-    FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
 
@@ -469,6 +486,7 @@ void select_carve(void *ws, SelectWs &w)
     w.keys = (unsigned long long *)p; p += align_up(kSelMaxK * 8, 256);
     w.counts = (int *)p; p += 256;
     w.cand = (Candidate *)p;
+    w.hist_clean = false;
 }
 
 }  // namespace fpsk

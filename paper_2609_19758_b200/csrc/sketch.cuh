@@ -73,6 +73,7 @@ struct SelectWs {           // all device memory
     unsigned long long *keys;    // selected keys (<= kmax)
     int *counts;            // [0] above-threshold count, [1] collected, [2] n_U
     Candidate *cand;        // <= kmax
+    bool hist_clean;        // host side: the histogram has been zeroed since this workspace was carved
 };
 constexpr int kSelMaxK = 1024;
 size_t select_ws_bytes();
