@@ -122,13 +122,17 @@ template <typename T, bool VEC, bool MOM, bool PLANES>
 __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A, long long lda, int n1, int n2,
                                                          int kpad, float inv_p1, const uint32_t *rowperm,
                                                          const int *rowstart, float *P, float *Pw, int kblocks,
-                                                         unsigned char *planesP, unsigned char *planesPw)
+                                                         unsigned char *planesP, unsigned char *planesPw, int m_b)
 {
-    const int a = blockIdx.y;
-    const long long col0 = ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    // FP32 output: CTA = one bucket, consecutive threads = consecutive columns.  Plane output: a warp covers
+    // eight consecutive buckets x four k-chunks, because the eight buckets of a k-chunk are one 128-byte
+    // line of the tiled plane (lone 16-byte chunks, one bucket per CTA, take three times as long to store).
+    const int a = PLANES ? (int)blockIdx.y * 8 + (int)(threadIdx.x & 7) : (int)blockIdx.y;
+    const long long col0 = PLANES ? ((long long)blockIdx.x * (blockDim.x / 8) + (threadIdx.x >> 3)) * 8
+                                  : ((long long)blockIdx.x * blockDim.x + threadIdx.x) * 8;
     if (col0 >= (PLANES ? kblocks * 32 : kpad)) return;
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, accw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
-    if (col0 < n2) {
+    if (col0 < n2 && a < m_b) {
         const int s0 = rowstart[a], s1 = rowstart[a + 1];
         for (int s = s0; s < s1; ++s) {
             const uint32_t e = __ldg(rowperm + s);
@@ -665,8 +669,8 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     {
         const bool vec = (reinterpret_cast<uintptr_t>(in.A) & 15) == 0 && in.lda % 8 == 0 && n2 % 8 == 0;
         const int kcols = w.tc ? kblocks * 32 : pl.kpad;
-        dim3 grid((kcols / 8 + 127) / 128, m_b);
-#define FPSK_CA(V, M, PL) compress_a_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw, kblocks, w.planes[0], w.planes[1])
+        dim3 grid = w.tc ? dim3((kcols / 8 + 15) / 16, (m_b + 7) / 8) : dim3((kcols / 8 + 127) / 128, m_b);
+#define FPSK_CA(V, M, PL) compress_a_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw, kblocks, w.planes[0], w.planes[1], m_b)
         if (w.tc) {
             if (vec) { if (mom) FPSK_CA(true, true, true); else FPSK_CA(true, false, true); }
             else     { if (mom) FPSK_CA(false, true, true); else FPSK_CA(false, false, true); }
