@@ -357,6 +357,13 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
 fpsk_status fpsk_apply_corrections(float *C, int64_t ldc, int64_t m, int64_t n, const fpsk_fault *h_faults,
                                    int32_t count, void *workspace, size_t ws_bytes, void *stream);
 
+/* Self-test of the give-up path that every device-side wait of this library has (no counterpart in
+ * the paper).  One thread waits for *d_flag (device, 4 bytes) to become non-zero, with a limit of about
+ * half a millisecond instead of the library's usual second, then writes d_result->status: FPSK_OK if the
+ * flag was set, FPSK_ERR_TIMEOUT if the wait gave up.  The kernel always returns; the context stays usable.
+ * Asynchronous on `stream`. */
+fpsk_status fpsk_selftest_bounded_wait(uint32_t *d_flag, fpsk_probe_result *d_result, void *stream);
+
 /* Number of kernels launched by this library since load (all entry points, all threads). */
 uint64_t fpsk_launch_count(void);
 

@@ -283,6 +283,20 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
     return FPSK_OK;
 }
 
+// Waits, with a short limit, for a flag that the caller leaves at zero: the wait gives up, the kernel
+// reports FPSK_ERR_TIMEOUT in the result and returns normally, like every bounded wait of the library
+// does after its (much longer) limit.
+__global__ void selftest_wait_kernel(const unsigned int *flag, fpsk_probe_result *result)
+{
+    if (threadIdx.x != 0) return;
+    const bool arrived = bounded_wait_ge(flag, 1u, 2048u);        // about half a millisecond
+    fpsk_probe_result r;
+    r.fired = 0; r.nonfinite = 0; r.argmax_col = -1;
+    r.status = arrived ? (int)FPSK_OK : (int)FPSK_ERR_TIMEOUT;
+    r.max_abs = 0.f; r.sigma_hat = 0.f; r.thr = 0.f; r.tau = 0.f;
+    *result = r;
+}
+
 }  // namespace fpsk
 
 using namespace fpsk;
@@ -457,6 +471,15 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
     }
     return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, q.tensor_cores, cache, cache_bytes, workspace, ws_bytes, st,
                          d_result, d_S, d_state);
+}
+
+// ---------------------------------------------------------------- give-up path of the device-side waits
+fpsk_status fpsk_selftest_bounded_wait(uint32_t *d_flag, fpsk_probe_result *d_result, void *stream)
+{
+    if (!d_flag || !d_result) return FPSK_ERR_NULL;
+    selftest_wait_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(d_flag, d_result);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
 }
 
 // ---------------------------------------------------------------- stateful probe

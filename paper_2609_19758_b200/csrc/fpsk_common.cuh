@@ -116,9 +116,9 @@ __device__ __forceinline__ uint4 ldg_nc_v4(const void *p)
 // ---------------------------------------------------------------- bounded device-side wait
 // Spin until *ctr >= target; gives up after a fixed number of polls and returns false, so
 // that a kernel can flag FPSK_ERR_TIMEOUT and leave instead of hanging.
-__device__ __forceinline__ bool bounded_wait_ge(const unsigned int *ctr, unsigned int target)
+__device__ __forceinline__ bool bounded_wait_ge(const unsigned int *ctr, unsigned int target, unsigned int max_polls = 1u << 21)
 {
-    for (unsigned int it = 0; it < (1u << 21); ++it) {
+    for (unsigned int it = 0; it < max_polls; ++it) {
         unsigned int v;
         asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(ctr));
         if (v >= target) return true;

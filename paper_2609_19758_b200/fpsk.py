@@ -145,6 +145,8 @@ def lib() -> C.CDLL:
                                          vp, sz, vp, C.POINTER(Fault), i32, C.POINTER(RepairReport)]
         L.fpsk_apply_corrections.restype = C.c_int
         L.fpsk_apply_corrections.argtypes = [vp, i64, i64, i64, C.POINTER(Fault), i32, vp, sz, vp]
+        L.fpsk_selftest_bounded_wait.restype = C.c_int
+        L.fpsk_selftest_bounded_wait.argtypes = [vp, vp, vp]
         L.fpsk_launch_count.restype = u64
         L.fpsk_launch_count.argtypes = []
         _lib = L
@@ -312,6 +314,13 @@ def probe_accumulate(result: torch.Tensor, state: torch.Tensor, stream=None) -> 
     rc = lib().fpsk_probe_accumulate(result.data_ptr(), state.data_ptr(), _stream_ptr(stream))
     if rc != STATUS_OK:
         raise FpskError(rc, "fpsk_probe_accumulate")
+
+
+def selftest_bounded_wait(flag: torch.Tensor, result: torch.Tensor, stream=None) -> None:
+    """Launch the wait self-test on a 4-byte device flag; read the status with read_probe_result."""
+    rc = lib().fpsk_selftest_bounded_wait(flag.data_ptr(), result.data_ptr(), _stream_ptr(stream))
+    if rc != STATUS_OK:
+        raise FpskError(rc, "fpsk_selftest_bounded_wait")
 
 
 def recalibration_due(calls: int) -> bool:

@@ -342,3 +342,20 @@ def test_localize_capacity_and_bucket_errors():
     with pytest.raises(fpsk.FpskError) as e:
         fpsk.localize(dA, dB, dC, 1, 64, ws, p)                         # workspace sized for 32
     assert e.value.status == fpsk.ERR_WORKSPACE
+
+
+def test_a_device_wait_that_runs_out_reports_timeout_and_leaves_the_context_usable():
+    """Every device-side wait of the library is bounded; this drives the give-up path with a short limit
+    (a flag that nothing sets), then checks that the same stream still runs a probe."""
+    flag = torch.zeros(1, dtype=torch.int32, device="cuda")
+    res = fpsk.new_probe_result()
+    fpsk.selftest_bounded_wait(flag, res)
+    torch.cuda.synchronize()
+    assert fpsk.read_probe_result(res).status == fpsk.ERR_TIMEOUT
+    flag.fill_(1)
+    fpsk.selftest_bounded_wait(flag, res)
+    torch.cuda.synchronize()
+    assert fpsk.read_probe_result(res).status == 0
+    A, Bm, Cm = _case("uniform", 64, 64, 64, W.FP16, 3)
+    got, _, _ = _run_probe(A, Bm, Cm)
+    assert got.status == 0 and got.fired == 0
