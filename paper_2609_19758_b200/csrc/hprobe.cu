@@ -255,19 +255,16 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
         // uA: unit being streamed; uB: the next one; both known, and so are their first chunks RA, RB
         // (lane l holds 16 bytes: ints 4 (l % 4) .. of record l / 4).  uC is fetched while uA streams.
         const int4 *chunks = reinterpret_cast<const int4 *>(p.stages);
-        int uA = 0, uB = 0;
-        if (lane == 0) {
-            uA = (int)atomicAdd(p.ctrl + 2, 1u);
-            uB = (int)atomicAdd(p.ctrl + 2, 1u);
-        }
-        uA = __shfl_sync(0xFFFFFFFFu, uA, 0);
-        uB = __shfl_sync(0xFFFFFFFFu, uB, 0);
+        // the first two units of every team are fixed (no round trip to the counter before the first copy);
+        // the counter hands out the units after those
+        const int nteams = 2 * (int)gridDim.x;
+        int uA = 2 * c + team, uB = uA + nteams;
         const int4 zero4 = make_int4(0, 0, 0, 0);
         int4 RA = uA < U ? __ldg(chunks + (long long)uA * 32 + lane) : zero4;
         int4 RB = uB < U ? __ldg(chunks + (long long)uB * 32 + lane) : zero4;
         while (uA < U && ok) {
             int uC = 0;
-            if (lane == 0) uC = (int)atomicAdd(p.ctrl + 2, 1u);          // needed when this unit is done
+            if (lane == 0) uC = 2 * nteams + (int)atomicAdd(p.ctrl + 2, 1u);          // needed when this unit is done
             int4 R = RA;
             for (;;) {
                 const unsigned int lastmask = __ballot_sync(0xFFFFFFFFu, (lane & 3) == 0 && (R.z & 0x100));
@@ -548,6 +545,7 @@ struct HvArgs {
     unsigned int *ctrl;      // [0] ticket, [1] error flag, [2] unit counter of the streaming kernel, [3] statistics published
     fpsk_probe_result *result;
     fpsk_probe_state *state; // accumulated into when not null
+    unsigned long long *ctrace;   // time stamps per CTA when tracing (8 each), else null
 };
 
 struct HvMax {
@@ -641,6 +639,10 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
     __shared__ int s_flag;
     const int c = blockIdx.x, G = gridDim.x, tid = threadIdx.x;
     const long long mm = (long long)p.m * p.m;
+    // time stamps for FPSK_HPROBE_TRACE (0 entry, 1 partials loaded, 2 joined, 3 all published, 4 totals,
+    // 5 clipped sum, 6 ticket, 7 verdict)
+#define CT(k) do { if (p.ctrace && tid == 0) p.ctrace[c * 8 + (k)] = hp_gtime(); } while (0)
+    CT(0);
     // ranges in units of 4 buckets (the tail CTA takes the remainder of an m^2 that is not a multiple of 4)
     const long long q4 = (mm + 3) / 4;
     const long long i0 = 4 * (q4 * c / G), i1 = min(mm, 4 * (q4 * (c + 1) / G));
@@ -669,7 +671,9 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
         if (!(av <= 3.4028234663852886e38f)) l.bad += 1.f;          // Inf or NaN
         else l.mx = hv_better(l.mx, HvMax{av, (int)i});
     }
+    CT(1);
     l = hv_block_join(l, slot0);
+    CT(2);
     if (tid == 0) {
         __stcg(p.vstat + c, make_float4(l.sum, l.bad, l.mx.v, __int_as_float(l.mx.i)));
         red_release_add(p.ctrl + 3);
@@ -677,6 +681,7 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
         if (!s_flag) atomicOr(p.ctrl + 1, 1u);
     }
     __syncthreads();
+    CT(3);
     const bool ok = s_flag != 0;
     // ---- the same totals in every CTA: records in CTA order, thread-strided, then the fixed shape
     HvStat t = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
@@ -687,6 +692,7 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
         }
     }
     t = hv_block_join(t, slot1);
+    CT(4);
     const float mean = t.sum / (float)mm;
     const bool slow = !(t.mx.v <= 5.f * mean) || t.bad > 0.f;
     if (slow) {
@@ -696,12 +702,14 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
         cs = hv_block_join(cs, slot2);
         if (tid == 0) __stcg(p.cstat + c, cs.sum);
     }
+    CT(5);
     if (tid == 0) {
         __threadfence();
         const unsigned int tk = atom_acq_rel_add(p.ctrl + 0);
         s_flag = (tk == (unsigned int)(G - 1)) ? 1 : 0;
     }
     __syncthreads();
+    CT(6);
     if (!s_flag) return;
     __threadfence();
     // ---- last CTA
@@ -734,10 +742,12 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
         r.thr = thr;
         r.tau = tau;
         *p.result = r;
+        if (p.ctrace) p.ctrace[c * 8 + 7] = hp_gtime();
         if (p.state) state_accumulate(p.state, r);
         // counters ready for the next call on this workspace
         p.ctrl[0] = 0; p.ctrl[1] = 0; p.ctrl[2] = 0; p.ctrl[3] = 0;
     }
+#undef CT
 }
 
 // ---------------------------------------------------------------- host side
@@ -836,7 +846,7 @@ static size_t hp_work_layout(void *base, long long n1, long long n2, long long n
     t.Pplanes = (unsigned char *)take(tc_planes_bytes(m, pl.kpad));
     t.partC = (float *)take((size_t)pl.segsC * m * m * 4);
     t.S = (float *)take((size_t)m * m * 4);
-    t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 128);       // 8 stamps per team
+    t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 256);       // 8 stamps per team
     if (w) *w = t;
     return off;
 }
@@ -973,6 +983,7 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);
     v.S = d_S ? d_S : w.S;
     v.vstat = w.vstat; v.cstat = w.cstat; v.ctrl = w.ctrl; v.result = d_result; v.state = d_state;
+    v.ctrace = a.trace_on ? w.trace + 8 * 2 * sms : nullptr;
     {
         // cooperative: every CTA waits (bounded) for the statistics of all others
         int grid = sms < kHvMaxGrid ? sms : kHvMaxGrid;
