@@ -23,6 +23,7 @@ struct SketchWs {
     SketchPlan pl;
     int *h1, *v1, *h2, *v2;
     uint32_t *rowperm, *colperm;
+    uint32_t *colpos;            // inverse of colperm: position (and sign) of every column in the bucket-sorted order
     int *rowcount, *rowstart, *colcount, *colstart;
     float *P, *Pw, *Q, *Qw, *partAB, *partC;
     bool tc;                     // split-BF16 tensor-core contraction
@@ -43,7 +44,7 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
 int sketch_max_buckets(long long n1, long long n2, long long n3);
 
 fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, int *bucket, int *sign,
-                            int *count, int *start, uint32_t *perm, cudaStream_t st);
+                            int *count, int *start, uint32_t *perm, cudaStream_t st, uint32_t *pos = nullptr);
 fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
                            SketchWs &w, cudaStream_t st, float *S, float *R, float *T);
 // start[0..n] = exclusive prefix sums of count[0..n)  (one CTA, any n)
