@@ -199,7 +199,8 @@ typedef struct {
     int32_t dtype, n_buckets, round;
     int32_t valid;        /* 0: nothing cached                                                 */
     int32_t rebuilds;     /* how many times the B side was (re)built through this record       */
-    int32_t reserved;
+    int32_t b_transposed; /* set by the caller before the first call: 0 = the B pointer is B (k x n, row-major);
+                             1 = it is W = B^T (n x k, row-major, ldb >= k), the x W^T weight layout  */
 } fpsk_bside;
 
 /* State of a probe across calls; see "what the probe keeps between calls" below. */
@@ -229,6 +230,8 @@ int32_t fpsk_bside_matches(const fpsk_bside *side, const void *B, int64_t ldb, u
  * over the n_buckets^2 buckets, thr = min(tau sqrt(m n / n_buckets^2), mu sqrt(2 ln n_buckets^2) sigma_hat)
  * (Section "Thresholds"; a bucket sums m n / n_buckets^2 entries of E on average, so the analytic
  * cap enters with the root of that population), dirty iff max|S| > thr or S is not finite.
+ *   B, ldb        B itself, or, with side->b_transposed = 1, the weight W = B^T as n x k row-major
+ *                 (C = A W^T); only the (re)build of the B side reads it
  *   side, cache   the B side.  When `side` does not match the key (see fpsk_bside), it is rebuilt
  *                 into `cache` first (reads B once; side->rebuilds is incremented); on a match B
  *                 is not read: the call reads 2mk + 4mn bytes.  Bump b_version after every in-place

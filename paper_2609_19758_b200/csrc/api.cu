@@ -453,8 +453,10 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
 {
     if (!c_is_fp32) return FPSK_ERR_DTYPE;      // a narrowed C is rejected, not tolerated
     if (!side || !cache || !workspace || !d_result) return FPSK_ERR_NULL;
-    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    const bool bt = side->b_transposed != 0;
+    fpsk_status rc = check_mats(A, lda, B, bt ? n : ldb, C, ldc, m, k, n, dtype);      // W is n x k: its own check below
     if (rc != FPSK_OK) return rc;
+    if (bt && ldb < k) return FPSK_ERR_SHAPE;
     if (n_buckets < 1 || n_buckets > 4096 || round < 0) return FPSK_ERR_BUCKETS;
     if ((reinterpret_cast<uintptr_t>(cache) & 255) || (reinterpret_cast<uintptr_t>(workspace) & 255)) return FPSK_ERR_ALIGN;
     if (cache_bytes < hprobe_cache_bytes(m, k, n, n_buckets) || ws_bytes < hprobe_ws_bytes(m, k, n, n_buckets))
@@ -463,7 +465,7 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!fpsk_bside_matches(side, B, ldb, b_version, m, k, n, dtype, seed, round, n_buckets, cache)) {
         side->valid = 0;
-        rc = hprobe_prepare(B, ldb, m, k, n, dtype, seed, round, n_buckets, cache, cache_bytes, st);
+        rc = hprobe_prepare(B, ldb, bt ? 1 : 0, m, k, n, dtype, seed, round, n_buckets, cache, cache_bytes, st);
         if (rc != FPSK_OK) return rc;
         side->B = B; side->cache = cache; side->ldb = ldb; side->m = m; side->k = k; side->n = n;
         side->seed = seed; side->version = b_version; side->dtype = (int32_t)dtype; side->n_buckets = n_buckets;

@@ -750,6 +750,28 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
 #undef CT
 }
 
+// Q = B H2^T from the transposed weight W = B^T (n3 x n2, row-major): thread (bucket b, column k) adds the
+// rows of W that fall in bucket b in ascending row order (the order in which the untransposed path adds
+// the columns of B).  Runs once per B side; Q is kpad x npad with zero padding.
+template <typename T>
+__global__ void __launch_bounds__(256) hp_compress_wt_kernel(const unsigned short *W, long long ldw, int n2, int m_b, int kpad,
+                                                             int npad, const uint32_t *colperm, const int *colstart, float *Q)
+{
+    const int k = blockIdx.x * blockDim.x + threadIdx.x;
+    const int b = blockIdx.y;
+    if (k >= kpad) return;
+    float q = 0.f;
+    if (k < n2 && b < m_b) {
+        const int s0 = __ldg(colstart + b), s1 = __ldg(colstart + b + 1);
+        for (int s = s0; s < s1; ++s) {
+            const uint32_t e = __ldg(colperm + s);
+            const float x = bits16_to_float<T>(W[(long long)(e & 0x7FFFFFFFu) * ldw + k]);
+            q += (e >> 31) ? -x : x;
+        }
+    }
+    Q[(long long)k * npad + b] = q;
+}
+
 // ---------------------------------------------------------------- host side
 struct HpPlan {
     int kpad, npad, segsA, segsC, tile, ksplit, kchunk;
@@ -888,7 +910,7 @@ static HpArgs hp_args(const void *A, long long lda, const float *C, long long ld
 }
 
 // Build the B side: both hash tables of the round, Q = B H2^T, max|B| and the unit partition.
-fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long n2, long long n3, fpsk_dtype dtype,
+fpsk_status hprobe_prepare(const void *B, long long ldb, int b_transposed, long long n1, long long n2, long long n3, fpsk_dtype dtype,
                            uint64_t seed, int rnd, int m, void *cache, size_t cache_bytes, cudaStream_t st)
 {
     const int sms = hp_sm_count();
@@ -900,11 +922,20 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long
     if (rc != FPSK_OK) return rc;
     rc = build_hash_side(seed, rnd, 1, (int)n3, m, c.h2, c.v2, c.colcount, c.colstart, c.colperm, st);
     if (rc != FPSK_OK) return rc;
-    rc = build_b_side(B, ldb, n2, n3, dtype, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q, st);
-    if (rc != FPSK_OK) return rc;
+    if (b_transposed) {
+        // the weight as W = B^T (n3 x n2): bucket b of Q = B H2^T is the signed sum of the rows of W in bucket b
+        dim3 grid((pl.kpad + 255) / 256, pl.npad);
+        if (dtype == FPSK_FP16) hp_compress_wt_kernel<__half><<<grid, 256, 0, st>>>(static_cast<const unsigned short *>(B), ldb, (int)n2, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q);
+        else hp_compress_wt_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<const unsigned short *>(B), ldb, (int)n2, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q);
+        FPSK_LAUNCH_CHECK();
+    } else {
+        rc = build_b_side(B, ldb, n2, n3, dtype, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q, st);
+        if (rc != FPSK_OK) return rc;
+    }
     rc = tc_split_launch(c.Q, 1, pl.npad, m, pl.kpad, 1, c.Qplanes, st);      // row b of Q^T is column b of Q
     if (rc != FPSK_OK) return rc;
-    rc = max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
+    rc = b_transposed ? max_abs_half_launch(B, ldb, n3, n2, dtype, c.maxB, c.scratch, st)
+                      : max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
     if (rc != FPSK_OK) return rc;
     const HpArgs a = hp_args(nullptr, 0, nullptr, 0, n1, n2, n3, m, pl, c, nullptr);
     hp_segment_lists_kernel<<<pl.segsC, 256, (size_t)(m + 1) * 4, st>>>(c.h2, c.v2, (int)n3, m, c.segperm, c.segstart);

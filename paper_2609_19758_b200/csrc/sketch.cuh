@@ -141,7 +141,7 @@ constexpr int kTcMinBuckets = 384;      // below this the FP32 FMA contraction i
 // ---- the S only probe with a cached B side (hprobe.cu) ------------------------------------------
 size_t hprobe_cache_bytes(long long n1, long long n2, long long n3, int m);
 size_t hprobe_ws_bytes(long long n1, long long n2, long long n3, int m);
-fpsk_status hprobe_prepare(const void *B, long long ldb, long long n1, long long n2, long long n3, fpsk_dtype dtype,
+fpsk_status hprobe_prepare(const void *B, long long ldb, int b_transposed, long long n1, long long n2, long long n3, fpsk_dtype dtype,
                            uint64_t seed, int rnd, int m, void *cache, size_t cache_bytes, cudaStream_t st);
 fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
                           long long n3, fpsk_dtype dtype, int m, double mu, int tensor_cores, void *cache, size_t cache_bytes, void *ws,

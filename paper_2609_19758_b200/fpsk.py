@@ -54,7 +54,7 @@ class BSide(C.Structure):
     _fields_ = [("B", C.c_void_p), ("cache", C.c_void_p), ("ldb", C.c_int64), ("m", C.c_int64), ("k", C.c_int64),
                 ("n", C.c_int64), ("seed", C.c_uint64), ("version", C.c_uint64), ("dtype", C.c_int32),
                 ("n_buckets", C.c_int32), ("round", C.c_int32), ("valid", C.c_int32), ("rebuilds", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("b_transposed", C.c_int32)]
 
 
 class ProbeState(C.Structure):
@@ -248,11 +248,29 @@ def probe_static(A, B, Cm, result: torch.Tensor, residual: Optional[torch.Tensor
         raise FpskError(rc, "fpsk_probe_static")
 
 
+class _ShapeOnly:
+    """Stands in for a k x n operand in the argument checks when the caller holds its transpose."""
+
+    def __init__(self, W: torch.Tensor, k: int, n: int):
+        self.is_cuda, self.dtype, self.shape, self._W = W.is_cuda, W.dtype, (k, n), W
+
+    def dim(self):
+        return 2
+
+    def stride(self, d):
+        return 1 if d == 1 else self.shape[1]
+
+    def data_ptr(self):
+        return self._W.data_ptr()
+
+
 class HashedProbe:
     """Buffers of the S only probe with a cached B side: the host record, the device cache and the
     per-call workspace (torch owns the memory).  ``__call__`` is one asynchronous probe."""
 
-    def __init__(self, m: int, k: int, n: int, n_buckets: int, seed: int, rnd: int = 0, device=None, stream=None):
+    def __init__(self, m: int, k: int, n: int, n_buckets: int, seed: int, rnd: int = 0, device=None, stream=None,
+                 b_transposed: bool = False):
+        """b_transposed: the B argument of the calls is the weight W = B^T (n x k, row-major): C = A W^T."""
         self.shape = (m, k, n)
         self.n_buckets, self.seed, self.round = n_buckets, seed, rnd
         cb = int(lib().fpsk_probe_hashed_cache_bytes(m, k, n, n_buckets))
@@ -265,17 +283,28 @@ class HashedProbe:
         if rc != STATUS_OK:
             raise FpskError(rc, "fpsk_probe_init")
         self.side = BSide()
+        self.side.b_transposed = 1 if b_transposed else 0
 
     def matches(self, B: torch.Tensor, b_version: int) -> bool:
         m, k, n = self.shape
-        ldb = B.stride(0) if k > 1 else max(n, B.stride(0))
+        if self.side.b_transposed:
+            ldb = B.stride(0) if n > 1 else max(k, B.stride(0))
+        else:
+            ldb = B.stride(0) if k > 1 else max(n, B.stride(0))
         return bool(lib().fpsk_bside_matches(C.byref(self.side), B.data_ptr(), ldb, b_version, m, k, n, dtype_of(B),
                                              self.seed, self.round, self.n_buckets, self.cache.data_ptr()))
 
     def __call__(self, A, B, Cm, result: torch.Tensor, b_version: int = 0, S: Optional[torch.Tensor] = None,
                  params: Optional[Params] = None, stream=None, c_is_fp32: Optional[bool] = None,
                  state: Optional[torch.Tensor] = None) -> None:
-        a = _mat_args(A, B, Cm)
+        if self.side.b_transposed:
+            # B is the weight W (n x k): marshal A and C as usual, W with its own leading dimension
+            m, k, n = self.shape
+            assert B.is_cuda and B.dim() == 2 and B.stride(1) == 1 and tuple(B.shape) == (n, k) and B.dtype == A.dtype
+            a = list(_mat_args(A, _ShapeOnly(B, k, n), Cm))
+            a[2], a[3] = B.data_ptr(), (B.stride(0) if n > 1 else max(k, B.stride(0)))
+        else:
+            a = _mat_args(A, B, Cm)
         assert (a[6], a[7], a[8]) == self.shape
         if c_is_fp32 is None:
             c_is_fp32 = Cm.dtype == torch.float32

@@ -283,3 +283,31 @@ def test_recalibration_from_the_accumulated_noise():
     # the oracle's sketch at the same bucket count gives the same plan input
     ref, _ = O.probe_hashed(_f64(A), _f64(Bm), Cm.numpy(), 6, 0, m)
     assert sigma_bar == pytest.approx(ref.sigma_hat, rel=0.05)
+
+
+# ---------------------------------------------------------------- weight stored transposed (C = A W^T)
+@pytest.mark.parametrize("shape,m,dtype", [((512, 256, 384), 32, W.BF16), ((1024, 1032, 2048), 128, W.FP16),
+                                           ((130, 72, 100), 5, W.BF16)])
+def test_transposed_weight_layout(shape, m, dtype):
+    n1, n2, n3 = shape
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, dtype, 23)
+    Cm[n1 // 2, n3 // 3] += 0.75
+    Wt = Bm.t().contiguous()                                   # n3 x n2, what an x W^T layer holds
+    ref, S_ref = O.probe_hashed(_f64(A), _f64(Wt).T, Cm.numpy(), 17, 1, m)
+    h1, _ = O.hash_round(17, 1, 0, n1, m)
+    h2, _ = O.hash_round(17, 1, 1, n3, m)
+    denom = O.abs_sketch(O.abs_product(_f64(A), _f64(Bm)), h1, h2, m)
+    hp_t = fpsk.HashedProbe(n1, n2, n3, m, seed=17, rnd=1, b_transposed=True)
+    got_t, S_t = _run(hp_t, A.cuda(), Wt.cuda(), Cm.cuda())
+    assert got_t.status == 0 and got_t.fired == 1 and ref.fired and got_t.argmax_col == ref.argmax_col
+    assert np.all(np.abs(S_t - S_ref) <= TOL * denom + 1e-30)
+    # same additions in the same order as the untransposed layout: identical bits
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=17, rnd=1)
+    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda())
+    assert np.array_equal(S, S_t) and got.tau == got_t.tau and got.sigma_hat == got_t.sigma_hat
+    # a padded leading dimension of W
+    big = torch.zeros(n3, n2 + 16, dtype=Wt.dtype, device="cuda")
+    big[:, :n2] = Wt.cuda()
+    hp_p = fpsk.HashedProbe(n1, n2, n3, m, seed=17, rnd=1, b_transposed=True)
+    got_p, S_p = _run(hp_p, A.cuda(), big[:, :n2], Cm.cuda())
+    assert np.array_equal(S_p, S_t)
