@@ -84,6 +84,11 @@ typedef struct {
     int32_t delta_max;   /* declared bound Delta on faults per row or column               */
     int32_t mad_of_abs;  /* 1: MAD of |S| as printed in the paper; 0: signed MAD of S      */
     int32_t tensor_cores;/* 0: FP32 FMA contraction; 1: split-BF16 tcgen05 contraction     */
+    int32_t b_transposed;/* fpsk_measure_noise, fpsk_localize: 1 = the B pointer is the weight
+                            W = B^T (n x k, row-major, ldb >= k), i.e. C = A W^T; 0 = B is k x n.
+                            Other entry points take B as k x n (fpsk_probe_hashed has its own
+                            switch in fpsk_bside).                                          */
+    int32_t reserved;
     double rho_min;      /* smallest fault to localize, in units of rms(C)                 */
     double c_valid;      /* c of tau_ij = c eps sum_k |A_ik||B_kj|                         */
     double mu;           /* probe margin                                                   */

@@ -79,7 +79,7 @@ static bool params_ok(const fpsk_params &p)
 {
     return p.rounds >= 1 && p.rounds <= 8 && p.r_star >= 0 && p.r_max >= 0 && p.r_max <= 16 && p.radius >= -1 &&
            p.radius <= 16 && p.s_budget >= 1 && p.delta_max >= 1 && p.rho_min > 0 && p.c_valid > 0 && p.mu > 0 &&
-           p.b_star > 0 && p.c_coll > 1.0 - 1e-12;
+           p.b_star > 0 && p.c_coll > 1.0 - 1e-12 && (p.b_transposed == 0 || p.b_transposed == 1);
 }
 
 static fpsk_params resolve_params(const fpsk_params *p)
@@ -91,11 +91,11 @@ static fpsk_params resolve_params(const fpsk_params *p)
 }
 
 static fpsk_status check_mats(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
-                              int64_t m, int64_t k, int64_t n, fpsk_dtype dtype)
+                              int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, bool b_transposed = false)
 {
     if (!A || !B || !C) return FPSK_ERR_NULL;
     if (dtype != FPSK_FP16 && dtype != FPSK_BF16) return FPSK_ERR_DTYPE;
-    if (m < 1 || k < 1 || n < 1 || lda < k || ldb < n || ldc < n) return FPSK_ERR_SHAPE;
+    if (m < 1 || k < 1 || n < 1 || lda < k || ldb < (b_transposed ? k : n) || ldc < n) return FPSK_ERR_SHAPE;
     if (m >= (1LL << 30) || k >= (1LL << 30) || n >= (1LL << 30)) return FPSK_ERR_SHAPE;
     return FPSK_OK;
 }
@@ -170,7 +170,8 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
     unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
     rc = max_abs_half_launch(in.A, in.lda, m, k, dtype, w.misc + 0, uscr, st);
     if (rc != FPSK_OK) return rc;
-    rc = max_abs_half_launch(in.B, in.ldb, k, n, dtype, w.misc + 1, uscr + 1, st);
+    rc = in.bt ? max_abs_half_launch(in.B, in.ldb, n, k, dtype, w.misc + 1, uscr + 1, st)
+               : max_abs_half_launch(in.B, in.ldb, k, n, dtype, w.misc + 1, uscr + 1, st);
     if (rc != FPSK_OK) return rc;
     tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
     FPSK_LAUNCH_CHECK();
@@ -377,7 +378,7 @@ fpsk_status fpsk_probe(const void *A, int64_t lda, const void *B, int64_t ldb, c
     if (!workspace || !d_result) return FPSK_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
     const fpsk_params q = resolve_params(p);
-    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    if (!params_ok(q) || q.b_transposed) return FPSK_ERR_PARAM;      // this probe streams B as k x n
     ProbeDims d{m, k, n, lda, ldb, ldc};
     return probe_launch(A, B, C, d, dtype, q.mu, workspace, ws_bytes, static_cast<cudaStream_t>(stream), d_result,
                         d_residual);
@@ -569,7 +570,7 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
                                int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t m0,
                                const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream, fpsk_noise *h_out)
 {
-    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype, p && p->b_transposed);
     if (rc != FPSK_OK) return rc;
     if (!workspace || !h_out) return FPSK_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
@@ -580,7 +581,7 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     LocWs w;
     if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
     rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
     if (rc != FPSK_OK) return rc;
     const long long mm = (long long)m0 * m0;
@@ -627,7 +628,7 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
                           const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream, fpsk_fault *h_faults,
                           int32_t capacity, int32_t *h_count)
 {
-    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype, p && p->b_transposed);
     if (rc != FPSK_OK) return rc;
     if (!workspace || !h_count || (capacity > 0 && !h_faults)) return FPSK_ERR_NULL;
     if (capacity < 0) return FPSK_ERR_PARAM;
@@ -637,7 +638,7 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
     if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     LocWs w;
     if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
-    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
     *h_count = 0;
     std::vector<fpsk_fault> F;
     bool truncated = false;
@@ -709,7 +710,7 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
     if (capacity < 0) return FPSK_ERR_PARAM;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
     const fpsk_params q = resolve_params(p);
-    if (!params_ok(q)) return FPSK_ERR_PARAM;
+    if (!params_ok(q) || q.b_transposed) return FPSK_ERR_PARAM;      // the repair path reads B as k x n
     if (n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     if (ws_bytes < fpsk_repair_workspace_bytes(m, k, n, n_buckets, p) || fpsk_repair_workspace_bytes(m, k, n, n_buckets, p) == 0)
         return FPSK_ERR_WORKSPACE;

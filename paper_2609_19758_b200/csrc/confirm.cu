@@ -16,7 +16,7 @@ template <typename T>
 __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
     const unsigned short *A, long long lda, const unsigned short *B, long long ldb, const float *C, long long ldc,
     long long n1, long long n2, long long n3, const Candidate *cand, const int *n_cand, int r, double c_valid, int force,
-    Hit *hits, int *n_hits, int hit_cap)
+    Hit *hits, int *n_hits, int hit_cap, int bt)
 {
     __shared__ double sg[kConfirmThreads];
     __shared__ double sa[kConfirmThreads];
@@ -33,10 +33,12 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
     double g = 0.0, ab = 0.0;
     if (active) {
         const unsigned short *arow = A + i * lda;
-        const unsigned short *bcol = B + j;
+        // column j of B: strided in B, or row j of the transposed weight
+        const unsigned short *bcol = bt ? B + j * ldb : B + j;
+        const long long bstep = bt ? 1 : ldb;
         for (long long k = ks; k < n2; k += slices) {
             const double a = (double)bits16_to_float<T>(arow[k]);
-            const double b = (double)bits16_to_float<T>(bcol[k * ldb]);
+            const double b = (double)bits16_to_float<T>(bcol[k * bstep]);
             const double p = a * b;          // exact: two <= 11-bit significands
             g += p;
             ab += fabs(p);
@@ -75,11 +77,11 @@ fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate
     const unsigned short *B = static_cast<const unsigned short *>(in.B);
     if (dtype == FPSK_FP16)
         confirm_kernel<__half><<<grid, kConfirmThreads, 0, st>>>(A, in.lda, B, in.ldb, in.C, in.ldc, in.n1, in.n2, in.n3,
-                                                                 cand, n_cand, radius, c_valid, force, hits, n_hits, hit_cap);
+                                                                 cand, n_cand, radius, c_valid, force, hits, n_hits, hit_cap, in.bt);
     else
         confirm_kernel<__nv_bfloat16><<<grid, kConfirmThreads, 0, st>>>(A, in.lda, B, in.ldb, in.C, in.ldc, in.n1, in.n2,
                                                                         in.n3, cand, n_cand, radius, c_valid, force, hits, n_hits,
-                                                                        hit_cap);
+                                                                        hit_cap, in.bt);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }

@@ -53,7 +53,7 @@ extern "C" fpsk_status fpsk_probe_static(const void *A, int64_t lda, const void 
     if (m >= (1LL << 30) || k >= (1LL << 30) || n >= (1LL << 30)) return FPSK_ERR_SHAPE;
     double mu = 4.0;
     if (p) {
-        if (!(p->mu > 0)) return FPSK_ERR_PARAM;
+        if (!(p->mu > 0) || p->b_transposed) return FPSK_ERR_PARAM;      // B is streamed as k x n here
         mu = p->mu;
     }
     // shapes whose scratch does not fit the built-in array are refused, never truncated

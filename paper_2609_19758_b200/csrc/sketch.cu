@@ -237,6 +237,78 @@ __global__ void __launch_bounds__(256) compress_b_kernel(const unsigned short *B
     }
 }
 
+// ---------------------------------------------------------------- B compression from the transposed weight
+// B given as W = B^T (n3 x n2, row-major: the x W^T layout of a linear layer).  Column j of B is row j of W, so
+// the fold over the columns of bucket b is a sum of rows of W, the mirror image of the A compression: a thread
+// owns eight adjacent k of one bucket and walks the bucket's rows in ascending j, which is the order of
+// additions of the kernels above (same bits).  Lanes: eight consecutive buckets x four k-chunks per warp, so
+// that a warp stores whole 128-byte lines of the tiled planes (32-byte runs of the FP32 rows of Q).  Writes the
+// padding too: buckets up to bmax and k up to kend are zeros.
+template <typename T, bool VEC, bool MOM, bool PLANES>
+__global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *Wt, long long ldw, int n2, int n3,
+                                                          int kpad, int m_b, int npad, float inv_p3,
+                                                          const uint32_t *colperm, const int *colstart, float *Q,
+                                                          float *Qw, int kblocks, int btiles, unsigned char *planesQ,
+                                                          unsigned char *planesQw)
+{
+    const int b = (int)blockIdx.y * 8 + (int)(threadIdx.x & 7);
+    const int k0 = ((int)blockIdx.x * (int)(blockDim.x / 8) + (int)(threadIdx.x >> 3)) * 8;
+    const int kend = PLANES ? kblocks * 32 : kpad;
+    const int bmax = PLANES ? btiles * 256 : npad;
+    if (k0 >= kend || b >= bmax) return;
+    float q[8] = {0, 0, 0, 0, 0, 0, 0, 0}, qw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (k0 < n2 && b < m_b) {
+        const int s0 = colstart[b], s1 = colstart[b + 1];
+        for (int s = s0; s < s1; ++s) {
+            const uint32_t e = __ldg(colperm + s);
+            const int j = (int)(e & 0x7FFFFFFFu);
+            const float sg = (e >> 31) ? -1.f : 1.f;
+            uint4 v;
+            if (VEC) v = ldg_nc_v4(Wt + (long long)j * ldw + k0);
+            else {
+                unsigned int w[4] = {0, 0, 0, 0};
+                for (int t = 0; t < 8; ++t)
+                    if (k0 + t < n2) w[t >> 1] |= (unsigned int)Wt[(long long)j * ldw + k0 + t] << ((t & 1) * 16);
+                v = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+            const float swj = sg * ((float)(j + 1) * inv_p3);
+            const unsigned int ww[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) {
+                float2 f = HalfTraits<T>::unpack2(ww[t]);
+                q[2 * t] += sg * f.x;
+                q[2 * t + 1] += sg * f.y;
+                if (MOM) {
+                    qw[2 * t] = fmaf(swj, f.x, qw[2 * t]);
+                    qw[2 * t + 1] = fmaf(swj, f.y, qw[2 * t + 1]);
+                }
+            }
+        }
+    }
+    if (PLANES) {
+        const size_t off = plane_chunk_offset<256>(b, k0, kblocks);
+        uint4 hi, mid, lo;
+        split8_bf16(q, hi, mid, lo);
+        *reinterpret_cast<uint4 *>(planesQ + off) = hi;
+        *reinterpret_cast<uint4 *>(planesQ + off + 256 * 64) = mid;
+        *reinterpret_cast<uint4 *>(planesQ + off + 2 * 256 * 64) = lo;
+        if (MOM) {
+            split8_bf16(qw, hi, mid, lo);
+            *reinterpret_cast<uint4 *>(planesQw + off) = hi;
+            *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = mid;
+            *reinterpret_cast<uint4 *>(planesQw + off + 2 * 256 * 64) = lo;
+        }
+        return;
+    }
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+        if (k0 + t < kpad) {
+            Q[(long long)(k0 + t) * npad + b] = q[t];
+            if (MOM) Qw[(long long)(k0 + t) * npad + b] = qw[t];
+        }
+    }
+}
+
 // ---------------------------------------------------------------- C scatter
 // CTA (x: bucket row a, y: split).  The rows of bucket a (ascending) are divided among the
 // splits; each row of C is staged in shared memory and folded over its columns by bucket;
@@ -804,7 +876,22 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
 #undef FPSK_CA
         FPSK_LAUNCH_CHECK();
     }
-    if (b8) {
+    if (in.bt) {
+        const bool vec = (reinterpret_cast<uintptr_t>(in.B) & 15) == 0 && in.ldb % 8 == 0 && n2 % 8 == 0;
+        const int kcols = w.tc ? kblocks * 32 : pl.kpad;
+        const int bmax = w.tc ? btiles * 256 : pl.npad;
+        dim3 grid((kcols / 8 + 15) / 16, (bmax + 7) / 8);
+#define FPSK_CW(V, M, PL) compress_wt_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3])
+        if (w.tc) {
+            if (vec) { if (mom) FPSK_CW(true, true, true); else FPSK_CW(true, false, true); }
+            else     { if (mom) FPSK_CW(false, true, true); else FPSK_CW(false, false, true); }
+        } else {
+            if (vec) { if (mom) FPSK_CW(true, true, false); else FPSK_CW(true, false, false); }
+            else     { if (mom) FPSK_CW(false, true, false); else FPSK_CW(false, false, false); }
+        }
+#undef FPSK_CW
+        FPSK_LAUNCH_CHECK();
+    } else if (b8) {
         const size_t smem = (size_t)16 * ((n3 + 7) & ~7);
         const int groups = (w.tc ? kblocks * 32 : pl.kpad) / 8;
         const int grid = groups < 888 ? groups : 888;
@@ -834,7 +921,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     if (w.tc) {
         // split-BF16 contraction on the tensor cores, one launch for all problems
         FPSK_CUDA_OK(cudaMemsetAsync(w.tc_err, 0, 4, st));
-        if (!b8) {
+        if (!b8 && !in.bt) {
             // wide B: Q, Qw came out as FP32 rows; split them here (row b of Q^T is column b of Q)
             rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], st);
             if (rc != FPSK_OK) return rc;

@@ -36,6 +36,7 @@ struct SketchIn {
     const void *A, *B;
     const float *C;
     long long n1, n2, n3, lda, ldb, ldc;
+    int bt = 0;      // 1: B points to W = B^T (n3 x n2, row-major, leading dimension ldb)
 };
 
 void sketch_plan(long long n1, long long n2, long long n3, int m_b, SketchPlan &pl);

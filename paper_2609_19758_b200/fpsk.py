@@ -34,6 +34,7 @@ class Fault(C.Structure):
 class Params(C.Structure):
     _fields_ = [("rounds", C.c_int32), ("r_star", C.c_int32), ("r_max", C.c_int32), ("radius", C.c_int32),
                 ("s_budget", C.c_int32), ("delta_max", C.c_int32), ("mad_of_abs", C.c_int32), ("tensor_cores", C.c_int32),
+                ("b_transposed", C.c_int32), ("reserved", C.c_int32),
                 ("rho_min", C.c_double), ("c_valid", C.c_double), ("mu", C.c_double), ("b_star", C.c_double),
                 ("c_coll", C.c_double)]
 
@@ -182,16 +183,21 @@ def _stream_ptr(stream: Optional[torch.cuda.Stream]) -> int:
     return int(s.cuda_stream)
 
 
-def _mat_args(A: torch.Tensor, B: torch.Tensor, Cm: torch.Tensor):
+def _mat_args(A: torch.Tensor, B: torch.Tensor, Cm: torch.Tensor, b_transposed: bool = False):
+    """(A, lda, B, ldb, C, ldc, m, k, n, dtype); with b_transposed, B is the weight W = B^T of shape (n, k)."""
     assert A.is_cuda and B.is_cuda and Cm.is_cuda, "A, B, C must be device tensors"
     assert A.dim() == 2 and B.dim() == 2 and Cm.dim() == 2
     assert A.stride(1) == 1 and B.stride(1) == 1 and Cm.stride(1) == 1, "row-major (unit column stride) required"
     m, k = A.shape
-    k2, n = B.shape
+    if b_transposed:
+        n, k2 = B.shape
+    else:
+        k2, n = B.shape
     assert k2 == k and tuple(Cm.shape) == (m, n) and A.dtype == B.dtype
+    brows, bcols = B.shape
     return (A.data_ptr(), A.stride(0) if m > 1 else max(k, A.stride(0)), B.data_ptr(),
-            B.stride(0) if k > 1 else max(n, B.stride(0)), Cm.data_ptr(), Cm.stride(0) if m > 1 else max(n, Cm.stride(0)),
-            m, k, n, dtype_of(A))
+            B.stride(0) if brows > 1 else max(bcols, B.stride(0)), Cm.data_ptr(),
+            Cm.stride(0) if m > 1 else max(n, Cm.stride(0)), m, k, n, dtype_of(A))
 
 
 def law_m_start(m: int, k: int, n: int, dtype: int, params: Optional[Params] = None) -> int:
@@ -436,7 +442,8 @@ def sketches(A, B, Cm, seed: int, rnd: int, n_buckets: int, ws: torch.Tensor, mo
 
 def measure_noise(A, B, Cm, seed: int, ws: torch.Tensor, m0: int = 0, params: Optional[Params] = None,
                   stream=None) -> Noise:
-    a = _mat_args(A, B, Cm)
+    """With params.b_transposed = 1, B is the weight W = B^T of shape (n, k) (C = A W^T)."""
+    a = _mat_args(A, B, Cm, bool(params is not None and params.b_transposed))
     out = Noise()
     rc = lib().fpsk_measure_noise(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, m0,
                                   C.byref(params) if params is not None else None, ws.data_ptr(), ws.numel(),
@@ -448,7 +455,8 @@ def measure_noise(A, B, Cm, seed: int, ws: torch.Tensor, m0: int = 0, params: Op
 
 def localize(A, B, Cm, seed: int, n_buckets: int, ws: torch.Tensor, params: Optional[Params] = None,
              capacity: int = 1024, stream=None) -> List[Fault]:
-    a = _mat_args(A, B, Cm)
+    """With params.b_transposed = 1, B is the weight W = B^T of shape (n, k) (C = A W^T)."""
+    a = _mat_args(A, B, Cm, bool(params is not None and params.b_transposed))
     buf = (Fault * capacity)()
     cnt = C.c_int32(0)
     rc = lib().fpsk_localize(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, n_buckets,

@@ -33,7 +33,7 @@ def test_exports_every_declared_symbol(lib):
 def test_struct_layouts_match_header():
     assert C.sizeof(fpsk.ProbeResult) == 32
     assert C.sizeof(fpsk.Fault) == 40 and fpsk.Fault.delta.offset == 8 and fpsk.Fault.bucket_b.offset == 36
-    assert C.sizeof(fpsk.Params) == 72 and fpsk.Params.rho_min.offset == 32
+    assert C.sizeof(fpsk.Params) == 80 and fpsk.Params.rho_min.offset == 40 and fpsk.Params.b_transposed.offset == 32
     assert C.sizeof(fpsk.Noise) == 56
 
 
@@ -89,6 +89,14 @@ def test_argument_validation_needs_no_device(lib):
     buf = (fpsk.Fault * 4)()
     assert g(one, 8, one, 8, one, 8, 8, 8, 8, 0, 1, 0, None, one, 1 << 20, None, buf, 4, C.byref(cnt)) == fpsk.ERR_BUCKETS
     assert g(one, 8, one, 8, one, 8, 8, 8, 8, 0, 1, 4, None, one, 16, None, buf, 4, C.byref(cnt)) == fpsk.ERR_WORKSPACE
+    # transposed weight (W = B^T, n x k): ldb is checked against k; only noise measurement and localization take it
+    wt = fpsk.default_params(b_transposed=1)
+    assert g(one, 8, one, 8, one, 16, 8, 8, 16, 0, 1, 4, C.byref(wt), one, 16, None, buf, 4, C.byref(cnt)) == fpsk.ERR_WORKSPACE
+    assert g(one, 8, one, 8, one, 16, 8, 8, 16, 0, 1, 4, None, one, 16, None, buf, 4, C.byref(cnt)) == fpsk.ERR_SHAPE
+    assert g(one, 16, one, 8, one, 8, 8, 16, 8, 0, 1, 4, C.byref(wt), one, 16, None, buf, 4, C.byref(cnt)) == fpsk.ERR_SHAPE
+    assert f(one, 8, one, 8, one, 8, 8, 8, 8, 0, 1, C.byref(wt), one, 1 << 20, None, one, None) == fpsk.ERR_PARAM
+    assert g(one, 8, one, 8, one, 8, 8, 8, 8, 0, 1, 4, C.byref(fpsk.default_params(b_transposed=2)), one, 1 << 20, None,
+             buf, 4, C.byref(cnt)) == fpsk.ERR_PARAM
     assert lib.fpsk_hash_tables(1, 0, 2, 10, 4, one, one, None) == fpsk.ERR_PARAM
     assert lib.fpsk_probe_workspace_bytes(0, 1, 1) == 0
     assert lib.fpsk_probe_workspace_bytes(4096, 4096, 4096) > 0
