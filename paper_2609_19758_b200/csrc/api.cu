@@ -183,14 +183,15 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
         rc = build_sketches(in, dtype, seed, 0, m_b, true, w.sk, st, w.S, w.R, w.T);
         if (rc != FPSK_OK) return rc;
         round0_built = true;
-        rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+        rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, in.C, in.ldc, m, n, w.samples, w.sel, w.misc + 3, st);
         if (rc != FPSK_OK) return rc;
         float h_scal[8], h_rms = 0.f;
         FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
-        rc = rms_c_launch(in.C, in.ldc, m, n, w.samples, w.sel, w.misc + 3, st);
-        if (rc != FPSK_OK) return rc;
         FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+        unsigned int h_sel_err = 0;
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_sel_err) return FPSK_ERR_TIMEOUT;
         double sig = h_scal[1], rms = h_rms;
         if (!(std::isfinite(sig) && sig > 0 && std::isfinite(rms) && rms > 0)) {
             sig = law_sigma((double)m, (double)k, (double)n, dtype, 1.0, (double)m_b);
@@ -225,11 +226,10 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
             rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, w.R, w.T, st);
             if (rc != FPSK_OK) return rc;
         }
-        if (!(t == 0 && round0_built)) {
-            rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
-            if (rc != FPSK_OK) return rc;
-        }
-        rc = select_candidates_launch(w.S, w.R, w.T, m_b, m, n, w.misc + 2, radius, K, w.sel, st);
+        // sigma_MAD of this round's S rides in the launches of the K-largest selection (round 0's is already
+        // there when it was needed for the radius)
+        const int mad_mode = (t == 0 && round0_built) ? -1 : (q.mad_of_abs ? 1 : 0);
+        rc = select_candidates_launch(w.S, w.R, w.T, m_b, m, n, w.misc + 2, radius, K, mad_mode, w.sel, st);
         if (rc != FPSK_OK) return rc;
         rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, st);
         if (rc != FPSK_OK) return rc;
@@ -238,8 +238,9 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
         FPSK_CUDA_OK(cudaMemcpyAsync(&h_nhits, w.n_hits, 4, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * kHitCap, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
-        unsigned int h_tc_err = 0;
+        unsigned int h_tc_err = 0, h_sel_err = 0;
         if (w.sk.tc) FPSK_CUDA_OK(cudaMemcpyAsync(&h_tc_err, w.sk.tc_err, 4, cudaMemcpyDeviceToHost, st));
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaEventRecord(round_done.e, st));
         if (t + 1 < q.rounds) {
             rc = build_sketches(in, dtype, seed, t + 1, m_b, true, w.sk, st, w.S, w.R, w.T);
@@ -247,7 +248,7 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
             built_ahead = true;
         }
         FPSK_CUDA_OK(cudaEventSynchronize(round_done.e));
-        if (h_tc_err) return FPSK_ERR_TIMEOUT;        // a bounded wait of the tensor-core contraction gave up
+        if (h_tc_err || h_sel_err) return FPSK_ERR_TIMEOUT;        // a bounded wait (contraction, selects) gave up
         if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
         const int nU = std::min(h_counts[2], K);
 
@@ -587,15 +588,16 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     const long long mm = (long long)m0 * m0;
     rc = sigma_clip_launch(w.S, mm, w.sel, st);
     if (rc != FPSK_OK) return rc;
-    rc = sigma_mad_launch(w.S, mm, q.mad_of_abs, w.sel, st);
+    rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
     if (rc != FPSK_OK) return rc;
     float h_scal[8];
     FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
-    rc = rms_c_launch(C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
-    if (rc != FPSK_OK) return rc;
     float h_rms = 0.f;
     FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+    unsigned int h_sel_err = 0;
+    FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
     FPSK_CUDA_OK(cudaStreamSynchronize(st));
+    if (h_sel_err) return FPSK_ERR_TIMEOUT;
 
     fpsk_noise out;
     memset(&out, 0, sizeof(out));
@@ -788,14 +790,15 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
         SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
         rc = build_sketches(in, dtype, seed, 0, m0, false, w0.sk, st, w0.S, nullptr, nullptr);
         if (rc != FPSK_OK) return rc;
-        rc = sigma_mad_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, w0.sel, st);
+        rc = sigma_mad_rms_c_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);
         if (rc != FPSK_OK) return rc;
         float h_scal[8], h_rms = 0.f;
         FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w0.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
-        rc = rms_c_launch(C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);
-        if (rc != FPSK_OK) return rc;
         FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w0.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+        unsigned int h_sel_err = 0;
+        FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w0.sel.err, 4, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        if (h_sel_err) return FPSK_ERR_TIMEOUT;
         int r;
         double B_;
         plan_of(m, k, n, dtype, h_scal[1], h_rms, m0, q, m_loc, r, B_);

@@ -531,7 +531,6 @@ constexpr int kSegMax = 4096;                 // bytes of one row segment: 256 x
 constexpr int kGatherFloats = 5120;           // staging of partial vectors in the final combine; lane-reduce scratch
 constexpr int kUChunkT = 1024;                // u values kept in shared memory
 constexpr int kTmaSmem = kStages * kStageBytes + (kGatherFloats + kUChunkT) * 4 + 256;
-constexpr int kMaxGridC = 256;                // grids up to this size combine their statistics in one batch of loads
 
 struct TDecomp {
     int cg;       // column groups

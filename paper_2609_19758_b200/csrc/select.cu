@@ -3,6 +3,7 @@
 // ratios of Eq. (recover)).  Medians and the K-th largest key come from an exact radix select
 // (integer histograms only), so every decision is deterministic.
 #include "sketch.cuh"
+#include "stream_pipe.cuh"
 
 #include <math.h>
 
@@ -13,14 +14,22 @@ enum SelMode {
     SEL_SIGNED = 1,     // key = order-preserving bits of S        (median of S)
     SEL_DEV_ABS = 2,    // key = bits(||S| - med|)
     SEL_DEV_SIGNED = 3, // key = bits(|S - med|)
-    SEL_TOPK = 4,       // valid iff |S| > thr; key = bits(|S|) << 32 | ~idx   (all keys distinct)
+    SEL_TOPK = 4,       // key = bits(|S|) << 32 | ~idx (all keys distinct; a NaN sorts below everything)
     SEL_SAMPLE = 5      // valid iff S >= 0 (sentinel -1 marks dropped samples); key = bits(S)
 };
 
-// state words
+// state words (per job slot)
 enum { ST_PREFIX = 0, ST_K = 1, ST_SKIP = 2, ST_WORDS = 4 };
 // scal slots
-enum { SC_MED = 0, SC_MAD = 1, SC_MEAN = 2, SC_CLIP = 3, SC_THR = 4, SC_TAUC = 5, SC_TAUD = 6, SC_WORDS = 16 };
+enum { SC_MED = 0, SC_MAD = 1, SC_MEAN = 2, SC_CLIP = 3, SC_THR = 4, SC_TAUC = 5, SC_TAUD = 6, SC_SMED = 7, SC_WORDS = 16 };
+// Histogram words.  Every CTA adds its 256 counts to one of kHistCopies copies (CTA index modulo the copies),
+// each copy in cache lines of its own, so that the CTAs' atomics do not all queue on the same eight lines.
+// Digit d, job slot s, copy r: hist[kHistBase + ((d * 2 + s) * kHistCopies + r) * 256 ...].
+enum { kHistCopies = 8, kHistBase = 64, kHistWords = 8 /*digits*/ * 2 * kHistCopies * 256,
+       kHistErr = kHistBase + kHistWords, kSumTicket = kHistErr + 1, kHistBytes = (kHistBase + kHistWords + 64) * 4 };
+// hist[0]: arrival counter of the running select launch (zeroed with the histograms before every launch);
+// hist[kHistErr]: set when a bounded wait gave up (zeroed once per call of the library, read by the host);
+// hist[kSumTicket]: ticket of the clipped-mean sums.
 
 __device__ __forceinline__ uint32_t ordered_bits(float x)
 {
@@ -33,29 +42,35 @@ __device__ __forceinline__ float from_ordered_bits(uint32_t k)
     return __uint_as_float(b);
 }
 
-__device__ __forceinline__ bool make_key(int mode, const float *S, long long idx, const float *scal,
-                                         unsigned long long &key)
+// key of the K-largest selection: descending |S|, ties by ascending flat index
+__device__ __forceinline__ unsigned long long topk_key(float a, long long idx)
 {
-    const float x = S[idx];
+    const uint32_t hi = (a == a) ? __float_as_uint(a) : 0u;
+    return ((unsigned long long)hi << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
+}
+
+// key of element idx with value x (med: the median that the deviation keys are taken from)
+__device__ __forceinline__ bool key_of(int mode, float x, long long idx, float med, unsigned long long &key)
+{
     switch (mode) {
     case SEL_ABS: key = __float_as_uint(fabsf(x)); return true;
     case SEL_SIGNED: key = ordered_bits(x); return true;
-    case SEL_DEV_ABS: key = __float_as_uint(fabsf(fabsf(x) - scal[SC_MED])); return true;
-    case SEL_DEV_SIGNED: key = __float_as_uint(fabsf(x - scal[SC_MED])); return true;
-    case SEL_TOPK: {
-        const float a = fabsf(x);
-        if (!(a > scal[SC_THR])) return false;
-        key = ((unsigned long long)__float_as_uint(a) << 32) | (unsigned long long)(0xFFFFFFFFu - (uint32_t)idx);
-        return true;
-    }
+    case SEL_DEV_ABS: key = __float_as_uint(fabsf(fabsf(x) - med)); return true;
+    case SEL_DEV_SIGNED: key = __float_as_uint(fabsf(x - med)); return true;
+    case SEL_TOPK: key = topk_key(fabsf(x), idx); return true;
     default:
         if (!(x >= 0.f)) return false;
         key = __float_as_uint(x);
         return true;
     }
 }
+__device__ __forceinline__ bool make_key(int mode, const float *S, long long idx, const float *scal,
+                                         unsigned long long &key)
+{
+    return key_of(mode, S[idx], idx, scal[SC_MED], key);
+}
 
-// counts[0] = number of valid keys (SEL_TOPK, SEL_SAMPLE)
+// counts[0] = number of valid keys (SEL_SAMPLE)
 __global__ void count_valid_kernel(int mode, const float *S, long long mm, const float *scal, int *counts)
 {
     int c = 0;
@@ -67,22 +82,33 @@ __global__ void count_valid_kernel(int mode, const float *S, long long mm, const
     if ((threadIdx.x & 31) == 0 && c) atomicAdd(counts, c);
 }
 
-// rank to select: median of N keys, or (count - K) for the K largest, from device counts
-__device__ __forceinline__ void select_initial(int mode, long long n_all, int K, const int *counts, bool &skip,
-                                               unsigned long long &k)
+constexpr int kSelThreads = 1024; // one CTA per SM
+constexpr int kSelItems = 8;      // elements per thread and batch (their keys stay in shared memory over the digits when one
+                                  // batch covers the source)
+
+// One radix select in flight: its source, key kind, digit position.  Up to two run in one launch (slot 0, 1).
+struct SelJob {
+    const float *src;
+    long long n;
+    int mode, nbits, shift, K;
+};
+
+// rank to select: median of N keys, or (N - K) for the K largest
+__device__ __forceinline__ void select_initial(const SelJob &j, const int *counts, bool &skip, unsigned long long &k)
 {
     skip = false;
     k = 0;
-    if (mode == SEL_TOPK) {
-        const int cnt = counts[0];
-        if (cnt <= K) skip = true;             // take everything above the threshold
-        else k = (unsigned long long)(cnt - K);
-    } else if (mode == SEL_SAMPLE) {
+    if (j.mode == SEL_TOPK) {
+        // The K largest of all keys.  The buckets above the detection threshold are a top segment of this
+        // order, so "the K largest above the threshold" is this selection cut at the threshold afterwards.
+        if (j.n <= (long long)j.K) skip = true;
+        else k = (unsigned long long)(j.n - j.K);
+    } else if (j.mode == SEL_SAMPLE) {
         const int cnt = counts[0];
         if (cnt <= 0) skip = true;
         else k = (unsigned long long)((cnt - 1) / 2);
     } else {
-        k = (unsigned long long)((n_all - 1) / 2);
+        k = (unsigned long long)((j.n - 1) / 2);
     }
 }
 
@@ -92,119 +118,322 @@ __device__ __forceinline__ void select_result(int mode, unsigned long long key, 
     if (mode == SEL_ABS) scal[SC_MED] = __uint_as_float((uint32_t)key);
     else if (mode == SEL_SIGNED) scal[SC_MED] = from_ordered_bits((uint32_t)key);
     else if (mode == SEL_DEV_ABS || mode == SEL_DEV_SIGNED) scal[SC_MAD] = 1.4826f * __uint_as_float((uint32_t)key);
-    else if (mode == SEL_SAMPLE) scal[SC_MED] = skip ? __uint_as_float(0x7FC00000u) : __uint_as_float((uint32_t)key);
+    else if (mode == SEL_SAMPLE) scal[SC_SMED] = skip ? __uint_as_float(0x7FC00000u) : __uint_as_float((uint32_t)key);
 }
 
-// One 8-bit digit of the radix select.  The last CTA to finish picks the digit.  The first pass of a
-// select derives the rank from the device counts itself and the last one writes the result, so a select
-// is nothing but its passes.  The histogram is left at zero by every pass (and zeroed once per call of
-// the library before the first select).
-__global__ void __launch_bounds__(256) radix_pass_kernel(int mode, int nbits, int shift, const float *S, long long mm,
-                                                         float *scal, unsigned long long *state, unsigned int *hist,
-                                                         long long n_all, int K, const int *counts)
+// The digits of up to three radix selects in ONE cooperative launch: `a` in slot 0 and, beside it digit by
+// digit, `b` and then `c` in slot 1 (independent sources, keys and ranks; one pass over memory when they
+// share the source; c may take its deviations from b's result, which every CTA derives for itself).  A
+// digit is: every CTA bins its keys in shared memory and adds the 256 counts to one of the copies of this
+// digit's histogram; a grid-wide arrival counter (bounded wait); every CTA sums the copies and finds the
+// bin of the k-th key by the same scan.  One CTA of 1024 threads per SM.  Measured at 10^6 keys: 8 us per
+// digit (binning 2-5, arrival wait 2, copies + scan 1.5-2), against 9.5 us for a launch per digit with a
+// last-CTA scan and the select state in global memory; the K-largest key needs only its upper four digits
+// when the K-th value is unique, and the median of the samples of C and the two medians of the MAD ride in
+// the same launches, so a localization round runs 8 digits in one launch instead of 16 launches.
+struct SelChain {
+    SelJob a, b, c;
+    int have_b, have_c;
+};
+constexpr int kChainSteps = 8;                 // digits of the longest key (64 bits)
+
+// inclusive scan of the 256 counts (one per thread) -> the bin whose running count passes k, and the
+// number of keys below it; the same values in every thread
+__device__ __forceinline__ void pick_digit(unsigned int h, unsigned long long k, unsigned long long *wsum, int *s_bin,
+                                           unsigned long long *s_before, int &bin, unsigned long long &before_out)
 {
-    __shared__ unsigned int sh[256];
-    __shared__ int last;
-    const bool first = shift == nbits - 8, final_ = shift == 0;
-    bool skip;
-    unsigned long long k_first = 0;
-    if (first) select_initial(mode, n_all, K, counts, skip, k_first);
-    else skip = state[ST_SKIP] != 0;
-    if (skip) {
-        if (first && blockIdx.x == 0 && threadIdx.x == 0) {
-            state[ST_SKIP] = 1;
-            state[ST_PREFIX] = 0;
-            select_result(mode, 0, true, scal);
-        }
-        return;
-    }
-    sh[threadIdx.x] = 0;
-    __syncthreads();
-    const unsigned long long prefix = first ? 0ull : state[ST_PREFIX];
-    const int hs = shift + 8;
-    // Keys of a noise sketch crowd into a few bins of the leading digits: lanes with the same bin are
-    // combined first (match_any), so a warp issues one shared-memory atomic per distinct bin.
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long i0 = (long long)blockIdx.x * blockDim.x; i0 < mm; i0 += stride) {
-        const long long i = i0 + threadIdx.x;
-        unsigned long long k = 0;
-        bool valid = i < mm && make_key(mode, S, i, scal, k);
-        if (valid && hs < nbits && (k >> hs) != (prefix >> hs)) valid = false;
-        const unsigned int bin = valid ? ((unsigned)(k >> shift) & 255u) : 256u;
-        const unsigned int peers = __match_any_sync(0xFFFFFFFFu, bin);
-        if (valid && (threadIdx.x & 31) == (unsigned)(__ffs(peers) - 1)) atomicAdd(&sh[bin], (unsigned)__popc(peers));
-    }
-    __syncthreads();
-    if (sh[threadIdx.x]) atomicAdd(&hist[threadIdx.x], sh[threadIdx.x]);
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last = (atomicAdd(&hist[256], 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    // the bin holding the k-th key: inclusive scan of the 256 counts (one per thread), then the first
-    // thread whose running count passes k
-    {
-        __shared__ unsigned long long wsum[8];
-        __shared__ int s_bin;
-        __shared__ unsigned long long s_before;
-        const unsigned long long k = first ? k_first : state[ST_K];
-        const unsigned int h = __ldcg(&hist[threadIdx.x]);
-        unsigned long long inc = h;
-        const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    unsigned long long inc = h;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-            if (lane >= o) inc += v;
-        }
-        if (lane == 31) wsum[wid] = inc;
-        if (threadIdx.x == 0) { s_bin = 255; s_before = 0; }
-        __syncthreads();
-        unsigned long long base = 0;
-        for (int w = 0; w < wid; ++w) base += wsum[w];
-        inc += base;                                   // keys in bins 0 .. threadIdx.x
-        const unsigned long long before = inc - h;     // keys in bins below this one
-        unsigned long long total = 0;
-        for (int w = 0; w < 8; ++w) total += wsum[w];
-        __syncthreads();
-        if (before <= k && k < inc) { s_bin = threadIdx.x; s_before = before; }        // exactly one thread, when k < total
-        if (threadIdx.x == 255 && k >= total) { s_bin = 255; s_before = total; }       // k beyond the keys (not reached: k is clamped to the count)
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            const unsigned long long key = prefix | ((unsigned long long)s_bin << shift);
-            state[ST_K] = k - s_before;
-            state[ST_PREFIX] = key;
-            if (first) state[ST_SKIP] = 0;
-            if (final_) select_result(mode, key, false, scal);
-            hist[256] = 0;
-        }
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
+        if (lane >= o) inc += v;
     }
+    __syncthreads();                               // earlier readers of wsum, s_bin are done
+    if (lane == 31 && wid < 8) wsum[wid] = inc;    // threads beyond the 256 bins come along with h = 0
+    if (threadIdx.x == 0) { *s_bin = 255; *s_before = 0; }
     __syncthreads();
-    hist[threadIdx.x] = 0;
+    unsigned long long base = 0;
+    for (int w = 0; w < wid && w < 8; ++w) base += wsum[w];
+    inc += base;                                   // keys in bins 0 .. threadIdx.x
+    const unsigned long long before = inc - h;     // keys in bins below this one
+    unsigned long long total = 0;
+    for (int w = 0; w < 8; ++w) total += wsum[w];
+    __syncthreads();
+    if (before <= k && k < inc) { *s_bin = threadIdx.x; *s_before = before; }        // exactly one thread, when k < total
+    if (threadIdx.x == 255 && k >= total) { *s_bin = 255; *s_before = total; }       // k beyond the keys (not reached: k is clamped to the count)
+    __syncthreads();
+    bin = *s_bin;
+    before_out = *s_before;
 }
 
-// after the passes: turn the selected key into a value
-
-static fpsk_status run_select(int mode, int nbits, const float *S, long long mm, int K, SelectWs &w, cudaStream_t st)
+__device__ __forceinline__ float median_value(int mode, unsigned long long key)
 {
+    return mode == SEL_SIGNED ? from_ordered_bits((uint32_t)key) : __uint_as_float((uint32_t)key);
+}
+
+// 32-bit part of a key that does not change over the digits (for the K-largest key: its upper half)
+__device__ __forceinline__ uint32_t key_base(int mode, float x, float med)
+{
+    switch (mode) {
+    case SEL_ABS: return __float_as_uint(fabsf(x));
+    case SEL_SIGNED: return ordered_bits(x);
+    case SEL_DEV_ABS: return __float_as_uint(fabsf(fabsf(x) - med));
+    case SEL_DEV_SIGNED: return __float_as_uint(fabsf(x - med));
+    case SEL_TOPK: { const float a = fabsf(x); return (a == a) ? __float_as_uint(a) : 0u; }
+    default: return (x >= 0.f) ? __float_as_uint(x) : 0xFFFFFFFFu;      // dropped sample: no key
+    }
+}
+
+__global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain ch, float *scal, unsigned long long *state,
+                                                              unsigned int *hist, const int *counts)
+{
+    __shared__ unsigned int sh[2][256];
+    __shared__ unsigned long long wsum[8];
+    __shared__ int s_bin, s_ok;
+    __shared__ unsigned long long s_before;
+    const int G = (int)gridDim.x, tid = (int)threadIdx.x;
+    SelJob job[2] = {ch.a, ch.b};
+    bool on[2] = {true, ch.have_b != 0};
+    bool have_c = ch.have_c != 0;
+    unsigned long long k[2] = {0, 0}, prefix[2] = {0, 0};
+    float med = scal[SC_MED];
+    const bool lead = blockIdx.x == 0 && tid == 0;
+    // a slot-1 job that has nothing to select makes room for its successor at once
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        for (int tries = 0; tries < 2 && on[j]; ++tries) {
+            bool skip;
+            select_initial(job[j], counts, skip, k[j]);
+            job[j].shift = job[j].nbits - 8;
+            if (!skip) break;
+            if (lead) {
+                state[j * ST_WORDS + ST_SKIP] = 1;
+                state[j * ST_WORDS + ST_PREFIX] = 0;
+                select_result(job[j].mode, 0, true, scal);
+            }
+            if (j == 1 && have_c) { job[1] = ch.c; have_c = false; }
+            else on[j] = false;
+        }
+    }
+    const int steps1 = (ch.have_b ? ch.b.nbits / 8 : 0) + (ch.have_c ? ch.c.nbits / 8 : 0);
+    const int nsteps = ch.a.nbits / 8 > steps1 ? ch.a.nbits / 8 : steps1;
+    const long long per_grid = (long long)G * (kSelThreads * kSelItems);
+    long long nall = ch.a.n;
+    if (ch.have_b && ch.b.n > nall) nall = ch.b.n;
+    if (ch.have_c && ch.c.n > nall) nall = ch.c.n;
+    // When one batch covers the sources a thread derives the keys of its elements once per select and keeps
+    // them (in shared memory) over the digits; otherwise it derives them again digit by digit.
+    const bool one_batch = nall <= per_grid;
+    extern __shared__ uint32_t kb_all[];           // [job][item][thread]
+    uint32_t (*kb)[kSelItems][kSelThreads] = reinterpret_cast<uint32_t (*)[kSelItems][kSelThreads]>(kb_all);
+    bool fresh[2] = {true, true};
+    for (int step = 0; step < nsteps; ++step) {
+        if (tid < 256) {
+            sh[0][tid] = 0;
+            sh[1][tid] = 0;
+        }
+        __syncthreads();
+        long long nmax = 0;
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            if (on[j] && job[j].n > nmax) nmax = job[j].n;
+        // Leading digits put nearly all keys into one or two bins: a lane that counts for a group keeps its last
+        // two bins in registers and adds them to shared memory when they change or the digit ends.
+        unsigned int cbin[2][2] = {{256u, 256u}, {256u, 256u}}, ccnt[2][2] = {{0u, 0u}, {0u, 0u}};
+        // All of a thread's loads are issued before it bins anything (the warp-wide votes keep the compiler
+        // from moving loads across them).
+        for (long long base = (long long)blockIdx.x * (kSelThreads * kSelItems); base < nmax; base += per_grid) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (!on[j] || !(fresh[j] || !one_batch)) continue;
+#pragma unroll 1
+                for (int u0 = 0; u0 < kSelItems; u0 += 8) {
+                    float x[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const long long i = base + (u0 + u) * kSelThreads + tid;
+                        x[u] = i < job[j].n ? __ldg(job[j].src + i) : 0.f;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) kb[j][u0 + u][tid] = key_base(job[j].mode, x[u], med);
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                if (!on[j]) continue;
+                const int shift = job[j].shift;
+                const bool wide = job[j].nbits == 64;              // K-largest key: kb is the upper half, ~index the lower
+                const bool low_half = wide && shift < 32;
+                const bool sample = job[j].mode == SEL_SAMPLE;
+                const uint32_t pre_hi = wide ? (uint32_t)(prefix[j] >> 32) : (uint32_t)prefix[j];
+                const uint32_t pre_lo = (uint32_t)prefix[j];
+                const int sh32 = low_half ? shift : (wide ? shift - 32 : shift);
+                // bits of the 32-bit word in play that are already fixed by earlier digits
+                const uint32_t fixed = sh32 + 8 >= 32 ? 0u : (0xFFFFFFFFu << (sh32 + 8));
+#pragma unroll 2
+                for (int u = 0; u < kSelItems; ++u) {
+                    const long long i = base + u * kSelThreads + tid;
+                    const uint32_t kbu = kb[j][u][tid];
+                    bool valid = i < job[j].n && !(sample && kbu == 0xFFFFFFFFu);
+                    uint32_t word;
+                    if (low_half) {
+                        valid = valid && kbu == pre_hi;
+                        word = 0xFFFFFFFFu - (uint32_t)i;
+                        valid = valid && ((word ^ pre_lo) & fixed) == 0u;
+                    } else {
+                        word = kbu;
+                        valid = valid && ((word ^ pre_hi) & fixed) == 0u;
+                    }
+                    const unsigned int vmask = __ballot_sync(0xFFFFFFFFu, valid);
+                    if (vmask == 0u) continue;                             // late digits: hardly any key still carries the prefix
+                    const unsigned int bin = (word >> sh32) & 255u;
+                    const unsigned int peers = __match_any_sync(0xFFFFFFFFu, valid ? bin : 256u);
+                    // the lowest lane of a group counts for the group; it keeps its last two bins in registers
+                    if (valid && (tid & 31) == __ffs(peers) - 1) {
+                        const unsigned int cnt = (unsigned)__popc(peers);
+                        if (bin == cbin[j][0]) ccnt[j][0] += cnt;
+                        else if (bin == cbin[j][1]) ccnt[j][1] += cnt;
+                        else {
+                            if (ccnt[j][1]) atomicAdd(&sh[j][cbin[j][1]], ccnt[j][1]);
+                            cbin[j][1] = cbin[j][0]; ccnt[j][1] = ccnt[j][0];
+                            cbin[j][0] = bin; ccnt[j][0] = cnt;
+                        }
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+#pragma unroll
+            for (int e = 0; e < 2; ++e)
+                if (ccnt[j][e]) atomicAdd(&sh[j][cbin[j][e]], ccnt[j][e]);
+        }
+        fresh[0] = false;
+        fresh[1] = false;
+        __syncthreads();
+        unsigned int *hstep = hist + kHistBase + (size_t)step * (2 * kHistCopies * 256);
+#pragma unroll
+        for (int j = 0; j < 2; ++j)
+            if (on[j] && tid < 256 && sh[j][tid]) atomicAdd(&hstep[(j * kHistCopies + (blockIdx.x % kHistCopies)) * 256 + tid], sh[j][tid]);
+        // ---- all CTAs' counts are in: arrival counter, bounded wait
+        __syncthreads();
+        if (tid == 0) {
+            __threadfence();
+            red_release_add(hist);
+            s_ok = bounded_wait_ge(hist, (unsigned)(step + 1) * (unsigned)G) ? 1 : 0;
+            if (!s_ok) atomicOr(hist + kHistErr, 1u);
+        }
+        __syncthreads();
+        if (!s_ok) return;
+        unsigned int hsum[2] = {0, 0};
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (!on[j]) continue;
+#pragma unroll
+            for (int r = 0; r < kHistCopies; ++r)
+                if (tid < 256) hsum[j] += __ldcg(&hstep[(j * kHistCopies + r) * 256 + tid]);
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (!on[j]) continue;
+            int bin;
+            unsigned long long before;
+            pick_digit(hsum[j], k[j], wsum, &s_bin, &s_before, bin, before);
+            k[j] -= before;
+            prefix[j] |= (unsigned long long)bin << job[j].shift;
+            job[j].shift -= 8;
+            // K-largest key: once the rank inside the remaining ties is 0, the lower digits cannot move the
+            // cut (every key of the tie is at or above "upper half, zeros"), so they are left at zero
+            if (job[j].nbits == 64 && job[j].shift < 32 && k[j] == 0) job[j].shift = -8;
+            if (job[j].shift >= 0) continue;
+            // the select in slot j is complete
+            if (lead) {
+                state[j * ST_WORDS + ST_SKIP] = 0;
+                state[j * ST_WORDS + ST_PREFIX] = prefix[j];
+                select_result(job[j].mode, prefix[j], false, scal);
+            }
+            if (job[j].mode == SEL_ABS || job[j].mode == SEL_SIGNED) med = median_value(job[j].mode, prefix[j]);
+            if (j == 1 && have_c) {
+                job[1] = ch.c;
+                have_c = false;
+                fresh[1] = true;
+                bool skip;
+                select_initial(job[1], counts, skip, k[1]);
+                job[1].shift = job[1].nbits - 8;
+                prefix[1] = 0;
+                if (skip) {
+                    if (lead) {
+                        state[ST_WORDS + ST_SKIP] = 1;
+                        state[ST_WORDS + ST_PREFIX] = 0;
+                        select_result(job[1].mode, 0, true, scal);
+                    }
+                    on[1] = false;
+                }
+            } else {
+                on[j] = false;
+            }
+        }
+        if (!on[0] && !on[1]) break;       // same decision in every CTA: nobody waits for a further digit
+    }
+}
+
+constexpr size_t kSelSmem = (size_t)2 * kSelItems * kSelThreads * 4;
+
+static int select_capacity()
+{
+    static int cap = 0;            // co-resident CTAs of the cooperative select kernel on this device
+    if (cap == 0) {
+        int dev = 0, sms = 0, occ = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
+        if (cudaFuncSetAttribute(select_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelSmem) != cudaSuccess) return sms;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, select_chain_kernel, kSelThreads, kSelSmem) != cudaSuccess || occ < 1) return sms;
+        cap = sms;
+    }
+    return cap;
+}
+
+static int select_grid(long long n)
+{
+    const long long want = (n + kSelThreads * kSelItems - 1) / (kSelThreads * kSelItems);
+    const int cap = select_capacity();
+    return (int)(want < 1 ? 1 : (want > cap ? cap : want));
+}
+
+// Runs select `a` in slot 0 and, beside it, `b` and then `c` in slot 1.  One memset (this launch's histograms
+// and arrival counter) and one cooperative launch.
+static fpsk_status run_selects(SelJob a, SelJob b, bool have_b, SelJob c, bool have_c, SelectWs &w, cudaStream_t st)
+{
+    const int da = a.nbits / 8, db = have_b ? b.nbits / 8 : 0, dc = have_c ? c.nbits / 8 : 0;
+    const int steps = da > db + dc ? da : db + dc;
+    if (steps > kChainSteps || (have_c && !have_b)) return FPSK_ERR_PARAM;
     if (!w.hist_clean) {
-        FPSK_CUDA_OK(cudaMemsetAsync(w.hist, 0, 257 * sizeof(unsigned int), st));
+        FPSK_CUDA_OK(cudaMemsetAsync(w.hist + kHistErr, 0, 64 * sizeof(unsigned int), st));      // sticky error word, sum ticket
         w.hist_clean = true;
     }
-    long long want = (mm + 256 * 16 - 1) / (256 * 16);
-    const int grid = (int)(want < 1 ? 1 : (want > 1184 ? 1184 : want));
-    for (int shift = nbits - 8; shift >= 0; shift -= 8) {
-        radix_pass_kernel<<<grid, 256, 0, st>>>(mode, nbits, shift, S, mm, w.scal, w.state, w.hist, mm, K, w.counts);
-        FPSK_LAUNCH_CHECK();
-    }
+    FPSK_CUDA_OK(cudaMemsetAsync(w.hist, 0, (size_t)(kHistBase + steps * 2 * kHistCopies * 256) * sizeof(unsigned int), st));
+    SelChain ch;
+    ch.a = a; ch.b = b; ch.c = c; ch.have_b = have_b ? 1 : 0; ch.have_c = have_c ? 1 : 0;
+    long long nmax = a.n;
+    if (have_b && b.n > nmax) nmax = b.n;
+    if (have_c && c.n > nmax) nmax = c.n;
+    const int grid = select_grid(nmax);
+    float *scal = w.scal;
+    unsigned long long *state = w.state;
+    unsigned int *hist = w.hist;
+    const int *counts = w.counts;
+    void *args[] = {(void *)&ch, (void *)&scal, (void *)&state, (void *)&hist, (void *)&counts};
+    FPSK_CUDA_OK(cudaLaunchCooperativeKernel((const void *)select_chain_kernel, dim3(grid), dim3(kSelThreads), args, kSelSmem, st));
+    count_launch();
     return FPSK_OK;
 }
 
-fpsk_status sigma_mad_launch(const float *S, long long mm, int mad_of_abs, SelectWs &w, cudaStream_t st)
+static SelJob sel_job(int mode, int nbits, const float *src, long long n, int K)
 {
-    fpsk_status rc = run_select(mad_of_abs ? SEL_ABS : SEL_SIGNED, 32, S, mm, 0, w, st);
-    if (rc != FPSK_OK) return rc;
-    return run_select(mad_of_abs ? SEL_DEV_ABS : SEL_DEV_SIGNED, 32, S, mm, 0, w, st);
+    SelJob j;
+    j.src = src; j.n = n; j.mode = mode; j.nbits = nbits; j.shift = nbits - 8; j.K = K;
+    return j;
 }
 
 // ---------------------------------------------------------------- clipped mean
@@ -246,9 +475,9 @@ __global__ void __launch_bounds__(256) abs_sum_kernel(int mode, const float *S, 
 
 fpsk_status sigma_clip_launch(const float *S, long long mm, SelectWs &w, cudaStream_t st)
 {
-    FPSK_CUDA_OK(cudaMemsetAsync(w.hist + 257, 0, 4, st));
+    FPSK_CUDA_OK(cudaMemsetAsync(w.hist + kSumTicket, 0, 4, st));
     for (int mode = 0; mode < 2; ++mode) {
-        abs_sum_kernel<<<kSumGrid, 256, 0, st>>>(mode, S, mm, w.scal, w.partial, w.hist + 257);
+        abs_sum_kernel<<<kSumGrid, 256, 0, st>>>(mode, S, mm, w.scal, w.partial, w.hist + kSumTicket);
         FPSK_LAUNCH_CHECK();
     }
     return FPSK_OK;
@@ -271,10 +500,13 @@ __global__ void thresholds_kernel(const float *taup, float nmax, float rad, floa
 __global__ void collect_kernel(const float *S, long long mm, const float *scal, const unsigned long long *state,
                                int cap, unsigned long long *keys, int *counts)
 {
+    // the K largest keys (slot 0 of the select state), cut at the detection threshold
     const unsigned long long kth = state[ST_SKIP] ? 0ull : state[ST_PREFIX];
+    const float thr = scal[SC_THR];
     for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < mm; i += (long long)gridDim.x * blockDim.x) {
-        unsigned long long k;
-        if (!make_key(SEL_TOPK, S, i, scal, k)) continue;
+        const float a = fabsf(S[i]);
+        if (!(a > thr)) continue;
+        const unsigned long long k = topk_key(a, i);
         if (k < kth) continue;
         const int slot = atomicAdd(counts + 1, 1);
         if (slot < cap) keys[slot] = k;
@@ -335,19 +567,22 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
 }
 
 fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
-                                     long long n3, const float *d_tau, int radius, int K, SelectWs &w, cudaStream_t st)
+                                     long long n3, const float *d_tau, int radius, int K, int mad_mode, SelectWs &w,
+                                     cudaStream_t st)
 {
     if (K > kSelMaxK) K = kSelMaxK;
     const long long mm = (long long)m_b * m_b;
+    // The K-th largest key does not depend on the thresholds, so its eight digits run beside the four of
+    // the median and the four of the MAD (mad_mode 1: of |S|, 0: signed; < 0: sigma_MAD is already in place).
+    const SelJob top = sel_job(SEL_TOPK, 64, S, mm, K);
+    const SelJob med = sel_job(mad_mode ? SEL_ABS : SEL_SIGNED, 32, S, mm, 0);
+    const SelJob dev = sel_job(mad_mode ? SEL_DEV_ABS : SEL_DEV_SIGNED, 32, S, mm, 0);
+    fpsk_status rc = run_selects(top, med, mad_mode >= 0, dev, mad_mode >= 0, w, st);
+    if (rc != FPSK_OK) return rc;
     thresholds_kernel<<<1, 32, 0, st>>>(d_tau, (float)(n1 > n3 ? n1 : n3), (float)radius, w.scal, w.counts);
     FPSK_LAUNCH_CHECK();
-    long long want = (mm + 256 * 16 - 1) / (256 * 16);
-    const int grid = (int)(want < 1 ? 1 : (want > 1184 ? 1184 : want));
-    count_valid_kernel<<<grid, 256, 0, st>>>(SEL_TOPK, S, mm, w.scal, w.counts);
-    FPSK_LAUNCH_CHECK();
-    fpsk_status rc = run_select(SEL_TOPK, 64, S, mm, K, w, st);
-    if (rc != FPSK_OK) return rc;
-    collect_kernel<<<grid, 256, 0, st>>>(S, mm, w.scal, w.state, kSelMaxK, w.keys, w.counts);
+    const long long cwant = (mm + 4095) / 4096;
+    collect_kernel<<<(int)(cwant < 1 ? 1 : (cwant > 1184 ? 1184 : cwant)), 256, 0, st>>>(S, mm, w.scal, w.state, kSelMaxK, w.keys, w.counts);
     FPSK_LAUNCH_CHECK();
     int p1 = 0, p3 = 0;
     while ((1LL << p1) < n1) ++p1;
@@ -429,7 +664,7 @@ __global__ void __launch_bounds__(1024) clipped_rms_kernel(const float *samples,
                                                            const int *counts, float *out)
 {
     __shared__ double sh[1024];
-    const float clip = 64.f * scal[SC_MED];
+    const float clip = 64.f * scal[SC_SMED];
     double acc = 0.0;
     for (long long i = threadIdx.x; i < nsamp; i += 1024) {
         const float a = samples[i];
@@ -450,19 +685,33 @@ __global__ void __launch_bounds__(1024) clipped_rms_kernel(const float *samples,
     }
 }
 
-fpsk_status rms_c_launch(const float *C, long long ldc, long long n1, long long n3, float *samples,
-                         SelectWs &w, float *out, cudaStream_t st)
+static long long rms_c_samples(const float *C, long long ldc, long long n1, long long n3, float *samples, SelectWs &w,
+                               cudaStream_t st)
 {
     const long long total = n1 * n3;
     long long stride = total / 65536;
     if (stride < 1) stride = 1;
     const long long nsamp = (total + stride - 1) / stride;
     sample_c_kernel<<<(unsigned)((nsamp + 255) / 256), 256, 0, st>>>(C, ldc, n3, total, stride, nsamp, samples);
-    FPSK_LAUNCH_CHECK();
-    FPSK_CUDA_OK(cudaMemsetAsync(w.counts, 0, 4 * 4, st));
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    if (cudaMemsetAsync(w.counts, 0, 4 * 4, st) != cudaSuccess) return -1;
     count_valid_kernel<<<64, 256, 0, st>>>(SEL_SAMPLE, samples, nsamp, w.scal, w.counts);
-    FPSK_LAUNCH_CHECK();
-    fpsk_status rc = run_select(SEL_SAMPLE, 32, samples, nsamp, 0, w, st);
+    if (cudaGetLastError() != cudaSuccess) return -1;
+    return nsamp;
+}
+
+// sigma_MAD of S (median -> scal[0], 1.4826 MAD -> scal[1]) and the strided, clipped rms of C (-> out[0]) from
+// one launch: the median of the samples of C in one slot, the median of S and then the median of the
+// deviations in the other.
+fpsk_status sigma_mad_rms_c_launch(const float *S, long long mm, int mad_of_abs, const float *C, long long ldc,
+                                   long long n1, long long n3, float *samples, SelectWs &w, float *out, cudaStream_t st)
+{
+    const long long nsamp = rms_c_samples(C, ldc, n1, n3, samples, w, st);
+    if (nsamp < 0) return FPSK_ERR_CUDA;
+    const SelJob med = sel_job(mad_of_abs ? SEL_ABS : SEL_SIGNED, 32, S, mm, 0);
+    const SelJob dev = sel_job(mad_of_abs ? SEL_DEV_ABS : SEL_DEV_SIGNED, 32, S, mm, 0);
+    const SelJob smp = sel_job(SEL_SAMPLE, 32, samples, nsamp, 0);
+    fpsk_status rc = run_selects(smp, med, true, dev, true, w, st);
     if (rc != FPSK_OK) return rc;
     clipped_rms_kernel<<<1, 1024, 0, st>>>(samples, nsamp, w.scal, w.counts, out);
     FPSK_LAUNCH_CHECK();
@@ -472,14 +721,15 @@ fpsk_status rms_c_launch(const float *C, long long ldc, long long n1, long long 
 // ---------------------------------------------------------------- workspace
 size_t select_ws_bytes()
 {
-    return 4096 /*hist+ticket*/ + 256 /*state*/ + 256 /*scal*/ + align_up(kSumGrid * 4, 256) +
+    return align_up(kHistBytes, 256) /*hist+tickets*/ + 256 /*state*/ + 256 /*scal*/ + align_up(kSumGrid * 4, 256) +
            align_up(kSelMaxK * 8, 256) + 256 /*counts*/ + align_up(kSelMaxK * sizeof(Candidate), 256);
 }
 
 void select_carve(void *ws, SelectWs &w)
 {
     char *p = static_cast<char *>(ws);
-    w.hist = (unsigned int *)p; p += 4096;
+    w.hist = (unsigned int *)p; p += align_up(kHistBytes, 256);
+    w.err = w.hist + kHistErr;
     w.state = (unsigned long long *)p; p += 256;
     w.scal = (float *)p; p += 256;
     w.partial = (float *)p; p += align_up(kSumGrid * 4, 256);

@@ -298,13 +298,13 @@ __global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *
             *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = mid;
             *reinterpret_cast<uint4 *>(planesQw + off + 2 * 256 * 64) = lo;
         }
-        return;
-    }
+    } else {
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
-        if (k0 + t < kpad) {
-            Q[(long long)(k0 + t) * npad + b] = q[t];
-            if (MOM) Qw[(long long)(k0 + t) * npad + b] = qw[t];
+        for (int t = 0; t < 8; ++t) {
+            if (k0 + t < kpad) {
+                Q[(long long)(k0 + t) * npad + b] = q[t];
+                if (MOM) Qw[(long long)(k0 + t) * npad + b] = qw[t];
+            }
         }
     }
 }

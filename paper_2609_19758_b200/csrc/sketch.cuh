@@ -67,13 +67,14 @@ struct Candidate {          // one decoded bucket of the set U (Algorithm 1)
 };
 
 struct SelectWs {           // all device memory
-    unsigned int *hist;     // 256 bins + control words
+    unsigned int *hist;     // histograms of the radix select (digits x two jobs x copies x 256 bins) + control words
+    unsigned int *err;      // nonzero after a bounded grid-wide wait of a select gave up (the host reads it)
     unsigned long long *state;   // radix-select state
     float *scal;            // scalar results: [0] median, [1] sigma_mad, [2] mean|S|, [3] sigma_clip,
                             //                 [4] thr, [5] tau_c, [6] tau_d
     float *partial;         // per-CTA partial sums
     unsigned long long *keys;    // selected keys (<= kmax)
-    int *counts;            // [0] above-threshold count, [1] collected, [2] n_U
+    int *counts;            // [0] valid samples of C, [1] collected, [2] n_U
     Candidate *cand;        // <= kmax
     bool hist_clean;        // host side: the histogram has been zeroed since this workspace was carved
 };
@@ -81,19 +82,20 @@ constexpr int kSelMaxK = 1024;
 size_t select_ws_bytes();
 void select_carve(void *ws, SelectWs &w);
 
-// sigma_MAD of S (mad_of_abs: of |S| as printed, else signed) -> scal[1]; median -> scal[0]
-fpsk_status sigma_mad_launch(const float *S, long long mm, int mad_of_abs, SelectWs &w, cudaStream_t st);
 // clipped-mean estimate 1.2533 mean(min(|S|, 5 mean|S|)) -> scal[3]
 fpsk_status sigma_clip_launch(const float *S, long long mm, SelectWs &w, cudaStream_t st);
-// thresholds from scal[1] and tau, K largest |S| above max(tau_c, tau_d), decoded candidates
+// thresholds from scal[1] and tau, K largest |S| above max(tau_c, tau_d), decoded candidates.
+// mad_mode >= 0: sigma_MAD of S (1: of |S|, 0: signed) is computed in the same launches first.
 fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
-                                     long long n3, const float *d_tau, int radius, int K, SelectWs &w, cudaStream_t st);
+                                     long long n3, const float *d_tau, int radius, int K, int mad_mode, SelectWs &w,
+                                     cudaStream_t st);
 // device max |X| of a half matrix -> out[0] (float)
 fpsk_status max_abs_half_launch(const void *X, long long ld, long long rows, long long cols, fpsk_dtype dtype,
                                 float *out, unsigned int *scratch, cudaStream_t st);
-// strided, clipped rms of C (Section "Calibration") -> scal_out[0]; uses SelectWs for the median
-fpsk_status rms_c_launch(const float *C, long long ldc, long long n1, long long n3, float *samples,
-                         SelectWs &w, float *out, cudaStream_t st);
+// sigma_MAD of S (mad_of_abs: of |S| as printed, else signed) -> scal[1], median -> scal[0]; and the strided,
+// clipped rms of C (Section "Calibration") -> out[0]; the three medians share one launch
+fpsk_status sigma_mad_rms_c_launch(const float *S, long long mm, int mad_of_abs, const float *C, long long ldc,
+                                   long long n1, long long n3, float *samples, SelectWs &w, float *out, cudaStream_t st);
 
 // ---- confirmation (confirm.cu) ---------------------------------------------------------------
 struct Hit {                // an accepted window entry
