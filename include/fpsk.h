@@ -14,7 +14,9 @@
  *   - The caller owns every buffer.  The library allocates no device memory and never writes
  *     to A or B; C is written only by fpsk_verify_repair and fpsk_apply_corrections (paper,
  *     Section "Overview": localization does not modify C; Algorithm 2, "Apply").
- *     fpsk_localize creates one CUDA event for the duration of the call.
+ *     fpsk_localize and fpsk_verify_repair create one CUDA event for the duration of the call and
+ *     stage each round's results through a small pinned host buffer (about 25 KB) that the
+ *     library creates on first use, one per concurrent call, and keeps for the life of the process.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Indices are 0-based.  The 1-based index weights of the paper are internal.
  *   - Errors are return codes.  Nothing throws, aborts or resets the device.  After

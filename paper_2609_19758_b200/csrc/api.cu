@@ -6,6 +6,7 @@
 #include <math.h>
 #include <string.h>
 #include <algorithm>
+#include <mutex>
 #include <vector>
 
 namespace fpsk {
@@ -13,6 +14,74 @@ std::atomic<unsigned long long> g_launches{0};
 
 constexpr int kHitCap = 2048;
 constexpr int kPeelCap = 4096;
+constexpr int kPackHits = 256;       // hits that travel with a round's results in one copy (more: a second copy)
+
+// What the host needs from a localization round, gathered on the device so that it is ONE copy:
+// header, the candidates, the first kPackHits hits.
+struct RoundHeader {
+    int counts[4];           // [2] = number of candidates (n_U)
+    int n_hits;
+    unsigned int tc_err, sel_err;
+    int pad[9];
+};
+static_assert(sizeof(RoundHeader) == 64, "RoundHeader is 64 bytes");
+constexpr size_t kPackBytes = sizeof(RoundHeader) + (size_t)kSelMaxK * sizeof(Candidate) + (size_t)kPackHits * sizeof(Hit);
+
+__global__ void pack_round_kernel(const int *counts, const int *n_hits, const unsigned int *tc_err,
+                                  const unsigned int *sel_err, const Candidate *cand, int K, const Hit *hits,
+                                  unsigned char *pack)
+{
+    RoundHeader *h = reinterpret_cast<RoundHeader *>(pack);
+    Candidate *pc = reinterpret_cast<Candidate *>(pack + sizeof(RoundHeader));
+    Hit *ph = reinterpret_cast<Hit *>(pack + sizeof(RoundHeader) + (size_t)K * sizeof(Candidate));
+    const int nh = *n_hits;
+    if (threadIdx.x == 0) {
+        for (int q = 0; q < 4; ++q) h->counts[q] = counts[q];
+        h->n_hits = nh;
+        h->tc_err = tc_err ? *tc_err : 0u;
+        h->sel_err = *sel_err;
+    }
+    for (int t = threadIdx.x; t < K; t += blockDim.x) pc[t] = cand[t];
+    const int np = nh < kPackHits ? nh : kPackHits;
+    for (int t = threadIdx.x; t < np; t += blockDim.x) ph[t] = hits[t];
+}
+
+// Pinned host staging for the per-round results.  A pageable destination makes cudaMemcpyAsync block the host
+// until the copy has run, so the next round could not be enqueued behind this one.  Buffers are created on
+// first use (one per concurrent call) and kept for the life of the process.
+struct PinnedPool {
+    std::mutex mu;
+    std::vector<void *> free_list;      // each kPackBytes
+};
+static PinnedPool &pinned_pool()
+{
+    static PinnedPool *p = new PinnedPool;      // never destroyed: no CUDA calls at process exit
+    return *p;
+}
+struct PinnedLease {
+    void *p = nullptr;
+    ~PinnedLease()
+    {
+        if (!p) return;
+        PinnedPool &pool = pinned_pool();
+        std::lock_guard<std::mutex> g(pool.mu);
+        pool.free_list.push_back(p);
+    }
+};
+static fpsk_status pinned_acquire(PinnedLease &l)
+{
+    PinnedPool &pool = pinned_pool();
+    {
+        std::lock_guard<std::mutex> g(pool.mu);
+        if (!pool.free_list.empty()) {
+            l.p = pool.free_list.back();
+            pool.free_list.pop_back();
+            return FPSK_OK;
+        }
+    }
+    FPSK_CUDA_OK(cudaHostAlloc(&l.p, kPackBytes, cudaHostAllocDefault));
+    return FPSK_OK;
+}
 
 // ---------------------------------------------------------------- scalar planner
 static double cf_of(fpsk_dtype d) { return d == FPSK_BF16 ? 0.19 : 1.76 * 0.19; }
@@ -110,6 +179,7 @@ struct LocWs {
     PeelEntry *peel;
     Hit *hits;
     int *n_hits;
+    unsigned char *pack;      // kPackBytes: a round's results in one piece
 };
 
 static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool tc = false)
@@ -123,6 +193,7 @@ static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bo
     b += align_up(sizeof(PeelEntry) * kPeelCap, 256);
     b += align_up(sizeof(Hit) * kHitCap, 256);
     b += 256;
+    b += align_up(kPackBytes, 256);
     return b;
 }
 
@@ -141,6 +212,7 @@ static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, lon
     w.peel = (PeelEntry *)take(sizeof(PeelEntry) * kPeelCap);
     w.hits = (Hit *)take(sizeof(Hit) * kHitCap);
     w.n_hits = (int *)take(256);
+    w.pack = (unsigned char *)take(kPackBytes);
     return true;
 }
 
@@ -203,7 +275,10 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
 
     std::vector<PeelEntry> peel;
     std::vector<Hit> hits(kHitCap);
-    std::vector<Candidate> cand(kSelMaxK);
+    PinnedLease stage;
+    rc = pinned_acquire(stage);
+    if (rc != FPSK_OK) return rc;
+    const size_t pack_bytes = sizeof(RoundHeader) + (size_t)K * sizeof(Candidate) + (size_t)kPackHits * sizeof(Hit);
     // The sketches of round t + 1 do not depend on what round t finds (only the peeling does), so they
     // are enqueued before the host waits for round t's results: the GPU builds them while the host
     // replays the search.  The event marks the end of round t's copies.
@@ -233,14 +308,10 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
         if (rc != FPSK_OK) return rc;
         rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, st);
         if (rc != FPSK_OK) return rc;
-        int h_counts[4] = {0, 0, 0, 0}, h_nhits = 0;
-        FPSK_CUDA_OK(cudaMemcpyAsync(h_counts, w.sel.counts, sizeof(h_counts), cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_nhits, w.n_hits, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * kHitCap, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(cand.data(), w.sel.cand, sizeof(Candidate) * K, cudaMemcpyDeviceToHost, st));
-        unsigned int h_tc_err = 0, h_sel_err = 0;
-        if (w.sk.tc) FPSK_CUDA_OK(cudaMemcpyAsync(&h_tc_err, w.sk.tc_err, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
+        pack_round_kernel<<<1, 256, 0, st>>>(w.sel.counts, w.n_hits, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.sel.cand, K,
+                                             w.hits, w.pack);
+        FPSK_LAUNCH_CHECK();
+        FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, pack_bytes, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaEventRecord(round_done.e, st));
         if (t + 1 < q.rounds) {
             rc = build_sketches(in, dtype, seed, t + 1, m_b, true, w.sk, st, w.S, w.R, w.T);
@@ -248,9 +319,22 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
             built_ahead = true;
         }
         FPSK_CUDA_OK(cudaEventSynchronize(round_done.e));
-        if (h_tc_err || h_sel_err) return FPSK_ERR_TIMEOUT;        // a bounded wait (contraction, selects) gave up
+        const RoundHeader *hdr = static_cast<const RoundHeader *>(stage.p);
+        const Candidate *cand = reinterpret_cast<const Candidate *>(static_cast<const char *>(stage.p) + sizeof(RoundHeader));
+        const Hit *packed_hits = reinterpret_cast<const Hit *>(static_cast<const char *>(stage.p) + sizeof(RoundHeader) +
+                                                               (size_t)K * sizeof(Candidate));
+        if (hdr->tc_err || hdr->sel_err) return FPSK_ERR_TIMEOUT;        // a bounded wait (contraction, selects) gave up
+        int h_nhits = hdr->n_hits;
         if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
-        const int nU = std::min(h_counts[2], K);
+        const int nU = std::min(hdr->counts[2], K);
+        if (h_nhits <= kPackHits) {
+            std::copy(packed_hits, packed_hits + h_nhits, hits.begin());
+        } else {
+            // more hits than travel with the header: fetch the list itself (the stream runs the next round's
+            // sketches meanwhile; they do not touch it)
+            FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * h_nhits, cudaMemcpyDeviceToHost, st));
+            FPSK_CUDA_OK(cudaStreamSynchronize(st));
+        }
 
         // replay of Algorithm 1's search: offsets in Chebyshev-then-Manhattan order, buckets of U
         // in selection order; a bucket leaves U at its first accepted entry

@@ -603,22 +603,44 @@ __global__ void __launch_bounds__(256) max_abs_half_kernel(const unsigned short 
     if (vec_ok) {
         const long long cv = cols / 8;               // 16-byte vectors per row
         const long long total = rows * cv;
-        for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-            const long long r = i / cv, c = i - r * cv;
-            const uint4 v = ldg_nc_v4(X + r * ld + c * 8);
-            const unsigned int w[4] = {v.x, v.y, v.z, v.w};
+        // four independent 16-byte loads in flight per thread
+        const long long stride = (long long)gridDim.x * blockDim.x;
+        for (long long i0 = (long long)blockIdx.x * blockDim.x + threadIdx.x; i0 < total; i0 += 4 * stride) {
+            uint4 v[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                m = max(m, (w[q] >> 16) & 0x7FFFu);
-                m = max(m, w[q] & 0x7FFFu);
+            for (int u = 0; u < 4; ++u) {
+                const long long i = i0 + u * stride;
+                long long off = i * 8;                   // rows back to back: no division
+                if (ld != cols) {
+                    const long long r = i / cv;
+                    off = r * ld + (i - r * cv) * 8;
+                }
+                v[u] = i < total ? ldg_nc_v4(X + off) : make_uint4(0, 0, 0, 0);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const unsigned int w[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    m = max(m, (w[q] >> 16) & 0x7FFFu);
+                    m = max(m, w[q] & 0x7FFFu);
+                }
             }
         }
     } else {
         for (long long r = blockIdx.x; r < rows; r += gridDim.x)
             for (long long c = threadIdx.x; c < cols; c += blockDim.x) m = max(m, (unsigned int)(X[r * ld + c] & 0x7FFFu));
     }
+    // one atomic per CTA: thousands of atomics on the one word took longer than reading the matrix
+    __shared__ unsigned int wmax[8];
     m = __reduce_max_sync(0xFFFFFFFFu, m);
-    if ((threadIdx.x & 31) == 0 && m) atomicMax(out, m);
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = m;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 1; w < 8; ++w) m = max(m, wmax[w]);
+        if (m) atomicMax(out, m);
+    }
 }
 template <typename T>
 __global__ void max_abs_finish_kernel(const unsigned int *bits, float *out)
@@ -633,7 +655,7 @@ fpsk_status max_abs_half_launch(const void *X, long long ld, long long rows, lon
     const unsigned short *x = static_cast<const unsigned short *>(X);
     const int vec_ok = ((reinterpret_cast<uintptr_t>(X) & 15) == 0 && ld % 8 == 0 && cols % 8 == 0) ? 1 : 0;
     long long want = vec_ok ? (rows * (cols / 8) + 256 * 4 - 1) / (256 * 4) : rows;
-    const int grid = (int)(want < 1 ? 1 : (want > 2368 ? 2368 : want));
+    const int grid = (int)(want < 1 ? 1 : (want > 1184 ? 1184 : want));
     if (dtype == FPSK_FP16) {
         max_abs_half_kernel<__half><<<grid, 256, 0, st>>>(x, ld, rows, cols, vec_ok, scratch);
         FPSK_LAUNCH_CHECK();
