@@ -238,6 +238,10 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
     const long long mm = (long long)m_b * m_b;
     const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
     fpsk_status rc;
+    SketchAuxLease aux;
+    rc = sketch_aux_acquire(aux);
+    if (rc != FPSK_OK) return rc;
+    w.sk.aux = aux.aux;
     // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
     unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
     rc = max_abs_half_launch(in.A, in.lda, m, k, dtype, w.misc + 0, uscr, st);
@@ -667,6 +671,10 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
+    SketchAuxLease aux;
+    rc = sketch_aux_acquire(aux);
+    if (rc != FPSK_OK) return rc;
+    w.sk.aux = aux.aux;
     rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
     if (rc != FPSK_OK) return rc;
     const long long mm = (long long)m0 * m0;

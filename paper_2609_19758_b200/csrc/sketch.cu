@@ -11,6 +11,9 @@
 //   combine_kernel      S = sum of AB partials - sum of C partials
 #include "sketch.cuh"
 
+#include <mutex>
+#include <vector>
+
 namespace fpsk {
 
 // ---------------------------------------------------------------- hash tables
@@ -811,6 +814,7 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
     if (ws_bytes < sketch_ws_bytes(n1, n2, n3, m_b, tc)) return false;
     tc = tc && m_b >= kTcMinBuckets;
     sketch_plan(n1, n2, n3, m_b, w.pl);
+    w.aux = nullptr;
     const size_t mm = (size_t)m_b * m_b;
     char *p = static_cast<char *>(ws);
     auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
@@ -841,6 +845,46 @@ int sketch_max_buckets(long long n1, long long n2, long long n3)
     return (int)m;
 }
 
+// ---------------------------------------------------------------- auxiliary streams
+struct SketchAuxPool {
+    std::mutex mu;
+    std::vector<SketchAux *> free_list;
+};
+static SketchAuxPool &sketch_aux_pool()
+{
+    static SketchAuxPool *p = new SketchAuxPool;       // never destroyed: no CUDA calls at process exit
+    return *p;
+}
+SketchAuxLease::~SketchAuxLease()
+{
+    if (!aux) return;
+    SketchAuxPool &pool = sketch_aux_pool();
+    std::lock_guard<std::mutex> g(pool.mu);
+    pool.free_list.push_back(aux);
+}
+fpsk_status sketch_aux_acquire(SketchAuxLease &lease)
+{
+    int dev = 0;
+    FPSK_CUDA_OK(cudaGetDevice(&dev));
+    SketchAuxPool &pool = sketch_aux_pool();
+    {
+        std::lock_guard<std::mutex> g(pool.mu);
+        for (size_t i = 0; i < pool.free_list.size(); ++i) {
+            if (pool.free_list[i]->device != dev) continue;
+            lease.aux = pool.free_list[i];
+            pool.free_list.erase(pool.free_list.begin() + (long)i);
+            return FPSK_OK;
+        }
+    }
+    SketchAux *a = new SketchAux;
+    a->device = dev;
+    lease.aux = a;                  // returned to the pool even when a creation below fails (unused handles stay null)
+    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a->s1, cudaStreamNonBlocking));
+    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a->s2, cudaStreamNonBlocking));
+    for (int e = 0; e < 5; ++e) FPSK_CUDA_OK(cudaEventCreateWithFlags(&a->ev[e], cudaEventDisableTiming));
+    return FPSK_OK;
+}
+
 template <typename T>
 static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, int m_b, bool mom, SketchWs &w,
                                     cudaStream_t st, float *S, float *R, float *Tt)
@@ -849,10 +893,25 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     const float inv_p1 = 1.0f / (float)(1LL << pow2_exp(n1));
     const float inv_p3 = 1.0f / (float)(1LL << pow2_exp(n3));
     fpsk_status rc;
+    // st: row side, A compression, contraction, combine; sB: column side, B compression; sC: C scatter
+    // (needs both sides).  Without auxiliary streams all three are st.
+    SketchAux *ax = (w.aux && w.aux->s1 && w.aux->s2 && w.aux->ev[4]) ? w.aux : nullptr;
+    cudaStream_t sB = ax ? ax->s1 : st, sC = ax ? ax->s2 : st;
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));             // everything queued before this build
+        FPSK_CUDA_OK(cudaStreamWaitEvent(sB, ax->ev[0], 0));
+        FPSK_CUDA_OK(cudaStreamWaitEvent(sC, ax->ev[0], 0));
+    }
     rc = build_hash_side(seed, rnd, 0, n1, m_b, w.h1, w.v1, w.rowcount, w.rowstart, w.rowperm, st);
     if (rc != FPSK_OK) return rc;
-    rc = build_hash_side(seed, rnd, 1, n3, m_b, w.h2, w.v2, w.colcount, w.colstart, w.colperm, st, w.colpos);
+    rc = build_hash_side(seed, rnd, 1, n3, m_b, w.h2, w.v2, w.colcount, w.colstart, w.colperm, sB, w.colpos);
     if (rc != FPSK_OK) return rc;
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[1], st));             // row side ready
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[2], sB));             // column side ready
+        FPSK_CUDA_OK(cudaStreamWaitEvent(sC, ax->ev[1], 0));
+        FPSK_CUDA_OK(cudaStreamWaitEvent(sC, ax->ev[2], 0));
+    }
 
     const unsigned short *A = static_cast<const unsigned short *>(in.A);
     const unsigned short *B = static_cast<const unsigned short *>(in.B);
@@ -881,7 +940,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         const int kcols = w.tc ? kblocks * 32 : pl.kpad;
         const int bmax = w.tc ? btiles * 256 : pl.npad;
         dim3 grid((kcols / 8 + 15) / 16, (bmax + 7) / 8);
-#define FPSK_CW(V, M, PL) compress_wt_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3])
+#define FPSK_CW(V, M, PL) compress_wt_kernel<T, V, M, PL><<<grid, 128, 0, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3])
         if (w.tc) {
             if (vec) { if (mom) FPSK_CW(true, true, true); else FPSK_CW(true, false, true); }
             else     { if (mom) FPSK_CW(false, true, true); else FPSK_CW(false, false, true); }
@@ -898,7 +957,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
 #define FPSK_CB8(M, PL)                                                                                                          \
     do {                                                                                                                         \
         FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b8_kernel<T, M, PL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        compress_b8_kernel<T, M, PL><<<grid, 256, smem, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm,      \
+        compress_b8_kernel<T, M, PL><<<grid, 256, smem, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm,      \
                                                               w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3]); \
     } while (0)
         if (w.tc) { if (mom) FPSK_CB8(true, true); else FPSK_CB8(false, true); }
@@ -910,26 +969,59 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         int grid = pl.kpad < 1184 ? pl.kpad : 1184;
         if (mom) {
             FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b_kernel<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            compress_b_kernel<T, true><<<grid, 256, smem, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw);
+            compress_b_kernel<T, true><<<grid, 256, smem, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw);
         } else {
             FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b_kernel<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            compress_b_kernel<T, false><<<grid, 256, smem, st>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw);
+            compress_b_kernel<T, false><<<grid, 256, smem, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw);
         }
         FPSK_LAUNCH_CHECK();
+    }
+    if (w.tc && !b8 && !in.bt) {
+        // wide B: Q, Qw came out as FP32 rows; split them here (row b of Q^T is column b of Q)
+        rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], sB);
+        if (rc != FPSK_OK) return rc;
+        if (mom) {
+            rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], sB);
+            if (rc != FPSK_OK) return rc;
+        }
+    }
+    // ---- C scatter: independent of the compressions and of the contraction
+    {
+        const size_t smem = ((size_t)2 * kScChunk + 3 * (size_t)m_b) * 4;
+        dim3 grid(m_b, pl.nsplit);
+        const bool vec = (reinterpret_cast<uintptr_t>(in.C) & 15) == 0 && in.ldc % 4 == 0 && n3 % 4 == 0;
+#define FPSK_SC(M, V)                                                                                                        \
+    do {                                                                                                                     \
+        FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<M, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
+        scatter_c_kernel<M, V><<<grid, 256, smem, sC>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart,  \
+                                                        w.colperm, w.colstart, pl.nsplit, w.partC);                          \
+    } while (0)
+        const size_t smem2 = (size_t)(mom ? 3 : 1) * ((n3 + 3) & ~3) * 4 + (size_t)(m_b + 1) * 4;
+#define FPSK_SC2(M, V)                                                                                                        \
+    do {                                                                                                                      \
+        FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c2_kernel<M, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)); \
+        scatter_c2_kernel<M, V><<<grid, 256, smem2, sC>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, \
+                                                          w.colpos, w.colstart, pl.nsplit, w.partC);                          \
+    } while (0)
+        if (n3 <= kSc2MaxCols) {
+            if (mom) { if (vec) FPSK_SC2(true, true); else FPSK_SC2(true, false); }
+            else     { if (vec) FPSK_SC2(false, true); else FPSK_SC2(false, false); }
+        } else {
+            if (mom) { if (vec) FPSK_SC(true, true); else FPSK_SC(true, false); }
+            else     { if (vec) FPSK_SC(false, true); else FPSK_SC(false, false); }
+        }
+#undef FPSK_SC2
+#undef FPSK_SC
+        FPSK_LAUNCH_CHECK();
+    }
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[3], sB));             // B side compressed
+        FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->ev[3], 0));
     }
     int ab_splits = pl.ksplit;
     if (w.tc) {
         // split-BF16 contraction on the tensor cores, one launch for all problems
         FPSK_CUDA_OK(cudaMemsetAsync(w.tc_err, 0, 4, st));
-        if (!b8 && !in.bt) {
-            // wide B: Q, Qw came out as FP32 rows; split them here (row b of Q^T is column b of Q)
-            rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], st);
-            if (rc != FPSK_OK) return rc;
-            if (mom) {
-                rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], st);
-                if (rc != FPSK_OK) return rc;
-            }
-        }
         const unsigned char *pa[2] = {w.planes[0], w.planes[1]}, *pb[2] = {w.planes[2], w.planes[3]};
         const int selA[3] = {0, 1, 0}, selB[3] = {0, 0, 1};
         ab_splits = w.tc_ksplit;
@@ -953,33 +1045,9 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         }
         FPSK_LAUNCH_CHECK();
     }
-    {
-        const size_t smem = ((size_t)2 * kScChunk + 3 * (size_t)m_b) * 4;
-        dim3 grid(m_b, pl.nsplit);
-        const bool vec = (reinterpret_cast<uintptr_t>(in.C) & 15) == 0 && in.ldc % 4 == 0 && n3 % 4 == 0;
-#define FPSK_SC(M, V)                                                                                                        \
-    do {                                                                                                                     \
-        FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c_kernel<M, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        scatter_c_kernel<M, V><<<grid, 256, smem, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart,  \
-                                                        w.colperm, w.colstart, pl.nsplit, w.partC);                          \
-    } while (0)
-        const size_t smem2 = (size_t)(mom ? 3 : 1) * ((n3 + 3) & ~3) * 4 + (size_t)(m_b + 1) * 4;
-#define FPSK_SC2(M, V)                                                                                                        \
-    do {                                                                                                                      \
-        FPSK_CUDA_OK(cudaFuncSetAttribute(scatter_c2_kernel<M, V>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2)); \
-        scatter_c2_kernel<M, V><<<grid, 256, smem2, st>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, \
-                                                          w.colpos, w.colstart, pl.nsplit, w.partC);                          \
-    } while (0)
-        if (n3 <= kSc2MaxCols) {
-            if (mom) { if (vec) FPSK_SC2(true, true); else FPSK_SC2(true, false); }
-            else     { if (vec) FPSK_SC2(false, true); else FPSK_SC2(false, false); }
-        } else {
-            if (mom) { if (vec) FPSK_SC(true, true); else FPSK_SC(true, false); }
-            else     { if (vec) FPSK_SC(false, true); else FPSK_SC(false, false); }
-        }
-#undef FPSK_SC2
-#undef FPSK_SC
-        FPSK_LAUNCH_CHECK();
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[4], sC));             // C sketches ready
+        FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->ev[4], 0));
     }
     {
         const long long mm = (long long)m_b * m_b;

@@ -19,8 +19,24 @@ struct SketchPlan {
     int tile;      // 64 or 128
 };
 
+// Two more streams and the events that tie them to the caller's stream: the parts of a sketch build that do
+// not depend on each other (row side + A compression, column side + B compression, C scatter) run side by
+// side, and the C scatter hides under the contraction.  Created on first use, kept for the life of the process,
+// one set per concurrent call and device.
+struct SketchAux {
+    int device = -1;
+    cudaStream_t s1 = nullptr, s2 = nullptr;
+    cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+};
+struct SketchAuxLease {          // returns the set to the pool when it goes out of scope
+    SketchAux *aux = nullptr;
+    ~SketchAuxLease();
+};
+fpsk_status sketch_aux_acquire(SketchAuxLease &lease);
+
 struct SketchWs {
     SketchPlan pl;
+    SketchAux *aux;              // nullptr: everything on the caller's stream
     int *h1, *v1, *h2, *v2;
     uint32_t *rowperm, *colperm;
     uint32_t *colpos;            // inverse of colperm: position (and sign) of every column in the bucket-sorted order
