@@ -216,6 +216,19 @@ static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, lon
     return true;
 }
 
+// max|A| -> misc[0], max|B| -> misc[1] (device); the tensor-core contraction scales its planes by them
+static fpsk_status loc_max_ab(const SketchIn &in, fpsk_dtype dtype, LocWs &w, cudaStream_t st)
+{
+    unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
+    fpsk_status rc = max_abs_half_launch(in.A, in.lda, in.n1, in.n2, dtype, w.misc + 0, uscr, st);
+    if (rc != FPSK_OK) return rc;
+    rc = in.bt ? max_abs_half_launch(in.B, in.ldb, in.n3, in.n2, dtype, w.misc + 1, uscr + 1, st)
+               : max_abs_half_launch(in.B, in.ldb, in.n2, in.n3, dtype, w.misc + 1, uscr + 1, st);
+    if (rc != FPSK_OK) return rc;
+    w.sk.d_maxab = w.misc;
+    return FPSK_OK;
+}
+
 __global__ void tau_kernel(float *misc, float n2)
 {
     if (threadIdx.x == 0) misc[2] = 100.f * n2 * 1.1920928955078125e-07f * misc[0] * misc[1];
@@ -243,11 +256,7 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
     if (rc != FPSK_OK) return rc;
     w.sk.aux = aux.aux;
     // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
-    unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
-    rc = max_abs_half_launch(in.A, in.lda, m, k, dtype, w.misc + 0, uscr, st);
-    if (rc != FPSK_OK) return rc;
-    rc = in.bt ? max_abs_half_launch(in.B, in.ldb, n, k, dtype, w.misc + 1, uscr + 1, st)
-               : max_abs_half_launch(in.B, in.ldb, k, n, dtype, w.misc + 1, uscr + 1, st);
+    rc = loc_max_ab(in, dtype, w, st);
     if (rc != FPSK_OK) return rc;
     tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
     FPSK_LAUNCH_CHECK();
@@ -675,6 +684,10 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     rc = sketch_aux_acquire(aux);
     if (rc != FPSK_OK) return rc;
     w.sk.aux = aux.aux;
+    if (w.sk.tc) {
+        rc = loc_max_ab(in, dtype, w, st);
+        if (rc != FPSK_OK) return rc;
+    }
     rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
     if (rc != FPSK_OK) return rc;
     const long long mm = (long long)m0 * m0;
@@ -880,6 +893,10 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
         LocWs w0;
         if (!loc_carve(loc_ws, loc_bytes, m, k, n, m0, w0, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
         SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+        if (w0.sk.tc) {
+            rc = loc_max_ab(in, dtype, w0, st);
+            if (rc != FPSK_OK) return rc;
+        }
         rc = build_sketches(in, dtype, seed, 0, m0, false, w0.sk, st, w0.S, nullptr, nullptr);
         if (rc != FPSK_OK) return rc;
         rc = sigma_mad_rms_c_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);

@@ -527,6 +527,27 @@ __global__ void __launch_bounds__(256) hp_fold_plain_kernel(const HpArgs p)
     }
 }
 
+// scale[0] = the power of two for the P planes, from the per-CTA maxima of |A| (16-bit patterns) and the
+// largest row bucket
+template <typename T>
+__global__ void __launch_bounds__(256) hp_scale_a_kernel(const unsigned int *maxA, int n_maxA, const int *rowcount, int m, float *scale)
+{
+    __shared__ unsigned int wbits[8];
+    __shared__ int wcnt[8];
+    unsigned int mb = 0;
+    int c = 0;
+    for (int r = threadIdx.x; r < n_maxA; r += blockDim.x) mb = max(mb, maxA[r]);
+    for (int b = threadIdx.x; b < m; b += blockDim.x) c = max(c, rowcount[b]);
+    mb = __reduce_max_sync(0xFFFFFFFFu, mb);
+    c = __reduce_max_sync(0xFFFFFFFFu, c);
+    if ((threadIdx.x & 31) == 0) { wbits[threadIdx.x >> 5] = mb; wcnt[threadIdx.x >> 5] = c; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) { mb = max(mb, wbits[w]); c = max(c, wcnt[w]); }
+        scale[0] = tc_scale_of(c, bits16_to_float<T>((unsigned short)mb));
+    }
+}
+
 // ---------------------------------------------------------------- combine + verdict
 struct HvArgs {
     const float *partAB;     // [ksplit][m*m]
@@ -536,7 +557,8 @@ struct HvArgs {
     int m, n1, n2, n3;
     const unsigned int *maxA;
     int n_maxA;
-    const float *maxB;       // [1] max|B|
+    const float *maxB;       // [0] max|B|, [1] scale of the Q planes
+    const float *scaleA;     // scale of the P planes when the partials come from the tensor cores, else null
     float thr_scale;         // mu sqrt(2 ln max(m^2, 2))
     float cap_scale;         // sqrt(n1 n3 / m^2)
     float *S;                // m*m
@@ -647,6 +669,7 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
     const long long q4 = (mm + 3) / 4;
     const long long i0 = 4 * (q4 * c / G), i1 = min(mm, 4 * (q4 * (c + 1) / G));
     HvStat l = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
+    const float unscale = p.scaleA ? 1.f / (__ldcg(p.scaleA) * __ldcg(p.maxB + 1)) : 1.f;      // powers of two: exact
     for (long long i = i0 + tid; i < i1; i += kHvThreads) {
         float ab = 0.f;
         for (int s0 = 0; s0 < p.ksplit; s0 += 8) {
@@ -656,6 +679,7 @@ __global__ void __launch_bounds__(kHvThreads) hp_combine_kernel(const HvArgs p)
 #pragma unroll
             for (int q = 0; q < 8; ++q) ab += v[q];
         }
+        ab *= unscale;
         float cf = 0.f;
         for (int s0 = 0; s0 < p.nseg; s0 += 8) {
             float v[8];
@@ -808,8 +832,8 @@ struct HpCache {          // the B side, device memory kept by the caller across
     uint32_t *segperm;
     int *segstart;
     float *Q;
-    unsigned char *Qplanes;   // Q^T as tiled BF16 planes (tensor-core contraction)
-    float *maxB;          // [0] max|B|
+    unsigned char *Qplanes;   // Q^T as tiled FP16 planes (tensor-core contraction), scaled by maxB[1]
+    float *maxB;          // [0] max|B|, [1] the power of two that brings Q into FP16 range
     unsigned int *scratch;
 };
 
@@ -847,6 +871,7 @@ struct HpWork {           // per-call scratch
     float4 *vstat;
     float *P, *Tc, *partAB, *partC, *S, *cstat;
     unsigned char *Pplanes;
+    float *scaleA;        // the power of two that brings P into FP16 range (tensor-core contraction)
     unsigned long long *trace;
 };
 
@@ -866,6 +891,7 @@ static size_t hp_work_layout(void *base, long long n1, long long n2, long long n
     t.Tc = (float *)take((size_t)m * n3 * 4);
     t.partAB = (float *)take((size_t)(pl.ksplit > pl.tc_ksplit ? pl.ksplit : pl.tc_ksplit) * m * m * 4);
     t.Pplanes = (unsigned char *)take(tc_planes_bytes(m, pl.kpad));
+    t.scaleA = (float *)take(256);
     t.partC = (float *)take((size_t)pl.segsC * m * m * 4);
     t.S = (float *)take((size_t)m * m * 4);
     t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 256);       // 8 stamps per team
@@ -932,10 +958,12 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, int b_transposed, long 
         rc = build_b_side(B, ldb, n2, n3, dtype, m, pl.kpad, pl.npad, c.colperm, c.colstart, c.Q, st);
         if (rc != FPSK_OK) return rc;
     }
-    rc = tc_split_launch(c.Q, 1, pl.npad, m, pl.kpad, 1, c.Qplanes, st);      // row b of Q^T is column b of Q
-    if (rc != FPSK_OK) return rc;
     rc = b_transposed ? max_abs_half_launch(B, ldb, n3, n2, dtype, c.maxB, c.scratch, st)
                       : max_abs_half_launch(B, ldb, n2, n3, dtype, c.maxB, c.scratch, st);
+    if (rc != FPSK_OK) return rc;
+    rc = tc_scale_launch(c.colcount, m, c.maxB, c.maxB + 1, st);
+    if (rc != FPSK_OK) return rc;
+    rc = tc_split_launch(c.Q, c.maxB + 1, 1, pl.npad, m, pl.kpad, 1, c.Qplanes, st);      // row b of Q^T is column b of Q
     if (rc != FPSK_OK) return rc;
     const HpArgs a = hp_args(nullptr, 0, nullptr, 0, n1, n2, n3, m, pl, c, nullptr);
     hp_segment_lists_kernel<<<pl.segsC, 256, (size_t)(m + 1) * 4, st>>>(c.h2, c.v2, (int)n3, m, c.segperm, c.segstart);
@@ -995,7 +1023,10 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     fpsk_status rc;
     int ksplit = pl.ksplit;
     if (tensor_cores) {
-        rc = tc_split_launch(w.P, pl.kpad, 1, m, pl.kpad, 0, w.Pplanes, st);
+        if (dtype == FPSK_FP16) hp_scale_a_kernel<__half><<<1, 256, 0, st>>>(w.maxA, n_maxA, c.rowcount, m, w.scaleA);
+        else hp_scale_a_kernel<__nv_bfloat16><<<1, 256, 0, st>>>(w.maxA, n_maxA, c.rowcount, m, w.scaleA);
+        FPSK_LAUNCH_CHECK();
+        rc = tc_split_launch(w.P, w.scaleA, pl.kpad, 1, m, pl.kpad, 0, w.Pplanes, st);
         if (rc != FPSK_OK) return rc;
         const unsigned char *pa[2] = {w.Pplanes, w.Pplanes}, *pb[2] = {c.Qplanes, c.Qplanes};
         const int sel[3] = {0, 0, 0};
@@ -1009,6 +1040,7 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     v.partAB = w.partAB; v.ksplit = ksplit; v.partC = w.partC; v.nseg = pl.segsC;
     v.m = m; v.n1 = (int)n1; v.n2 = (int)n2; v.n3 = (int)n3;
     v.maxA = w.maxA; v.n_maxA = n_maxA; v.maxB = c.maxB;
+    v.scaleA = tensor_cores ? w.scaleA : nullptr;
     const double mm = (double)m * (double)m;
     v.thr_scale = (float)(mu * sqrt(2.0 * log(mm > 2.0 ? mm : 2.0)));
     v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);

@@ -96,30 +96,49 @@ fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, in
     return FPSK_OK;
 }
 
-// Eight FP32 values -> the 16-byte chunks of their three BF16 terms (x = hi + mid + lo, remainders exact).
-__device__ __forceinline__ void split8_bf16(const float (&x)[8], uint4 &hi, uint4 &mid, uint4 &lo)
+// Eight FP32 values, scaled by a power of two -> the 16-byte chunks of their two FP16 terms (x = hi + lo up to
+// 2^-24 |x|: the remainder x - hi is exact in FP32 and lo rounds it to 11 bits).
+__device__ __forceinline__ void split8_f16(const float (&x)[8], float scale, uint4 &hi, uint4 &lo)
 {
-    unsigned short h[8], m[8], l[8];
+    unsigned short h[8], l[8];
 #pragma unroll
     for (int j = 0; j < 8; ++j) {
-        const __nv_bfloat16 bh = __float2bfloat16_rn(x[j]);
-        const float r1 = x[j] - __bfloat162float(bh);
-        const __nv_bfloat16 bm = __float2bfloat16_rn(r1);
-        const float r2 = r1 - __bfloat162float(bm);
-        const __nv_bfloat16 bl = __float2bfloat16_rn(r2);
-        h[j] = __bfloat16_as_ushort(bh); m[j] = __bfloat16_as_ushort(bm); l[j] = __bfloat16_as_ushort(bl);
+        const float xs = x[j] * scale;
+        const __half bh = __float2half_rn(xs);
+        const float r1 = xs - __half2float(bh);
+        const __half bl = __float2half_rn(r1);
+        h[j] = __half_as_ushort(bh); l[j] = __half_as_ushort(bl);
     }
     hi = make_uint4(h[0] | ((unsigned)h[1] << 16), h[2] | ((unsigned)h[3] << 16), h[4] | ((unsigned)h[5] << 16), h[6] | ((unsigned)h[7] << 16));
-    mid = make_uint4(m[0] | ((unsigned)m[1] << 16), m[2] | ((unsigned)m[3] << 16), m[4] | ((unsigned)m[5] << 16), m[6] | ((unsigned)m[7] << 16));
     lo = make_uint4(l[0] | ((unsigned)l[1] << 16), l[2] | ((unsigned)l[3] << 16), l[4] | ((unsigned)l[5] << 16), l[6] | ((unsigned)l[7] << 16));
 }
 // Where the chunk (row r, eight k starting at k0) of a tiled operand plane sits (layout of tc_contract.cu):
-// tiles of R rows by 32 k, the three planes of a tile back to back.
+// tiles of R rows by 32 k, the planes of a tile back to back.
 template <int R>
 __device__ __forceinline__ size_t plane_chunk_offset(int r, int k0, int kblocks)
 {
     const int rt = r / R, rr = r % R, kb = k0 >> 5, kc = (k0 & 31) >> 3;
-    return ((size_t)rt * kblocks + kb) * 3 * (size_t)(R * 64) + (size_t)(kc * (R / 8) + rr / 8) * 128 + (size_t)(rr % 8) * 16;
+    return ((size_t)rt * kblocks + kb) * kTcPlanes * (size_t)(R * 64) + (size_t)(kc * (R / 8) + rr / 8) * 128 + (size_t)(rr % 8) * 16;
+}
+
+__global__ void __launch_bounds__(256) tc_scale_kernel(const int *count, int m_b, const float *maxv, float *scale)
+{
+    __shared__ int wmax[8];
+    int c = 0;
+    for (int b = threadIdx.x; b < m_b; b += blockDim.x) c = max(c, count[b]);
+    c = __reduce_max_sync(0xFFFFFFFFu, c);
+    if ((threadIdx.x & 31) == 0) wmax[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) c = max(c, wmax[w]);
+        scale[0] = tc_scale_of(c, maxv[0]);
+    }
+}
+fpsk_status tc_scale_launch(const int *count, int m_b, const float *maxv, float *scale, cudaStream_t st)
+{
+    tc_scale_kernel<<<1, 256, 0, st>>>(count, m_b, maxv, scale);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
 }
 
 // ---------------------------------------------------------------- A compression
@@ -131,7 +150,8 @@ template <typename T, bool VEC, bool MOM, bool PLANES>
 __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A, long long lda, int n1, int n2,
                                                          int kpad, float inv_p1, const uint32_t *rowperm,
                                                          const int *rowstart, float *P, float *Pw, int kblocks,
-                                                         unsigned char *planesP, unsigned char *planesPw, int m_b)
+                                                         unsigned char *planesP, unsigned char *planesPw, int m_b,
+                                                         const float *tc_scale)
 {
     // FP32 output: CTA = one bucket, consecutive threads = consecutive columns.  Plane output: a warp covers
     // eight consecutive buckets x four k-chunks, because the eight buckets of a k-chunk are one 128-byte
@@ -171,16 +191,15 @@ __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A
     }
     if (PLANES) {
         const size_t off = plane_chunk_offset<128>(a, (int)col0, kblocks);
-        uint4 hi, mid, lo;
-        split8_bf16(acc, hi, mid, lo);
+        const float sc = __ldg(tc_scale);
+        uint4 hi, lo;
+        split8_f16(acc, sc, hi, lo);
         *reinterpret_cast<uint4 *>(planesP + off) = hi;
-        *reinterpret_cast<uint4 *>(planesP + off + 128 * 64) = mid;
-        *reinterpret_cast<uint4 *>(planesP + off + 2 * 128 * 64) = lo;
+        *reinterpret_cast<uint4 *>(planesP + off + 128 * 64) = lo;
         if (MOM) {
-            split8_bf16(accw, hi, mid, lo);
+            split8_f16(accw, sc, hi, lo);
             *reinterpret_cast<uint4 *>(planesPw + off) = hi;
-            *reinterpret_cast<uint4 *>(planesPw + off + 128 * 64) = mid;
-            *reinterpret_cast<uint4 *>(planesPw + off + 2 * 128 * 64) = lo;
+            *reinterpret_cast<uint4 *>(planesPw + off + 128 * 64) = lo;
         }
         return;
     }
@@ -252,7 +271,7 @@ __global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *
                                                           int kpad, int m_b, int npad, float inv_p3,
                                                           const uint32_t *colperm, const int *colstart, float *Q,
                                                           float *Qw, int kblocks, int btiles, unsigned char *planesQ,
-                                                          unsigned char *planesQw)
+                                                          unsigned char *planesQw, const float *tc_scale)
 {
     const int b = (int)blockIdx.y * 8 + (int)(threadIdx.x & 7);
     const int k0 = ((int)blockIdx.x * (int)(blockDim.x / 8) + (int)(threadIdx.x >> 3)) * 8;
@@ -290,16 +309,15 @@ __global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *
     }
     if (PLANES) {
         const size_t off = plane_chunk_offset<256>(b, k0, kblocks);
-        uint4 hi, mid, lo;
-        split8_bf16(q, hi, mid, lo);
+        const float sc = __ldg(tc_scale);
+        uint4 hi, lo;
+        split8_f16(q, sc, hi, lo);
         *reinterpret_cast<uint4 *>(planesQ + off) = hi;
-        *reinterpret_cast<uint4 *>(planesQ + off + 256 * 64) = mid;
-        *reinterpret_cast<uint4 *>(planesQ + off + 2 * 256 * 64) = lo;
+        *reinterpret_cast<uint4 *>(planesQ + off + 256 * 64) = lo;
         if (MOM) {
-            split8_bf16(qw, hi, mid, lo);
+            split8_f16(qw, sc, hi, lo);
             *reinterpret_cast<uint4 *>(planesQw + off) = hi;
-            *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = mid;
-            *reinterpret_cast<uint4 *>(planesQw + off + 2 * 256 * 64) = lo;
+            *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = lo;
         }
     } else {
 #pragma unroll
@@ -325,7 +343,7 @@ __global__ void __launch_bounds__(256) compress_b8_kernel(const unsigned short *
                                                           int kpad, int m_b, int npad, float inv_p3,
                                                           const uint32_t *colperm, const int *colstart, float *Q,
                                                           float *Qw, int kblocks, int btiles, unsigned char *planesQ,
-                                                          unsigned char *planesQw)
+                                                          unsigned char *planesQw, const float *tc_scale)
 {
     extern __shared__ __align__(16) unsigned short rowbuf8[];
     const int n3p = (n3 + 7) & ~7;
@@ -366,16 +384,15 @@ __global__ void __launch_bounds__(256) compress_b8_kernel(const unsigned short *
             }
             if (PLANES) {
                 const size_t off = plane_chunk_offset<256>(b, k0, kblocks);
-                uint4 hi, mid, lo;
-                split8_bf16(q, hi, mid, lo);
+                const float sc = __ldg(tc_scale);
+                uint4 hi, lo;
+                split8_f16(q, sc, hi, lo);
                 *reinterpret_cast<uint4 *>(planesQ + off) = hi;
-                *reinterpret_cast<uint4 *>(planesQ + off + 256 * 64) = mid;
-                *reinterpret_cast<uint4 *>(planesQ + off + 2 * 256 * 64) = lo;
+                *reinterpret_cast<uint4 *>(planesQ + off + 256 * 64) = lo;
                 if (MOM) {
-                    split8_bf16(qw, hi, mid, lo);
+                    split8_f16(qw, sc, hi, lo);
                     *reinterpret_cast<uint4 *>(planesQw + off) = hi;
-                    *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = mid;
-                    *reinterpret_cast<uint4 *>(planesQw + off + 2 * 256 * 64) = lo;
+                    *reinterpret_cast<uint4 *>(planesQw + off + 256 * 64) = lo;
                 }
             } else {
 #pragma unroll
@@ -719,14 +736,17 @@ __global__ void __launch_bounds__(256, 2) sgemm_kernel(const GemmBatch g)
 }
 
 // ---------------------------------------------------------------- combine
+// tc_scale (tensor-core contraction only): the partials carry the two sides' powers of two, undone here.
 __global__ void combine_kernel(const float *partAB, int ksplit, const float *partC, int nsplit, long long mm,
-                               int nsk, float *S, float *R, float *T)
+                               int nsk, float *S, float *R, float *T, const float *tc_scale)
 {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= mm) return;
+    const float unscale = tc_scale ? 1.f / (tc_scale[0] * tc_scale[1]) : 1.f;        // a power of two: exact
     for (int q = 0; q < nsk; ++q) {
         float ab = partAB[(long long)q * mm + idx];
         for (int s = 1; s < ksplit; ++s) ab += partAB[((long long)s * 3 + q) * mm + idx];
+        ab *= unscale;
         float c = partC[(long long)q * mm + idx];
         for (int s = 1; s < nsplit; ++s) c += partC[((long long)s * 3 + q) * mm + idx];
         float *dst = q == 0 ? S : (q == 1 ? R : T);
@@ -804,7 +824,7 @@ size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool t
     b += align_up((size_t)m_b * pl.kpad * 4, 256) * 2;       // P, Pw
     b += align_up((size_t)pl.kpad * pl.npad * 4, 256) * 2;   // Q, Qw
     b += align_up((size_t)(pl.ksplit > tcks ? pl.ksplit : tcks) * 3 * mm * 4, 256);      // AB partials
-    if (tc) b += align_up(tc_planes_bytes(m_b, pl.kpad), 256) * 4 + 256;          // BF16 planes of P, Pw, Q^T, Qw^T; error word
+    if (tc) b += align_up(tc_planes_bytes(m_b, pl.kpad), 256) * 4 + 512;          // FP16 planes of P, Pw, Q^T, Qw^T; error word; scales
     b += align_up((size_t)pl.nsplit * 3 * mm * 4, 256);      // C partials
     return b;
 }
@@ -830,6 +850,8 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
     w.partAB = (float *)take((size_t)(w.pl.ksplit > w.tc_ksplit ? w.pl.ksplit : w.tc_ksplit) * 3 * mm * 4);
     for (int i = 0; i < 4; ++i) w.planes[i] = tc ? (unsigned char *)take(tc_planes_bytes(m_b, w.pl.kpad)) : nullptr;
     w.tc_err = tc ? (unsigned int *)take(256) : nullptr;
+    w.tc_scale = tc ? (float *)take(256) : nullptr;
+    w.d_maxab = nullptr;
     w.partC = (float *)take((size_t)w.pl.nsplit * 3 * mm * 4);
     return true;
 }
@@ -906,6 +928,14 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     if (rc != FPSK_OK) return rc;
     rc = build_hash_side(seed, rnd, 1, n3, m_b, w.h2, w.v2, w.colcount, w.colstart, w.colperm, sB, w.colpos);
     if (rc != FPSK_OK) return rc;
+    const float *scA = w.tc ? w.tc_scale : nullptr, *scB = w.tc ? w.tc_scale + 1 : nullptr;
+    if (w.tc) {
+        if (!w.d_maxab) return FPSK_ERR_PARAM;
+        rc = tc_scale_launch(w.rowcount, m_b, w.d_maxab, w.tc_scale, st);
+        if (rc != FPSK_OK) return rc;
+        rc = tc_scale_launch(w.colcount, m_b, w.d_maxab + 1, w.tc_scale + 1, sB);
+        if (rc != FPSK_OK) return rc;
+    }
     if (ax) {
         FPSK_CUDA_OK(cudaEventRecord(ax->ev[1], st));             // row side ready
         FPSK_CUDA_OK(cudaEventRecord(ax->ev[2], sB));             // column side ready
@@ -924,7 +954,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         const bool vec = (reinterpret_cast<uintptr_t>(in.A) & 15) == 0 && in.lda % 8 == 0 && n2 % 8 == 0;
         const int kcols = w.tc ? kblocks * 32 : pl.kpad;
         dim3 grid = w.tc ? dim3((kcols / 8 + 15) / 16, (m_b + 7) / 8) : dim3((kcols / 8 + 127) / 128, m_b);
-#define FPSK_CA(V, M, PL) compress_a_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw, kblocks, w.planes[0], w.planes[1], m_b)
+#define FPSK_CA(V, M, PL) compress_a_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw, kblocks, w.planes[0], w.planes[1], m_b, scA)
         if (w.tc) {
             if (vec) { if (mom) FPSK_CA(true, true, true); else FPSK_CA(true, false, true); }
             else     { if (mom) FPSK_CA(false, true, true); else FPSK_CA(false, false, true); }
@@ -940,7 +970,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         const int kcols = w.tc ? kblocks * 32 : pl.kpad;
         const int bmax = w.tc ? btiles * 256 : pl.npad;
         dim3 grid((kcols / 8 + 15) / 16, (bmax + 7) / 8);
-#define FPSK_CW(V, M, PL) compress_wt_kernel<T, V, M, PL><<<grid, 128, 0, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3])
+#define FPSK_CW(V, M, PL) compress_wt_kernel<T, V, M, PL><<<grid, 128, 0, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3], scB)
         if (w.tc) {
             if (vec) { if (mom) FPSK_CW(true, true, true); else FPSK_CW(true, false, true); }
             else     { if (mom) FPSK_CW(false, true, true); else FPSK_CW(false, false, true); }
@@ -958,7 +988,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     do {                                                                                                                         \
         FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b8_kernel<T, M, PL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
         compress_b8_kernel<T, M, PL><<<grid, 256, smem, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm,      \
-                                                              w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3]); \
+                                                              w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3], scB); \
     } while (0)
         if (w.tc) { if (mom) FPSK_CB8(true, true); else FPSK_CB8(false, true); }
         else      { if (mom) FPSK_CB8(true, false); else FPSK_CB8(false, false); }
@@ -978,10 +1008,10 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     }
     if (w.tc && !b8 && !in.bt) {
         // wide B: Q, Qw came out as FP32 rows; split them here (row b of Q^T is column b of Q)
-        rc = tc_split_launch(w.Q, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], sB);
+        rc = tc_split_launch(w.Q, scB, 1, pl.npad, m_b, pl.kpad, 1, w.planes[2], sB);
         if (rc != FPSK_OK) return rc;
         if (mom) {
-            rc = tc_split_launch(w.Qw, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], sB);
+            rc = tc_split_launch(w.Qw, scB, 1, pl.npad, m_b, pl.kpad, 1, w.planes[3], sB);
             if (rc != FPSK_OK) return rc;
         }
     }
@@ -1051,7 +1081,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     }
     {
         const long long mm = (long long)m_b * m_b;
-        combine_kernel<<<(unsigned)((mm + 255) / 256), 256, 0, st>>>(w.partAB, ab_splits, w.partC, pl.nsplit, mm, mom ? 3 : 1, S, R, Tt);
+        combine_kernel<<<(unsigned)((mm + 255) / 256), 256, 0, st>>>(w.partAB, ab_splits, w.partC, pl.nsplit, mm, mom ? 3 : 1, S, R, Tt, w.tc ? w.tc_scale : nullptr);
         FPSK_LAUNCH_CHECK();
     }
     return FPSK_OK;

@@ -44,8 +44,10 @@ struct SketchWs {
     float *P, *Pw, *Q, *Qw, *partAB, *partC;
     bool tc;                     // split-BF16 tensor-core contraction
     int tc_ksplit;
-    unsigned char *planes[4];    // P, Pw, Q^T, Qw^T as tiled BF16 planes
+    unsigned char *planes[4];    // P, Pw, Q^T, Qw^T as tiled FP16 planes (hi, lo)
     unsigned int *tc_err;        // set by the contraction when a wait gave up
+    float *tc_scale;             // [0], [1]: powers of two that bring P, Pw and Q, Qw into FP16 range (device)
+    const float *d_maxab;        // [0] max|A|, [1] max|B| (device; set by the caller before a tensor-core build)
 };
 
 struct SketchIn {
@@ -148,13 +150,27 @@ fpsk_status patch_launch(float *C, long long ldc, const PatchEntry *d_entries, i
 // bytes of the three tiled BF16 planes of a rows x kk FP32 matrix
 size_t tc_planes_bytes(int rows, int kk);
 // planes of X(r, k) = src[r * ldr + k * ldk], tiled for the A side (b_side = 0) or the B side (1) of the contraction
-fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, int b_side, unsigned char *planes,
+fpsk_status tc_split_launch(const float *src, const float *d_scale, long long ldr, long long ldk, int rows, int kk, int b_side, unsigned char *planes,
                             cudaStream_t st);
 // part[ks][prob] = A_selA[prob] (M x K) times B_selB[prob] (N x K) transposed, over the ks-th range of K
 fpsk_status tc_contract_launch(const unsigned char *const *planesA, const unsigned char *const *planesB, const int *selA,
                                const int *selB, int nprob, int pstride, float *part, int M, int N, int K, int ksplit,
                                unsigned int *d_err, cudaStream_t st);
 int tc_plan_ksplit(int M, int N, int K, int nprob, int sms);
+constexpr int kTcPlanes = 2;            // FP16 terms per FP32 value (hi, lo)
+// The power of two that brings the bucket sums of one side into FP16 range: |sum| <= (largest bucket) x max|X|
+// is scaled to at most 2^14 (FP16 reaches 65504).  Exact to undo; elements more than 2^16 below the largest
+// lose bits of their lo term, an absolute error below 2^-39 of the largest.
+__device__ __forceinline__ float tc_scale_of(int max_count, float max_abs)
+{
+    const float bound = (float)max_count * max_abs;
+    if (!(bound > 0.f && bound <= 3.0e38f)) return 1.f;
+    int e = 14 - (ilogbf(bound) + 1);                  // bound < 2^(ilogb + 1)
+    e = e > 100 ? 100 : (e < -100 ? -100 : e);
+    return ldexpf(1.f, e);
+}
+// scale[0] = tc_scale_of(max of count[0..m_b), maxv[0])   (all device)
+fpsk_status tc_scale_launch(const int *count, int m_b, const float *maxv, float *scale, cudaStream_t st);
 constexpr int kTcMinBuckets = 384;      // below this the FP32 FMA contraction is the faster one (measured)
 
 // ---- the S only probe with a cached B side (hprobe.cu) ------------------------------------------

@@ -2,18 +2,20 @@
 //
 // The sketches need S_AB = P Q (and the weighted forms) to FP32 accuracy: the sketch noise is the
 // measured quantity, and a single-pass reduced-precision product raises it by orders of magnitude
-// (Section "Implementation": TF32 raised the floor 419x).  An FP32 value is therefore split into
-// three BF16 terms x = hi + mid + lo (8 + 8 + 8 significand bits, each remainder exact in FP32), and
-// the product is formed from the six term pairs whose weight is above 2^-24:
-//   (hi,hi) (hi,mid) (mid,hi) (hi,lo) (lo,hi) (mid,mid),
-// every pair one BF16 tcgen05.mma with FP32 accumulation into the same TMEM accumulator.
+// (Section "Implementation": TF32 raised the floor 419x).  An FP32 value, scaled by a power of two
+// into FP16 range, is therefore split into two FP16 terms x = hi + lo (11 + 11 significand bits; the
+// remainder x - hi is exact in FP32, so hi + lo misses x by at most 2^-24 |x|), and the product is formed
+// from the three term pairs whose weight is above 2^-22:
+//   (lo,hi) (hi,lo) (hi,hi),
+// every pair one FP16 tcgen05.mma with FP32 accumulation into the same TMEM accumulator.  (Three BF16
+// terms need six pairs for the same accuracy: twice the tensor-core work.)
 //
-//   tc_split_kernel      FP32 matrix -> three BF16 planes, laid out tile by tile exactly as the
+//   tc_split_kernel      FP32 matrix -> two FP16 planes, laid out tile by tile exactly as the
 //                        tensor core reads shared memory (K-major, no swizzle: 8 x 16-byte core
-//                        matrices), so that the three planes of an operand tile are one contiguous block
+//                        matrices), so that the planes of an operand tile are one contiguous block
 //   tc_contract_kernel   one 128 x 256 output tile per CTA and K split: a producer warp brings the operand
 //                        tiles of a 32-deep K block with two bulk copies (mbarrier complete_tx), one
-//                        thread issues the 12 MMAs of the block and commits them to the stage's
+//                        thread issues the 6 MMAs of the block and commits them to the stage's
 //                        "empty" barrier, four warps read the accumulator back (tcgen05.ld) and
 //                        store the split-K partial.
 // Every wait is bounded; on expiry the CTA flags the error word, frees its TMEM and leaves.
@@ -25,24 +27,25 @@
 namespace fpsk {
 
 constexpr int kTcBM = 128, kTcBN = 256, kTcBK = 32;
-constexpr int kTcTileA = kTcBM * kTcBK * 2;              // one BF16 plane of an A tile (8 KB)
+constexpr int kTcTileA = kTcBM * kTcBK * 2;              // one FP16 plane of an A tile (8 KB)
 constexpr int kTcTileB = kTcBN * kTcBK * 2;              // of a B tile (16 KB)
-constexpr int kTcStageBytes = 3 * kTcTileA + 3 * kTcTileB;   // A hi, mid, lo; B hi, mid, lo (72 KB)
-constexpr int kTcStages = 3;
+constexpr int kTcStageBytes = kTcPlanes * kTcTileA + kTcPlanes * kTcTileB;   // A hi, lo; B hi, lo (48 KB)
+constexpr int kTcStages = 4;
 constexpr int kTcSmem = kTcStages * kTcStageBytes + 256;
 constexpr int kTcThreads = 192;                          // warps 0-3 epilogue, warp 4 producer, warp 5 MMA
 constexpr int kTcCols = 256;                             // TMEM columns of the accumulator
 static_assert(kTcBM * (kTcBN + 1) * 4 <= kTcStages * kTcStageBytes, "epilogue tile fits in the operand stages");
 
-// ---------------------------------------------------------------- FP32 -> three BF16 planes, tiled
-// X(r, k) = src[r * ldr + k * ldk] for r < rows, k < kk, else 0.  Tiles of R rows (128 for the A side, 256
-// for the B side) by 32 k.  Output: row tile rt, K block kb, plane p at ((rt * kblocks + kb) * 3 + p) * R * 64
-// bytes, so the three planes of an operand tile are one contiguous block (one bulk copy); inside a plane
+// ---------------------------------------------------------------- FP32 -> two FP16 planes, tiled
+// X(r, k) = scale * src[r * ldr + k * ldk] for r < rows, k < kk, else 0 (scale: a device scalar, a power of two).
+// Tiles of R rows (128 for the A side, 256 for the B side) by 32 k.  Output: row tile rt, K block kb, plane p at
+// ((rt * kblocks + kb) * 2 + p) * R * 64 bytes, so the planes of an operand tile are one contiguous block (one bulk copy); inside a plane
 // tile the 16-byte chunk (row r, k chunk kc) sits at (kc * (R / 8) + r / 8) * 128 + (r % 8) * 16.
 template <int R>
-__global__ void __launch_bounds__(256) tc_split_kernel(const float *src, long long ldr, long long ldk, int rows, int kk,
-                                                       int kblocks, unsigned char *planes)
+__global__ void __launch_bounds__(256) tc_split_kernel(const float *src, const float *d_scale, long long ldr, long long ldk,
+                                                       int rows, int kk, int kblocks, unsigned char *planes)
 {
+    const float scale = d_scale ? __ldg(d_scale) : 1.f;
     __shared__ float tile[R][kTcBK + 1];
     constexpr int kTile = R * kTcBK * 2;
     const int kb = blockIdx.x, rt = blockIdx.y;
@@ -61,21 +64,18 @@ __global__ void __launch_bounds__(256) tc_split_kernel(const float *src, long lo
         }
     }
     __syncthreads();
-    unsigned char *out = planes + ((size_t)rt * kblocks + kb) * 3 * kTile;
+    unsigned char *out = planes + ((size_t)rt * kblocks + kb) * kTcPlanes * kTile;
     for (int id = threadIdx.x; id < R * (kTcBK / 8); id += 256) {
         const int kc = id / R, r = id % R;
-        unsigned short h[8], m[8], l[8];
+        unsigned short h[8], l[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-            const float x = tile[r][kc * 8 + j];
-            const __nv_bfloat16 bh = __float2bfloat16_rn(x);
-            const float r1 = x - __bfloat162float(bh);           // exact
-            const __nv_bfloat16 bm = __float2bfloat16_rn(r1);
-            const float r2 = r1 - __bfloat162float(bm);          // exact
-            const __nv_bfloat16 bl = __float2bfloat16_rn(r2);
-            h[j] = __bfloat16_as_ushort(bh);
-            m[j] = __bfloat16_as_ushort(bm);
-            l[j] = __bfloat16_as_ushort(bl);
+            const float x = tile[r][kc * 8 + j] * scale;
+            const __half bh = __float2half_rn(x);
+            const float r1 = x - __half2float(bh);               // exact
+            const __half bl = __float2half_rn(r1);
+            h[j] = __half_as_ushort(bh);
+            l[j] = __half_as_ushort(bl);
         }
         const size_t off = (size_t)(kc * (R / 8) + r / 8) * 128 + (size_t)(r % 8) * 16;
         auto pack = [](const unsigned short *v) {
@@ -83,8 +83,7 @@ __global__ void __launch_bounds__(256) tc_split_kernel(const float *src, long lo
                               v[6] | ((unsigned)v[7] << 16));
         };
         *reinterpret_cast<uint4 *>(out + off) = pack(h);
-        *reinterpret_cast<uint4 *>(out + kTile + off) = pack(m);
-        *reinterpret_cast<uint4 *>(out + 2 * kTile + off) = pack(l);
+        *reinterpret_cast<uint4 *>(out + kTile + off) = pack(l);
     }
 }
 
@@ -104,7 +103,7 @@ __device__ __forceinline__ void tc_commit(uint32_t bar)
 {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-// D[tmem] (+)= A[smem desc] * B[smem desc]^T, BF16 operands, FP32 accumulate; 128 x 256 x 16
+// D[tmem] (+)= A[smem desc] * B[smem desc]^T, 16-bit operands (type in idesc), FP32 accumulate; 128 x 256 x 16
 __device__ __forceinline__ void tc_mma(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate)
 {
     asm volatile(
@@ -192,18 +191,19 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
             if (lane == 0) mbar_expect_tx(full0 + 8 * stage, kTcStageBytes);
             __syncwarp();
             if (lane < 2) {
-                // lane 0: the three planes of the A tile (24 KB), lane 1: of the B tile (48 KB)
-                const unsigned char *src = lane ? pb + ((size_t)nt * g.kblocks + kb) * 3 * kTcTileB
-                                                : pa + ((size_t)mt * g.kblocks + kb) * 3 * kTcTileA;
-                bulk_g2s(smem_u32(smem + (size_t)stage * kTcStageBytes + (size_t)lane * 3 * kTcTileA), src,
-                         lane ? 3 * kTcTileB : 3 * kTcTileA, full0 + 8 * stage);
+                // lane 0: the planes of the A tile (16 KB), lane 1: of the B tile (32 KB)
+                const unsigned char *src = lane ? pb + ((size_t)nt * g.kblocks + kb) * kTcPlanes * kTcTileB
+                                                : pa + ((size_t)mt * g.kblocks + kb) * kTcPlanes * kTcTileA;
+                bulk_g2s(smem_u32(smem + (size_t)stage * kTcStageBytes + (size_t)lane * kTcPlanes * kTcTileA), src,
+                         lane ? kTcPlanes * kTcTileB : kTcPlanes * kTcTileA, full0 + 8 * stage);
             }
             if (++stage == kTcStages) { stage = 0; phase ^= 1u; }
         }
     } else if (warp == 5) {
         // ------------------------------------------------------------ MMA issue (one thread)
-        // instruction descriptor: FP32 accumulator, BF16 x BF16, both K-major, N = 128, M = 128
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
+        // instruction descriptor: FP32 accumulator (bit 4), FP16 x FP16 (operand format fields 0), both K-major,
+        // N = 256, M = 128
+        const uint32_t idesc = (1u << 4) | ((uint32_t)(kTcBN >> 3) << 17) | ((uint32_t)(kTcBM >> 4) << 24);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -217,13 +217,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) tc_contract_kernel(const TcArgs
             if (lane == 0) {
                 const uint32_t sbase = smem_u32(smem + (size_t)stage * kTcStageBytes);
                 // term pairs (A plane, B plane), small weights first
-                const int pairA[6] = {2, 0, 1, 1, 0, 0}, pairB[6] = {0, 2, 1, 0, 1, 0};
+                const int pairA[3] = {1, 0, 0}, pairB[3] = {0, 1, 0};
 #pragma unroll
                 for (int kstep = 0; kstep < kTcBK / 16; ++kstep) {
 #pragma unroll
-                    for (int q = 0; q < 6; ++q) {
+                    for (int q = 0; q < 3; ++q) {
                         const uint32_t sa = sbase + pairA[q] * kTcTileA + kstep * 2 * (kTcBM / 8) * 128;
-                        const uint32_t sb = sbase + 3 * kTcTileA + pairB[q] * kTcTileB + kstep * 2 * (kTcBN / 8) * 128;
+                        const uint32_t sb = sbase + kTcPlanes * kTcTileA + pairB[q] * kTcTileB + kstep * 2 * (kTcBN / 8) * 128;
                         tc_mma(tmem, tc_smem_desc(sa, (kTcBM / 8) * 128, 128), tc_smem_desc(sb, (kTcBN / 8) * 128, 128), idesc, acc);
                         acc = 1;
                     }
@@ -287,15 +287,15 @@ size_t tc_planes_bytes(int rows, int kk)
 {
     // sized for either side: rows rounded up to the B side's 256
     const size_t rt = (size_t)(rows + kTcBN - 1) / kTcBN, kb = (size_t)(kk + kTcBK - 1) / kTcBK;
-    return 3 * rt * kb * kTcTileB;
+    return kTcPlanes * rt * kb * kTcTileB;
 }
 
-fpsk_status tc_split_launch(const float *src, long long ldr, long long ldk, int rows, int kk, int b_side, unsigned char *planes,
-                            cudaStream_t st)
+fpsk_status tc_split_launch(const float *src, const float *d_scale, long long ldr, long long ldk, int rows, int kk, int b_side,
+                            unsigned char *planes, cudaStream_t st)
 {
     const int kb = (kk + kTcBK - 1) / kTcBK;
-    if (b_side) tc_split_kernel<kTcBN><<<dim3(kb, (rows + kTcBN - 1) / kTcBN), 256, 0, st>>>(src, ldr, ldk, rows, kk, kb, planes);
-    else tc_split_kernel<kTcBM><<<dim3(kb, (rows + kTcBM - 1) / kTcBM), 256, 0, st>>>(src, ldr, ldk, rows, kk, kb, planes);
+    if (b_side) tc_split_kernel<kTcBN><<<dim3(kb, (rows + kTcBN - 1) / kTcBN), 256, 0, st>>>(src, d_scale, ldr, ldk, rows, kk, kb, planes);
+    else tc_split_kernel<kTcBM><<<dim3(kb, (rows + kTcBM - 1) / kTcBM), 256, 0, st>>>(src, d_scale, ldr, ldk, rows, kk, kb, planes);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }
