@@ -8,7 +8,7 @@
 
 namespace fpsk {
 
-constexpr int kConfirmThreads = 256;
+constexpr int kConfirmThreads = 1024;     // many k slices per window entry: the dot products are load latency
 
 // CTA (x: candidate, y: row offset d_i + r).  Thread (slice, d_j) accumulates every
 // `slices`-th k of column j_hat + d_j; slices are then summed in slice order.
@@ -36,7 +36,23 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
         // column j of B: strided in B, or row j of the transposed weight
         const unsigned short *bcol = bt ? B + j * ldb : B + j;
         const long long bstep = bt ? 1 : ldb;
-        for (long long k = ks; k < n2; k += slices) {
+        // eight loads of each operand in flight per thread; the sums run in ascending k of the slice
+        long long k = ks;
+        for (; k + 7 * (long long)slices < n2; k += 8 * (long long)slices) {
+            unsigned short av[8], bv[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                av[q] = arow[k + q * slices];
+                bv[q] = bcol[(k + q * slices) * bstep];
+            }
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                const double p = (double)bits16_to_float<T>(av[q]) * (double)bits16_to_float<T>(bv[q]);   // exact
+                g += p;
+                ab += fabs(p);
+            }
+        }
+        for (; k < n2; k += slices) {
             const double a = (double)bits16_to_float<T>(arow[k]);
             const double b = (double)bits16_to_float<T>(bcol[k * bstep]);
             const double p = a * b;          // exact: two <= 11-bit significands
