@@ -159,14 +159,14 @@ fpsk_status tc_contract_launch(const unsigned char *const *planesA, const unsign
 int tc_plan_ksplit(int M, int N, int K, int nprob, int sms);
 constexpr int kTcPlanes = 2;            // FP16 terms per FP32 value (hi, lo)
 // The power of two that brings the bucket sums of one side into FP16 range: |sum| <= (largest bucket) x max|X|
-// is scaled to at most 2^14 (FP16 reaches 65504).  Exact to undo; elements more than 2^16 below the largest
+// is scaled below 2^14 (FP16 reaches 65504).  Exact to undo; elements more than 2^16 below the largest
 // lose bits of their lo term, an absolute error below 2^-39 of the largest.
 __device__ __forceinline__ float tc_scale_of(int max_count, float max_abs)
 {
-    const float bound = (float)max_count * max_abs;
-    if (!(bound > 0.f && bound <= 3.0e38f)) return 1.f;
-    int e = 14 - (ilogbf(bound) + 1);                  // bound < 2^(ilogb + 1)
-    e = e > 100 ? 100 : (e < -100 ? -100 : e);
+    if (!(max_abs > 0.f && max_abs <= 3.4028234663852886e38f) || max_count < 1) return 1.f;
+    // max_abs < 2^(ilogb + 1), max_count < 2^(bits of max_count): exponents only, so nothing overflows here
+    int e = 14 - (ilogbf(max_abs) + 1 + (32 - __clz(max_count)));
+    e = e > 126 ? 126 : (e < -126 ? -126 : e);
     return ldexpf(1.f, e);
 }
 // scale[0] = tc_scale_of(max of count[0..m_b), maxv[0])   (all device)

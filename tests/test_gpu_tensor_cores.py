@@ -1,7 +1,8 @@
-"""The split-BF16 tensor-core contraction (tcgen05) behind `tensor_cores = 1`: same results as the FP32
+"""The split-FP16 tensor-core contraction (tcgen05) behind `tensor_cores = 1`: same results as the FP32
 FMA contraction within the 1e-5 tolerance, bit-exact on integer products, and a measured sketch noise
 that is not above the FMA path's (the gate for using it; Section "Implementation" warns that a
-single-pass reduced-precision product raised the floor 419x)."""
+single-pass reduced-precision product raised the floor 419x).  The bucket sums are scaled by a power of
+two into FP16 range before they are split, so operands of any magnitude must behave the same."""
 import numpy as np
 import pytest
 import torch
@@ -103,3 +104,48 @@ def test_small_bucket_counts_keep_the_fma_contraction():
         ws = fpsk.workspace(n, n, n, m_b, p)
         out.append(fpsk.measure_noise(dA, dB, dC, 5, ws, m_b, p))
     assert out[0].sigma_clip == out[1].sigma_clip and out[0].sigma_mad == out[1].sigma_mad
+
+
+@pytest.mark.parametrize("log2_scale_a,log2_scale_b", [(40, 0), (-40, 0), (60, -60), (-30, -30), (100, 10)])
+def test_operand_magnitude_does_not_matter(log2_scale_a, log2_scale_b):
+    """Powers of two on A and B only move exponents: the same faults are found, with deltas scaled exactly."""
+    n1, n2, n3, m_b = 1024, 768, 1280, 400
+    A, Bm = W.operands("gauss_scaled", n1, n2, n3, W.BF16, 12)
+    base = None
+    for sa, sb in ((0, 0), (log2_scale_a, log2_scale_b)):
+        As = (A.double() * 2.0 ** sa).to(torch.bfloat16)
+        Bs = (Bm.double() * 2.0 ** sb).to(torch.bfloat16)
+        Cm = harness.vendor_gemm_fp32(As.cuda(), Bs.cuda()).cpu()
+        faults = W.faults_additive(n1, n3, W.rms(Cm), 3, 4, 0.05, 0.09, "small")
+        Cf, _ = W.inject(Cm, faults)
+        p = fpsk.default_params(s_budget=4, radius=4, tensor_cores=1)
+        ws = fpsk.workspace(n1, n2, n3, m_b, p)
+        got = fpsk.localize(As.cuda(), Bs.cuda(), Cf.cuda(), 77, m_b, ws, p)
+        nz = fpsk.measure_noise(As.cuda(), Bs.cuda(), Cm.cuda(), 5, ws, m_b, p)
+        assert {(f.i, f.j) for f in got} == {(f.i, f.j) for f in faults}
+        rec = (sorted((f.i, f.j, f.delta * 2.0 ** -(sa + sb)) for f in got), nz.sigma_clip * 2.0 ** -(sa + sb))
+        if base is None:
+            base = rec
+        else:
+            # scaling by powers of two is exact in every step of the verifier (no over- or underflow here)
+            assert [(i, j) for i, j, _ in rec[0]] == [(i, j) for i, j, _ in base[0]]
+            for (_, _, d), (_, _, d0) in zip(rec[0], base[0]):
+                assert d == pytest.approx(d0, rel=1e-6)
+            assert rec[1] == pytest.approx(base[1], rel=1e-3)
+
+
+def test_all_zero_and_huge_operands_do_not_break_the_scaling():
+    n, m_b = 512, 384
+    A = torch.zeros(n, n, dtype=torch.bfloat16)
+    Bm = torch.zeros(n, n, dtype=torch.bfloat16)
+    Cm = torch.zeros(n, n, dtype=torch.float32)
+    p = fpsk.default_params(tensor_cores=1, radius=2)
+    ws = fpsk.workspace(n, n, n, m_b, p)
+    assert fpsk.localize(A.cuda(), Bm.cuda(), Cm.cuda(), 1, m_b, ws, p) == []
+    # the largest finite BF16 in A: the bound (largest bucket) x max|A| overflows FP32 -> scale 1, sums may overflow
+    # FP16 planes; the call must still return (nonfinite sketches select nothing that confirms)
+    A2, B2 = W.operands("gauss_scaled", n, n, n, W.BF16, 4)
+    A2[3, 5] = torch.finfo(torch.bfloat16).max
+    C2 = harness.vendor_gemm_fp32(A2.cuda(), B2.cuda())
+    got = fpsk.localize(A2.cuda(), B2.cuda(), C2, 1, m_b, ws, p)
+    assert isinstance(got, list)
