@@ -300,21 +300,34 @@ fpsk_status tc_split_launch(const float *src, const float *d_scale, long long ld
     return FPSK_OK;
 }
 
-// K splits: enough CTAs to fill the GPU, and no accumulation chain longer than kTcMaxChain K blocks.
-// The tensor core's FP32 accumulation is not round-to-nearest: measured on sketches of clean products,
-// chains of 1024 terms give the lowest noise (about a third below the FP32 FMA contraction), chains of
-// 8192 terms double it; shorter chains move the additions into the FP32 combine and approach its noise.
-constexpr int kTcMaxChain = 32;        // K blocks of 32: 1024 terms
+// K splits.  The tensor core's FP32 accumulation is not round-to-nearest: measured on sketches of clean
+// products, chains of 1024 terms give the lowest noise, 2048 terms 9 % more, 8192 terms 2.4 times as much;
+// shorter chains move the additions into the FP32 combine and approach its noise.  So no chain is longer than
+// kTcMaxChain K blocks, and among the splits that respect this the one with the least estimated time wins:
+// one CTA per SM, so the launch takes ceil(CTAs / SMs) rounds of (fixed cost + K blocks per CTA), the fixed
+// cost (set-up, TMEM allocation, epilogue) being worth about nine K blocks of six MMAs; every split also adds a
+// partial that the combine has to read.
+constexpr int kTcMaxChain = 32;        // K blocks of 32: 1024 terms (chains of 1376 terms: 5 us less per round at
+                                       // m = 1024, n2 = 4096, and a third more noise on a correctly rounded product)
+constexpr int kTcFixedCost = 9;        // in K blocks
 int tc_plan_ksplit(int M, int N, int K, int nprob, int sms)
 {
     const int tiles = ((M + kTcBM - 1) / kTcBM) * ((N + kTcBN - 1) / kTcBN) * nprob;
     const int kblocks = (K + kTcBK - 1) / kTcBK;
-    int s = sms / (tiles > 0 ? tiles : 1);
-    if (s < 1) s = 1;
-    if (s > kblocks) s = kblocks;
-    int per = (kblocks + s - 1) / s;
-    if (per > kTcMaxChain) per = kTcMaxChain;
-    return (kblocks + per - 1) / per;
+    if (sms < 1) sms = 1;
+    int best = 1;
+    long long best_cost = -1;
+    for (int s = 1; s <= kblocks && s <= 64; ++s) {
+        const int per = (kblocks + s - 1) / s;
+        if (per > kTcMaxChain) continue;
+        if ((kblocks + per - 1) / per != s) continue;          // the same chains with fewer, empty splits
+        const long long rounds = ((long long)tiles * s + sms - 1) / sms;
+        // plus what a further partial costs the combine that follows (about 2.4e-6 K-block times per output element)
+        const long long cost = 16 * rounds * (kTcFixedCost + per) + (long long)s * (1 + ((long long)M * N * nprob * 16) / 420000);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; best = s; }
+    }
+    if (best_cost < 0) best = (kblocks + kTcMaxChain - 1) / kTcMaxChain;     // more than 64 splits needed
+    return best;
 }
 
 // part[ks][prob] = A_sel(prob) B_sel(prob)^T over the ks-th range of K blocks.  planesA[i] holds an M x K
