@@ -149,3 +149,58 @@ def test_all_zero_and_huge_operands_do_not_break_the_scaling():
     C2 = harness.vendor_gemm_fp32(A2.cuda(), B2.cuda())
     got = fpsk.localize(A2.cuda(), B2.cuda(), C2, 1, m_b, ws, p)
     assert isinstance(got, list)
+
+
+@pytest.mark.parametrize("tc", [0, 1])
+def test_more_keys_than_one_pass_of_the_select_kernel_holds(tc):
+    """1200^2 = 1.44 M buckets: the radix selects take their keys in more than one batch per digit."""
+    n1, n2, n3, m_b = 4800, 128, 4800, 1200
+    A, Bm = W.operands("gauss_scaled", n1, n2, n3, W.BF16, 8)
+    Cm = harness.vendor_gemm_fp32(A.cuda(), Bm.cuda()).cpu()
+    faults = W.faults_additive(n1, n3, W.rms(Cm), 6, 5, 0.05, 0.09, "small")
+    Cf, _ = W.inject(Cm, faults)
+    A64, B64 = _f64(A), _f64(Bm)
+    ref = O.localize(A64, B64, Cf.numpy(), 31, m_b, W.BF16, O.Params(s_budget=5, radius=3))
+    rmap = {(f.i, f.j): f.delta for f in ref}
+    p = fpsk.default_params(s_budget=5, radius=3, tensor_cores=tc)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    got = fpsk.localize(A.cuda(), Bm.cuda(), Cf.cuda(), 31, m_b, ws, p)
+    assert {(f.i, f.j) for f in got} == set(rmap) == {(f.i, f.j) for f in faults}
+    for f in got:
+        a = np.abs(A64[f.i, :]) @ np.abs(B64[:, f.j])
+        assert abs(f.delta - rmap[(f.i, f.j)]) <= TOL * a
+    if tc == 0:
+        # the estimates against the definitions applied to the very sketch they were taken from (FP32, as the kernels
+        # compute them): lower medians by exact selection, so equality is bit for bit
+        S, _, _ = fpsk.sketches(A.cuda(), Bm.cuda(), Cm.cuda(), 5, 0, m_b, ws, moments=False)
+        a = np.abs(S.cpu().numpy().ravel())
+        rank = (a.size - 1) // 2
+        med = np.partition(a, rank)[rank]
+        dev = np.abs(a - med)
+        mad = np.float32(1.4826) * np.partition(dev, rank)[rank]
+        mean = np.float32(a.astype(np.float64).sum() / a.size)
+        nz = fpsk.measure_noise(A.cuda(), Bm.cuda(), Cm.cuda(), 5, ws, m_b, p)
+        assert np.float32(nz.sigma_mad) == mad
+        clip = np.float32(1.2533) * np.float32(np.minimum(a, np.float32(5) * mean).astype(np.float64).sum() / a.size)
+        assert nz.sigma_clip == pytest.approx(float(clip), rel=1e-5)
+
+
+@pytest.mark.parametrize("m_b,mad_of_abs", [(300, 1), (300, 0), (1024, 1), (1024, 0), (17, 1)])
+def test_sigma_mad_is_the_exact_selection_on_the_sketch(m_b, mad_of_abs):
+    """sigma_MAD of `fpsk_measure_noise` = 1.4826 x lower median of the deviations from the lower median, bit for
+    bit, on the sketch the same kernels produce (FMA contraction, so that `fpsk_sketches` gives that sketch)."""
+    n = 1536
+    A, Bm = W.operands("gauss_scaled", n, n, n, W.FP16, 41)
+    dA, dB = A.cuda(), Bm.cuda()
+    dC = harness.vendor_gemm_fp32(dA, dB)
+    p = fpsk.default_params(tensor_cores=0, mad_of_abs=mad_of_abs)
+    ws = fpsk.workspace(n, n, n, m_b, p)
+    S, _, _ = fpsk.sketches(dA, dB, dC, 9, 0, m_b, ws, moments=False)
+    x = S.cpu().numpy().ravel()
+    a = np.abs(x) if mad_of_abs else x
+    rank = (a.size - 1) // 2
+    med = np.partition(a, rank)[rank]
+    dev = np.abs(a - med)
+    mad = np.float32(1.4826) * np.partition(dev, rank)[rank]
+    nz = fpsk.measure_noise(dA, dB, dC, 9, ws, m_b, p)
+    assert np.float32(nz.sigma_mad) == mad
