@@ -5,10 +5,13 @@
 //
 //   hash_kernel / scan_kernel / place_kernel   hash tables and bucket-sorted permutations
 //   compress_a_kernel   P = H1 A, Pw = H1 W1 A          (m_b x n2, rows grouped by bucket)
-//   compress_b_kernel   Q = B H2^T, Qw = B W2 H2^T      (n2 x m_b, one row of B per pass)
-//   sgemm_kernel        S_AB = P Q, R_AB = Pw Q, T_AB = P Qw   (FP32 SIMT, split-K partials)
-//   scatter_c_kernel    S_C, R_C, T_C: one streaming pass over C per round (row sums in registers, one fold per chunk)
+//   compress_b_kernel / compress_b8_kernel (B as k x n) / compress_wt_kernel (the weight W = B^T)
+//                       Q = B H2^T, Qw = B W2 H2^T      (n2 x m_b)
+//   sgemm_kernel        S_AB = P Q, R_AB = Pw Q, T_AB = P Qw   (FP32 SIMT, split-K partials); with the tensor-core
+//                       contraction (tc_contract.cu) the compressions write scaled FP16 planes instead of P, Q
+//   scatter_c_kernel / scatter_c2_kernel   S_C, R_C, T_C: one streaming pass over C per round
 //   combine_kernel      S = sum of AB partials - sum of C partials
+// The column side + B compression and the C scatter run on auxiliary streams when the caller provides them.
 #include "sketch.cuh"
 
 #include <mutex>
