@@ -14,13 +14,13 @@
  *   - The caller owns every buffer.  The library allocates no device memory and never writes
  *     to A or B; C is written only by fpsk_verify_repair and fpsk_apply_corrections (paper,
  *     Section "Overview": localization does not modify C; Algorithm 2, "Apply").
- *     fpsk_localize and fpsk_verify_repair create one CUDA event for the duration of the call and
- *     stage each round's results through a small pinned host buffer (about 25 KB).  They and
- *     fpsk_measure_noise run independent parts of a sketch build on two auxiliary non-blocking
- *     streams, tied to `stream` by events on both sides (work queued on `stream` before the call
- *     is complete before any of it starts; everything is complete when the call returns).  The
- *     buffer, the two streams and their five events are created on first use, one set per
- *     concurrent call and device, and kept for the life of the process.
+ *     fpsk_localize and fpsk_verify_repair create one CUDA event for the duration of the call.  They and
+ *     fpsk_measure_noise read their results back through a small pinned host buffer (about 25 KB) and run
+ *     independent parts of a sketch build on two auxiliary non-blocking streams, tied to `stream` by
+ *     events on both sides (work queued on `stream` before the call is complete before any of it
+ *     starts; everything is complete when the call returns).  The buffer, the two streams and their
+ *     five events are created on first use, one set per concurrent call and device, and kept for the
+ *     life of the process.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Indices are 0-based.  The 1-based index weights of the paper are internal.
  *   - Errors are return codes.  Nothing throws, aborts or resets the device.  After

@@ -79,7 +79,7 @@ static fpsk_status pinned_acquire(PinnedLease &l)
             return FPSK_OK;
         }
     }
-    FPSK_CUDA_OK(cudaHostAlloc(&l.p, kPackBytes, cudaHostAllocDefault));
+    FPSK_CUDA_OK(cudaHostAlloc(&l.p, kPackBytes, cudaHostAllocPortable));
     return FPSK_OK;
 }
 
@@ -229,6 +229,25 @@ static fpsk_status loc_max_ab(const SketchIn &in, fpsk_dtype dtype, LocWs &w, cu
     return FPSK_OK;
 }
 
+// The scalars of a noise measurement (the select's eight scalars, rms(C), the select's error word) to the host
+// through pinned staging: three small asynchronous copies and one wait (a pageable destination blocks per copy).
+static fpsk_status read_noise_scalars(const LocWs &w, cudaStream_t st, float (&h_scal)[8], float &h_rms)
+{
+    PinnedLease stage;
+    fpsk_status rc = pinned_acquire(stage);
+    if (rc != FPSK_OK) return rc;
+    char *h = static_cast<char *>(stage.p);
+    FPSK_CUDA_OK(cudaMemcpyAsync(h, w.sel.scal, 32, cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaMemcpyAsync(h + 32, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaMemcpyAsync(h + 36, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
+    FPSK_CUDA_OK(cudaStreamSynchronize(st));
+    memcpy(h_scal, h, 32);
+    memcpy(&h_rms, h + 32, 4);
+    unsigned int err = 0;
+    memcpy(&err, h + 36, 4);
+    return err ? FPSK_ERR_TIMEOUT : FPSK_OK;
+}
+
 __global__ void tau_kernel(float *misc, float n2)
 {
     if (threadIdx.x == 0) misc[2] = 100.f * n2 * 1.1920928955078125e-07f * misc[0] * misc[1];
@@ -271,12 +290,8 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
         rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, in.C, in.ldc, m, n, w.samples, w.sel, w.misc + 3, st);
         if (rc != FPSK_OK) return rc;
         float h_scal[8], h_rms = 0.f;
-        FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
-        unsigned int h_sel_err = 0;
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaStreamSynchronize(st));
-        if (h_sel_err) return FPSK_ERR_TIMEOUT;
+        rc = read_noise_scalars(w, st, h_scal, h_rms);
+        if (rc != FPSK_OK) return rc;
         double sig = h_scal[1], rms = h_rms;
         if (!(std::isfinite(sig) && sig > 0 && std::isfinite(rms) && rms > 0)) {
             sig = law_sigma((double)m, (double)k, (double)n, dtype, 1.0, (double)m_b);
@@ -696,13 +711,9 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
     if (rc != FPSK_OK) return rc;
     float h_scal[8];
-    FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
     float h_rms = 0.f;
-    FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
-    unsigned int h_sel_err = 0;
-    FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
-    FPSK_CUDA_OK(cudaStreamSynchronize(st));
-    if (h_sel_err) return FPSK_ERR_TIMEOUT;
+    rc = read_noise_scalars(w, st, h_scal, h_rms);
+    if (rc != FPSK_OK) return rc;
 
     fpsk_noise out;
     memset(&out, 0, sizeof(out));
@@ -902,12 +913,8 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
         rc = sigma_mad_rms_c_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);
         if (rc != FPSK_OK) return rc;
         float h_scal[8], h_rms = 0.f;
-        FPSK_CUDA_OK(cudaMemcpyAsync(h_scal, w0.sel.scal, sizeof(h_scal), cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_rms, w0.misc + 3, 4, cudaMemcpyDeviceToHost, st));
-        unsigned int h_sel_err = 0;
-        FPSK_CUDA_OK(cudaMemcpyAsync(&h_sel_err, w0.sel.err, 4, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaStreamSynchronize(st));
-        if (h_sel_err) return FPSK_ERR_TIMEOUT;
+        rc = read_noise_scalars(w0, st, h_scal, h_rms);
+        if (rc != FPSK_OK) return rc;
         int r;
         double B_;
         plan_of(m, k, n, dtype, h_scal[1], h_rms, m0, q, m_loc, r, B_);
