@@ -180,9 +180,11 @@ struct LocWs {
     Hit *hits;
     int *n_hits;
     unsigned char *pack;      // kPackBytes: a round's results in one piece
+    unsigned short *Wt;       // room for W = B^T (n3 x ldw) when B comes as k x n, else null
+    long long ldw;
 };
 
-static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool tc = false)
+static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool tc = false, bool wt = false)
 {
     const size_t mm = (size_t)m_b * m_b;
     size_t b = sketch_ws_bytes(n1, n2, n3, m_b, tc);
@@ -194,12 +196,14 @@ static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bo
     b += align_up(sizeof(Hit) * kHitCap, 256);
     b += 256;
     b += align_up(kPackBytes, 256);
+    if (wt) b += align_up((size_t)n3 * (size_t)((n2 + 7) & ~7LL) * 2, 256);
     return b;
 }
 
-static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, LocWs &w, bool tc = false)
+static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long long n3, int m_b, LocWs &w, bool tc = false,
+                      bool wt = false)
 {
-    if (ws_bytes < loc_ws_bytes(n1, n2, n3, m_b, tc)) return false;
+    if (ws_bytes < loc_ws_bytes(n1, n2, n3, m_b, tc, wt)) return false;
     const size_t mm = (size_t)m_b * m_b;
     const size_t skb = sketch_ws_bytes(n1, n2, n3, m_b, tc);
     if (!sketch_carve(ws, skb, n1, n2, n3, m_b, w.sk, tc)) return false;
@@ -213,6 +217,8 @@ static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, lon
     w.hits = (Hit *)take(sizeof(Hit) * kHitCap);
     w.n_hits = (int *)take(256);
     w.pack = (unsigned char *)take(kPackBytes);
+    w.ldw = (n2 + 7) & ~7LL;
+    w.Wt = wt ? (unsigned short *)take((size_t)n3 * (size_t)w.ldw * 2) : nullptr;
     return true;
 }
 
@@ -263,9 +269,10 @@ static int offset_rank_key(int di, int dj, int r)
 // The localize part of Algorithm 2: p.rounds rounds of Algorithm 1 at m_b buckets, carrying F.
 // Entries already in F with round < 0 are absolute repairs (Section "Nonfinite"): they count as
 // found but are not peeled, their error is already absent from the sketches.
-static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int m_b, const fpsk_params &q, LocWs &w,
+static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, uint64_t seed, int m_b, const fpsk_params &q, LocWs &w,
                                  cudaStream_t st, std::vector<fpsk_fault> &F, bool &truncated, int &radius_used)
 {
+    SketchIn in = in_caller;
     const long long m = in.n1, k = in.n2, n = in.n3;
     const long long mm = (long long)m_b * m_b;
     const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
@@ -279,6 +286,15 @@ static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t 
     if (rc != FPSK_OK) return rc;
     tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
     FPSK_LAUNCH_CHECK();
+    if (!in.bt && w.Wt) {
+        // B as k x n: transpose it once and let every round read rows of W = B^T (the B compression sums rows
+        // instead of gathering columns, the confirmation reads a row instead of a strided column; same bits)
+        rc = transpose_b_launch(in.B, in.ldb, k, n, w.Wt, w.ldw, st);
+        if (rc != FPSK_OK) return rc;
+        in.B = w.Wt;
+        in.ldb = w.ldw;
+        in.bt = 1;
+    }
 
     int radius = q.radius;
     bool round0_built = false;
@@ -657,7 +673,7 @@ size_t fpsk_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, 
     // n_buckets <= 0: size for the law's starting count of either operand type
     if (n_buckets <= 0) n_buckets = std::max(m_start_of(m, k, n, FPSK_FP16, q), m_start_of(m, k, n, FPSK_BF16, q));
     if (n_buckets > sketch_max_buckets(m, k, n)) return 0;
-    return loc_ws_bytes(m, k, n, n_buckets, q.tensor_cores != 0);
+    return loc_ws_bytes(m, k, n, n_buckets, q.tensor_cores != 0, !q.b_transposed);
 }
 
 fpsk_status fpsk_sketches(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
@@ -755,7 +771,7 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
     if (!params_ok(q)) return FPSK_ERR_PARAM;
     if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     LocWs w;
-    if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
+    if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w, q.tensor_cores != 0, !q.b_transposed)) return FPSK_ERR_WORKSPACE;
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
     *h_count = 0;
     std::vector<fpsk_fault> F;
@@ -786,7 +802,7 @@ size_t fpsk_repair_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_bu
         mb = std::min(mb, sketch_max_buckets(m, k, n));
     }
     if (mb < 1 || mb > sketch_max_buckets(m, k, n)) return 0;
-    return align_up(probe_ws_bytes(m, k, n), 256) + align_up(loc_ws_bytes(m, k, n, mb, q.tensor_cores != 0), 256) +
+    return align_up(probe_ws_bytes(m, k, n), 256) + align_up(loc_ws_bytes(m, k, n, mb, q.tensor_cores != 0, true), 256) +
            align_up(repair_scratch_bytes(), 256) + 256;
 }
 
@@ -922,7 +938,7 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
         if (qq.radius < 0) qq.radius = r;
     }
     LocWs w;
-    if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
+    if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w, q.tensor_cores != 0, true)) return FPSK_ERR_WORKSPACE;
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
     bool truncated = false;
     int radius_used = 0;

@@ -11,7 +11,9 @@ namespace fpsk {
 constexpr int kConfirmThreads = 1024;     // many k slices per window entry: the dot products are load latency
 
 // CTA (x: candidate, y: row offset d_i + r).  Thread (slice, d_j) accumulates every
-// `slices`-th k of column j_hat + d_j; slices are then summed in slice order.
+// `slices`-th k of column j_hat + d_j; slices are then summed in slice order.  Adjacent lanes take adjacent
+// columns when B is k x n (a row of B is contiguous in j) and adjacent slices when B comes as W = B^T (a row of W
+// is contiguous in k).
 template <typename T>
 __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
     const unsigned short *A, long long lda, const unsigned short *B, long long ldb, const float *C, long long ldc,
@@ -27,9 +29,10 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
     const long long i = (long long)cand[u].ih + di;
     if (i < 0 || i >= n1) return;
     const int slices = kConfirmThreads / W;
-    const int dj = threadIdx.x % W, ks = threadIdx.x / W;
+    const int dj = bt ? (int)threadIdx.x / slices : (int)threadIdx.x % W;
+    const int ks = bt ? (int)threadIdx.x % slices : (int)threadIdx.x / W;
     const long long j = (long long)cand[u].jh - r + dj;
-    const bool active = ks < slices && j >= 0 && j < n3;
+    const bool active = ks < slices && dj < W && j >= 0 && j < n3;
     double g = 0.0, ab = 0.0;
     if (active) {
         const unsigned short *arow = A + i * lda;
@@ -60,8 +63,10 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
             ab += fabs(p);
         }
     }
-    sg[threadIdx.x] = g;
-    sa[threadIdx.x] = ab;
+    if (ks < slices && dj < W) {
+        sg[ks * W + dj] = g;
+        sa[ks * W + dj] = ab;
+    }
     __syncthreads();
     if (active && ks == 0) {
         for (int s = 1; s < slices; ++s) {

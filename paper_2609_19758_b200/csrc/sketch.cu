@@ -870,6 +870,63 @@ int sketch_max_buckets(long long n1, long long n2, long long n3)
     return (int)m;
 }
 
+// ---------------------------------------------------------------- B -> W = B^T (16-bit elements)
+// 64 x 64 tiles through shared memory.  VEC (16-byte aligned rows on both sides, n2 and n3 multiples of 8): a thread
+// reads 8 consecutive columns of a row of B with one load and writes 8 consecutive k of a row of W with one store.
+template <bool VEC>
+__global__ void __launch_bounds__(256) transpose16_kernel(const unsigned short *B, long long ldb, int n2, int n3,
+                                                          unsigned short *W, long long ldw)
+{
+    __shared__ __align__(16) unsigned short tile[64][66];      // row pitch 33 words: rows 8 apart fall into different banks
+    const int k0 = blockIdx.y * 64, j0 = blockIdx.x * 64;
+    if (VEC) {
+        for (int e = threadIdx.x; e < 64 * 8; e += 256) {
+            const int r = e >> 3, c8 = (e & 7) * 8;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (k0 + r < n2 && j0 + c8 < n3) v = ldg_nc_v4(B + (long long)(k0 + r) * ldb + j0 + c8);
+            uint32_t *dst = reinterpret_cast<uint32_t *>(&tile[r][c8]);
+            dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < 64 * 8; e += 256) {
+            const int r8 = (e & 7) * 8, c = e >> 3;            // eight consecutive lanes write 128 contiguous bytes of a row of W
+            if (j0 + c >= n3 || k0 + r8 >= n2) continue;
+            unsigned short x[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) x[t] = tile[r8 + t][c];
+            *reinterpret_cast<uint4 *>(W + (long long)(j0 + c) * ldw + k0 + r8) =
+                make_uint4(x[0] | ((unsigned)x[1] << 16), x[2] | ((unsigned)x[3] << 16), x[4] | ((unsigned)x[5] << 16),
+                           x[6] | ((unsigned)x[7] << 16));
+        }
+    } else {
+        for (int e = threadIdx.x; e < 64 * 64; e += 256) {
+            const int r = e >> 6, c = e & 63;                  // a warp reads 32 consecutive columns of one row of B
+            tile[r][c] = (k0 + r < n2 && j0 + c < n3) ? B[(long long)(k0 + r) * ldb + j0 + c] : (unsigned short)0;
+        }
+        __syncthreads();
+        for (int e = threadIdx.x; e < 64 * 64; e += 256) {
+            const int c = e >> 6, r = e & 63;                  // ... and writes 32 consecutive k of one row of W
+            if (j0 + c < n3 && k0 + r < n2) W[(long long)(j0 + c) * ldw + k0 + r] = tile[r][c];
+        }
+    }
+}
+
+fpsk_status transpose_b_launch(const void *B, long long ldb, long long n2, long long n3, void *W, long long ldw,
+                               cudaStream_t st)
+{
+    dim3 grid((unsigned)((n3 + 63) / 64), (unsigned)((n2 + 63) / 64));
+    const bool vec = ((reinterpret_cast<uintptr_t>(B) | reinterpret_cast<uintptr_t>(W)) & 15) == 0 && ldb % 8 == 0 &&
+                     ldw % 8 == 0 && n2 % 8 == 0 && n3 % 8 == 0;
+    if (vec)
+        transpose16_kernel<true><<<grid, 256, 0, st>>>(static_cast<const unsigned short *>(B), ldb, (int)n2, (int)n3,
+                                                       static_cast<unsigned short *>(W), ldw);
+    else
+        transpose16_kernel<false><<<grid, 256, 0, st>>>(static_cast<const unsigned short *>(B), ldb, (int)n2, (int)n3,
+                                                        static_cast<unsigned short *>(W), ldw);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
 // ---------------------------------------------------------------- auxiliary streams
 struct SketchAuxPool {
     std::mutex mu;

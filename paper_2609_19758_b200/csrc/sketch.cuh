@@ -64,6 +64,9 @@ int sketch_max_buckets(long long n1, long long n2, long long n3);
 
 fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, int *bucket, int *sign,
                             int *count, int *start, uint32_t *perm, cudaStream_t st, uint32_t *pos = nullptr);
+// W = B^T for 16-bit elements: W[j * ldw + k] = B[k * ldb + j], k < n2, j < n3 (ldw >= n2)
+fpsk_status transpose_b_launch(const void *B, long long ldb, long long n2, long long n3, void *W, long long ldw,
+                               cudaStream_t st);
 fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
                            SketchWs &w, cudaStream_t st, float *S, float *R, float *T);
 // start[0..n] = exclusive prefix sums of count[0..n)  (one CTA, any n)
