@@ -137,34 +137,48 @@ struct SelChain {
 };
 constexpr int kChainSteps = 8;                 // digits of the longest key (64 bits)
 
-// inclusive scan of the 256 counts (one per thread) -> the bin whose running count passes k, and the
-// number of keys below it; the same values in every thread
-__device__ __forceinline__ void pick_digit(unsigned int h, unsigned long long k, unsigned long long *wsum, int *s_bin,
-                                           unsigned long long *s_before, int &bin, unsigned long long &before_out)
+// For both select slots at once: inclusive scan of the 256 counts (thread t < 256 holds bin t) -> the bin whose
+// running count passes k, and the number of keys below it; the same values in every thread of the CTA.  The first
+// eight warps work among themselves (named barrier); the other warps only join the closing barrier.
+__device__ __forceinline__ void pick_digits(const unsigned int (&h)[2], const unsigned long long (&k)[2], const bool (&on)[2],
+                                            unsigned long long (*wsum)[8], int *s_bin, unsigned long long *s_before,
+                                            int (&bin)[2], unsigned long long (&before_out)[2])
 {
-    unsigned long long inc = h;
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    if (threadIdx.x < 256) {
+        unsigned long long inc[2] = {h[0], h[1]};
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, inc, o);
-        if (lane >= o) inc += v;
+        for (int o = 1; o < 32; o <<= 1) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                const unsigned long long v = __shfl_up_sync(0xFFFFFFFFu, inc[j], o);
+                if (lane >= o) inc[j] += v;
+            }
+        }
+        if (lane == 31) { wsum[0][wid] = inc[0]; wsum[1][wid] = inc[1]; }
+        if (threadIdx.x < 2) { s_bin[threadIdx.x] = 255; s_before[threadIdx.x] = 0; }
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (!on[j]) continue;
+            unsigned long long base = 0, total = 0;
+            for (int w = 0; w < 8; ++w) {
+                const unsigned long long v = wsum[j][w];
+                if (w < wid) base += v;
+                total += v;
+            }
+            const unsigned long long incl = inc[j] + base;          // keys in bins 0 .. threadIdx.x
+            const unsigned long long before = incl - h[j];          // keys in bins below this one
+            if (before <= k[j] && k[j] < incl) { s_bin[j] = (int)threadIdx.x; s_before[j] = before; }     // exactly one thread, when k < total
+            if (threadIdx.x == 255 && k[j] >= total) { s_bin[j] = 255; s_before[j] = total; }              // k beyond the keys (not reached: k is clamped to the count)
+        }
     }
-    __syncthreads();                               // earlier readers of wsum, s_bin are done
-    if (lane == 31 && wid < 8) wsum[wid] = inc;    // threads beyond the 256 bins come along with h = 0
-    if (threadIdx.x == 0) { *s_bin = 255; *s_before = 0; }
     __syncthreads();
-    unsigned long long base = 0;
-    for (int w = 0; w < wid && w < 8; ++w) base += wsum[w];
-    inc += base;                                   // keys in bins 0 .. threadIdx.x
-    const unsigned long long before = inc - h;     // keys in bins below this one
-    unsigned long long total = 0;
-    for (int w = 0; w < 8; ++w) total += wsum[w];
-    __syncthreads();
-    if (before <= k && k < inc) { *s_bin = threadIdx.x; *s_before = before; }        // exactly one thread, when k < total
-    if (threadIdx.x == 255 && k >= total) { *s_bin = 255; *s_before = total; }       // k beyond the keys (not reached: k is clamped to the count)
-    __syncthreads();
-    bin = *s_bin;
-    before_out = *s_before;
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        bin[j] = s_bin[j];
+        before_out[j] = s_before[j];
+    }
 }
 
 __device__ __forceinline__ float median_value(int mode, unsigned long long key)
@@ -185,13 +199,53 @@ __device__ __forceinline__ uint32_t key_base(int mode, float x, float med)
     }
 }
 
+// One digit of one select over the kSelItems elements of this thread (keys in shared memory): lanes with equal
+// bins are combined and the lowest lane of a group counts for it, keeping its last two bins in registers.
+// LOW: the digit lies in the lower half of a 64-bit K-largest key (~element index) and the upper half must match.
+template <bool LOW, bool CACHE>
+__device__ __forceinline__ void bin_items(const uint32_t (*kbj)[kSelThreads], uint32_t ibase, uint32_t n32, bool sample,
+                                          uint32_t pre_hi, uint32_t pre_lo, uint32_t fixed, int sh32, unsigned int *shj,
+                                          unsigned int (&cbin)[2], unsigned int (&ccnt)[2])
+{
+    const int tid = (int)threadIdx.x;
+#pragma unroll 2
+    for (int u = 0; u < kSelItems; ++u) {
+        const uint32_t i32 = ibase + (uint32_t)(u * kSelThreads);
+        const uint32_t kbu = kbj[u][tid];
+        bool valid = i32 < n32 && !(sample && kbu == 0xFFFFFFFFu);
+        uint32_t word;
+        if (LOW) {
+            word = 0xFFFFFFFFu - i32;
+            valid = valid && kbu == pre_hi && ((word ^ pre_lo) & fixed) == 0u;
+        } else {
+            word = kbu;
+            valid = valid && ((word ^ pre_hi) & fixed) == 0u;
+        }
+        const unsigned int vmask = __ballot_sync(0xFFFFFFFFu, valid);
+        if (vmask == 0u) continue;                             // late digits: hardly any key still carries the prefix
+        const unsigned int bin = (word >> sh32) & 255u;
+        const unsigned int peers = __match_any_sync(0xFFFFFFFFu, valid ? bin : 256u);
+        if (valid && (tid & 31) == __ffs(peers) - 1) {
+            const unsigned int cnt = (unsigned)__popc(peers);
+            if (!CACHE) atomicAdd(&shj[bin], cnt);
+            else if (bin == cbin[0]) ccnt[0] += cnt;
+            else if (bin == cbin[1]) ccnt[1] += cnt;
+            else {
+                if (ccnt[1]) atomicAdd(&shj[cbin[1]], ccnt[1]);
+                cbin[1] = cbin[0]; ccnt[1] = ccnt[0];
+                cbin[0] = bin; ccnt[0] = cnt;
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain ch, float *scal, unsigned long long *state,
                                                               unsigned int *hist, const int *counts)
 {
     __shared__ unsigned int sh[2][256];
-    __shared__ unsigned long long wsum[8];
-    __shared__ int s_bin, s_ok;
-    __shared__ unsigned long long s_before;
+    __shared__ unsigned long long wsum[2][8];
+    __shared__ int s_bin[2], s_ok;
+    __shared__ unsigned long long s_before[2];
     const int G = (int)gridDim.x, tid = (int)threadIdx.x;
     SelJob job[2] = {ch.a, ch.b};
     bool on[2] = {true, ch.have_b != 0};
@@ -271,36 +325,12 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
                 const int sh32 = low_half ? shift : (wide ? shift - 32 : shift);
                 // bits of the 32-bit word in play that are already fixed by earlier digits
                 const uint32_t fixed = sh32 + 8 >= 32 ? 0u : (0xFFFFFFFFu << (sh32 + 8));
-#pragma unroll 2
-                for (int u = 0; u < kSelItems; ++u) {
-                    const long long i = base + u * kSelThreads + tid;
-                    const uint32_t kbu = kb[j][u][tid];
-                    bool valid = i < job[j].n && !(sample && kbu == 0xFFFFFFFFu);
-                    uint32_t word;
-                    if (low_half) {
-                        valid = valid && kbu == pre_hi;
-                        word = 0xFFFFFFFFu - (uint32_t)i;
-                        valid = valid && ((word ^ pre_lo) & fixed) == 0u;
-                    } else {
-                        word = kbu;
-                        valid = valid && ((word ^ pre_hi) & fixed) == 0u;
-                    }
-                    const unsigned int vmask = __ballot_sync(0xFFFFFFFFu, valid);
-                    if (vmask == 0u) continue;                             // late digits: hardly any key still carries the prefix
-                    const unsigned int bin = (word >> sh32) & 255u;
-                    const unsigned int peers = __match_any_sync(0xFFFFFFFFu, valid ? bin : 256u);
-                    // the lowest lane of a group counts for the group; it keeps its last two bins in registers
-                    if (valid && (tid & 31) == __ffs(peers) - 1) {
-                        const unsigned int cnt = (unsigned)__popc(peers);
-                        if (bin == cbin[j][0]) ccnt[j][0] += cnt;
-                        else if (bin == cbin[j][1]) ccnt[j][1] += cnt;
-                        else {
-                            if (ccnt[j][1]) atomicAdd(&sh[j][cbin[j][1]], ccnt[j][1]);
-                            cbin[j][1] = cbin[j][0]; ccnt[j][1] = ccnt[j][0];
-                            cbin[j][0] = bin; ccnt[j][0] = cnt;
-                        }
-                    }
-                }
+                const uint32_t ibase = (uint32_t)base + (uint32_t)tid;      // element indices fit 32 bits (<= 2^24 buckets)
+                // the register cache pays on a select's leading digit (one or two bins take nearly every key);
+                // later digits spread over the bins or have few keys left
+                if (low_half) bin_items<true, false>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j], cbin[j], ccnt[j]);
+                else if (shift == job[j].nbits - 8) bin_items<false, true>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j], cbin[j], ccnt[j]);
+                else bin_items<false, false>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j], cbin[j], ccnt[j]);
             }
         }
 #pragma unroll
@@ -334,14 +364,17 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
             for (int r = 0; r < kHistCopies; ++r)
                 if (tid < 256) hsum[j] += __ldcg(&hstep[(j * kHistCopies + r) * 256 + tid]);
         }
+        int dbin[2];
+        unsigned long long dbefore[2];
+        {
+            const bool on_now[2] = {on[0], on[1]};
+            pick_digits(hsum, k, on_now, wsum, s_bin, s_before, dbin, dbefore);
+        }
 #pragma unroll
         for (int j = 0; j < 2; ++j) {
             if (!on[j]) continue;
-            int bin;
-            unsigned long long before;
-            pick_digit(hsum[j], k[j], wsum, &s_bin, &s_before, bin, before);
-            k[j] -= before;
-            prefix[j] |= (unsigned long long)bin << job[j].shift;
+            k[j] -= dbefore[j];
+            prefix[j] |= (unsigned long long)dbin[j] << job[j].shift;
             job[j].shift -= 8;
             // K-largest key: once the rank inside the remaining ties is 0, the lower digits cannot move the
             // cut (every key of the tie is at or above "upper half, zeros"), so they are left at zero
