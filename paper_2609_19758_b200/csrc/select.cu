@@ -83,7 +83,7 @@ __global__ void count_valid_kernel(int mode, const float *S, long long mm, const
 }
 
 constexpr int kSelThreads = 1024; // one CTA per SM
-constexpr int kSelItems = 8;      // elements per thread and batch (their keys stay in shared memory over the digits when one
+constexpr int kSelItems = 8;      // elements per thread and batch (their keys stay in registers over the digits when one
                                   // batch covers the source)
 
 // One radix select in flight: its source, key kind, digit position.  Up to two run in one launch (slot 0, 1).
@@ -126,8 +126,8 @@ __device__ __forceinline__ void select_result(int mode, unsigned long long key, 
 // share the source; c may take its deviations from b's result, which every CTA derives for itself).  A
 // digit is: every CTA bins its keys in shared memory and adds the 256 counts to one of the copies of this
 // digit's histogram; a grid-wide arrival counter (bounded wait); every CTA sums the copies and finds the
-// bin of the k-th key by the same scan.  One CTA of 1024 threads per SM.  Measured at 10^6 keys: 8 us per
-// digit (binning 2-5, arrival wait 2, copies + scan 1.5-2), against 9.5 us for a launch per digit with a
+// bin of the k-th key by the same scan.  One CTA of 1024 threads per SM.  Measured at 10^6 keys: 5 us per
+// digit (binning 1-2, arrival wait 2, copies + scan 1), against 9.5 us for a launch per digit with a
 // last-CTA scan and the select state in global memory; the K-largest key needs only its upper four digits
 // when the K-th value is unique, and the median of the samples of C and the two medians of the MAD ride in
 // the same launches, so a localization round runs 8 digits in one launch instead of 16 launches.
@@ -199,19 +199,19 @@ __device__ __forceinline__ uint32_t key_base(int mode, float x, float med)
     }
 }
 
-// One digit of one select over the kSelItems elements of this thread (keys in shared memory): lanes with equal
-// bins are combined and the lowest lane of a group counts for it, keeping its last two bins in registers.
+// One digit of one select over the kSelItems elements of this thread (keys in registers): every lane whose
+// key still carries the prefix adds one to its bin in shared memory.  Plain atomics: lanes of a warp that hit the
+// same address cost no more than lanes that spread (measured on sketches of exact zeros), and combining equal bins
+// first (match.any, a register cache of the last bins) only added instructions: 67 us per round against 43.
 // LOW: the digit lies in the lower half of a 64-bit K-largest key (~element index) and the upper half must match.
-template <bool LOW, bool CACHE>
-__device__ __forceinline__ void bin_items(const uint32_t (*kbj)[kSelThreads], uint32_t ibase, uint32_t n32, bool sample,
-                                          uint32_t pre_hi, uint32_t pre_lo, uint32_t fixed, int sh32, unsigned int *shj,
-                                          unsigned int (&cbin)[2], unsigned int (&ccnt)[2])
+template <bool LOW>
+__device__ __forceinline__ void bin_items(const uint32_t (&kbj)[kSelItems], uint32_t ibase, uint32_t n32, bool sample,
+                                          uint32_t pre_hi, uint32_t pre_lo, uint32_t fixed, int sh32, unsigned int *shj)
 {
-    const int tid = (int)threadIdx.x;
-#pragma unroll 2
+#pragma unroll
     for (int u = 0; u < kSelItems; ++u) {
         const uint32_t i32 = ibase + (uint32_t)(u * kSelThreads);
-        const uint32_t kbu = kbj[u][tid];
+        const uint32_t kbu = kbj[u];
         bool valid = i32 < n32 && !(sample && kbu == 0xFFFFFFFFu);
         uint32_t word;
         if (LOW) {
@@ -221,21 +221,7 @@ __device__ __forceinline__ void bin_items(const uint32_t (*kbj)[kSelThreads], ui
             word = kbu;
             valid = valid && ((word ^ pre_hi) & fixed) == 0u;
         }
-        const unsigned int vmask = __ballot_sync(0xFFFFFFFFu, valid);
-        if (vmask == 0u) continue;                             // late digits: hardly any key still carries the prefix
-        const unsigned int bin = (word >> sh32) & 255u;
-        const unsigned int peers = __match_any_sync(0xFFFFFFFFu, valid ? bin : 256u);
-        if (valid && (tid & 31) == __ffs(peers) - 1) {
-            const unsigned int cnt = (unsigned)__popc(peers);
-            if (!CACHE) atomicAdd(&shj[bin], cnt);
-            else if (bin == cbin[0]) ccnt[0] += cnt;
-            else if (bin == cbin[1]) ccnt[1] += cnt;
-            else {
-                if (ccnt[1]) atomicAdd(&shj[cbin[1]], ccnt[1]);
-                cbin[1] = cbin[0]; ccnt[1] = ccnt[0];
-                cbin[0] = bin; ccnt[0] = cnt;
-            }
-        }
+        if (valid) atomicAdd(&shj[(word >> sh32) & 255u], 1u);
     }
 }
 
@@ -277,10 +263,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
     if (ch.have_b && ch.b.n > nall) nall = ch.b.n;
     if (ch.have_c && ch.c.n > nall) nall = ch.c.n;
     // When one batch covers the sources a thread derives the keys of its elements once per select and keeps
-    // them (in shared memory) over the digits; otherwise it derives them again digit by digit.
+    // them (in registers) over the digits; otherwise it derives them again digit by digit.
     const bool one_batch = nall <= per_grid;
-    extern __shared__ uint32_t kb_all[];           // [job][item][thread]
-    uint32_t (*kb)[kSelItems][kSelThreads] = reinterpret_cast<uint32_t (*)[kSelItems][kSelThreads]>(kb_all);
+    uint32_t kb[2][kSelItems];                     // the keys of this thread's elements, in registers
     bool fresh[2] = {true, true};
     for (int step = 0; step < nsteps; ++step) {
         if (tid < 256) {
@@ -292,16 +277,11 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
 #pragma unroll
         for (int j = 0; j < 2; ++j)
             if (on[j] && job[j].n > nmax) nmax = job[j].n;
-        // Leading digits put nearly all keys into one or two bins: a lane that counts for a group keeps its last
-        // two bins in registers and adds them to shared memory when they change or the digit ends.
-        unsigned int cbin[2][2] = {{256u, 256u}, {256u, 256u}}, ccnt[2][2] = {{0u, 0u}, {0u, 0u}};
-        // All of a thread's loads are issued before it bins anything (the warp-wide votes keep the compiler
-        // from moving loads across them).
         for (long long base = (long long)blockIdx.x * (kSelThreads * kSelItems); base < nmax; base += per_grid) {
 #pragma unroll
             for (int j = 0; j < 2; ++j) {
                 if (!on[j] || !(fresh[j] || !one_batch)) continue;
-#pragma unroll 1
+#pragma unroll
                 for (int u0 = 0; u0 < kSelItems; u0 += 8) {
                     float x[8];
 #pragma unroll
@@ -310,7 +290,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
                         x[u] = i < job[j].n ? __ldg(job[j].src + i) : 0.f;
                     }
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) kb[j][u0 + u][tid] = key_base(job[j].mode, x[u], med);
+                    for (int u = 0; u < 8; ++u) kb[j][u0 + u] = key_base(job[j].mode, x[u], med);
                 }
             }
 #pragma unroll
@@ -326,18 +306,9 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
                 // bits of the 32-bit word in play that are already fixed by earlier digits
                 const uint32_t fixed = sh32 + 8 >= 32 ? 0u : (0xFFFFFFFFu << (sh32 + 8));
                 const uint32_t ibase = (uint32_t)base + (uint32_t)tid;      // element indices fit 32 bits (<= 2^24 buckets)
-                // the register cache pays on a select's leading digit (one or two bins take nearly every key);
-                // later digits spread over the bins or have few keys left
-                if (low_half) bin_items<true, false>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j], cbin[j], ccnt[j]);
-                else if (shift == job[j].nbits - 8) bin_items<false, true>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j], cbin[j], ccnt[j]);
-                else bin_items<false, false>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j], cbin[j], ccnt[j]);
+                if (low_half) bin_items<true>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j]);
+                else bin_items<false>(kb[j], ibase, (uint32_t)job[j].n, sample, pre_hi, pre_lo, fixed, sh32, sh[j]);
             }
-        }
-#pragma unroll
-        for (int j = 0; j < 2; ++j) {
-#pragma unroll
-            for (int e = 0; e < 2; ++e)
-                if (ccnt[j][e]) atomicAdd(&sh[j][cbin[j][e]], ccnt[j][e]);
         }
         fresh[0] = false;
         fresh[1] = false;
@@ -411,8 +382,6 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
     }
 }
 
-constexpr size_t kSelSmem = (size_t)2 * kSelItems * kSelThreads * 4;
-
 static int select_capacity()
 {
     static int cap = 0;            // co-resident CTAs of the cooperative select kernel on this device
@@ -420,8 +389,7 @@ static int select_capacity()
         int dev = 0, sms = 0, occ = 0;
         if (cudaGetDevice(&dev) != cudaSuccess) return 148;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) return 148;
-        if (cudaFuncSetAttribute(select_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSelSmem) != cudaSuccess) return sms;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, select_chain_kernel, kSelThreads, kSelSmem) != cudaSuccess || occ < 1) return sms;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&occ, select_chain_kernel, kSelThreads, 0) != cudaSuccess || occ < 1) return sms;
         cap = sms;
     }
     return cap;
@@ -457,7 +425,7 @@ static fpsk_status run_selects(SelJob a, SelJob b, bool have_b, SelJob c, bool h
     unsigned int *hist = w.hist;
     const int *counts = w.counts;
     void *args[] = {(void *)&ch, (void *)&scal, (void *)&state, (void *)&hist, (void *)&counts};
-    FPSK_CUDA_OK(cudaLaunchCooperativeKernel((const void *)select_chain_kernel, dim3(grid), dim3(kSelThreads), args, kSelSmem, st));
+    FPSK_CUDA_OK(cudaLaunchCooperativeKernel((const void *)select_chain_kernel, dim3(grid), dim3(kSelThreads), args, 0, st));
     count_launch();
     return FPSK_OK;
 }
