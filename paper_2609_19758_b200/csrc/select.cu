@@ -526,10 +526,13 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
     if (n > cap) n = cap;
     sk[t] = t < n ? keys[t] : 0ull;
     __syncthreads();
-    for (int k = 2; k <= kSelMaxK; k <<= 1) {
+    // the network only has to cover the keys that are there (a power of two; zeros fill the rest)
+    int np2 = 2;
+    while (np2 < n) np2 <<= 1;
+    for (int k = 2; k <= np2; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
             const int ixj = t ^ j;
-            if (ixj > t) {
+            if (ixj > t && ixj < np2) {
                 const bool desc = (t & k) == 0;
                 const unsigned long long a = sk[t], b = sk[ixj];
                 if (desc ? (a < b) : (a > b)) { sk[t] = b; sk[ixj] = a; }
@@ -557,14 +560,14 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
     flag[t] = keep;
     __syncthreads();
     // inclusive scan of the keep flags (order-preserving compaction)
-    for (int o = 1; o < kSelMaxK; o <<= 1) {
+    for (int o = 1; o < np2; o <<= 1) {
         const int v = t >= o ? flag[t - o] : 0;
         __syncthreads();
         flag[t] += v;
         __syncthreads();
     }
     if (keep) cand[flag[t] - 1] = c;
-    if (t == kSelMaxK - 1) counts[2] = flag[t];
+    if (t == np2 - 1) counts[2] = flag[t];
 }
 
 fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
