@@ -719,13 +719,29 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
         rc = loc_max_ab(in, dtype, w, st);
         if (rc != FPSK_OK) return rc;
     }
+    // The samples of C need nothing from the sketch: they are taken on the stream that will run the C scatter, ahead of
+    // the build (which joins that stream before its combine).  The clipped mean and the selects both only read S:
+    // the two sums run on the other auxiliary stream beside the select launch.
+    SketchAux *ax = (aux.aux && aux.aux->s1 && aux.aux->s2 && aux.aux->ev[4]) ? aux.aux : nullptr;
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));             // whatever the caller queued before this call (the GEMM, say)
+        FPSK_CUDA_OK(cudaStreamWaitEvent(ax->s2, ax->ev[0], 0));
+    }
+    const long long nsamp = rms_c_samples(C, ldc, m, n, w.samples, w.sel, ax ? ax->s2 : st);
+    if (nsamp < 0) return FPSK_ERR_CUDA;
     rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
     if (rc != FPSK_OK) return rc;
     const long long mm = (long long)m0 * m0;
-    rc = sigma_clip_launch(w.S, mm, w.sel, st);
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));
+        FPSK_CUDA_OK(cudaStreamWaitEvent(ax->s1, ax->ev[0], 0));
+    }
+    rc = sigma_clip_launch(w.S, mm, w.sel, ax ? ax->s1 : st);
     if (rc != FPSK_OK) return rc;
-    rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, C, ldc, m, n, w.samples, w.sel, w.misc + 3, st);
+    if (ax) FPSK_CUDA_OK(cudaEventRecord(ax->ev[1], ax->s1));
+    rc = sigma_mad_rms_c_select_launch(w.S, mm, q.mad_of_abs, w.samples, nsamp, w.sel, w.misc + 3, st);
     if (rc != FPSK_OK) return rc;
+    if (ax) FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->ev[1], 0));
     float h_scal[8];
     float h_rms = 0.f;
     rc = read_noise_scalars(w, st, h_scal, h_rms);

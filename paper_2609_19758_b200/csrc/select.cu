@@ -711,8 +711,10 @@ __global__ void __launch_bounds__(1024) clipped_rms_kernel(const float *samples,
     }
 }
 
-static long long rms_c_samples(const float *C, long long ldc, long long n1, long long n3, float *samples, SelectWs &w,
-                               cudaStream_t st)
+// Strided samples of |C| (-1 marks Inf / NaN) and the number of valid ones -> counts[0]; returns the sample count
+// (< 0: a launch failed).
+long long rms_c_samples(const float *C, long long ldc, long long n1, long long n3, float *samples, SelectWs &w,
+                        cudaStream_t st)
 {
     const long long total = n1 * n3;
     long long stride = total / 65536;
@@ -734,6 +736,13 @@ fpsk_status sigma_mad_rms_c_launch(const float *S, long long mm, int mad_of_abs,
 {
     const long long nsamp = rms_c_samples(C, ldc, n1, n3, samples, w, st);
     if (nsamp < 0) return FPSK_ERR_CUDA;
+    return sigma_mad_rms_c_select_launch(S, mm, mad_of_abs, samples, nsamp, w, out, st);
+}
+
+// The second half of the above, for a caller that took the samples earlier (on another stream, joined since).
+fpsk_status sigma_mad_rms_c_select_launch(const float *S, long long mm, int mad_of_abs, float *samples, long long nsamp,
+                                          SelectWs &w, float *out, cudaStream_t st)
+{
     const SelJob med = sel_job(mad_of_abs ? SEL_ABS : SEL_SIGNED, 32, S, mm, 0);
     const SelJob dev = sel_job(mad_of_abs ? SEL_DEV_ABS : SEL_DEV_SIGNED, 32, S, mm, 0);
     const SelJob smp = sel_job(SEL_SAMPLE, 32, samples, nsamp, 0);

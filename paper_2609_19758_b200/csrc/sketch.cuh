@@ -115,6 +115,10 @@ fpsk_status max_abs_half_launch(const void *X, long long ld, long long rows, lon
                                 float *out, unsigned int *scratch, cudaStream_t st);
 // sigma_MAD of S (mad_of_abs: of |S| as printed, else signed) -> scal[1], median -> scal[0]; and the strided,
 // clipped rms of C (Section "Calibration") -> out[0]; the three medians share one launch
+long long rms_c_samples(const float *C, long long ldc, long long n1, long long n3, float *samples, SelectWs &w,
+                        cudaStream_t st);          // the samples alone (count -> w.counts[0]); returns how many, < 0 on a launch error
+fpsk_status sigma_mad_rms_c_select_launch(const float *S, long long mm, int mad_of_abs, float *samples, long long nsamp,
+                                          SelectWs &w, float *out, cudaStream_t st);      // the selects and the rms on samples taken before
 fpsk_status sigma_mad_rms_c_launch(const float *S, long long mm, int mad_of_abs, const float *C, long long ldc,
                                    long long n1, long long n3, float *samples, SelectWs &w, float *out, cudaStream_t st);
 
