@@ -294,7 +294,10 @@ fpsk_status fpsk_probe_recalibrate(int64_t m, int64_t n, double sigma_bar, doubl
 fpsk_status fpsk_hash_tables(uint64_t seed, int32_t round, int32_t side, int64_t count,
                              int32_t n_buckets, int32_t *d_bucket, int32_t *d_sign, void *stream);
 
-/* Bytes of device workspace for fpsk_sketches / fpsk_measure_noise / fpsk_localize. */
+/* Bytes of device workspace for fpsk_sketches / fpsk_measure_noise / fpsk_localize with these parameters
+ * (0 for a bad shape, bad parameters or a bucket count out of range).  Covers, with tensor_cores = 1 and at least
+ * 384 buckets, the FP16 planes of the compressed operands, and, with b_transposed = 0, room for W = B^T
+ * (n x k rounded up to 8, 16-bit): fpsk_localize transposes B into it once per call and runs its rounds on W. */
 size_t fpsk_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, const fpsk_params *p);
 
 /* Largest bucket count the kernels accept for this shape (shared-memory limits). */
