@@ -410,7 +410,9 @@ static fpsk_status run_selects(SelJob a, SelJob b, bool have_b, SelJob c, bool h
     const int steps = da > db + dc ? da : db + dc;
     if (steps > kChainSteps || (have_c && !have_b)) return FPSK_ERR_PARAM;
     if (!w.hist_clean) {
-        FPSK_CUDA_OK(cudaMemsetAsync(w.hist + kHistErr, 0, 64 * sizeof(unsigned int), st));      // sticky error word, sum ticket
+        // the sticky error word only: the ticket next to it belongs to the clipped-mean sums, which may be running
+        // on another stream at this moment
+        FPSK_CUDA_OK(cudaMemsetAsync(w.hist + kHistErr, 0, sizeof(unsigned int), st));
         w.hist_clean = true;
     }
     FPSK_CUDA_OK(cudaMemsetAsync(w.hist, 0, (size_t)(kHistBase + steps * 2 * kHistCopies * 256) * sizeof(unsigned int), st));
