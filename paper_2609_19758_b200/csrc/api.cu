@@ -300,7 +300,7 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
     bool round0_built = false;
     if (radius < 0) {
         // no calibration handed in: sigma_MAD of the first round's S and the strided rms of C
-        rc = build_sketches(in, dtype, seed, 0, m_b, true, w.sk, st, w.S, w.R, w.T);
+        rc = build_sketches(in, dtype, seed, 0, m_b, false, w.sk, st, w.S, nullptr, nullptr);
         if (rc != FPSK_OK) return rc;
         round0_built = true;
         rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, in.C, in.ldc, m, n, w.samples, w.sel, w.misc + 3, st);
@@ -331,24 +331,32 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
         ~EventGuard() { if (e) cudaEventDestroy(e); }
     } round_done;
     FPSK_CUDA_OK(cudaEventCreateWithFlags(&round_done.e, cudaEventDisableTiming));
+    // Only S is built whole.  The first moments R, T are read at the K buckets the selection keeps and nowhere else
+    // (Eq. (recover)), so they are computed for those buckets alone once the keys are collected: a third of the
+    // contraction, of the combine and of the plane writes.
     bool built_ahead = false;
     for (int t = 0; t < q.rounds; ++t) {
         if (!(t == 0 && round0_built) && !built_ahead) {
-            rc = build_sketches(in, dtype, seed, t, m_b, true, w.sk, st, w.S, w.R, w.T);
+            rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
             if (rc != FPSK_OK) return rc;
         }
         built_ahead = false;
+        int np = 0;
         if (!peel.empty()) {
-            const int np = (int)std::min<size_t>(peel.size(), kPeelCap);
+            np = (int)std::min<size_t>(peel.size(), kPeelCap);
             if ((int)peel.size() > kPeelCap) truncated = true;
             FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, st));
-            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, w.R, w.T, st);
+            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, nullptr, nullptr, st);
             if (rc != FPSK_OK) return rc;
         }
         // sigma_MAD of this round's S rides in the launches of the K-largest selection (round 0's is already
         // there when it was needed for the radius)
         const int mad_mode = (t == 0 && round0_built) ? -1 : (q.mad_of_abs ? 1 : 0);
-        rc = select_candidates_launch(w.S, w.R, w.T, m_b, m, n, w.misc + 2, radius, K, mad_mode, w.sel, st);
+        rc = select_collect_launch(w.S, m_b, m, n, w.misc + 2, radius, K, mad_mode, w.sel, st);
+        if (rc != FPSK_OK) return rc;
+        rc = candidate_moments_launch(in, dtype, w.sk, m_b, K, w.sel, w.peel, np, seed, t, st);
+        if (rc != FPSK_OK) return rc;
+        rc = decode_launch(w.S, nullptr, nullptr, w.sel.Rc, w.sel.Tc, m, n, w.sel, st);
         if (rc != FPSK_OK) return rc;
         rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, st);
         if (rc != FPSK_OK) return rc;
@@ -358,7 +366,7 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
         FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, pack_bytes, cudaMemcpyDeviceToHost, st));
         FPSK_CUDA_OK(cudaEventRecord(round_done.e, st));
         if (t + 1 < q.rounds) {
-            rc = build_sketches(in, dtype, seed, t + 1, m_b, true, w.sk, st, w.S, w.R, w.T);
+            rc = build_sketches(in, dtype, seed, t + 1, m_b, false, w.sk, st, w.S, nullptr, nullptr);
             if (rc != FPSK_OK) return rc;
             built_ahead = true;
         }

@@ -87,6 +87,162 @@ __global__ void __launch_bounds__(kConfirmThreads) confirm_kernel(
     }
 }
 
+// ---------------------------------------------------------------- first moments of the candidate buckets only
+// Only the K buckets that the selection keeps ever have their R and T read (Eq. (recover)), so the two weighted
+// sketches are not built whole: for a kept bucket (a, b)
+//   R = sum_k Pw[a,k] Q[k,b] - sum_{i in a, j in b} v1 v2 w_i C_ij,    T = sum_k P[a,k] Qw[k,b] - sum v1 v2 w_j C_ij,
+// with the compressed rows and columns formed on the fly from the bucket's rows of A and columns of B (same FP32
+// order as the compressions), the products accumulated in FP64, and the peeled faults of the bucket subtracted.
+// One CTA per collected key.
+constexpr int kMomThreads = 1024;         // few CTAs do any work (one per kept bucket): wide ones
+template <typename T>
+__global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
+    const unsigned short *A, long long lda, const unsigned short *B, long long ldb, int bt, const float *C, long long ldc,
+    int n2, int m_b, float inv_p1, float inv_p3, const uint32_t *rowperm, const int *rowstart, const uint32_t *colperm,
+    const int *colstart, const unsigned long long *keys, const int *counts, int cap, const PeelEntry *peel, int n_peel,
+    uint32_t key1, uint32_t key2, float *Rc, float *Tc, int vec)
+{
+    __shared__ double sr[kMomThreads], st_[kMomThreads];
+    const int slot = blockIdx.x;
+    int n = counts[1];
+    if (n > cap) n = cap;
+    if (slot >= n) return;
+    const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(keys[slot] & 0xFFFFFFFFull);
+    const int a = (int)(idx / (uint32_t)m_b), b = (int)(idx % (uint32_t)m_b);
+    const int r0 = rowstart[a], r1 = rowstart[a + 1], c0 = colstart[b], c1 = colstart[b + 1];
+    double accR = 0.0, accT = 0.0;
+    if (vec) {
+        // eight consecutive k per thread, four rows (columns) of the bucket in flight: the walk is load latency
+        for (int k0 = threadIdx.x * 8; k0 < n2; k0 += kMomThreads * 8) {
+            float p[8] = {0, 0, 0, 0, 0, 0, 0, 0}, pw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+            float q[8] = {0, 0, 0, 0, 0, 0, 0, 0}, qw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+#pragma unroll
+            for (int side = 0; side < 2; ++side) {
+                const uint32_t *perm = side ? colperm : rowperm;
+                const unsigned short *X = side ? B : A;
+                const long long ld = side ? ldb : lda;
+                const float inv_p = side ? inv_p3 : inv_p1;
+                const int b0 = side ? c0 : r0, b1 = side ? c1 : r1;
+                for (int sb = b0; sb < b1; sb += 4) {
+                    uint32_t e4[4];
+                    uint4 v4[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) e4[u] = sb + u < b1 ? __ldg(perm + sb + u) : 0u;
+#pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        v4[u] = sb + u < b1 ? ldg_nc_v4(X + (long long)(e4[u] & 0x7FFFFFFFu) * ld + k0) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        if (sb + u >= b1) break;
+                        const int i = (int)(e4[u] & 0x7FFFFFFFu);
+                        const float sg = (e4[u] >> 31) ? -1.f : 1.f;
+                        const float sw = sg * ((float)(i + 1) * inv_p);
+                        const unsigned int ww[4] = {v4[u].x, v4[u].y, v4[u].z, v4[u].w};
+#pragma unroll
+                        for (int t = 0; t < 4; ++t) {
+                            const float2 f = HalfTraits<T>::unpack2(ww[t]);
+                            if (side == 0) {
+                                p[2 * t] += sg * f.x; p[2 * t + 1] += sg * f.y;
+                                pw[2 * t] = fmaf(sw, f.x, pw[2 * t]); pw[2 * t + 1] = fmaf(sw, f.y, pw[2 * t + 1]);
+                            } else {
+                                q[2 * t] += sg * f.x; q[2 * t + 1] += sg * f.y;
+                                qw[2 * t] = fmaf(sw, f.x, qw[2 * t]); qw[2 * t + 1] = fmaf(sw, f.y, qw[2 * t + 1]);
+                            }
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int t = 0; t < 8; ++t) {
+                accR += (double)pw[t] * (double)q[t];
+                accT += (double)p[t] * (double)qw[t];
+            }
+        }
+    } else {
+        for (int k = threadIdx.x; k < n2; k += kMomThreads) {
+            float p = 0.f, pw = 0.f, q = 0.f, qw = 0.f;
+            for (int s = r0; s < r1; ++s) {
+                const uint32_t e = __ldg(rowperm + s);
+                const int i = (int)(e & 0x7FFFFFFFu);
+                const float sg = (e >> 31) ? -1.f : 1.f;
+                const float x = bits16_to_float<T>(A[(long long)i * lda + k]);
+                p += sg * x;
+                pw = fmaf(sg * ((float)(i + 1) * inv_p1), x, pw);
+            }
+            for (int s = c0; s < c1; ++s) {
+                const uint32_t e = __ldg(colperm + s);
+                const int j = (int)(e & 0x7FFFFFFFu);
+                const float sg = (e >> 31) ? -1.f : 1.f;
+                const float y = bits16_to_float<T>(bt ? B[(long long)j * ldb + k] : B[(long long)k * ldb + j]);
+                q += sg * y;
+                qw = fmaf(sg * ((float)(j + 1) * inv_p3), y, qw);
+            }
+            accR += (double)pw * (double)q;
+            accT += (double)p * (double)qw;
+        }
+    }
+    // the bucket's entries of C, one (row, column) pair per thread and step
+    const int nr = r1 - r0, nc = c1 - c0;
+    for (int e = threadIdx.x; e < nr * nc; e += kMomThreads) {
+        const uint32_t er = __ldg(rowperm + r0 + e / nc), ec = __ldg(colperm + c0 + e % nc);
+        const int i = (int)(er & 0x7FFFFFFFu), j = (int)(ec & 0x7FFFFFFFu);
+        const double v = ((er >> 31) != (ec >> 31)) ? -1.0 : 1.0;
+        const double c = (double)C[(long long)i * ldc + j];
+        accR -= v * (double)((float)(i + 1) * inv_p1) * c;
+        accT -= v * (double)((float)(j + 1) * inv_p3) * c;
+    }
+    sr[threadIdx.x] = accR;
+    st_[threadIdx.x] = accT;
+    __syncthreads();
+    for (int s = kMomThreads / 2; s > 0; s >>= 1) {
+        if ((int)threadIdx.x < s) { sr[threadIdx.x] += sr[threadIdx.x + s]; st_[threadIdx.x] += st_[threadIdx.x + s]; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        double R = sr[0], Tm = st_[0];
+        // faults confirmed in earlier rounds that hash into this bucket (Algorithm 1, peeling)
+        for (int f = 0; f < n_peel; ++f) {
+            int a2, b2, s1, s2;
+            hash_index(key1, (uint32_t)peel[f].i, (uint32_t)m_b, a2, s1);
+            if (a2 != a) continue;
+            hash_index(key2, (uint32_t)peel[f].j, (uint32_t)m_b, b2, s2);
+            if (b2 != b) continue;
+            const double g = (double)(s1 * s2) * peel[f].delta;
+            R -= g * ((double)(peel[f].i + 1) * (double)inv_p1);
+            Tm -= g * ((double)(peel[f].j + 1) * (double)inv_p3);
+        }
+        Rc[slot] = (float)R;
+        Tc[slot] = (float)Tm;
+    }
+}
+
+fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const SketchWs &sk, int m_b, int K, SelectWs &sel,
+                                     const PeelEntry *d_peel, int n_peel, uint64_t seed, int rnd, cudaStream_t st)
+{
+    if (K < 1) return FPSK_OK;
+    int p1 = 0, p3 = 0;
+    while ((1LL << p1) < in.n1) ++p1;
+    while ((1LL << p3) < in.n3) ++p3;
+    const float inv_p1 = 1.0f / (float)(1LL << p1), inv_p3 = 1.0f / (float)(1LL << p3);
+    const unsigned short *A = static_cast<const unsigned short *>(in.A);
+    const unsigned short *B = static_cast<const unsigned short *>(in.B);
+    const uint32_t key1 = round_key(seed, rnd, 0), key2 = round_key(seed, rnd, 1);
+    // 16-byte loads along k need both operands as rows contiguous in k (B as W = B^T) and aligned
+    const int vec = (in.bt && ((reinterpret_cast<uintptr_t>(in.A) | reinterpret_cast<uintptr_t>(in.B)) & 15) == 0 && in.lda % 8 == 0 &&
+                     in.ldb % 8 == 0 && in.n2 % 8 == 0) ? 1 : 0;
+    if (dtype == FPSK_FP16)
+        candidate_moments_kernel<__half><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n2, m_b, inv_p1,
+                                                            inv_p3, sk.rowperm, sk.rowstart, sk.colperm, sk.colstart, sel.keys,
+                                                            sel.counts, kSelMaxK, d_peel, n_peel, key1, key2, sel.Rc, sel.Tc, vec);
+    else
+        candidate_moments_kernel<__nv_bfloat16><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n2, m_b,
+                                                                   inv_p1, inv_p3, sk.rowperm, sk.rowstart, sk.colperm,
+                                                                   sk.colstart, sel.keys, sel.counts, kSelMaxK, d_peel, n_peel,
+                                                                   key1, key2, sel.Rc, sel.Tc, vec);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
                            int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
                            cudaStream_t st)

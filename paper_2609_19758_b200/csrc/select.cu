@@ -518,15 +518,20 @@ __global__ void collect_kernel(const float *S, long long mm, const float *scal, 
 
 // Sort the selected keys (descending |S|, ties by ascending flat index), keep those with
 // S != 0 and S, R, T finite (the set U), decode Eq. (recover) with 1-based -> 0-based indices.
-__global__ void __launch_bounds__(1024) decode_kernel(const float *S, const float *R, const float *T, int p1, int p3,
-                                                      const unsigned long long *keys, int *counts, int cap, Candidate *cand)
+// The moments come either from whole sketches R, T (indexed by bucket) or, when Rc is given, from the values
+// computed for the collected keys only (Rc, Tc indexed by the key's slot in `keys`).
+__global__ void __launch_bounds__(1024) decode_kernel(const float *S, const float *R, const float *T, const float *Rc,
+                                                      const float *Tc, int p1, int p3, const unsigned long long *keys,
+                                                      int *counts, int cap, Candidate *cand)
 {
     __shared__ unsigned long long sk[kSelMaxK];
     __shared__ int flag[kSelMaxK];
+    __shared__ unsigned short sl[kSelMaxK];           // the slot a key came from
     const int t = threadIdx.x;
     int n = counts[1];
     if (n > cap) n = cap;
     sk[t] = t < n ? keys[t] : 0ull;
+    sl[t] = (unsigned short)t;
     __syncthreads();
     // the network only has to cover the keys that are there (a power of two; zeros fill the rest)
     int np2 = 2;
@@ -537,7 +542,10 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
             if (ixj > t && ixj < np2) {
                 const bool desc = (t & k) == 0;
                 const unsigned long long a = sk[t], b = sk[ixj];
-                if (desc ? (a < b) : (a > b)) { sk[t] = b; sk[ixj] = a; }
+                if (desc ? (a < b) : (a > b)) {
+                    sk[t] = b; sk[ixj] = a;
+                    const unsigned short u = sl[t]; sl[t] = sl[ixj]; sl[ixj] = u;
+                }
             }
             __syncthreads();
         }
@@ -547,7 +555,7 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
     int keep = 0;
     if (t < n) {
         const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(sk[t] & 0xFFFFFFFFull);
-        const float s = S[idx], r = R ? R[idx] : 0.f, q = T ? T[idx] : 0.f;
+        const float s = S[idx], r = Rc ? Rc[sl[t]] : (R ? R[idx] : 0.f), q = Tc ? Tc[sl[t]] : (T ? T[idx] : 0.f);
         const bool fin = (fabsf(s) <= 3.402823466e38f) && (fabsf(r) <= 3.402823466e38f) && (fabsf(q) <= 3.402823466e38f);
         if (s != 0.f && fin) {
             float fi = rintf(ldexpf(r / s, p1)) - 1.f;
@@ -572,9 +580,10 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
     if (t == np2 - 1) counts[2] = flag[t];
 }
 
-fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
-                                     long long n3, const float *d_tau, int radius, int K, int mad_mode, SelectWs &w,
-                                     cudaStream_t st)
+// Thresholds from scal[1] and tau, then the K largest |S| above max(tau_c, tau_d) into w.keys (unsorted; count in
+// w.counts[1]).  mad_mode >= 0: sigma_MAD of S (1: of |S|, 0: signed) is computed in the same launch first.
+fpsk_status select_collect_launch(const float *S, int m_b, long long n1, long long n3, const float *d_tau, int radius, int K,
+                                  int mad_mode, SelectWs &w, cudaStream_t st)
 {
     if (K > kSelMaxK) K = kSelMaxK;
     const long long mm = (long long)m_b * m_b;
@@ -590,12 +599,29 @@ fpsk_status select_candidates_launch(const float *S, const float *R, const float
     const long long cwant = (mm + 4095) / 4096;
     collect_kernel<<<(int)(cwant < 1 ? 1 : (cwant > 1184 ? 1184 : cwant)), 256, 0, st>>>(S, mm, w.scal, w.state, kSelMaxK, w.keys, w.counts);
     FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// The collected keys sorted and decoded into w.cand (count in w.counts[2]); moments from the sketches R, T or, when
+// Rc is given, from the per-key values Rc, Tc.
+fpsk_status decode_launch(const float *S, const float *R, const float *T, const float *Rc, const float *Tc, long long n1,
+                          long long n3, SelectWs &w, cudaStream_t st)
+{
     int p1 = 0, p3 = 0;
     while ((1LL << p1) < n1) ++p1;
     while ((1LL << p3) < n3) ++p3;
-    decode_kernel<<<1, kSelMaxK, 0, st>>>(S, R, T, p1, p3, w.keys, w.counts, kSelMaxK, w.cand);
+    decode_kernel<<<1, kSelMaxK, 0, st>>>(S, R, T, Rc, Tc, p1, p3, w.keys, w.counts, kSelMaxK, w.cand);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
+}
+
+fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
+                                     long long n3, const float *d_tau, int radius, int K, int mad_mode, SelectWs &w,
+                                     cudaStream_t st)
+{
+    fpsk_status rc = select_collect_launch(S, m_b, n1, n3, d_tau, radius, K, mad_mode, w, st);
+    if (rc != FPSK_OK) return rc;
+    return decode_launch(S, R, T, nullptr, nullptr, n1, n3, w, st);
 }
 
 // ---------------------------------------------------------------- max |X| of a half matrix
@@ -759,7 +785,8 @@ fpsk_status sigma_mad_rms_c_select_launch(const float *S, long long mm, int mad_
 size_t select_ws_bytes()
 {
     return align_up(kHistBytes, 256) /*hist+tickets*/ + 256 /*state*/ + 256 /*scal*/ + align_up(kSumGrid * 4, 256) +
-           align_up(kSelMaxK * 8, 256) + 256 /*counts*/ + align_up(kSelMaxK * sizeof(Candidate), 256);
+           align_up(kSelMaxK * 8, 256) + 256 /*counts*/ + align_up(kSelMaxK * sizeof(Candidate), 256) +
+           2 * align_up(kSelMaxK * 4, 256) /*moments of the collected keys*/;
 }
 
 void select_carve(void *ws, SelectWs &w)
@@ -772,7 +799,9 @@ void select_carve(void *ws, SelectWs &w)
     w.partial = (float *)p; p += align_up(kSumGrid * 4, 256);
     w.keys = (unsigned long long *)p; p += align_up(kSelMaxK * 8, 256);
     w.counts = (int *)p; p += 256;
-    w.cand = (Candidate *)p;
+    w.cand = (Candidate *)p; p += align_up(kSelMaxK * sizeof(Candidate), 256);
+    w.Rc = (float *)p; p += align_up(kSelMaxK * 4, 256);
+    w.Tc = (float *)p;
     w.hist_clean = false;
 }
 

@@ -810,8 +810,8 @@ __global__ void peel_kernel(const PeelEntry *F, int nF, uint32_t key1, uint32_t 
         const double g = (double)(s1 * s2) * F[f].delta;
         const long long o = (long long)a * m_b + b;
         S[o] = (float)((double)S[o] - g);
-        R[o] = (float)((double)R[o] - g * ((double)(F[f].i + 1) * (double)inv_p1));
-        T[o] = (float)((double)T[o] - g * ((double)(F[f].j + 1) * (double)inv_p3));
+        if (R) R[o] = (float)((double)R[o] - g * ((double)(F[f].i + 1) * (double)inv_p1));
+        if (T) T[o] = (float)((double)T[o] - g * ((double)(F[f].j + 1) * (double)inv_p3));
     }
 }
 

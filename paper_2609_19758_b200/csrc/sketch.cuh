@@ -97,6 +97,7 @@ struct SelectWs {           // all device memory
     unsigned long long *keys;    // selected keys (<= kmax)
     int *counts;            // [0] valid samples of C, [1] collected, [2] n_U
     Candidate *cand;        // <= kmax
+    float *Rc, *Tc;         // first moments of the collected keys' buckets (slot order of `keys`)
     bool hist_clean;        // host side: the histogram has been zeroed since this workspace was carved
 };
 constexpr int kSelMaxK = 1024;
@@ -107,6 +108,11 @@ void select_carve(void *ws, SelectWs &w);
 fpsk_status sigma_clip_launch(const float *S, long long mm, SelectWs &w, cudaStream_t st);
 // thresholds from scal[1] and tau, K largest |S| above max(tau_c, tau_d), decoded candidates.
 // mad_mode >= 0: sigma_MAD of S (1: of |S|, 0: signed) is computed in the same launches first.
+// the two halves of select_candidates_launch, for a caller that computes the moments of the collected keys in between
+fpsk_status select_collect_launch(const float *S, int m_b, long long n1, long long n3, const float *d_tau, int radius, int K,
+                                  int mad_mode, SelectWs &w, cudaStream_t st);
+fpsk_status decode_launch(const float *S, const float *R, const float *T, const float *Rc, const float *Tc, long long n1,
+                          long long n3, SelectWs &w, cudaStream_t st);
 fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
                                      long long n3, const float *d_tau, int radius, int K, int mad_mode, SelectWs &w,
                                      cudaStream_t st);
@@ -131,6 +137,11 @@ struct Hit {                // an accepted window entry
     double gamma;           // FP64 recomputation
 };
 // force != 0: report every in-range window entry, whatever its test says
+// R, T of Eq. (recover) for the collected keys only (w.keys, count w.counts[1]) -> w.Rc, w.Tc: per key, the dot
+// products of the bucket's compressed rows of A and columns of B, the bucket's entries of C, and the peeled faults
+// that fall into the bucket.  Uses the hash tables of the round held in `sk`.
+fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const SketchWs &sk, int m_b, int K, SelectWs &sel,
+                                     const PeelEntry *d_peel, int n_peel, uint64_t seed, int rnd, cudaStream_t st);
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
                            int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
                            cudaStream_t st);
