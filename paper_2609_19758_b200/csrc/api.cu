@@ -172,7 +172,7 @@ static fpsk_status check_mats(const void *A, int64_t lda, const void *B, int64_t
 // ---------------------------------------------------------------- localize workspace
 struct LocWs {
     SketchWs sk;
-    float *S, *R, *T;
+    float *S;                 // the sum sketch of the round (R, T exist only at the kept buckets: SelectWs::Rc, Tc)
     SelectWs sel;
     float *samples;
     float *misc;              // [0] max|A| [1] max|B| [2] tau [3] rms_c ; [8..] uint scratch
@@ -188,7 +188,7 @@ static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bo
 {
     const size_t mm = (size_t)m_b * m_b;
     size_t b = sketch_ws_bytes(n1, n2, n3, m_b, tc);
-    b += align_up(mm * 4, 256) * 3;
+    b += align_up(mm * 4, 256);
     b += align_up(select_ws_bytes(), 256);
     b += align_up((size_t)131072 * 4, 256);
     b += 256;
@@ -209,7 +209,7 @@ static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, lon
     if (!sketch_carve(ws, skb, n1, n2, n3, m_b, w.sk, tc)) return false;
     char *p = static_cast<char *>(ws) + skb;
     auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
-    w.S = (float *)take(mm * 4); w.R = (float *)take(mm * 4); w.T = (float *)take(mm * 4);
+    w.S = (float *)take(mm * 4);
     select_carve(take(select_ws_bytes()), w.sel);
     w.samples = (float *)take((size_t)131072 * 4);
     w.misc = (float *)take(256);
