@@ -296,6 +296,10 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
         in.bt = 1;
     }
 
+    // the hash tables of all rounds in one batch of three launches (they depend on the seed only)
+    rc = prepare_hash_rounds(seed, 0, std::min(q.rounds, (int)kHashSets), m, n, m_b, w.sk, st);
+    if (rc != FPSK_OK) return rc;
+
     int radius = q.radius;
     bool round0_built = false;
     if (radius < 0) {

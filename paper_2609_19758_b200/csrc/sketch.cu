@@ -815,6 +815,112 @@ __global__ void peel_kernel(const PeelEntry *F, int nF, uint32_t key1, uint32_t 
     }
 }
 
+// ---------------------------------------------------------------- hash tables of several rounds at once
+static void sketch_use_set(SketchWs &w, int q)
+{
+    const HashSet &hs = w.sets[q];
+    w.h1 = hs.h1; w.v1 = hs.v1; w.h2 = hs.h2; w.v2 = hs.v2;
+    w.rowperm = hs.rowperm; w.colperm = hs.colperm; w.colpos = hs.colpos;
+    w.rowcount = hs.rowcount; w.rowstart = hs.rowstart; w.colcount = hs.colcount; w.colstart = hs.colstart;
+}
+
+struct HashJob {                 // one side of one round
+    uint32_t key;
+    int n;
+    int *bucket, *sign, *count, *start;
+    uint32_t *perm, *pos;
+};
+struct HashBatch {
+    HashJob job[2 * kHashSets];
+};
+// blockIdx.y = job: the three kernels of build_hash_side for all jobs of the batch in one launch each
+__global__ void hash_batch_kernel(HashBatch hb, int m_b)
+{
+    const HashJob &j = hb.job[blockIdx.y];
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= j.n) return;
+    int b, s;
+    hash_index(j.key, (uint32_t)idx, (uint32_t)m_b, b, s);
+    j.bucket[idx] = b;
+    j.sign[idx] = s;
+    atomicAdd(j.count + b, 1);
+}
+__global__ void scan_batch_kernel(HashBatch hb, int m_b)
+{
+    const HashJob &j = hb.job[blockIdx.x];
+    __shared__ int carry;
+    __shared__ int buf[1024];
+    if (threadIdx.x == 0) carry = 0;
+    __syncthreads();
+    for (int base = 0; base < m_b; base += 1024) {
+        const int i = base + threadIdx.x;
+        const int v = i < m_b ? j.count[i] : 0;
+        buf[threadIdx.x] = v;
+        __syncthreads();
+        for (int o = 1; o < 1024; o <<= 1) {
+            const int t = threadIdx.x >= o ? buf[threadIdx.x - o] : 0;
+            __syncthreads();
+            buf[threadIdx.x] += t;
+            __syncthreads();
+        }
+        if (i < m_b) j.start[i] = carry + buf[threadIdx.x] - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry += buf[1023];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) j.start[m_b] = carry;
+}
+__global__ void __launch_bounds__(256) place_batch_kernel(HashBatch hb)
+{
+    const HashJob &jb = hb.job[blockIdx.y];
+    const int idx = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (idx >= jb.n) return;
+    const int b = __ldg(jb.bucket + idx);
+    int cnt = 0;
+    int j = lane;
+    for (; j + 96 < idx; j += 128) {
+        const int b0 = __ldg(jb.bucket + j), b1 = __ldg(jb.bucket + j + 32), b2 = __ldg(jb.bucket + j + 64), b3 = __ldg(jb.bucket + j + 96);
+        cnt += (b0 == b) + (b1 == b) + (b2 == b) + (b3 == b);
+    }
+    for (; j < idx; j += 32) cnt += (__ldg(jb.bucket + j) == b);
+    cnt = __reduce_add_sync(0xFFFFFFFFu, cnt);
+    if (lane == 0) {
+        const uint32_t sbit = __ldg(jb.sign + idx) < 0 ? 0x80000000u : 0u;
+        const uint32_t where = (uint32_t)(__ldg(jb.start + b) + cnt);
+        jb.perm[where] = (uint32_t)idx | sbit;
+        if (jb.pos) jb.pos[idx] = where | sbit;
+    }
+}
+
+fpsk_status prepare_hash_rounds(uint64_t seed, int first, int count, long long n1, long long n3, int m_b, SketchWs &w,
+                                cudaStream_t st)
+{
+    if (count > kHashSets) count = kHashSets;
+    w.prepared_count = 0;
+    if (count < 1) return FPSK_OK;
+    HashBatch hb;
+    int nmax = 0;
+    for (int q = 0; q < count; ++q) {
+        const HashSet &hs = w.sets[q];
+        FPSK_CUDA_OK(cudaMemsetAsync(hs.rowcount, 0, sizeof(int) * (size_t)m_b, st));
+        FPSK_CUDA_OK(cudaMemsetAsync(hs.colcount, 0, sizeof(int) * (size_t)m_b, st));
+        hb.job[2 * q] = HashJob{round_key(seed, first + q, 0), (int)n1, hs.h1, hs.v1, hs.rowcount, hs.rowstart, hs.rowperm, nullptr};
+        hb.job[2 * q + 1] = HashJob{round_key(seed, first + q, 1), (int)n3, hs.h2, hs.v2, hs.colcount, hs.colstart, hs.colperm, hs.colpos};
+    }
+    nmax = (int)(n1 > n3 ? n1 : n3);
+    hash_batch_kernel<<<dim3((nmax + 255) / 256, 2 * count), 256, 0, st>>>(hb, m_b);
+    FPSK_LAUNCH_CHECK();
+    scan_batch_kernel<<<2 * count, 1024, 0, st>>>(hb, m_b);
+    FPSK_LAUNCH_CHECK();
+    place_batch_kernel<<<dim3((nmax + 7) / 8, 2 * count), 256, 0, st>>>(hb);
+    FPSK_LAUNCH_CHECK();
+    w.prepared_first = first;
+    w.prepared_count = count;
+    w.prepared_seed = seed;
+    return FPSK_OK;
+}
+
 // ---------------------------------------------------------------- host orchestration
 static int pow2_exp(long long n)
 {
@@ -861,9 +967,9 @@ size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool t
     tc = tc && m_b >= kTcMinBuckets;
     const int tcks = tc ? tc_plan_ksplit(m_b, m_b, pl.kpad, 3, sketch_sms()) : 0;
     size_t b = 0;
-    b += align_up((size_t)n1 * 4, 256) * 3;          // h1, v1, rowperm
-    b += align_up((size_t)n3 * 4, 256) * 4;          // h2, v2, colperm, colpos
-    b += align_up((size_t)(m_b + 1) * 4, 256) * 4;   // rowcount, rowstart, colcount, colstart
+    b += kHashSets * align_up((size_t)n1 * 4, 256) * 3;          // h1, v1, rowperm           (per prepared hash round)
+    b += kHashSets * align_up((size_t)n3 * 4, 256) * 4;          // h2, v2, colperm, colpos
+    b += kHashSets * align_up((size_t)(m_b + 1) * 4, 256) * 4;   // rowcount, rowstart, colcount, colstart
     b += align_up((size_t)m_b * pl.kpad * 4, 256) * 2;       // P, Pw
     b += align_up((size_t)pl.kpad * pl.npad * 4, 256) * 2;   // Q, Qw
     b += align_up((size_t)(pl.ksplit > tcks ? pl.ksplit : tcks) * 3 * mm * 4, 256);      // AB partials
@@ -881,11 +987,16 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
     const size_t mm = (size_t)m_b * m_b;
     char *p = static_cast<char *>(ws);
     auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
-    w.h1 = (int *)take((size_t)n1 * 4); w.v1 = (int *)take((size_t)n1 * 4); w.rowperm = (uint32_t *)take((size_t)n1 * 4);
-    w.h2 = (int *)take((size_t)n3 * 4); w.v2 = (int *)take((size_t)n3 * 4); w.colperm = (uint32_t *)take((size_t)n3 * 4);
-    w.colpos = (uint32_t *)take((size_t)n3 * 4);
-    w.rowcount = (int *)take((size_t)(m_b + 1) * 4); w.rowstart = (int *)take((size_t)(m_b + 1) * 4);
-    w.colcount = (int *)take((size_t)(m_b + 1) * 4); w.colstart = (int *)take((size_t)(m_b + 1) * 4);
+    for (int q = 0; q < kHashSets; ++q) {
+        HashSet &hs = w.sets[q];
+        hs.h1 = (int *)take((size_t)n1 * 4); hs.v1 = (int *)take((size_t)n1 * 4); hs.rowperm = (uint32_t *)take((size_t)n1 * 4);
+        hs.h2 = (int *)take((size_t)n3 * 4); hs.v2 = (int *)take((size_t)n3 * 4); hs.colperm = (uint32_t *)take((size_t)n3 * 4);
+        hs.colpos = (uint32_t *)take((size_t)n3 * 4);
+        hs.rowcount = (int *)take((size_t)(m_b + 1) * 4); hs.rowstart = (int *)take((size_t)(m_b + 1) * 4);
+        hs.colcount = (int *)take((size_t)(m_b + 1) * 4); hs.colstart = (int *)take((size_t)(m_b + 1) * 4);
+    }
+    w.prepared_first = 0; w.prepared_count = 0; w.prepared_seed = 0;
+    sketch_use_set(w, 0);
     w.P = (float *)take((size_t)m_b * w.pl.kpad * 4); w.Pw = (float *)take((size_t)m_b * w.pl.kpad * 4);
     w.Q = (float *)take((size_t)w.pl.kpad * w.pl.npad * 4); w.Qw = (float *)take((size_t)w.pl.kpad * w.pl.npad * 4);
     w.tc = tc;
@@ -1024,10 +1135,17 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         FPSK_CUDA_OK(cudaStreamWaitEvent(sB, ax->ev[0], 0));
         FPSK_CUDA_OK(cudaStreamWaitEvent(sC, ax->ev[0], 0));
     }
-    rc = build_hash_side(seed, rnd, 0, n1, m_b, w.h1, w.v1, w.rowcount, w.rowstart, w.rowperm, st);
-    if (rc != FPSK_OK) return rc;
-    rc = build_hash_side(seed, rnd, 1, n3, m_b, w.h2, w.v2, w.colcount, w.colstart, w.colperm, sB, w.colpos);
-    if (rc != FPSK_OK) return rc;
+    if (w.prepared_count > 0 && seed == w.prepared_seed && rnd >= w.prepared_first && rnd < w.prepared_first + w.prepared_count) {
+        sketch_use_set(w, rnd - w.prepared_first);         // tables prepared ahead (on st, before this point)
+    } else {
+        // built here, into the first set (whatever was prepared is overwritten: forget it)
+        w.prepared_count = 0;
+        sketch_use_set(w, 0);
+        rc = build_hash_side(seed, rnd, 0, n1, m_b, w.h1, w.v1, w.rowcount, w.rowstart, w.rowperm, st);
+        if (rc != FPSK_OK) return rc;
+        rc = build_hash_side(seed, rnd, 1, n3, m_b, w.h2, w.v2, w.colcount, w.colstart, w.colperm, sB, w.colpos);
+        if (rc != FPSK_OK) return rc;
+    }
     const float *scA = w.tc ? w.tc_scale : nullptr, *scB = w.tc ? w.tc_scale + 1 : nullptr;
     if (w.tc) {
         if (!w.d_maxab) return FPSK_ERR_PARAM;

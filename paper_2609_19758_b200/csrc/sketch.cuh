@@ -34,9 +34,19 @@ struct SketchAuxLease {          // returns the set to the pool when it goes out
 };
 fpsk_status sketch_aux_acquire(SketchAuxLease &lease);
 
+constexpr int kHashSets = 3;     // hash rounds whose tables can be prepared ahead in one batch
+struct HashSet {                 // the tables of one hash round
+    int *h1, *v1, *h2, *v2;
+    uint32_t *rowperm, *colperm, *colpos;
+    int *rowcount, *rowstart, *colcount, *colstart;
+};
 struct SketchWs {
     SketchPlan pl;
     SketchAux *aux;              // nullptr: everything on the caller's stream
+    HashSet sets[kHashSets];
+    int prepared_first, prepared_count;      // rounds whose tables sit in sets[0 .. prepared_count) (host side)
+    unsigned long long prepared_seed;
+    // the tables of the round in progress (one of the sets)
     int *h1, *v1, *h2, *v2;
     uint32_t *rowperm, *colperm;
     uint32_t *colpos;            // inverse of colperm: position (and sign) of every column in the bucket-sorted order
@@ -67,6 +77,10 @@ fpsk_status build_hash_side(uint64_t seed, int rnd, int side, int n, int m_b, in
 // W = B^T for 16-bit elements: W[j * ldw + k] = B[k * ldb + j], k < n2, j < n3 (ldw >= n2)
 fpsk_status transpose_b_launch(const void *B, long long ldb, long long n2, long long n3, void *W, long long ldw,
                                cudaStream_t st);
+// Hash tables and bucket-sorted permutations of rounds first .. first + count - 1 (count <= kHashSets), both sides, in
+// three batched launches; build_sketches then finds them ready.
+fpsk_status prepare_hash_rounds(uint64_t seed, int first, int count, long long n1, long long n3, int m_b, SketchWs &w,
+                                cudaStream_t st);
 fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int rnd, int m_b, bool mom,
                            SketchWs &w, cudaStream_t st, float *S, float *R, float *T);
 // start[0..n] = exclusive prefix sums of count[0..n)  (one CTA, any n)
