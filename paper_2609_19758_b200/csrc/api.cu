@@ -281,24 +281,39 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
     rc = sketch_aux_acquire(aux);
     if (rc != FPSK_OK) return rc;
     w.sk.aux = aux.aux;
-    // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
-    rc = loc_max_ab(in, dtype, w, st);
+    // Once per call, side by side: max|A| and the hash tables of all rounds (they depend on the seed only) on the
+    // caller's stream; max|B| and, for B given as k x n, its transpose on an auxiliary stream.  With W = B^T every round
+    // reads rows of W: the B compression sums rows instead of gathering columns, the confirmation reads a row instead
+    // of a strided column; same bits.
+    SketchAux *ax = (aux.aux && aux.aux->s1 && aux.aux->s2 && aux.aux->ev[4]) ? aux.aux : nullptr;
+    cudaStream_t sB0 = ax ? ax->s1 : st;
+    unsigned int *uscr = reinterpret_cast<unsigned int *>(w.misc + 8);
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));             // whatever the caller queued before this call
+        FPSK_CUDA_OK(cudaStreamWaitEvent(sB0, ax->ev[0], 0));
+    }
+    rc = max_abs_half_launch(in.A, in.lda, m, k, dtype, w.misc + 0, uscr, st);
     if (rc != FPSK_OK) return rc;
-    tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
-    FPSK_LAUNCH_CHECK();
+    rc = in.bt ? max_abs_half_launch(in.B, in.ldb, n, k, dtype, w.misc + 1, uscr + 1, sB0)
+               : max_abs_half_launch(in.B, in.ldb, k, n, dtype, w.misc + 1, uscr + 1, sB0);
+    if (rc != FPSK_OK) return rc;
+    w.sk.d_maxab = w.misc;
     if (!in.bt && w.Wt) {
-        // B as k x n: transpose it once and let every round read rows of W = B^T (the B compression sums rows
-        // instead of gathering columns, the confirmation reads a row instead of a strided column; same bits)
-        rc = transpose_b_launch(in.B, in.ldb, k, n, w.Wt, w.ldw, st);
+        rc = transpose_b_launch(in.B, in.ldb, k, n, w.Wt, w.ldw, sB0);
         if (rc != FPSK_OK) return rc;
         in.B = w.Wt;
         in.ldb = w.ldw;
         in.bt = 1;
     }
-
-    // the hash tables of all rounds in one batch of three launches (they depend on the seed only)
     rc = prepare_hash_rounds(seed, 0, std::min(q.rounds, (int)kHashSets), m, n, m_b, w.sk, st);
     if (rc != FPSK_OK) return rc;
+    if (ax) {
+        FPSK_CUDA_OK(cudaEventRecord(ax->ev[1], sB0));
+        FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->ev[1], 0));
+    }
+    // tau = 100 n2 eps max|A| max|B| (device scalar misc[2])
+    tau_kernel<<<1, 32, 0, st>>>(w.misc, (float)k);
+    FPSK_LAUNCH_CHECK();
 
     int radius = q.radius;
     bool round0_built = false;

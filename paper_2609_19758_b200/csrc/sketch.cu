@@ -901,10 +901,10 @@ fpsk_status prepare_hash_rounds(uint64_t seed, int first, int count, long long n
     if (count < 1) return FPSK_OK;
     HashBatch hb;
     int nmax = 0;
+    // the counts of sets 0 .. count - 1 are one contiguous block (see sketch_carve)
+    FPSK_CUDA_OK(cudaMemsetAsync(w.sets[0].rowcount, 0, (size_t)count * 2 * align_up((size_t)(m_b + 1) * 4, 256), st));
     for (int q = 0; q < count; ++q) {
         const HashSet &hs = w.sets[q];
-        FPSK_CUDA_OK(cudaMemsetAsync(hs.rowcount, 0, sizeof(int) * (size_t)m_b, st));
-        FPSK_CUDA_OK(cudaMemsetAsync(hs.colcount, 0, sizeof(int) * (size_t)m_b, st));
         hb.job[2 * q] = HashJob{round_key(seed, first + q, 0), (int)n1, hs.h1, hs.v1, hs.rowcount, hs.rowstart, hs.rowperm, nullptr};
         hb.job[2 * q + 1] = HashJob{round_key(seed, first + q, 1), (int)n3, hs.h2, hs.v2, hs.colcount, hs.colstart, hs.colperm, hs.colpos};
     }
@@ -987,13 +987,18 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
     const size_t mm = (size_t)m_b * m_b;
     char *p = static_cast<char *>(ws);
     auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
+    // the bucket counts of all sets side by side: one memset clears them when several rounds are prepared at once
+    for (int q = 0; q < kHashSets; ++q) {
+        w.sets[q].rowcount = (int *)take((size_t)(m_b + 1) * 4);
+        w.sets[q].colcount = (int *)take((size_t)(m_b + 1) * 4);
+    }
     for (int q = 0; q < kHashSets; ++q) {
         HashSet &hs = w.sets[q];
         hs.h1 = (int *)take((size_t)n1 * 4); hs.v1 = (int *)take((size_t)n1 * 4); hs.rowperm = (uint32_t *)take((size_t)n1 * 4);
         hs.h2 = (int *)take((size_t)n3 * 4); hs.v2 = (int *)take((size_t)n3 * 4); hs.colperm = (uint32_t *)take((size_t)n3 * 4);
         hs.colpos = (uint32_t *)take((size_t)n3 * 4);
-        hs.rowcount = (int *)take((size_t)(m_b + 1) * 4); hs.rowstart = (int *)take((size_t)(m_b + 1) * 4);
-        hs.colcount = (int *)take((size_t)(m_b + 1) * 4); hs.colstart = (int *)take((size_t)(m_b + 1) * 4);
+        hs.rowstart = (int *)take((size_t)(m_b + 1) * 4);
+        hs.colstart = (int *)take((size_t)(m_b + 1) * 4);
     }
     w.prepared_first = 0; w.prepared_count = 0; w.prepared_seed = 0;
     sketch_use_set(w, 0);
