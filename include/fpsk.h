@@ -89,12 +89,16 @@ typedef struct {
     int32_t s_budget;    /* declared fault count s (sets K = max(64, 8 s) and m_comb)      */
     int32_t delta_max;   /* declared bound Delta on faults per row or column               */
     int32_t mad_of_abs;  /* 1: MAD of |S| as printed in the paper; 0: signed MAD of S      */
-    int32_t tensor_cores;/* 0: FP32 FMA contraction; 1: split-BF16 tcgen05 contraction     */
+    int32_t tensor_cores;/* 0: FP32 FMA contraction; 1: tcgen05 contraction on two scaled FP16
+                            terms per FP32 value (three products, FP32 accumulation in TMEM)   */
     int32_t b_transposed;/* fpsk_measure_noise, fpsk_localize: 1 = the B pointer is the weight
                             W = B^T (n x k, row-major, ldb >= k), i.e. C = A W^T; 0 = B is k x n.
                             Other entry points take B as k x n (fpsk_probe_hashed has its own
                             switch in fpsk_bside).                                          */
-    int32_t reserved;
+    int32_t scale_cap;   /* fpsk_probe_hashed only.  0 (default): thr = min(tau, ...) exactly as Section
+                            "Thresholds" prints it; 1: the analytic cap enters as tau sqrt(m n / n_buckets^2)
+                            (not in the paper: for sketches so coarse that a clean bucket, which sums
+                            m n / n_buckets^2 entries of E, can exceed the bound on ONE inner product)     */
     double rho_min;      /* smallest fault to localize, in units of rms(C)                 */
     double c_valid;      /* c of tau_ij = c eps sum_k |A_ik||B_kj|                         */
     double mu;           /* probe margin                                                   */
@@ -201,7 +205,10 @@ fpsk_status fpsk_probe_static(const void *A, int64_t lda, const void *B, int64_t
 /* Host-side record of a cached B side (Section "Implementation": the sketch of the B side is
  * cached and keyed on tensor identity and version, so an in-place optimizer update invalidates
  * it).  Zero-initialise it once (valid = 0); fpsk_probe_hashed fills and checks it.  The key is
- * (B pointer, ldb, b_version, shape, dtype, seed, round, n_buckets, cache pointer). */
+ * (B pointer, ldb, b_version, shape, dtype, seed, round, n_buckets, cache pointer, layout of B).
+ * The record only says what was ENQUEUED: the (re)build runs asynchronously on the stream of the call
+ * that missed, so a cache and its record belong to one stream (or to streams the caller orders after
+ * that call). */
 typedef struct {
     const void *B;
     void *cache;
@@ -212,6 +219,8 @@ typedef struct {
     int32_t rebuilds;     /* how many times the B side was (re)built through this record       */
     int32_t b_transposed; /* set by the caller before the first call: 0 = the B pointer is B (k x n, row-major);
                              1 = it is W = B^T (n x k, row-major, ldb >= k), the x W^T weight layout  */
+    int32_t built_transposed; /* layout the cached B side was built from (part of the key; library-written) */
+    int32_t reserved;
 } fpsk_bside;
 
 /* State of a probe across calls; see "what the probe keeps between calls" below. */
@@ -238,9 +247,8 @@ int32_t fpsk_bside_matches(const fpsk_bside *side, const void *B, int64_t ldb, u
 
 /* The S only probe (Section "The Cheap S Only Probe"): S = (H1 A)(B H2^T) - H1 C H2^T for hash
  * round `round` of `seed` at n_buckets buckets per side, sigma_hat = 1.2533 mean(min(|S|, 5 mean|S|))
- * over the n_buckets^2 buckets, thr = min(tau sqrt(m n / n_buckets^2), mu sqrt(2 ln n_buckets^2) sigma_hat)
- * (Section "Thresholds"; a bucket sums m n / n_buckets^2 entries of E on average, so the analytic
- * cap enters with the root of that population), dirty iff max|S| > thr or S is not finite.
+ * over the n_buckets^2 buckets, thr = min(tau, mu sqrt(2 ln n_buckets^2) sigma_hat) (Section "Thresholds";
+ * p->scale_cap = 1 widens the cap to tau sqrt(m n / n_buckets^2)), dirty iff max|S| > thr or S is not finite.
  *   B, ldb        B itself, or, with side->b_transposed = 1, the weight W = B^T as n x k row-major
  *                 (C = A W^T); only the (re)build of the B side reads it
  *   side, cache   the B side.  When `side` does not match the key (see fpsk_bside), it is rebuilt

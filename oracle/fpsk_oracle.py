@@ -14,13 +14,17 @@ Indices are 0-based in every interface; the 1-based index weights
 w_i = (i+1)/2^ceil(log2 n1) are internal.
 
 Parity pins (tests/test_oracle_*.py): integer brute force for Eq. (S),
-exact single-fault recovery for Eq. (recover), the printed bucket counts of
-Table "rect" and the other integers the paper prints for the sizing law,
-Gaussian closed forms for the two noise estimators, collision statistics for
-the hash rounds, Lemma 1 on a clean product.  Two readings have no pin in the
-paper and are "parity unpinned": the probe threshold applied to the un-hashed
-column sketch (bucket count taken as n3), and the noise constant itself (the
-paper states that it belongs to the BLAS).
+exact single-fault recovery for Eq. (recover), peeling against the term-by-term
+sketch of the faults left behind (exact on integer products), the printed bucket
+counts of Table "rect" and the other integers the paper prints for the sizing law,
+Gaussian closed forms for the two noise estimators and for the normalisation of
+the noise constant, brute force for the tolerance denominators, collision
+statistics for the hash rounds, Lemma 1 on a clean product.  Two readings have no
+pin in the paper and are "parity unpinned": the probe threshold applied to the
+un-hashed column sketch (bucket count taken as n3, analytic cap scaled by
+sqrt(n1)), and the value of the noise constant on a given GPU (the paper states
+that it belongs to the BLAS).  The hashed S only probe follows the rule of
+Section "Thresholds" as printed.
 """
 from __future__ import annotations
 
@@ -72,6 +76,8 @@ class Params:
     s_budget: int = 8
     delta_max: int = 8
     mad_of_abs: int = 1         # 1: MAD of |S| as printed; 0: signed MAD of S
+    scale_cap: int = 0          # hashed probe only. 0: thr = min(tau, ...) as printed in Section
+                                # "Thresholds"; 1: the cap enters as tau sqrt(n1 n3 / m^2)
 
 
 @dataclass
@@ -230,10 +236,10 @@ def hashed_sum_sketch(E, h1, v1, h2, v2, m_b: int) -> np.ndarray:
 
 def probe_hashed(A, B, C, seed: int, rnd: int, m_b: int, params: Params = None):
     """The S only probe: hash round (seed, rnd) with m_b buckets per side, S = H1 (AB - C) H2^T,
-    sigma_hat = clipped mean over the m_b^2 buckets, thr = min(cap, mu sqrt(2 ln m_b^2) sigma_hat),
-    dirty iff max|S| > thr or S is not finite.  The analytic cap enters as tau sqrt(n1 n3 / m_b^2):
-    tau bounds one inner product's rounding and a bucket sums n1 n3 / m_b^2 of them on average
-    (the reading taken for the un-hashed sketch, applied to the bucket population).
+    sigma_hat = clipped mean over the m_b^2 buckets, thr = min(tau, mu sqrt(2 ln m_b^2) sigma_hat)
+    as Section "Thresholds" prints it, dirty iff max|S| > thr or S is not finite.  Only with
+    params.scale_cap = 1 (off by default, not in the paper) the cap enters as
+    tau sqrt(n1 n3 / m_b^2), the root of the number of entries of E a bucket sums on average.
     Returns (ProbeResult with argmax_col = flat bucket index a*m_b + b, S)."""
     params = params or Params()
     A64, B64 = _f64(A), _f64(B)
@@ -245,7 +251,7 @@ def probe_hashed(A, B, C, seed: int, rnd: int, m_b: int, params: Params = None):
         E = A64 @ B64 - np.asarray(C, dtype=np.float64)
     S = hashed_sum_sketch(E, h1, v1, h2, v2, m_b)
     tau = analytic_tau(A64, B64, n2)
-    pop = float(n1) * float(n3) / (float(m_b) * float(m_b))
+    pop = float(n1) * float(n3) / (float(m_b) * float(m_b)) if params.scale_cap else 1.0
     return probe_verdict(S.ravel(), tau, params, n_rows=pop), S
 
 

@@ -61,14 +61,16 @@ def run_case(tag, kind, n1, n2, n3, dtype, seed, make_faults, params, probe_buck
     pws = fpsk.probe_workspace(n1, n2, n3)
     res = fpsk.new_probe_result()
     fpsk.probe(dA, dB, dC, pws, res, None, params)
-    clean_fired = fpsk.read_probe_result(res).fired
+    r_c = fpsk.read_probe_result(res)
+    clean_fired = r_c.fired
     dirty_fired = None
     if faults:
         fpsk.probe(dA, dB, dCf, pws, res, None, params)
         dirty_fired = fpsk.read_probe_result(res).fired
     hp = fpsk.HashedProbe(n1, n2, n3, probe_buckets, seed=seed + 1000)
     hp(dA, dB, dC, res, params=params)
-    h_clean = fpsk.read_probe_result(res).fired
+    r_h = fpsk.read_probe_result(res)
+    h_clean = r_h.fired
     h_dirty = None
     if faults:
         hp(dA, dB, dCf, res, params=params)
@@ -104,7 +106,10 @@ def run_case(tag, kind, n1, n2, n3, dtype, seed, make_faults, params, probe_buck
     print(json.dumps(dict(case=tag, shape=[n1, n2, n3], dtype="fp16" if dtype == W.FP16 else "bf16", seed=seed,
                           c_hat=nz.c_hat, plan=[nz.m0, nz.m_loc, nz.radius], injected=len(faults), found=len(want & have),
                           false_positives=len(have - want) + len(got_clean), probe=[int(clean_fired), dirty_fired],
-                          hashed_probe=[int(h_clean), h_dirty])), flush=True)
+                          hashed_probe=[int(h_clean), h_dirty],
+                          probe_clean=dict(max_abs=r_c.max_abs, sigma_hat=r_c.sigma_hat, thr=r_c.thr, tau=r_c.tau),
+                          hashed_clean=dict(m=probe_buckets, max_abs=r_h.max_abs, sigma_hat=r_h.sigma_hat, thr=r_h.thr,
+                                            tau=r_h.tau))), flush=True)
     del ws, dA, dB, dC, dCf
     torch.cuda.empty_cache()
 

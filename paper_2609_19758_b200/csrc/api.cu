@@ -148,7 +148,8 @@ static bool params_ok(const fpsk_params &p)
 {
     return p.rounds >= 1 && p.rounds <= 8 && p.r_star >= 0 && p.r_max >= 0 && p.r_max <= 16 && p.radius >= -1 &&
            p.radius <= 16 && p.s_budget >= 1 && p.delta_max >= 1 && p.rho_min > 0 && p.c_valid > 0 && p.mu > 0 &&
-           p.b_star > 0 && p.c_coll > 1.0 - 1e-12 && (p.b_transposed == 0 || p.b_transposed == 1);
+           p.b_star > 0 && p.c_coll > 1.0 - 1e-12 && (p.b_transposed == 0 || p.b_transposed == 1) &&
+           (p.scale_cap == 0 || p.scale_cap == 1);
 }
 
 static fpsk_params resolve_params(const fpsk_params *p)
@@ -619,16 +620,18 @@ fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, cons
     if (cache_bytes < hprobe_cache_bytes(m, k, n, n_buckets) || ws_bytes < hprobe_ws_bytes(m, k, n, n_buckets))
         return FPSK_ERR_WORKSPACE;
     const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (side->valid && side->built_transposed != side->b_transposed) side->valid = 0;      // the layout is part of the key
     if (!fpsk_bside_matches(side, B, ldb, b_version, m, k, n, dtype, seed, round, n_buckets, cache)) {
         side->valid = 0;
         rc = hprobe_prepare(B, ldb, bt ? 1 : 0, m, k, n, dtype, seed, round, n_buckets, cache, cache_bytes, st);
         if (rc != FPSK_OK) return rc;
         side->B = B; side->cache = cache; side->ldb = ldb; side->m = m; side->k = k; side->n = n;
         side->seed = seed; side->version = b_version; side->dtype = (int32_t)dtype; side->n_buckets = n_buckets;
-        side->round = round; side->valid = 1; side->rebuilds += 1;
+        side->round = round; side->built_transposed = side->b_transposed; side->valid = 1; side->rebuilds += 1;
     }
-    return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, q.tensor_cores, cache, cache_bytes, workspace, ws_bytes, st,
+    return hprobe_launch(A, lda, C, ldc, m, k, n, dtype, n_buckets, q.mu, q.scale_cap, q.tensor_cores, cache, cache_bytes, workspace, ws_bytes, st,
                          d_result, d_S, d_state);
 }
 

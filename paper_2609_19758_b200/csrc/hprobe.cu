@@ -560,7 +560,7 @@ struct HvArgs {
     const float *maxB;       // [0] max|B|, [1] scale of the Q planes
     const float *scaleA;     // scale of the P planes when the partials come from the tensor cores, else null
     float thr_scale;         // mu sqrt(2 ln max(m^2, 2))
-    float cap_scale;         // sqrt(n1 n3 / m^2)
+    float cap_scale;         // 1 (the printed rule), or sqrt(n1 n3 / m^2) when the caller asked for the scaled cap
     float *S;                // m*m
     float4 *vstat;           // per CTA: sum|S|, nonfinite count, max, argmax (as int bits)
     float *cstat;            // per CTA: sum of min(|S|, clip)
@@ -982,7 +982,7 @@ fpsk_status hprobe_prepare(const void *B, long long ldb, int b_transposed, long 
 
 // One probe on a prepared B side.  d_S may be NULL (S then stays in the workspace).
 fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
-                          long long n3, fpsk_dtype dtype, int m, double mu, int tensor_cores, void *cache, size_t cache_bytes, void *ws,
+                          long long n3, fpsk_dtype dtype, int m, double mu, int scale_cap, int tensor_cores, void *cache, size_t cache_bytes, void *ws,
                           size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S, fpsk_probe_state *d_state)
 {
     const int sms = hp_sm_count();
@@ -1043,7 +1043,7 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     v.scaleA = tensor_cores ? w.scaleA : nullptr;
     const double mm = (double)m * (double)m;
     v.thr_scale = (float)(mu * sqrt(2.0 * log(mm > 2.0 ? mm : 2.0)));
-    v.cap_scale = (float)sqrt((double)n1 * (double)n3 / mm);
+    v.cap_scale = scale_cap ? (float)sqrt((double)n1 * (double)n3 / mm) : 1.0f;
     v.S = d_S ? d_S : w.S;
     v.vstat = w.vstat; v.cstat = w.cstat; v.ctrl = w.ctrl; v.result = d_result; v.state = d_state;
     v.ctrace = a.trace_on ? w.trace + 8 * 2 * sms : nullptr;

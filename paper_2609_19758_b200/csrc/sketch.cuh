@@ -211,7 +211,7 @@ size_t hprobe_ws_bytes(long long n1, long long n2, long long n3, int m);
 fpsk_status hprobe_prepare(const void *B, long long ldb, int b_transposed, long long n1, long long n2, long long n3, fpsk_dtype dtype,
                            uint64_t seed, int rnd, int m, void *cache, size_t cache_bytes, cudaStream_t st);
 fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long long ldc, long long n1, long long n2,
-                          long long n3, fpsk_dtype dtype, int m, double mu, int tensor_cores, void *cache, size_t cache_bytes, void *ws,
+                          long long n3, fpsk_dtype dtype, int m, double mu, int scale_cap, int tensor_cores, void *cache, size_t cache_bytes, void *ws,
                           size_t ws_bytes, cudaStream_t st, fpsk_probe_result *d_result, float *d_S, fpsk_probe_state *d_state);
 fpsk_status probe_accumulate_launch(const fpsk_probe_result *d_result, fpsk_probe_state *d_state, cudaStream_t st);
 

@@ -34,7 +34,7 @@ class Fault(C.Structure):
 class Params(C.Structure):
     _fields_ = [("rounds", C.c_int32), ("r_star", C.c_int32), ("r_max", C.c_int32), ("radius", C.c_int32),
                 ("s_budget", C.c_int32), ("delta_max", C.c_int32), ("mad_of_abs", C.c_int32), ("tensor_cores", C.c_int32),
-                ("b_transposed", C.c_int32), ("reserved", C.c_int32),
+                ("b_transposed", C.c_int32), ("scale_cap", C.c_int32),
                 ("rho_min", C.c_double), ("c_valid", C.c_double), ("mu", C.c_double), ("b_star", C.c_double),
                 ("c_coll", C.c_double)]
 
@@ -55,7 +55,7 @@ class BSide(C.Structure):
     _fields_ = [("B", C.c_void_p), ("cache", C.c_void_p), ("ldb", C.c_int64), ("m", C.c_int64), ("k", C.c_int64),
                 ("n", C.c_int64), ("seed", C.c_uint64), ("version", C.c_uint64), ("dtype", C.c_int32),
                 ("n_buckets", C.c_int32), ("round", C.c_int32), ("valid", C.c_int32), ("rebuilds", C.c_int32),
-                ("b_transposed", C.c_int32)]
+                ("b_transposed", C.c_int32), ("built_transposed", C.c_int32), ("reserved", C.c_int32)]
 
 
 class ProbeState(C.Structure):

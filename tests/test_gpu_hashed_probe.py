@@ -56,21 +56,22 @@ SHAPES = [
 
 @pytest.mark.parametrize("shape", SHAPES)
 @pytest.mark.parametrize("dtype", [W.FP16, W.BF16])
-@pytest.mark.parametrize("tensor_cores", [0, 1])
-def test_sketch_and_verdict(shape, dtype, tensor_cores):
+@pytest.mark.parametrize("tensor_cores,scale_cap", [(0, 0), (1, 0), (0, 1)])
+def test_sketch_and_verdict(shape, dtype, tensor_cores, scale_cap):
     n1, n2, n3, m = shape
     A, Bm, Cm = _case("uniform" if dtype == W.FP16 else "gauss_scaled", n1, n2, n3, dtype, 5)
     A64, B64 = _f64(A), _f64(Bm)
-    ref, S_ref = O.probe_hashed(A64, B64, Cm.numpy(), 21, 4, m)
+    ref, S_ref = O.probe_hashed(A64, B64, Cm.numpy(), 21, 4, m, O.Params(scale_cap=scale_cap))
     h1, _ = O.hash_round(21, 4, 0, n1, m)
     h2, _ = O.hash_round(21, 4, 1, n3, m)
     denom = O.abs_sketch(O.abs_product(A64, B64), h1, h2, m)
     hp = fpsk.HashedProbe(n1, n2, n3, m, seed=21, rnd=4)
-    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda(), params=fpsk.default_params(tensor_cores=tensor_cores))
+    got, S = _run(hp, A.cuda(), Bm.cuda(), Cm.cuda(), params=fpsk.default_params(tensor_cores=tensor_cores, scale_cap=scale_cap))
     assert got.status == 0
     assert np.all(np.abs(S - S_ref) <= TOL * denom + 1e-30)
     assert got.tau == pytest.approx(ref.tau, rel=1e-6)
-    v = O.probe_verdict(S.ravel(), ref.tau, n_rows=n1 * n3 / float(m * m))     # the rule on the GPU's own S
+    # the rule on the GPU's own S: the printed one, or with the cap widened by the root of the bucket population
+    v = O.probe_verdict(S.ravel(), ref.tau, n_rows=n1 * n3 / float(m * m) if scale_cap else 1)
     assert got.sigma_hat == pytest.approx(v.sigma_hat, rel=1e-4, abs=1e-30)
     assert got.thr == pytest.approx(v.thr, rel=1e-4, abs=1e-30)
     assert got.max_abs == pytest.approx(v.max_abs, rel=1e-6, abs=1e-30)

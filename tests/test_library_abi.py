@@ -107,7 +107,7 @@ def test_argument_validation_needs_no_device(lib):
 
 def test_bside_record_and_key_logic(lib):
     """The cache key of the B side (tensor identity and version; Section "Implementation") is host logic."""
-    assert C.sizeof(fpsk.BSide) == 88 and fpsk.BSide.valid.offset == 76
+    assert C.sizeof(fpsk.BSide) == 96 and fpsk.BSide.valid.offset == 76 and fpsk.BSide.built_transposed.offset == 88
     s = fpsk.BSide()
     Bp, cache = C.c_void_p(0x1000), C.c_void_p(0x2000)
     args = (Bp, 64, 7, 32, 48, 64, fpsk.BF16, 99, 3, 16, cache)

@@ -92,13 +92,21 @@ def test_rule_closed_form_and_population_cap():
     assert math.isclose(r2.thr, 1.0, rel_tol=1e-12) and r2.fired
 
 
-def test_population_enters_probe_hashed():
+def test_printed_rule_is_the_default_and_the_population_cap_is_opt_in():
+    # Section "Thresholds": thr = min(tau, mu sqrt(2 ln m^2) sigma_hat).  A tiny inner dimension with large
+    # entries of C makes the cap bind, so the two forms of the cap can be told apart.
     A, B, C = _ops("uniform", 64, 32, 48, o.FP16, 9)
-    res, _ = o.probe_hashed(A, B, C, 1, 0, 4)
+    C = C + 3.0 * np.sign(np.random.default_rng(3).standard_normal(C.shape))       # noise far above tau
     tau = o.analytic_tau(_np(A), _np(B), 32)
-    cap = tau * math.sqrt(64 * 48 / 16.0)
+    res, S = o.probe_hashed(A, B, C, 1, 0, 4)
+    sig = 1.2533 * np.minimum(np.abs(S), 5.0 * np.abs(S).mean()).mean()
+    assert 4.0 * math.sqrt(2.0 * math.log(16)) * sig > 10.0 * tau               # the noise term is not the minimum
     assert math.isclose(res.tau, tau, rel_tol=1e-12)
-    assert res.thr <= cap * (1 + 1e-12)
+    assert math.isclose(res.thr, tau, rel_tol=1e-12) and res.fired
+    res1, _ = o.probe_hashed(A, B, C, 1, 0, 4, o.Params(scale_cap=1))
+    assert math.isclose(res1.thr, min(tau * math.sqrt(64 * 48 / 16.0), 4.0 * math.sqrt(2.0 * math.log(16)) * sig),
+                        rel_tol=1e-12)
+    assert res1.thr > res.thr
 
 
 @pytest.mark.parametrize("bad", [np.inf, -np.inf, np.nan])

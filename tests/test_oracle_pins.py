@@ -311,3 +311,108 @@ def test_recovery_over_rounds_bound_theorem2():
         assert {(f.i, f.j) for f in F} <= coords
         miss_trials += int(len(F) < s)
     assert miss_trials / trials <= s * 2.0 ** -k
+
+
+# ---------------------------------------------------------------- peeling, pinned directly
+def _fault_only_sketch(faults, h1, v1, h2, v2, m_b, n1, n3):
+    """Sketches of an error matrix that is zero except E_ij = e at the listed (i, j, e):
+    written out term by term, 1-based weights over the next power of two."""
+    p1 = 1
+    while p1 < n1:
+        p1 *= 2
+    p3 = 1
+    while p3 < n3:
+        p3 *= 2
+    S = np.zeros((m_b, m_b))
+    R = np.zeros((m_b, m_b))
+    T = np.zeros((m_b, m_b))
+    for (i, j, e) in faults:
+        sg = v1[i] * v2[j]
+        S[h1[i], h2[j]] += sg * e
+        R[h1[i], h2[j]] += sg * e * (i + 1) / p1
+        T[h1[i], h2[j]] += sg * e * (j + 1) / p3
+    return S, R, T
+
+
+@pytest.mark.parametrize("n1,n3,m_b,seed", [(24, 40, 3, 5), (64, 64, 8, 6), (17, 9, 2, 7)])
+def test_peel_removes_exactly_what_a_confirmed_fault_put_into_the_sketches(n1, n3, m_b, seed):
+    """Algorithm 1, peeling loop; Section "Peeling Across Hash Rounds".  On an exact integer product the
+    sketches hold nothing but the faults, so peeling all of them must leave exact zeros in S, R and T, and
+    peeling a subset must leave the sketches of the others (every value is a dyadic rational: exact)."""
+    n2 = 6
+    A, B, C, _ = _int_case(n1, n2, n3, seed)
+    g = np.random.default_rng(seed)
+    coords = set()
+    row = int(g.integers(n1))
+    while len(coords) < 3:                      # three in one row: some share a row bucket
+        coords.add((row, int(g.integers(n3))))
+    while len(coords) < 7:
+        coords.add((int(g.integers(n1)), int(g.integers(n3))))
+    written = []
+    for t, (i, j) in enumerate(sorted(coords)):
+        d = float((t + 1) * (1 if t % 2 else -1))
+        C[i, j] += d
+        written.append((i, j, d))
+    E = O.error_matrix(A, B, C)
+    for rnd in (0, 1):
+        h1, v1 = O.hash_round(99, rnd, 0, n1, m_b)
+        h2, v2 = O.hash_round(99, rnd, 1, n3, m_b)
+        # the correction of a fault written as C_ij += d is delta = gamma - C_ij = -d
+        F = [O.Fault(i, j, -d, 0.0, 0.0, 0, -1, -1) for (i, j, d) in written]
+        S, R, T = O.moment_sketches(E, h1, v1, h2, v2, m_b)
+        assert np.count_nonzero(S) > 0
+        O.peel(S, R, T, F, h1, v1, h2, v2, n1, n3)
+        assert not S.any() and not R.any() and not T.any()
+        for keep in (1, 3, 6):
+            S, R, T = O.moment_sketches(E, h1, v1, h2, v2, m_b)
+            O.peel(S, R, T, F[keep:], h1, v1, h2, v2, n1, n3)
+            Sx, Rx, Tx = _fault_only_sketch([(i, j, -d) for (i, j, d) in written[:keep]], h1, v1, h2, v2, m_b, n1, n3)
+            assert np.array_equal(S, Sx) and np.array_equal(R, Rx) and np.array_equal(T, Tx)
+
+
+# ---------------------------------------------------------------- normalisation of the noise constant
+def test_noise_constant_normalisation_on_a_known_error_matrix():
+    """Eq. (sigma) normalises the bucket noise as sigma m / (2^-24 sqrt(n1 n2 n3) rms(C)).  Feed the
+    measurement an error matrix of i.i.d. N(0, s^2) entries and a constant C: a bucket that sums c entries
+    is N(0, c s^2), the clipped mean of a Gaussian is its sigma (clipping at 5 mean|x| = 4 sigma removes
+    1e-4), so c_hat has a closed form in s, the bucket populations and the constant."""
+    n1, n2, n3, m0 = 3072, 8, 2048, 160
+    s_e, c0 = 3.0e-4, 2.5
+    g = np.random.default_rng(20)
+    E = s_e * g.standard_normal((n1, n3))
+    A = np.zeros((n1, n2))
+    B = np.zeros((n2, n3))
+    C = np.full((n1, n3), c0, dtype=np.float32)
+    nz = O.measure_noise(A, B, C, seed=5, dtype=O.BF16, m0=m0, E=E)
+    assert nz.m0 == m0 and nz.rms_c == c0
+    h1, _ = O.hash_round(5, 0, 0, n1, m0)
+    h2, _ = O.hash_round(5, 0, 1, n3, m0)
+    pop = np.outer(np.bincount(h1, minlength=m0), np.bincount(h2, minlength=m0)).astype(float)
+    sigma_expected = 1.2533 * math.sqrt(2.0 / math.pi) * s_e * np.sqrt(pop).mean()
+    assert nz.sigma_clip == pytest.approx(sigma_expected, rel=1e-2)
+    c_expected = sigma_expected * m0 / (2.0 ** -24 * math.sqrt(float(n1) * n2 * n3) * c0)
+    assert nz.c_hat == pytest.approx(c_expected, rel=1e-2)
+    # and against the plain population n1 n3 / m0^2 (the sqrt of a varying count loses under 2 %)
+    plain = s_e * math.sqrt(n1 * n3) / (2.0 ** -24 * math.sqrt(float(n1) * n2 * n3) * c0)
+    assert nz.c_hat == pytest.approx(plain, rel=3e-2)
+
+
+# ---------------------------------------------------------------- the tolerance denominators
+def test_abs_product_and_abs_sketch_brute_force():
+    g = np.random.default_rng(8)
+    n1, n2, n3, m_b = 9, 5, 11, 3
+    A = g.integers(-4, 5, (n1, n2)).astype(float)
+    B = g.integers(-4, 5, (n2, n3)).astype(float)
+    h1, _ = O.hash_round(3, 0, 0, n1, m_b)
+    h2, _ = O.hash_round(3, 0, 1, n3, m_b)
+    ABS = O.abs_product(A, B)
+    want = np.zeros((n1, n3))
+    wantS = np.zeros((m_b, m_b))
+    for i in range(n1):
+        for j in range(n3):
+            for k in range(n2):
+                want[i, j] += abs(A[i, k]) * abs(B[k, j])
+            wantS[h1[i], h2[j]] += want[i, j]
+    assert np.array_equal(ABS, want)
+    assert np.array_equal(O.abs_sketch(ABS, h1, h2, m_b), wantS)
+    assert ABS.min() >= 0 and O.abs_sketch(ABS, h1, h2, m_b).sum() == want.sum()
