@@ -314,11 +314,13 @@ int32_t fpsk_max_buckets(int64_t m, int64_t k, int64_t n);
 /* Sum and first-moment sketches of E = AB - C for one hash round (Eq. (S) and the weighted
  * forms R, T of Section "Moment Sketches"), from compressed operands
  * (H1 A)(B H2^T) - H1 C H2^T, without forming AB.  d_S, d_R, d_T: device, n_buckets^2 floats
- * each, row-major [a][b]; d_R and d_T may both be NULL for the S-only form.  Asynchronous. */
+ * each, row-major [a][b]; d_R and d_T may both be NULL for the S-only form.  p (NULL = defaults) selects the
+ * contraction (p->tensor_cores, effective from 384 buckets) and the layout of B (p->b_transposed), as in
+ * fpsk_localize; the workspace is the one fpsk_workspace_bytes sizes for these parameters.  Asynchronous. */
 fpsk_status fpsk_sketches(const void *A, int64_t lda, const void *B, int64_t ldb,
                           const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
                           fpsk_dtype dtype, uint64_t seed, int32_t round, int32_t n_buckets,
-                          void *workspace, size_t ws_bytes, void *stream,
+                          const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream,
                           float *d_S, float *d_R, float *d_T);
 
 /* Run-time noise measurement on a (clean) product: S of round 0 at m0 buckets (m0 <= 0: the

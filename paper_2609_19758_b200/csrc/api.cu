@@ -708,21 +708,27 @@ size_t fpsk_workspace_bytes(int64_t m, int64_t k, int64_t n, int32_t n_buckets, 
 
 fpsk_status fpsk_sketches(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,
                           int64_t m, int64_t k, int64_t n, fpsk_dtype dtype, uint64_t seed, int32_t round,
-                          int32_t n_buckets, void *workspace, size_t ws_bytes, void *stream, float *d_S, float *d_R,
-                          float *d_T)
+                          int32_t n_buckets, const fpsk_params *p, void *workspace, size_t ws_bytes, void *stream,
+                          float *d_S, float *d_R, float *d_T)
 {
-    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype);
+    fpsk_status rc = check_mats(A, lda, B, ldb, C, ldc, m, k, n, dtype, p && p->b_transposed);
     if (rc != FPSK_OK) return rc;
+    const fpsk_params q = resolve_params(p);
+    if (!params_ok(q)) return FPSK_ERR_PARAM;
     if (!workspace || !d_S) return FPSK_ERR_NULL;
     if ((d_R == nullptr) != (d_T == nullptr)) return FPSK_ERR_NULL;
     if (reinterpret_cast<uintptr_t>(workspace) & 255) return FPSK_ERR_ALIGN;
     if (n_buckets < 1 || n_buckets > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     if (round < 0) return FPSK_ERR_PARAM;
-    SketchWs w;
-    if (!sketch_carve(workspace, ws_bytes, m, k, n, n_buckets, w)) return FPSK_ERR_WORKSPACE;
-    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
-    return build_sketches(in, dtype, seed, round, n_buckets, d_R != nullptr, w, static_cast<cudaStream_t>(stream), d_S,
-                          d_R, d_T);
+    LocWs w;
+    if (!loc_carve(workspace, ws_bytes, m, k, n, n_buckets, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
+    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (w.sk.tc) {      // the tensor-core contraction scales its planes by max|A|, max|B|
+        rc = loc_max_ab(in, dtype, w, st);
+        if (rc != FPSK_OK) return rc;
+    }
+    return build_sketches(in, dtype, seed, round, n_buckets, d_R != nullptr, w.sk, st, d_S, d_R, d_T);
 }
 
 fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_t ldb, const float *C, int64_t ldc,

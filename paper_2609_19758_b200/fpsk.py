@@ -131,7 +131,7 @@ def lib() -> C.CDLL:
         L.fpsk_max_buckets.restype = i32
         L.fpsk_max_buckets.argtypes = [i64, i64, i64]
         L.fpsk_sketches.restype = C.c_int
-        L.fpsk_sketches.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32, i32, vp, sz, vp,
+        L.fpsk_sketches.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32, i32, C.POINTER(Params), vp, sz, vp,
                                     vp, vp, vp]
         L.fpsk_measure_noise.restype = C.c_int
         L.fpsk_measure_noise.argtypes = [vp, i64, vp, i64, vp, i64, i64, i64, i64, C.c_int, u64, i32,
@@ -427,12 +427,15 @@ def max_buckets(m: int, k: int, n: int) -> int:
     return int(lib().fpsk_max_buckets(m, k, n))
 
 
-def sketches(A, B, Cm, seed: int, rnd: int, n_buckets: int, ws: torch.Tensor, moments: bool = True, stream=None):
-    a = _mat_args(A, B, Cm)
+def sketches(A, B, Cm, seed: int, rnd: int, n_buckets: int, ws: torch.Tensor, moments: bool = True, stream=None,
+             params: Optional[Params] = None):
+    """With params.b_transposed = 1, B is the weight W = B^T of shape (n, k) (C = A W^T)."""
+    a = _mat_args(A, B, Cm, bool(params is not None and params.b_transposed))
     S = torch.empty((n_buckets, n_buckets), dtype=torch.float32, device=A.device)
     R = torch.empty_like(S) if moments else None
     T = torch.empty_like(S) if moments else None
     rc = lib().fpsk_sketches(a[0], a[1], a[2], a[3], a[4], a[5], a[6], a[7], a[8], a[9], seed, rnd, n_buckets,
+                             C.byref(params) if params is not None else None,
                              ws.data_ptr(), ws.numel(), _stream_ptr(stream), S.data_ptr(),
                              R.data_ptr() if moments else None, T.data_ptr() if moments else None)
     if rc != STATUS_OK:

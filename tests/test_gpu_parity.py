@@ -223,10 +223,14 @@ def test_measure_noise_matches_oracle(n, dtype, kind):
     ref = O.measure_noise(_f64(A), _f64(Bm), Cm.numpy(), 5, dtype, 0, po)
     assert got.m0 == ref.m0
     assert got.rms_c == pytest.approx(ref.rms_c, rel=1e-5)
-    # the GPU estimate contains the verifier's own FP32 rounding on top of the GEMM's: it may
-    # only be larger, and by a bounded factor
-    assert 0.9 * ref.sigma_clip <= got.sigma_clip <= 3.0 * ref.sigma_clip
-    assert 0.8 * ref.sigma_mad <= got.sigma_mad <= 3.0 * ref.sigma_mad
+    # the GPU estimate contains the verifier's own FP32 rounding on top of the GEMM's.  Observed ratios on
+    # these shapes: sigma_clip 1.19 / 1.03 / 1.02, sigma_MAD 1.05 / 1.02 / 1.04 (largest at n = 256, where
+    # the GEMM's own noise is smallest)
+    print("sigma_clip gpu/oracle", got.sigma_clip / ref.sigma_clip, "sigma_mad gpu/oracle", got.sigma_mad / ref.sigma_mad)
+    assert 0.97 * ref.sigma_clip <= got.sigma_clip <= 1.3 * ref.sigma_clip
+    assert 0.97 * ref.sigma_mad <= got.sigma_mad <= 1.3 * ref.sigma_mad
+    # and so the plan drawn from it is the oracle's
+    assert (got.m_loc, got.radius) == (ref.m_loc, ref.radius)
     # the plan is the oracle's plan for the GPU's own measurements (same scalar rule)
     ml, r, Bv = O.plan(n, n, n, dtype, got.sigma_clip, got.rms_c, got.m0, po)
     assert (got.m_loc, got.radius) == (ml, r)

@@ -204,3 +204,81 @@ def test_sigma_mad_is_the_exact_selection_on_the_sketch(m_b, mad_of_abs):
     mad = np.float32(1.4826) * np.partition(dev, rank)[rank]
     nz = fpsk.measure_noise(dA, dB, dC, 9, ws, m_b, p)
     assert np.float32(nz.sigma_mad) == mad
+
+
+# ------------------------------------------------------------------ the sketch builder itself, element by element
+def _sketch_refs(A, Bm, Cm, seed, rnd, m_b):
+    n1, n3 = A.shape[0], Bm.shape[1]
+    A64, B64 = _f64(A), _f64(Bm)
+    E = O.error_matrix(A64, B64, Cm.numpy())
+    h1, v1 = O.hash_round(seed, rnd, 0, n1, m_b)
+    h2, v2 = O.hash_round(seed, rnd, 1, n3, m_b)
+    return O.moment_sketches(E, h1, v1, h2, v2, m_b), O.abs_sketch(O.abs_product(A64, B64), h1, h2, m_b)
+
+
+@pytest.mark.parametrize("shape,m_b,dtype", [((1024, 1024, 1024), 384, W.BF16), ((1536, 520, 1280), 400, W.FP16),
+                                             ((2048, 1032, 4096), 1024, W.BF16), ((4096, 512, 2048), 1024, W.FP16)])
+@pytest.mark.parametrize("b_transposed", [0, 1])
+def test_tensor_core_sketches_element_by_element(shape, m_b, dtype, b_transposed):
+    """S, R and T of the tcgen05 sketch builder (planes written by the compressions, split-K partials, combine)
+    against the oracle's definition, every bucket, for B as k x n and as the weight W = B^T."""
+    n1, n2, n3 = shape
+    A, Bm, Cm = _case("uniform" if dtype == W.FP16 else "gauss_scaled", n1, n2, n3, dtype, 19)
+    Cf, _ = W.inject(Cm, W.faults_additive(n1, n3, W.rms(Cm), 3, 4, 0.02, 1.0, "small"))
+    (So, Ro, To), ABS = _sketch_refs(A, Bm, Cf, 2024, 1, m_b)
+    p = fpsk.default_params(tensor_cores=1, b_transposed=b_transposed)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    dB = Bm.t().contiguous().cuda() if b_transposed else Bm.cuda()
+    S, R, T = fpsk.sketches(A.cuda(), dB, Cf.cuda(), 2024, 1, m_b, ws, params=p)
+    S2, _, _ = fpsk.sketches(A.cuda(), dB, Cf.cuda(), 2024, 1, m_b, ws, moments=False, params=p)
+    torch.cuda.synchronize()
+    for g, o in ((S, So), (R, Ro), (T, To), (S2, So)):
+        assert np.all(np.abs(g.cpu().numpy().astype(np.float64) - o) <= TOL * ABS + 1e-30)
+
+
+@pytest.mark.parametrize("b_transposed", [0, 1])
+def test_tensor_core_sketches_are_bit_exact_on_integer_products(b_transposed):
+    n1, n2, n3, m_b = 768, 264, 640, 384
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 31, lim=8)
+    Cm = W.cpu_fp32_product(A, Bm)
+    Cm[5, 1] += 3.0
+    Cm[767, 639] -= 7.0
+    Cm[300, 630] += 1.0
+    (So, Ro, To), _ = _sketch_refs(A, Bm, Cm, 77, 2, m_b)
+    p = fpsk.default_params(tensor_cores=1, b_transposed=b_transposed)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    dB = Bm.t().contiguous().cuda() if b_transposed else Bm.cuda()
+    S, R, T = fpsk.sketches(A.cuda(), dB, Cm.cuda(), 77, 2, m_b, ws, params=p)
+    for g, o in ((S, So), (R, Ro), (T, To)):
+        assert np.array_equal(g.cpu().numpy().astype(np.float64), o)
+
+
+# ------------------------------------------------------------------ Eq. (recover) with no window to hide behind
+@pytest.mark.parametrize("shape,m_b,tc", [((64, 16, 48), 16, 0), ((300, 40, 520), 64, 0), ((768, 256, 640), 384, 0),
+                                          ((768, 256, 640), 384, 1), ((1000, 72, 1536), 512, 1)])
+@pytest.mark.parametrize("n_faults", [1, 5])
+def test_radius_zero_decodes_the_exact_coordinate(shape, m_b, tc, n_faults):
+    """Exact integer products, radius 0: the only entry ever recomputed for a bucket is the one Eq. (recover)
+    names, so the moments at the kept buckets and the decode must be right to the unit.  The fault list must be
+    the oracle's: coordinates, round, bucket and exact magnitude (faults that collide in every round are missed
+    by both)."""
+    n1, n2, n3 = shape
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 31, lim=8)
+    Cm = W.cpu_fp32_product(A, Bm)
+    g = np.random.default_rng(n1 + n_faults)
+    coords = [(n1 - 1, n3 - 1)] if n_faults == 1 else []
+    while len(coords) < n_faults:
+        c = (int(g.integers(n1)), int(g.integers(n3)))
+        if c not in coords:
+            coords.append(c)
+    faults = [W.InjectedFault(i, j, "add", float((t + 2) * (1 if t % 2 else -1)), "typical") for t, (i, j) in enumerate(coords)]
+    Cf, _ = W.inject(Cm, faults)
+    p = fpsk.default_params(radius=0, tensor_cores=tc)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    got = fpsk.localize(A.cuda(), Bm.cuda(), Cf.cuda(), 4242, m_b, ws, p)
+    ref = O.localize(_f64(A), _f64(Bm), Cf.numpy(), 4242, m_b, W.FP16, O.Params(radius=0))
+    assert [(f.i, f.j, f.delta, f.round, f.bucket_a, f.bucket_b) for f in got] == \
+           [(f.i, f.j, f.delta, f.round, f.bucket_a, f.bucket_b) for f in ref]
+    assert {(f.i, f.j) for f in got} == set(coords)
+    for f in got:
+        assert f.delta == -faults[coords.index((f.i, f.j))].value

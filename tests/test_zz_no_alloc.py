@@ -6,11 +6,14 @@ from a fixed array inside the library.  The test calls the entry point through t
 in a row and checks each result against fpsk_probe with a caller-owned workspace: the kernel
 is the same and its summation order is fixed, so the two must agree bit for bit, which is well
 inside the 1e-5 tolerance the other probe tests use.  The second call runs on a different
-product, so it also shows that nothing stale from the first call leaks into it.
+product, so it also shows that nothing stale from the first call leaks into it.  The residual
+is also held against the definition (column sums of E = AB - C in FP64) like in the other
+probe tests.
 """
 import ctypes as C
 
 import numpy as np
+import oracle as O
 import pytest
 import torch
 
@@ -27,12 +30,13 @@ def _fields(r):
 def test_probe_static_matches_probe_on_two_calls_in_a_row():
     B.build()
     n1, n2, n3 = 512, 768, 1024
-    cases = []
+    cases, hosts = [], []
     for seed in (3, 4):
         A, Bm = W.operands("gauss_scaled", n1, n2, n3, W.BF16, seed)
         dA, dB = A.cuda(), Bm.cuda()
         dC = harness.vendor_gemm_fp32(dA, dB)
         cases.append((dA, dB, dC))
+        hosts.append((A, Bm))
     # the second product carries a fault, so the two calls must give different verdicts
     cases[1][2][17, 33] += 0.25
 
@@ -60,6 +64,14 @@ def test_probe_static_matches_probe_on_two_calls_in_a_row():
         assert float((g_resid - w_resid).abs().max()) <= 1e-5 * scale
         assert torch.equal(g_resid, w_resid)              # same kernel, fixed order: identical
         assert _fields(g) == _fields(w_res)
+    for (A, Bm), (_, _, dC), (g_res, g_resid) in zip(hosts, cases, got):
+        A64, B64 = A.double().numpy(), Bm.double().numpy()
+        E = O.error_matrix(A64, B64, dC.cpu().numpy())
+        abs_j = O.abs_product(A64, B64).sum(axis=0)
+        assert np.all(np.abs(g_resid.cpu().double().numpy() - O.probe_sketch(E)) <= 1e-5 * abs_j)
+        g = fpsk.read_probe_result(g_res)
+        v = O.probe_verdict(O.probe_sketch(E), O.analytic_tau(A64, B64, n2), n_rows=n1)
+        assert bool(g.fired) == v.fired
     assert fpsk.read_probe_result(got[0][0]).fired == 0
     assert fpsk.read_probe_result(got[1][0]).fired == 1 and fpsk.read_probe_result(got[1][0]).argmax_col == 33
 
