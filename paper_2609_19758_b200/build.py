@@ -39,6 +39,8 @@ def build(verbose: bool = False, force: bool = False) -> str:
     cmd = [nvcc_path(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared", "-I", os.path.join(ROOT, "include"),
            "-I", os.path.join(HERE, "csrc")]
+    # extra flags, e.g. FPSK_NVCC_FLAGS=-DFPSK_MEASURE for the build that records in-kernel time stamps
+    cmd += os.environ.get("FPSK_NVCC_FLAGS", "").split()
     if verbose:
         cmd += ["-Xptxas", "-v"]
     cmd += sources() + ["-o", LIB]

@@ -44,10 +44,15 @@ struct ProbeArgs {
 
 __device__ __forceinline__ void trace_mark(const ProbeArgs &p, int c, int k)
 {
+    // SM cycle counter (cheap to read); slots 12 and 13 (kernel entry and exit) also record the global
+    // nanosecond timer in slots 30 and 31, from which the reader calibrates each CTA's cycle counts
     if (p.trace) {
-        unsigned long long t;
-        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-        p.trace[c * 32 + k] = (long long)t;
+        p.trace[c * 32 + k] = clock64();
+        if (k == 12 || k == 13) {
+            unsigned long long t;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+            p.trace[c * 32 + (k == 12 ? 30 : 31)] = (long long)t;
+        }
     }
 }
 
@@ -314,6 +319,14 @@ struct SyncAll {
 struct SyncConsumers {   // named barrier over the 512 consumer threads of the TMA kernel
     static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
 };
+__device__ __forceinline__ void bar_sync_named(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive_named(int id, int count)      // counts this thread in, does not wait
+{
+    asm volatile("bar.arrive %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 
 // Deterministic block reductions over NT threads: xor-shuffle tree inside each warp, then the
 // warp results combined in warp order.  Two barriers each.
@@ -520,11 +533,7 @@ __global__ void __launch_bounds__(kProbeThreads, 2) probe_kernel(const ProbeArgs
 // several hundred cycles), so those parts are short loops with as few dependent global round
 // trips as possible.
 constexpr int kTmaConsumers = 512;
-#ifndef FPSK_TMA_PRODUCERS
-#define FPSK_TMA_PRODUCERS 1
-#endif
-constexpr int kTmaProducers = FPSK_TMA_PRODUCERS;   // producer warps (a second one gains 1 % at 16384^3 and costs 2 us at 4096^3)
-constexpr int kTmaThreads = kTmaConsumers + 32 * kTmaProducers;
+constexpr int kTmaThreads = kTmaConsumers + 32;      // one producer warp (a second one gained 1 % at 16384^3 and cost 2 us at 4096^3)
 constexpr int kStageBytes = 32768;
 constexpr int kStages = 6;
 constexpr int kSegMax = 4096;                 // bytes of one row segment: 256 x 16 B; two row lanes of consumers
@@ -631,7 +640,7 @@ __device__ __forceinline__ void write_verdict(const ProbeArgs &p, float thr_scal
     *p.result = r;
 }
 
-// Verdict in the last CTA.  Warp 0 combines the per-slice statistics (one batch of loads, warp
+// Verdict in the last CTA.  Warp 0 combines the per-slice statistics (one batch of plain loads, warp
 // shuffles, no block barrier) and finishes alone when nothing exceeds the clip level; otherwise
 // all consumers make the second pass over s (staged into shared memory by one bulk copy).
 template <typename T>
@@ -643,26 +652,32 @@ __device__ __forceinline__ void verdict_tma(const ProbeArgs &p, int grid, float 
     float sum = 0.f, bad = 0.f, clip = 0.f;
     ArgMax am = {-1.f, 0x7FFFFFFF};
     if (ctid < 32) {
-        // the per-CTA records (slice statistics, operand maxima) come in by three bulk copies:
-        // one round trip and a few instructions, then a short loop over shared memory
-        float4 *sv = reinterpret_cast<float4 *>(red);
-        unsigned int *sa = reinterpret_cast<unsigned int *>(red + 4 * 512), *sb = sa + 512;
-        const uint32_t mbytes = ((uint32_t)grid * 4u + 15u) & ~15u;
-        if (ctid == 0) {
-            fence_proxy_async();
-            mbar_expect_tx(gbar, (uint32_t)grid * 16u + 2u * mbytes);
-            bulk_g2s(smem_u32(sv), p.vstat, (uint32_t)grid * 16u, gbar);
-            bulk_g2s(smem_u32(sa), p.maxA, mbytes, gbar);
-            bulk_g2s(smem_u32(sb), p.maxB, mbytes, gbar);
-        }
-        mbar_wait_warp(gbar, gpar);
-        for (int g = ctid; g < grid; g += 32) {
-            const float4 st = sv[g];
-            sum += st.x;
-            bad += st.y;
-            am = amax(am, ArgMax{st.z, __float_as_int(st.w)});
-            ma = max(ma, sa[g]);
-            mb = max(mb, sb[g]);
+        // the per-CTA records (slice statistics, operand maxima): plain loads, all of a lane's in flight
+        // together, then combined in index order
+        constexpr int UB = 5;             // one batch for grids of up to 160 CTAs
+        for (int g0 = ctid; g0 < grid; g0 += 32 * UB) {
+            float4 st[UB];
+            unsigned int xa[UB], xb[UB];
+#pragma unroll
+            for (int q = 0; q < UB; ++q) {
+                const int g = g0 + 32 * q;
+                if (g < grid) {
+                    st[q] = __ldcg(p.vstat + g);
+                    xa[q] = __ldcg(p.maxA + g);
+                    xb[q] = __ldcg(p.maxB + g);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < UB; ++q) {
+                const int g = g0 + 32 * q;
+                if (g < grid) {
+                    sum += st[q].x;
+                    bad += st[q].y;
+                    am = amax(am, ArgMax{st[q].z, __float_as_int(st[q].w)});
+                    ma = max(ma, xa[q]);
+                    mb = max(mb, xb[q]);
+                }
+            }
         }
         ma = __reduce_max_sync(0xFFFFFFFFu, ma);
         mb = __reduce_max_sync(0xFFFFFFFFu, mb);
@@ -686,7 +701,6 @@ __device__ __forceinline__ void verdict_tma(const ProbeArgs &p, int grid, float 
             }
         }
     }
-    gpar ^= 1u;                 // warp 0 has used one phase of gbar; every thread tracks it
     SyncConsumers::sync();
     if (!*s_slow) return;
     // some entry exceeds the clip level (or is not finite): second pass over all of s
@@ -735,20 +749,18 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
     const int tid = threadIdx.x;
     if (tid == 0) trace_mark(p, c, 12);
     const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kStages), gbar = smem_u32(bars + 2 * kStages);
-    if (tid == 0) {
+    // The producer warp sets up the barriers itself, counts itself in at the set-up barrier (id 3) without
+    // waiting and starts copying at once; the consumers wait there before they touch a barrier of the ring.
+    if (tid == kTmaConsumers) {
         for (int s = 0; s < kStages; ++s) {
             mbar_init(full0 + 8 * s, 1);
             mbar_init(empty0 + 8 * s, kTmaConsumers / 32);
         }
         mbar_init(gbar, 1);
-        s_err = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    // With programmatic dependent launch this kernel may start while its predecessor in the
-    // stream is still draining; nothing produced by earlier work is touched before this point.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    __syncthreads();
+    if (tid == 0) s_err = 0;
 
     Piece pc[3];
     pc[0] = make_piece(p.A, p.lda, p.n2 * 2, 2, a.tA, c);
@@ -765,8 +777,8 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
         // Both walk the same sequence of stages; warp w fills the stages whose running number is
         // congruent to w, so two streams of copy instructions are in flight.
         const int lane = tid & 31;
-        const int pw = (tid - kTmaConsumers) >> 5;
-        unsigned int nstage = 0;
+        __syncwarp();                     // lane 0's barrier set-up before any lane's copy names a barrier
+        bar_arrive_named(3, kTmaThreads);
         int stage = 0;
         uint32_t phase = 0;
         bool ok = true;
@@ -782,20 +794,18 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                 fence_proxy_async();
                 for (int t0 = 0; t0 < ngA && ok; t0 += ut_rows) {
                     const int nt = min(ut_rows, ngA - t0);
-                    if ((nstage++ % kTmaProducers) == (unsigned)pw) {
-                        w = 1;
-                        if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
-                        w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                        if (!w) { ok = false; break; }
-                        if (lane == 0) {
-                            // this row group's block of partA is [ngA][ucnt]: rows t0..t0+nt are contiguous
-                            const uint32_t bytes = (uint32_t)nt * (uint32_t)ucnt * 4u;
-                            mbar_expect_tx(full0 + 8 * stage, bytes);
-                            bulk_g2s(smem_u32(ring + (size_t)stage * kStageBytes),
-                                     p.partA + (long long)pc[2].r0 * ngA + (long long)t0 * ucnt, bytes, full0 + 8 * stage);
-                        }
-                        __syncwarp();
+                    w = 1;
+                    if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                    w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                    if (!w) { ok = false; break; }
+                    if (lane == 0) {
+                        // this row group's block of partA is [ngA][ucnt]: rows t0..t0+nt are contiguous
+                        const uint32_t bytes = (uint32_t)nt * (uint32_t)ucnt * 4u;
+                        mbar_expect_tx(full0 + 8 * stage, bytes);
+                        bulk_g2s(smem_u32(ring + (size_t)stage * kStageBytes),
+                                 p.partA + (long long)pc[2].r0 * ngA + (long long)t0 * ucnt, bytes, full0 + 8 * stage);
                     }
+                    __syncwarp();
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -803,18 +813,16 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
             if (!q.has) continue;
             for (int row = q.r0; row < q.r1 && ok; row += q.tr) {
                 const int nr = min(q.tr, q.r1 - row);
-                if ((nstage++ % kTmaProducers) == (unsigned)pw) {
-                    int w = 1;
-                    if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
-                    w = __shfl_sync(0xFFFFFFFFu, w, 0);
-                    if (!w) { ok = false; break; }
-                    if (lane == 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)nr * (uint32_t)q.wbytes);
-                    __syncwarp();
-                    const uint32_t dst0 = smem_u32(ring + (size_t)stage * kStageBytes);
-                    for (int r = lane; r < nr; r += 32)
-                        bulk_g2s(dst0 + (uint32_t)r * (uint32_t)q.segb, q.base + (long long)(row + r) * q.ldb, (uint32_t)q.wbytes,
-                                 full0 + 8 * stage);
-                }
+                int w = 1;
+                if (lane == 0) w = mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u) ? 1 : 0;
+                w = __shfl_sync(0xFFFFFFFFu, w, 0);
+                if (!w) { ok = false; break; }
+                if (lane == 0) mbar_expect_tx(full0 + 8 * stage, (uint32_t)nr * (uint32_t)q.wbytes);
+                __syncwarp();
+                const uint32_t dst0 = smem_u32(ring + (size_t)stage * kStageBytes);
+                for (int r = lane; r < nr; r += 32)
+                    bulk_g2s(dst0 + (uint32_t)r * (uint32_t)q.segb, q.base + (long long)(row + r) * q.ldb, (uint32_t)q.wbytes,
+                             full0 + 8 * stage);
                 if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
         }
@@ -861,6 +869,7 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
                 }
             }
         }
+        bar_sync_named(3, kTmaThreads);          // the ring's barriers are set up, s_err is written
         if (ctid == 0) trace_mark(p, c, 0);
 #pragma unroll
         for (int m = 0; m < 3; ++m) {
@@ -1049,39 +1058,40 @@ __global__ void __launch_bounds__(kTmaThreads, 1) probe_tma_kernel(const TmaArgs
             const int nsub = jn <= kTmaConsumers ? kTmaConsumers / uw : 1;
             const int sub = jn <= kTmaConsumers ? ctid / uw : 0;
             const int kk = jn <= kTmaConsumers ? ctid - sub * uw : ctid;
-            constexpr int kData = kGatherFloats - 2 * kTmaConsumers;    // staging; the tail of `red` holds the sub-sums
-            const int tmax = jn > 0 ? kData / jn : ntot;                 // partial rows per pass (>= 1: jn <= 1024)
+            // Plain coalesced loads straight from L2 (the block of a slice is contiguous): every thread has its
+            // few rows in flight together.  A bulk copy into shared memory of the same block took longer
+            // (proxy fence, copy engine, barrier).
             float sp0 = 0.f, sc0 = 0.f, sp1 = 0.f, sc1 = 0.f;
-            for (int t0 = 0; t0 < ntot && jn > 0; t0 += tmax) {
-                const int nt = min(tmax, ntot - t0);
-                if (ctid == 0) {
-                    fence_proxy_async();
-                    const uint32_t bytes = (uint32_t)nt * (uint32_t)jn * 4u;
-                    mbar_expect_tx(gbar, bytes);
-                    bulk_g2s(smem_u32(red), blk + (long long)t0 * jn, bytes, gbar);
-                }
-                const bool got = mbar_wait_warp(gbar, gpar);
-                gpar ^= 1u;
-                if (!got) s_err = 1;
-                if (kk < jn) {
-                    int t = (sub - t0 % nsub + nsub) % nsub;              // global row t0 + t is congruent to sub
-#pragma unroll 4
-                    for (; t < nt; t += nsub) {
-                        const float v = red[t * jn + kk];
-                        if (t0 + t < ngP) sp0 += v; else sc0 += v;
+            if (kk < jn) {
+                constexpr int UB = 8;
+                for (int t0 = sub; t0 < ntot; t0 += UB * nsub) {
+                    float v[UB];
+#pragma unroll
+                    for (int q = 0; q < UB; ++q) {
+                        const int t = t0 + q * nsub;
+                        v[q] = t < ntot ? __ldcg(blk + (long long)t * jn + kk) : 0.f;
+                    }
+#pragma unroll
+                    for (int q = 0; q < UB; ++q) {
+                        const int t = t0 + q * nsub;
+                        if (t < ntot) { if (t < ngP) sp0 += v[q]; else sc0 += v[q]; }
                     }
                 }
-                if (kk + kTmaConsumers < jn) {
-#pragma unroll 4
-                    for (int t = 0; t < nt; ++t) {
-                        const float v = red[t * jn + kk + kTmaConsumers];
-                        if (t0 + t < ngP) sp1 += v; else sc1 += v;
-                    }
+            }
+            if (kk + kTmaConsumers < jn) {
+                constexpr int UB = 8;
+                for (int t0 = 0; t0 < ntot; t0 += UB) {
+                    float v[UB];
+#pragma unroll
+                    for (int q = 0; q < UB; ++q)
+                        v[q] = t0 + q < ntot ? __ldcg(blk + (long long)(t0 + q) * jn + kk + kTmaConsumers) : 0.f;
+#pragma unroll
+                    for (int q = 0; q < UB; ++q)
+                        if (t0 + q < ntot) { if (t0 + q < ngP) sp1 += v[q]; else sc1 += v[q]; }
                 }
-                SyncConsumers::sync();
             }
             if (nsub > 1) {
-                float *tmp = red + kData;
+                float *tmp = red + 1024;       // clear of the per-warp statistics records at the head of `red`
                 tmp[sub * uw + kk] = sp0;
                 tmp[kTmaConsumers + sub * uw + kk] = sc0;
                 SyncConsumers::sync();
@@ -1314,9 +1324,12 @@ fpsk_status probe_launch(const void *A, const void *B, const float *C, const Pro
     p.maxB = reinterpret_cast<unsigned int *>(w); w += align_up((size_t)kMaxGrid * 4, 256);
     p.s = d_residual ? d_residual : reinterpret_cast<float *>(w);
     w += align_up((size_t)d.n3 * 4, 256);
-    // FPSK_PROBE_TRACE=1 records per-CTA phase timestamps in the workspace tail (a measurement aid)
+    p.trace = nullptr;
+#ifdef FPSK_MEASURE
+    // measurement build only: FPSK_PROBE_TRACE=1 records per-CTA phase stamps in the workspace
     static const bool want_trace = [] { const char *e = getenv("FPSK_PROBE_TRACE"); return e && e[0] == '1'; }();
-    p.trace = want_trace ? reinterpret_cast<long long *>(w) : nullptr;
+    if (want_trace) p.trace = reinterpret_cast<long long *>(w);
+#endif
     w += (size_t)kMaxGrid * 32 * 8;
     p.vstat = reinterpret_cast<float4 *>(w);
     p.result = d_result;
@@ -1326,8 +1339,12 @@ fpsk_status probe_launch(const void *A, const void *B, const float *C, const Pro
                        reinterpret_cast<uintptr_t>(C)) & 15) == 0 &&
                      d.lda % 8 == 0 && d.ldb % 8 == 0 && d.ldc % 4 == 0 && d.n2 % 8 == 0 &&
                      d.n3 % 8 == 0;
-    // FPSK_PROBE_PLAIN=1 forces the plain-load kernel (a measurement aid)
-    static const bool force_plain = [] { const char *e = getenv("FPSK_PROBE_PLAIN"); return e && e[0] == '1'; }();
+    bool force_plain = false;
+#ifdef FPSK_MEASURE
+    // measurement build only: FPSK_PROBE_PLAIN=1 forces the plain-load kernel
+    static const bool env_plain = [] { const char *e = getenv("FPSK_PROBE_PLAIN"); return e && e[0] == '1'; }();
+    force_plain = env_plain;
+#endif
     if (vec && !force_plain) {
         int grid = 0;
         fpsk_status rc = tma_grid(grid);
@@ -1341,24 +1358,8 @@ fpsk_status probe_launch(const void *A, const void *B, const float *C, const Pro
             void *args[] = {&ta};
             const void *fn = dtype == FPSK_FP16 ? (const void *)probe_tma_kernel<__half>
                                                 : (const void *)probe_tma_kernel<__nv_bfloat16>;
-            // FPSK_PROBE_PDL=1: programmatic dependent launch instead of a cooperative launch (measurement aid)
-            static const bool pdl = [] { const char *e = getenv("FPSK_PROBE_PDL"); return e && e[0] == '1'; }();
-            if (pdl) {
-                cudaLaunchConfig_t cfg;
-                memset(&cfg, 0, sizeof(cfg));
-                cfg.gridDim = dim3(grid);
-                cfg.blockDim = dim3(kTmaThreads);
-                cfg.dynamicSmemBytes = kTmaSmem;
-                cfg.stream = st;
-                cudaLaunchAttribute at[1];
-                at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-                at[0].val.programmaticStreamSerializationAllowed = 1;
-                cfg.attrs = at;
-                cfg.numAttrs = 1;
-                FPSK_CUDA_OK(cudaLaunchKernelExC(&cfg, fn, args));
-            } else {
-                FPSK_CUDA_OK(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kTmaThreads), args, kTmaSmem, st));
-            }
+            // cooperative: the CTAs wait on one another's partial sums, so all of them must be resident
+            FPSK_CUDA_OK(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(kTmaThreads), args, kTmaSmem, st));
             FPSK_LAUNCH_CHECK();
             return FPSK_OK;
         }
@@ -1382,3 +1383,15 @@ fpsk_status probe_launch(const void *A, const void *B, const float *C, const Pro
 }
 
 }  // namespace fpsk
+
+#ifdef FPSK_MEASURE
+// measurement build only: where the phase stamps of the probe kernel sit in its workspace
+// ([CTA][32] 64-bit words), for the script that reads them
+extern "C" size_t fpsk_probe_trace_offset(int64_t m, int64_t k, int64_t n)
+{
+    using namespace fpsk;
+    (void)m;
+    return 256 + align_up(part_floats(k, 8) * 4, 256) + align_up(part_floats(n, 8) * 4, 256) + align_up(part_floats(n, 4) * 4, 256) +
+           2 * align_up((size_t)kMaxGrid * 4, 256) + align_up((size_t)n * 4, 256);
+}
+#endif
