@@ -2,17 +2,22 @@
 """Benchmark of the FP-Sketch verifier hot path on B200.
 
 One step = one pass of the whole path over one batch of synthetic input:
-    probe (detection sketch + verdict)  ->  run-time noise measurement on the clean product
+    probe of the clean product (detection sketch + verdict; the clean-path cost)
+    ->  run-time noise measurement on the clean product (bucket count and radius)
+    ->  probe of the faulty product (must fire)
     ->  localization of the injected faults (hash rounds, candidates, FP64 confirmation).
-Workload: square BF16 product m=k=n=4096, A ~ N(0,1), B ~ N(0, sd 1/sqrt(k)), FP32 C from the
-vendor GEMM, 4 additive faults of 2-9 % of rms(C) per batch; batches rotate so that no input
-is served from L2, and a 256 MiB read flushes L2 before every probe.
+Headline workload: the largest shape of the clean-path sweep, the square BF16 product m=k=n=16384 with
+A, B ~ N(0,1) and FP32 C from the vendor GEMM (2.1 GB read per probe), 4 additive faults of 2-9 % of rms(C)
+in the faulty copy; two input batches rotate (each is larger than L2) and a 256 MiB read flushes L2 before
+every probe.  The same JSON line carries the sweep over the other square sizes and both operand types
+(probe time per launch and back to back, GB/s, fraction of the copy peak, vendor GEMM, noise constant, plan,
+fitted exponent), a short recovery campaign split by fault population, and the CPU oracle's time for the
+probe and for the localization leg.
 
-Prints ONE JSON line.  The headline metric is the clean-path probe's HBM throughput
-(algorithmic bytes 2mk + 2kn + 4mn over the probe kernel's device time); probe ms, vendor
-GEMM ms, localize ms, recovery and the measured noise constant ride along.
+Prints ONE JSON line.  The headline metric is the clean-path probe's HBM throughput (algorithmic bytes
+2mk + 2kn + 4mn over the probe kernel's device time).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--shape m,k,n] [--dtype bf16|fp16]
 """
 from __future__ import annotations
 
@@ -38,17 +43,21 @@ FALLBACK_HBM_GBS = 6650.0
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--shape", default="4096,4096,4096", help="m,k,n (default: the benchmark configuration)")
+    ap.add_argument("--shape", default="16384,16384,16384", help="m,k,n (default: the largest square of the clean-path sweep)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16"])
-    ap.add_argument("--kind", default="gauss_scaled")
-    ap.add_argument("--sets", type=int, default=3, help="rotating input batches")
+    ap.add_argument("--kind", default="gauss", choices=["gauss", "gauss_scaled", "uniform", "transformer"],
+                    help="operand recipe (gauss: A, B ~ N(0,1), the clean-path sweep's)")
+    ap.add_argument("--sets", type=int, default=0, help="rotating input batches (0: 2 above 1 GB per batch, else 3)")
+    ap.add_argument("--sweep", default="1024,2048,4096,8192,16384", help="square sizes of the clean-path sweep in the same line ('' to skip)")
+    ap.add_argument("--campaign", default="short", choices=["none", "short", "full"],
+                    help="recovery campaign by fault population: short = a bounded subset of the configurations")
     ap.add_argument("--probe-only", action="store_true", help="time only the probe (profiling aid)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tensor-cores", type=int, default=1, choices=[0, 1],
-                    help="contraction of the moment sketches: 1 = split-BF16 tcgen05 (bucket counts >= 384), 0 = FP32 FMA")
+                    help="contraction of the moment sketches: 1 = split-FP16 tcgen05 (bucket counts >= 384), 0 = FP32 FMA")
     ap.add_argument("--probe-buckets", type=int, default=256, help="bucket count of the S only probe leg (0: skip it)")
     return ap.parse_args()
 
@@ -120,25 +129,52 @@ def algorithmic_bytes(m, k, n):
     return 2 * m * k + 2 * k * n + 4 * m * n
 
 
+RECIPES = {
+    "gauss": "A, B ~ N(0,1)",
+    "gauss_scaled": "A ~ N(0,1), B ~ N(0, 1/sqrt(k))",
+    "uniform": "A, B ~ U(-1,1)",
+    "transformer": "A ~ N(0,1), B ~ N(0, sd 0.02)",
+}
+
+
+def draw_operands(kind, m, k, n, td, seed):
+    """Seeded operands drawn on the device (the largest case is 1 GB of operands): same recipes as the host
+    generators of the tests, torch's generator instead of numpy's."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(0x5EED0000 + seed)
+    if kind == "uniform":
+        A = (torch.rand(m, k, device="cuda", generator=g) * 2 - 1).to(td)
+        B = (torch.rand(k, n, device="cuda", generator=g) * 2 - 1).to(td)
+    else:
+        A = torch.randn(m, k, device="cuda", generator=g).to(td)
+        B = torch.randn(k, n, device="cuda", generator=g)
+        if kind == "gauss_scaled":
+            B = B * (1.0 / k ** 0.5)
+        elif kind == "transformer":
+            B = B * 0.02
+        B = B.to(td)
+    return A, B
+
+
 def make_batches(args, m, k, n, dt, nsets, seed0=0):
     from paper_2609_19758_b200 import harness, workloads as W
+    td = W.TORCH_DTYPE[dt]
     batches = []
     for s in range(nsets):
-        A, B = W.operands(args.kind, m, k, n, dt, seed0 + s)
-        dA, dB = A.cuda(), B.cuda()
+        dA, dB = draw_operands(args.kind, m, k, n, td, seed0 + s)
         C = harness.vendor_gemm_fp32(dA, dB)
-        rms = float(torch.sqrt(torch.mean(C.double() ** 2)))
+        rms = float(torch.sqrt(torch.mean(C[:: max(1, m // 2048)].double() ** 2)))
         faults = W.faults_additive(m, n, rms, seed0 + s, 4, 0.02, 0.09, "small")
         Cf = C.clone()
         for f in faults:
             Cf[f.i, f.j] += f.value
-        batches.append(dict(A=dA, B=dB, C=C, Cf=Cf, faults=faults, rms=rms, hA=A, hB=B))
+        batches.append(dict(A=dA, B=dB, C=C, Cf=Cf, faults=faults, rms=rms))
     return batches
 
 
 def run_ours(args):
     from paper_2609_19758_b200 import build as Bld
-    from paper_2609_19758_b200 import fpsk, harness, replicas, workloads as W
+    from paper_2609_19758_b200 import campaign, fpsk, harness, replicas, sweep, workloads as W
 
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -158,25 +194,27 @@ def run_ours(args):
     m, k, n = (int(x) for x in args.shape.split(","))
     dt = W.BF16 if args.dtype == "bf16" else W.FP16
     K, Wm = args.steps, max(args.warmup, 3)
-    nsets = max(args.sets, 3 if algorithmic_bytes(m, k, n) < 512e6 else 2)
+    nbytes = algorithmic_bytes(m, k, n)
+    nsets = args.sets if args.sets > 0 else (2 if nbytes > 1e9 else 3)
     batches = make_batches(args, m, k, n, dt, nsets, seed0=100 * rank)
     params = fpsk.default_params(s_budget=4, tensor_cores=args.tensor_cores)
     pws = fpsk.probe_workspace(m, k, n)
     res = fpsk.new_probe_result()
+    res_f = fpsk.new_probe_result()
     resid = torch.empty(n, dtype=torch.float32, device="cuda")
     # workspace sized for the largest bucket count the plan can ask for
     mb_cap = min(fpsk.max_buckets(m, k, n), max(16, int((m * n // 16) ** 0.5)))
     mb_cap = max(mb_cap, fpsk.law_m_start(m, k, n, dt, params))
     ws = fpsk.workspace(m, k, n, mb_cap, params)
     flush = torch.zeros(64 << 20, dtype=torch.int32, device="cuda")     # 256 MiB, read (not written) to evict L2
-    nbytes = algorithmic_bytes(m, k, n)
 
     ev = lambda: torch.cuda.Event(enable_timing=True)
     pe = [(ev(), ev()) for _ in range(K)]
+    fe = [(ev(), ev()) for _ in range(K)]
     ne = [(ev(), ev()) for _ in range(K)]
     le = [(ev(), ev()) for _ in range(K)]
     t0, t1 = ev(), ev()
-    found = injected = false_pos = fired_n = 0
+    found = injected = false_pos = fired_faulty = fired_clean = 0
     c_hats, plans = [], []
     launches0 = 0
     sampler = None
@@ -190,23 +228,31 @@ def run_ours(args):
             t0.record()
         b = batches[s % nsets]
         i = s - Wm
-        flush_sink = flush.max()                        # a 256 MiB READ evicts the inputs from L2 and leaves no dirty lines
+        flush.max()                                     # a 256 MiB READ evicts the inputs from L2 and leaves no dirty lines
         if i >= 0:
             pe[i][0].record()
-        fpsk.probe(b["A"], b["B"], b["Cf"], pws, res, resid, params)
+        fpsk.probe(b["A"], b["B"], b["C"], pws, res, resid, params)          # the clean path: this is the timed probe
         if i >= 0:
             pe[i][1].record()
         if args.probe_only:
             continue
-        verdict = fpsk.read_probe_result(res)           # the one host read of the verdict
         if i >= 0:
             ne[i][0].record()
         nz = fpsk.measure_noise(b["A"], b["B"], b["C"], 1000 + s, ws, 0, params)
         if i >= 0:
             ne[i][1].record()
+        clean = fpsk.read_probe_result(res)
+        flush.max()
+        if i >= 0:
+            fe[i][0].record()
+        fpsk.probe(b["A"], b["B"], b["Cf"], pws, res_f, None, params)        # the product under test: must fire
+        if i >= 0:
+            fe[i][1].record()
+        verdict = fpsk.read_probe_result(res_f)         # the one host read of the verdict
+        if i >= 0:
             le[i][0].record()
         params.radius = nz.radius
-        got = fpsk.localize(b["A"], b["B"], b["Cf"], 1000 + s, min(nz.m_loc, mb_cap), ws, params)
+        got = fpsk.localize(b["A"], b["B"], b["Cf"], 1000 + s, min(nz.m_loc, mb_cap), ws, params) if verdict.fired else []
         if i >= 0:
             le[i][1].record()
             want = {(f.i, f.j) for f in b["faults"]}
@@ -214,7 +260,8 @@ def run_ours(args):
             found += len(want & have)
             injected += len(want)
             false_pos += len(have - want)
-            fired_n += int(verdict.fired)
+            fired_faulty += int(verdict.fired)
+            fired_clean += int(clean.fired)
             c_hats.append(nz.c_hat)
             plans.append((nz.m0, nz.m_loc, nz.radius))
     t1.record()
@@ -225,33 +272,22 @@ def run_ours(args):
     clocks = sampler.stop() if sampler else None
     total_ms = t0.elapsed_time(t1)
     probe_ms = [a.elapsed_time(b_) for a, b_ in pe]
+    faulty_ms = [a.elapsed_time(b_) for a, b_ in fe] if not args.probe_only else [0.0]
     noise_ms = [a.elapsed_time(b_) for a, b_ in ne] if not args.probe_only else [0.0]
     loc_ms = [a.elapsed_time(b_) for a, b_ in le] if not args.probe_only else [0.0]
     probe_mean = sum(probe_ms) / len(probe_ms)
 
-    # the same probe launched back to back over the rotating batches (each batch is larger than L2, so every
-    # launch still reads its operands from HBM): one event pair around the burst, i.e. the launch duration
-    # without the per-launch cost of an event pair (an empty kernel between two events reads about 6 us here)
+    # the same probe back to back from a CUDA graph over the rotating batches (each larger than L2): the launch
+    # duration without the per-launch cost of an event pair (an empty kernel between two events reads 5-6 us here)
     burst_ms = None
-    if nsets >= 3 and algorithmic_bytes(m, k, n) >= 128e6:
-        Kb = max(30, min(K, 120))
-        for q in range(nsets):
-            fpsk.probe(batches[q]["A"], batches[q]["B"], batches[q]["Cf"], pws, res, resid, params)
-        torch.cuda.synchronize()
-        b0, b1 = ev(), ev()
-        b0.record()
-        for q in range(Kb):
-            bq = batches[q % nsets]
-            fpsk.probe(bq["A"], bq["B"], bq["Cf"], pws, res, resid, params)
-        b1.record()
-        torch.cuda.synchronize()
-        burst_ms = b0.elapsed_time(b1) / Kb
+    if nbytes >= 128e6:
+        burst_ms = sweep._burst(lambda q: (lambda: fpsk.probe(batches[q]["A"], batches[q]["B"], batches[q]["C"], pws, res, resid, params)),
+                                nsets, launches=30 if nbytes < 1e9 else 12)
 
     # vendor GEMM under test, timed alongside (not part of the product)
     g0, g1 = ev(), ev()
-    b = batches[0]
     for _ in range(3):
-        harness.vendor_gemm_fp32(b["A"], b["B"])
+        harness.vendor_gemm_fp32(batches[0]["A"], batches[0]["B"])
     torch.cuda.synchronize()
     g0.record()
     for q in range(10):
@@ -268,15 +304,15 @@ def run_ours(args):
         mb = args.probe_buckets
         hps = [fpsk.HashedProbe(m, k, n, mb, seed=77) for _ in range(nsets)]
         hres = fpsk.new_probe_result()
-        fired_clean = fired_faulty = 0
+        hfired_clean = hfired_faulty = 0
         for q in range(nsets):                          # builds every B side; also the detection check
             hps[q](batches[q]["A"], batches[q]["B"], batches[q]["C"], hres)
             torch.cuda.synchronize()
             r_clean = fpsk.read_probe_result(hres)
             hps[q](batches[q]["A"], batches[q]["B"], batches[q]["Cf"], hres)
             torch.cuda.synchronize()
-            fired_clean += int(r_clean.fired)
-            fired_faulty += int(fpsk.read_probe_result(hres).fired)
+            hfired_clean += int(r_clean.fired)
+            hfired_faulty += int(fpsk.read_probe_result(hres).fired)
         Kh = min(K, 50)
         he = [(ev(), ev()) for _ in range(Kh)]
         for q in range(Kh + 3):
@@ -313,24 +349,27 @@ def run_ours(args):
         hbytes = 2 * m * k + 4 * m * n
         hashed = {"n_buckets": mb, "ms": hms, "bytes_per_call": hbytes, "gbs": hbytes / (hms * 1e-3) / 1e9,
                   "over_gemm": hms / gemm_ms, "sigma_hat": r_clean.sigma_hat, "thr": r_clean.thr,
-                  "fired_on_clean": fired_clean, "fired_on_faulty": fired_faulty, "batches": nsets,
+                  "fired_on_clean": hfired_clean, "fired_on_faulty": hfired_faulty, "batches": nsets,
                   "b_side_rebuilds": sum(h.side.rebuilds for h in hps), "kernels_per_call": 3,
                   "graph_replay_ms": gms,
                   "state_after_replays": {"calls": hst.calls, "clean_calls": hst.clean_calls, "fired_any": hst.fired_any,
                                           "sigma_bar": (hst.sigma_sum / hst.clean_calls) if hst.clean_calls else None}}
+        del hps, graphs
 
-    # end to end through the C ABI with HOST buffers: H2D of A, B, C and D2H of the verdict inside
+    # end to end through the C ABI with HOST buffers: H2D of A, B, C and D2H of the verdict inside the timed region
     hws = fpsk.probe_host_workspace(m, k, n)
-    hb = [dict(A=x["hA"].pin_memory(), B=x["hB"].pin_memory(), C=x["Cf"].cpu().pin_memory()) for x in batches[:2]]
-    Ke = min(K, 20)
+    nhost = 1 if nbytes > 1e9 else 2
+    hb = [dict(A=x["A"].cpu().pin_memory(), B=x["B"].cpu().pin_memory(), C=x["C"].cpu().pin_memory()) for x in batches[:nhost]]
+    Ke = min(K, 5 if nbytes > 1e9 else 20)
     for q in range(2):
-        fpsk.probe_host(hb[q % 2]["A"], hb[q % 2]["B"], hb[q % 2]["C"], hws, params)
+        fpsk.probe_host(hb[q % nhost]["A"], hb[q % nhost]["B"], hb[q % nhost]["C"], hws, params)
     torch.cuda.synchronize()
     w0 = time.perf_counter()
     for q in range(Ke):
-        r_ = fpsk.probe_host(hb[q % 2]["A"], hb[q % 2]["B"], hb[q % 2]["C"], hws, params)
+        fpsk.probe_host(hb[q % nhost]["A"], hb[q % nhost]["B"], hb[q % nhost]["C"], hws, params)
     torch.cuda.synchronize()
     e2e_ms = (time.perf_counter() - w0) * 1e3 / Ke
+    del hws
 
     # max over ranks (replicas only: no data-path collective)
     probe_mean_x, step_ms_x, e2e_ms_x = replicas.max_over_ranks([probe_mean, total_ms / K, e2e_ms], dist, device="cuda")
@@ -356,55 +395,107 @@ def run_ours(args):
         "data": "synthetic",
         "config": {
             "workload": f"square {args.dtype.upper()} product m=k=n={m}" if m == k == n else f"{m}x{k}x{n} {args.dtype}",
-            "recipe": f"{args.kind}: A~N(0,1), B~N(0,1/sqrt(k)); FP32 C from the vendor GEMM; 4 faults of 2-9% rms(C) per batch",
-            "step": "probe + noise measurement (clean C) + localize (3 hash rounds, FP64 confirm)",
-            "contraction": "split-BF16 tcgen05 at >= 384 buckets, FP32 FMA below" if args.tensor_cores else "FP32 FMA",
-            "l2": f"256 MiB flush read before every probe; {nsets} rotating input batches (each 134 MB > L2)",
+            "recipe": f"{args.kind}: {RECIPES[args.kind]}, drawn on the device (seeded); FP32 C from the vendor GEMM; "
+                      "the faulty copy carries 4 additive faults of 2-9% rms(C)",
+            "step": "probe (clean product) + noise measurement + probe (faulty product) + localize (3 hash rounds, FP64 confirm)",
+            "contraction": "split-FP16 tcgen05 at >= 384 buckets, FP32 FMA below" if args.tensor_cores else "FP32 FMA",
+            "l2": f"256 MiB flush read before every probe; {nsets} rotating input batches ({nbytes / 1e6:.0f} MB each > L2)",
             "parallelism": "replicas only" if world > 1 else "single GPU",
+            "also_in_this_line": "sweep: the other square sizes and FP16; recovery_by_population: short campaign",
         },
         "probe_ms": probe_mean_x,
         "probe_ms_median": statistics.median(probe_ms),
         "probe_ms_min": min(probe_ms),
         "probe_ms_burst": burst_ms,
+        "probe_faulty_ms": statistics.median(faulty_ms),
         "gemm_ms": gemm_ms,
         "probe_over_gemm": probe_mean_x / gemm_ms,
         "measure_noise_ms": statistics.median(noise_ms),
         "localize_ms": statistics.median(loc_ms),
         "recovery": {"found": found, "injected": injected, "rate": (found / injected) if injected else None,
-                     "false_positives": false_pos, "probe_fired": fired_n, "steps": K},
+                     "false_positives": false_pos, "probe_fired_on_faulty": fired_faulty, "probe_fired_on_clean": fired_clean,
+                     "steps": K},
         "noise": {"c_hat_median": statistics.median(c_hats) if c_hats else None,
                   "plan_m0_mloc_r": list(plans[len(plans) // 2]) if plans else None},
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peak, "unit": "GB/s", "frac": gbs / peak,
                      "peak_source": peak_src + " copy bandwidth (MEASURED_PEAKS.json)" if peak_src == "measured" else "fallback 6650",
                      "frac_of_nominal_8TBs": gbs / 8000.0, "kernel": "probe_tma_kernel", "bytes_per_launch": nbytes,
-                     "traffic": None,
+                     "traffic": None, "traffic_source": None,
                      "achieved_burst": (nbytes / (burst_ms * 1e-3) / 1e9) if burst_ms else None,
                      "frac_burst": (nbytes / (burst_ms * 1e-3) / 1e9 / peak) if burst_ms else None,
-                     "note": "achieved/frac: one CUDA-event pair per launch, L2 flushed by a read before each; "
-                             "*_burst: launches back to back over rotating batches larger than L2, one event pair"},
+                     "note": "achieved/frac: one CUDA-event pair per launch inside the timed step loop, L2 flushed by a read "
+                             "before each; *_burst: launches back to back from a CUDA graph over rotating batches larger than L2"},
         "e2e": {"value": replicas.whole_job_throughput(nbytes / 1e9, e2e_ms_x * 1e-3, world), "unit": "GB/s", "ms": e2e_ms_x,
                 "h2d_bytes_per_step": nbytes, "d2h_bytes_per_step": 32},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
     if hashed is not None:
-        peak_h, _ = measured_peak()
-        hashed["frac_of_copy_peak"] = hashed["gbs"] / peak_h
+        hashed["frac_of_copy_peak"] = hashed["gbs"] / peak
         out["hashed_probe"] = hashed
-    # DRAM traffic per launch of the probe kernel, from the committed ncu summary (text, "key bytes")
+    # DRAM traffic per launch of the probe kernel: not measurable inside the run; the figure of the committed ncu
+    # capture of the same kernel (a text file, "key bytes"), scaled by the bytes of this shape when it was taken on another
     try:
         with open(os.path.join(ROOT, "profiles", "probe_traffic.txt")) as f:
+            table = {}
             for line in f:
                 parts = line.split("#")[0].split()
-                if len(parts) == 2 and parts[0] == f"{m}x{k}x{n}_{args.dtype}":
-                    out["roofline"]["traffic"] = int(parts[1])
+                if len(parts) == 2:
+                    table[parts[0]] = int(parts[1])
+        key = f"{m}x{k}x{n}_{args.dtype}"
+        if key in table:
+            out["roofline"]["traffic"] = table[key]
+            out["roofline"]["traffic_source"] = "profiles/probe_traffic.txt (ncu capture of this shape)"
+        elif f"4096x4096x4096_{args.dtype}" in table:
+            ref = table[f"4096x4096x4096_{args.dtype}"]
+            out["roofline"]["traffic"] = int(ref / algorithmic_bytes(4096, 4096, 4096) * nbytes)
+            out["roofline"]["traffic_source"] = "profiles/probe_traffic.txt: ncu capture at 4096^3 scaled by algorithmic bytes (traffic grows in proportion)"
     except Exception:
         pass
+    host_sample = None
     if not args.no_cpu_baseline and not args.probe_only:
-        out["cpu_baseline"] = cpu_baseline(args, batches[0], m, k, n, dt, nbytes)
+        host_sample = host_slab(batches[0], m, k, n)
+    del batches, ws, hb
+    torch.cuda.empty_cache()
+
+    # the clean-path sweep of the benchmark's fifth configuration, in the same run: square sizes, both operand types
+    if args.sweep and not args.probe_only:
+        sizes = [int(x) for x in args.sweep.split(",") if x]
+        rows, fits = sweep.run(sizes, iters=12, tensor_cores=args.tensor_cores, emit=None, with_localize=True)
+        for r in rows:
+            r["frac"] = r["probe_gbs"] / peak
+            r["frac_burst"] = (r["probe_gbs_burst"] / peak) if r.get("probe_gbs_burst") else None
+        out["sweep"] = {"rows": rows, "noise_exponent_fit": fits,
+                        "note": "A, B ~ N(0,1), no faults; probe_ms: median of event pairs, L2 flushed by a read; probe_ms_burst: "
+                                "back to back from a CUDA graph over rotating batches larger than L2 (sizes from 4096); localize "
+                                "forced on the clean product at the planned bucket count; c_hat = sigma m0 / (2^-24 n^1.5 rms(C)), "
+                                "fit c_hat ~ n^e over the sizes"}
+    # recovery by fault population over the benchmark configurations (bounded here; the whole campaign is
+    # python -m paper_2609_19758_b200.campaign)
+    if args.campaign != "none" and not args.probe_only:
+        campaign.EMIT = lambda line: sys.stderr.write(line + "\n")
+        if args.campaign == "short":
+            summ = campaign.run((1, 2, 3, 4), seeds2=3, seeds4=1, tensor_cores=args.tensor_cores, probe_buckets=256)
+            what = "configs 1-4: 256^3 FP16 (4 cases), 4096^3 BF16 (3 seeds), all transformer shapes in both types, 8192^3 FP16 (1 seed)"
+        else:
+            summ = campaign.run((1, 2, 3, 4), tensor_cores=args.tensor_cores, probe_buckets=256)
+            what = "configs 1-4 at their full seed counts"
+        out["recovery_by_population"] = {"cases": what, "summary": summ}
+    if host_sample is not None:
+        out["cpu_baseline"] = cpu_baseline(host_sample, m, k, n, dt)
     print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
+
+
+SLAB_COLS = 256
+
+
+def host_slab(batch, m, k, n):
+    """Host copies of a bounded sample of the workload: all of A, and the first SLAB_COLS columns of B and C (all of
+    them when the product is at most 4096^3).  The oracle's probe of the slab is the column slab of the full probe."""
+    w = n if m * k * n <= 4096 ** 3 else min(n, SLAB_COLS)
+    return dict(A=batch["A"].cpu(), B=batch["B"][:, :w].contiguous().cpu(), C=batch["C"][:, :w].contiguous().cpu(), w=w)
 
 
 def oracle_probe_once(A64, B64, C64):
@@ -414,50 +505,92 @@ def oracle_probe_once(A64, B64, C64):
     return O.probe_verdict(s, O.analytic_tau(A64, B64, A64.shape[1]), n_rows=A64.shape[0])
 
 
-def cpu_baseline(args, batch, m, k, n, dt, nbytes):
-    """The oracle as it stands, timed on this machine's host cores: one full-size probe
-    (explicit E = AB - C in FP64, column sums, verdict)."""
-    A64 = batch["hA"].double().numpy()
-    B64 = batch["hB"].double().numpy()
-    C64 = batch["Cf"].cpu().numpy()
+def oracle_localize_leg():
+    """The oracle's localization leg on the 4096^3 BF16 configuration (explicit E, then sketches + rounds from E),
+    timed separately: (E seconds, sketch + localize seconds, faults found)."""
+    import oracle as O
+    from paper_2609_19758_b200 import workloads as W
+    nl = 4096
+    A, B = W.operands("gauss_scaled", nl, nl, nl, W.BF16, 0)
+    C = W.cpu_fp32_product(A, B)
+    faults = W.faults_additive(nl, nl, W.rms(C), 0, 4, 0.02, 0.09, "small")
+    Cf, _ = W.inject(C, faults)
+    A64, B64 = A.double().numpy(), B.double().numpy()
     t = time.perf_counter()
-    v = oracle_probe_once(A64, B64, C64)
+    E = O.error_matrix(A64, B64, Cf.numpy())
+    t_e = time.perf_counter() - t
+    t = time.perf_counter()
+    got = O.localize(A64, B64, Cf.numpy(), 11, 1024, W.BF16, O.Params(s_budget=4, radius=10), E=E)
+    t_l = time.perf_counter() - t
+    return t_e, t_l, len({(f.i, f.j) for f in got} & {(f.i, f.j) for f in faults}), len(faults)
+
+
+def cpu_baseline(sample, m, k, n, dt, with_localize=True):
+    """The oracle as it stands, timed on this machine's host cores on a bounded sample of the workload: the probe of a
+    column slab (explicit E = A B - C in FP64 for those columns, column sums, verdict), and the localization leg at
+    4096^3 (explicit E, then sketches and rounds from E) reported separately."""
+    A64 = sample["A"].double().numpy()
+    B64 = sample["B"].double().numpy()
+    C32 = sample["C"].numpy()
+    w = sample["w"]
+    t = time.perf_counter()
+    v = oracle_probe_once(A64, B64, C32)
     dt_s = time.perf_counter() - t
-    return {"value": nbytes / dt_s / 1e9, "unit": "GB/s", "ms": dt_s * 1e3, "cores": os.cpu_count(), "kind": "oracle",
-            "fired": bool(v.fired),
-            "sample": f"one full-size oracle probe of the {m}x{k}x{n} workload (FP64 explicit E, numpy/OpenBLAS threads)"}
+    sbytes = 2 * m * k + 2 * k * w + 4 * m * w
+    out = {"value": sbytes / dt_s / 1e9, "unit": "GB/s", "ms": dt_s * 1e3, "cores": os.cpu_count(), "kind": "oracle",
+           "fired": bool(v.fired), "sample_bytes": sbytes,
+           "sample": (f"one oracle probe of the full {m}x{k}x{n} workload" if w == n else
+                      f"one oracle probe of a slab of the {m}x{k}x{n} workload: all of A, the first {w} of {n} columns of B and C")
+                     + " (FP64 explicit E, numpy/OpenBLAS threads); GB/s over the sample's own algorithmic bytes"}
+    if with_localize:
+        t_e, t_l, nf, ni = oracle_localize_leg()
+        out["localize_leg"] = {"workload": "4096^3 BF16, 4 faults of 2-9% rms(C), 1024 buckets, radius 10, 3 rounds",
+                               "explicit_E_ms": t_e * 1e3, "sketch_and_localize_from_E_ms": t_l * 1e3, "found": nf, "injected": ni}
+    return out
 
 
 def run_reference(args):
-    """The CPU oracle timed as the reference arm: each step is one oracle probe of the same
-    workload (bounded: a step is a few seconds at 4096^3)."""
+    """The CPU oracle timed as the reference arm on the same workload: each step is one oracle probe of a bounded
+    sample (a column slab above 4096^3), so that the run ends within minutes."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from paper_2609_19758_b200 import workloads as W
     m, k, n = (int(x) for x in args.shape.split(","))
     dt = W.BF16 if args.dtype == "bf16" else W.FP16
-    nbytes = algorithmic_bytes(m, k, n)
-    A, B = W.operands(args.kind, m, k, n, dt, 0)
+    w = n if m * k * n <= 4096 ** 3 else min(n, SLAB_COLS)
+    g = torch.Generator()
+    g.manual_seed(0x5EED0000)
+    td = W.TORCH_DTYPE[dt]
+    scale = (1.0 / k ** 0.5) if args.kind == "gauss_scaled" else (0.02 if args.kind == "transformer" else 1.0)
+    if args.kind == "uniform":
+        A = (torch.rand(m, k, generator=g) * 2 - 1).to(td)
+        B = (torch.rand(k, w, generator=g) * 2 - 1).to(td)
+    else:
+        A = torch.randn(m, k, generator=g).to(td)
+        B = (torch.randn(k, w, generator=g) * scale).to(td)
     C = W.cpu_fp32_product(A, B)
-    C[3, 5] += 0.05
-    A64, B64, C64 = A.double().numpy(), B.double().numpy(), C.numpy()
-    K = min(args.steps, 30)
+    C[3, 5] += 0.05 * float(C.abs().mean())
+    A64, B64, C32 = A.double().numpy(), B.double().numpy(), C.numpy()
+    sbytes = 2 * m * k + 2 * k * w + 4 * m * w
+    K = min(args.steps, 10 if w < n else 30)
     Wm = min(max(args.warmup, 1), 2)
     for _ in range(Wm):
-        oracle_probe_once(A64, B64, C64)
+        oracle_probe_once(A64, B64, C32)
     t = time.perf_counter()
     for _ in range(K):
-        oracle_probe_once(A64, B64, C64)
+        oracle_probe_once(A64, B64, C32)
     ms = (time.perf_counter() - t) * 1e3 / K
-    gbs = nbytes / (ms * 1e-3) / 1e9
-    sample = f"{K} oracle probes of the full {m}x{k}x{n} workload (steps capped at 30 to bound the run)"
+    gbs = sbytes / (ms * 1e-3) / 1e9
+    sample = (f"{K} oracle probes of the full {m}x{k}x{n} workload" if w == n else
+              f"{K} oracle probes of a slab of the {m}x{k}x{n} workload (all of A, {w} of {n} columns of B and C)") + \
+             "; GB/s over the sample's own algorithmic bytes; steps capped to bound the run"
     print(json.dumps({
         "impl": "reference", "metric": "clean-path probe HBM GB/s (probe ms beside vendor GEMM ms; fault recovery rate)",
         "value": gbs, "unit": "GB/s", "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": K, "warmup": Wm,
         "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
         "data": "synthetic",
-        "config": {"workload": f"square {args.dtype.upper()} product m=k=n={m}" if m == k == n else f"{m}x{k}x{n}"},
+        "config": {"workload": f"square {args.dtype.upper()} product m=k=n={m}" if m == k == n else f"{m}x{k}x{n} {args.dtype}"},
         "probe_ms": ms,
         "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": os.cpu_count(), "kind": "oracle", "sample": sample},
         "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},

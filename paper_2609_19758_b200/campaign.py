@@ -24,6 +24,13 @@ from . import build as B
 from . import fpsk, harness, workloads as W
 
 
+def _print_line(line: str) -> None:
+    print(line, flush=True)
+
+
+EMIT = _print_line          # where the per-case JSON lines go (a caller that owns stdout redirects them)
+
+
 def wilson(k: int, n: int, z: float = 1.959964):
     if n == 0:
         return None
@@ -103,15 +110,57 @@ def run_case(tag, kind, n1, n2, n3, dtype, seed, make_faults, params, probe_buck
             tally.setdefault(key, [0, 0])
             tally[key][0] += int(v)
             tally[key][1] += 1
-    print(json.dumps(dict(case=tag, shape=[n1, n2, n3], dtype="fp16" if dtype == W.FP16 else "bf16", seed=seed,
+    EMIT(json.dumps(dict(case=tag, shape=[n1, n2, n3], dtype="fp16" if dtype == W.FP16 else "bf16", seed=seed,
                           c_hat=nz.c_hat, plan=[nz.m0, nz.m_loc, nz.radius], injected=len(faults), found=len(want & have),
                           false_positives=len(have - want) + len(got_clean), probe=[int(clean_fired), dirty_fired],
                           hashed_probe=[int(h_clean), h_dirty],
                           probe_clean=dict(max_abs=r_c.max_abs, sigma_hat=r_c.sigma_hat, thr=r_c.thr, tau=r_c.tau),
                           hashed_clean=dict(m=probe_buckets, max_abs=r_h.max_abs, sigma_hat=r_h.sigma_hat, thr=r_h.thr,
-                                            tau=r_h.tau))), flush=True)
+                                            tau=r_h.tau))))
     del ws, dA, dB, dC, dCf
     torch.cuda.empty_cache()
+
+
+def run(configs=(1, 2, 3, 4), seeds2=20, seeds4=10, tensor_cores=1, probe_buckets=256, shapes3=None):
+    """Runs the chosen configurations and returns the summary (per-population recovery, false positives, probes)."""
+    B.build()
+    fpsk.lib()
+    todo = set(configs)
+    tally = {}
+    tc = tensor_cores
+    if 1 in todo:
+        p = fpsk.default_params(s_budget=1, delta_max=1, tensor_cores=tc)
+        run_case("cfg1", "uniform", 256, 256, 256, W.FP16, 1, lambda dC, rms: [], p, 16, tally)
+        for s in (1, 2, 3):
+            run_case("cfg1", "uniform", 256, 256, 256, W.FP16, 1,
+                     lambda dC, rms, s=s: W.faults_additive(256, 256, rms, s, 1, 0.5, 0.5, "typical"), p, 16, tally)
+    if 2 in todo:
+        p = fpsk.default_params(s_budget=4, tensor_cores=tc)
+        for s in range(seeds2):
+            run_case("cfg2", "gauss_scaled", 4096, 4096, 4096, W.BF16, s,
+                     lambda dC, rms, s=s: W.faults_additive(4096, 4096, rms, s, 4, 0.02, 0.09, "small"), p,
+                     probe_buckets, tally)
+    if 3 in todo:
+        p = fpsk.default_params(tensor_cores=tc)
+        for (n1, n2, n3) in (shapes3 if shapes3 is not None else W.TRANSFORMER_SHAPES):
+            for dt in (W.FP16, W.BF16):
+                def mk(dC, rms, n1=n1, n3=n3):
+                    a = W.faults_additive(n1, n3, rms, 7, 4, 1.0, 1.0, "typical")
+                    b = W.faults_additive(n1, n3, rms, 8, 4, 0.02, 0.09, "small", taken=[(f.i, f.j) for f in a])
+                    return a + b
+                run_case("cfg3", "transformer", n1, n2, n3, dt, 7, mk, p, probe_buckets, tally)
+    if 4 in todo:
+        p = fpsk.default_params(s_budget=16, delta_max=4, tensor_cores=tc)
+        for s in range(seeds4):
+            run_case("cfg4", "uniform", 8192, 8192, 8192, W.FP16, s,
+                     lambda dC, rms, s=s: W.faults_mixed16(dC.cpu(), rms, s), p, probe_buckets, tally)
+    summary = {}
+    for k, v in tally.items():
+        if isinstance(v, list):
+            summary[k] = dict(hits=v[0], of=v[1], rate=(v[0] / v[1]) if v[1] else None, wilson95=wilson(v[0], v[1]))
+        else:
+            summary[k] = v
+    return summary
 
 
 def main():
@@ -122,45 +171,9 @@ def main():
     ap.add_argument("--tensor-cores", type=int, default=1, choices=[0, 1])
     ap.add_argument("--probe-buckets", type=int, default=256)
     args = ap.parse_args()
-    B.build()
-    fpsk.lib()
     torch.cuda.set_device(0)
-    todo = {int(x) for x in args.configs.split(",")}
-    tally = {}
-    tc = args.tensor_cores
-    if 1 in todo:
-        p = fpsk.default_params(s_budget=1, delta_max=1, tensor_cores=tc)
-        run_case("cfg1", "uniform", 256, 256, 256, W.FP16, 1, lambda dC, rms: [], p, 16, tally)
-        for s in (1, 2, 3):
-            run_case("cfg1", "uniform", 256, 256, 256, W.FP16, 1,
-                     lambda dC, rms, s=s: W.faults_additive(256, 256, rms, s, 1, 0.5, 0.5, "typical"), p, 16, tally)
-    if 2 in todo:
-        p = fpsk.default_params(s_budget=4, tensor_cores=tc)
-        for s in range(args.seeds2):
-            run_case("cfg2", "gauss_scaled", 4096, 4096, 4096, W.BF16, s,
-                     lambda dC, rms, s=s: W.faults_additive(4096, 4096, rms, s, 4, 0.02, 0.09, "small"), p,
-                     args.probe_buckets, tally)
-    if 3 in todo:
-        p = fpsk.default_params(tensor_cores=tc)
-        for (n1, n2, n3) in W.TRANSFORMER_SHAPES:
-            for dt in (W.FP16, W.BF16):
-                def mk(dC, rms, n1=n1, n3=n3):
-                    a = W.faults_additive(n1, n3, rms, 7, 4, 1.0, 1.0, "typical")
-                    b = W.faults_additive(n1, n3, rms, 8, 4, 0.02, 0.09, "small", taken=[(f.i, f.j) for f in a])
-                    return a + b
-                run_case("cfg3", "transformer", n1, n2, n3, dt, 7, mk, p, args.probe_buckets, tally)
-    if 4 in todo:
-        p = fpsk.default_params(s_budget=16, delta_max=4, tensor_cores=tc)
-        for s in range(args.seeds4):
-            run_case("cfg4", "uniform", 8192, 8192, 8192, W.FP16, s,
-                     lambda dC, rms, s=s: W.faults_mixed16(dC.cpu(), rms, s), p, args.probe_buckets, tally)
-    summary = {}
-    for k, v in tally.items():
-        if isinstance(v, list):
-            summary[k] = dict(hits=v[0], of=v[1], rate=(v[0] / v[1]) if v[1] else None, wilson95=wilson(v[0], v[1]))
-        else:
-            summary[k] = v
-    print(json.dumps(dict(summary=summary, tensor_cores=tc, probe_buckets=args.probe_buckets)))
+    summary = run({int(x) for x in args.configs.split(",")}, args.seeds2, args.seeds4, args.tensor_cores, args.probe_buckets)
+    print(json.dumps(dict(summary=summary, tensor_cores=args.tensor_cores, probe_buckets=args.probe_buckets)))
 
 
 if __name__ == "__main__":
