@@ -14,13 +14,13 @@
  *   - The caller owns every buffer.  The library allocates no device memory and never writes
  *     to A or B; C is written only by fpsk_verify_repair and fpsk_apply_corrections (paper,
  *     Section "Overview": localization does not modify C; Algorithm 2, "Apply").
- *     fpsk_localize and fpsk_verify_repair create one CUDA event for the duration of the call.  They and
- *     fpsk_measure_noise read their results back through a small pinned host buffer (about 25 KB) and run
- *     independent parts of a sketch build on two auxiliary non-blocking streams, tied to `stream` by
- *     events on both sides (work queued on `stream` before the call is complete before any of it
- *     starts; everything is complete when the call returns).  The buffer, the two streams and their
- *     five events are created on first use, one set per concurrent call and device, and kept for the
- *     life of the process.
+ *     fpsk_measure_noise, fpsk_localize and fpsk_verify_repair read their results back through a small
+ *     pinned host buffer (about 25 KB) and run independent parts of a sketch build on two auxiliary
+ *     non-blocking streams, tied to `stream` by events on both sides (work queued on `stream` before the
+ *     call is complete before any of it starts; everything is complete when the call returns, also when
+ *     it returns an error).  These host resources are the caller's when it passes a context
+ *     (fpsk_context_create, fpsk_params.context); otherwise they are created on first use, one set per
+ *     concurrent call and device, and kept for the life of the process.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).
  *   - Indices are 0-based.  The 1-based index weights of the paper are internal.
  *   - Errors are return codes.  Nothing throws, aborts or resets the device.  After
@@ -104,6 +104,8 @@ typedef struct {
     double mu;           /* probe margin                                                   */
     double b_star;       /* target index budget                                            */
     double c_coll;       /* collision constant of m_comb                                   */
+    void *context;       /* fpsk_context* of the caller (see fpsk_context_create), or NULL: the library then
+                            creates the auxiliary streams, events and pinned buffer itself on first use      */
 } fpsk_params;
 
 /* Result of the run-time noise measurement (Section "Fault Magnitude, Calibration, and the
@@ -384,15 +386,17 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
 fpsk_status fpsk_apply_corrections(float *C, int64_t ldc, int64_t m, int64_t n, const fpsk_fault *h_faults,
                                    int32_t count, void *workspace, size_t ws_bytes, void *stream);
 
-/* Self-test of the give-up path that every device-side wait of this library has (no counterpart in
- * the paper).  One thread waits for *d_flag (device, 4 bytes) to become non-zero, with a limit of about
- * half a millisecond instead of the library's usual second, then writes d_result->status: FPSK_OK if the
- * flag was set, FPSK_ERR_TIMEOUT if the wait gave up.  The kernel always returns; the context stays usable.
- * Asynchronous on `stream`. */
-fpsk_status fpsk_selftest_bounded_wait(uint32_t *d_flag, fpsk_probe_result *d_result, void *stream);
-
-/* Number of kernels launched by this library since load (all entry points, all threads). */
-uint64_t fpsk_launch_count(void);
+/* ---- caller-owned host resources ------------------------------------------------------------
+ * fpsk_measure_noise, fpsk_localize and fpsk_verify_repair need, besides the device workspace, two auxiliary
+ * non-blocking streams, six events and about 25 KB of pinned host memory (their results come back through it).
+ * A caller that wants to own them (no creation inside those calls, release at a time of its choosing) creates a
+ * context on the device it will run on, puts it into fpsk_params.context and destroys it when no call that uses
+ * it is in flight.  A context serves one call at a time.  With context = NULL the library creates one such set
+ * per concurrent call and device on first use and keeps it for the life of the process.  (The paper has no
+ * counterpart: its engine runs under a framework that owns streams and staging memory.) */
+typedef struct fpsk_context fpsk_context;
+fpsk_status fpsk_context_create(fpsk_context **out);
+fpsk_status fpsk_context_destroy(fpsk_context *ctx);
 
 #ifdef __cplusplus
 }

@@ -2,6 +2,7 @@
 // (Sections "Sketch Noise Sets the Bucket Count" and "Calibration") and the round loop of
 // Algorithm 2's localize part with the ordered replay of Algorithm 1's search over the hits.
 #include "sketch.cuh"
+#include "fpsk_test.h"
 
 #include <math.h>
 #include <string.h>
@@ -11,6 +12,25 @@
 
 namespace fpsk {
 std::atomic<unsigned long long> g_launches{0};
+std::atomic<unsigned long long> g_lazy_resources{0};
+
+#ifdef FPSK_DEBUG_BOUNDS
+// the bounds records of the source files of the library (each registers its own at load)
+struct BoundsSource {
+    const char *file;
+    cudaError_t (*read)(BoundsRecord *);
+    cudaError_t (*clear)();
+};
+static std::vector<BoundsSource> &bounds_sources()
+{
+    static std::vector<BoundsSource> *v = new std::vector<BoundsSource>;
+    return *v;
+}
+void bounds_register(const char *file, cudaError_t (*read)(BoundsRecord *), cudaError_t (*clear)())
+{
+    bounds_sources().push_back(BoundsSource{file, read, clear});
+}
+#endif
 
 constexpr int kHitCap = 2048;
 constexpr int kPeelCap = 4096;
@@ -60,9 +80,10 @@ static PinnedPool &pinned_pool()
 }
 struct PinnedLease {
     void *p = nullptr;
+    bool borrowed = false;      // the buffer of a caller's context: not returned to the pool
     ~PinnedLease()
     {
-        if (!p) return;
+        if (!p || borrowed) return;
         PinnedPool &pool = pinned_pool();
         std::lock_guard<std::mutex> g(pool.mu);
         pool.free_list.push_back(p);
@@ -79,9 +100,63 @@ static fpsk_status pinned_acquire(PinnedLease &l)
             return FPSK_OK;
         }
     }
+    g_lazy_resources.fetch_add(1, std::memory_order_relaxed);
     FPSK_CUDA_OK(cudaHostAlloc(&l.p, kPackBytes, cudaHostAllocPortable));
     return FPSK_OK;
 }
+
+}  // namespace fpsk
+
+// What a caller's context holds: the host-side resources of one call at a time.
+struct fpsk_context {
+    fpsk::SketchAux aux;
+    void *pinned = nullptr;           // kPackBytes
+    cudaEvent_t round_done = nullptr;
+};
+
+namespace fpsk {
+
+// The host-side resources of one call: from the caller's context when it passed one (nothing is created),
+// else leased from the library's own pools (created on first use).
+struct HostRes {
+    SketchAuxLease aux;
+    PinnedLease pin;
+    cudaEvent_t round_done = nullptr;
+    bool own_event = false;
+    ~HostRes() { if (own_event && round_done) cudaEventDestroy(round_done); }
+    fpsk_status acquire(const fpsk_params &q, bool need_event)
+    {
+        if (q.context) {
+            fpsk_context *c = static_cast<fpsk_context *>(q.context);
+            int dev = 0;
+            FPSK_CUDA_OK(cudaGetDevice(&dev));
+            if (c->aux.device != dev) return FPSK_ERR_PARAM;       // a context belongs to the device it was created on
+            aux.aux = &c->aux; aux.borrowed = true;
+            pin.p = c->pinned; pin.borrowed = true;
+            round_done = c->round_done;
+            return FPSK_OK;
+        }
+        fpsk_status rc = sketch_aux_acquire(aux);
+        if (rc != FPSK_OK) return rc;
+        rc = pinned_acquire(pin);
+        if (rc != FPSK_OK) return rc;
+        if (need_event) {
+            FPSK_CUDA_OK(cudaEventCreateWithFlags(&round_done, cudaEventDisableTiming));
+            own_event = true;
+        }
+        return FPSK_OK;
+    }
+    // Error exits: whatever was queued on the auxiliary streams and on the caller's stream is complete before
+    // the call returns, as the header promises for every return.
+    void drain(cudaStream_t st) const
+    {
+        if (aux.aux) {
+            if (aux.aux->s1) cudaStreamSynchronize(aux.aux->s1);
+            if (aux.aux->s2) cudaStreamSynchronize(aux.aux->s2);
+        }
+        cudaStreamSynchronize(st);
+    }
+};
 
 // ---------------------------------------------------------------- scalar planner
 static double cf_of(fpsk_dtype d) { return d == FPSK_BF16 ? 0.19 : 1.76 * 0.19; }
@@ -238,12 +313,9 @@ static fpsk_status loc_max_ab(const SketchIn &in, fpsk_dtype dtype, LocWs &w, cu
 
 // The scalars of a noise measurement (the select's eight scalars, rms(C), the select's error word) to the host
 // through pinned staging: three small asynchronous copies and one wait (a pageable destination blocks per copy).
-static fpsk_status read_noise_scalars(const LocWs &w, cudaStream_t st, float (&h_scal)[8], float &h_rms)
+static fpsk_status read_noise_scalars(const LocWs &w, cudaStream_t st, float (&h_scal)[8], float &h_rms, void *pinned)
 {
-    PinnedLease stage;
-    fpsk_status rc = pinned_acquire(stage);
-    if (rc != FPSK_OK) return rc;
-    char *h = static_cast<char *>(stage.p);
+    char *h = static_cast<char *>(pinned);
     FPSK_CUDA_OK(cudaMemcpyAsync(h, w.sel.scal, 32, cudaMemcpyDeviceToHost, st));
     FPSK_CUDA_OK(cudaMemcpyAsync(h + 32, w.misc + 3, 4, cudaMemcpyDeviceToHost, st));
     FPSK_CUDA_OK(cudaMemcpyAsync(h + 36, w.sel.err, 4, cudaMemcpyDeviceToHost, st));
@@ -270,17 +342,15 @@ static int offset_rank_key(int di, int dj, int r)
 // The localize part of Algorithm 2: p.rounds rounds of Algorithm 1 at m_b buckets, carrying F.
 // Entries already in F with round < 0 are absolute repairs (Section "Nonfinite"): they count as
 // found but are not peeled, their error is already absent from the sketches.
-static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, uint64_t seed, int m_b, const fpsk_params &q, LocWs &w,
-                                 cudaStream_t st, std::vector<fpsk_fault> &F, bool &truncated, int &radius_used)
+static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, uint64_t seed, int m_b, const fpsk_params &q, LocWs &w,
+                                   cudaStream_t st, HostRes &hr, std::vector<fpsk_fault> &F, bool &truncated, int &radius_used)
 {
     SketchIn in = in_caller;
     const long long m = in.n1, k = in.n2, n = in.n3;
     const long long mm = (long long)m_b * m_b;
     const int K = std::min(std::max(64, 8 * q.s_budget), kSelMaxK);
     fpsk_status rc;
-    SketchAuxLease aux;
-    rc = sketch_aux_acquire(aux);
-    if (rc != FPSK_OK) return rc;
+    SketchAuxLease &aux = hr.aux;
     w.sk.aux = aux.aux;
     // Once per call, side by side: max|A| and the hash tables of all rounds (they depend on the seed only) on the
     // caller's stream; max|B| and, for B given as k x n, its transpose on an auxiliary stream.  With W = B^T every round
@@ -326,7 +396,7 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
         rc = sigma_mad_rms_c_launch(w.S, mm, q.mad_of_abs, in.C, in.ldc, m, n, w.samples, w.sel, w.misc + 3, st);
         if (rc != FPSK_OK) return rc;
         float h_scal[8], h_rms = 0.f;
-        rc = read_noise_scalars(w, st, h_scal, h_rms);
+        rc = read_noise_scalars(w, st, h_scal, h_rms, hr.pin.p);
         if (rc != FPSK_OK) return rc;
         double sig = h_scal[1], rms = h_rms;
         if (!(std::isfinite(sig) && sig > 0 && std::isfinite(rms) && rms > 0)) {
@@ -339,18 +409,12 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
 
     std::vector<PeelEntry> peel;
     std::vector<Hit> hits(kHitCap);
-    PinnedLease stage;
-    rc = pinned_acquire(stage);
-    if (rc != FPSK_OK) return rc;
+    PinnedLease &stage = hr.pin;
     const size_t pack_bytes = sizeof(RoundHeader) + (size_t)K * sizeof(Candidate) + (size_t)kPackHits * sizeof(Hit);
     // The sketches of round t + 1 do not depend on what round t finds (only the peeling does), so they
     // are enqueued before the host waits for round t's results: the GPU builds them while the host
     // replays the search.  The event marks the end of round t's copies.
-    struct EventGuard {
-        cudaEvent_t e = nullptr;
-        ~EventGuard() { if (e) cudaEventDestroy(e); }
-    } round_done;
-    FPSK_CUDA_OK(cudaEventCreateWithFlags(&round_done.e, cudaEventDisableTiming));
+    struct { cudaEvent_t e; } round_done{hr.round_done};
     // Only S is built whole.  The first moments R, T are read at the K buckets the selection keeps and nowhere else
     // (Eq. (recover)), so they are computed for those buckets alone once the keys are collected: a third of the
     // contraction, of the combine and of the plane writes.
@@ -439,6 +503,15 @@ static fpsk_status localize_core(const SketchIn &in_caller, fpsk_dtype dtype, ui
         }
     }
     return FPSK_OK;
+}
+
+static fpsk_status localize_core(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, int m_b, const fpsk_params &q, LocWs &w,
+                                 cudaStream_t st, HostRes &hr, std::vector<fpsk_fault> &F, bool &truncated, int &radius_used)
+{
+    const fpsk_status rc = localize_rounds(in, dtype, seed, m_b, q, w, st, hr, F, truncated, radius_used);
+    // an error may leave a round's sketch build queued on the auxiliary streams: finish it before returning
+    if (rc != FPSK_OK) hr.drain(st);
+    return rc;
 }
 
 // Waits, with a short limit, for a flag that the caller leaves at zero: the wait gives up, the kernel
@@ -747,41 +820,49 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
-    SketchAuxLease aux;
-    rc = sketch_aux_acquire(aux);
+    HostRes hr;
+    rc = hr.acquire(q, false);
     if (rc != FPSK_OK) return rc;
+    SketchAuxLease &aux = hr.aux;
     w.sk.aux = aux.aux;
-    if (w.sk.tc) {
-        rc = loc_max_ab(in, dtype, w, st);
-        if (rc != FPSK_OK) return rc;
-    }
-    // The samples of C need nothing from the sketch: they are taken on the stream that will run the C scatter, ahead of
-    // the build (which joins that stream before its combine).  The clipped mean and the selects both only read S:
-    // the two sums run on the other auxiliary stream beside the select launch.
-    SketchAux *ax = (aux.aux && aux.aux->s1 && aux.aux->s2 && aux.aux->ev[4]) ? aux.aux : nullptr;
-    if (ax) {
-        FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));             // whatever the caller queued before this call (the GEMM, say)
-        FPSK_CUDA_OK(cudaStreamWaitEvent(ax->s2, ax->ev[0], 0));
-    }
-    const long long nsamp = rms_c_samples(C, ldc, m, n, w.samples, w.sel, ax ? ax->s2 : st);
-    if (nsamp < 0) return FPSK_ERR_CUDA;
-    rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
-    if (rc != FPSK_OK) return rc;
-    const long long mm = (long long)m0 * m0;
-    if (ax) {
-        FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));
-        FPSK_CUDA_OK(cudaStreamWaitEvent(ax->s1, ax->ev[0], 0));
-    }
-    rc = sigma_clip_launch(w.S, mm, w.sel, ax ? ax->s1 : st);
-    if (rc != FPSK_OK) return rc;
-    if (ax) FPSK_CUDA_OK(cudaEventRecord(ax->ev[1], ax->s1));
-    rc = sigma_mad_rms_c_select_launch(w.S, mm, q.mad_of_abs, w.samples, nsamp, w.sel, w.misc + 3, st);
-    if (rc != FPSK_OK) return rc;
-    if (ax) FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->ev[1], 0));
     float h_scal[8];
     float h_rms = 0.f;
-    rc = read_noise_scalars(w, st, h_scal, h_rms);
-    if (rc != FPSK_OK) return rc;
+    // one exit path: an error leaves nothing queued behind the call
+    rc = [&]() -> fpsk_status {
+        fpsk_status rc;
+        if (w.sk.tc) {
+            rc = loc_max_ab(in, dtype, w, st);
+            if (rc != FPSK_OK) return rc;
+        }
+        // The samples of C need nothing from the sketch: they are taken on the stream that will run the C scatter, ahead of
+        // the build (which joins that stream before its combine).  The clipped mean and the selects both only read S:
+        // the two sums run on the other auxiliary stream beside the select launch.
+        SketchAux *ax = (aux.aux && aux.aux->s1 && aux.aux->s2 && aux.aux->ev[4]) ? aux.aux : nullptr;
+        if (ax) {
+            FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));             // whatever the caller queued before this call (the GEMM, say)
+            FPSK_CUDA_OK(cudaStreamWaitEvent(ax->s2, ax->ev[0], 0));
+        }
+        const long long nsamp = rms_c_samples(C, ldc, m, n, w.samples, w.sel, ax ? ax->s2 : st);
+        if (nsamp < 0) return FPSK_ERR_CUDA;
+        rc = build_sketches(in, dtype, seed, 0, m0, false, w.sk, st, w.S, nullptr, nullptr);
+        if (rc != FPSK_OK) return rc;
+        const long long mm = (long long)m0 * m0;
+        if (ax) {
+            FPSK_CUDA_OK(cudaEventRecord(ax->ev[0], st));
+            FPSK_CUDA_OK(cudaStreamWaitEvent(ax->s1, ax->ev[0], 0));
+        }
+        rc = sigma_clip_launch(w.S, mm, w.sel, ax ? ax->s1 : st);
+        if (rc != FPSK_OK) return rc;
+        if (ax) FPSK_CUDA_OK(cudaEventRecord(ax->ev[1], ax->s1));
+        rc = sigma_mad_rms_c_select_launch(w.S, mm, q.mad_of_abs, w.samples, nsamp, w.sel, w.misc + 3, st);
+        if (rc != FPSK_OK) return rc;
+        if (ax) FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->ev[1], 0));
+        return read_noise_scalars(w, st, h_scal, h_rms, hr.pin.p);
+    }();
+    if (rc != FPSK_OK) {
+        hr.drain(st);
+        return rc;
+    }
 
     fpsk_noise out;
     memset(&out, 0, sizeof(out));
@@ -829,7 +910,10 @@ fpsk_status fpsk_localize(const void *A, int64_t lda, const void *B, int64_t ldb
     std::vector<fpsk_fault> F;
     bool truncated = false;
     int radius_used = 0;
-    rc = localize_core(in, dtype, seed, n_buckets, q, w, static_cast<cudaStream_t>(stream), F, truncated, radius_used);
+    HostRes hr;
+    rc = hr.acquire(q, true);
+    if (rc != FPSK_OK) return rc;
+    rc = localize_core(in, dtype, seed, n_buckets, q, w, static_cast<cudaStream_t>(stream), hr, F, truncated, radius_used);
     if (rc != FPSK_OK) return rc;
     std::sort(F.begin(), F.end(), [](const fpsk_fault &x, const fpsk_fault &y) {
         return x.i != y.i ? x.i < y.i : x.j < y.j;
@@ -967,41 +1051,49 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
     // ---- plan from the noise measured on this call, then k rounds of Algorithm 1
     fpsk_params qq = q;
     int m_loc = n_buckets;
-    if (m_loc <= 0) {
-        const int m0 = std::min(m_start_of(m, k, n, dtype, q), sketch_max_buckets(m, k, n));
-        LocWs w0;
-        if (!loc_carve(loc_ws, loc_bytes, m, k, n, m0, w0, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
-        SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
-        if (w0.sk.tc) {
-            rc = loc_max_ab(in, dtype, w0, st);
-            if (rc != FPSK_OK) return rc;
-        }
-        rc = build_sketches(in, dtype, seed, 0, m0, false, w0.sk, st, w0.S, nullptr, nullptr);
-        if (rc != FPSK_OK) return rc;
-        rc = sigma_mad_rms_c_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);
-        if (rc != FPSK_OK) return rc;
-        float h_scal[8], h_rms = 0.f;
-        rc = read_noise_scalars(w0, st, h_scal, h_rms);
-        if (rc != FPSK_OK) return rc;
-        int r;
-        double B_;
-        plan_of(m, k, n, dtype, h_scal[1], h_rms, m0, q, m_loc, r, B_);
-        m_loc = std::min(m_loc, sketch_max_buckets(m, k, n));
-        if (qq.radius < 0) qq.radius = r;
-    }
-    LocWs w;
-    if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w, q.tensor_cores != 0, true)) return FPSK_ERR_WORKSPACE;
-    SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
     bool truncated = false;
     int radius_used = 0;
-    rc = localize_core(in, dtype, seed, m_loc, qq, w, st, F, truncated, radius_used);
+    HostRes hr;
+    rc = [&]() -> fpsk_status {
+        fpsk_status rc = hr.acquire(q, true);
+        if (rc != FPSK_OK) return rc;
+        if (m_loc <= 0) {
+            const int m0 = std::min(m_start_of(m, k, n, dtype, q), sketch_max_buckets(m, k, n));
+            LocWs w0;
+            if (!loc_carve(loc_ws, loc_bytes, m, k, n, m0, w0, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
+            SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+            if (w0.sk.tc) {
+                rc = loc_max_ab(in, dtype, w0, st);
+                if (rc != FPSK_OK) return rc;
+            }
+            rc = build_sketches(in, dtype, seed, 0, m0, false, w0.sk, st, w0.S, nullptr, nullptr);
+            if (rc != FPSK_OK) return rc;
+            rc = sigma_mad_rms_c_launch(w0.S, (long long)m0 * m0, q.mad_of_abs, C, ldc, m, n, w0.samples, w0.sel, w0.misc + 3, st);
+            if (rc != FPSK_OK) return rc;
+            float h_scal[8], h_rms = 0.f;
+            rc = read_noise_scalars(w0, st, h_scal, h_rms, hr.pin.p);
+            if (rc != FPSK_OK) return rc;
+            int r;
+            double B_;
+            plan_of(m, k, n, dtype, h_scal[1], h_rms, m0, q, m_loc, r, B_);
+            m_loc = std::min(m_loc, sketch_max_buckets(m, k, n));
+            if (qq.radius < 0) qq.radius = r;
+        }
+        LocWs w;
+        if (!loc_carve(loc_ws, loc_bytes, m, k, n, m_loc, w, q.tensor_cores != 0, true)) return FPSK_ERR_WORKSPACE;
+        SketchIn in{A, B, C, m, k, n, lda, ldb, ldc};
+        return localize_core(in, dtype, seed, m_loc, qq, w, st, hr, F, truncated, radius_used);
+    }();
+    if (rc != FPSK_OK) hr.drain(st);
     // ---- the absolute entries go back into C whatever happened above
     if (!restore.empty()) {
         PatchEntry *d = static_cast<PatchEntry *>(rep_ws);
-        FPSK_CUDA_OK(cudaMemcpyAsync(d, restore.data(), sizeof(PatchEntry) * restore.size(), cudaMemcpyHostToDevice, st));
-        fpsk_status rc2 = patch_launch(C, ldc, d, (int)restore.size(), st);
-        FPSK_CUDA_OK(cudaStreamSynchronize(st));
-        if (rc2 != FPSK_OK) return rc2;
+        fpsk_status rc2 = FPSK_OK;
+        if (cudaMemcpyAsync(d, restore.data(), sizeof(PatchEntry) * restore.size(), cudaMemcpyHostToDevice, st) != cudaSuccess)
+            rc2 = FPSK_ERR_CUDA;
+        if (rc2 == FPSK_OK) rc2 = patch_launch(C, ldc, d, (int)restore.size(), st);
+        if (cudaStreamSynchronize(st) != cudaSuccess && rc2 == FPSK_OK) rc2 = FPSK_ERR_CUDA;
+        if (rc == FPSK_OK) rc = rc2;
     }
     if (rc != FPSK_OK) return rc;
     h_report->m_loc = m_loc;
@@ -1031,5 +1123,78 @@ fpsk_status fpsk_verify_repair(const void *A, int64_t lda, const void *B, int64_
 }
 
 uint64_t fpsk_launch_count(void) { return g_launches.load(); }
+uint64_t fpsk_lazy_resource_count(void) { return g_lazy_resources.load(); }
+
+int32_t fpsk_debug_bounds_report(int64_t *violations, int32_t *line, int64_t *index, int64_t *limit, char *file, size_t file_cap)
+{
+#ifdef FPSK_DEBUG_BOUNDS
+    long long total = 0;
+    bool first = true;
+    if (file && file_cap) file[0] = 0;
+    for (const BoundsSource &src : bounds_sources()) {
+        BoundsRecord r;
+        if (src.read(&r) != cudaSuccess) return -1;
+        total += r.count;
+        if (r.count && first) {
+            first = false;
+            if (line) *line = r.line;
+            if (index) *index = r.index;
+            if (limit) *limit = r.limit;
+            if (file && file_cap) {
+                strncpy(file, src.file, file_cap - 1);
+                file[file_cap - 1] = 0;
+            }
+        }
+    }
+    if (violations) *violations = total;
+    return 1;
+#else
+    (void)line; (void)index; (void)limit; (void)file; (void)file_cap;
+    if (violations) *violations = -1;
+    return 0;
+#endif
+}
+
+fpsk_status fpsk_debug_bounds_clear(void)
+{
+#ifdef FPSK_DEBUG_BOUNDS
+    for (const BoundsSource &src : bounds_sources())
+        if (src.clear() != cudaSuccess) return FPSK_ERR_CUDA;
+#endif
+    return FPSK_OK;
+}
+
+fpsk_status fpsk_context_create(fpsk_context **out)
+{
+    if (!out) return FPSK_ERR_NULL;
+    *out = nullptr;
+    fpsk_context *c = new fpsk_context;
+    bool ok = cudaGetDevice(&c->aux.device) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->aux.s1, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->aux.s2, cudaStreamNonBlocking) == cudaSuccess;
+    for (int e = 0; e < 5 && ok; ++e) ok = cudaEventCreateWithFlags(&c->aux.ev[e], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->round_done, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaHostAlloc(&c->pinned, kPackBytes, cudaHostAllocPortable) == cudaSuccess;
+    if (!ok) {
+        fpsk_context_destroy(c);
+        return FPSK_ERR_CUDA;
+    }
+    *out = c;
+    return FPSK_OK;
+}
+
+fpsk_status fpsk_context_destroy(fpsk_context *c)
+{
+    if (!c) return FPSK_OK;
+    bool ok = true;
+    if (c->aux.s1) ok = (cudaStreamDestroy(c->aux.s1) == cudaSuccess) && ok;
+    if (c->aux.s2) ok = (cudaStreamDestroy(c->aux.s2) == cudaSuccess) && ok;
+    for (int e = 0; e < 5; ++e)
+        if (c->aux.ev[e]) ok = (cudaEventDestroy(c->aux.ev[e]) == cudaSuccess) && ok;
+    if (c->round_done) ok = (cudaEventDestroy(c->round_done) == cudaSuccess) && ok;
+    if (c->pinned) ok = (cudaFreeHost(c->pinned) == cudaSuccess) && ok;
+    delete c;
+    return ok ? FPSK_OK : FPSK_ERR_CUDA;
+}
 
 }  // extern "C"

@@ -98,7 +98,7 @@ constexpr int kMomThreads = 1024;         // few CTAs do any work (one per kept 
 template <typename T>
 __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
     const unsigned short *A, long long lda, const unsigned short *B, long long ldb, int bt, const float *C, long long ldc,
-    int n2, int m_b, float inv_p1, float inv_p3, const uint32_t *rowperm, const int *rowstart, const uint32_t *colperm,
+    int n1, int n2, int n3, int m_b, float inv_p1, float inv_p3, const uint32_t *rowperm, const int *rowstart, const uint32_t *colperm,
     const int *colstart, const unsigned long long *keys, const int *counts, int cap, const PeelEntry *peel, int n_peel,
     uint32_t key1, uint32_t key2, float *Rc, float *Tc, int vec)
 {
@@ -109,6 +109,7 @@ __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
     if (slot >= n) return;
     const uint32_t idx = 0xFFFFFFFFu - (uint32_t)(keys[slot] & 0xFFFFFFFFull);
     const int a = (int)(idx / (uint32_t)m_b), b = (int)(idx % (uint32_t)m_b);
+    if (!FPSK_IN_BOUNDS(a, m_b)) return;          // a key that does not name a bucket
     const int r0 = rowstart[a], r1 = rowstart[a + 1], c0 = colstart[b], c1 = colstart[b + 1];
     double accR = 0.0, accT = 0.0;
     if (vec) {
@@ -164,6 +165,7 @@ __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
             for (int s = r0; s < r1; ++s) {
                 const uint32_t e = __ldg(rowperm + s);
                 const int i = (int)(e & 0x7FFFFFFFu);
+                if (!FPSK_IN_BOUNDS(i, n1)) continue;
                 const float sg = (e >> 31) ? -1.f : 1.f;
                 const float x = bits16_to_float<T>(A[(long long)i * lda + k]);
                 p += sg * x;
@@ -172,6 +174,7 @@ __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
             for (int s = c0; s < c1; ++s) {
                 const uint32_t e = __ldg(colperm + s);
                 const int j = (int)(e & 0x7FFFFFFFu);
+                if (!FPSK_IN_BOUNDS(j, n3)) continue;
                 const float sg = (e >> 31) ? -1.f : 1.f;
                 const float y = bits16_to_float<T>(bt ? B[(long long)j * ldb + k] : B[(long long)k * ldb + j]);
                 q += sg * y;
@@ -186,6 +189,7 @@ __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
     for (int e = threadIdx.x; e < nr * nc; e += kMomThreads) {
         const uint32_t er = __ldg(rowperm + r0 + e / nc), ec = __ldg(colperm + c0 + e % nc);
         const int i = (int)(er & 0x7FFFFFFFu), j = (int)(ec & 0x7FFFFFFFu);
+        if (!FPSK_IN_BOUNDS(i, n1) || !FPSK_IN_BOUNDS(j, n3)) continue;
         const double v = ((er >> 31) != (ec >> 31)) ? -1.0 : 1.0;
         const double c = (double)C[(long long)i * ldc + j];
         accR -= v * (double)((float)(i + 1) * inv_p1) * c;
@@ -231,11 +235,11 @@ fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const
     const int vec = (in.bt && ((reinterpret_cast<uintptr_t>(in.A) | reinterpret_cast<uintptr_t>(in.B)) & 15) == 0 && in.lda % 8 == 0 &&
                      in.ldb % 8 == 0 && in.n2 % 8 == 0) ? 1 : 0;
     if (dtype == FPSK_FP16)
-        candidate_moments_kernel<__half><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n2, m_b, inv_p1,
+        candidate_moments_kernel<__half><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n1, (int)in.n2, (int)in.n3, m_b, inv_p1,
                                                             inv_p3, sk.rowperm, sk.rowstart, sk.colperm, sk.colstart, sel.keys,
                                                             sel.counts, kSelMaxK, d_peel, n_peel, key1, key2, sel.Rc, sel.Tc, vec);
     else
-        candidate_moments_kernel<__nv_bfloat16><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n2, m_b,
+        candidate_moments_kernel<__nv_bfloat16><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n1, (int)in.n2, (int)in.n3, m_b,
                                                                    inv_p1, inv_p3, sk.rowperm, sk.rowstart, sk.colperm,
                                                                    sk.colstart, sel.keys, sel.counts, kSelMaxK, d_peel, n_peel,
                                                                    key1, key2, sel.Rc, sel.Tc, vec);

@@ -113,6 +113,45 @@ __device__ __forceinline__ uint4 ldg_nc_v4(const void *p)
     return r;
 }
 
+// ---------------------------------------------------------------- bounds-checked build
+// With -DFPSK_DEBUG_BOUNDS every index that a kernel takes from a table (a permutation entry, a bucket
+// number, a decoded coordinate, a slot from a counter) is checked before it addresses memory: an index out of
+// range is recorded (first one per source file: line, index, limit; and a count) and the access is skipped,
+// so the kernel returns normally.  fpsk_debug_bounds_report (fpsk_test.h) reads the records.  In the product
+// build the check compiles to `true`.
+#ifdef FPSK_DEBUG_BOUNDS
+struct BoundsRecord {
+    unsigned int count;
+    int line;
+    long long index, limit;
+};
+static __device__ BoundsRecord g_bounds_tu;
+__device__ __forceinline__ bool bounds_ok(long long idx, long long limit, int line)
+{
+    if (idx >= 0 && idx < limit) return true;
+    if (atomicAdd(&g_bounds_tu.count, 1u) == 0u) {
+        g_bounds_tu.line = line;
+        g_bounds_tu.index = idx;
+        g_bounds_tu.limit = limit;
+    }
+    return false;
+}
+#define FPSK_IN_BOUNDS(idx, limit) fpsk::bounds_ok((long long)(idx), (long long)(limit), __LINE__)
+void bounds_register(const char *file, cudaError_t (*read)(BoundsRecord *), cudaError_t (*clear)());
+namespace {
+struct BoundsRegistration {
+    BoundsRegistration()
+    {
+        bounds_register(__BASE_FILE__,
+                        [](BoundsRecord *r) { return cudaMemcpyFromSymbol(r, g_bounds_tu, sizeof(*r)); },
+                        []() { BoundsRecord z = {0u, 0, 0, 0}; return cudaMemcpyToSymbol(g_bounds_tu, &z, sizeof(z)); });
+    }
+} g_bounds_registration;
+}  // namespace
+#else
+#define FPSK_IN_BOUNDS(idx, limit) true
+#endif
+
 // ---------------------------------------------------------------- bounded device-side wait
 // Spin until *ctr >= target; gives up after a fixed number of polls and returns false, so
 // that a kernel can flag FPSK_ERR_TIMEOUT and leave instead of hanging.

@@ -930,8 +930,12 @@ static HpArgs hp_args(const void *A, long long lda, const float *C, long long ld
     a.P = w ? w->P : nullptr; a.Tc = w ? w->Tc : nullptr; a.partC = w ? w->partC : nullptr;
     a.maxA = w ? w->maxA : nullptr; a.ctrl = w ? w->ctrl : nullptr;
     a.trace = w ? w->trace : nullptr;
+    a.trace_on = 0;
+#ifdef FPSK_MEASURE
+    // measurement build only: FPSK_HPROBE_TRACE records per-team phase stamps in the workspace
     static const bool trace_env = getenv("FPSK_HPROBE_TRACE") != nullptr;
     a.trace_on = trace_env ? 1 : 0;
+#endif
     return a;
 }
 
@@ -993,7 +997,12 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
     HpPlan pl;
     hp_plan(n2, n3, m, sms, pl);
     const HpArgs a = hp_args(A, lda, C, ldc, n1, n2, n3, m, pl, c, &w);
-    static const bool force_plain = getenv("FPSK_HPROBE_PLAIN") != nullptr;
+    bool force_plain = false;
+#ifdef FPSK_MEASURE
+    // measurement build only: FPSK_HPROBE_PLAIN forces the plain-load kernels
+    static const bool env_plain = getenv("FPSK_HPROBE_PLAIN") != nullptr;
+    force_plain = env_plain;
+#endif
     const bool bulk_ok = !force_plain && (reinterpret_cast<uintptr_t>(A) & 15) == 0 && (reinterpret_cast<uintptr_t>(C) & 15) == 0 &&
                          lda % 8 == 0 && ldc % 4 == 0 && n2 % 8 == 0 && n3 % 4 == 0;
     int n_maxA = sms;

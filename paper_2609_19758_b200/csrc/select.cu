@@ -576,7 +576,7 @@ __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const floa
         flag[t] += v;
         __syncthreads();
     }
-    if (keep) cand[flag[t] - 1] = c;
+    if (keep && FPSK_IN_BOUNDS(flag[t] - 1, np2)) cand[flag[t] - 1] = c;
     if (t == np2 - 1) counts[2] = flag[t];
 }
 

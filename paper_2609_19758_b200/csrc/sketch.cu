@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(256) place_kernel(const int *bucket, const int
     if (lane == 0) {
         const uint32_t sbit = __ldg(sign + idx) < 0 ? 0x80000000u : 0u;
         const uint32_t where = (uint32_t)(__ldg(start + b) + cnt);
-        perm[where] = (uint32_t)idx | sbit;
+        if (FPSK_IN_BOUNDS(where, n)) perm[where] = (uint32_t)idx | sbit;
         if (pos) pos[idx] = where | sbit;        // the inverse: where entry idx sits in the sorted order (and its sign)
     }
 }
@@ -169,6 +169,7 @@ __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A
         for (int s = s0; s < s1; ++s) {
             const uint32_t e = __ldg(rowperm + s);
             const int i = (int)(e & 0x7FFFFFFFu);
+            if (!FPSK_IN_BOUNDS(s, n1) || !FPSK_IN_BOUNDS(i, n1)) continue;
             const float sg = (e >> 31) ? -1.f : 1.f;
             uint4 v;
             if (VEC) v = ldg_nc_v4(A + (long long)i * lda + col0);
@@ -250,6 +251,7 @@ __global__ void __launch_bounds__(256) compress_b_kernel(const unsigned short *B
                 for (int s = s0; s < s1; ++s) {
                     const uint32_t e = __ldg(colperm + s);
                     const int j = (int)(e & 0x7FFFFFFFu);
+                    if (!FPSK_IN_BOUNDS(s, n3) || !FPSK_IN_BOUNDS(j, n3)) continue;
                     const float sg = (e >> 31) ? -1.f : 1.f;
                     const float x = bits16_to_float<T>(rowbuf[j]);
                     q += sg * x;
@@ -287,6 +289,7 @@ __global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *
         for (int s = s0; s < s1; ++s) {
             const uint32_t e = __ldg(colperm + s);
             const int j = (int)(e & 0x7FFFFFFFu);
+            if (!FPSK_IN_BOUNDS(s, n3) || !FPSK_IN_BOUNDS(j, n3)) continue;
             const float sg = (e >> 31) ? -1.f : 1.f;
             uint4 v;
             if (VEC) v = ldg_nc_v4(Wt + (long long)j * ldw + k0);
@@ -375,6 +378,7 @@ __global__ void __launch_bounds__(256) compress_b8_kernel(const unsigned short *
                 for (int s = s0; s < s1; ++s) {
                     const uint32_t e = __ldg(colperm + s);
                     const int j = (int)(e & 0x7FFFFFFFu);
+                    if (!FPSK_IN_BOUNDS(s, n3) || !FPSK_IN_BOUNDS(j, n3)) continue;
                     const float sg = (e >> 31) ? -1.f : 1.f;
                     const float swj = sg * ((float)(j + 1) * inv_p3);
 #pragma unroll
@@ -443,6 +447,7 @@ __global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long lon
         for (int s = q0; s < q1; ++s) {
             const uint32_t e = __ldg(rowperm + s);
             const int i = (int)(e & 0x7FFFFFFFu);
+            if (!FPSK_IN_BOUNDS(s, n1) || !FPSK_IN_BOUNDS(i, n1)) continue;
             const float v1 = (e >> 31) ? -1.f : 1.f;
             const float v1w = v1 * ((float)(i + 1) * inv_p1);
             const float *src = C + (long long)i * ldc + c0;
@@ -482,6 +487,7 @@ __global__ void __launch_bounds__(256) scatter_c_kernel(const float *C, long lon
             float fs = 0.f, fr = 0.f, ft = 0.f;
             for (int c = k0; c < k1; ++c) {
                 const uint32_t ce = __ldg(colperm + c);
+                if (!FPSK_IN_BOUNDS(c, n3) || !FPSK_IN_BOUNDS(ce & 0x7FFFFFFFu, n3)) continue;
                 const int j = (int)(ce & 0x7FFFFFFFu) - c0;
                 if (j < 0 || j >= cw) continue;
                 const float sg = (ce >> 31) ? -1.f : 1.f;
@@ -556,7 +562,7 @@ __global__ void __launch_bounds__(256, 2) scatter_c2_kernel(const float *C, long
 #pragma unroll
             for (int u = 0; u < 4; ++u) {
                 const float *src = C + (long long)(e4[u] & 0x7FFFFFFFu) * ldc + c0;
-                const bool live = sb + u < q1;
+                const bool live = sb + u < q1 && FPSK_IN_BOUNDS(sb + u, n1) && FPSK_IN_BOUNDS(e4[u] & 0x7FFFFFFFu, n1);
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
                     const int j = q * 1024 + threadIdx.x * 4;
@@ -597,6 +603,7 @@ __global__ void __launch_bounds__(256, 2) scatter_c2_kernel(const float *C, long
             for (int e = 0; e < 4; ++e) {
                 if (j + e >= cw) continue;
                 const uint32_t pos = cpe[e] & 0x7FFFFFFFu;
+                if (!FPSK_IN_BOUNDS(pos, n3)) continue;
                 const float sg = (cpe[e] >> 31) ? -1.f : 1.f;
                 ts[pos] = sg * rse[e];
                 if (MOM) {
@@ -809,6 +816,7 @@ __global__ void peel_kernel(const PeelEntry *F, int nF, uint32_t key1, uint32_t 
         hash_index(key2, (uint32_t)F[f].j, (uint32_t)m_b, b, s2);
         const double g = (double)(s1 * s2) * F[f].delta;
         const long long o = (long long)a * m_b + b;
+        if (!FPSK_IN_BOUNDS(a, m_b) || !FPSK_IN_BOUNDS(b, m_b)) continue;
         S[o] = (float)((double)S[o] - g);
         if (R) R[o] = (float)((double)R[o] - g * ((double)(F[f].i + 1) * (double)inv_p1));
         if (T) T[o] = (float)((double)T[o] - g * ((double)(F[f].j + 1) * (double)inv_p3));
@@ -888,7 +896,7 @@ __global__ void __launch_bounds__(256) place_batch_kernel(HashBatch hb)
     if (lane == 0) {
         const uint32_t sbit = __ldg(jb.sign + idx) < 0 ? 0x80000000u : 0u;
         const uint32_t where = (uint32_t)(__ldg(jb.start + b) + cnt);
-        jb.perm[where] = (uint32_t)idx | sbit;
+        if (FPSK_IN_BOUNDS(where, jb.n)) jb.perm[where] = (uint32_t)idx | sbit;
         if (jb.pos) jb.pos[idx] = where | sbit;
     }
 }
@@ -1095,7 +1103,7 @@ static SketchAuxPool &sketch_aux_pool()
 }
 SketchAuxLease::~SketchAuxLease()
 {
-    if (!aux) return;
+    if (!aux || borrowed) return;
     SketchAuxPool &pool = sketch_aux_pool();
     std::lock_guard<std::mutex> g(pool.mu);
     pool.free_list.push_back(aux);
@@ -1115,6 +1123,7 @@ fpsk_status sketch_aux_acquire(SketchAuxLease &lease)
         }
     }
     SketchAux *a = new SketchAux;
+    g_lazy_resources.fetch_add(1, std::memory_order_relaxed);
     a->device = dev;
     lease.aux = a;                  // returned to the pool even when a creation below fails (unused handles stay null)
     FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a->s1, cudaStreamNonBlocking));

@@ -28,10 +28,12 @@ struct SketchAux {
     cudaStream_t s1 = nullptr, s2 = nullptr;
     cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
 };
-struct SketchAuxLease {          // returns the set to the pool when it goes out of scope
+struct SketchAuxLease {          // returns the set to the pool when it goes out of scope (unless it is borrowed from a context)
     SketchAux *aux = nullptr;
+    bool borrowed = false;
     ~SketchAuxLease();
 };
+extern std::atomic<unsigned long long> g_lazy_resources;      // stream sets and pinned buffers the library created by itself
 fpsk_status sketch_aux_acquire(SketchAuxLease &lease);
 
 constexpr int kHashSets = 3;     // hash rounds whose tables can be prepared ahead in one batch

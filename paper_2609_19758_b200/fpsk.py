@@ -15,6 +15,9 @@ import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libfpsk.so")
+# FPSK_LIBRARY names another build of the same library to load instead (the index-checked libfpsk_bounds.so)
+if os.environ.get("FPSK_LIBRARY"):
+    LIB_PATH = os.path.abspath(os.environ["FPSK_LIBRARY"])
 
 FP16, BF16 = 0, 1
 STATUS_OK = 0
@@ -36,7 +39,7 @@ class Params(C.Structure):
                 ("s_budget", C.c_int32), ("delta_max", C.c_int32), ("mad_of_abs", C.c_int32), ("tensor_cores", C.c_int32),
                 ("b_transposed", C.c_int32), ("scale_cap", C.c_int32),
                 ("rho_min", C.c_double), ("c_valid", C.c_double), ("mu", C.c_double), ("b_star", C.c_double),
-                ("c_coll", C.c_double)]
+                ("c_coll", C.c_double), ("context", C.c_void_p)]
 
 
 class Noise(C.Structure):
@@ -150,6 +153,16 @@ def lib() -> C.CDLL:
         L.fpsk_selftest_bounded_wait.argtypes = [vp, vp, vp]
         L.fpsk_launch_count.restype = u64
         L.fpsk_launch_count.argtypes = []
+        L.fpsk_lazy_resource_count.restype = u64
+        L.fpsk_lazy_resource_count.argtypes = []
+        L.fpsk_debug_bounds_report.restype = i32
+        L.fpsk_debug_bounds_report.argtypes = [C.POINTER(i64), C.POINTER(i32), C.POINTER(i64), C.POINTER(i64), C.c_char_p, sz]
+        L.fpsk_debug_bounds_clear.restype = C.c_int
+        L.fpsk_debug_bounds_clear.argtypes = []
+        L.fpsk_context_create.restype = C.c_int
+        L.fpsk_context_create.argtypes = [C.POINTER(vp)]
+        L.fpsk_context_destroy.restype = C.c_int
+        L.fpsk_context_destroy.argtypes = [vp]
         _lib = L
     return _lib
 
@@ -168,6 +181,43 @@ def default_params(**kw) -> Params:
 
 def launch_count() -> int:
     return int(lib().fpsk_launch_count())
+
+
+def debug_bounds_report():
+    """(built_with_checks, violations, line, index, limit, source file) of the loaded library."""
+    v, ln, ix, lm = C.c_int64(-1), C.c_int32(0), C.c_int64(0), C.c_int64(0)
+    buf = C.create_string_buffer(256)
+    rc = lib().fpsk_debug_bounds_report(C.byref(v), C.byref(ln), C.byref(ix), C.byref(lm), buf, 256)
+    return int(rc), int(v.value), int(ln.value), int(ix.value), int(lm.value), buf.value.decode()
+
+
+def lazy_resource_count() -> int:
+    return int(lib().fpsk_lazy_resource_count())
+
+
+class Context:
+    """Caller-owned host resources (auxiliary streams, events, pinned buffer) of fpsk_measure_noise,
+    fpsk_localize and fpsk_verify_repair: put `ctx.ptr` into Params.context.  One call at a time."""
+
+    def __init__(self):
+        h = C.c_void_p()
+        rc = lib().fpsk_context_create(C.byref(h))
+        if rc != STATUS_OK:
+            raise FpskError(rc, "fpsk_context_create")
+        self.ptr = h.value
+
+    def close(self):
+        if self.ptr:
+            rc = lib().fpsk_context_destroy(self.ptr)
+            self.ptr = None
+            if rc != STATUS_OK:
+                raise FpskError(rc, "fpsk_context_destroy")
+
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
 
 
 def dtype_of(t: torch.Tensor) -> int:

@@ -22,10 +22,15 @@ def lib():
 
 
 def test_exports_every_declared_symbol(lib):
-    hdr = open(os.path.join(ROOT, "include", "fpsk.h")).read()
-    hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
-    names = set(re.findall(r"\b(fpsk_[a-z_0-9]+)\s*\(", hdr))
-    assert {"fpsk_probe", "fpsk_localize", "fpsk_measure_noise", "fpsk_sketches", "fpsk_plan"} <= names
+    names = set()
+    for h in sorted(os.listdir(os.path.join(ROOT, "include"))):
+        if not h.endswith(".h"):
+            continue
+        hdr = open(os.path.join(ROOT, "include", h)).read()
+        hdr = re.sub(r"/\*.*?\*/", "", hdr, flags=re.S)
+        names |= set(re.findall(r"\b(fpsk_[a-z_0-9]+)\s*\(", hdr))
+    assert {"fpsk_probe", "fpsk_localize", "fpsk_measure_noise", "fpsk_sketches", "fpsk_plan", "fpsk_context_create",
+            "fpsk_context_destroy", "fpsk_selftest_bounded_wait", "fpsk_launch_count"} <= names
     for n in names:
         assert hasattr(lib, n), n
 
@@ -33,7 +38,8 @@ def test_exports_every_declared_symbol(lib):
 def test_struct_layouts_match_header():
     assert C.sizeof(fpsk.ProbeResult) == 32
     assert C.sizeof(fpsk.Fault) == 40 and fpsk.Fault.delta.offset == 8 and fpsk.Fault.bucket_b.offset == 36
-    assert C.sizeof(fpsk.Params) == 80 and fpsk.Params.rho_min.offset == 40 and fpsk.Params.b_transposed.offset == 32
+    assert C.sizeof(fpsk.Params) == 88 and fpsk.Params.rho_min.offset == 40 and fpsk.Params.b_transposed.offset == 32
+    assert fpsk.Params.context.offset == 80
     assert C.sizeof(fpsk.Noise) == 56
 
 
