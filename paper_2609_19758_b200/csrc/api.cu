@@ -153,6 +153,7 @@ struct HostRes {
         if (aux.aux) {
             if (aux.aux->s1) cudaStreamSynchronize(aux.aux->s1);
             if (aux.aux->s2) cudaStreamSynchronize(aux.aux->s2);
+            if (aux.aux->s3) cudaStreamSynchronize(aux.aux->s3);
         }
         cudaStreamSynchronize(st);
     }
@@ -249,6 +250,7 @@ static fpsk_status check_mats(const void *A, int64_t lda, const void *B, int64_t
 struct LocWs {
     SketchWs sk;
     float *S;                 // the sum sketch of the round (R, T exist only at the kept buckets: SelectWs::Rc, Tc)
+    float *Sr[kHashSets];     // one S per round prepared ahead (Sr[0] == S): their builds run before the tails
     SelectWs sel;
     float *samples;
     float *misc;              // [0] max|A| [1] max|B| [2] tau [3] rms_c ; [8..] uint scratch
@@ -264,7 +266,7 @@ static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bo
 {
     const size_t mm = (size_t)m_b * m_b;
     size_t b = sketch_ws_bytes(n1, n2, n3, m_b, tc);
-    b += align_up(mm * 4, 256);
+    b += kHashSets * align_up(mm * 4, 256);
     b += align_up(select_ws_bytes(), 256);
     b += align_up((size_t)131072 * 4, 256);
     b += 256;
@@ -285,7 +287,8 @@ static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, lon
     if (!sketch_carve(ws, skb, n1, n2, n3, m_b, w.sk, tc)) return false;
     char *p = static_cast<char *>(ws) + skb;
     auto take = [&](size_t bytes) { void *r = p; p += align_up(bytes, 256); return r; };
-    w.S = (float *)take(mm * 4);
+    for (int q = 0; q < kHashSets; ++q) w.Sr[q] = (float *)take(mm * 4);
+    w.S = w.Sr[0];
     select_carve(take(select_ws_bytes()), w.sel);
     w.samples = (float *)take((size_t)131072 * 4);
     w.misc = (float *)take(256);
@@ -411,48 +414,83 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
     std::vector<Hit> hits(kHitCap);
     PinnedLease &stage = hr.pin;
     const size_t pack_bytes = sizeof(RoundHeader) + (size_t)K * sizeof(Candidate) + (size_t)kPackHits * sizeof(Hit);
-    // The sketches of round t + 1 do not depend on what round t finds (only the peeling does), so they
-    // are enqueued before the host waits for round t's results: the GPU builds them while the host
-    // replays the search.  The event marks the end of round t's copies.
+    // The sketches of a round do not depend on what earlier rounds find (only the peeling does; Section "Peeling
+    // Across Hash Rounds"), and the tail of a round (peel, selection, moments of the kept buckets, decode,
+    // confirmation) touches none of a build's buffers but its S.  So the builds of all rounds whose tables were
+    // prepared ahead are queued at once on the caller's stream, each into an S of its own, and every tail runs on the
+    // auxiliary stream s3 behind its build's event: the GPU runs round t's tail beside round t + 1's build, and the
+    // host replays the search of round t meanwhile.  Without auxiliary streams everything runs on the caller's stream
+    // in order, the next build queued before the host waits (as the only overlap).
     struct { cudaEvent_t e; } round_done{hr.round_done};
     // Only S is built whole.  The first moments R, T are read at the K buckets the selection keeps and nowhere else
     // (Eq. (recover)), so they are computed for those buckets alone once the keys are collected: a third of the
     // contraction, of the combine and of the plane writes.
+    const bool overlap = ax && ax->s3 && ax->evb[0] && ax->evb[1] && ax->evb[2] && ax->evt;
+    cudaStream_t ts = overlap ? ax->s3 : st;
+    const int nprep = w.sk.prepared_count > 0 ? std::min(q.rounds, w.sk.prepared_count) : 0;
+    if (overlap) {
+        if (round0_built) FPSK_CUDA_OK(cudaEventRecord(ax->evb[0], st));
+        for (int t = round0_built ? 1 : 0; t < nprep; ++t) {
+            rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.Sr[t], nullptr, nullptr);
+            if (rc != FPSK_OK) return rc;
+            FPSK_CUDA_OK(cudaEventRecord(ax->evb[t], st));
+        }
+    }
     bool built_ahead = false;
     for (int t = 0; t < q.rounds; ++t) {
-        if (!(t == 0 && round0_built) && !built_ahead) {
-            rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
-            if (rc != FPSK_OK) return rc;
+        float *S = w.S;
+        if (overlap) {
+            if (t < nprep || (t == 0 && round0_built)) {
+                S = w.Sr[t];
+                FPSK_CUDA_OK(cudaStreamWaitEvent(ts, ax->evb[t], 0));
+            } else {
+                // a round beyond the prepared ones: its tables replace those of set 0, whose round is long finished
+                rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
+                if (rc != FPSK_OK) return rc;
+                FPSK_CUDA_OK(cudaEventRecord(ax->evb[0], st));
+                FPSK_CUDA_OK(cudaStreamWaitEvent(ts, ax->evb[0], 0));
+            }
+            sketch_select_round(w.sk, seed, t);        // host side: the tables the kept buckets' moments are taken from
+        } else {
+            if (!(t == 0 && round0_built) && !built_ahead) {
+                rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
+                if (rc != FPSK_OK) return rc;
+            }
+            built_ahead = false;
         }
-        built_ahead = false;
         int np = 0;
         if (!peel.empty()) {
             np = (int)std::min<size_t>(peel.size(), kPeelCap);
             if ((int)peel.size() > kPeelCap) truncated = true;
-            FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, st));
-            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, w.S, nullptr, nullptr, st);
+            FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, ts));
+            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, S, nullptr, nullptr, ts);
             if (rc != FPSK_OK) return rc;
         }
         // sigma_MAD of this round's S rides in the launches of the K-largest selection (round 0's is already
         // there when it was needed for the radius)
         const int mad_mode = (t == 0 && round0_built) ? -1 : (q.mad_of_abs ? 1 : 0);
-        rc = select_collect_launch(w.S, m_b, m, n, w.misc + 2, radius, K, mad_mode, w.sel, st);
+        rc = select_collect_launch(S, m_b, m, n, w.misc + 2, radius, K, mad_mode, w.sel, ts);
         if (rc != FPSK_OK) return rc;
-        rc = candidate_moments_launch(in, dtype, w.sk, m_b, K, w.sel, w.peel, np, seed, t, st);
+        rc = candidate_moments_launch(in, dtype, w.sk, m_b, K, w.sel, w.peel, np, seed, t, ts);
         if (rc != FPSK_OK) return rc;
-        rc = decode_launch(w.S, nullptr, nullptr, w.sel.Rc, w.sel.Tc, m, n, w.sel, st);
+        rc = decode_launch(S, nullptr, nullptr, w.sel.Rc, w.sel.Tc, m, n, w.sel, ts);
         if (rc != FPSK_OK) return rc;
-        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, st);
+        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, ts);
         if (rc != FPSK_OK) return rc;
-        pack_round_kernel<<<1, 256, 0, st>>>(w.sel.counts, w.n_hits, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.sel.cand, K,
+        pack_round_kernel<<<1, 256, 0, ts>>>(w.sel.counts, w.n_hits, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.sel.cand, K,
                                              w.hits, w.pack);
         FPSK_LAUNCH_CHECK();
-        FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, pack_bytes, cudaMemcpyDeviceToHost, st));
-        FPSK_CUDA_OK(cudaEventRecord(round_done.e, st));
-        if (t + 1 < q.rounds) {
+        FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, pack_bytes, cudaMemcpyDeviceToHost, ts));
+        FPSK_CUDA_OK(cudaEventRecord(round_done.e, ts));
+        if (!overlap && t + 1 < q.rounds) {
             rc = build_sketches(in, dtype, seed, t + 1, m_b, false, w.sk, st, w.S, nullptr, nullptr);
             if (rc != FPSK_OK) return rc;
             built_ahead = true;
+        }
+        if (overlap && t + 1 == q.rounds) {
+            // the caller's stream continues behind the last tail
+            FPSK_CUDA_OK(cudaEventRecord(ax->evt, ts));
+            FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->evt, 0));
         }
         FPSK_CUDA_OK(cudaEventSynchronize(round_done.e));
         const RoundHeader *hdr = static_cast<const RoundHeader *>(stage.p);
@@ -468,8 +506,8 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
         } else {
             // more hits than travel with the header: fetch the list itself (the stream runs the next round's
             // sketches meanwhile; they do not touch it)
-            FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * h_nhits, cudaMemcpyDeviceToHost, st));
-            FPSK_CUDA_OK(cudaStreamSynchronize(st));
+            FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * h_nhits, cudaMemcpyDeviceToHost, ts));
+            FPSK_CUDA_OK(cudaStreamSynchronize(ts));
         }
 
         // replay of Algorithm 1's search: offsets in Chebyshev-then-Manhattan order, buckets of U
@@ -1169,10 +1207,7 @@ fpsk_status fpsk_context_create(fpsk_context **out)
     if (!out) return FPSK_ERR_NULL;
     *out = nullptr;
     fpsk_context *c = new fpsk_context;
-    bool ok = cudaGetDevice(&c->aux.device) == cudaSuccess;
-    ok = ok && cudaStreamCreateWithFlags(&c->aux.s1, cudaStreamNonBlocking) == cudaSuccess;
-    ok = ok && cudaStreamCreateWithFlags(&c->aux.s2, cudaStreamNonBlocking) == cudaSuccess;
-    for (int e = 0; e < 5 && ok; ++e) ok = cudaEventCreateWithFlags(&c->aux.ev[e], cudaEventDisableTiming) == cudaSuccess;
+    bool ok = sketch_aux_create(c->aux) == FPSK_OK;
     ok = ok && cudaEventCreateWithFlags(&c->round_done, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaHostAlloc(&c->pinned, kPackBytes, cudaHostAllocPortable) == cudaSuccess;
     if (!ok) {
@@ -1186,11 +1221,7 @@ fpsk_status fpsk_context_create(fpsk_context **out)
 fpsk_status fpsk_context_destroy(fpsk_context *c)
 {
     if (!c) return FPSK_OK;
-    bool ok = true;
-    if (c->aux.s1) ok = (cudaStreamDestroy(c->aux.s1) == cudaSuccess) && ok;
-    if (c->aux.s2) ok = (cudaStreamDestroy(c->aux.s2) == cudaSuccess) && ok;
-    for (int e = 0; e < 5; ++e)
-        if (c->aux.ev[e]) ok = (cudaEventDestroy(c->aux.ev[e]) == cudaSuccess) && ok;
+    bool ok = sketch_aux_destroy(c->aux);
     if (c->round_done) ok = (cudaEventDestroy(c->round_done) == cudaSuccess) && ok;
     if (c->pinned) ok = (cudaFreeHost(c->pinned) == cudaSuccess) && ok;
     delete c;

@@ -1124,12 +1124,44 @@ fpsk_status sketch_aux_acquire(SketchAuxLease &lease)
     }
     SketchAux *a = new SketchAux;
     g_lazy_resources.fetch_add(1, std::memory_order_relaxed);
-    a->device = dev;
     lease.aux = a;                  // returned to the pool even when a creation below fails (unused handles stay null)
-    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a->s1, cudaStreamNonBlocking));
-    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a->s2, cudaStreamNonBlocking));
-    for (int e = 0; e < 5; ++e) FPSK_CUDA_OK(cudaEventCreateWithFlags(&a->ev[e], cudaEventDisableTiming));
+    return sketch_aux_create(*a);
+}
+
+fpsk_status sketch_aux_create(SketchAux &a)
+{
+    FPSK_CUDA_OK(cudaGetDevice(&a.device));
+    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a.s1, cudaStreamNonBlocking));
+    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a.s2, cudaStreamNonBlocking));
+    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a.s3, cudaStreamNonBlocking));
+    for (int e = 0; e < 5; ++e) FPSK_CUDA_OK(cudaEventCreateWithFlags(&a.ev[e], cudaEventDisableTiming));
+    for (int e = 0; e < 3; ++e) FPSK_CUDA_OK(cudaEventCreateWithFlags(&a.evb[e], cudaEventDisableTiming));
+    FPSK_CUDA_OK(cudaEventCreateWithFlags(&a.evt, cudaEventDisableTiming));
     return FPSK_OK;
+}
+
+bool sketch_aux_destroy(SketchAux &a)
+{
+    bool ok = true;
+    if (a.s1) ok = (cudaStreamDestroy(a.s1) == cudaSuccess) && ok;
+    if (a.s2) ok = (cudaStreamDestroy(a.s2) == cudaSuccess) && ok;
+    if (a.s3) ok = (cudaStreamDestroy(a.s3) == cudaSuccess) && ok;
+    for (int e = 0; e < 5; ++e)
+        if (a.ev[e]) ok = (cudaEventDestroy(a.ev[e]) == cudaSuccess) && ok;
+    for (int e = 0; e < 3; ++e)
+        if (a.evb[e]) ok = (cudaEventDestroy(a.evb[e]) == cudaSuccess) && ok;
+    if (a.evt) ok = (cudaEventDestroy(a.evt) == cudaSuccess) && ok;
+    a = SketchAux();
+    return ok;
+}
+
+bool sketch_select_round(SketchWs &w, uint64_t seed, int rnd)
+{
+    if (w.prepared_count > 0 && seed == w.prepared_seed && rnd >= w.prepared_first && rnd < w.prepared_first + w.prepared_count) {
+        sketch_use_set(w, rnd - w.prepared_first);
+        return true;
+    }
+    return false;
 }
 
 template <typename T>

@@ -27,7 +27,14 @@ struct SketchAux {
     int device = -1;
     cudaStream_t s1 = nullptr, s2 = nullptr;
     cudaEvent_t ev[5] = {nullptr, nullptr, nullptr, nullptr, nullptr};
+    // localization: the tail of a round (selection, decode, confirmation) runs on s3 behind the event of the
+    // round's sketch build, beside the next round's build on the caller's stream
+    cudaStream_t s3 = nullptr;
+    cudaEvent_t evb[3] = {nullptr, nullptr, nullptr};       // build of prepared round q is complete
+    cudaEvent_t evt = nullptr;                              // the tails are complete
 };
+fpsk_status sketch_aux_create(SketchAux &a);     // streams and events on the current device (a.device is set)
+bool sketch_aux_destroy(SketchAux &a);
 struct SketchAuxLease {          // returns the set to the pool when it goes out of scope (unless it is borrowed from a context)
     SketchAux *aux = nullptr;
     bool borrowed = false;
@@ -35,6 +42,9 @@ struct SketchAuxLease {          // returns the set to the pool when it goes out
 };
 extern std::atomic<unsigned long long> g_lazy_resources;      // stream sets and pinned buffers the library created by itself
 fpsk_status sketch_aux_acquire(SketchAuxLease &lease);
+struct SketchWs;
+// host side only: point w at the tables of round rnd when they were prepared ahead (prepare_hash_rounds)
+bool sketch_select_round(SketchWs &w, uint64_t seed, int rnd);
 
 constexpr int kHashSets = 3;     // hash rounds whose tables can be prepared ahead in one batch
 struct HashSet {                 // the tables of one hash round

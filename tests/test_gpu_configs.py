@@ -140,7 +140,7 @@ def _run_case(kind, n1, n2, n3, dtype, seed, make_faults, params, oparams, probe
 
 
 # ------------------------------------------------------------------ config: square BF16 4096, 4 small faults
-@pytest.mark.parametrize("seed", [0, 1, 2])
+@pytest.mark.parametrize("seed", list(range(20)))          # the configuration's 20 seeds
 def test_square_bf16_4096_four_small_faults(seed):
     p = fpsk.default_params(s_budget=4)
     po = O.Params(s_budget=4)
@@ -199,7 +199,7 @@ def test_transformer_shapes_eight_faults(shape, dtype):
 
 
 # ------------------------------------------------------------------ config: square FP16 8192, 16 simultaneous faults
-@pytest.mark.parametrize("seed", [0, 1])
+@pytest.mark.parametrize("seed", list(range(10)))          # the configuration's 10 seeds
 def test_square_fp16_8192_sixteen_faults_sharing_lines(seed):
     n = 8192
     p = fpsk.default_params(s_budget=16, delta_max=4)
