@@ -336,6 +336,93 @@ __global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *
     }
 }
 
+// ---------------------------------------------------------------- compressions straight into the tiled planes
+// Row-bucket sums of a row-major half-precision matrix X (rows of A grouped by h1, or rows of W = B^T grouped by
+// h2), written as the scaled FP16 hi/lo planes of the tensor-core contraction (R-row tiles, see plane_chunk_offset).
+// A CTA takes eight consecutive buckets and 256 consecutive k: warp w owns bucket 8 * blockIdx.y + w and its lanes
+// run along k, so every row is read in one 512-byte piece (the kernels above give a warp eight buckets and read
+// 64 bytes per row and warp); up to four rows of the bucket are in flight per thread.  The sums are split, turned
+// through shared memory, and leave as full 128-byte lines: the eight buckets of a k-chunk are one line of the plane.
+// Same additions in the same order as compress_a_kernel / compress_wt_kernel: same bits.
+template <typename T, int R, bool VEC, bool MOM>
+__global__ void __launch_bounds__(256, 6) compress_planes_kernel(const unsigned short *X, long long ld, int nrows, int n2,
+                                                                 float inv_p, const uint32_t *perm, const int *start, int m_b,
+                                                                 int kblocks, unsigned char *planes, unsigned char *planes_w,
+                                                                 const float *tc_scale)
+{
+    __shared__ uint4 tile[MOM ? 4 : 2][32 * 9];          // [plane][k-chunk l][bucket w] as l * 9 + w (padded: no bank conflicts)
+    const int w = (int)threadIdx.x >> 5, l = (int)threadIdx.x & 31;
+    const int a = (int)blockIdx.y * 8 + w;
+    const int k0 = ((int)blockIdx.x * 32 + l) * 8;
+    const int kend = kblocks * 32;
+    float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, accw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    if (k0 < n2 && a < m_b) {
+        const int s0 = start[a], s1 = start[a + 1];
+        for (int sb = s0; sb < s1; sb += 4) {
+            uint32_t e[4];
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) e[u] = sb + u < s1 ? __ldg(perm + sb + u) : 0u;
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = (int)(e[u] & 0x7FFFFFFFu);
+                v[u] = make_uint4(0u, 0u, 0u, 0u);
+                if (sb + u >= s1 || !FPSK_IN_BOUNDS(sb + u, nrows) || !FPSK_IN_BOUNDS(i, nrows)) continue;
+                if (VEC) v[u] = ldg_nc_v4(X + (long long)i * ld + k0);
+                else {
+                    unsigned int ww[4] = {0, 0, 0, 0};
+                    for (int q = 0; q < 8; ++q)
+                        if (k0 + q < n2) ww[q >> 1] |= (unsigned int)X[(long long)i * ld + k0 + q] << ((q & 1) * 16);
+                    v[u] = make_uint4(ww[0], ww[1], ww[2], ww[3]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (sb + u >= s1) break;
+                const int i = (int)(e[u] & 0x7FFFFFFFu);
+                const float sg = (e[u] >> 31) ? -1.f : 1.f;
+                const float swi = sg * ((float)(i + 1) * inv_p);
+                const unsigned int ww[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float2 f = HalfTraits<T>::unpack2(ww[q]);
+                    acc[2 * q] += sg * f.x;
+                    acc[2 * q + 1] += sg * f.y;
+                    if (MOM) {
+                        accw[2 * q] = fmaf(swi, f.x, accw[2 * q]);
+                        accw[2 * q + 1] = fmaf(swi, f.y, accw[2 * q + 1]);
+                    }
+                }
+            }
+        }
+    }
+    const float sc = __ldg(tc_scale);
+    uint4 hi, lo;
+    split8_f16(acc, sc, hi, lo);
+    tile[0][l * 9 + w] = hi;
+    tile[1][l * 9 + w] = lo;
+    if (MOM) {
+        split8_f16(accw, sc, hi, lo);
+        tile[2][l * 9 + w] = hi;
+        tile[3][l * 9 + w] = lo;
+    }
+    __syncthreads();
+    // thread t stores 16-byte slot t & 7 of line t >> 3 (k-chunk): a warp writes four full lines
+    const int t = (int)threadIdx.x, lc = t >> 3, slot = t & 7;
+    const int kc0 = ((int)blockIdx.x * 32 + lc) * 8;
+    const int ab = (int)blockIdx.y * 8 + slot;
+    if (kc0 < kend) {
+        const size_t off = plane_chunk_offset<R>(ab, kc0, kblocks);
+        const int ti = lc * 9 + slot;
+        *reinterpret_cast<uint4 *>(planes + off) = tile[0][ti];
+        *reinterpret_cast<uint4 *>(planes + off + R * 64) = tile[1][ti];
+        if (MOM) {
+            *reinterpret_cast<uint4 *>(planes_w + off) = tile[2][ti];
+            *reinterpret_cast<uint4 *>(planes_w + off + R * 64) = tile[3][ti];
+        }
+    }
+}
+
 // ---------------------------------------------------------------- C scatter
 // CTA (x: bucket row a, y: split).  The rows of bucket a (ascending) are divided among the
 // splits; each row of C is staged in shared memory and folded over its columns by bucket;
@@ -1133,7 +1220,12 @@ fpsk_status sketch_aux_create(SketchAux &a)
     FPSK_CUDA_OK(cudaGetDevice(&a.device));
     FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a.s1, cudaStreamNonBlocking));
     FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a.s2, cudaStreamNonBlocking));
-    FPSK_CUDA_OK(cudaStreamCreateWithFlags(&a.s3, cudaStreamNonBlocking));
+    {
+        // the tails are short and latency-bound: their CTAs go ahead of the builds' in the queue for free SMs
+        int lo = 0, hi = 0;
+        FPSK_CUDA_OK(cudaDeviceGetStreamPriorityRange(&lo, &hi));
+        FPSK_CUDA_OK(cudaStreamCreateWithPriority(&a.s3, cudaStreamNonBlocking, hi));
+    }
     for (int e = 0; e < 5; ++e) FPSK_CUDA_OK(cudaEventCreateWithFlags(&a.ev[e], cudaEventDisableTiming));
     for (int e = 0; e < 3; ++e) FPSK_CUDA_OK(cudaEventCreateWithFlags(&a.evb[e], cudaEventDisableTiming));
     FPSK_CUDA_OK(cudaEventCreateWithFlags(&a.evt, cudaEventDisableTiming));
@@ -1220,8 +1312,11 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         dim3 grid = w.tc ? dim3((kcols / 8 + 15) / 16, (m_b + 7) / 8) : dim3((kcols / 8 + 127) / 128, m_b);
 #define FPSK_CA(V, M, PL) compress_a_kernel<T, V, M, PL><<<grid, 128, 0, st>>>(A, in.lda, n1, n2, pl.kpad, inv_p1, w.rowperm, w.rowstart, w.P, w.Pw, kblocks, w.planes[0], w.planes[1], m_b, scA)
         if (w.tc) {
-            if (vec) { if (mom) FPSK_CA(true, true, true); else FPSK_CA(true, false, true); }
-            else     { if (mom) FPSK_CA(false, true, true); else FPSK_CA(false, false, true); }
+            dim3 gp((kblocks * 32 / 8 + 31) / 32, (m_b + 7) / 8);
+#define FPSK_CP(V, M) compress_planes_kernel<T, 128, V, M><<<gp, 256, 0, st>>>(A, in.lda, n1, n2, inv_p1, w.rowperm, w.rowstart, m_b, kblocks, w.planes[0], w.planes[1], scA)
+            if (vec) { if (mom) FPSK_CP(true, true); else FPSK_CP(true, false); }
+            else     { if (mom) FPSK_CP(false, true); else FPSK_CP(false, false); }
+#undef FPSK_CP
         } else {
             if (vec) { if (mom) FPSK_CA(true, true, false); else FPSK_CA(true, false, false); }
             else     { if (mom) FPSK_CA(false, true, false); else FPSK_CA(false, false, false); }
@@ -1236,8 +1331,12 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         dim3 grid((kcols / 8 + 15) / 16, (bmax + 7) / 8);
 #define FPSK_CW(V, M, PL) compress_wt_kernel<T, V, M, PL><<<grid, 128, 0, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm, w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3], scB)
         if (w.tc) {
-            if (vec) { if (mom) FPSK_CW(true, true, true); else FPSK_CW(true, false, true); }
-            else     { if (mom) FPSK_CW(false, true, true); else FPSK_CW(false, false, true); }
+            // buckets up to the padded extent of the plane (btiles * 256): the ones beyond m_b are written as zeros
+            dim3 gp((kblocks * 32 / 8 + 31) / 32, btiles * 256 / 8);
+#define FPSK_CP(V, M) compress_planes_kernel<T, 256, V, M><<<gp, 256, 0, sB>>>(B, in.ldb, n3, n2, inv_p3, w.colperm, w.colstart, m_b, kblocks, w.planes[2], w.planes[3], scB)
+            if (vec) { if (mom) FPSK_CP(true, true); else FPSK_CP(true, false); }
+            else     { if (mom) FPSK_CP(false, true); else FPSK_CP(false, false); }
+#undef FPSK_CP
         } else {
             if (vec) { if (mom) FPSK_CW(true, true, false); else FPSK_CW(true, false, false); }
             else     { if (mom) FPSK_CW(false, true, false); else FPSK_CW(false, false, false); }
