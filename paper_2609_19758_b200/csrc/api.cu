@@ -855,7 +855,11 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
     if (m0 <= 0) m0 = m_start_of(m, k, n, dtype, q);
     if (m0 > sketch_max_buckets(m, k, n)) return FPSK_ERR_BUCKETS;
     LocWs w;
-    if (!loc_carve(workspace, ws_bytes, m, k, n, m0, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
+    // With the tensor-core contraction the B side is compressed from W = B^T (rows of W are contiguous along k):
+    // a B that comes as k x n is transposed into the workspace first, when the workspace has the room that
+    // fpsk_workspace_bytes sizes for it.  Same bits as the k x n kernels, a third less time at 16384^3.
+    bool own_wt = q.tensor_cores != 0 && !q.b_transposed && loc_carve(workspace, ws_bytes, m, k, n, m0, w, true, true) && w.sk.tc;
+    if (!own_wt && !loc_carve(workspace, ws_bytes, m, k, n, m0, w, q.tensor_cores != 0)) return FPSK_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     SketchIn in{A, B, C, m, k, n, lda, ldb, ldc, q.b_transposed};
     HostRes hr;
@@ -871,6 +875,13 @@ fpsk_status fpsk_measure_noise(const void *A, int64_t lda, const void *B, int64_
         if (w.sk.tc) {
             rc = loc_max_ab(in, dtype, w, st);
             if (rc != FPSK_OK) return rc;
+        }
+        if (own_wt && w.Wt) {
+            rc = transpose_b_launch(in.B, in.ldb, k, n, w.Wt, w.ldw, st);
+            if (rc != FPSK_OK) return rc;
+            in.B = w.Wt;
+            in.ldb = w.ldw;
+            in.bt = 1;
         }
         // The samples of C need nothing from the sketch: they are taken on the stream that will run the C scatter, ahead of
         // the build (which joins that stream before its combine).  The clipped mean and the selects both only read S:
