@@ -22,6 +22,8 @@ from . import fpsk, harness
 
 def _time(fn, iters, flush):
     evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(iters)]
+    for _ in range(2):                  # untimed: first-call set-up (kernel attributes, pooled streams, first touch of the workspace)
+        fn()
     for i in range(iters):
         flush.max()                     # evict L2 with a read; also keeps the GPU busy before the timed call
         evs[i][0].record()
