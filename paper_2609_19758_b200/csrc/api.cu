@@ -473,9 +473,9 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
         if (rc != FPSK_OK) return rc;
         rc = candidate_moments_launch(in, dtype, w.sk, m_b, K, w.sel, w.peel, np, seed, t, ts);
         if (rc != FPSK_OK) return rc;
-        rc = decode_launch(S, nullptr, nullptr, w.sel.Rc, w.sel.Tc, m, n, w.sel, ts);
+        rc = decode_launch(S, nullptr, nullptr, w.sel.Rc, w.sel.Tc, m, n, w.sel, ts, w.n_hits);
         if (rc != FPSK_OK) return rc;
-        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, ts);
+        rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, ts, true);
         if (rc != FPSK_OK) return rc;
         pack_round_kernel<<<1, 256, 0, ts>>>(w.sel.counts, w.n_hits, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.sel.cand, K,
                                              w.hits, w.pack);

@@ -249,10 +249,10 @@ fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const
 
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
                            int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
-                           cudaStream_t st)
+                           cudaStream_t st, bool hits_cleared)
 {
     if (radius < 0 || 2 * radius + 1 > kConfirmThreads) return FPSK_ERR_PARAM;
-    FPSK_CUDA_OK(cudaMemsetAsync(n_hits, 0, sizeof(int), st));
+    if (!hits_cleared) FPSK_CUDA_OK(cudaMemsetAsync(n_hits, 0, sizeof(int), st));
     dim3 grid(max_cand, 2 * radius + 1);
     const unsigned short *A = static_cast<const unsigned short *>(in.A);
     const unsigned short *B = static_cast<const unsigned short *>(in.B);

@@ -134,6 +134,15 @@ __device__ __forceinline__ void select_result(int mode, unsigned long long key, 
 struct SelChain {
     SelJob a, b, c;
     int have_b, have_c;
+    // Epilogue of a localization round's launch (collect != 0; `a` is then the K-largest selection over S): the
+    // thresholds tau_c, tau_d from sigma_MAD (just selected in slot 1, or already in scal) and the analytic cap, and
+    // the keys at or above the K-th that exceed max(tau_c, tau_d) gathered into `keys` (unsorted, count in counts[1]).
+    // Every CTA knows the K-th key and sigma_MAD when the digits are done, so this needs no further launch.
+    int collect, cap;
+    const float *taup;
+    float nmax, rad;
+    unsigned long long *keys;
+    int *counts_out;
 };
 constexpr int kChainSteps = 8;                 // digits of the longest key (64 bits)
 
@@ -239,6 +248,14 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
     unsigned long long k[2] = {0, 0}, prefix[2] = {0, 0};
     float med = scal[SC_MED];
     const bool lead = blockIdx.x == 0 && tid == 0;
+    // for the collect epilogue: sigma_MAD as it stands (replaced when this launch selects it) and the K-th key
+    float mad_local = scal[SC_MAD];
+    unsigned long long kth_local = 0ull;
+    bool top_skipped = false;
+    if (ch.collect && lead) {
+        // cleared here, used after at least one grid-wide arrival: the lead's stores precede its release there
+        ch.counts_out[0] = 0; ch.counts_out[1] = 0; ch.counts_out[2] = 0;
+    }
     // a slot-1 job that has nothing to select makes room for its successor at once
 #pragma unroll
     for (int j = 0; j < 2; ++j) {
@@ -247,6 +264,7 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
             select_initial(job[j], counts, skip, k[j]);
             job[j].shift = job[j].nbits - 8;
             if (!skip) break;
+            if (j == 0) top_skipped = true;
             if (lead) {
                 state[j * ST_WORDS + ST_SKIP] = 1;
                 state[j * ST_WORDS + ST_PREFIX] = 0;
@@ -358,6 +376,8 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
                 select_result(job[j].mode, prefix[j], false, scal);
             }
             if (job[j].mode == SEL_ABS || job[j].mode == SEL_SIGNED) med = median_value(job[j].mode, prefix[j]);
+            if (job[j].mode == SEL_DEV_ABS || job[j].mode == SEL_DEV_SIGNED) mad_local = 1.4826f * __uint_as_float((uint32_t)prefix[j]);
+            if (j == 0) kth_local = prefix[0];
             if (j == 1 && have_c) {
                 job[1] = ch.c;
                 have_c = false;
@@ -379,6 +399,26 @@ __global__ void __launch_bounds__(kSelThreads, 1) select_chain_kernel(SelChain c
             }
         }
         if (!on[0] && !on[1]) break;       // same decision in every CTA: nobody waits for a further digit
+    }
+    if (!ch.collect) return;
+    // ---- thresholds (Section "Thresholds"; Algorithm 1) and the collection of the keys above them
+    const float tau = __ldg(ch.taup);
+    const float tau_c = fminf(tau, 2.f * mad_local);
+    const float tau_d = ch.nmax * mad_local / fmaxf(ch.rad, 0.5f);
+    const float thr = fmaxf(tau_c, tau_d);
+    if (lead) {
+        scal[SC_TAUC] = tau_c;
+        scal[SC_TAUD] = tau_d;
+        scal[SC_THR] = thr;
+    }
+    const unsigned long long kth = top_skipped ? 0ull : kth_local;
+    for (long long i = (long long)blockIdx.x * kSelThreads + tid; i < ch.a.n; i += (long long)G * kSelThreads) {
+        const float av = fabsf(__ldg(ch.a.src + i));
+        if (!(av > thr)) continue;
+        const unsigned long long key = topk_key(av, i);
+        if (key < kth) continue;
+        const int slot = atomicAdd(ch.counts_out + 1, 1);
+        if (slot < ch.cap) ch.keys[slot] = key;
     }
 }
 
@@ -404,7 +444,12 @@ static int select_grid(long long n)
 
 // Runs select `a` in slot 0 and, beside it, `b` and then `c` in slot 1.  One memset (this launch's histograms
 // and arrival counter) and one cooperative launch.
-static fpsk_status run_selects(SelJob a, SelJob b, bool have_b, SelJob c, bool have_c, SelectWs &w, cudaStream_t st)
+struct SelCollect {
+    const float *taup = nullptr;
+    float nmax = 0.f, rad = 0.f;
+};
+static fpsk_status run_selects(SelJob a, SelJob b, bool have_b, SelJob c, bool have_c, SelectWs &w, cudaStream_t st,
+                               const SelCollect *collect = nullptr)
 {
     const int da = a.nbits / 8, db = have_b ? b.nbits / 8 : 0, dc = have_c ? c.nbits / 8 : 0;
     const int steps = da > db + dc ? da : db + dc;
@@ -418,6 +463,9 @@ static fpsk_status run_selects(SelJob a, SelJob b, bool have_b, SelJob c, bool h
     FPSK_CUDA_OK(cudaMemsetAsync(w.hist, 0, (size_t)(kHistBase + steps * 2 * kHistCopies * 256) * sizeof(unsigned int), st));
     SelChain ch;
     ch.a = a; ch.b = b; ch.c = c; ch.have_b = have_b ? 1 : 0; ch.have_c = have_c ? 1 : 0;
+    ch.collect = collect ? 1 : 0; ch.cap = kSelMaxK;
+    ch.taup = collect ? collect->taup : nullptr; ch.nmax = collect ? collect->nmax : 0.f; ch.rad = collect ? collect->rad : 0.f;
+    ch.keys = w.keys; ch.counts_out = w.counts;
     long long nmax = a.n;
     if (have_b && b.n > nmax) nmax = b.n;
     if (have_c && c.n > nmax) nmax = c.n;
@@ -522,9 +570,10 @@ __global__ void collect_kernel(const float *S, long long mm, const float *scal, 
 // computed for the collected keys only (Rc, Tc indexed by the key's slot in `keys`).
 __global__ void __launch_bounds__(1024) decode_kernel(const float *S, const float *R, const float *T, const float *Rc,
                                                       const float *Tc, int p1, int p3, const unsigned long long *keys,
-                                                      int *counts, int cap, Candidate *cand)
+                                                      int *counts, int cap, Candidate *cand, int *zero_word)
 {
     __shared__ unsigned long long sk[kSelMaxK];
+    if (zero_word && threadIdx.x == 0) *zero_word = 0;       // the hit counter of the confirmation launched next
     __shared__ int flag[kSelMaxK];
     __shared__ unsigned short sl[kSelMaxK];           // the slot a key came from
     const int t = threadIdx.x;
@@ -592,25 +641,21 @@ fpsk_status select_collect_launch(const float *S, int m_b, long long n1, long lo
     const SelJob top = sel_job(SEL_TOPK, 64, S, mm, K);
     const SelJob med = sel_job(mad_mode ? SEL_ABS : SEL_SIGNED, 32, S, mm, 0);
     const SelJob dev = sel_job(mad_mode ? SEL_DEV_ABS : SEL_DEV_SIGNED, 32, S, mm, 0);
-    fpsk_status rc = run_selects(top, med, mad_mode >= 0, dev, mad_mode >= 0, w, st);
-    if (rc != FPSK_OK) return rc;
-    thresholds_kernel<<<1, 32, 0, st>>>(d_tau, (float)(n1 > n3 ? n1 : n3), (float)radius, w.scal, w.counts);
-    FPSK_LAUNCH_CHECK();
-    const long long cwant = (mm + 4095) / 4096;
-    collect_kernel<<<(int)(cwant < 1 ? 1 : (cwant > 1184 ? 1184 : cwant)), 256, 0, st>>>(S, mm, w.scal, w.state, kSelMaxK, w.keys, w.counts);
-    FPSK_LAUNCH_CHECK();
-    return FPSK_OK;
+    // thresholds and collection ride at the end of the same launch (every CTA knows the K-th key and sigma_MAD there)
+    SelCollect col;
+    col.taup = d_tau; col.nmax = (float)(n1 > n3 ? n1 : n3); col.rad = (float)radius;
+    return run_selects(top, med, mad_mode >= 0, dev, mad_mode >= 0, w, st, &col);
 }
 
 // The collected keys sorted and decoded into w.cand (count in w.counts[2]); moments from the sketches R, T or, when
 // Rc is given, from the per-key values Rc, Tc.
 fpsk_status decode_launch(const float *S, const float *R, const float *T, const float *Rc, const float *Tc, long long n1,
-                          long long n3, SelectWs &w, cudaStream_t st)
+                          long long n3, SelectWs &w, cudaStream_t st, int *zero_word)
 {
     int p1 = 0, p3 = 0;
     while ((1LL << p1) < n1) ++p1;
     while ((1LL << p3) < n3) ++p3;
-    decode_kernel<<<1, kSelMaxK, 0, st>>>(S, R, T, Rc, Tc, p1, p3, w.keys, w.counts, kSelMaxK, w.cand);
+    decode_kernel<<<1, kSelMaxK, 0, st>>>(S, R, T, Rc, Tc, p1, p3, w.keys, w.counts, kSelMaxK, w.cand, zero_word);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }

@@ -138,7 +138,7 @@ fpsk_status sigma_clip_launch(const float *S, long long mm, SelectWs &w, cudaStr
 fpsk_status select_collect_launch(const float *S, int m_b, long long n1, long long n3, const float *d_tau, int radius, int K,
                                   int mad_mode, SelectWs &w, cudaStream_t st);
 fpsk_status decode_launch(const float *S, const float *R, const float *T, const float *Rc, const float *Tc, long long n1,
-                          long long n3, SelectWs &w, cudaStream_t st);
+                          long long n3, SelectWs &w, cudaStream_t st, int *zero_word = nullptr);   // zero_word: a counter cleared by the launch (the next confirmation's hits)
 fpsk_status select_candidates_launch(const float *S, const float *R, const float *T, int m_b, long long n1,
                                      long long n3, const float *d_tau, int radius, int K, int mad_mode, SelectWs &w,
                                      cudaStream_t st);
@@ -170,7 +170,7 @@ fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const
                                      const PeelEntry *d_peel, int n_peel, uint64_t seed, int rnd, cudaStream_t st);
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
                            int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
-                           cudaStream_t st);
+                           cudaStream_t st, bool hits_cleared = false);      // hits_cleared: *n_hits was zeroed by an earlier launch on st
 
 // ---- scan / patch / apply (repair.cu) ----------------------------------------------------------
 constexpr int kRepairCap = 4096;      // entries one call can scan out, patch or apply
