@@ -34,40 +34,37 @@ void bounds_register(const char *file, cudaError_t (*read)(BoundsRecord *), cuda
 
 constexpr int kHitCap = 2048;
 constexpr int kPeelCap = 4096;
-constexpr int kPackHits = 256;       // hits that travel with a round's results in one copy (more: a second copy)
 
-// What the host needs from a localization round, gathered on the device so that it is ONE copy:
-// header, the candidates, the first kPackHits hits.
-struct RoundHeader {
-    int counts[4];           // [2] = number of candidates (n_U)
-    int n_hits;
+// What the host needs from a localization, gathered on the device so that it is ONE copy at the end of the
+// call: header and the first kPackFaults confirmed faults (more: a second copy).
+constexpr int kPackFaults = 512;
+struct FinalHeader {
+    int n_faults, n_peel, truncated;
     unsigned int tc_err, sel_err;
-    int pad[9];
+    int pad[11];
 };
-static_assert(sizeof(RoundHeader) == 64, "RoundHeader is 64 bytes");
-constexpr size_t kPackBytes = sizeof(RoundHeader) + (size_t)kSelMaxK * sizeof(Candidate) + (size_t)kPackHits * sizeof(Hit);
+static_assert(sizeof(FinalHeader) == 64, "FinalHeader is 64 bytes");
+constexpr size_t kPackBytes = sizeof(FinalHeader) + (size_t)kPackFaults * sizeof(DevFault);
 
-__global__ void pack_round_kernel(const int *counts, const int *n_hits, const unsigned int *tc_err,
-                                  const unsigned int *sel_err, const Candidate *cand, int K, const Hit *hits,
+__global__ void pack_final_kernel(const int *rstate, const unsigned int *tc_err, const unsigned int *sel_err, const DevFault *F,
                                   unsigned char *pack)
 {
-    RoundHeader *h = reinterpret_cast<RoundHeader *>(pack);
-    Candidate *pc = reinterpret_cast<Candidate *>(pack + sizeof(RoundHeader));
-    Hit *ph = reinterpret_cast<Hit *>(pack + sizeof(RoundHeader) + (size_t)K * sizeof(Candidate));
-    const int nh = *n_hits;
+    FinalHeader *h = reinterpret_cast<FinalHeader *>(pack);
+    DevFault *pf = reinterpret_cast<DevFault *>(pack + sizeof(FinalHeader));
+    const int nf = rstate[0];
     if (threadIdx.x == 0) {
-        for (int q = 0; q < 4; ++q) h->counts[q] = counts[q];
-        h->n_hits = nh;
+        h->n_faults = nf;
+        h->n_peel = rstate[1];
+        h->truncated = rstate[2];
         h->tc_err = tc_err ? *tc_err : 0u;
         h->sel_err = *sel_err;
     }
-    for (int t = threadIdx.x; t < K; t += blockDim.x) pc[t] = cand[t];
-    const int np = nh < kPackHits ? nh : kPackHits;
-    for (int t = threadIdx.x; t < np; t += blockDim.x) ph[t] = hits[t];
+    const int np = nf < kPackFaults ? nf : kPackFaults;
+    for (int t = threadIdx.x; t < np; t += blockDim.x) pf[t] = F[t];
 }
 
-// Pinned host staging for the per-round results.  A pageable destination makes cudaMemcpyAsync block the host
-// until the copy has run, so the next round could not be enqueued behind this one.  Buffers are created on
+// Pinned host staging for the results.  A pageable destination makes cudaMemcpyAsync block the host until the copy
+// has run.  Buffers are created on
 // first use (one per concurrent call) and kept for the life of the process.
 struct PinnedPool {
     std::mutex mu;
@@ -254,10 +251,12 @@ struct LocWs {
     SelectWs sel;
     float *samples;
     float *misc;              // [0] max|A| [1] max|B| [2] tau [3] rms_c ; [8..] uint scratch
-    PeelEntry *peel;
+    PeelEntry *peel;          // confirmed finite faults, as the peeling needs them (device list, kPeelCap)
+    DevFault *dfaults;        // Algorithm 1's set F on the device (kPeelCap)
+    int *rstate;              // [0] faults in F, [1] entries of the peel list, [2] a list overflowed
     Hit *hits;
     int *n_hits;
-    unsigned char *pack;      // kPackBytes: a round's results in one piece
+    unsigned char *pack;      // kPackBytes: the call's results in one piece
     unsigned short *Wt;       // room for W = B^T (n3 x ldw) when B comes as k x n, else null
     long long ldw;
 };
@@ -271,6 +270,7 @@ static size_t loc_ws_bytes(long long n1, long long n2, long long n3, int m_b, bo
     b += align_up((size_t)131072 * 4, 256);
     b += 256;
     b += align_up(sizeof(PeelEntry) * kPeelCap, 256);
+    b += align_up(sizeof(DevFault) * kPeelCap, 256) + 256;
     b += align_up(sizeof(Hit) * kHitCap, 256);
     b += 256;
     b += align_up(kPackBytes, 256);
@@ -293,6 +293,8 @@ static bool loc_carve(void *ws, size_t ws_bytes, long long n1, long long n2, lon
     w.samples = (float *)take((size_t)131072 * 4);
     w.misc = (float *)take(256);
     w.peel = (PeelEntry *)take(sizeof(PeelEntry) * kPeelCap);
+    w.dfaults = (DevFault *)take(sizeof(DevFault) * kPeelCap);
+    w.rstate = (int *)take(256);
     w.hits = (Hit *)take(sizeof(Hit) * kHitCap);
     w.n_hits = (int *)take(256);
     w.pack = (unsigned char *)take(kPackBytes);
@@ -333,13 +335,6 @@ static fpsk_status read_noise_scalars(const LocWs &w, cudaStream_t st, float (&h
 __global__ void tau_kernel(float *misc, float n2)
 {
     if (threadIdx.x == 0) misc[2] = 100.f * n2 * 1.1920928955078125e-07f * misc[0] * misc[1];
-}
-
-static int offset_rank_key(int di, int dj, int r)
-{
-    // Chebyshev, then Manhattan, then d_i, then d_j (all ascending) packed into one integer
-    const int ch = std::max(abs(di), abs(dj)), mh = abs(di) + abs(dj);
-    return ((ch * 64 + mh) * 64 + (di + r)) * 64 + (dj + r);
 }
 
 // The localize part of Algorithm 2: p.rounds rounds of Algorithm 1 at m_b buckets, carrying F.
@@ -410,17 +405,15 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
     }
     radius_used = radius;
 
-    std::vector<PeelEntry> peel;
-    std::vector<Hit> hits(kHitCap);
     PinnedLease &stage = hr.pin;
-    const size_t pack_bytes = sizeof(RoundHeader) + (size_t)K * sizeof(Candidate) + (size_t)kPackHits * sizeof(Hit);
     // The sketches of a round do not depend on what earlier rounds find (only the peeling does; Section "Peeling
     // Across Hash Rounds"), and the tail of a round (peel, selection, moments of the kept buckets, decode,
-    // confirmation) touches none of a build's buffers but its S.  So the builds of all rounds whose tables were
-    // prepared ahead are queued at once on the caller's stream, each into an S of its own, and every tail runs on the
-    // auxiliary stream s3 behind its build's event: the GPU runs round t's tail beside round t + 1's build, and the
-    // host replays the search of round t meanwhile.  Without auxiliary streams everything runs on the caller's stream
-    // in order, the next build queued before the host waits (as the only overlap).
+    // confirmation, ordered search) touches none of a build's buffers but its S.  So the builds of all rounds whose
+    // tables were prepared ahead are queued at once on the caller's stream, each into an S of its own, and every tail
+    // runs on the auxiliary stream s3 behind its build's event: the GPU runs round t's tail beside round t + 1's
+    // build.  The set F and the peel list live on the device (the ordered search of Algorithm 1 over a round's hits
+    // is a one-CTA kernel), so the rounds chain on the stream and the host reads ONE packed result at the end of the
+    // call.  Without auxiliary streams everything runs on the caller's stream in order.
     struct { cudaEvent_t e; } round_done{hr.round_done};
     // Only S is built whole.  The first moments R, T are read at the K buckets the selection keeps and nowhere else
     // (Eq. (recover)), so they are computed for those buckets alone once the keys are collected: a third of the
@@ -428,6 +421,31 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
     const bool overlap = ax && ax->s3 && ax->evb[0] && ax->evb[1] && ax->evb[2] && ax->evt;
     cudaStream_t ts = overlap ? ax->s3 : st;
     const int nprep = w.sk.prepared_count > 0 ? std::min(q.rounds, w.sk.prepared_count) : 0;
+    // F as the caller hands it in (absolute repairs: found, never peeled) goes to the device first
+    const int n_fixed = (int)std::min<size_t>(F.size(), kPeelCap);
+    if ((int)F.size() > kPeelCap) truncated = true;
+    std::vector<DevFault> fixed((size_t)n_fixed);
+    for (int f = 0; f < n_fixed; ++f) {
+        DevFault d;
+        d.i = F[f].i; d.j = F[f].j; d.gamma = F[f].recompute; d.c_value = F[f].c_value; d.round = F[f].round; d.flat = -1; d.pad = 0;
+        fixed[f] = d;
+    }
+    {
+        // through the pinned staging (read again only at the end of the call, behind these copies in stream order),
+        // so that nothing here waits for the device
+        const int init[4] = {n_fixed, 0, 0, 0};
+        const bool fits = sizeof(init) + sizeof(DevFault) * (size_t)n_fixed <= kPackBytes;
+        char *hp = static_cast<char *>(stage.p);
+        if (fits) {
+            memcpy(hp, init, sizeof(init));
+            if (n_fixed) memcpy(hp + sizeof(init), fixed.data(), sizeof(DevFault) * (size_t)n_fixed);
+        }
+        FPSK_CUDA_OK(cudaMemcpyAsync(w.rstate, fits ? (const void *)hp : (const void *)init, sizeof(init), cudaMemcpyHostToDevice, st));
+        if (n_fixed)
+            FPSK_CUDA_OK(cudaMemcpyAsync(w.dfaults, fits ? (const void *)(hp + sizeof(init)) : (const void *)fixed.data(),
+                                         sizeof(DevFault) * (size_t)n_fixed, cudaMemcpyHostToDevice, st));
+        if (!fits) FPSK_CUDA_OK(cudaStreamSynchronize(st));      // pageable sources are read by the copies until here
+    }
     if (overlap) {
         if (round0_built) FPSK_CUDA_OK(cudaEventRecord(ax->evb[0], st));
         for (int t = round0_built ? 1 : 0; t < nprep; ++t) {
@@ -436,7 +454,6 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
             FPSK_CUDA_OK(cudaEventRecord(ax->evb[t], st));
         }
     }
-    bool built_ahead = false;
     for (int t = 0; t < q.rounds; ++t) {
         float *S = w.S;
         if (overlap) {
@@ -444,26 +461,21 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
                 S = w.Sr[t];
                 FPSK_CUDA_OK(cudaStreamWaitEvent(ts, ax->evb[t], 0));
             } else {
-                // a round beyond the prepared ones: its tables replace those of set 0, whose round is long finished
+                // a round beyond the prepared ones: its tables replace those of set 0, whose round must be finished
+                FPSK_CUDA_OK(cudaEventRecord(ax->evt, ts));
+                FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->evt, 0));
                 rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
                 if (rc != FPSK_OK) return rc;
                 FPSK_CUDA_OK(cudaEventRecord(ax->evb[0], st));
                 FPSK_CUDA_OK(cudaStreamWaitEvent(ts, ax->evb[0], 0));
             }
             sketch_select_round(w.sk, seed, t);        // host side: the tables the kept buckets' moments are taken from
-        } else {
-            if (!(t == 0 && round0_built) && !built_ahead) {
-                rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
-                if (rc != FPSK_OK) return rc;
-            }
-            built_ahead = false;
+        } else if (!(t == 0 && round0_built)) {
+            rc = build_sketches(in, dtype, seed, t, m_b, false, w.sk, st, w.S, nullptr, nullptr);
+            if (rc != FPSK_OK) return rc;
         }
-        int np = 0;
-        if (!peel.empty()) {
-            np = (int)std::min<size_t>(peel.size(), kPeelCap);
-            if ((int)peel.size() > kPeelCap) truncated = true;
-            FPSK_CUDA_OK(cudaMemcpyAsync(w.peel, peel.data(), sizeof(PeelEntry) * np, cudaMemcpyHostToDevice, ts));
-            rc = peel_launch(w.peel, np, seed, t, m, n, m_b, S, nullptr, nullptr, ts);
+        if (t > 0) {
+            rc = peel_launch(w.peel, 0, seed, t, m, n, m_b, S, nullptr, nullptr, ts, w.rstate + 1);
             if (rc != FPSK_OK) return rc;
         }
         // sigma_MAD of this round's S rides in the launches of the K-largest selection (round 0's is already
@@ -471,74 +483,52 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
         const int mad_mode = (t == 0 && round0_built) ? -1 : (q.mad_of_abs ? 1 : 0);
         rc = select_collect_launch(S, m_b, m, n, w.misc + 2, radius, K, mad_mode, w.sel, ts);
         if (rc != FPSK_OK) return rc;
-        rc = candidate_moments_launch(in, dtype, w.sk, m_b, K, w.sel, w.peel, np, seed, t, ts);
+        rc = candidate_moments_launch(in, dtype, w.sk, m_b, K, w.sel, w.peel, w.rstate + 1, seed, t, ts);
         if (rc != FPSK_OK) return rc;
         rc = decode_launch(S, nullptr, nullptr, w.sel.Rc, w.sel.Tc, m, n, w.sel, ts, w.n_hits);
         if (rc != FPSK_OK) return rc;
         rc = confirm_launch(in, dtype, w.sel.cand, w.sel.counts + 2, K, radius, q.c_valid, 0, w.hits, w.n_hits, kHitCap, ts, true);
         if (rc != FPSK_OK) return rc;
-        pack_round_kernel<<<1, 256, 0, ts>>>(w.sel.counts, w.n_hits, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.sel.cand, K,
-                                             w.hits, w.pack);
-        FPSK_LAUNCH_CHECK();
-        FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, pack_bytes, cudaMemcpyDeviceToHost, ts));
-        FPSK_CUDA_OK(cudaEventRecord(round_done.e, ts));
-        if (!overlap && t + 1 < q.rounds) {
-            rc = build_sketches(in, dtype, seed, t + 1, m_b, false, w.sk, st, w.S, nullptr, nullptr);
-            if (rc != FPSK_OK) return rc;
-            built_ahead = true;
-        }
-        if (overlap && t + 1 == q.rounds) {
-            // the caller's stream continues behind the last tail
-            FPSK_CUDA_OK(cudaEventRecord(ax->evt, ts));
-            FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->evt, 0));
-        }
-        FPSK_CUDA_OK(cudaEventSynchronize(round_done.e));
-        const RoundHeader *hdr = static_cast<const RoundHeader *>(stage.p);
-        const Candidate *cand = reinterpret_cast<const Candidate *>(static_cast<const char *>(stage.p) + sizeof(RoundHeader));
-        const Hit *packed_hits = reinterpret_cast<const Hit *>(static_cast<const char *>(stage.p) + sizeof(RoundHeader) +
-                                                               (size_t)K * sizeof(Candidate));
-        if (hdr->tc_err || hdr->sel_err) return FPSK_ERR_TIMEOUT;        // a bounded wait (contraction, selects) gave up
-        int h_nhits = hdr->n_hits;
-        if (h_nhits > kHitCap) { truncated = true; h_nhits = kHitCap; }
-        const int nU = std::min(hdr->counts[2], K);
-        if (h_nhits <= kPackHits) {
-            std::copy(packed_hits, packed_hits + h_nhits, hits.begin());
-        } else {
-            // more hits than travel with the header: fetch the list itself (the stream runs the next round's
-            // sketches meanwhile; they do not touch it)
-            FPSK_CUDA_OK(cudaMemcpyAsync(hits.data(), w.hits, sizeof(Hit) * h_nhits, cudaMemcpyDeviceToHost, ts));
-            FPSK_CUDA_OK(cudaStreamSynchronize(ts));
-        }
-
-        // replay of Algorithm 1's search: offsets in Chebyshev-then-Manhattan order, buckets of U
-        // in selection order; a bucket leaves U at its first accepted entry
-        std::sort(hits.begin(), hits.begin() + h_nhits, [&](const Hit &x, const Hit &y) {
-            const int kx = offset_rank_key(x.di, x.dj, radius), ky = offset_rank_key(y.di, y.dj, radius);
-            if (kx != ky) return kx < ky;
-            return x.cand < y.cand;
-        });
-        std::vector<char> alive((size_t)std::max(nU, 1), 1);
-        for (int h = 0; h < h_nhits; ++h) {
-            const Hit &x = hits[h];
-            if (x.cand < 0 || x.cand >= nU || !alive[x.cand]) continue;
-            bool inF = false;
-            for (const fpsk_fault &f : F)
-                if (f.i == x.i && f.j == x.j) { inF = true; break; }
-            if (inF) continue;
-            fpsk_fault f;
-            memset(&f, 0, sizeof(f));
-            f.i = x.i; f.j = x.j;
-            f.recompute = x.gamma;
-            f.c_value = x.c_value;
-            f.delta = x.gamma - (double)x.c_value;
-            f.round = t;
-            f.bucket_a = cand[x.cand].flat / m_b;
-            f.bucket_b = cand[x.cand].flat % m_b;
-            F.push_back(f);
-            // only finite faults are peeled (Section "Peeling Across Hash Rounds")
-            if (std::isfinite(f.delta)) peel.push_back(PeelEntry{f.i, f.j, f.delta});
-            alive[x.cand] = 0;
-        }
+        rc = replay_launch(w.hits, w.n_hits, kHitCap, w.sel.cand, w.sel.counts + 2, K, radius, t, w.dfaults, kPeelCap, w.peel,
+                           w.rstate, ts);
+        if (rc != FPSK_OK) return rc;
+    }
+    // ---- the one read of the call: header and the first kPackFaults faults
+    pack_final_kernel<<<1, 256, 0, ts>>>(w.rstate, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.dfaults, w.pack);
+    FPSK_LAUNCH_CHECK();
+    FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, kPackBytes, cudaMemcpyDeviceToHost, ts));
+    FPSK_CUDA_OK(cudaEventRecord(round_done.e, ts));
+    if (overlap) {
+        // the caller's stream continues behind the last tail
+        FPSK_CUDA_OK(cudaEventRecord(ax->evt, ts));
+        FPSK_CUDA_OK(cudaStreamWaitEvent(st, ax->evt, 0));
+    }
+    FPSK_CUDA_OK(cudaEventSynchronize(round_done.e));
+    const FinalHeader *hdr = static_cast<const FinalHeader *>(stage.p);
+    if (hdr->tc_err || hdr->sel_err) return FPSK_ERR_TIMEOUT;        // a bounded wait (contraction, selects) gave up
+    if (hdr->truncated) truncated = true;
+    const int nF = std::min(hdr->n_faults, (int)kPeelCap);
+    std::vector<DevFault> all((size_t)std::max(nF, 0));
+    const DevFault *packed = reinterpret_cast<const DevFault *>(static_cast<const char *>(stage.p) + sizeof(FinalHeader));
+    std::copy(packed, packed + std::min(nF, (int)kPackFaults), all.begin());
+    if (nF > kPackFaults) {
+        // more faults than travel with the header: fetch the rest of the list
+        FPSK_CUDA_OK(cudaMemcpyAsync(all.data() + kPackFaults, w.dfaults + kPackFaults, sizeof(DevFault) * (size_t)(nF - kPackFaults),
+                                     cudaMemcpyDeviceToHost, ts));
+        FPSK_CUDA_OK(cudaStreamSynchronize(ts));
+    }
+    for (int f = n_fixed; f < nF; ++f) {
+        const DevFault &d = all[f];
+        fpsk_fault o;
+        memset(&o, 0, sizeof(o));
+        o.i = d.i; o.j = d.j;
+        o.recompute = d.gamma;
+        o.c_value = d.c_value;
+        o.delta = d.gamma - (double)d.c_value;
+        o.round = d.round;
+        o.bucket_a = d.flat / m_b;
+        o.bucket_b = d.flat % m_b;
+        F.push_back(o);
     }
     return FPSK_OK;
 }

@@ -99,7 +99,7 @@ template <typename T>
 __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
     const unsigned short *A, long long lda, const unsigned short *B, long long ldb, int bt, const float *C, long long ldc,
     int n1, int n2, int n3, int m_b, float inv_p1, float inv_p3, const uint32_t *rowperm, const int *rowstart, const uint32_t *colperm,
-    const int *colstart, const unsigned long long *keys, const int *counts, int cap, const PeelEntry *peel, int n_peel,
+    const int *colstart, const unsigned long long *keys, const int *counts, int cap, const PeelEntry *peel, const int *d_n_peel,
     uint32_t key1, uint32_t key2, float *Rc, float *Tc, int vec)
 {
     __shared__ double sr[kMomThreads], st_[kMomThreads];
@@ -205,6 +205,7 @@ __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
     if (threadIdx.x == 0) {
         double R = sr[0], Tm = st_[0];
         // faults confirmed in earlier rounds that hash into this bucket (Algorithm 1, peeling)
+        const int n_peel = d_n_peel ? *d_n_peel : 0;
         for (int f = 0; f < n_peel; ++f) {
             int a2, b2, s1, s2;
             hash_index(key1, (uint32_t)peel[f].i, (uint32_t)m_b, a2, s1);
@@ -221,7 +222,7 @@ __global__ void __launch_bounds__(kMomThreads) candidate_moments_kernel(
 }
 
 fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const SketchWs &sk, int m_b, int K, SelectWs &sel,
-                                     const PeelEntry *d_peel, int n_peel, uint64_t seed, int rnd, cudaStream_t st)
+                                     const PeelEntry *d_peel, const int *d_n_peel, uint64_t seed, int rnd, cudaStream_t st)
 {
     if (K < 1) return FPSK_OK;
     int p1 = 0, p3 = 0;
@@ -237,11 +238,11 @@ fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const
     if (dtype == FPSK_FP16)
         candidate_moments_kernel<__half><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n1, (int)in.n2, (int)in.n3, m_b, inv_p1,
                                                             inv_p3, sk.rowperm, sk.rowstart, sk.colperm, sk.colstart, sel.keys,
-                                                            sel.counts, kSelMaxK, d_peel, n_peel, key1, key2, sel.Rc, sel.Tc, vec);
+                                                            sel.counts, kSelMaxK, d_peel, d_n_peel, key1, key2, sel.Rc, sel.Tc, vec);
     else
         candidate_moments_kernel<__nv_bfloat16><<<K, kMomThreads, 0, st>>>(A, in.lda, B, in.ldb, in.bt, in.C, in.ldc, (int)in.n1, (int)in.n2, (int)in.n3, m_b,
                                                                    inv_p1, inv_p3, sk.rowperm, sk.rowstart, sk.colperm,
-                                                                   sk.colstart, sel.keys, sel.counts, kSelMaxK, d_peel, n_peel,
+                                                                   sk.colstart, sel.keys, sel.counts, kSelMaxK, d_peel, d_n_peel,
                                                                    key1, key2, sel.Rc, sel.Tc, vec);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
@@ -263,6 +264,99 @@ fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate
         confirm_kernel<__nv_bfloat16><<<grid, kConfirmThreads, 0, st>>>(A, in.lda, B, in.ldb, in.C, in.ldc, in.n1, in.n2,
                                                                         in.n3, cand, n_cand, radius, c_valid, force, hits, n_hits,
                                                                         hit_cap, in.bt);
+    FPSK_LAUNCH_CHECK();
+    return FPSK_OK;
+}
+
+// ---------------------------------------------------------------- ordered search over a round's hits, on the device
+constexpr int kReplayThreads = 1024;
+constexpr int kReplayMaxHits = 2048;
+
+__device__ __forceinline__ unsigned int offset_rank(int di, int dj, int r)
+{
+    // Chebyshev, then Manhattan, then d_i, then d_j (all ascending) packed into one integer (< 2^23 for r <= 16)
+    const int ch = max(abs(di), abs(dj)), mh = abs(di) + abs(dj);
+    return (unsigned int)(((ch * 64 + mh) * 64 + (di + r)) * 64 + (dj + r));
+}
+
+__global__ void __launch_bounds__(kReplayThreads) replay_kernel(const Hit *hits, const int *n_hits, int hit_cap,
+                                                               const Candidate *cand, const int *n_cand, int K, int radius,
+                                                               int round, DevFault *F, int f_cap, PeelEntry *peel, int *rstate)
+{
+    __shared__ unsigned long long keys[kReplayMaxHits];       // (offset rank, candidate, hit index): all distinct
+    __shared__ unsigned char in_f[kReplayMaxHits];            // the hit's entry was confirmed in an earlier round
+    __shared__ unsigned char alive[kSelMaxK];
+    const int tid = (int)threadIdx.x;
+    int nh = *n_hits;
+    const bool over = nh > hit_cap || nh > kReplayMaxHits;
+    if (nh > hit_cap) nh = hit_cap;
+    if (nh > kReplayMaxHits) nh = kReplayMaxHits;
+    const int nU = min(*n_cand, K);
+    const int nF0 = min(rstate[0], f_cap);
+    int np2 = 1;
+    while (np2 < nh) np2 <<= 1;
+    for (int h = tid; h < np2; h += kReplayThreads) {
+        unsigned long long key = ~0ull;
+        unsigned char seen = 0;
+        if (h < nh) {
+            const Hit x = hits[h];
+            key = ((unsigned long long)offset_rank(x.di, x.dj, radius) << 32) | ((unsigned long long)(unsigned int)(x.cand & 0xFFFF) << 16) |
+                  (unsigned long long)h;
+            for (int f = 0; f < nF0; ++f)
+                if (F[f].i == x.i && F[f].j == x.j) { seen = 1; break; }
+        }
+        keys[h] = key;
+        in_f[h] = seen;
+    }
+    for (int u = tid; u < kSelMaxK; u += kReplayThreads) alive[u] = 1;
+    __syncthreads();
+    // bitonic sort, ascending, over the next power of two of the hits present
+    for (int k2 = 2; k2 <= np2; k2 <<= 1) {
+        for (int j2 = k2 >> 1; j2 > 0; j2 >>= 1) {
+            for (int t = tid; t < np2; t += kReplayThreads) {
+                const int p = t ^ j2;
+                if (p > t) {
+                    const unsigned long long a = keys[t], b = keys[p];
+                    const bool up = (t & k2) == 0;
+                    if ((a > b) == up) { keys[t] = b; keys[p] = a; }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    if (tid != 0) return;
+    int nF = nF0, nP = rstate[1], trunc = over ? 1 : 0;
+    for (int s = 0; s < nh; ++s) {
+        const int h = (int)(keys[s] & 0xFFFFull);
+        const Hit x = hits[h];
+        if (x.cand < 0 || x.cand >= nU || !alive[x.cand] || in_f[h]) continue;
+        bool dup = false;                       // the same entry reached through another bucket of this round
+        for (int f = nF0; f < nF; ++f)
+            if (F[f].i == x.i && F[f].j == x.j) { dup = true; break; }
+        if (dup) continue;
+        if (nF >= f_cap) { trunc = 1; break; }
+        DevFault d;
+        d.i = x.i; d.j = x.j; d.gamma = x.gamma; d.c_value = x.c_value; d.round = round; d.flat = cand[x.cand].flat; d.pad = 0;
+        F[nF++] = d;
+        const double delta = x.gamma - (double)x.c_value;
+        // only finite faults are peeled (Section "Peeling Across Hash Rounds")
+        if (isfinite(delta)) {
+            PeelEntry e;
+            e.i = x.i; e.j = x.j; e.delta = delta;
+            peel[nP++] = e;                     // nP <= nF <= f_cap: the lists have the same capacity
+        }
+        alive[x.cand] = 0;
+    }
+    rstate[0] = nF;
+    rstate[1] = nP;
+    if (trunc) rstate[2] = 1;
+}
+
+fpsk_status replay_launch(const Hit *hits, const int *n_hits, int hit_cap, const Candidate *cand, const int *n_cand, int K,
+                          int radius, int round, DevFault *F, int f_cap, PeelEntry *peel, int *rstate, cudaStream_t st)
+{
+    if (K > kSelMaxK) return FPSK_ERR_PARAM;
+    replay_kernel<<<1, kReplayThreads, 0, st>>>(hits, n_hits, hit_cap, cand, n_cand, K, radius, round, F, f_cap, peel, rstate);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }

@@ -893,10 +893,11 @@ __global__ void __launch_bounds__(256) combine4_kernel(const float *partAB, int 
 
 // Subtract every confirmed fault from its bucket (Algorithm 1, peeling loop).  One thread:
 // the list is short and the order of subtractions is then fixed.
-__global__ void peel_kernel(const PeelEntry *F, int nF, uint32_t key1, uint32_t key2, int m_b, float inv_p1,
+__global__ void peel_kernel(const PeelEntry *F, int nF_host, const int *d_nF, uint32_t key1, uint32_t key2, int m_b, float inv_p1,
                             float inv_p3, float *S, float *R, float *T)
 {
     if (blockIdx.x != 0 || threadIdx.x != 0) return;
+    const int nF = d_nF ? *d_nF : nF_host;
     for (int f = 0; f < nF; ++f) {
         int a, b, s1, s2;
         hash_index(key1, (uint32_t)F[f].i, (uint32_t)m_b, a, s1);
@@ -1506,12 +1507,12 @@ fpsk_status build_sketches(const SketchIn &in, fpsk_dtype dtype, uint64_t seed, 
 }
 
 fpsk_status peel_launch(const PeelEntry *dF, int nF, uint64_t seed, int rnd, long long n1, long long n3, int m_b,
-                        float *S, float *R, float *T, cudaStream_t st)
+                        float *S, float *R, float *T, cudaStream_t st, const int *d_nF)
 {
-    if (nF <= 0) return FPSK_OK;
+    if (!d_nF && nF <= 0) return FPSK_OK;
     const float inv_p1 = 1.0f / (float)(1LL << pow2_exp(n1));
     const float inv_p3 = 1.0f / (float)(1LL << pow2_exp(n3));
-    peel_kernel<<<1, 32, 0, st>>>(dF, nF, round_key(seed, rnd, 0), round_key(seed, rnd, 1), m_b, inv_p1, inv_p3, S, R, T);
+    peel_kernel<<<1, 32, 0, st>>>(dF, nF, d_nF, round_key(seed, rnd, 0), round_key(seed, rnd, 1), m_b, inv_p1, inv_p3, S, R, T);
     FPSK_LAUNCH_CHECK();
     return FPSK_OK;
 }

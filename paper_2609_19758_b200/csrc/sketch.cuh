@@ -104,7 +104,8 @@ fpsk_status contraction_launch(const float *P, const float *Q, float *part, int 
 fpsk_status build_b_side(const void *B, long long ldb, long long n2, long long n3, fpsk_dtype dtype, int m_b, int kpad,
                          int npad, const uint32_t *colperm, const int *colstart, float *Q, cudaStream_t st);
 fpsk_status peel_launch(const PeelEntry *dF, int nF, uint64_t seed, int rnd, long long n1, long long n3, int m_b,
-                        float *S, float *R, float *T, cudaStream_t st);
+                        float *S, float *R, float *T, cudaStream_t st,
+                        const int *d_nF = nullptr);      // d_nF: the count is read on the device instead (nF is ignored)
 
 // ---- selection (select.cu) -----------------------------------------------------------------
 struct Candidate {          // one decoded bucket of the set U (Algorithm 1)
@@ -162,12 +163,28 @@ struct Hit {                // an accepted window entry
     float c_value;
     double gamma;           // FP64 recomputation
 };
+// A confirmed fault as the device keeps it over the rounds of a localization (Algorithm 1's set F).
+struct DevFault {
+    int i, j;
+    double gamma;           // FP64 recomputation
+    float c_value;          // the delivered C_ij
+    int round;              // hash round that found it; < 0: an absolute repair handed in by the caller (never peeled)
+    int flat;               // its bucket a * m_b + b in that round
+    int pad;
+};
+static_assert(sizeof(DevFault) == 32, "DevFault is 32 bytes");
+// Replay of Algorithm 1's ordered search over a round's hits, on the device (one CTA): the hits sorted by offset
+// (Chebyshev, Manhattan, d_i, d_j) and then by candidate; a bucket leaves U at its first accepted entry; an entry
+// already in F is skipped.  Accepted entries are appended to F (count in rstate[0]) and, when their error is finite,
+// to the peel list (count in rstate[1]); rstate[2] is set when a list overflowed (hits, F).
+fpsk_status replay_launch(const Hit *hits, const int *n_hits, int hit_cap, const Candidate *cand, const int *n_cand, int K,
+                          int radius, int round, DevFault *F, int f_cap, PeelEntry *peel, int *rstate, cudaStream_t st);
 // force != 0: report every in-range window entry, whatever its test says
 // R, T of Eq. (recover) for the collected keys only (w.keys, count w.counts[1]) -> w.Rc, w.Tc: per key, the dot
 // products of the bucket's compressed rows of A and columns of B, the bucket's entries of C, and the peeled faults
 // that fall into the bucket.  Uses the hash tables of the round held in `sk`.
 fpsk_status candidate_moments_launch(const SketchIn &in, fpsk_dtype dtype, const SketchWs &sk, int m_b, int K, SelectWs &sel,
-                                     const PeelEntry *d_peel, int n_peel, uint64_t seed, int rnd, cudaStream_t st);
+                                     const PeelEntry *d_peel, const int *d_n_peel, uint64_t seed, int rnd, cudaStream_t st);
 fpsk_status confirm_launch(const SketchIn &in, fpsk_dtype dtype, const Candidate *cand, const int *n_cand,
                            int max_cand, int radius, double c_valid, int force, Hit *hits, int *n_hits, int hit_cap,
                            cudaStream_t st, bool hits_cleared = false);      // hits_cleared: *n_hits was zeroed by an earlier launch on st
