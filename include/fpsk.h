@@ -15,7 +15,7 @@
  *     to A or B; C is written only by fpsk_verify_repair and fpsk_apply_corrections (paper,
  *     Section "Overview": localization does not modify C; Algorithm 2, "Apply").
  *     fpsk_measure_noise, fpsk_localize and fpsk_verify_repair read their results back through a small
- *     pinned host buffer (about 25 KB) and run independent parts of a sketch build on two auxiliary
+ *     pinned host buffer (about 16 KB) and run independent parts of their work on three auxiliary
  *     non-blocking streams, tied to `stream` by events on both sides (work queued on `stream` before the
  *     call is complete before any of it starts; everything is complete when the call returns, also when
  *     it returns an error).  These host resources are the caller's when it passes a context
@@ -387,8 +387,8 @@ fpsk_status fpsk_apply_corrections(float *C, int64_t ldc, int64_t m, int64_t n, 
                                    int32_t count, void *workspace, size_t ws_bytes, void *stream);
 
 /* ---- caller-owned host resources ------------------------------------------------------------
- * fpsk_measure_noise, fpsk_localize and fpsk_verify_repair need, besides the device workspace, two auxiliary
- * non-blocking streams, six events and about 25 KB of pinned host memory (their results come back through it).
+ * fpsk_measure_noise, fpsk_localize and fpsk_verify_repair need, besides the device workspace, three auxiliary
+ * non-blocking streams, ten events and about 16 KB of pinned host memory (their results come back through it).
  * A caller that wants to own them (no creation inside those calls, release at a time of its choosing) creates a
  * context on the device it will run on, puts it into fpsk_params.context and destroys it when no call that uses
  * it is in flight.  A context serves one call at a time.  With context = NULL the library creates one such set
