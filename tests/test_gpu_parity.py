@@ -363,3 +363,50 @@ def test_a_device_wait_that_runs_out_reports_timeout_and_leaves_the_context_usab
     A, Bm, Cm = _case("uniform", 64, 64, 64, W.FP16, 3)
     got, _, _ = _run_probe(A, Bm, Cm)
     assert got.status == 0 and got.fired == 0
+
+
+# ------------------------------------------------------------------ the ordered search over the hits (device walk)
+@pytest.mark.parametrize("m_b,radius,tc", [(12, 3, 0), (24, 2, 0), (384, 4, 1)])
+def test_localize_clustered_faults_equal_the_oracle_round_by_round(m_b, radius, tc):
+    """Many faults, several of them neighbours (one bucket's window then holds several true entries, and the same
+    entry lies in the windows of several buckets), few buckets (collisions, so later rounds and the peeling matter):
+    the fault list must be the oracle's entry by entry - coordinates, the round and bucket of discovery, magnitudes -
+    which pins the order of the walk over the hits, the one-accept-per-bucket rule and the membership test in F."""
+    n1, n2, n3 = (96, 24, 80) if not tc else (768, 64, 640)
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 77, lim=6)
+    Cm = W.cpu_fp32_product(A, Bm)
+    g = np.random.default_rng(m_b * 31 + radius)
+    coords = set()
+    for _ in range(9):                                   # nine clusters of up to four adjacent entries
+        i, j = int(g.integers(1, n1 - 2)), int(g.integers(1, n3 - 2))
+        for (di, dj) in [(0, 0), (0, 1), (1, 0), (1, 1)][: int(g.integers(1, 5))]:
+            coords.add((i + di, j + dj))
+    coords = sorted(coords)
+    faults = [W.InjectedFault(i, j, "add", float(2 + (t % 7)) * (1 if t % 2 else -1), "typical") for t, (i, j) in enumerate(coords)]
+    Cf, _ = W.inject(Cm, faults)
+    p = fpsk.default_params(radius=radius, rounds=5, s_budget=len(coords), tensor_cores=tc)
+    po = O.Params(radius=radius, rounds=5, s_budget=len(coords))
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    got = fpsk.localize(A.cuda(), Bm.cuda(), Cf.cuda(), 99, m_b, ws, p)
+    ref = O.localize(_f64(A), _f64(Bm), Cf.numpy(), 99, m_b, W.FP16, po)
+    key = lambda f: (f.i, f.j, f.round, f.bucket_a, f.bucket_b, f.delta, f.c_value)
+    assert [key(f) for f in got] == [key(f) for f in ref]
+    assert {(f.i, f.j) for f in got} <= set(coords) and len(got) >= len(coords) // 2
+    # and again on the same workspace: nothing of the first call's device lists survives into the second
+    again = fpsk.localize(A.cuda(), Bm.cuda(), Cf.cuda(), 99, m_b, ws, p)
+    assert [key(f) for f in again] == [key(f) for f in got]
+
+
+def test_localize_reports_overflow_of_the_hit_list():
+    """A corrupted block larger than the hit list of a round (2048 entries): the call says so (FPSK_ERR_CAPACITY)
+    instead of returning a silently shortened list, and what it does return are true entries."""
+    n1, n2, n3, m_b = 256, 32, 256, 16
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 5, lim=6)
+    Cm = W.cpu_fp32_product(A, Bm)
+    Cf = Cm.clone()
+    Cf[100:160, 100:160] += 5.0                          # 3600 faulty entries in one 60 x 60 block
+    p = fpsk.default_params(radius=16, rounds=1, s_budget=128)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    with pytest.raises(fpsk.FpskError) as e:
+        fpsk.localize(A.cuda(), Bm.cuda(), Cf.cuda(), 3, m_b, ws, p)
+    assert e.value.status == fpsk.ERR_CAPACITY
