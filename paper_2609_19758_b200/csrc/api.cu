@@ -46,8 +46,8 @@ struct FinalHeader {
 static_assert(sizeof(FinalHeader) == 64, "FinalHeader is 64 bytes");
 constexpr size_t kPackBytes = sizeof(FinalHeader) + (size_t)kPackFaults * sizeof(DevFault);
 
-__global__ void pack_final_kernel(const int *rstate, const unsigned int *tc_err, const unsigned int *sel_err, const DevFault *F,
-                                  unsigned char *pack)
+__global__ void pack_final_kernel(const int *rstate, const unsigned int *tc_err, const unsigned int *sc_err, const unsigned int *sel_err,
+                                  const DevFault *F, unsigned char *pack)
 {
     FinalHeader *h = reinterpret_cast<FinalHeader *>(pack);
     DevFault *pf = reinterpret_cast<DevFault *>(pack + sizeof(FinalHeader));
@@ -56,7 +56,7 @@ __global__ void pack_final_kernel(const int *rstate, const unsigned int *tc_err,
         h->n_faults = nf;
         h->n_peel = rstate[1];
         h->truncated = rstate[2];
-        h->tc_err = tc_err ? *tc_err : 0u;
+        h->tc_err = (tc_err ? *tc_err : 0u) | (sc_err ? *sc_err : 0u);
         h->sel_err = *sel_err;
     }
     const int np = nf < kPackFaults ? nf : kPackFaults;
@@ -494,7 +494,7 @@ static fpsk_status localize_rounds(const SketchIn &in_caller, fpsk_dtype dtype, 
         if (rc != FPSK_OK) return rc;
     }
     // ---- the one read of the call: header and the first kPackFaults faults
-    pack_final_kernel<<<1, 256, 0, ts>>>(w.rstate, w.sk.tc ? w.sk.tc_err : nullptr, w.sel.err, w.dfaults, w.pack);
+    pack_final_kernel<<<1, 256, 0, ts>>>(w.rstate, w.sk.tc ? w.sk.tc_err : nullptr, w.sk.sc_ctrl + 1, w.sel.err, w.dfaults, w.pack);
     FPSK_LAUNCH_CHECK();
     FPSK_CUDA_OK(cudaMemcpyAsync(stage.p, w.pack, kPackBytes, cudaMemcpyDeviceToHost, ts));
     FPSK_CUDA_OK(cudaEventRecord(round_done.e, ts));

@@ -13,6 +13,7 @@
 //   combine_kernel      S = sum of AB partials - sum of C partials
 // The column side + B compression and the C scatter run on auxiliary streams when the caller provides them.
 #include "sketch.cuh"
+#include "stream_pipe.cuh"
 
 #include <mutex>
 #include <vector>
@@ -715,6 +716,327 @@ __global__ void __launch_bounds__(256, 2) scatter_c2_kernel(const float *C, long
     }
 }
 
+// ---------------------------------------------------------------- the C scatter as a producer/consumer ring
+// The same reduction as scatter_c2_kernel<false, true> (S only, aligned C), same additions in the same order, as a
+// persistent kernel: one CTA per SM; a producer warp that streams the rows of a unit (row bucket a, row split) with
+// one bulk copy per 16 KB piece of a row into a ring of shared-memory stages of two rows; sixteen consumer warps that
+// add the signed rows in registers and write the column sums of a unit to their bucket-sorted positions; and, where
+// shared memory has room for two such buffers, eight folder warps that add them up by column bucket while the
+// consumers are already on the next unit (with one buffer the consumers fold themselves).  The rows of the next
+// units are in flight all the while (in the kernels above a CTA streams, scatters and folds in turn).  Units are
+// handed out by a device counter, so CTAs that meet small buckets take more of them.  Every wait is bounded: a
+// thread that gives up sets ctrl[1], which the caller reads after the launch.
+constexpr int kSrStageBytes0 = 16384;
+constexpr int kSrConsumers = 512;
+struct SrSync {   // named barrier over the consumer warps of scatter_ring_kernel
+    static __device__ __forceinline__ void sync() { asm volatile("bar.sync 1, 512;" ::: "memory"); }
+};
+constexpr int kSrQ = kSrStageBytes0 / 16 / kSrConsumers;     // float4 per consumer thread and stage
+constexpr int kSrFolders = 256;                // warps that fold a unit's sorted column sums while the next unit's rows are added
+constexpr int kSrThreads = kSrConsumers + 32 + kSrFolders;
+constexpr int kSrRowBytes = kSrStageBytes0;   // one row of a 4096-column chunk
+constexpr int kSrRows = 2;                    // rows of a chunk per stage: the per-stage hand-over is paid once for both
+constexpr int kSrStageBytes = kSrRows * kSrRowBytes;
+constexpr int kSrStages = 4;                  // at most; fewer where the two buffers of column sums leave less room
+struct SrUnit { int a, sp, flags, pad; };     // flags: 1 nothing was added (write zeros), 2 no more units
+struct SrMeta {                               // what the consumers need to know about a stage
+    int flags;                                // 1 first rows of a chunk, 2 last rows of a chunk, 4 last stage of the unit, 8 no more units
+    int valid;                                // bit r: row r of the stage was copied
+    float sign[kSrRows];
+    int a, sp, c0, cw;
+};
+struct SrArgs {
+    const float *C;
+    long long ldc;
+    int n1, n3, m_b, nsplit, n_units, nst;    // nst: ring stages in use
+    const uint32_t *rowperm, *colpos;
+    const int *rowstart, *colstart;
+    float *part;
+    unsigned int *ctrl;                       // [0] unit counter (zero before the launch), [1] set when a bounded wait gave up
+};
+
+// Bucket sums of one unit from its sorted column sums: thread per column bucket, the columns of a bucket added in
+// their sorted order; two buckets per thread at a time, so that their loads are independent.
+static __device__ __forceinline__ void sr_fold(const float *ts, const int *cs, float *dst, int m_b, int t, int nt, bool empty_unit)
+{
+    for (int b = t; b < m_b; b += 2 * nt) {
+        const int b2 = b + nt;
+        float fa = 0.f, fb = 0.f;
+        if (!empty_unit) {
+            int ca = cs[b], cb = 0, eb = 0;
+            const int ea = cs[b + 1];
+            if (b2 < m_b) { cb = cs[b2]; eb = cs[b2 + 1]; }
+            while (ca < ea || cb < eb) {
+                const float xa = ca < ea ? ts[ca] : 0.f;
+                const float xb = cb < eb ? ts[cb] : 0.f;
+                if (ca < ea) { fa += xa; ++ca; }
+                if (cb < eb) { fb += xb; ++cb; }
+            }
+        }
+        dst[b] = fa;
+        if (b2 < m_b) dst[b2] = fb;
+    }
+}
+
+template <bool FW>     // FW: a group of folder warps and two buffers of column sums; otherwise the consumers fold, one buffer
+__global__ void __launch_bounds__(FW ? kSrThreads : kSrConsumers + 32, 1) scatter_ring_kernel(const SrArgs p)
+{
+    extern __shared__ __align__(128) unsigned char sr_smem[];
+    unsigned char *ring = sr_smem;
+    const int n3p = (p.n3 + 3) & ~3;
+    float *ts0 = reinterpret_cast<float *>(sr_smem + (size_t)p.nst * kSrStageBytes);  // sorted, signed column sums of a unit, two buffers
+    int *cs = reinterpret_cast<int *>(ts0 + (FW ? 2 : 1) * n3p);                               // bucket boundaries in the sorted order
+    SrMeta *meta = reinterpret_cast<SrMeta *>(cs + ((p.m_b + 1 + 3) & ~3));
+    SrUnit *umeta = reinterpret_cast<SrUnit *>(meta + kSrStages);
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(umeta + 2);
+    const uint32_t full0 = smem_u32(bars), empty0 = smem_u32(bars + kSrStages);
+    const uint32_t tsfull0 = smem_u32(bars + 2 * kSrStages), tsfree0 = smem_u32(bars + 2 * kSrStages + 2);
+    const int tid = (int)threadIdx.x;
+    if (tid == kSrConsumers) {
+        for (int s = 0; s < kSrStages; ++s) {
+            mbar_init(full0 + 8 * s, 1);
+            mbar_init(empty0 + 8 * s, kSrConsumers / 32);
+        }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(tsfull0 + 8 * s, kSrConsumers);
+            mbar_init(tsfree0 + 8 * s, kSrFolders);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (tid < kSrConsumers)
+        for (int b = tid; b <= p.m_b; b += kSrConsumers) cs[b] = __ldg(p.colstart + b);
+    __syncthreads();
+    const long long mm = (long long)p.m_b * p.m_b;
+    if (FW && tid >= kSrConsumers + 32) {
+        // ------------------------------------------------------------ folder warps
+        // Bucket sums of one unit: thread per column bucket, the columns of a bucket added in their sorted order.
+        const int ft = tid - (kSrConsumers + 32);
+        int fb = 0;
+        uint32_t fph = 0;                     // bit b: parity of the next phase of buffer b
+        for (;;) {
+            if (!mbar_wait_warp(tsfull0 + 8 * fb, (fph >> fb) & 1u)) { if (ft == 0) atomicOr(p.ctrl + 1, 1u); break; }
+            const SrUnit um = umeta[fb];
+            if (um.flags & 2) break;
+            const float *ts = ts0 + (size_t)fb * n3p;
+            float *dst = p.part + (long long)um.sp * 3 * mm + (long long)um.a * p.m_b;
+            const bool empty_unit = um.flags & 1;
+            sr_fold(ts, cs, dst, p.m_b, ft, kSrFolders, empty_unit);
+            mbar_arrive(tsfree0 + 8 * fb);    // every folder thread: its reads of the buffer are done
+            fph ^= 1u << fb;
+            fb ^= 1;
+        }
+        return;
+    }
+    if (tid >= kSrConsumers) {
+        // ------------------------------------------------------------ producer warp
+        // What a unit needs before its first copy can be issued is a chain of three dependent loads (unit counter,
+        // bucket boundaries, row indices), about 2 us when taken one after the other - longer than the copies of the
+        // unit take.  So the chain is a three-deep pipeline over the units: while the rows of unit k are issued, the
+        // row indices of unit k + 1, the boundaries of unit k + 2 and the number of unit k + 3 are in flight.  Lane l
+        // holds the index of row l of a unit (further groups of 32 rows are fetched in place); lane 0 issues.
+        const int lane = tid & 31;
+        int stage = 0;
+        uint32_t phase = 0;
+        bool ok = true;
+        auto next_stage = [&](const SrMeta &m, const float *src0, const float *src1, uint32_t bytes) {      // lane 0 only
+            if (!mbar_wait_bounded(empty0 + 8 * stage, phase ^ 1u)) { ok = false; return; }
+            meta[stage] = m;
+            if (m.valid) {
+                mbar_expect_tx(full0 + 8 * stage, bytes * (uint32_t)__popc(m.valid));
+                const uint32_t dst = smem_u32(ring + (size_t)stage * kSrStageBytes);
+                if (m.valid & 1) bulk_g2s(dst, src0, bytes, full0 + 8 * stage);
+                if (m.valid & 2) bulk_g2s(dst + kSrRowBytes, src1, bytes, full0 + 8 * stage);
+            } else {
+                mbar_arrive(full0 + 8 * stage);
+            }
+            if (++stage == p.nst) { stage = 0; phase ^= 1u; }
+        };
+        auto take_unit = [&]() {
+            int u = 0;
+            if (lane == 0) u = (int)atomicAdd(p.ctrl, 1u);
+            return __shfl_sync(0xFFFFFFFFu, u, 0);
+        };
+        auto bounds_of = [&](int u, int &q0, int &q1) {
+            q0 = q1 = 0;
+            if (u >= p.n_units) return;
+            const int a = u % p.m_b, sp = u / p.m_b;
+            const int s0 = __ldg(p.rowstart + a), s1 = __ldg(p.rowstart + a + 1);
+            const int cnt = s1 - s0;
+            q0 = s0 + (int)((long long)cnt * sp / p.nsplit);
+            q1 = s0 + (int)((long long)cnt * (sp + 1) / p.nsplit);
+        };
+        // prologue: fill the pipeline
+        int u_c = take_unit();                                  // unit whose rows are issued next
+        int q0_c, q1_c;
+        bounds_of(u_c, q0_c, q1_c);
+        uint32_t e_c = q0_c + lane < q1_c ? __ldg(p.rowperm + q0_c + lane) : 0u;
+        int u_b = take_unit();                                  // unit one behind: boundaries known
+        int q0_b, q1_b;
+        bounds_of(u_b, q0_b, q1_b);
+        int u_a = take_unit();                                  // unit two behind: number known
+        while (u_c < p.n_units) {
+            // the loads of the following units first (independent of one another and of the copies below)
+            const int u_new = take_unit();
+            int q0_a, q1_a;
+            bounds_of(u_a, q0_a, q1_a);
+            const uint32_t e_b = q0_b + lane < q1_b ? __ldg(p.rowperm + q0_b + lane) : 0u;
+            // ---- the rows of the present unit
+            const int a = u_c % p.m_b, sp = u_c / p.m_b;
+            if (q1_c <= q0_c) {
+                if (lane == 0) {
+                    SrMeta m = {1 | 2 | 4, 0, {0.f, 0.f}, a, sp, 0, 0};        // nothing to add: the consumers write zeros
+                    next_stage(m, nullptr, nullptr, 0);
+                }
+            } else {
+                for (int c0 = 0; c0 < p.n3; c0 += kSrRowBytes / 4) {
+                    const int cw = min(kSrRowBytes / 4, p.n3 - c0);
+                    const bool last_chunk = c0 + kSrRowBytes / 4 >= p.n3;
+                    for (int base = q0_c; base < q1_c; base += 32) {
+                        const uint32_t eg = base == q0_c ? e_c : (base + lane < q1_c ? __ldg(p.rowperm + base + lane) : 0u);
+                        const int ng = min(32, q1_c - base);
+                        for (int r = 0; r < ng; r += kSrRows) {
+                            const uint32_t e0 = __shfl_sync(0xFFFFFFFFu, eg, r);
+                            const uint32_t e1 = __shfl_sync(0xFFFFFFFFu, eg, (r + 1) & 31);
+                            if (lane != 0 || !ok) continue;
+                            const int sidx = base + r;
+                            const bool two = r + 1 < ng;
+                            const int last = sidx + (two ? 1 : 0);
+                            const int i0 = (int)(e0 & 0x7FFFFFFFu), i1 = (int)(e1 & 0x7FFFFFFFu);
+                            SrMeta m;
+                            m.flags = (sidx == q0_c ? 1 : 0) | (last == q1_c - 1 ? 2 : 0) | ((last == q1_c - 1 && last_chunk) ? 4 : 0);
+                            m.valid = 0;
+                            if (FPSK_IN_BOUNDS(sidx, p.n1) && FPSK_IN_BOUNDS(i0, p.n1)) m.valid |= 1;
+                            if (two && FPSK_IN_BOUNDS(last, p.n1) && FPSK_IN_BOUNDS(i1, p.n1)) m.valid |= 2;
+                            m.sign[0] = (e0 >> 31) ? -1.f : 1.f;
+                            m.sign[1] = (e1 >> 31) ? -1.f : 1.f;
+                            m.a = a; m.sp = sp; m.c0 = c0; m.cw = cw;
+                            next_stage(m, p.C + (long long)i0 * p.ldc + c0, p.C + (long long)i1 * p.ldc + c0, (uint32_t)cw * 4u);
+                        }
+                    }
+                }
+            }
+            if (!__shfl_sync(0xFFFFFFFFu, ok ? 1 : 0, 0)) break;
+            // ---- rotate the pipeline
+            u_c = u_b; q0_c = q0_b; q1_c = q1_b; e_c = e_b;
+            u_b = u_a; q0_b = q0_a; q1_b = q1_a;
+            u_a = u_new;
+        }
+        if (lane == 0) {
+            if (ok) {
+                SrMeta m = {8, 0, {0.f, 0.f}, 0, 0, 0, 0};
+                next_stage(m, nullptr, nullptr, 0);
+            }
+            if (!ok) {
+                atomicOr(p.ctrl + 1, 1u);
+                // before the CTA can leave: copies that may still be landing in its shared memory (bounded)
+                for (int s = 0; s < p.nst; ++s) {
+                    mbar_wait_bounded(full0 + 8 * s, 0);
+                    mbar_wait_bounded(full0 + 8 * s, 1);
+                }
+            }
+        }
+        return;
+    }
+    // ------------------------------------------------------------ consumer warps
+    int stage = 0;
+    uint32_t phase = 0;
+    int buf = 0;                              // buffer of column sums the present unit is scattered to
+    uint32_t aph = 0;                         // bit b: number of units handed over in buffer b, mod 2
+    bool unit_open = false;                   // the present unit has its buffer
+    float4 acc[kSrQ];
+    uint4 cp[kSrQ];
+    for (;;) {
+        if (!mbar_wait_warp(full0 + 8 * stage, phase)) { if (tid == 0) atomicOr(p.ctrl + 1, 1u); break; }
+        const SrMeta m = meta[stage];
+        if (m.flags & 8) {
+            if (!FW) break;
+            // no more units: tell the folders through the next buffer
+            if (!mbar_wait_warp(tsfree0 + 8 * buf, ((aph >> buf) & 1u) ^ 1u)) { if (tid == 0) atomicOr(p.ctrl + 1, 1u); break; }
+            if (tid == 0) umeta[buf] = SrUnit{0, 0, 2, 0};
+            mbar_arrive(tsfull0 + 8 * buf);
+            break;
+        }
+        if (m.flags & 1) {
+#pragma unroll
+            for (int q = 0; q < kSrQ; ++q) {
+                acc[q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                const int j = q * (kSrConsumers * 4) + tid * 4;
+                cp[q] = j < m.cw ? __ldg(reinterpret_cast<const uint4 *>(p.colpos + m.c0 + j)) : make_uint4(0, 0, 0, 0);
+            }
+        }
+#pragma unroll
+        for (int r = 0; r < kSrRows; ++r) {
+            if (!((m.valid >> r) & 1)) continue;
+            const float *row = reinterpret_cast<const float *>(ring + (size_t)stage * kSrStageBytes + (size_t)r * kSrRowBytes);
+            const float sg = m.sign[r];
+#pragma unroll
+            for (int q = 0; q < kSrQ; ++q) {
+                const int j = q * (kSrConsumers * 4) + tid * 4;
+                if (j < m.cw) {
+                    const float4 x = *reinterpret_cast<const float4 *>(row + j);
+                    acc[q].x = fmaf(sg, x.x, acc[q].x); acc[q].y = fmaf(sg, x.y, acc[q].y);
+                    acc[q].z = fmaf(sg, x.z, acc[q].z); acc[q].w = fmaf(sg, x.w, acc[q].w);
+                }
+            }
+        }
+        __syncwarp();
+        if ((tid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
+        if (++stage == p.nst) { stage = 0; phase ^= 1u; }
+        if (m.flags & 2) {
+            // the chunk's column sums, signed, to the positions their columns have in the bucket-sorted order; the
+            // buffer must have been folded (two units ago) before the first of them is written
+            if (FW && !unit_open) {
+                if (!mbar_wait_warp(tsfree0 + 8 * buf, ((aph >> buf) & 1u) ^ 1u)) { if (tid == 0) atomicOr(p.ctrl + 1, 1u); break; }
+                unit_open = true;
+            }
+            float *ts = ts0 + (size_t)buf * n3p;
+#pragma unroll
+            for (int q = 0; q < kSrQ; ++q) {
+                const int j = q * (kSrConsumers * 4) + tid * 4;
+                const uint32_t cpe[4] = {cp[q].x, cp[q].y, cp[q].z, cp[q].w};
+                const float rse[4] = {acc[q].x, acc[q].y, acc[q].z, acc[q].w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (j + e >= m.cw) continue;
+                    const uint32_t pos = cpe[e] & 0x7FFFFFFFu;
+                    if (!FPSK_IN_BOUNDS(pos, p.n3)) continue;
+                    ts[pos] = ((cpe[e] >> 31) ? -1.f : 1.f) * rse[e];
+                }
+            }
+        }
+        if (m.flags & 4) {
+            if (FW) {
+                // hand the unit to the folders: every consumer thread arrives after its own writes
+                if (tid == 0) umeta[buf] = SrUnit{m.a, m.sp, m.cw == 0 ? 1 : 0, 0};
+                mbar_arrive(tsfull0 + 8 * buf);
+                aph ^= 1u << buf;
+                buf ^= 1;
+                unit_open = false;
+            } else {
+                float *dst = p.part + (long long)m.sp * 3 * mm + (long long)m.a * p.m_b;
+                SrSync::sync();
+                sr_fold(ts0, cs, dst, p.m_b, tid, kSrConsumers, m.cw == 0);
+                SrSync::sync();       // the buffer is rewritten by the next unit
+            }
+        }
+    }
+}
+
+static size_t scatter_ring_fixed(int n3, int m_b, bool fw)
+{
+    return (size_t)(fw ? 2 : 1) * ((n3 + 3) & ~3) * 4 + (size_t)((m_b + 1 + 3) & ~3) * 4 + kSrStages * sizeof(SrMeta) + 2 * sizeof(SrUnit) +
+           (2 * kSrStages + 4) * 8 + 128;
+}
+// Ring stages that fit beside the buffers of column sums (0: this form does not fit).
+static int scatter_ring_stages(int n3, int m_b, bool fw)
+{
+    const size_t fixed = scatter_ring_fixed(n3, m_b, fw), budget = 224 * 1024;
+    if (fixed + 2 * (size_t)kSrStageBytes > budget) return 0;
+    const size_t nst = (budget - fixed) / kSrStageBytes;
+    return (int)(nst > (size_t)kSrStages ? kSrStages : nst);
+}
+
 // ---------------------------------------------------------------- FP32 SIMT contraction
 // C[M x N] = A[M x K] * B[K x N], all row-major, K a multiple of BK, FP32 FMA only (the
 // sketch noise is the measured quantity, so no reduced-precision tensor-core path here).
@@ -1071,6 +1393,7 @@ size_t sketch_ws_bytes(long long n1, long long n2, long long n3, int m_b, bool t
     b += align_up((size_t)(pl.ksplit > tcks ? pl.ksplit : tcks) * 3 * mm * 4, 256);      // AB partials
     if (tc) b += align_up(tc_planes_bytes(m_b, pl.kpad), 256) * 4 + 512;          // FP16 planes of P, Pw, Q^T, Qw^T; error word; scales
     b += align_up((size_t)pl.nsplit * 3 * mm * 4, 256);      // C partials
+    b += 256;                                                // control words of the ring scatter
     return b;
 }
 
@@ -1108,6 +1431,7 @@ bool sketch_carve(void *ws, size_t ws_bytes, long long n1, long long n2, long lo
     w.tc_scale = tc ? (float *)take(256) : nullptr;
     w.d_maxab = nullptr;
     w.partC = (float *)take((size_t)w.pl.nsplit * 3 * mm * 4);
+    w.sc_ctrl = (unsigned int *)take(256);
     return true;
 }
 
@@ -1397,7 +1721,33 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
         scatter_c2_kernel<M, V><<<grid, 256, smem2, sC>>>(in.C, in.ldc, n1, n3, m_b, inv_p1, inv_p3, w.rowperm, w.rowstart, \
                                                           w.colpos, w.colstart, pl.nsplit, w.partC);                          \
     } while (0)
-        if (n3 <= kSc2MaxCols) {
+        // the ring form with folder warps where both buffers leave room for the whole ring, with folding consumers where one does
+        const bool ring_fw = scatter_ring_stages(n3, m_b, true) == kSrStages;
+        const bool ring_fits = ring_fw || scatter_ring_stages(n3, m_b, false) == kSrStages;
+        // measured: the ring form wins from about 150 MB of C (268 MB: 73 against 83 us, 1 GB: 233 against 302 us) and loses
+        // below (67 MB: 30 against 27 us), where its longer start is not made up
+        const bool ring_any = ring_fits && (long long)n1 * n3 >= (40LL << 20);
+        FPSK_CUDA_OK(cudaMemsetAsync(w.sc_ctrl, 0, 8, sC));       // unit counter and give-up flag of the ring form (the flag is read whichever form runs)
+        if (!mom && vec && n3 <= kSc2MaxCols && ring_any) {
+            // S only, aligned C: the persistent producer/consumer form (same bits)
+            static std::once_flag once;
+            static cudaError_t attr_err = cudaSuccess;
+            std::call_once(once, [] {
+                attr_err = cudaFuncSetAttribute(scatter_ring_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+                if (attr_err == cudaSuccess)
+                    attr_err = cudaFuncSetAttribute(scatter_ring_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024);
+            });
+            if (attr_err != cudaSuccess) return FPSK_ERR_CUDA;
+            SrArgs sa;
+            sa.C = in.C; sa.ldc = in.ldc; sa.n1 = n1; sa.n3 = n3; sa.m_b = m_b; sa.nsplit = pl.nsplit; sa.n_units = m_b * pl.nsplit; sa.nst = kSrStages;
+            sa.rowperm = w.rowperm; sa.colpos = w.colpos; sa.rowstart = w.rowstart; sa.colstart = w.colstart;
+            sa.part = w.partC; sa.ctrl = w.sc_ctrl;
+            const int sms = sketch_sms();
+            const size_t smem_ring = (size_t)kSrStages * kSrStageBytes + scatter_ring_fixed(n3, m_b, ring_fw);
+            const int grid = sa.n_units < sms ? sa.n_units : sms;
+            if (ring_fw) scatter_ring_kernel<true><<<grid, kSrThreads, smem_ring, sC>>>(sa);
+            else scatter_ring_kernel<false><<<grid, kSrConsumers + 32, smem_ring, sC>>>(sa);
+        } else if (n3 <= kSc2MaxCols) {
             if (mom) { if (vec) FPSK_SC2(true, true); else FPSK_SC2(true, false); }
             else     { if (vec) FPSK_SC2(false, true); else FPSK_SC2(false, false); }
         } else {

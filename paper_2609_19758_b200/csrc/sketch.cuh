@@ -68,6 +68,7 @@ struct SketchWs {
     int tc_ksplit;
     unsigned char *planes[4];    // P, Pw, Q^T, Qw^T as tiled FP16 planes (hi, lo)
     unsigned int *tc_err;        // set by the contraction when a wait gave up
+    unsigned int *sc_ctrl;       // ring scatter: [0] unit counter, [1] set when a bounded wait gave up
     float *tc_scale;             // [0], [1]: powers of two that bring P, Pw and Q, Qw into FP16 range (device)
     const float *d_maxab;        // [0] max|A|, [1] max|B| (device; set by the caller before a tensor-core build)
 };
