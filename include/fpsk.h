@@ -263,7 +263,12 @@ int32_t fpsk_bside_matches(const fpsk_bside *side, const void *B, int64_t ldb, u
  *   d_S           device, n_buckets^2 floats receiving S, or NULL
  *   d_state       device, accumulated into by the last kernel of the call, or NULL
  * sigma_hat is the noise at this bucket count and feeds fpsk_plan directly.
- * Asynchronous on `stream`, no host synchronisation; deterministic. */
+ * Launches on a matching B side: three kernels (stream of A and C, contraction, combine and verdict).  With
+ * p->tensor_cores = 1, n_buckets <= 256, A and C aligned to 16 bytes and k % 8 == 0, n % 4 == 0, lda % 8 == 0,
+ * ldc % 4 == 0: one cooperative kernel (A streams first and leaves as FP16 planes scaled per bucket and column
+ * segment, the first CTAs contract them with the cached planes of B H2^T on the tensor cores while the others
+ * stream C, then all combine); S then differs from the three-kernel form by the rounding of the contraction only.
+ * Asynchronous on `stream`, no host synchronisation; deterministic (bit-identical from call to call in either form). */
 fpsk_status fpsk_probe_hashed(fpsk_bside *side, const void *A, int64_t lda, const void *B, int64_t ldb,
                               uint64_t b_version, const float *C, int64_t ldc, int64_t m, int64_t k, int64_t n,
                               fpsk_dtype dtype, int c_is_fp32, uint64_t seed, int32_t round, int32_t n_buckets,

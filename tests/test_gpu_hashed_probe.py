@@ -312,3 +312,110 @@ def test_transposed_weight_layout(shape, m, dtype):
     hp_p = fpsk.HashedProbe(n1, n2, n3, m, seed=17, rnd=1, b_transposed=True)
     got_p, S_p = _run(hp_p, A.cuda(), big[:, :n2], Cm.cuda())
     assert np.array_equal(S_p, S_t)
+
+
+# ---------------------------------------------------------------- the probe as one launch
+# With tensor_cores = 1, at most 256 buckets and inputs the bulk copies can address, stream, contraction, combine and
+# verdict run as one cooperative kernel (P goes to the tensor cores as FP16 planes scaled per bucket and column
+# segment of A).  What it returns is held to the same bars as the three-launch form.
+FUSED_SHAPES = [
+    # (n1, n2, n3, m)
+    (1024, 4096, 1024, 256),      # two column segments of A, one item per contracting CTA
+    (512, 6152, 768, 128),        # a ragged last segment, one row tile
+    (384, 2048 * 20, 256, 256),   # twenty segments: more items than contracting CTAs (a CTA takes several in turn)
+    (2048, 520, 1028, 200),       # buckets that do not fill the second row tile, K below one segment
+]
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES)
+@pytest.mark.parametrize("dtype", [W.FP16, W.BF16])
+def test_one_launch_form_against_the_oracle(shape, dtype):
+    n1, n2, n3, m = shape
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, dtype, 7)
+    A64, B64 = _f64(A), _f64(Bm)
+    ref, S_ref = O.probe_hashed(A64, B64, Cm.numpy(), 33, 2, m)
+    h1, _ = O.hash_round(33, 2, 0, n1, m)
+    h2, _ = O.hash_round(33, 2, 1, n3, m)
+    denom = O.abs_sketch(O.abs_product(A64, B64), h1, h2, m)
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=33, rnd=2)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    pr = fpsk.default_params(tensor_cores=1)
+    _run(hp, dA, dB, dC, params=pr)                                   # builds the B side
+    n0 = fpsk.launch_count()
+    got, S = _run(hp, dA, dB, dC, params=pr)
+    assert fpsk.launch_count() - n0 == 1                              # the whole probe was one kernel
+    assert got.status == 0
+    assert np.all(np.abs(S - S_ref) <= TOL * denom + 1e-30)
+    assert got.tau == pytest.approx(ref.tau, rel=1e-6)
+    v = O.probe_verdict(S.ravel(), ref.tau, n_rows=1)
+    assert got.sigma_hat == pytest.approx(v.sigma_hat, rel=1e-4, abs=1e-30)
+    assert got.thr == pytest.approx(v.thr, rel=1e-4, abs=1e-30)
+    assert got.max_abs == pytest.approx(v.max_abs, rel=1e-6, abs=1e-30)
+    assert got.argmax_col == v.argmax_col and got.nonfinite == 0
+    # bit-identical from call to call, and against the three-launch form within the rounding of the two contractions
+    got2, S2 = _run(hp, dA, dB, dC, params=pr)
+    assert np.array_equal(S, S2) and got2.sigma_hat == got.sigma_hat
+    n0 = fpsk.launch_count()
+    got3, S3 = _run(hp, dA, dB, dC, params=fpsk.default_params(tensor_cores=0))
+    assert fpsk.launch_count() - n0 == 3
+    assert np.all(np.abs(S3 - S) <= 2 * TOL * denom + 1e-30)
+    # a fault of a few percent of rms(C) fires in both forms at the same bucket
+    f = W.faults_additive(n1, n3, W.rms(Cm), 3, 1, 0.05, 0.09, "small")
+    Cf, _ = W.inject(Cm, f)
+    dCf = Cf.cuda()
+    g1, _ = _run(hp, dA, dB, dCf, params=pr)
+    g0, _ = _run(hp, dA, dB, dCf, params=fpsk.default_params(tensor_cores=0))
+    want = int(h1[f[0].i]) * m + int(h2[f[0].j])
+    assert g1.fired == 1 and g0.fired == 1 and g1.argmax_col == g0.argmax_col == want
+
+
+def test_one_launch_form_integer_products_and_nonfinite():
+    n1, n2, n3, m = 768, 4104, 512, 256
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 9)
+    Cm = W.cpu_fp32_product(A, Bm)
+    Cm[5, 7] += 4.0
+    ref, S_ref = O.probe_hashed(_f64(A), _f64(Bm), Cm.numpy(), 2, 0, m)
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=2)
+    pr = fpsk.default_params(tensor_cores=1)
+    dA, dB = A.cuda(), Bm.cuda()
+    got, S = _run(hp, dA, dB, Cm.cuda(), params=pr)
+    assert np.array_equal(S, S_ref)                                   # integers survive the split into two FP16 terms exactly
+    assert got.fired == 1 and got.argmax_col == ref.argmax_col and got.max_abs == ref.max_abs
+    for bad in (float("nan"), float("inf")):
+        Cb = Cm.clone()
+        Cb[100, 100] = bad
+        got, _ = _run(hp, dA, dB, Cb.cuda(), params=pr)
+        assert got.status == 0 and got.fired == 1 and got.nonfinite == 1
+    Ab = A.clone()
+    Ab[17, 2050] = float("inf")                                       # a non-finite operand: its bucket's planes carry it
+    got, _ = _run(hp, Ab.cuda(), dB, Cm.cuda(), params=pr)
+    assert got.status == 0 and got.fired == 1 and got.nonfinite == 1
+
+
+def test_one_launch_form_replays_from_a_cuda_graph():
+    n1, n2, n3, m = 1024, 4096, 1024, 256
+    A, Bm, Cm = _case("gauss_scaled", n1, n2, n3, W.BF16, 23)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda().clone()
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=4)
+    pr = fpsk.default_params(tensor_cores=1)
+    res = fpsk.new_probe_result()
+    state = fpsk.new_probe_state()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        hp(dA, dB, dC, res, params=pr)
+    side.synchronize()
+    r0 = fpsk.read_probe_result(res)
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        hp(dA, dB, dC, res, params=pr, state=state)
+    for _ in range(4):
+        g.replay()
+    torch.cuda.synchronize()
+    st = fpsk.read_probe_state(state)
+    assert (st.calls, st.clean_calls, st.fired_any) == (4, 4, 0)
+    assert st.sigma_sum == 4 * float(np.float32(r0.sigma_hat))
+    dC[10, 20] += 0.5
+    g.replay()
+    torch.cuda.synchronize()
+    st = fpsk.read_probe_state(state)
+    assert (st.calls, st.fired_any, st.first_fired_call) == (5, 1, 5)
