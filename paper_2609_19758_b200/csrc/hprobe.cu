@@ -724,9 +724,15 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
                         }
                         __syncwarp();
                         if (tr && lane == 0 && first) { p.trace[(c * 2 + team) * 8 + 1] = hp_gtime(); first = false; }
-                        if (lane < np)
-                            bulk_g2s(smem_u32(ring + (size_t)stage * kHpStageBytes) + (uint32_t)lane * kHpPieceBytes,
-                                     base_p + (long long)row * ldb, (uint32_t)wbytes, full0 + 8 * stage);
+                        if (lane < np) {
+                            // a row index or a segment out of range (bounds-checked build): row 0 of segment 0 is copied
+                            // instead, so that the stage still completes
+                            const bool in = FPSK_IN_BOUNDS(row, p.n1) && FPSK_IN_BOUNDS(seg, isC ? p.segsC : p.segsA);
+                            const unsigned char *src = in ? base_p + (long long)row * ldb
+                                                          : (isC ? reinterpret_cast<const unsigned char *>(p.C) : reinterpret_cast<const unsigned char *>(p.A));
+                            bulk_g2s(smem_u32(ring + (size_t)stage * kHpStageBytes) + (uint32_t)lane * kHpPieceBytes, src, (uint32_t)wbytes,
+                                     full0 + 8 * stage);
+                        }
                         if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
                     }
                     if (lastmask || !ok || nxt < 0) break;
@@ -975,8 +981,11 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
             if ((tid & 31) == 0) mbar_arrive(empty0 + 8 * stage);
             if (++stage == kHpStages) { stage = 0; phase ^= 1u; }
             if (last) {
-                // unit complete
-                if (isC) {
+                // unit complete (a bucket or a segment out of range, bounds-checked build: its sums are dropped)
+                const bool unit_ok = FPSK_IN_BOUNDS(a, p.m) && FPSK_IN_BOUNDS(seg, isC ? p.segsC : p.segsA);
+                if (!unit_ok) {
+                    if (isC) ++ncunit; else ++naunit;
+                } else if (isC) {
                     // the segment's signed row-bucket sums go through shared memory; thread b then folds the
                     // columns of bucket b (ascending) into partC[seg][a][b].  Two buffers: the barrier of
                     // the next C unit separates this unit's reads from the writes of the one after.
@@ -998,7 +1007,8 @@ __global__ void __launch_bounds__(kHpThreads, 1) hp_stream_kernel(const HpArgs p
                             for (int q = 0; q < 4; ++q) e[q] = s + q < s1 ? __ldg(sp + s + q) : 0u;
 #pragma unroll
                             for (int q = 0; q < 4; ++q) {
-                                const float x = tb[e[q] & 0x7FFFFFFFu];
+                                const uint32_t ci = e[q] & 0x7FFFFFFFu;
+                                const float x = FPSK_IN_BOUNDS(ci, kHpSegC) ? tb[ci] : 0.f;
                                 if (s + q < s1) cf += (e[q] >> 31) ? -x : x;
                             }
                         }

@@ -50,7 +50,11 @@ for (n1, n2, n3, dt, m_b) in [(77, 33, 255, W.FP16, 16), (300, 40, 520, W.BF16, 
         _, rrep = fpsk.verify_repair(A.cuda(), Bm.cuda(), Cr, 5, rws, m_b, p)
         hp = fpsk.HashedProbe(n1, n2, n3, min(m_b, 64), seed=9)
         hp(dA, dB, dC, res)
+        # contiguous operands: where the sizes allow, the bulk-copy kernels (with tc = 1 the single-launch form)
+        hp2 = fpsk.HashedProbe(n1, n2, n3, min(m_b, 64), seed=9)
+        hp2(A.cuda(), Bm.cuda(), Cf.cuda(), res, params=p)
         torch.cuda.synchronize()
+        fired = fired and fpsk.read_probe_result(res).fired and fpsk.read_probe_result(res).status == 0
         done.append(dict(shape=[n1, n2, n3], tc=tc, fired=int(fired), found=sorted((f.i, f.j) for f in got) == sorted(coords),
                          found_t=sorted((f.i, f.j) for f in got_t) == sorted(coords), repaired=int(rrep.state == 1),
                          restored=bool(torch.equal(Cr.cpu(), Cm))))
