@@ -167,29 +167,44 @@ __global__ void __launch_bounds__(128) compress_a_kernel(const unsigned short *A
     float acc[8] = {0, 0, 0, 0, 0, 0, 0, 0}, accw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (col0 < n2 && a < m_b) {
         const int s0 = rowstart[a], s1 = rowstart[a + 1];
-        for (int s = s0; s < s1; ++s) {
-            const uint32_t e = __ldg(rowperm + s);
-            const int i = (int)(e & 0x7FFFFFFFu);
-            if (!FPSK_IN_BOUNDS(s, n1) || !FPSK_IN_BOUNDS(i, n1)) continue;
-            const float sg = (e >> 31) ? -1.f : 1.f;
-            uint4 v;
-            if (VEC) v = ldg_nc_v4(A + (long long)i * lda + col0);
-            else {
-                unsigned int w[4] = {0, 0, 0, 0};
-                for (int q = 0; q < 8; ++q)
-                    if (col0 + q < n2) w[q >> 1] |= (unsigned int)A[(long long)i * lda + col0 + q] << ((q & 1) * 16);
-                v = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            const float swi = sg * ((float)(i + 1) * inv_p1);
-            const unsigned int ww[4] = {v.x, v.y, v.z, v.w};
+        // eight rows in flight (a bucket of the noise measurement has a hundred rows: one load at a time is all latency);
+        // the additions stay in row order
+        for (int s = s0; s < s1; s += 8) {
+            uint32_t e[8];
+            uint4 v[8];
+            bool ok[8];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                float2 f = HalfTraits<T>::unpack2(ww[q]);
-                acc[2 * q] += sg * f.x;
-                acc[2 * q + 1] += sg * f.y;
-                if (MOM) {
-                    accw[2 * q] = fmaf(swi, f.x, accw[2 * q]);
-                    accw[2 * q + 1] = fmaf(swi, f.y, accw[2 * q + 1]);
+            for (int u = 0; u < 8; ++u) {
+                e[u] = s + u < s1 ? __ldg(rowperm + s + u) : 0u;
+                const int i = (int)(e[u] & 0x7FFFFFFFu);
+                ok[u] = s + u < s1 && FPSK_IN_BOUNDS(s + u, n1) && FPSK_IN_BOUNDS(i, n1);
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (ok[u]) {
+                    if (VEC) v[u] = ldg_nc_v4(A + (long long)i * lda + col0);
+                    else {
+                        unsigned int w[4] = {0, 0, 0, 0};
+                        for (int q = 0; q < 8; ++q)
+                            if (col0 + q < n2) w[q >> 1] |= (unsigned int)A[(long long)i * lda + col0 + q] << ((q & 1) * 16);
+                        v[u] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (!ok[u]) continue;
+                const int i = (int)(e[u] & 0x7FFFFFFFu);
+                const float sg = (e[u] >> 31) ? -1.f : 1.f;
+                const float swi = sg * ((float)(i + 1) * inv_p1);
+                const unsigned int ww[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    float2 f = HalfTraits<T>::unpack2(ww[q]);
+                    acc[2 * q] += sg * f.x;
+                    acc[2 * q + 1] += sg * f.y;
+                    if (MOM) {
+                        accw[2 * q] = fmaf(swi, f.x, accw[2 * q]);
+                        accw[2 * q + 1] = fmaf(swi, f.y, accw[2 * q + 1]);
+                    }
                 }
             }
         }
@@ -287,29 +302,43 @@ __global__ void __launch_bounds__(128) compress_wt_kernel(const unsigned short *
     float q[8] = {0, 0, 0, 0, 0, 0, 0, 0}, qw[8] = {0, 0, 0, 0, 0, 0, 0, 0};
     if (k0 < n2 && b < m_b) {
         const int s0 = colstart[b], s1 = colstart[b + 1];
-        for (int s = s0; s < s1; ++s) {
-            const uint32_t e = __ldg(colperm + s);
-            const int j = (int)(e & 0x7FFFFFFFu);
-            if (!FPSK_IN_BOUNDS(s, n3) || !FPSK_IN_BOUNDS(j, n3)) continue;
-            const float sg = (e >> 31) ? -1.f : 1.f;
-            uint4 v;
-            if (VEC) v = ldg_nc_v4(Wt + (long long)j * ldw + k0);
-            else {
-                unsigned int w[4] = {0, 0, 0, 0};
-                for (int t = 0; t < 8; ++t)
-                    if (k0 + t < n2) w[t >> 1] |= (unsigned int)Wt[(long long)j * ldw + k0 + t] << ((t & 1) * 16);
-                v = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-            const float swj = sg * ((float)(j + 1) * inv_p3);
-            const unsigned int ww[4] = {v.x, v.y, v.z, v.w};
+        // eight rows of W in flight, the additions in row order (as in compress_a_kernel)
+        for (int s = s0; s < s1; s += 8) {
+            uint32_t e[8];
+            uint4 v[8];
+            bool ok[8];
 #pragma unroll
-            for (int t = 0; t < 4; ++t) {
-                float2 f = HalfTraits<T>::unpack2(ww[t]);
-                q[2 * t] += sg * f.x;
-                q[2 * t + 1] += sg * f.y;
-                if (MOM) {
-                    qw[2 * t] = fmaf(swj, f.x, qw[2 * t]);
-                    qw[2 * t + 1] = fmaf(swj, f.y, qw[2 * t + 1]);
+            for (int u = 0; u < 8; ++u) {
+                e[u] = s + u < s1 ? __ldg(colperm + s + u) : 0u;
+                const int j = (int)(e[u] & 0x7FFFFFFFu);
+                ok[u] = s + u < s1 && FPSK_IN_BOUNDS(s + u, n3) && FPSK_IN_BOUNDS(j, n3);
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (ok[u]) {
+                    if (VEC) v[u] = ldg_nc_v4(Wt + (long long)j * ldw + k0);
+                    else {
+                        unsigned int w[4] = {0, 0, 0, 0};
+                        for (int t = 0; t < 8; ++t)
+                            if (k0 + t < n2) w[t >> 1] |= (unsigned int)Wt[(long long)j * ldw + k0 + t] << ((t & 1) * 16);
+                        v[u] = make_uint4(w[0], w[1], w[2], w[3]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                if (!ok[u]) continue;
+                const int j = (int)(e[u] & 0x7FFFFFFFu);
+                const float sg = (e[u] >> 31) ? -1.f : 1.f;
+                const float swj = sg * ((float)(j + 1) * inv_p3);
+                const unsigned int ww[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                    float2 f = HalfTraits<T>::unpack2(ww[t]);
+                    q[2 * t] += sg * f.x;
+                    q[2 * t + 1] += sg * f.y;
+                    if (MOM) {
+                        qw[2 * t] = fmaf(swj, f.x, qw[2 * t]);
+                        qw[2 * t + 1] = fmaf(swj, f.y, qw[2 * t + 1]);
+                    }
                 }
             }
         }
@@ -433,16 +462,65 @@ __global__ void __launch_bounds__(256, 6) compress_planes_kernel(const unsigned 
 // BF16 planes (PLANES: emitted directly, K extent kblocks * 32 and bucket extent btiles * 256, zero
 // padded; otherwise FP32 rows of Q, Qw as above).  Same order of additions per row as the kernel above.
 template <typename T, bool MOM, bool PLANES>
-__global__ void __launch_bounds__(256) compress_b8_kernel(const unsigned short *B, long long ldb, int n2, int n3,
+__global__ void __launch_bounds__(1024) compress_b8_kernel(const unsigned short *B, long long ldb, int n2, int n3,
                                                           int kpad, int m_b, int npad, float inv_p3,
                                                           const uint32_t *colperm, const int *colstart, float *Q,
                                                           float *Qw, int kblocks, int btiles, unsigned char *planesQ,
-                                                          unsigned char *planesQw, const float *tc_scale)
+                                                          unsigned char *planesQw, const float *tc_scale, const uint32_t *colpos)
 {
     extern __shared__ __align__(16) unsigned short rowbuf8[];
     const int n3p = (n3 + 7) & ~7;
     const int kend = PLANES ? kblocks * 32 : kpad;
     const int bmax = PLANES ? btiles * 256 : npad;
+    // S only into FP32 Q, aligned B (the noise measurement below the tensor cores' bucket count): the eight rows go into
+    // shared memory in bucket-sorted column order, sign applied (colpos: position and sign of every column), and a
+    // thread per (bucket, row) adds a contiguous run - the bucket's columns in ascending order, as below: the same
+    // additions in the same order, without the gather through the column list and with every thread at work also
+    // when the buckets are few.
+    const bool sorted_rows = !PLANES && !MOM && n3 % 8 == 0 && ldb % 8 == 0 && (reinterpret_cast<uintptr_t>(B) & 15) == 0;
+    if (sorted_rows) {
+        const int rs = n3p + 2;               // row stride in shared memory: the eight rows of a bucket's run fall into eight banks
+        for (int k0 = blockIdx.x * 8; k0 < kend; k0 += gridDim.x * 8) {
+            __syncthreads();
+            for (int j = threadIdx.x * 8; j < n3; j += blockDim.x * 8) {
+                const uint4 c0 = __ldg(reinterpret_cast<const uint4 *>(colpos + j)), c1 = __ldg(reinterpret_cast<const uint4 *>(colpos + j + 4));
+                const uint32_t cp[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                uint4 v[8];
+#pragma unroll
+                for (int r = 0; r < 8; ++r) v[r] = k0 + r < n2 ? ldg_nc_v4(B + (long long)(k0 + r) * ldb + j) : make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int r = 0; r < 8; ++r) {
+                    const unsigned int ww[4] = {v[r].x, v[r].y, v[r].z, v[r].w};
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        const uint32_t pos = cp[q] & 0x7FFFFFFFu;
+                        if (!FPSK_IN_BOUNDS(pos, n3)) continue;
+                        const unsigned short h = (unsigned short)(ww[q >> 1] >> ((q & 1) * 16));
+                        rowbuf8[(size_t)r * rs + pos] = (unsigned short)(h ^ ((cp[q] >> 31) ? 0x8000u : 0u));
+                    }
+                }
+            }
+            __syncthreads();
+            for (int it = threadIdx.x; it < bmax * 8; it += blockDim.x) {
+                const int b = it >> 3, r = it & 7;
+                float q1 = 0.f;
+                if (b < m_b) {
+                    const int s0 = __ldg(colstart + b), s1 = __ldg(colstart + b + 1);
+                    const unsigned short *rowp = rowbuf8 + (size_t)r * rs;
+                    for (int sx = s0; sx < s1; sx += 8) {
+                        unsigned short h[8];              // eight loads in flight, then added in order
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) h[u] = sx + u < s1 ? rowp[sx + u] : (unsigned short)0;
+#pragma unroll
+                        for (int u = 0; u < 8; ++u)
+                            if (sx + u < s1) q1 += bits16_to_float<T>(h[u]);
+                    }
+                }
+                if (k0 + r < kpad) Q[(long long)(k0 + r) * npad + b] = q1;
+            }
+        }
+        return;
+    }
     for (int k0 = blockIdx.x * 8; k0 < kend; k0 += gridDim.x * 8) {
         __syncthreads();
         for (int r = 0; r < 8; ++r) {
@@ -1630,7 +1708,7 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
     // With the tensor-core contraction the compressions emit the tiled BF16 planes themselves (no FP32 P, Q).
     const int kblocks = (pl.kpad + 31) / 32;
     const int btiles = (m_b + 255) / 256;
-    const bool b8 = (size_t)16 * ((n3 + 7) & ~7) <= 160 * 1024;      // eight rows of B fit in shared memory
+    const bool b8 = (size_t)16 * (((n3 + 7) & ~7) + 2) <= 160 * 1024;      // eight rows of B fit in shared memory
     {
         const bool vec = (reinterpret_cast<uintptr_t>(in.A) & 15) == 0 && in.lda % 8 == 0 && n2 % 8 == 0;
         const int kcols = w.tc ? kblocks * 32 : pl.kpad;
@@ -1669,14 +1747,17 @@ static fpsk_status build_sketches_t(const SketchIn &in, uint64_t seed, int rnd, 
 #undef FPSK_CW
         FPSK_LAUNCH_CHECK();
     } else if (b8) {
-        const size_t smem = (size_t)16 * ((n3 + 7) & ~7);
+        const size_t smem = (size_t)16 * (((n3 + 7) & ~7) + 2);      // eight rows of 16-bit values (+ the padding of the sorted form)
         const int groups = (w.tc ? kblocks * 32 : pl.kpad) / 8;
         const int grid = groups < 888 ? groups : 888;
+        // the sorted-row form (S only, FP32 Q, aligned B) is instruction-bound on its scattered 16-bit stores and holds one
+        // CTA per SM at 8192 columns: 32 warps instead of 8
+        const bool sorted8 = n3 % 8 == 0 && in.ldb % 8 == 0 && (reinterpret_cast<uintptr_t>(B) & 15) == 0;
 #define FPSK_CB8(M, PL)                                                                                                          \
     do {                                                                                                                         \
         FPSK_CUDA_OK(cudaFuncSetAttribute(compress_b8_kernel<T, M, PL>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)); \
-        compress_b8_kernel<T, M, PL><<<grid, 256, smem, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm,      \
-                                                              w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3], scB); \
+        compress_b8_kernel<T, M, PL><<<grid, (!PL && !M && sorted8) ? 1024 : 256, smem, sB>>>(B, in.ldb, n2, n3, pl.kpad, m_b, pl.npad, inv_p3, w.colperm,      \
+                                                              w.colstart, w.Q, w.Qw, kblocks, btiles, w.planes[2], w.planes[3], scB, w.colpos); \
     } while (0)
         if (w.tc) { if (mom) FPSK_CB8(true, true); else FPSK_CB8(false, true); }
         else      { if (mom) FPSK_CB8(true, false); else FPSK_CB8(false, false); }
