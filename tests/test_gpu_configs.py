@@ -274,3 +274,39 @@ def test_noise_constant_sweep_and_exponent():
         assert 0.05 < a.c_hat < 5.0
     e = math.log(chat[4096] / chat[1024]) / math.log(4.0)
     assert -0.3 < e < 1.0
+
+
+# ---------------------------------------------------------------- the C scatter at the sizes where it runs as a ring
+# From about 160 MB of C the S only scatter is the persistent producer/consumer kernel (with folder warps up to 8192
+# columns, with folding consumers at 16384).  Integer operands make every FP32 sum exact, so S must equal the oracle's
+# explicit-E sketch bit for bit whichever kernel, split count or tail shape produced it; the inner dimension is kept
+# short so that the oracle's E is cheap.
+@pytest.mark.parametrize("n1,n3,m_b,tensor_cores", [
+    (8192, 8192, 2048, 1),      # folder warps, one row split, tensor-core contraction behind it
+    (8200, 8192, 48, 0),        # few buckets: many row splits per bucket, a ragged row count
+    (4096, 16384, 1024, 1),     # 16384 columns: one buffer of column sums, the consumers fold
+    (5000, 12288, 384, 0),      # three column chunks, the last rows of a bucket split unevenly
+])
+def test_ring_scatter_shapes_bit_exact_on_integers(n1, n3, m_b, tensor_cores):
+    n2 = 32
+    A, Bm = W.operands("integer", n1, n2, n3, W.FP16, 6, lim=4)
+    Cm = W.cpu_fp32_product(A, Bm)
+    Cm[n1 - 1, n3 - 1] += 3.0
+    Cm[n1 // 2, 7] -= 2.0
+    Cm[3, n3 // 2] += 1.0
+    p = fpsk.default_params(tensor_cores=tensor_cores)
+    ws = fpsk.workspace(n1, n2, n3, m_b, p)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    n0 = fpsk.launch_count()
+    S, _, _ = fpsk.sketches(dA, dB, dC, 91, 2, m_b, ws, moments=False, params=p)
+    S_again, _, _ = fpsk.sketches(dA, dB, dC, 91, 2, m_b, ws, moments=False, params=p)
+    torch.cuda.synchronize()
+    assert fpsk.launch_count() > n0
+    E = O.error_matrix(A.double().numpy(), Bm.double().numpy(), Cm.numpy())
+    h1, v1 = O.hash_round(91, 2, 0, n1, m_b)
+    h2, v2 = O.hash_round(91, 2, 1, n3, m_b)
+    So = O.hashed_sum_sketch(E, h1, v1, h2, v2, m_b)
+    got = S.cpu().numpy().astype(np.float64)
+    assert np.array_equal(got, So)
+    assert np.array_equal(S_again.cpu().numpy(), S.cpu().numpy())
+    assert int(np.count_nonzero(So)) == 3
