@@ -77,7 +77,11 @@ def run(sizes=(1024, 2048, 4096, 8192, 16384), iters=20, tensor_cores=0, dtypes=
                 sets.append((A, Bm, harness.vendor_gemm_fp32(A, Bm)))
             A, Bm, C = sets[0]
             p = fpsk.default_params(tensor_cores=tensor_cores)
-            ws0 = fpsk.workspace(n, n, n, 0, p)
+            # one workspace for the measurement and the localization, sized for the largest bucket count the plan can ask
+            # for (as bench.py does): the measurement then has room to transpose B once instead of compressing it as k x n
+            mb_cap = min(fpsk.max_buckets(n, n, n), max(16, int((n * n // 16) ** 0.5)))
+            mb_cap = max(mb_cap, fpsk.law_m_start(n, n, n, dt_name == "bf16" and 1 or 0, p))
+            ws0 = fpsk.workspace(n, n, n, mb_cap, p)
             nz = fpsk.measure_noise(A, Bm, C, 7, ws0, 0, p)
             pws = fpsk.probe_workspace(n, n, n)
             res = fpsk.new_probe_result()
@@ -89,7 +93,6 @@ def run(sizes=(1024, 2048, 4096, 8192, 16384), iters=20, tensor_cores=0, dtypes=
                 burst_ms = _burst(lambda q: (lambda: fpsk.probe(sets[q][0], sets[q][1], sets[q][2], pws, res, None, p)), nsets)
             gemm_ms, _ = _time(lambda: harness.vendor_gemm_fp32(A, Bm), it, flush)
             noise_ms, _ = _time(lambda: fpsk.measure_noise(A, Bm, C, 7, ws0, 0, p), max(3, it // 4), flush)
-            del ws0
             row = dict(n=n, dtype=dt_name, tensor_cores=tensor_cores, c_hat=nz.c_hat, sigma_clip=nz.sigma_clip, sigma_mad=nz.sigma_mad,
                        rms_c=nz.rms_c, m0=nz.m0, m_probe=nz.m_probe, m_loc=nz.m_loc, radius=nz.radius, probe_ms=probe_ms,
                        probe_ms_min=probe_min, probe_gbs=nbytes / probe_ms / 1e6, probe_ms_burst=burst_ms,
@@ -97,12 +100,11 @@ def run(sizes=(1024, 2048, 4096, 8192, 16384), iters=20, tensor_cores=0, dtypes=
                        measure_noise_ms=noise_ms, clean_fired=int(verdict.fired))
             if with_localize:
                 p.radius = nz.radius
-                m_loc = min(nz.m_loc, fpsk.max_buckets(n, n, n))
-                ws = fpsk.workspace(n, n, n, m_loc, p)
+                m_loc = min(nz.m_loc, mb_cap)
                 found = []
-                loc_ms, _ = _time(lambda: found.append(len(fpsk.localize(A, Bm, C, 7, m_loc, ws, p))), max(3, it // 4), flush)
+                loc_ms, _ = _time(lambda: found.append(len(fpsk.localize(A, Bm, C, 7, m_loc, ws0, p))), max(3, it // 4), flush)
                 row.update(localize_ms=loc_ms, clean_faults_reported=max(found) if found else 0)
-                del ws
+            del ws0
             rows.append(row)
             if emit:
                 emit(row)
