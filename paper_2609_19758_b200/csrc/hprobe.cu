@@ -1573,9 +1573,16 @@ fpsk_status hprobe_launch(const void *A, long long lda, const float *C, long lon
             v.partAB = w.partAB; v.ksplit = pl.segsA * pl.f_nsub; v.n_maxA = sms;
             void *args[] = {(void *)&a, (void *)&v};
             const void *fn = dtype == FPSK_FP16 ? (const void *)hp_stream_kernel<__half, true> : (const void *)hp_stream_kernel<__nv_bfloat16, true>;
-            FPSK_CUDA_OK(cudaLaunchCooperativeKernel(fn, dim3(sms), dim3(kHpThreads), args, kHpSmem, st));
-            count_launch();
-            return FPSK_OK;
+            // (fn is hp_stream_kernel<T, true>)  Where the device cannot hold the whole grid at once (fewer SMs available to
+            // this context than it reports), the launch is refused and the three-launch form below runs instead.
+            const cudaError_t le = cudaLaunchCooperativeKernel(fn, dim3(sms), dim3(kHpThreads), args, kHpSmem, st);
+            if (le == cudaSuccess) {
+                count_launch();
+                return FPSK_OK;
+            }
+            if (le != cudaErrorCooperativeLaunchTooLarge) return FPSK_ERR_CUDA;
+            (void)cudaGetLastError();
+            v.partAB = w.partAB; v.ksplit = 0; v.n_maxA = 0;
         }
         if (dtype == FPSK_FP16) hp_stream_kernel<__half, false><<<sms, kHpThreads, kHpSmem, st>>>(a, v);
         else hp_stream_kernel<__nv_bfloat16, false><<<sms, kHpThreads, kHpSmem, st>>>(a, v);
