@@ -419,3 +419,31 @@ def test_one_launch_form_replays_from_a_cuda_graph():
     torch.cuda.synchronize()
     st = fpsk.read_probe_state(state)
     assert (st.calls, st.fired_any, st.first_fired_call) == (5, 1, 5)
+
+
+@pytest.mark.parametrize("shape", [(100, 512, 64, 256), (40, 8, 8, 256), (4096, 16, 4096, 200), (2056, 6152, 1028, 129)])
+def test_one_launch_form_sparse_buckets_and_short_inner_dimensions(shape):
+    """More buckets than rows or columns (most buckets empty), an inner dimension below one K block, a bucket count
+    that fills neither row tile: S, tau and the verdict still follow the oracle's."""
+    n1, n2, n3, m = shape
+    A, Bm = W.operands("gauss_scaled", n1, n2, n3, W.BF16, 3)
+    Cm = W.cpu_fp32_product(A, Bm)
+    A64, B64 = _f64(A), _f64(Bm)
+    ref, S_ref = O.probe_hashed(A64, B64, Cm.numpy(), 5, 1, m)
+    h1, _ = O.hash_round(5, 1, 0, n1, m)
+    h2, _ = O.hash_round(5, 1, 1, n3, m)
+    denom = O.abs_sketch(O.abs_product(A64, B64), h1, h2, m)
+    hp = fpsk.HashedProbe(n1, n2, n3, m, seed=5, rnd=1)
+    pr = fpsk.default_params(tensor_cores=1)
+    dA, dB, dC = A.cuda(), Bm.cuda(), Cm.cuda()
+    _run(hp, dA, dB, dC, params=pr)
+    n0 = fpsk.launch_count()
+    got, S = _run(hp, dA, dB, dC, params=pr)
+    assert fpsk.launch_count() - n0 == 1 and got.status == 0
+    assert np.all(np.abs(S - S_ref) <= TOL * denom + 1e-30)
+    assert got.tau == pytest.approx(ref.tau, rel=1e-6)
+    v = O.probe_verdict(S.ravel(), ref.tau, n_rows=1)
+    assert got.sigma_hat == pytest.approx(v.sigma_hat, rel=1e-4, abs=1e-30)
+    assert got.argmax_col == v.argmax_col and got.nonfinite == 0
+    if abs(v.max_abs - v.thr) > 1e-3 * v.thr:
+        assert bool(got.fired) == v.fired
