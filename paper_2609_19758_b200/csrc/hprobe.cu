@@ -78,7 +78,9 @@ struct HpArgs {
     int nsub;                      // K ranges per column segment of A: a range never spans two scales
     int kblocks;                   // K blocks of 32 in the planes
     int trace_on;
-    unsigned long long *trace;     // 8 time stamps per CTA when trace_on
+    unsigned long long *trace;     // measurement build, when trace_on: 32 words per CTA - [0, 16 G) eight stamps per team (entry, first
+                                   // copy, through with A, first stage, end, hand-over done, contraction done, units), [16 G, 24 G)
+                                   // eight per CTA of the combine, [24 G, 32 G) per contracting CTA: K blocks landed, tile ready, rows stored
 };
 
 // Units are (matrix, column segment, row bucket); all units of A go out before those of C.  A unit's rows go
@@ -1431,7 +1433,7 @@ static size_t hp_work_layout(void *base, long long n1, long long n2, long long n
     t.scaleP = (float *)take((size_t)m * pl.segsA * 4);
     t.partC = (float *)take((size_t)pl.segsC * m * m * 4);
     t.S = (float *)take((size_t)m * m * 4);
-    t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 256);       // 8 stamps per team
+    t.trace = (unsigned long long *)take((size_t)(sms > 1 ? sms : 1) * 256);       // 32 words per CTA (see HpArgs::trace)
     if (w) *w = t;
     return off;
 }
