@@ -514,8 +514,9 @@ __device__ __forceinline__ void hv_combine_fused(const HvArgs &p)
     Sync::sync();
     CT(6);
     if (!s_last) return;
-    __threadfence();
-    // ---- last CTA: totals in CTA order (thread-strided, then the fixed shape), max|A|
+    // ---- last CTA (thread 0's ticket was an acquire and the barrier above passes it on to the other threads; the
+    // records and S were stored to L2 and are loaded from there): totals in CTA order (thread-strided, then the fixed
+    // shape), max|A|
     HvStat t = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
     for (int r = tid; r < G; r += kHvThreads) {
         const float4 v = __ldcg(p.vstat + r);
@@ -529,17 +530,17 @@ __device__ __forceinline__ void hv_combine_fused(const HvArgs &p)
     const bool slow = !(t.mx.v <= 5.f * mean) || t.bad > 0.f;
     float clipped = t.sum;
     if (slow) {
-        // all of S again (m^2 values, still in L2), four 16-byte loads in flight per thread
+        // all of S again (m^2 values, still in L2), eight 16-byte loads in flight per thread
         const float clip = 5.f * mean;
         HvStat cs = {0.f, 0.f, {-1.f, 0x7FFFFFFF}};
         const long long nq = (reinterpret_cast<uintptr_t>(p.S) & 15) ? 0 : mm / 4;      // a caller's S may be aligned to 4 bytes only
         const float4 *S4 = reinterpret_cast<const float4 *>(p.S);
-        for (long long q0 = tid; q0 < nq; q0 += 4 * kHvThreads) {
-            float4 v[4];
+        for (long long q0 = tid; q0 < nq; q0 += 8 * kHvThreads) {
+            float4 v[8];
 #pragma unroll
-            for (int u = 0; u < 4; ++u) v[u] = q0 + (long long)u * kHvThreads < nq ? __ldcg(S4 + q0 + (long long)u * kHvThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int u = 0; u < 8; ++u) v[u] = q0 + (long long)u * kHvThreads < nq ? __ldcg(S4 + q0 + (long long)u * kHvThreads) : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-            for (int u = 0; u < 4; ++u)
+            for (int u = 0; u < 8; ++u)
                 cs.sum += (fminf(fabsf(v[u].x), clip) + fminf(fabsf(v[u].y), clip)) + (fminf(fabsf(v[u].z), clip) + fminf(fabsf(v[u].w), clip));
         }
         for (long long i = 4 * nq + tid; i < mm; i += kHvThreads) cs.sum += fminf(fabsf(__ldcg(p.S + i)), clip);
